@@ -1,0 +1,286 @@
+/*
+ * KVzap CPU oracle -- TEST INFRASTRUCTURE, NOT A PRODUCT PATH.
+ *
+ * A plain, slow, obviously-correct restatement of what the KVzap pruning path
+ * computes, written from the paper's definition (Method section, "KVzap";
+ * Algorithm 1 / Listing 1; Experiments, "KVzap training"; Appendix B).
+ * It shares no code, header, table or helper with the CUDA library and is
+ * only ever called by the tests, the smoke check and the benchmark's
+ * cpu_baseline / reference legs.
+ *
+ * Arithmetic: every bf16 input is widened exactly to double; products and
+ * sums are carried in double in the index order of the definition; one
+ * rounding to fp32 at the end.  OpenMP only splits the independent token /
+ * head loops across cores.
+ *
+ * All matrices are row-major.  bf16 values are passed as raw uint16_t bit
+ * patterns.  Weight matrices are stored [out, in].
+ *
+ * Parity pins (tests/test_oracle_*.py): exact rational brute force on tiny
+ * inputs, one-hot / zero weights, torch-fp64 library composition, GELU
+ * identities, the paper's parameter totals and overhead table, mask and
+ * compaction invariants, decode == prefill-on-concatenation.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* exact widening of a bf16 bit pattern (upper half of an IEEE fp32) */
+static double bf16_to_double(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int kvzap_oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* GELU as used by the MLP surrogate (Experiments, "KVzap training": one hidden
+ * layer followed by a GELU).  Exact form: x * Phi(x), Phi the standard normal CDF. */
+double kvzap_oracle_gelu(double x)
+{
+    return 0.5 * x * (1.0 + erf(x / sqrt(2.0)));
+}
+
+/*
+ * KVzap-Linear (Method, "KVzap"): a per-layer linear map from the hidden state
+ * h_t in R^{D_h} to H scores, applied independently at each position t.
+ *   scores[t,h] = b[h] + sum_k X[t,k] * W[h,k]
+ * X [T,Dh] bf16, W [H,Dh] bf16, b [H] fp32 or NULL (= 0), scores [T,H] fp32.
+ */
+void kvzap_oracle_score_linear(const uint16_t *X, int64_t T, int Dh,
+                               const uint16_t *W, const float *b, int H,
+                               float *scores)
+{
+    int64_t t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < T; ++t) {
+        for (int h = 0; h < H; ++h) {
+            double acc = b ? (double)b[h] : 0.0;
+            for (int k = 0; k < Dh; ++k)
+                acc += bf16_to_double(X[t * Dh + k]) * bf16_to_double(W[(int64_t)h * Dh + k]);
+            scores[t * H + h] = (float)acc;
+        }
+    }
+}
+
+/*
+ * KVzap-MLP (Method, "KVzap"; Experiments, "KVzap training"; Appendix B):
+ * two linear layers W1 in R^{D_h x N1}, W2 in R^{N1 x H} with a GELU between.
+ *   z[j]        = b1[j] + sum_k X[t,k] * W1[j,k]
+ *   g[j]        = GELU(z[j])
+ *   scores[t,h] = b2[h] + sum_j g[j] * W2[h,j]
+ * W1 [N1,Dh] bf16, b1 [N1] fp32|NULL, W2 [H,N1] bf16, b2 [H] fp32|NULL.
+ * Returns 0, or -1 if scratch memory could not be allocated.
+ */
+int kvzap_oracle_score_mlp(const uint16_t *X, int64_t T, int Dh,
+                           const uint16_t *W1, const float *b1, int N1,
+                           const uint16_t *W2, const float *b2, int H,
+                           float *scores)
+{
+    /* widen the weights once; W1 is kept as [Dh][N1] so that the hidden units,
+     * which are independent sums, sit next to each other in memory */
+    double *w1 = (double *)malloc(sizeof(double) * (size_t)Dh * (size_t)N1);
+    double *w2 = (double *)malloc(sizeof(double) * (size_t)H * (size_t)N1);
+    if (!w1 || !w2) { free(w1); free(w2); return -1; }
+    for (int j = 0; j < N1; ++j)
+        for (int k = 0; k < Dh; ++k)
+            w1[(size_t)k * N1 + j] = bf16_to_double(W1[(size_t)j * Dh + k]);
+    for (int h = 0; h < H; ++h)
+        for (int j = 0; j < N1; ++j)
+            w2[(size_t)h * N1 + j] = bf16_to_double(W2[(size_t)h * N1 + j]);
+
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *z = (double *)malloc(sizeof(double) * (size_t)N1);
+        if (!z) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+            int64_t t;
+#pragma omp for schedule(static)
+            for (t = 0; t < T; ++t) {
+                for (int j = 0; j < N1; ++j) z[j] = b1 ? (double)b1[j] : 0.0;
+                /* each z[j] accumulates its products in increasing k */
+                for (int k = 0; k < Dh; ++k) {
+                    const double x = bf16_to_double(X[t * Dh + k]);
+                    const double *row = w1 + (size_t)k * N1;
+                    for (int j = 0; j < N1; ++j) z[j] += x * row[j];
+                }
+                for (int j = 0; j < N1; ++j) z[j] = kvzap_oracle_gelu(z[j]);
+                for (int h = 0; h < H; ++h) {
+                    double acc = b2 ? (double)b2[h] : 0.0;
+                    for (int j = 0; j < N1; ++j) acc += z[j] * w2[(size_t)h * N1 + j];
+                    scores[t * H + h] = (float)acc;
+                }
+            }
+        }
+        free(z);
+    }
+    free(w1);
+    free(w2);
+    return failed ? -1 : 0;
+}
+
+/*
+ * Window + threshold (Algorithm 1: the last `window` positions are forced to
+ * +inf, then positions with score >= threshold are kept; Method, "KVzap":
+ * pairs whose score falls below tau are discarded; the most recent w tokens
+ * are always kept).
+ *   keep[h, t] = (t_in_seq >= T_b - w) || (scores[t,h] >= tau)
+ * The window is per sequence: sequence b owns packed rows
+ * [cu_seqlens[b], cu_seqlens[b+1]).  w = 0 protects nothing; T_b <= w keeps all.
+ * The comparison is an ordinary fp32 >= (NaN compares false).
+ * scores [T_total,H] fp32; keep [H,T_total] bytes (0/1).
+ */
+void kvzap_oracle_keep_mask(const float *scores, const int32_t *cu_seqlens, int B,
+                            int H, float tau, int w, uint8_t *keep)
+{
+    const int64_t T_total = cu_seqlens[B];
+    for (int b = 0; b < B; ++b) {
+        const int64_t t0 = cu_seqlens[b], t1 = cu_seqlens[b + 1];
+        const int64_t Tb = t1 - t0;
+        for (int h = 0; h < H; ++h) {
+            for (int64_t t = t0; t < t1; ++t) {
+                const int in_window = (t - t0) >= Tb - (int64_t)w;
+                const int above = scores[t * H + h] >= tau;
+                keep[(int64_t)h * T_total + t] = (uint8_t)(in_window || above);
+            }
+        }
+    }
+}
+
+/*
+ * Per-(sequence, head) ordered compaction (Algorithm 1: keys[indices],
+ * values[indices]; contribution list: per-head compression).
+ * For each (b,h) walk the sequence's positions in order and copy row t of K
+ * and of V, bytes verbatim, to output slot n++ of that (b,h) list.
+ * K,V,K_out,V_out [H,T_total,D] bf16; list (b,h) starts at packed row
+ * cu_seqlens[b] of head h in the outputs.  Rows past lengths[b,h] are not
+ * written.  lengths [B,H] int32.
+ */
+void kvzap_oracle_compact(const uint16_t *K, const uint16_t *V, const uint8_t *keep,
+                          const int32_t *cu_seqlens, int B, int H, int D,
+                          uint16_t *K_out, uint16_t *V_out, int32_t *lengths)
+{
+    const int64_t T_total = cu_seqlens[B];
+    const size_t row_bytes = sizeof(uint16_t) * (size_t)D;
+    int bh;
+#pragma omp parallel for schedule(static)
+    for (bh = 0; bh < B * H; ++bh) {
+        const int b = bh / H, h = bh % H;
+        const int64_t t0 = cu_seqlens[b], t1 = cu_seqlens[b + 1];
+        int64_t n = 0;
+        for (int64_t t = t0; t < t1; ++t) {
+            if (!keep[(int64_t)h * T_total + t]) continue;
+            const int64_t src = ((int64_t)h * T_total + t) * D;
+            const int64_t dst = ((int64_t)h * T_total + t0 + n) * D;
+            memcpy(K_out + dst, K + src, row_bytes);
+            memcpy(V_out + dst, V + src, row_bytes);
+            ++n;
+        }
+        lengths[b * H + h] = (int32_t)n;
+    }
+}
+
+/*
+ * Paged variant of the same compaction.  The paper gives no page format
+ * (Discussion, "Implementation Challenges": non-uniform per-head lengths need
+ * paged kernels with variable-length blocks), so the reading used here is:
+ * a page holds page_tokens rows of K (and a page of the same index in the V
+ * pool holds the matching V rows); list (b,h) owns ceil(len/page_tokens)
+ * pages, numbered contiguously from first_page in (b,h) order.
+ * K_pool,V_pool [n_pages_pool, page_tokens, D] bf16;
+ * page_table [B*H, max_pages_per_list] int32 (unused entries left untouched);
+ * n_pages_used = total pages assigned.  Returns 0, or -1 if the pool or the
+ * table is too small (nothing is then written).
+ */
+int kvzap_oracle_compact_paged(const uint16_t *K, const uint16_t *V, const uint8_t *keep,
+                               const int32_t *cu_seqlens, int B, int H, int D,
+                               int page_tokens, int32_t first_page, int64_t n_pages_pool,
+                               int max_pages_per_list,
+                               uint16_t *K_pool, uint16_t *V_pool, int32_t *page_table,
+                               int32_t *lengths, int32_t *n_pages_used)
+{
+    const int64_t T_total = cu_seqlens[B];
+    const size_t row_bytes = sizeof(uint16_t) * (size_t)D;
+    /* pass 1: lengths and the page budget */
+    int64_t pages = 0;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int64_t n = 0;
+            for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t)
+                n += keep[(int64_t)h * T_total + t] ? 1 : 0;
+            lengths[b * H + h] = (int32_t)n;
+            const int64_t need = (n + page_tokens - 1) / page_tokens;
+            if (need > max_pages_per_list) return -1;
+            pages += need;
+        }
+    if ((int64_t)first_page + pages > n_pages_pool) return -1;
+    /* pass 2: assign pages in (b,h) order and copy rows */
+    int64_t cursor = first_page;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            const int list = b * H + h;
+            const int64_t need = ((int64_t)lengths[list] + page_tokens - 1) / page_tokens;
+            for (int64_t p = 0; p < need; ++p)
+                page_table[(int64_t)list * max_pages_per_list + p] = (int32_t)(cursor + p);
+            int64_t n = 0;
+            for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t) {
+                if (!keep[(int64_t)h * T_total + t]) continue;
+                const int64_t page = cursor + n / page_tokens;
+                const int64_t dst = (page * page_tokens + n % page_tokens) * D;
+                const int64_t src = ((int64_t)h * T_total + t) * D;
+                memcpy(K_pool + dst, K + src, row_bytes);
+                memcpy(V_pool + dst, V + src, row_bytes);
+                ++n;
+            }
+            cursor += need;
+        }
+    *n_pages_used = (int32_t)pages;
+    return 0;
+}
+
+/*
+ * Closed forms of Appendix B (per token, per layer).
+ *   C        = 4 D_h (H_Q D + H D) + 6 D_h D_int      linear-projection FLOPs of a layer
+ *   C_MLP    = 2 D_h (D_h/8) + 2 (D_h/8) H = D_h/4 (D_h + H)
+ *   C_Linear = 2 D_h H
+ */
+double kvzap_oracle_layer_flops(int H_Q, int H, int D, int Dh, int D_int)
+{
+    return 4.0 * Dh * ((double)H_Q * D + (double)H * D) + 6.0 * (double)Dh * D_int;
+}
+
+double kvzap_oracle_mlp_flops(int Dh, int N1, int H)
+{
+    return 2.0 * (double)Dh * N1 + 2.0 * (double)N1 * H;
+}
+
+double kvzap_oracle_linear_flops(int Dh, int H)
+{
+    return 2.0 * (double)Dh * H;
+}
+
+/* parameter count of one layer's surrogate, biases included; N1 = 0 means Linear */
+int64_t kvzap_oracle_param_count(int Dh, int N1, int H)
+{
+    if (N1 == 0) return (int64_t)Dh * H + H;
+    return (int64_t)Dh * N1 + N1 + (int64_t)N1 * H + H;
+}
