@@ -1,0 +1,157 @@
+/*
+ * kvzap.h -- C ABI of the KVzap pruning hot path for NVIDIA B200 (sm_100a).
+ *
+ * KVzap (Method section, "KVzap"; Algorithm 1) prunes a transformer layer's
+ * KV cache per KV head: a small per-layer surrogate (a linear map, or a
+ * two-layer MLP with a GELU) turns each token's hidden state into one
+ * log-importance score per KV head; a key/value pair is discarded when its
+ * score is below a fixed threshold tau, except that the most recent w tokens
+ * are always kept; the kept keys and values of every (sequence, head) are
+ * gathered, in token order, into a list whose length differs from head to
+ * head.
+ *
+ * General conventions
+ *   - Every tensor argument is a DEVICE pointer owned by the caller, unless a
+ *     comment says "host".  The library owns only its context (a private
+ *     copy of the surrogate weights and a few MB of scratch).
+ *   - bf16 tensors are passed as `const void*` (raw 16-bit patterns),
+ *     row-major, innermost dimension last.  Pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as `void*` (NULL = default stream).
+ *     Calls enqueue work on it and return without synchronising.  A context
+ *     must not be used from two streams at the same time: its scratch is
+ *     shared by all calls.
+ *   - Errors the host can see (bad argument, unsupported shape) return at once
+ *     and launch nothing.  Conditions only the device can see set a status
+ *     word that kvzap_poll_status() reads; kernels never trap and every
+ *     device-side wait is bounded.
+ *   - Token packing: a batch of B sequences is passed packed along the token
+ *     axis; `cu_seqlens` (device, int32 [B+1], cu_seqlens[0] = 0,
+ *     cu_seqlens[B] = n_tokens) gives each sequence's rows.  NULL means one
+ *     sequence of n_tokens.
+ */
+#ifndef KVZAP_H_
+#define KVZAP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KVZAP_OK = 0,
+    KVZAP_ERR_INVALID_ARG = 1,   /* null pointer, negative size, out-of-range layer, ...        */
+    KVZAP_ERR_UNSUPPORTED = 2,   /* shape outside the limits listed at kvzap_create             */
+    KVZAP_ERR_CUDA = 3,          /* a CUDA runtime/driver call failed; see kvzap_last_error     */
+    KVZAP_ERR_OOM_PAGES = 4,     /* device side: page pool or page table exhausted              */
+    KVZAP_ERR_TIMEOUT = 5,       /* device side: a bounded wait inside a kernel expired         */
+    KVZAP_ERR_STATE = 6          /* call order violated, e.g. scoring a layer without weights   */
+} kvzap_status;
+
+typedef struct kvzap_ctx kvzap_ctx;
+
+/*
+ * Shapes of one model's surrogate and cache (Experiments, "KVzap training":
+ * input size D_h, one hidden layer of width D_h/8 for the MLP, H outputs;
+ * Introduction: cache of shape (2, L, H, T, D)).
+ */
+typedef struct {
+    int32_t d_model;      /* D_h; multiple of 64, 64..16384                                     */
+    int32_t hidden;       /* 0 = KVzap-Linear; else MLP hidden width N1: multiple of 64 up to
+                             512, or a multiple of 128 up to 1024                               */
+    int32_t n_kv_heads;   /* H, 1..8                                                            */
+    int32_t head_dim;     /* D; multiple of 8 (rows are whole 16-byte units), 8..1024           */
+    int32_t n_layers;     /* L >= 1: number of per-layer surrogates held by the context         */
+    int32_t device;       /* CUDA device ordinal                                                */
+    int64_t max_tokens;   /* largest n_tokens any call will pass (sizes the scratch)            */
+    int32_t max_seqs;     /* largest number of sequences in one call (>= 1)                     */
+    int32_t reserved;     /* set to 0                                                           */
+} kvzap_config;
+
+/* Creates a context on cfg->device (allocates weights storage and scratch with
+ * cudaMalloc; synchronous).  *out is NULL on failure. */
+kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg);
+
+/* Synchronises the device, frees everything the context owns.  NULL is allowed. */
+kvzap_status kvzap_destroy(kvzap_ctx *ctx);
+
+/* Message of the last failing call on this context ("" if none).  The string is
+ * owned by the context and valid until the next call on it.  With ctx == NULL
+ * returns the message of the last failing kvzap_create of this process. */
+const char *kvzap_last_error(const kvzap_ctx *ctx);
+
+/*
+ * Installs one layer's surrogate (Method, "KVzap": a linear layer or a
+ * two-layer MLP; Appendix B: W1 in R^{D_h x D_h/8}, W2 in R^{D_h/8 x H}).
+ * Matrices are bf16, stored [out, in] row-major; biases are fp32, NULL = zero.
+ *   KVzap-Linear (cfg.hidden == 0): W1 [H, d_model], b1 [H]; W2 and b2 must be NULL.
+ *   KVzap-MLP:                      W1 [hidden, d_model], b1 [hidden],
+ *                                   W2 [H, hidden],       b2 [H].
+ * The context keeps its own repacked copy (copy kernels run on `stream`); the
+ * caller's buffers may be freed once that stream work has completed.
+ */
+kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer,
+                               const void *W1, const float *b1,
+                               const void *W2, const float *b2, void *stream);
+
+/*
+ * Surrogate scoring (Method, "KVzap"; Algorithm 1, first line): maps each
+ * hidden state h_t to H scores, independently per position.
+ *   Linear: scores[t,h] = b1[h] + sum_k hidden[t,k] W1[h,k]
+ *   MLP:    scores[t,h] = b2[h] + sum_j GELU(b1[j] + sum_k hidden[t,k] W1[j,k]) W2[h,j]
+ * GELU is the exact (erf) form.  bf16 products are accumulated in fp32.
+ *   hidden [n_tokens, d_model] bf16 (in)   scores [n_tokens, H] fp32 (out)
+ * n_tokens may be 0 (nothing is launched) and need not be a multiple of anything.
+ */
+kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens,
+                         float *scores, void *stream);
+
+/*
+ * Threshold + sliding window + per-(sequence, head) ordered compaction
+ * (Algorithm 1, lines 2-4; Method, "KVzap": pairs whose score falls below tau
+ * are discarded, the most recent w tokens are kept).
+ *   keep[b,h,t] = (t >= T_b - w) || (scores[t,h] >= tau)        (fp32 compare; NaN is not kept)
+ * with t counted inside sequence b of length T_b.  w = 0 protects nothing;
+ * T_b <= w keeps the whole sequence.
+ *   K, V         [H, n_tokens, D] bf16 (in)    packed sequences along the token axis
+ *   scores       [n_tokens, H] fp32 (in)
+ *   K_out, V_out [H, n_tokens, D] bf16 (out)   list (b,h) occupies rows
+ *                cu_seqlens[b] .. cu_seqlens[b] + lengths[b,h] - 1 of head h, in token order,
+ *                rows copied bit for bit; all other rows are left untouched.
+ *   lengths      [n_seqs, H] int32 (out)
+ * K_out/V_out must not overlap K/V.  tau may be any fp32 (+-inf included); w >= 0.
+ */
+kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                 float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths, void *stream);
+
+/*
+ * Algorithm 1 in one call: kvzap_score on `hidden` with the threshold and
+ * window test fused into the scoring kernel's epilogue, then the compaction of
+ * kvzap_prune_prefill.  `scores_out` ([n_tokens, H] fp32) may be NULL when the
+ * caller does not need the scores.  Other arguments as above.
+ */
+kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                 const void *K, const void *V,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                 float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths,
+                                 float *scores_out, void *stream);
+
+/*
+ * Reads the context's device status word (synchronises `stream` first) and
+ * clears it.  Returns KVZAP_OK, or the first device-side condition recorded
+ * since the last poll (KVZAP_ERR_TIMEOUT, KVZAP_ERR_OOM_PAGES).
+ */
+kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream);
+
+/* Number of kernels the library has launched through this context since it was
+ * created (for launch accounting in benchmarks). */
+int64_t kvzap_launch_count(const kvzap_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVZAP_H_ */

@@ -1,0 +1,211 @@
+"""ctypes binding of ``libkvzap.so`` (the C ABI declared in ``include/kvzap.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch is used for device memory and streams.  There is no CPU
+fallback: if the library cannot be loaded, importing a symbol from it raises.
+
+The module-level ``kvzap_*`` functions mirror the C entry points one to one
+(tensors instead of raw pointers); :class:`Kvzap` is a small convenience
+wrapper that owns a context and allocates outputs.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libkvzap.so")
+_lib = None
+
+KVZAP_OK = 0
+STATUS_NAMES = {0: "KVZAP_OK", 1: "KVZAP_ERR_INVALID_ARG", 2: "KVZAP_ERR_UNSUPPORTED", 3: "KVZAP_ERR_CUDA",
+                4: "KVZAP_ERR_OOM_PAGES", 5: "KVZAP_ERR_TIMEOUT", 6: "KVZAP_ERR_STATE"}
+
+
+class KvzapError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("%s: %s" % (STATUS_NAMES.get(status, str(status)), message))
+        self.status = status
+
+
+class KvzapConfig(ctypes.Structure):
+    _fields_ = [("d_model", ctypes.c_int32), ("hidden", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("n_layers", ctypes.c_int32), ("device", ctypes.c_int32),
+                ("max_tokens", ctypes.c_int64), ("max_seqs", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+_vp, _i32, _i64, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+
+# name -> (restype, argtypes); also the list of symbols the header declares
+SIGNATURES = {
+    "kvzap_create": (_i32, [ctypes.POINTER(_vp), ctypes.POINTER(KvzapConfig)]),
+    "kvzap_destroy": (_i32, [_vp]),
+    "kvzap_last_error": (ctypes.c_char_p, [_vp]),
+    "kvzap_set_weights": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "kvzap_score": (_i32, [_vp, _i32, _vp, _i64, _vp, _vp]),
+    "kvzap_prune_prefill": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_fused": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "kvzap_poll_status": (_i32, [_vp, _vp]),
+    "kvzap_launch_count": (_i64, [_vp]),
+}
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Loads libkvzap.so (building it with nvcc first if it is missing or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    try:
+        _build.build()
+    except Exception as e:  # no nvcc on this machine: fall through to whatever was shipped
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("libkvzap.so is not built and could not be built here (%s); run "
+                               "`python -m paper_2601_07891_b200.build` on a machine with nvcc" % (e,)) from e
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError("libkvzap.so not found at %s" % _LIB_PATH)
+    lib = ctypes.CDLL(_LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)          # AttributeError if the symbol is not exported
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(handle, st):
+    if st != KVZAP_OK:
+        msg = load().kvzap_last_error(handle)
+        raise KvzapError(st, msg.decode() if msg else "")
+
+
+def kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0):
+    cfg = KvzapConfig(d_model, hidden, n_kv_heads, head_dim, n_layers, device, max_tokens, max_seqs, 0)
+    handle = ctypes.c_void_p()
+    st = load().kvzap_create(ctypes.byref(handle), ctypes.byref(cfg))
+    _check(None, st)
+    return handle
+
+
+def kvzap_destroy(handle):
+    _check(handle, load().kvzap_destroy(handle))
+
+
+def kvzap_set_weights(handle, layer, W1, b1=None, W2=None, b2=None, stream=None):
+    _check(handle, load().kvzap_set_weights(handle, layer, _ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _stream(stream)))
+
+
+def kvzap_score(handle, layer, hidden, scores, stream=None):
+    n_tokens = hidden.shape[0]
+    _check(handle, load().kvzap_score(handle, layer, _ptr(hidden) if n_tokens else None, n_tokens,
+                                      _ptr(scores) if n_tokens else None, _stream(stream)))
+
+
+def kvzap_prune_prefill(handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prune_prefill(
+        handle, _ptr(K) if nz else None, _ptr(V) if nz else None, _ptr(scores) if nz else None, _ptr(cu_seqlens),
+        n_seqs, n_tokens, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None, _ptr(lengths),
+        _stream(stream)))
+
+
+def kvzap_prefill_fused(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                        scores_out=None, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_fused(
+        handle, layer, _ptr(hidden) if nz else None, _ptr(K) if nz else None, _ptr(V) if nz else None,
+        _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
+        _ptr(lengths), _ptr(scores_out) if nz else None, _stream(stream)))
+
+
+def kvzap_poll_status(handle, stream=None) -> int:
+    return int(load().kvzap_poll_status(handle, _stream(stream)))
+
+
+def kvzap_launch_count(handle) -> int:
+    return int(load().kvzap_launch_count(handle))
+
+
+class Kvzap:
+    """Owns one context; allocates outputs with torch; same calls as the C ABI."""
+
+    def __init__(self, d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0):
+        self.d_model, self.hidden, self.n_kv_heads, self.head_dim = d_model, hidden, n_kv_heads, head_dim
+        self.n_layers, self.max_tokens, self.max_seqs = n_layers, max_tokens, max_seqs
+        self.device = torch.device("cuda", device)
+        self.handle = kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs, device)
+
+    def close(self):
+        if self.handle is not None:
+            kvzap_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_weights(self, layer, *weights, stream=None):
+        """weights = (W, b) for KVzap-Linear or (W1, b1, W2, b2) for KVzap-MLP."""
+        if len(weights) == 2:
+            kvzap_set_weights(self.handle, layer, weights[0], weights[1], None, None, stream)
+        else:
+            kvzap_set_weights(self.handle, layer, *weights, stream=stream)
+
+    def score(self, layer, hidden, out=None, stream=None):
+        if out is None:
+            out = torch.empty(hidden.shape[0], self.n_kv_heads, dtype=torch.float32, device=self.device)
+        kvzap_score(self.handle, layer, hidden, out, stream)
+        return out
+
+    def _outputs(self, K, n_seqs, K_out, V_out, lengths):
+        if K_out is None:
+            K_out = torch.empty_like(K)
+        if V_out is None:
+            V_out = torch.empty_like(K)
+        if lengths is None:
+            lengths = torch.empty(n_seqs, self.n_kv_heads, dtype=torch.int32, device=self.device)
+        return K_out, V_out, lengths
+
+    def prune_prefill(self, K, V, scores, tau, w, cu_seqlens=None, K_out=None, V_out=None, lengths=None, stream=None):
+        n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        K_out, V_out, lengths = self._outputs(K, n_seqs, K_out, V_out, lengths)
+        kvzap_prune_prefill(self.handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths, stream)
+        return K_out, V_out, lengths
+
+    def prefill_fused(self, layer, hidden, K, V, tau, w, cu_seqlens=None, K_out=None, V_out=None, lengths=None,
+                      scores_out=None, stream=None):
+        n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        K_out, V_out, lengths = self._outputs(K, n_seqs, K_out, V_out, lengths)
+        kvzap_prefill_fused(self.handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                            scores_out, stream)
+        return K_out, V_out, lengths
+
+    def poll_status(self, stream=None) -> int:
+        return kvzap_poll_status(self.handle, stream)
+
+    def launch_count(self) -> int:
+        return kvzap_launch_count(self.handle)

@@ -1,0 +1,497 @@
+// Host side of the C ABI declared in include/kvzap.h: context, weight
+// repacking, TMA descriptors, argument checks and kernel launches.
+#include "../../include/kvzap.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "prune_kernels.cuh"
+#include "score_kernel.cuh"
+
+namespace kvzap {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct LayerWeights {
+    void *w1 = nullptr;      // bf16 [rows_padded, d_model]
+    float *b1 = nullptr;     // [rows_padded]
+    float *w2t = nullptr;    // [hidden][8] fp32 (MLP)
+    float *b2 = nullptr;     // [8] (MLP)
+    CUtensorMap tmap_w;
+    bool set = false;
+};
+
+static char g_create_error[512] = "";
+
+}  // namespace kvzap
+
+struct kvzap_ctx {
+    kvzap_config cfg;
+    int sm_count = 0;
+    int w1_rows = 0;                 // rows of the stored first-layer matrix (Linear: padded to 16)
+    // scoring schedule (see ScoreParams)
+    int group_w = 0, n_groups = 0, chunk_n = 0, n_chunks = 0, n_stages = 0, acc_bufs = 0, acc_stride = 0,
+        tmem_cols = 0;
+    uint32_t score_smem = 0;
+    std::vector<kvzap::LayerWeights> layers;
+    kvzap::EncodeTiledFn encode = nullptr;
+    // scratch
+    int64_t max_blocks = 0, max_words = 0;
+    uint32_t *maskbits = nullptr;    // [H][max_words]
+    int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
+    int32_t *seqbase = nullptr;      // [H][max_seqs + 1]
+    int32_t *status_dev = nullptr;
+    int32_t *status_host = nullptr;  // pinned
+    int64_t launches = 0;
+    char err[512] = "";
+};
+
+namespace kvzap {
+
+static kvzap_status fail(kvzap_ctx *ctx, kvzap_status st, const char *fmt, ...)
+{
+    char *dst = ctx ? ctx->err : g_create_error;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(dst, 512, fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+#define KVZAP_CUDA(ctx, call)                                                                        \
+    do {                                                                                             \
+        cudaError_t e_ = (call);                                                                     \
+        if (e_ != cudaSuccess)                                                                       \
+            return kvzap::fail(ctx, KVZAP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+    } while (0)
+
+static int next_pow2(int v)
+{
+    int p = 32;
+    while (p < v) p <<= 1;
+    return p;
+}
+
+// 2-D bf16 tensor map: `rows` x `cols` row-major, box `box_rows` x 64 elements, 128-byte swizzle.
+static kvzap_status make_tmap(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
+                              uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, KVZAP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d (rows=%llu cols=%llu box_rows=%u)",
+                    static_cast<int>(r), static_cast<unsigned long long>(rows), static_cast<unsigned long long>(cols),
+                    box_rows);
+    return KVZAP_OK;
+}
+
+// W2 [H, hidden] bf16 -> w2t [hidden][8] fp32 (zero for heads >= H); b2 -> [8] fp32.
+__global__ void pack_w2_kernel(const uint16_t *__restrict__ W2, const float *__restrict__ b2, int n_heads, int hidden,
+                               float *__restrict__ w2t, float *__restrict__ b2p)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < hidden * kMaxHeads) {
+        const int j = idx / kMaxHeads, h = idx % kMaxHeads;
+        float v = 0.0f;
+        if (h < n_heads) v = __uint_as_float(static_cast<uint32_t>(W2[static_cast<int64_t>(h) * hidden + j]) << 16);
+        w2t[idx] = v;
+    }
+    if (idx < kMaxHeads) b2p[idx] = (b2 != nullptr && idx < n_heads) ? b2[idx] : 0.0f;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+static void free_all(kvzap_ctx *ctx)
+{
+    for (auto &lw : ctx->layers) {
+        cudaFree(lw.w1);
+        cudaFree(lw.b1);
+        cudaFree(lw.w2t);
+        cudaFree(lw.b2);
+    }
+    cudaFree(ctx->maskbits);
+    cudaFree(ctx->blockprefix);
+    cudaFree(ctx->seqbase);
+    cudaFree(ctx->status_dev);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
+}
+
+static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seqs, const int32_t *cu_seqlens)
+{
+    if (n_tokens < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "n_tokens is negative");
+    if (n_tokens > ctx->cfg.max_tokens)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "n_tokens %lld exceeds the context's max_tokens %lld",
+                    static_cast<long long>(n_tokens), static_cast<long long>(ctx->cfg.max_tokens));
+    if (n_seqs < 1 || n_seqs > ctx->cfg.max_seqs)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "n_seqs %d outside 1..max_seqs (%d)", n_seqs, ctx->cfg.max_seqs);
+    if (cu_seqlens == nullptr && n_seqs != 1)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "cu_seqlens is NULL but n_seqs is %d", n_seqs);
+    return KVZAP_OK;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launches the scoring kernel; maskbits != nullptr fuses the threshold/window test.
+static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens, float *scores,
+                                 uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs, float tau, int32_t w,
+                                 cudaStream_t stream)
+{
+    const kvzap_config &c = ctx->cfg;
+    LayerWeights &lw = ctx->layers[layer];
+    const int64_t n_tiles = (n_tokens + kTileM - 1) / kTileM;
+    CUtensorMap tmap_x;
+    kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model),
+                                kTileM);
+    if (st != KVZAP_OK) return st;
+    ScoreParams p;
+    memset(&p, 0, sizeof p);
+    p.n_tokens = n_tokens;
+    p.n_tiles = static_cast<int32_t>(n_tiles);
+    p.d_model = c.d_model;
+    p.group_w = ctx->group_w;
+    p.n_groups = ctx->n_groups;
+    p.chunk_n = ctx->chunk_n;
+    p.n_chunks = ctx->n_chunks;
+    p.n_stages = ctx->n_stages;
+    p.acc_bufs = ctx->acc_bufs;
+    p.acc_stride = ctx->acc_stride;
+    p.tmem_cols = ctx->tmem_cols;
+    p.n_hidden = c.hidden;
+    p.n_heads = c.n_kv_heads;
+    p.b1 = lw.b1;
+    p.w2t = lw.w2t;
+    p.b2 = lw.b2;
+    p.scores = scores;
+    p.maskbits = maskbits;
+    p.n_words = n_tiles * 4;
+    p.cu_seqlens = cu_seqlens;
+    p.n_seqs = n_seqs;
+    p.window = w;
+    p.tau = tau;
+    p.status = ctx->status_dev;
+    const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
+    if (c.hidden > 0)
+        score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+    else
+        score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+// scan + compaction over mask words already in ctx->maskbits
+static kvzap_status launch_compaction(kvzap_ctx *ctx, const void *K, const void *V, const int32_t *cu_seqlens,
+                                      int32_t n_seqs, int64_t n_tokens, void *K_out, void *V_out, int32_t *lengths,
+                                      cudaStream_t stream)
+{
+    const kvzap_config &c = ctx->cfg;
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    const int64_t n_words = n_blocks * 4;
+    scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs, n_tokens,
+                                        ctx->blockprefix, ctx->seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr,
+                                        ctx->status_dev);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
+    compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
+        static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
+        static_cast<uint4 *>(V_out), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
+        n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, 0, nullptr);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 2;
+    return KVZAP_OK;
+}
+
+static kvzap_status check_prune_args(kvzap_ctx *ctx, const void *K, const void *V, const void *K_out,
+                                     const void *V_out, const int32_t *lengths, int32_t w)
+{
+    if (!K || !V || !K_out || !V_out || !lengths)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "K, V, K_out, V_out and lengths must not be NULL");
+    if (!aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "K/V pointers must be 16-byte aligned");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    return KVZAP_OK;
+}
+
+}  // namespace kvzap
+
+using namespace kvzap;
+
+extern "C" {
+
+kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
+{
+    if (!out) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (!cfg) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "cfg is NULL");
+    const kvzap_config c = *cfg;
+    if (c.d_model < 64 || c.d_model > 16384 || c.d_model % 64)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "d_model %d: need a multiple of 64 in 64..16384", c.d_model);
+    if (c.hidden < 0 || c.hidden > 1024 || (c.hidden <= 512 && c.hidden % 64) || (c.hidden > 512 && c.hidden % 128))
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED,
+                    "hidden %d: need 0, a multiple of 64 up to 512, or a multiple of 128 up to 1024", c.hidden);
+    if (c.n_kv_heads < 1 || c.n_kv_heads > kMaxHeads)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "n_kv_heads %d: need 1..8", c.n_kv_heads);
+    if (c.head_dim < 8 || c.head_dim > 1024 || c.head_dim % 8)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "head_dim %d: need a multiple of 8 in 8..1024", c.head_dim);
+    if (c.n_layers < 1) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "n_layers %d: need >= 1", c.n_layers);
+    if (c.max_tokens < 1 || c.max_tokens > (int64_t(1) << 30))
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "max_tokens out of range (1..2^30)");
+    if (c.max_seqs < 1 || c.max_seqs > (1 << 20))
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "max_seqs out of range (1..2^20)");
+
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || c.device < 0 || c.device >= n_dev)
+        return fail(nullptr, KVZAP_ERR_CUDA, "CUDA device %d not available (%d devices)", c.device, n_dev);
+    DeviceGuard guard(c.device);
+    if (!guard.ok) return fail(nullptr, KVZAP_ERR_CUDA, "cudaSetDevice(%d) failed", c.device);
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c.device) != cudaSuccess)
+        return fail(nullptr, KVZAP_ERR_CUDA, "cudaGetDeviceProperties failed");
+    if (prop.major != 10)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "device %d is sm_%d%d; this library is built for sm_100a only",
+                    c.device, prop.major, prop.minor);
+
+    kvzap_ctx *ctx = new (std::nothrow) kvzap_ctx();
+    if (!ctx) return fail(nullptr, KVZAP_ERR_CUDA, "out of host memory");
+    ctx->cfg = c;
+    ctx->sm_count = prop.multiProcessorCount;
+
+    // scoring schedule
+    if (c.hidden == 0) {
+        ctx->w1_rows = 16;            // H <= 8 outputs padded to the smallest N of a 128-row MMA
+        ctx->group_w = 16; ctx->n_groups = 1; ctx->chunk_n = 16; ctx->n_chunks = 1;
+        ctx->acc_bufs = 2; ctx->acc_stride = 32;
+    } else {
+        ctx->w1_rows = c.hidden;
+        ctx->n_groups = c.hidden > 512 ? 2 : 1;
+        ctx->group_w = c.hidden / ctx->n_groups;
+        ctx->n_chunks = ctx->group_w > 256 ? 2 : 1;
+        ctx->chunk_n = ctx->group_w / ctx->n_chunks;
+        ctx->acc_bufs = 512 / ctx->group_w >= 2 ? 2 : 1;
+        ctx->acc_stride = ctx->group_w;
+    }
+    ctx->tmem_cols = next_pow2(ctx->acc_bufs * ctx->acc_stride);
+    {
+        const int budget = static_cast<int>(prop.sharedMemPerBlockOptin) - 1024;
+        int stages = kMaxStages;
+        for (; stages >= 2; --stages)
+            if (static_cast<int>(score_smem_layout(ctx->group_w, stages, c.hidden).total) <= budget) break;
+        if (stages < 2) {
+            delete ctx;
+            return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "shared memory too small for this surrogate shape");
+        }
+        ctx->n_stages = stages;
+        ctx->score_smem = score_smem_layout(ctx->group_w, stages, c.hidden).total + 1024;
+    }
+
+#define CREATE_CUDA(call)                                                                              \
+    do {                                                                                               \
+        cudaError_t e_ = (call);                                                                       \
+        if (e_ != cudaSuccess) {                                                                       \
+            fail(nullptr, KVZAP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));             \
+            free_all(ctx);                                                                             \
+            delete ctx;                                                                                \
+            return KVZAP_ERR_CUDA;                                                                     \
+        }                                                                                              \
+    } while (0)
+
+    {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        CREATE_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || fn == nullptr) {
+            delete ctx;
+            return fail(nullptr, KVZAP_ERR_CUDA, "driver entry point cuTensorMapEncodeTiled not found");
+        }
+        ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(ctx->score_smem)));
+    CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(ctx->score_smem)));
+
+    ctx->layers.resize(c.n_layers);
+    for (auto &lw : ctx->layers) {
+        const size_t w1_bytes = static_cast<size_t>(ctx->w1_rows) * c.d_model * 2;
+        CREATE_CUDA(cudaMalloc(&lw.w1, w1_bytes));
+        CREATE_CUDA(cudaMemset(lw.w1, 0, w1_bytes));
+        CREATE_CUDA(cudaMalloc(&lw.b1, sizeof(float) * ctx->w1_rows));
+        CREATE_CUDA(cudaMemset(lw.b1, 0, sizeof(float) * ctx->w1_rows));
+        if (c.hidden > 0) {
+            CREATE_CUDA(cudaMalloc(&lw.w2t, sizeof(float) * c.hidden * kMaxHeads));
+            CREATE_CUDA(cudaMalloc(&lw.b2, sizeof(float) * kMaxHeads));
+        }
+        ctx->err[0] = 0;
+        if (make_tmap(ctx, &lw.tmap_w, lw.w1, static_cast<uint64_t>(ctx->w1_rows), static_cast<uint64_t>(c.d_model),
+                      static_cast<uint32_t>(ctx->chunk_n)) != KVZAP_OK) {
+            snprintf(g_create_error, sizeof g_create_error, "%s", ctx->err);
+            free_all(ctx);
+            delete ctx;
+            return KVZAP_ERR_CUDA;
+        }
+    }
+    ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
+    ctx->max_words = ctx->max_blocks * 4;
+    CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * ctx->max_words * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
+    CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
+    CREATE_CUDA(cudaMallocHost(&ctx->status_host, sizeof(int32_t)));
+    CREATE_CUDA(cudaDeviceSynchronize());
+#undef CREATE_CUDA
+    g_create_error[0] = 0;
+    *out = ctx;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_destroy(kvzap_ctx *ctx)
+{
+    if (!ctx) return KVZAP_OK;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaDeviceSynchronize();
+    free_all(ctx);
+    delete ctx;
+    return KVZAP_OK;
+}
+
+const char *kvzap_last_error(const kvzap_ctx *ctx) { return ctx ? ctx->err : g_create_error; }
+
+int64_t kvzap_launch_count(const kvzap_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, const float *b1, const void *W2,
+                               const float *b2, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    if (!W1) return fail(ctx, KVZAP_ERR_INVALID_ARG, "W1 is NULL");
+    if (c.hidden == 0 && (W2 || b2)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-Linear takes no W2/b2");
+    if (c.hidden > 0 && !W2) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-MLP needs W2");
+    DeviceGuard guard(c.device);
+    LayerWeights &lw = ctx->layers[layer];
+    const int rows = c.hidden > 0 ? c.hidden : c.n_kv_heads;
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(lw.w1, W1, static_cast<size_t>(rows) * c.d_model * 2, cudaMemcpyDeviceToDevice,
+                                    stream));
+    if (b1)
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(lw.b1, b1, sizeof(float) * rows, cudaMemcpyDeviceToDevice, stream));
+    else
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lw.b1, 0, sizeof(float) * rows, stream));
+    if (c.hidden > 0) {
+        const int n = c.hidden * kMaxHeads;
+        pack_w2_kernel<<<(n + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t *>(W2), b2, c.n_kv_heads,
+                                                            c.hidden, lw.w2t, lw.b2);
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    }
+    lw.set = true;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens, float *scores,
+                         void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layers[layer].set) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (n_tokens == 0) return KVZAP_OK;
+    if (!hidden || !scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden and scores must not be NULL");
+    if (!aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be 16-byte aligned");
+    DeviceGuard guard(ctx->cfg.device);
+    return launch_score(ctx, layer, hidden, n_tokens, scores, nullptr, nullptr, 1, 0.0f, 0,
+                        static_cast<cudaStream_t>(stream_));
+}
+
+kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    DeviceGuard guard(ctx->cfg.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * ctx->cfg.n_kv_heads, stream));
+        return KVZAP_OK;
+    }
+    st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
+    if (st != KVZAP_OK) return st;
+    if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads, cu_seqlens,
+                                                                     n_seqs, tau, w, ctx->maskbits, n_blocks * 4);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+}
+
+kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths, float *scores_out, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layers[layer].set) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    DeviceGuard guard(ctx->cfg.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * ctx->cfg.n_kv_heads, stream));
+        return KVZAP_OK;
+    }
+    st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
+    if (st != KVZAP_OK) return st;
+    if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
+    st = launch_score(ctx, layer, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
+    if (st != KVZAP_OK) return st;
+    return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+}
+
+kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    DeviceGuard guard(ctx->cfg.device);
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->status_host, ctx->status_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    KVZAP_CUDA(ctx, cudaMemsetAsync(ctx->status_dev, 0, sizeof(int32_t), stream));
+    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
+    const int32_t v = *ctx->status_host;
+    if (v == 0) return KVZAP_OK;
+    fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
+    return static_cast<kvzap_status>(v);
+}
+
+}  // extern "C"

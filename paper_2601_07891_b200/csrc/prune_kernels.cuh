@@ -1,0 +1,281 @@
+// Threshold/window mask, per-head prefix sums and ordered K/V compaction
+// (Algorithm 1, lines 2-4).  Everything here is integer / byte work and must
+// be bit-exact.
+//
+// Data flow (all on one stream, no CTA ever waits for another):
+//   mask words  [H][n_words]   one keep bit per (head, packed token), 32 tokens per word,
+//                              written either by the scoring epilogue or by mask_kernel
+//   scan_kernel                per head: exclusive prefix of the kept count over 128-token
+//                              blocks; kept count before each sequence start; lengths[b,h]
+//   compact_kernel             one CTA per (128-token block, head): ranks its kept rows with
+//                              popc over the mask words and copies whole K and V rows with
+//                              16-byte accesses to their slot in the (b,h) list
+#pragma once
+
+#include "score_kernel.cuh"
+
+namespace kvzap {
+
+constexpr int kBlockTokens = 128;     // tokens per mask block = 4 words (same as the scoring tile)
+
+// ---------------------------------------------------------------------------
+// keep[h,t] = in_window(t) || scores[t,h] >= tau, as 32-token ballot words.
+// One warp per 32 tokens; 4 warps per CTA = one 128-token block.
+__global__ void __launch_bounds__(128)
+mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
+            const int32_t *__restrict__ cu_seqlens, int n_seqs, float tau, int window,
+            uint32_t *__restrict__ maskbits, int64_t n_words)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t word = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+    const int64_t t = word * 32 + lane;
+    const bool valid = t < n_tokens;
+    float s[kMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+    bool in_window = false;
+    if (valid) {
+        const float *src = scores + t * n_heads;
+        if (n_heads == kMaxHeads) {
+            const float4 a = __ldg(reinterpret_cast<const float4 *>(src));
+            const float4 b = __ldg(reinterpret_cast<const float4 *>(src) + 1);
+            s[0] = a.x; s[1] = a.y; s[2] = a.z; s[3] = a.w;
+            s[4] = b.x; s[5] = b.y; s[6] = b.z; s[7] = b.w;
+        } else {
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h)
+                if (h < n_heads) s[h] = __ldg(src + h);
+        }
+        int64_t seq_end = n_tokens;
+        if (cu_seqlens != nullptr && n_seqs > 1)
+            seq_end = __ldg(cu_seqlens + seq_of_token(cu_seqlens, n_seqs, t) + 1);
+        in_window = t >= seq_end - static_cast<int64_t>(window);
+    }
+    uint32_t my_word = 0;
+#pragma unroll
+    for (int h = 0; h < kMaxHeads; ++h) {
+        const bool keep = valid && (in_window || s[h] >= tau);
+        const uint32_t w = __ballot_sync(0xffffffffu, keep);
+        if (lane == h) my_word = w;
+    }
+    if (lane < n_heads) maskbits[static_cast<int64_t>(lane) * n_words + word] = my_word;
+}
+
+// Number of kept tokens of head h among packed tokens [0, t), given the block prefix.
+__device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ maskbits, int64_t n_words,
+                                               const int32_t *__restrict__ blockprefix, int64_t n_blocks, int h,
+                                               int64_t t)
+{
+    const int64_t blk = t / kBlockTokens;
+    int32_t n = blockprefix[static_cast<int64_t>(h) * (n_blocks + 1) + blk];
+    if (blk < n_blocks) {
+        const uint32_t *w = maskbits + static_cast<int64_t>(h) * n_words + blk * 4;
+        const int r = static_cast<int>(t - blk * kBlockTokens);       // 0..127 bits of this block
+        for (int i = 0; i < 4; ++i) {
+            const int lo = i * 32;
+            if (r >= lo + 32) n += __popc(w[i]);
+            else if (r > lo) n += __popc(w[i] & ((1u << (r - lo)) - 1u));
+        }
+    }
+    return n;
+}
+
+// ---------------------------------------------------------------------------
+// One CTA of 1024 threads.  blockprefix [H][n_blocks+1], seqbase [H][n_seqs+1],
+// lengths [n_seqs][H].  Paged output (page_tokens > 0): list (b,h) gets
+// ceil(len/page_tokens) pages numbered contiguously from first_page in (b,h)
+// order; list_page0 [n_seqs*H] receives each list's first page and page_table
+// [n_seqs*H][max_pages] its page numbers; *n_pages_used the total.  A pool or
+// table that is too small sets the status word and marks every list with
+// list_page0 = -1 so that the compaction writes nothing.
+__global__ void __launch_bounds__(1024)
+scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
+            const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens,
+            int32_t *__restrict__ blockprefix, int32_t *__restrict__ seqbase, int32_t *__restrict__ lengths,
+            int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
+            int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
+            int32_t *__restrict__ status)
+{
+    __shared__ int32_t warp_sums[32];
+    __shared__ int32_t carry_s;
+    __shared__ int32_t fail_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    auto block_scan = [&](int32_t v, int32_t &total) -> int32_t {   // inclusive scan over the CTA
+        int32_t x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        __syncthreads();
+        if (lane == 31) warp_sums[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t w = warp_sums[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t y = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += y;
+            }
+            warp_sums[lane] = w;
+        }
+        __syncthreads();
+        total = warp_sums[31];
+        return x + (warp > 0 ? warp_sums[warp - 1] : 0);
+    };
+
+    for (int h = 0; h < n_heads; ++h) {
+        if (tid == 0) carry_s = 0;
+        __syncthreads();
+        for (int64_t base = 0; base < n_blocks; base += 1024) {
+            const int64_t blk = base + tid;
+            int32_t cnt = 0;
+            if (blk < n_blocks) {
+                const uint4 w = *reinterpret_cast<const uint4 *>(maskbits + static_cast<int64_t>(h) * n_words + blk * 4);
+                cnt = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
+            }
+            int32_t total;
+            const int32_t incl = block_scan(cnt, total);
+            const int32_t carry = carry_s;
+            if (blk < n_blocks) blockprefix[static_cast<int64_t>(h) * (n_blocks + 1) + blk] = carry + incl - cnt;
+            __syncthreads();
+            if (tid == 0) carry_s = carry + total;
+            __syncthreads();
+        }
+        if (tid == 0) blockprefix[static_cast<int64_t>(h) * (n_blocks + 1) + n_blocks] = carry_s;
+    }
+    __syncthreads();      // blockprefix written by this CTA is visible to it from here on
+
+    for (int idx = tid; idx < n_heads * (n_seqs + 1); idx += 1024) {
+        const int h = idx / (n_seqs + 1), b = idx % (n_seqs + 1);
+        const int64_t t = cu_seqlens != nullptr ? static_cast<int64_t>(cu_seqlens[b]) : (b == 0 ? 0 : n_tokens);
+        seqbase[idx] = kept_before(maskbits, n_words, blockprefix, n_blocks, h, t);
+    }
+    __syncthreads();
+    for (int idx = tid; idx < n_heads * n_seqs; idx += 1024) {
+        const int b = idx / n_heads, h = idx % n_heads;
+        lengths[idx] = seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
+    }
+    if (page_tokens <= 0) return;
+
+    // paged output: exclusive scan of the per-list page counts in (b,h) order
+    __syncthreads();
+    if (tid == 0) { carry_s = 0; fail_s = 0; }
+    __syncthreads();
+    const int n_lists = n_heads * n_seqs;
+    for (int base = 0; base < n_lists; base += 1024) {
+        const int idx = base + tid;
+        int32_t need = 0;
+        if (idx < n_lists) {
+            need = (lengths[idx] + page_tokens - 1) / page_tokens;
+            if (need > max_pages) fail_s = 1;
+        }
+        int32_t total;
+        const int32_t incl = block_scan(need, total);
+        const int32_t carry = carry_s;
+        if (idx < n_lists) list_page0[idx] = first_page + carry + incl - need;
+        __syncthreads();
+        if (tid == 0) carry_s = carry + total;
+        __syncthreads();
+    }
+    const int32_t used = carry_s;
+    const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + used > n_pages_pool;
+    if (fail) {
+        for (int idx = tid; idx < n_lists; idx += 1024) list_page0[idx] = -1;
+        if (tid == 0) { atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */); *n_pages_used = 0; }
+        return;
+    }
+    if (tid == 0) *n_pages_used = used;
+    for (int idx = tid; idx < n_lists; idx += 1024) {
+        const int32_t p0 = list_page0[idx];
+        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens;
+        for (int32_t i = 0; i < need; ++i) page_table[static_cast<int64_t>(idx) * max_pages + i] = p0 + i;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// One CTA per (128-token block, head).  Rows are row_bytes = 2*D bytes, moved
+// as 16-byte units by 16-lane groups; up to kRowsInFlight rows of K and of V
+// are loaded before any is stored.
+constexpr int kCompactThreads = 256;
+constexpr int kRowsInFlight = 4;
+
+template <bool kPaged>
+__global__ void __launch_bounds__(kCompactThreads)
+compact_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ K_out,
+               uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks,
+               const int32_t *__restrict__ blockprefix, const int32_t *__restrict__ seqbase,
+               const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens, int n_heads, int row_units,
+               int page_tokens, const int32_t *__restrict__ list_page0)
+{
+    __shared__ int32_t src_tok[kBlockTokens];     // packed token index of the i-th kept row of this block
+    __shared__ int64_t dst_row[kBlockTokens];     // its destination row (dense: within head h; paged: pool row)
+    const int64_t blk = blockIdx.x;
+    const int h = blockIdx.y;
+    const int tid = threadIdx.x;
+    const uint32_t *words = maskbits + static_cast<int64_t>(h) * n_words + blk * 4;
+    const uint32_t w0 = words[0], w1 = words[1], w2 = words[2], w3 = words[3];
+    const int cnt = __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
+    if (cnt == 0) return;
+    if (tid < kBlockTokens) {
+        const int wi = tid >> 5, bit = tid & 31;
+        const uint32_t w = wi == 0 ? w0 : wi == 1 ? w1 : wi == 2 ? w2 : w3;
+        if ((w >> bit) & 1u) {
+            int r = __popc(w & ((1u << bit) - 1u));
+            if (wi > 0) r += __popc(w0);
+            if (wi > 1) r += __popc(w1);
+            if (wi > 2) r += __popc(w2);
+            const int64_t t = blk * kBlockTokens + tid;
+            const int32_t before = blockprefix[static_cast<int64_t>(h) * (n_blocks + 1) + blk] + r;
+            int b = 0;
+            int64_t seq_start = 0;
+            if (cu_seqlens != nullptr && n_seqs > 1) {
+                b = seq_of_token(cu_seqlens, n_seqs, t);
+                seq_start = cu_seqlens[b];
+            }
+            const int64_t n = before - seqbase[h * (n_seqs + 1) + b];     // rank inside list (b,h)
+            int64_t dst;
+            if constexpr (kPaged) {
+                const int32_t p0 = list_page0[b * n_heads + h];
+                dst = p0 < 0 ? -1 : (static_cast<int64_t>(p0) + n / page_tokens) * page_tokens + n % page_tokens;
+            } else {
+                dst = static_cast<int64_t>(h) * n_tokens + seq_start + n;
+            }
+            src_tok[r] = static_cast<int32_t>(t - blk * kBlockTokens);
+            dst_row[r] = dst;
+        }
+    }
+    __syncthreads();
+
+    const int group = tid >> 4, gl = tid & 15;            // 16 groups of 16 lanes
+    constexpr int kGroups = kCompactThreads / 16;
+    const int64_t head_row0 = static_cast<int64_t>(h) * n_tokens + blk * kBlockTokens;
+    for (int i0 = group; i0 < cnt; i0 += kGroups * kRowsInFlight) {
+        for (int u0 = gl; u0 < row_units; u0 += 16) {
+            uint4 kv[kRowsInFlight], vv[kRowsInFlight];
+#pragma unroll
+            for (int j = 0; j < kRowsInFlight; ++j) {
+                const int i = i0 + j * kGroups;
+                if (i < cnt) {
+                    const int64_t src = (head_row0 + src_tok[i]) * row_units + u0;
+                    kv[j] = __ldg(K + src);
+                    vv[j] = __ldg(V + src);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kRowsInFlight; ++j) {
+                const int i = i0 + j * kGroups;
+                if (i < cnt) {
+                    const int64_t d = dst_row[i];
+                    if (d >= 0) {
+                        K_out[d * row_units + u0] = kv[j];
+                        V_out[d * row_units + u0] = vv[j];
+                    }
+                }
+            }
+        }
+    }
+}
+
+}  // namespace kvzap
