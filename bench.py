@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the KVzap pruning hot path on B200.
+
+A "step" is one pass of the whole hot path -- surrogate scoring, threshold and
+window mask, per-head prefix sums, K/V compaction -- over one batch of synthetic
+input for every layer of the workload.  Metric: tokens pruned per second per
+layer = B*T / (step time / n_layers).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line.  ``--impl reference`` times the CPU oracle (as it
+stands) on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tokens pruned/sec per layer"
+UNIT = "tokens/s/layer"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (bytes); None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            with open(path) as f:
+                d = json.load(f)
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def surrogate_flops_per_token(wl):
+    """Algorithmic FLOPs per token per layer (Appendix B): 2 D_h N1 + 2 N1 H, or 2 D_h H."""
+    if wl.surrogate == "mlp":
+        return 2.0 * wl.d_model * wl.hidden + 2.0 * wl.hidden * wl.n_kv_heads
+    return 2.0 * wl.d_model * wl.n_kv_heads
+
+
+def algorithmic_bytes_per_layer(wl, n_tokens, kept_rows):
+    """Hidden states read + scores written + kept K and V rows read and written + weights read once."""
+    row = 2 * wl.head_dim
+    w_bytes = (wl.hidden * wl.d_model * 2 + wl.hidden * wl.n_kv_heads * 2) if wl.surrogate == "mlp" \
+        else wl.n_kv_heads * wl.d_model * 2
+    return n_tokens * wl.d_model * 2 + n_tokens * wl.n_kv_heads * 4 + kept_rows * row * 2 * 2 + w_bytes
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.max_mhz = period, [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = [("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap")]
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for label, attr in names:
+                    if mask & int(getattr(nv, attr, 0)):
+                        self.reasons.add(label)
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2.0)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_sample(wl, n_tokens, seed=424242):
+    """Times the CPU oracle (scoring + mask + compaction) on the first n_tokens of one layer.
+    Returns (tokens per second per layer, seconds, threads)."""
+    import torch
+    from oracle import kvzap_oracle as oracle
+    from paper_2601_07891_b200 import synth
+    weights = synth.surrogate_weights(wl, 0, "cpu")
+    X = synth.hidden_states(n_tokens, wl.d_model, seed, "cpu", wl.token_scale_sigma)
+    K, V = synth.keys_values(wl.n_kv_heads, n_tokens, wl.head_dim, seed + 1, "cpu")
+    ow = tuple(synth.bits(t) if t.dtype == torch.bfloat16 else t.numpy() for t in weights)
+    Xb, Kb, Vb = synth.bits(X), synth.bits(K), synth.bits(V)
+    oracle.lib()
+    t0 = time.perf_counter()
+    oracle.prune_prefill(Xb, ow, Kb, Vb, wl.tau, wl.window)
+    dt = time.perf_counter() - t0
+    return n_tokens / dt, dt, oracle.num_threads()
+
+
+def run_reference(args, wl):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_sample = min(wl.batch * wl.seq_len, args.ref_tokens)
+    for _ in range(args.warmup):
+        oracle_sample(wl, min(n_sample, 256))
+    vals, secs, threads = [], 0.0, 1
+    for _ in range(args.steps):
+        v, dt, threads = oracle_sample(wl, n_sample)
+        vals.append(v)
+        secs += dt
+    value = n_sample * len(vals) / secs
+    sample = "one layer, first %d tokens of the prompt: scoring + mask + compaction, per step" % n_sample
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(len(vals), 1),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
+                       "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "n_layers": wl.n_layers,
+                       "batch": wl.batch, "seq_len": wl.seq_len, "tau": wl.tau, "window": wl.window},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2601_07891_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        # replicas only: the path needs no exchange; the process group carries the barrier and the max
+        dist.init_process_group("nccl", device_id=dev)
+
+    L, B, T = wl.n_layers, wl.batch, wl.seq_len
+    if args.layers > 0:
+        L = min(L, args.layers)          # small case for profiler captures; reported in config.n_layers
+    n_tokens = B * T
+    H, D = wl.n_kv_heads, wl.head_dim
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=local_rank)
+    cu = torch.from_numpy(synth.cu_seqlens([T] * B)).to(dev) if B > 1 else None
+
+    # resident inputs, one set per layer while they fit (every layer's inputs exceed L2, so no flush is
+    # needed); beyond ~60 GB the layers rotate over fewer input sets (weights stay distinct per layer)
+    per_layer_bytes = n_tokens * wl.d_model * 2 + 4 * H * n_tokens * D * 2
+    n_sets = L if L * per_layer_bytes <= 60e9 else max(2, int(60e9 // per_layer_bytes))
+    Xs, Ks, Vs, Kos, Vos, lens, scs = [], [], [], [], [], [], []
+    for l in range(L):
+        weights = synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index)
+        ctx.set_weights(l, *weights)
+        if l >= n_sets:
+            for lst in (Xs, Ks, Vs, Kos, Vos, scs):
+                lst.append(lst[l % n_sets])
+            lens.append(torch.zeros(B, H, dtype=torch.int32, device=dev))
+            continue
+        seed = 1000 * args.workload_index + l + 100000 * rank
+        Xs.append(synth.hidden_states(n_tokens, wl.d_model, seed, dev, wl.token_scale_sigma))
+        K, V = synth.keys_values(H, n_tokens, D, seed + 500, dev)
+        Ks.append(K)
+        Vs.append(V)
+        Kos.append(torch.empty_like(K))
+        Vos.append(torch.empty_like(V))
+        lens.append(torch.zeros(B, H, dtype=torch.int32, device=dev))
+        scs.append(torch.empty(n_tokens, H, dtype=torch.float32, device=dev))
+    torch.cuda.synchronize()
+
+    def step():
+        for l in range(L):
+            binding.kvzap_prefill_fused(ctx.handle, l, Xs[l], Ks[l], Vs[l], cu, B, wl.tau, wl.window,
+                                        Kos[l], Vos[l], lens[l], scs[l])
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n_warm = args.warmup if args.layers > 0 else max(args.warmup, 3)
+    for _ in range(n_warm):
+        step()
+    barrier()
+    if ctx.poll_status() != 0:
+        raise RuntimeError("device status word set during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count()
+    sampler.start()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    gpu_launches = ctx.launch_count() - launches0
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * n_tokens / (ms_per_step * 1e-3 / L)
+    if ctx.poll_status() != 0:
+        raise RuntimeError("device status word set during the timed region")
+
+    # per-kernel durations, measured live with CUDA events around every launch of a second pass
+    kept_rows = float(sum(int(x.sum().item()) for x in lens)) / L          # kept (head, token) rows per layer
+    binding.kvzap_set_profiling(ctx.handle, True)
+    prof_steps = max(1, min(args.steps, 5))
+    for _ in range(prof_steps):
+        step()
+    prof = {k: binding.kvzap_get_profile(ctx.handle, k) for k in ("score", "scan", "compact")}
+    binding.kvzap_set_profiling(ctx.handle, False)
+    peaks, peak_src = load_peaks()
+    score_ms = prof["score"][0] / max(prof["score"][1], 1)
+    compact_ms = prof["compact"][0] / max(prof["compact"][1], 1)
+    scan_ms = prof["scan"][0] / max(prof["scan"][1], 1)
+    flops_per_launch = surrogate_flops_per_token(wl) * n_tokens
+    score_bytes = n_tokens * wl.d_model * 2 + n_tokens * H * 4
+    t_tensor = flops_per_launch / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_hbm = score_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        achieved = flops_per_launch / (score_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
+                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"]}
+    else:
+        achieved = score_bytes / (score_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"]}
+    roofline.update({"traffic": NCU_TRAFFIC_BYTES.get(wl.name), "kernel": "score_kernel", "peak_source": peak_src,
+                     "kernel_ms": score_ms})
+    # whole layer against max(tensor time, HBM time of all algorithmic bytes)
+    layer_bytes = algorithmic_bytes_per_layer(wl, n_tokens, kept_rows)
+    t_roof_layer = max(t_tensor, layer_bytes / (peaks["hbm_gbs"] * 1e9))
+    compact_bytes = kept_rows * 2 * D * 2 * 2
+    extra = {"layer_ms": ms_per_step / L, "layer_roofline_ms": t_roof_layer * 1e3,
+             "layer_frac_of_roofline": t_roof_layer * 1e3 / (ms_per_step / L),
+             "score_ms": score_ms, "scan_ms": scan_ms, "compact_ms": compact_ms,
+             "compact_GBps": compact_bytes / (compact_ms * 1e-3) / 1e9 if compact_ms > 0 else None,
+             "compact_frac_of_hbm": (compact_bytes / (compact_ms * 1e-3) / 1e9) / peaks["hbm_gbs"] if compact_ms > 0 else None,
+             "kept_fraction": kept_rows / (H * n_tokens)}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
+                       "n_kv_heads": H, "head_dim": D, "n_layers": L, "batch": B, "seq_len": T, "tau": wl.tau,
+                       "window": wl.window, "input_sets": n_sets,
+                       "l2": "inputs larger than L2 (distinct resident buffers per layer)",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
+
+    if rank == 0 and world == 1 and not args.skip_e2e:
+        # end to end through the host-buffer entry point: H2D of the layer's inputs and D2H of its
+        # result happen inside the timed region; host inputs rotate over a few pinned layer sets
+        n_sets = min(L, 2)
+        hX = [Xs[i].cpu().pin_memory() for i in range(n_sets)]
+        hK = [Ks[i].cpu().pin_memory() for i in range(n_sets)]
+        hV = [Vs[i].cpu().pin_memory() for i in range(n_sets)]
+        hKo, hVo = torch.empty_like(hK[0]).pin_memory(), torch.empty_like(hV[0]).pin_memory()
+        hlen = torch.zeros(B, H, dtype=torch.int32).pin_memory()
+        hcu = torch.from_numpy(synth.cu_seqlens([T] * B)) if B > 1 else None
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+
+        def e2e_step():
+            for l in range(L):
+                i = l % n_sets
+                binding.kvzap_prefill_fused_host(ctx.handle, l, hX[i], hK[i], hV[i], hcu, B, wl.tau, wl.window,
+                                                 hKo, hVo, hlen, None)
+        e2e_step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+        h2d = L * (n_tokens * wl.d_model * 2 + 2 * H * n_tokens * D * 2 + (4 * (B + 1) if B > 1 else 0))
+        d2h = int(L * (kept_rows * 2 * D * 2 + B * H * 4))
+        line["e2e"] = {"value": n_tokens / (e2e_ms * 1e-3 / L), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                       "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
+                       "note": "kvzap_prefill_fused_host: pinned host buffers, copies inside the timed region"}
+        del hX, hK, hV, hKo, hVo
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        # the oracle on the host cores, bounded sample
+        n_sample = min(n_tokens, args.ref_tokens)
+        v, dt, threads = oracle_sample(wl, n_sample)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": "one layer, first %d tokens: scoring + mask + compaction (%.1f s)" % (n_sample, dt)}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    from paper_2601_07891_b200 import synth
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_8b_prefill_32k", choices=[w for w in synth.WORKLOAD_ORDER
+                                                                         if synth.WORKLOADS[w].decode_steps == 0])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (small case for profiling)")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--ref-tokens", type=int, default=32768,
+                    help="tokens of one layer the CPU oracle is timed on (bounded sample)")
+    args = ap.parse_args()
+    args.workload_index = synth.WORKLOAD_ORDER.index(args.workload) + 1
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        if args.steps > 3:
+            args.ref_tokens = min(args.ref_tokens, 4096)     # keep the whole run within minutes
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -141,6 +141,37 @@ kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidd
                                  float *scores_out, void *stream);
 
 /*
+ * kvzap_prefill_fused for callers whose tensors live in HOST memory (pinned
+ * memory recommended).  Every pointer argument, cu_seqlens included, is a HOST
+ * pointer with the same shapes as above.  The call copies the inputs into
+ * device staging buffers owned by the context (allocated at the first call,
+ * sized for max_tokens), runs Algorithm 1 on the device, synchronises
+ * `stream`, and copies back lengths, the scores (if scores_out != NULL) and,
+ * for every (sequence, head) list, exactly its lengths[b,h] kept rows into the
+ * same positions of K_out / V_out; other rows of the host outputs are left
+ * untouched.  Returns after the results are in host memory.
+ */
+kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                      const void *K, const void *V,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                      float tau, int32_t w,
+                                      void *K_out, void *V_out, int32_t *lengths,
+                                      float *scores_out, void *stream);
+
+/* Kernel identifiers for kvzap_get_profile. */
+enum { KVZAP_KERNEL_SCORE = 0, KVZAP_KERNEL_MASK = 1, KVZAP_KERNEL_SCAN = 2, KVZAP_KERNEL_COMPACT = 3 };
+
+/*
+ * Per-kernel timing with CUDA events on the launching stream (a measurement
+ * aid; the paper has no counterpart).  While enabled, every kernel launch is
+ * bracketed by two events.  kvzap_set_profiling(ctx, 0/1) switches it and
+ * discards earlier records; kvzap_get_profile synchronises the device and
+ * returns the summed duration and the number of launches of one kernel.
+ */
+kvzap_status kvzap_set_profiling(kvzap_ctx *ctx, int32_t enable);
+kvzap_status kvzap_get_profile(kvzap_ctx *ctx, int32_t kernel, double *total_ms, int64_t *n_launches);
+
+/*
  * Reads the context's device status word (synchronises `stream` first) and
  * clears it.  Returns KVZAP_OK, or the first device-side condition recorded
  * since the last poll (KVZAP_ERR_TIMEOUT, KVZAP_ERR_OOM_PAGES).

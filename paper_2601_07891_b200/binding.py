@@ -49,6 +49,10 @@ SIGNATURES = {
     "kvzap_score": (_i32, [_vp, _i32, _vp, _i64, _vp, _vp]),
     "kvzap_prune_prefill": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_fused": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_fused_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp,
+                                        _vp]),
+    "kvzap_set_profiling": (_i32, [_vp, _i32]),
+    "kvzap_get_profile": (_i32, [_vp, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)]),
     "kvzap_poll_status": (_i32, [_vp, _vp]),
     "kvzap_launch_count": (_i64, [_vp]),
 }
@@ -138,6 +142,37 @@ def kvzap_prefill_fused(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w,
         handle, layer, _ptr(hidden) if nz else None, _ptr(K) if nz else None, _ptr(V) if nz else None,
         _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
         _ptr(lengths), _ptr(scores_out) if nz else None, _stream(stream)))
+
+
+def _hptr(t):
+    if t is None:
+        return None
+    assert not t.is_cuda and t.is_contiguous(), "host entry point takes contiguous CPU tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def kvzap_prefill_fused_host(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                             scores_out=None, stream=None):
+    """All tensors are HOST tensors (pinned recommended); returns after the results are on the host."""
+    n_tokens = K.shape[1]
+    _check(handle, load().kvzap_prefill_fused_host(
+        handle, layer, _hptr(hidden), _hptr(K), _hptr(V), _hptr(cu_seqlens), n_seqs, n_tokens, tau, w,
+        _hptr(K_out), _hptr(V_out), _hptr(lengths), _hptr(scores_out), _stream(stream)))
+
+
+KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3}
+
+
+def kvzap_set_profiling(handle, enable):
+    _check(handle, load().kvzap_set_profiling(handle, 1 if enable else 0))
+
+
+def kvzap_get_profile(handle, kernel):
+    """-> (total_ms, n_launches) of one kernel since profiling was switched on."""
+    ms, n = ctypes.c_double(0.0), ctypes.c_int64(0)
+    _check(handle, load().kvzap_get_profile(handle, KERNEL_IDS[kernel] if isinstance(kernel, str) else kernel,
+                                            ctypes.byref(ms), ctypes.byref(n)))
+    return float(ms.value), int(n.value)
 
 
 def kvzap_poll_status(handle, stream=None) -> int:

@@ -51,6 +51,15 @@ struct kvzap_ctx {
     int32_t *status_dev = nullptr;
     int32_t *status_host = nullptr;  // pinned
     int64_t launches = 0;
+    // optional per-kernel timing (kvzap_set_profiling)
+    bool profiling = false;
+    struct ProfRec { int kind; cudaEvent_t start, stop; };
+    std::vector<ProfRec> prof;
+    // device staging for the host-buffer entry point (allocated on first use)
+    void *stage_x = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_ko = nullptr, *stage_vo = nullptr;
+    float *stage_scores = nullptr;
+    int32_t *stage_lengths = nullptr, *stage_cu = nullptr;
+    int32_t *lengths_pinned = nullptr;
     char err[512] = "";
 };
 
@@ -112,6 +121,25 @@ __global__ void pack_w2_kernel(const uint16_t *__restrict__ W2, const float *__r
     if (idx < kMaxHeads) b2p[idx] = (b2 != nullptr && idx < n_heads) ? b2[idx] : 0.0f;
 }
 
+// Brackets one kernel launch with events when profiling is on.
+struct ProfScope {
+    kvzap_ctx *ctx;
+    cudaStream_t stream;
+    cudaEvent_t stop = nullptr;
+    ProfScope(kvzap_ctx *c, int kind, cudaStream_t s) : ctx(c), stream(s)
+    {
+        if (!ctx->profiling) return;
+        cudaEvent_t start = nullptr;
+        if (cudaEventCreate(&start) != cudaSuccess || cudaEventCreate(&stop) != cudaSuccess) { stop = nullptr; return; }
+        cudaEventRecord(start, stream);
+        ctx->prof.push_back({kind, start, stop});
+    }
+    ~ProfScope()
+    {
+        if (stop) cudaEventRecord(stop, stream);
+    }
+};
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;
@@ -138,6 +166,12 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->seqbase);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
+    for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    ctx->prof.clear();
+    cudaFree(ctx->stage_x); cudaFree(ctx->stage_k); cudaFree(ctx->stage_v);
+    cudaFree(ctx->stage_ko); cudaFree(ctx->stage_vo); cudaFree(ctx->stage_scores);
+    cudaFree(ctx->stage_lengths); cudaFree(ctx->stage_cu);
+    if (ctx->lengths_pinned) cudaFreeHost(ctx->lengths_pinned);
 }
 
 static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seqs, const int32_t *cu_seqlens)
@@ -194,10 +228,13 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, const void *hidd
     p.tau = tau;
     p.status = ctx->status_dev;
     const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
-    if (c.hidden > 0)
-        score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
-    else
-        score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
+        if (c.hidden > 0)
+            score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+        else
+            score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+    }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
     return KVZAP_OK;
@@ -211,15 +248,21 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const void *K, const void 
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     const int64_t n_words = n_blocks * 4;
-    scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs, n_tokens,
-                                        ctx->blockprefix, ctx->seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr,
-                                        ctx->status_dev);
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
+        scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
+                                            n_tokens, ctx->blockprefix, ctx->seqbase, lengths, 0, 0, 0, 0, nullptr,
+                                            nullptr, nullptr, ctx->status_dev);
+    }
     KVZAP_CUDA(ctx, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
-    compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
-        static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
-        static_cast<uint4 *>(V_out), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
-        n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, 0, nullptr);
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
+        compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
+            static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
+            static_cast<uint4 *>(V_out), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
+            n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, 0, nullptr);
+    }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 2;
     return KVZAP_OK;
@@ -448,8 +491,12 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     if (st != KVZAP_OK) return st;
     if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-    mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads, cu_seqlens,
-                                                                     n_seqs, tau, w, ctx->maskbits, n_blocks * 4);
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
+        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
+                                                                         cu_seqlens, n_seqs, tau, w, ctx->maskbits,
+                                                                         n_blocks * 4);
+    }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
     return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
@@ -492,6 +539,102 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     if (v == 0) return KVZAP_OK;
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
+}
+
+kvzap_status kvzap_set_profiling(kvzap_ctx *ctx, int32_t enable)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    ctx->prof.clear();
+    ctx->profiling = enable != 0;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_get_profile(kvzap_ctx *ctx, int32_t kernel, double *total_ms, int64_t *n_launches)
+{
+    if (!ctx || !total_ms || !n_launches) return KVZAP_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    KVZAP_CUDA(ctx, cudaDeviceSynchronize());
+    double sum = 0.0;
+    int64_t n = 0;
+    for (auto &r : ctx->prof) {
+        if (r.kind != kernel) continue;
+        float ms = 0.0f;
+        KVZAP_CUDA(ctx, cudaEventElapsedTime(&ms, r.start, r.stop));
+        sum += ms;
+        ++n;
+    }
+    *total_ms = sum;
+    *n_launches = n;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                      int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
+                                      void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
+    if (n_tokens == 0) {
+        memset(lengths, 0, sizeof(int32_t) * n_seqs * c.n_kv_heads);
+        return KVZAP_OK;
+    }
+    if (!hidden || !K || !V || !K_out || !V_out)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden, K, V, K_out and V_out must not be NULL");
+    DeviceGuard guard(c.device);
+    const size_t row_bytes = static_cast<size_t>(c.head_dim) * 2;
+    const size_t kv_cap = static_cast<size_t>(c.n_kv_heads) * c.max_tokens * row_bytes;
+    if (!ctx->stage_x) {
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_x, static_cast<size_t>(c.max_tokens) * c.d_model * 2));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_k, kv_cap));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_v, kv_cap));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_ko, kv_cap));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_vo, kv_cap));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_scores, sizeof(float) * c.max_tokens * c.n_kv_heads));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_lengths, sizeof(int32_t) * c.max_seqs * c.n_kv_heads));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_cu, sizeof(int32_t) * (static_cast<size_t>(c.max_seqs) + 1)));
+        KVZAP_CUDA(ctx, cudaMallocHost(&ctx->lengths_pinned, sizeof(int32_t) * c.max_seqs * c.n_kv_heads));
+    }
+    const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * row_bytes;
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_x, hidden, static_cast<size_t>(n_tokens) * c.d_model * 2,
+                                    cudaMemcpyHostToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_k, K, kv_bytes, cudaMemcpyHostToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_v, V, kv_bytes, cudaMemcpyHostToDevice, stream));
+    if (cu_seqlens)
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_cu, cu_seqlens, sizeof(int32_t) * (n_seqs + 1),
+                                        cudaMemcpyHostToDevice, stream));
+    st = kvzap_prefill_fused(ctx, layer, ctx->stage_x, ctx->stage_k, ctx->stage_v, cu_seqlens ? ctx->stage_cu : nullptr,
+                             n_seqs, n_tokens, tau, w, ctx->stage_ko, ctx->stage_vo, ctx->stage_lengths,
+                             scores_out ? ctx->stage_scores : nullptr, stream);
+    if (st != KVZAP_OK) return st;
+    const size_t n_lists = static_cast<size_t>(n_seqs) * c.n_kv_heads;
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->lengths_pinned, ctx->stage_lengths, sizeof(int32_t) * n_lists,
+                                    cudaMemcpyDeviceToHost, stream));
+    if (scores_out)
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(scores_out, ctx->stage_scores, sizeof(float) * n_tokens * c.n_kv_heads,
+                                        cudaMemcpyDeviceToHost, stream));
+    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
+    memcpy(lengths, ctx->lengths_pinned, sizeof(int32_t) * n_lists);
+    for (int b = 0; b < n_seqs; ++b) {
+        const int64_t seq_start = cu_seqlens ? cu_seqlens[b] : 0;
+        for (int h = 0; h < c.n_kv_heads; ++h) {
+            const int32_t n = lengths[b * c.n_kv_heads + h];
+            if (n <= 0) continue;
+            const size_t off = (static_cast<size_t>(h) * n_tokens + seq_start) * row_bytes;
+            KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(K_out) + off, static_cast<char *>(ctx->stage_ko) + off,
+                                            n * row_bytes, cudaMemcpyDeviceToHost, stream));
+            KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(V_out) + off, static_cast<char *>(ctx->stage_vo) + off,
+                                            n * row_bytes, cudaMemcpyDeviceToHost, stream));
+        }
+    }
+    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
+    return KVZAP_OK;
 }
 
 }  // extern "C"
