@@ -172,6 +172,44 @@ kvzap_status kvzap_set_profiling(kvzap_ctx *ctx, int32_t enable);
 kvzap_status kvzap_get_profile(kvzap_ctx *ctx, int32_t kernel, double *total_ms, int64_t *n_launches);
 
 /*
+ * kvzap_prune_prefill for callers that cannot allocate device memory.  (The
+ * paper has no counterpart; this is a deployment variant of the same
+ * operation.)
+ *
+ * Who needs it: a serving process that handed all of the GPU's memory to its
+ * own KV-cache pool at start-up, so that a later cudaMalloc (which
+ * kvzap_create performs) fails or steals from that pool; and latency-critical
+ * loops that may not call cudaMalloc/cudaFree because those calls stall every
+ * stream of the device while they run.  This entry point needs no context and
+ * never calls cudaMalloc, cudaFree or any other allocating routine.
+ *
+ * Instead of a context's scratch it uses one fixed array compiled into the
+ * library's device image (about 170 KB, held by every GPU that loads the
+ * library until the process exits).  Consequences:
+ *   - sizes are capped: n_tokens <= KVZAP_NOALLOC_MAX_TOKENS and
+ *     n_seqs <= KVZAP_NOALLOC_MAX_SEQS, else KVZAP_ERR_UNSUPPORTED is returned
+ *     and nothing is launched;
+ *   - it works on the CURRENT device (cudaSetDevice), where all pointers must
+ *     live; the first call on each device also looks up the array's device
+ *     address, so make that first call before starting any stream capture;
+ *   - all calls on a device share the array, which still holds the previous
+ *     call's contents (the call rewrites everything it reads, and clears its
+ *     status word): two calls that overlap on the GPU -- different streams, or
+ *     different host threads -- race on it and produce garbage.  Serialise
+ *     them on one stream.
+ * Arguments and results are exactly those of kvzap_prune_prefill, with the
+ * two shape parameters a context would have carried (n_kv_heads 1..8, head_dim
+ * a multiple of 8 in 8..1024) passed explicitly.  Error text is available
+ * from kvzap_last_error(NULL).
+ */
+#define KVZAP_NOALLOC_MAX_TOKENS 131072
+#define KVZAP_NOALLOC_MAX_SEQS 256
+kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V, const float *scores,
+                                         const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                         int32_t n_kv_heads, int32_t head_dim, float tau, int32_t w,
+                                         void *K_out, void *V_out, int32_t *lengths, void *stream);
+
+/*
  * Reads the context's device status word (synchronises `stream` first) and
  * clears it.  Returns KVZAP_OK, or the first device-side condition recorded
  * since the last poll (KVZAP_ERR_TIMEOUT, KVZAP_ERR_OOM_PAGES).

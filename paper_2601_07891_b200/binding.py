@@ -51,6 +51,7 @@ SIGNATURES = {
     "kvzap_prefill_fused": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_fused_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp,
                                         _vp]),
+    "kvzap_prune_prefill_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _f32, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_set_profiling": (_i32, [_vp, _i32]),
     "kvzap_get_profile": (_i32, [_vp, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)]),
     "kvzap_poll_status": (_i32, [_vp, _vp]),
@@ -160,6 +161,22 @@ def kvzap_prefill_fused_host(handle, layer, hidden, K, V, cu_seqlens, n_seqs, ta
         _hptr(K_out), _hptr(V_out), _hptr(lengths), _hptr(scores_out), _stream(stream)))
 
 
+NOALLOC_MAX_TOKENS = 131072
+NOALLOC_MAX_SEQS = 256
+
+
+def kvzap_prune_prefill_noalloc(K, V, scores, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths, stream=None):
+    """kvzap_prune_prefill without a context and without any allocation: the scratch is a fixed
+    array inside the library (limits NOALLOC_MAX_TOKENS / NOALLOC_MAX_SEQS).  Works on the current
+    device; calls that overlap on the GPU race on that array, so keep them on one stream."""
+    n_heads, n_tokens, head_dim = K.shape
+    nz = n_tokens > 0
+    _check(None, load().kvzap_prune_prefill_noalloc(
+        _ptr(K) if nz else None, _ptr(V) if nz else None, _ptr(scores) if nz else None, _ptr(cu_seqlens), n_seqs,
+        n_tokens, n_heads, head_dim, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
+        _ptr(lengths), _stream(stream)))
+
+
 KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3}
 
 
@@ -211,10 +228,22 @@ class Kvzap:
             kvzap_set_weights(self.handle, layer, *weights, stream=stream)
 
     def score(self, layer, hidden, out=None, stream=None):
+        if hidden.dim() != 2 or hidden.shape[1] != self.d_model or hidden.dtype != torch.bfloat16:
+            raise ValueError("hidden must be bf16 [T, %d], got %s" % (self.d_model, tuple(hidden.shape)))
         if out is None:
             out = torch.empty(hidden.shape[0], self.n_kv_heads, dtype=torch.float32, device=self.device)
         kvzap_score(self.handle, layer, hidden, out, stream)
         return out
+
+    def _check_shapes(self, K, V, hidden=None, scores=None):
+        """Shape errors are raised here, on the host: the C ABI takes raw pointers and trusts them."""
+        if tuple(K.shape[::2]) != (self.n_kv_heads, self.head_dim) or K.shape != V.shape or K.dtype != torch.bfloat16:
+            raise ValueError("K/V must be bf16 [%d, T, %d], got %s / %s" % (self.n_kv_heads, self.head_dim,
+                                                                            tuple(K.shape), tuple(V.shape)))
+        if hidden is not None and (hidden.shape != (K.shape[1], self.d_model) or hidden.dtype != torch.bfloat16):
+            raise ValueError("hidden must be bf16 [%d, %d], got %s" % (K.shape[1], self.d_model, tuple(hidden.shape)))
+        if scores is not None and (scores.shape != (K.shape[1], self.n_kv_heads) or scores.dtype != torch.float32):
+            raise ValueError("scores must be fp32 [%d, %d], got %s" % (K.shape[1], self.n_kv_heads, tuple(scores.shape)))
 
     def _outputs(self, K, n_seqs, K_out, V_out, lengths):
         if K_out is None:
@@ -227,6 +256,7 @@ class Kvzap:
 
     def prune_prefill(self, K, V, scores, tau, w, cu_seqlens=None, K_out=None, V_out=None, lengths=None, stream=None):
         n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        self._check_shapes(K, V, scores=scores)
         K_out, V_out, lengths = self._outputs(K, n_seqs, K_out, V_out, lengths)
         kvzap_prune_prefill(self.handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths, stream)
         return K_out, V_out, lengths
@@ -234,6 +264,7 @@ class Kvzap:
     def prefill_fused(self, layer, hidden, K, V, tau, w, cu_seqlens=None, K_out=None, V_out=None, lengths=None,
                       scores_out=None, stream=None):
         n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        self._check_shapes(K, V, hidden=hidden, scores=scores_out)
         K_out, V_out, lengths = self._outputs(K, n_seqs, K_out, V_out, lengths)
         kvzap_prefill_fused(self.handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
                             scores_out, stream)

@@ -638,3 +638,104 @@ kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void 
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Allocation-free variant of kvzap_prune_prefill.
+//
+// Its scratch (mask words, block prefix sums, per-sequence bases, a status word)
+// lives in the file-scope device array below instead of a context's cudaMalloc'd
+// buffers, so that a caller who must not allocate can still prune.  Every GPU that
+// loads this library carries the array (about 170 KB) until the process exits.
+namespace kvzap {
+
+constexpr int64_t kNoAllocMaxTokens = KVZAP_NOALLOC_MAX_TOKENS;
+constexpr int kNoAllocMaxSeqs = KVZAP_NOALLOC_MAX_SEQS;
+constexpr int64_t kNoAllocMaxBlocks = (kNoAllocMaxTokens + kBlockTokens - 1) / kBlockTokens;
+constexpr size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+constexpr size_t kNoAllocMaskOff = 0;
+constexpr size_t kNoAllocMaskBytes = round256(sizeof(uint32_t) * kMaxHeads * kNoAllocMaxBlocks * 4);
+constexpr size_t kNoAllocPrefixOff = kNoAllocMaskOff + kNoAllocMaskBytes;
+constexpr size_t kNoAllocPrefixBytes = round256(sizeof(int32_t) * kMaxHeads * (kNoAllocMaxBlocks + 1));
+constexpr size_t kNoAllocSeqOff = kNoAllocPrefixOff + kNoAllocPrefixBytes;
+constexpr size_t kNoAllocSeqBytes = round256(sizeof(int32_t) * kMaxHeads * (kNoAllocMaxSeqs + 1));
+constexpr size_t kNoAllocStatusOff = kNoAllocSeqOff + kNoAllocSeqBytes;
+constexpr size_t kNoAllocBytes = kNoAllocStatusOff + 256;
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kNoAllocMaxDevices = 64;
+static void *g_noalloc_dev_ptr[kNoAllocMaxDevices];      // device address of the array, per device ordinal
+
+}  // namespace kvzap
+
+extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V, const float *scores,
+                                                    const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                                    int32_t n_kv_heads, int32_t head_dim, float tau, int32_t w,
+                                                    void *K_out, void *V_out, int32_t *lengths, void *stream_)
+{
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (n_kv_heads < 1 || n_kv_heads > kMaxHeads)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "noalloc: n_kv_heads %d: need 1..8", n_kv_heads);
+    if (head_dim < 8 || head_dim > 1024 || head_dim % 8)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "noalloc: head_dim %d: need a multiple of 8 in 8..1024", head_dim);
+    if (n_tokens < 0) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: n_tokens is negative");
+    if (n_tokens > kNoAllocMaxTokens)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED,
+                    "noalloc: n_tokens %lld exceeds the static scratch's limit KVZAP_NOALLOC_MAX_TOKENS = %lld",
+                    static_cast<long long>(n_tokens), static_cast<long long>(kNoAllocMaxTokens));
+    if (n_seqs < 1 || n_seqs > kNoAllocMaxSeqs)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED,
+                    "noalloc: n_seqs %d outside 1..KVZAP_NOALLOC_MAX_SEQS (%d)", n_seqs, kNoAllocMaxSeqs);
+    if (cu_seqlens == nullptr && n_seqs != 1)
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: cu_seqlens is NULL but n_seqs is %d", n_seqs);
+    if (!lengths) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: lengths is NULL");
+    if (w < 0) return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: window w is negative");
+
+    // once per device, with that device current: resolve the array's device address
+    int dev = -1;
+    KVZAP_CUDA(nullptr, cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kNoAllocMaxDevices)
+        return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "noalloc: device ordinal %d not supported", dev);
+    void *base = g_noalloc_dev_ptr[dev];
+    if (base == nullptr) {
+        void *ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+        if (e != cudaSuccess || ptr == nullptr)
+            return fail(nullptr, KVZAP_ERR_CUDA, "noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        g_noalloc_dev_ptr[dev] = ptr;
+        base = ptr;
+    }
+    if (n_tokens == 0) {
+        KVZAP_CUDA(nullptr, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * n_kv_heads, stream));
+        return KVZAP_OK;
+    }
+    if (!K || !V || !K_out || !V_out || !scores)
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: K, V, scores, K_out and V_out must not be NULL");
+    if (!aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out))
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "noalloc: K/V pointers must be 16-byte aligned");
+
+    unsigned char *b8 = static_cast<unsigned char *>(base);
+    uint32_t *maskbits = reinterpret_cast<uint32_t *>(b8 + kNoAllocMaskOff);
+    int32_t *blockprefix = reinterpret_cast<int32_t *>(b8 + kNoAllocPrefixOff);
+    int32_t *seqbase = reinterpret_cast<int32_t *>(b8 + kNoAllocSeqOff);
+    int32_t *status = reinterpret_cast<int32_t *>(b8 + kNoAllocStatusOff);
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    const int64_t n_words = n_blocks * 4;
+    // The array keeps whatever the previous call left.  Every mask word, prefix and base entry
+    // that this call reads is first written by it; only the status word must start at zero.
+    KVZAP_CUDA(nullptr, cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
+    mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, n_kv_heads, cu_seqlens, n_seqs,
+                                                                     tau, w, maskbits, n_words);
+    KVZAP_CUDA(nullptr, cudaGetLastError());
+    scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
+                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, status);
+    KVZAP_CUDA(nullptr, cudaGetLastError());
+    const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(n_kv_heads));
+    compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
+        static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
+        static_cast<uint4 *>(V_out), maskbits, n_words, n_blocks, blockprefix, seqbase, cu_seqlens, n_seqs, n_tokens,
+        n_kv_heads, head_dim / 8, 0, nullptr);
+    KVZAP_CUDA(nullptr, cudaGetLastError());
+    return KVZAP_OK;
+}
