@@ -20,14 +20,6 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-struct LayerWeights {
-    void *w1 = nullptr;      // bf16 [rows_padded, d_model]
-    float *b1 = nullptr;     // [rows_padded]
-    float *w2t = nullptr;    // [hidden][8] fp32 (MLP)
-    float *b2 = nullptr;     // [8] (MLP)
-    CUtensorMap tmap_w;
-    bool set = false;
-};
 
 static char g_create_error[512] = "";
 
@@ -41,7 +33,13 @@ struct kvzap_ctx {
     int group_w = 0, n_groups = 0, chunk_n = 0, n_chunks = 0, n_stages = 0, acc_bufs = 0, acc_stride = 0,
         tmem_cols = 0;
     uint32_t score_smem = 0;
-    std::vector<kvzap::LayerWeights> layers;
+    // weights of all layers, stacked so that one tensor map / one base pointer serves any layer range
+    void *w1_all = nullptr;          // bf16 [L * w1_rows, d_model]
+    float *b1_all = nullptr;         // [L][w1_rows]
+    float *w2t_all = nullptr;        // [L][hidden][8] fp32 (MLP)
+    float *b2_all = nullptr;         // [L][8] (MLP)
+    CUtensorMap tmap_w;
+    std::vector<char> layer_set;
     kvzap::EncodeTiledFn encode = nullptr;
     // scratch
     int64_t max_blocks = 0, max_words = 0;
@@ -89,16 +87,17 @@ static int next_pow2(int v)
     return p;
 }
 
-// 2-D bf16 tensor map: `rows` x `cols` row-major, box `box_rows` x 64 elements, 128-byte swizzle.
+// bf16 tensor map over `slabs` matrices of `rows` x `cols` (row-major, slabs contiguous); box = one slab,
+// `box_rows` rows, 64 elements; 128-byte swizzle.  slabs == 0 makes a 2-D map.
 static kvzap_status make_tmap(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
-                              uint32_t box_rows)
+                              uint32_t box_rows, uint64_t slabs = 0)
 {
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(kBlockK), box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
-                                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    const cuuint64_t dims[3] = {cols, rows, slabs ? slabs : 1};
+    const cuuint64_t strides[2] = {cols * 2, cols * 2 * rows};
+    const cuuint32_t box[3] = {static_cast<cuuint32_t>(kBlockK), box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, slabs ? 3 : 2, const_cast<void *>(base), dims,
+                                   strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(ctx, KVZAP_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d (rows=%llu cols=%llu box_rows=%u)",
@@ -155,12 +154,10 @@ struct DeviceGuard {
 
 static void free_all(kvzap_ctx *ctx)
 {
-    for (auto &lw : ctx->layers) {
-        cudaFree(lw.w1);
-        cudaFree(lw.b1);
-        cudaFree(lw.w2t);
-        cudaFree(lw.b2);
-    }
+    cudaFree(ctx->w1_all);
+    cudaFree(ctx->b1_all);
+    cudaFree(ctx->w2t_all);
+    cudaFree(ctx->b2_all);
     cudaFree(ctx->maskbits);
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
@@ -189,22 +186,27 @@ static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seq
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Launches the scoring kernel; maskbits != nullptr fuses the threshold/window test.
-static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens, float *scores,
-                                 uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs, float tau, int32_t w,
-                                 cudaStream_t stream)
+// Launches the scoring kernel over layers [layer, layer + n_layers); hidden is [n_layers][n_tokens][d_model],
+// scores [n_layers][n_tokens][H]; maskbits != nullptr fuses the threshold/window test.
+static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
+                                 float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
+                                 float tau, int32_t w, cudaStream_t stream)
 {
     const kvzap_config &c = ctx->cfg;
-    LayerWeights &lw = ctx->layers[layer];
-    const int64_t n_tiles = (n_tokens + kTileM - 1) / kTileM;
+    const int64_t tiles_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    const int64_t n_tiles = tiles_per_layer * n_layers;
     CUtensorMap tmap_x;
     kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model),
-                                kTileM);
+                                kTileM, static_cast<uint64_t>(n_layers));
     if (st != KVZAP_OK) return st;
     ScoreParams p;
     memset(&p, 0, sizeof p);
     p.n_tokens = n_tokens;
     p.n_tiles = static_cast<int32_t>(n_tiles);
+    p.tiles_per_layer = static_cast<int32_t>(tiles_per_layer);
+    p.n_layers_call = n_layers;
+    p.layer0 = layer;
+    p.w_rows = ctx->w1_rows;
     p.d_model = c.d_model;
     p.group_w = ctx->group_w;
     p.n_groups = ctx->n_groups;
@@ -216,12 +218,12 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, const void *hidd
     p.tmem_cols = ctx->tmem_cols;
     p.n_hidden = c.hidden;
     p.n_heads = c.n_kv_heads;
-    p.b1 = lw.b1;
-    p.w2t = lw.w2t;
-    p.b2 = lw.b2;
+    p.b1 = ctx->b1_all;
+    p.w2t = ctx->w2t_all;
+    p.b2 = ctx->b2_all;
     p.scores = scores;
     p.maskbits = maskbits;
-    p.n_words = n_tiles * 4;
+    p.n_words = tiles_per_layer * 4;
     p.cu_seqlens = cu_seqlens;
     p.n_seqs = n_seqs;
     p.window = w;
@@ -231,9 +233,9 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, const void *hidd
     {
         ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
         if (c.hidden > 0)
-            score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+            score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, ctx->tmap_w, p);
         else
-            score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, lw.tmap_w, p);
+            score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, ctx->tmap_w, p);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
@@ -377,20 +379,20 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      static_cast<int>(ctx->score_smem)));
 
-    ctx->layers.resize(c.n_layers);
-    for (auto &lw : ctx->layers) {
-        const size_t w1_bytes = static_cast<size_t>(ctx->w1_rows) * c.d_model * 2;
-        CREATE_CUDA(cudaMalloc(&lw.w1, w1_bytes));
-        CREATE_CUDA(cudaMemset(lw.w1, 0, w1_bytes));
-        CREATE_CUDA(cudaMalloc(&lw.b1, sizeof(float) * ctx->w1_rows));
-        CREATE_CUDA(cudaMemset(lw.b1, 0, sizeof(float) * ctx->w1_rows));
+    ctx->layer_set.assign(c.n_layers, 0);
+    {
+        const size_t w1_bytes = static_cast<size_t>(c.n_layers) * ctx->w1_rows * c.d_model * 2;
+        CREATE_CUDA(cudaMalloc(&ctx->w1_all, w1_bytes));
+        CREATE_CUDA(cudaMemset(ctx->w1_all, 0, w1_bytes));
+        CREATE_CUDA(cudaMalloc(&ctx->b1_all, sizeof(float) * c.n_layers * ctx->w1_rows));
+        CREATE_CUDA(cudaMemset(ctx->b1_all, 0, sizeof(float) * c.n_layers * ctx->w1_rows));
         if (c.hidden > 0) {
-            CREATE_CUDA(cudaMalloc(&lw.w2t, sizeof(float) * c.hidden * kMaxHeads));
-            CREATE_CUDA(cudaMalloc(&lw.b2, sizeof(float) * kMaxHeads));
+            CREATE_CUDA(cudaMalloc(&ctx->w2t_all, sizeof(float) * c.n_layers * c.hidden * kMaxHeads));
+            CREATE_CUDA(cudaMalloc(&ctx->b2_all, sizeof(float) * c.n_layers * kMaxHeads));
         }
         ctx->err[0] = 0;
-        if (make_tmap(ctx, &lw.tmap_w, lw.w1, static_cast<uint64_t>(ctx->w1_rows), static_cast<uint64_t>(c.d_model),
-                      static_cast<uint32_t>(ctx->chunk_n)) != KVZAP_OK) {
+        if (make_tmap(ctx, &ctx->tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
+                      static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(ctx->chunk_n)) != KVZAP_OK) {
             snprintf(g_create_error, sizeof g_create_error, "%s", ctx->err);
             free_all(ctx);
             delete ctx;
@@ -437,22 +439,25 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, co
     if (c.hidden == 0 && (W2 || b2)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-Linear takes no W2/b2");
     if (c.hidden > 0 && !W2) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-MLP needs W2");
     DeviceGuard guard(c.device);
-    LayerWeights &lw = ctx->layers[layer];
     const int rows = c.hidden > 0 ? c.hidden : c.n_kv_heads;
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(lw.w1, W1, static_cast<size_t>(rows) * c.d_model * 2, cudaMemcpyDeviceToDevice,
+    char *w1_dst = static_cast<char *>(ctx->w1_all) + static_cast<size_t>(layer) * ctx->w1_rows * c.d_model * 2;
+    float *b1_dst = ctx->b1_all + static_cast<size_t>(layer) * ctx->w1_rows;
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(w1_dst, W1, static_cast<size_t>(rows) * c.d_model * 2, cudaMemcpyDeviceToDevice,
                                     stream));
     if (b1)
-        KVZAP_CUDA(ctx, cudaMemcpyAsync(lw.b1, b1, sizeof(float) * rows, cudaMemcpyDeviceToDevice, stream));
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(b1_dst, b1, sizeof(float) * rows, cudaMemcpyDeviceToDevice, stream));
     else
-        KVZAP_CUDA(ctx, cudaMemsetAsync(lw.b1, 0, sizeof(float) * rows, stream));
+        KVZAP_CUDA(ctx, cudaMemsetAsync(b1_dst, 0, sizeof(float) * rows, stream));
     if (c.hidden > 0) {
         const int n = c.hidden * kMaxHeads;
         pack_w2_kernel<<<(n + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t *>(W2), b2, c.n_kv_heads,
-                                                            c.hidden, lw.w2t, lw.b2);
+                                                            c.hidden,
+                                                            ctx->w2t_all + static_cast<size_t>(layer) * n,
+                                                            ctx->b2_all + static_cast<size_t>(layer) * kMaxHeads);
         KVZAP_CUDA(ctx, cudaGetLastError());
         ctx->launches += 1;
     }
-    lw.set = true;
+    ctx->layer_set[layer] = 1;
     return KVZAP_OK;
 }
 
@@ -463,12 +468,12 @@ kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int6
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
     if (st != KVZAP_OK) return st;
-    if (!ctx->layers[layer].set) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
     if (n_tokens == 0) return KVZAP_OK;
     if (!hidden || !scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden and scores must not be NULL");
     if (!aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be 16-byte aligned");
     DeviceGuard guard(ctx->cfg.device);
-    return launch_score(ctx, layer, hidden, n_tokens, scores, nullptr, nullptr, 1, 0.0f, 0,
+    return launch_score(ctx, layer, 1, hidden, n_tokens, scores, nullptr, nullptr, 1, 0.0f, 0,
                         static_cast<cudaStream_t>(stream_));
 }
 
@@ -511,7 +516,7 @@ kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidd
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
     if (st != KVZAP_OK) return st;
-    if (!ctx->layers[layer].set) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
     if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
     if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
     DeviceGuard guard(ctx->cfg.device);
@@ -522,7 +527,7 @@ kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidd
     st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
     if (st != KVZAP_OK) return st;
     if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
-    st = launch_score(ctx, layer, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
     return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
 }

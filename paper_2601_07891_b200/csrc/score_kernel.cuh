@@ -30,8 +30,12 @@ constexpr int kScoreThreads = 320;
 constexpr int kMaxHeads = 8;
 
 struct ScoreParams {
-    int64_t n_tokens;
-    int32_t n_tiles;
+    int64_t n_tokens;        // rows (tokens) per layer
+    int32_t n_tiles;         // tiles_per_layer * n_layers_call
+    int32_t tiles_per_layer;
+    int32_t n_layers_call;   // layers scored by this launch (hidden is [n_layers_call][n_tokens][d_model])
+    int32_t layer0;          // first layer: selects the rows of the stacked weights
+    int32_t w_rows;          // rows of W1 per layer in the stacked weight matrix
     int32_t d_model;
     int32_t group_w;      // accumulator columns computed together (one pass over K)
     int32_t n_groups;     // passes per tile
@@ -43,12 +47,12 @@ struct ScoreParams {
     int32_t tmem_cols;    // allocation, power of two >= 32
     int32_t n_hidden;     // MLP hidden width (0 for Linear)
     int32_t n_heads;
-    const float *b1;      // MLP: [n_hidden]; Linear: [16] (padded with zeros)
-    const float *w2t;     // MLP: [n_hidden][8] fp32, heads beyond n_heads are zero
-    const float *b2;      // MLP: [8]
-    float *scores;        // [n_tokens, n_heads] or nullptr
-    uint32_t *maskbits;   // [n_heads][n_words] or nullptr
-    int64_t n_words;      // 32-token words per head (= 4 * n_tiles)
+    const float *b1;      // stacked over all layers: MLP [L][n_hidden]; Linear [L][16] (zero padded)
+    const float *w2t;     // MLP: [L][n_hidden][8] fp32, heads beyond n_heads are zero
+    const float *b2;      // MLP: [L][8]
+    float *scores;        // [n_layers_call][n_tokens, n_heads] or nullptr
+    uint32_t *maskbits;   // [n_layers_call][n_heads][n_words] or nullptr
+    int64_t n_words;      // 32-token words per head and layer (= 4 * tiles_per_layer)
     const int32_t *cu_seqlens;   // [n_seqs + 1] or nullptr (one sequence)
     int32_t n_seqs;
     int32_t window;
@@ -112,8 +116,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     const uint32_t bar_done = bar_tempty + 16;           // [1] abort path only
     const uint32_t bar_pfull = bar_done + 8;             // [1] MLP: second column half -> first
     const uint32_t bar_pempty = bar_pfull + 8;           // [1] MLP: first column half -> second
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 64);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 68);
+    const uint32_t bar_epi = bar_pempty + 8;             // [1] MLP: all epilogue warps (weight reload)
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 72);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 76);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -131,6 +136,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         mbar_init(bar_done, 1);
         mbar_init(bar_pfull, 4);
         mbar_init(bar_pempty, 4);
+        mbar_init(bar_epi, kEpiWarps);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
@@ -139,12 +145,6 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
         tmem_relinquish();
-    }
-    if (kMlp && warp >= 2) {
-        const int tid = threadIdx.x - 64;
-        const float4 *w2g = reinterpret_cast<const float4 *>(p.w2t);
-        for (int i = tid; i < p.n_hidden * 2; i += kScoreThreads - 64) w2s[i] = __ldg(w2g + i);
-        for (int i = tid; i < p.n_hidden; i += kScoreThreads - 64) b1s[i] = __ldg(p.b1 + i);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -172,10 +172,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     if (lane == 0) {
                         const uint32_t sa = smem_base + s * L.stage_bytes;
                         mbar_arrive_expect_tx(bar_full + 8 * s, stage_tx);
-                        tma_load_2d(sa, &tmap_x, bar_full + 8 * s, kb * kBlockK, tile * kTileM, pol_x);
+                        const int l_rel = tile / p.tiles_per_layer;
+                        const int m_tile = tile - l_rel * p.tiles_per_layer;
+                        const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w;
+                        tma_load_3d(sa, &tmap_x, bar_full + 8 * s, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
                         for (int c = 0; c < p.n_chunks; ++c)
                             tma_load_2d(sa + kATileBytes + c * p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * s,
-                                        kb * kBlockK, g * p.group_w + c * p.chunk_n, pol_w);
+                                        kb * kBlockK, w_row0 + c * p.chunk_n, pol_w);
                     }
                     __syncwarp();
                 }
@@ -249,10 +252,37 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         const int hsel = ew >> 2;           // MLP: which half of the group's columns
         const int row = q * 32 + lane;      // token row inside the tile
         const bool active = kMlp || hsel == 0;
-        uint32_t acc_it = 0, tile_it = 0;
+        uint32_t acc_it = 0, tile_it = 0, epi_it = 0;
+        int cur_layer = -1;
         bool ok = true;
         if (active) {
             for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_it) {
+                const int l_rel = tile / p.tiles_per_layer;
+                const int m_tile = tile - l_rel * p.tiles_per_layer;
+                const int layer = p.layer0 + l_rel;
+                if constexpr (kMlp) {
+                    if (layer != cur_layer) {
+                        // (re)load this layer's b1 and W2 into shared memory; all epilogue warps have
+                        // finished the previous tile's reads once they have all arrived here
+                        const int etid = threadIdx.x - 64;
+                        if (cur_layer >= 0) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(bar_epi);
+                            if (!mbar_wait(bar_epi, epi_it & 1u, abort_flag)) { ok = false; break; }
+                            ++epi_it;
+                        }
+                        const float4 *w2g = reinterpret_cast<const float4 *>(p.w2t) +
+                                            static_cast<int64_t>(layer) * p.n_hidden * 2;
+                        const float *b1g = p.b1 + static_cast<int64_t>(layer) * p.n_hidden;
+                        for (int i = etid; i < p.n_hidden * 2; i += kEpiWarps * 32) w2s[i] = __ldg(w2g + i);
+                        for (int i = etid; i < p.n_hidden; i += kEpiWarps * 32) b1s[i] = __ldg(b1g + i);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_epi);
+                        if (!mbar_wait(bar_epi, epi_it & 1u, abort_flag)) { ok = false; break; }
+                        ++epi_it;
+                        cur_layer = layer;
+                    }
+                }
                 float s[kMaxHeads];
 #pragma unroll
                 for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
@@ -290,7 +320,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         tmem_ld_x16(t_row, r);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int h = 0; h < kMaxHeads; ++h) s[h] = __uint_as_float(r[h]) + __ldg(p.b1 + h);
+                        for (int h = 0; h < kMaxHeads; ++h)
+                            s[h] = __uint_as_float(r[h]) + __ldg(p.b1 + layer * p.w_rows + h);
                     }
                     // this warp is done reading the accumulator buffer
                     tc_fence_before_sync();
@@ -313,21 +344,21 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         const float4 pa = src[0], pb = src[1];
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_pempty);
-                        s[0] += pa.x + __ldg(p.b2 + 0);
-                        s[1] += pa.y + __ldg(p.b2 + 1);
-                        s[2] += pa.z + __ldg(p.b2 + 2);
-                        s[3] += pa.w + __ldg(p.b2 + 3);
-                        s[4] += pb.x + __ldg(p.b2 + 4);
-                        s[5] += pb.y + __ldg(p.b2 + 5);
-                        s[6] += pb.z + __ldg(p.b2 + 6);
-                        s[7] += pb.w + __ldg(p.b2 + 7);
+                        s[0] += pa.x + __ldg(p.b2 + layer * kMaxHeads + 0);
+                        s[1] += pa.y + __ldg(p.b2 + layer * kMaxHeads + 1);
+                        s[2] += pa.z + __ldg(p.b2 + layer * kMaxHeads + 2);
+                        s[3] += pa.w + __ldg(p.b2 + layer * kMaxHeads + 3);
+                        s[4] += pb.x + __ldg(p.b2 + layer * kMaxHeads + 4);
+                        s[5] += pb.y + __ldg(p.b2 + layer * kMaxHeads + 5);
+                        s[6] += pb.z + __ldg(p.b2 + layer * kMaxHeads + 6);
+                        s[7] += pb.w + __ldg(p.b2 + layer * kMaxHeads + 7);
                     }
                 }
                 if (hsel == 0) {
-                    const int64_t t = static_cast<int64_t>(tile) * kTileM + row;
+                    const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;      // row inside the layer
                     const bool valid = t < p.n_tokens;
                     if (valid && p.scores != nullptr) {
-                        float *dst = p.scores + t * p.n_heads;
+                        float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
                         if (p.n_heads == kMaxHeads) {
                             reinterpret_cast<float4 *>(dst)[0] = make_float4(s[0], s[1], s[2], s[3]);
                             reinterpret_cast<float4 *>(dst)[1] = make_float4(s[4], s[5], s[6], s[7]);
@@ -353,8 +384,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                             if (lane == h) my_word = word;
                         }
                         if (lane < p.n_heads)
-                            p.maskbits[static_cast<int64_t>(lane) * p.n_words + static_cast<int64_t>(tile) * 4 + q] =
-                                my_word;
+                            p.maskbits[(static_cast<int64_t>(l_rel) * p.n_heads + lane) * p.n_words +
+                                       static_cast<int64_t>(m_tile) * 4 + q] = my_word;
                     }
                 }
             }
