@@ -158,8 +158,115 @@ kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void 
                                       void *K_out, void *V_out, int32_t *lengths,
                                       float *scores_out, void *stream);
 
+/*
+ * Paged output of the same pruning (Discussion, "Implementation Challenges":
+ * per-head lengths differ, so the pruned cache needs paged kernels with
+ * variable-length blocks; the paper fixes no page format, this one is ours).
+ * A page holds page_tokens rows; page p of the K pool and page p of the V pool
+ * hold matching rows.  List (b,h) receives ceil(lengths[b,h] / page_tokens)
+ * pages, numbered contiguously from first_page in (b,h) order (list index
+ * b*H + h), and its rows fill them in token order.
+ *   K_pool, V_pool [n_pages_pool, page_tokens, D] bf16 (out; caller-owned)
+ *   page_table     [n_seqs*H, max_pages_per_list] int32 (out): page numbers of each list; entries
+ *                  beyond a list's page count are left untouched
+ *   lengths        [n_seqs, H] int32 (out)
+ *   n_pages_used   [1] int32 (out, device): pages assigned by this call
+ * If the pool (first_page + pages needed > n_pages_pool) or the table (a list
+ * needs more than max_pages_per_list) is too small, nothing is copied,
+ * *n_pages_used = 0, lengths are still written, and the status word is set to
+ * KVZAP_ERR_OOM_PAGES (kvzap_poll_status).
+ */
+kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                       float tau, int32_t w,
+                                       void *K_pool, void *V_pool, int64_t n_pages_pool, int32_t page_tokens,
+                                       int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
+                                       int32_t *lengths, int32_t *n_pages_used, void *stream);
+
+/* kvzap_prefill_fused with the paged output above. */
+kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                       const void *K, const void *V,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                       float tau, int32_t w,
+                                       void *K_pool, void *V_pool, int64_t n_pages_pool, int32_t page_tokens,
+                                       int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
+                                       int32_t *lengths, int32_t *n_pages_used,
+                                       float *scores_out, void *stream);
+
+/*
+ * Decode-time cache (caption of Algorithm 1: decoding is like prefilling but
+ * needs a buffer of scores to enforce the sliding window; contributions:
+ * delayed eviction with a sliding window).  One list per (sequence, layer, KV
+ * head).  The most recent `window` tokens of a list sit in a ring owned by the
+ * cache together with their scores; a token that leaves the window joins the
+ * list's permanent, position-ordered prefix iff its score >= tau, otherwise it
+ * is dropped.  The prefix lives in pages of the caller's pools
+ * ([n_pages_pool, page_tokens, D] bf16 each), taken one at a time from a bump
+ * allocator.  The logical content of a list is prefix ++ window, oldest first;
+ * for a fixed tau it equals the prefill pruning of the whole sequence.
+ * kvzap_cache_create allocates (cudaMalloc) the rings
+ * (2 * n_seqs*L*H*window*D*2 bytes), score buffers, lengths and page tables.
+ */
+typedef struct kvzap_cache kvzap_cache;
+kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seqs, int32_t window,
+                                int32_t page_tokens, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                int32_t max_pages_per_list);
+kvzap_status kvzap_cache_destroy(kvzap_cache *cache);
+
+/*
+ * One decode step for layers [layer_begin, layer_end) and all n_seqs sequences:
+ * scores the new token of every sequence with each layer's surrogate, appends
+ * its key/value row and score to the window, and decides the token that leaves
+ * the window (kept iff its buffered score >= tau).
+ *   hidden       [layer_end-layer_begin, n_seqs, d_model] bf16
+ *   K_new, V_new [layer_end-layer_begin, n_seqs, H, D] bf16
+ *   scores_out   [layer_end-layer_begin, n_seqs, H] fp32 or NULL
+ * A full pool or page table drops the row that needed the page and sets the
+ * status word to KVZAP_ERR_OOM_PAGES.
+ */
+kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                               const void *hidden, const void *K_new, const void *V_new, float tau,
+                               float *scores_out, void *stream);
+
+/* lengths [n_seqs, L, H] int32 (device): rows currently held by each list (prefix + window). */
+kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream);
+
+/* Copies one list, oldest row first, into K_out / V_out [capacity_rows, D] bf16 (device) and
+ * writes its row count to *n_rows (device); rows beyond capacity_rows are not copied. */
+kvzap_status kvzap_cache_export(kvzap_cache *cache, int32_t seq, int32_t layer, int32_t head,
+                                void *K_out, void *V_out, int64_t capacity_rows, int32_t *n_rows,
+                                void *stream);
+
+/*
+ * Prefill of one sequence's prompt for one layer straight into the decode
+ * cache, so that decoding can continue from it: scores the prompt, sends the
+ * tokens before the last `window` ones through the threshold (kept ones form
+ * the list's paged prefix, pages taken from the cache's allocator), and puts
+ * the last min(n_tokens, window) tokens with their scores into the window
+ * ring, where later decode steps will decide them.  After it, the lists
+ * (seq, layer, *) hold exactly what kvzap_prefill_fused would keep, and
+ * prefill(T) followed by k decode steps equals prefill(T + k).
+ *   hidden [n_tokens, d_model] bf16, K, V [H, n_tokens, D] bf16 (one sequence)
+ *   scores_out [n_tokens, H] fp32 (device) -- required, it also serves as scratch
+ * The lists must be empty (fresh cache) when this is called.
+ */
+kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, int32_t seq,
+                                    const void *hidden, const void *K, const void *V, int64_t n_tokens,
+                                    float tau, float *scores_out, void *stream);
+
+/*
+ * Installs prefix bookkeeping produced elsewhere (used to set up synthetic
+ * cache states): prefix_len [n_seqs*L*H] and page_table
+ * [n_seqs*L*H, max_pages_per_list], device int32 in list order (seq, layer,
+ * head); next_free_page is the first pool page the allocator may hand out.
+ * Every list's window becomes empty.  Synchronises `stream`.
+ */
+kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, const int32_t *page_table,
+                                int32_t next_free_page, void *stream);
+
 /* Kernel identifiers for kvzap_get_profile. */
-enum { KVZAP_KERNEL_SCORE = 0, KVZAP_KERNEL_MASK = 1, KVZAP_KERNEL_SCAN = 2, KVZAP_KERNEL_COMPACT = 3 };
+enum { KVZAP_KERNEL_SCORE = 0, KVZAP_KERNEL_MASK = 1, KVZAP_KERNEL_SCAN = 2, KVZAP_KERNEL_COMPACT = 3,
+       KVZAP_KERNEL_DECODE_UPDATE = 4 };
 
 /*
  * Per-kernel timing with CUDA events on the launching stream (a measurement

@@ -52,6 +52,17 @@ SIGNATURES = {
     "kvzap_prefill_fused_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp,
                                         _vp]),
     "kvzap_prune_prefill_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _f32, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prune_prefill_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32, _i32,
+                                         _vp, _i32, _vp, _vp, _vp]),
+    "kvzap_prefill_fused_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
+                                         _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_cache_create": (_i32, [_vp, ctypes.POINTER(_vp), _i32, _i32, _i32, _vp, _vp, _i64, _i32]),
+    "kvzap_cache_destroy": (_i32, [_vp]),
+    "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
+    "kvzap_cache_lengths": (_i32, [_vp, _vp, _vp]),
+    "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
+    "kvzap_prefill_to_cache": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
+    "kvzap_cache_import": (_i32, [_vp, _vp, _vp, _i32, _vp]),
     "kvzap_set_profiling": (_i32, [_vp, _i32]),
     "kvzap_get_profile": (_i32, [_vp, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)]),
     "kvzap_poll_status": (_i32, [_vp, _vp]),
@@ -177,7 +188,63 @@ def kvzap_prune_prefill_noalloc(K, V, scores, cu_seqlens, n_seqs, tau, w, K_out,
         _ptr(lengths), _stream(stream)))
 
 
-KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3}
+def kvzap_prune_prefill_paged(handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                              first_page, page_table, lengths, n_pages_used, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prune_prefill_paged(
+        handle, _ptr(K) if nz else None, _ptr(V) if nz else None, _ptr(scores) if nz else None, _ptr(cu_seqlens),
+        n_seqs, n_tokens, tau, w, _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens, first_page,
+        _ptr(page_table), page_table.shape[1], _ptr(lengths), _ptr(n_pages_used), _stream(stream)))
+
+
+def kvzap_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                              first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_fused_paged(
+        handle, layer, _ptr(hidden) if nz else None, _ptr(K) if nz else None, _ptr(V) if nz else None,
+        _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens,
+        first_page, _ptr(page_table), page_table.shape[1], _ptr(lengths), _ptr(n_pages_used),
+        _ptr(scores_out) if nz else None, _stream(stream)))
+
+
+def kvzap_cache_create(handle, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list):
+    cache = ctypes.c_void_p()
+    _check(handle, load().kvzap_cache_create(handle, ctypes.byref(cache), n_seqs, window, page_tokens, _ptr(K_pool),
+                                             _ptr(V_pool), K_pool.shape[0], max_pages_per_list))
+    return cache
+
+
+def kvzap_cache_destroy(cache):
+    _check(None, load().kvzap_cache_destroy(cache))
+
+
+def kvzap_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None, stream=None):
+    _check(handle, load().kvzap_decode_step(handle, cache, layer_begin, layer_end, _ptr(hidden), _ptr(K_new),
+                                            _ptr(V_new), tau, _ptr(scores_out), _stream(stream)))
+
+
+def kvzap_cache_lengths(handle, cache, lengths, stream=None):
+    _check(handle, load().kvzap_cache_lengths(cache, _ptr(lengths), _stream(stream)))
+
+
+def kvzap_cache_export(handle, cache, seq, layer, head, K_out, V_out, n_rows, stream=None):
+    _check(handle, load().kvzap_cache_export(cache, seq, layer, head, _ptr(K_out), _ptr(V_out), K_out.shape[0],
+                                             _ptr(n_rows), _stream(stream)))
+
+
+def kvzap_prefill_to_cache(handle, cache, layer, seq, hidden, K, V, tau, scores_out, stream=None):
+    _check(handle, load().kvzap_prefill_to_cache(handle, cache, layer, seq, _ptr(hidden), _ptr(K), _ptr(V), K.shape[1],
+                                                 tau, _ptr(scores_out), _stream(stream)))
+
+
+def kvzap_cache_import(handle, cache, prefix_len, page_table, next_free_page, stream=None):
+    _check(handle, load().kvzap_cache_import(cache, _ptr(prefix_len), _ptr(page_table), next_free_page,
+                                             _stream(stream)))
+
+
+KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3, "decode_update": 4}
 
 
 def kvzap_set_profiling(handle, enable):

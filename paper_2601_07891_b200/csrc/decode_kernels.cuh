@@ -1,0 +1,180 @@
+// Decode-time pruning on a paged, ragged cache (caption of Algorithm 1: decoding
+// applies the same rule with a buffer of the scores of the tokens still inside the
+// sliding window; contribution list: delayed eviction with a sliding window).
+//
+// One list per (sequence b, layer l, KV head h), index li = (b * L + l) * H + h:
+//   window ring   k_ring / v_ring [li][w][D], score_ring [li][w]: the most recent w tokens,
+//                 position p lives in slot p % w
+//   prefix        the tokens that left the window with score >= tau, in position order,
+//                 stored in pages of page_tokens rows taken from the caller's pool;
+//                 page_table [li][max_pages], prefix_len [li]
+//   n_tokens [li] tokens appended so far
+// A step appends one token per sequence: the token that leaves the window (position
+// n - w, found in the very slot the new token will take) is copied to the prefix iff
+// its buffered score >= tau, then the new row and its score overwrite the slot.
+// Logical cache = prefix ++ window in age order.  Pages come from a bump allocator
+// (atomicAdd on one cursor); an exhausted pool or page table sets the status word and
+// drops the row instead of writing out of bounds.
+#pragma once
+
+#include "ptx.cuh"
+
+namespace kvzap {
+
+struct CacheView {
+    int32_t n_seqs, n_layers, n_heads, row_units, window, page_tokens, max_pages;
+    int64_t n_pages_pool;
+    uint4 *k_ring, *v_ring;
+    float *score_ring;
+    int32_t *n_tokens, *prefix_len, *page_table, *page_cursor;
+    uint4 *k_pool, *v_pool;
+};
+
+constexpr int kDecodeThreads = 256;
+
+// 16 lanes per list; lists of layers [layer0, layer0 + n_layers_call).
+// scores [n_layers_call][B][H] fp32, K_new/V_new [n_layers_call][B][H][D] bf16.
+__global__ void __launch_bounds__(kDecodeThreads)
+decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const float *__restrict__ scores,
+                     const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, float tau,
+                     int32_t *__restrict__ status)
+{
+    const int gl = threadIdx.x & 15;
+    const int64_t group = (static_cast<int64_t>(blockIdx.x) * kDecodeThreads + threadIdx.x) >> 4;
+    const int64_t n_groups = static_cast<int64_t>(n_layers_call) * c.n_seqs * c.n_heads;
+    const bool live = group < n_groups;
+    // every lane of the warp runs the whole body (the shuffles below need all 32 lanes)
+    const int64_t g = live ? group : 0;
+    const int l_rel = static_cast<int>(g / (static_cast<int64_t>(c.n_seqs) * c.n_heads));
+    const int rem = static_cast<int>(g - static_cast<int64_t>(l_rel) * c.n_seqs * c.n_heads);
+    const int b = rem / c.n_heads, h = rem % c.n_heads;
+    const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
+    const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+    const int32_t n = c.n_tokens[li];
+    const float s_new = scores[src_row];
+
+    // which row (if any) moves to the prefix now
+    bool append = false;
+    const uint4 *app_k = nullptr, *app_v = nullptr;
+    int slot = 0;
+    if (c.window > 0) {
+        slot = n % c.window;
+        if (n >= c.window) {
+            const float s_old = c.score_ring[li * c.window + slot];
+            append = s_old >= tau;
+            app_k = c.k_ring + (li * c.window + slot) * c.row_units;
+            app_v = c.v_ring + (li * c.window + slot) * c.row_units;
+        }
+    } else {
+        append = s_new >= tau;
+        app_k = K_new + src_row * c.row_units;
+        app_v = V_new + src_row * c.row_units;
+    }
+    append = append && live;
+
+    // page for the appended row: lane 0 of the group allocates when the row opens a new page
+    const int32_t idx = c.prefix_len[li];
+    const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
+    int32_t page = -1;
+    if (append && gl == 0) {
+        if (page_i >= c.max_pages) {
+            atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+        } else if (in_page == 0) {
+            const int32_t got = atomicAdd(c.page_cursor, 1);
+            if (got >= c.n_pages_pool) {
+                atomicCAS(status, 0, 4);
+            } else {
+                page = got;
+                c.page_table[li * c.max_pages + page_i] = got;
+            }
+        } else {
+            page = c.page_table[li * c.max_pages + page_i];
+        }
+    }
+    page = __shfl_sync(0xffffffffu, page, 0, 16);
+    if (append && page >= 0) {
+        const int64_t dst = (static_cast<int64_t>(page) * c.page_tokens + in_page) * c.row_units;
+        for (int u = gl; u < c.row_units; u += 16) {
+            c.k_pool[dst + u] = app_k[u];
+            c.v_pool[dst + u] = app_v[u];
+        }
+        if (gl == 0) c.prefix_len[li] = idx + 1;
+    }
+    if (!live) return;
+    if (c.window > 0) {
+        // each lane overwrites exactly the 16-byte units it read above, so no lane races another
+        const int64_t ring = (li * c.window + slot) * c.row_units;
+        for (int u = gl; u < c.row_units; u += 16) {
+            c.k_ring[ring + u] = K_new[src_row * c.row_units + u];
+            c.v_ring[ring + u] = V_new[src_row * c.row_units + u];
+        }
+        if (gl == 0) c.score_ring[li * c.window + slot] = s_new;
+    }
+    if (gl == 0) c.n_tokens[li] = n + 1;
+}
+
+// After a prompt's prefix has been compacted: copies the last min(T, w) tokens of the prompt (rows of
+// K, V [H][T][D], scores [T][H]) into the window rings of lists li0 .. li0+H-1 and sets n_tokens = T.
+__global__ void __launch_bounds__(256)
+ring_fill_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
+                 const uint4 *__restrict__ V, int64_t T)
+{
+    const int h = blockIdx.y;
+    const int64_t li = li0 + h;
+    const int64_t n_win = T < c.window ? T : c.window;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_win * c.row_units;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t j = i / c.row_units;
+        const int u = static_cast<int>(i % c.row_units);
+        const int64_t pos = T - n_win + j;
+        const int64_t dst = (li * c.window + pos % c.window) * c.row_units + u;
+        const int64_t src = (static_cast<int64_t>(h) * T + pos) * c.row_units + u;
+        c.k_ring[dst] = K[src];
+        c.v_ring[dst] = V[src];
+        if (u == 0) c.score_ring[li * c.window + pos % c.window] = scores[pos * c.n_heads + h];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) c.n_tokens[li] = static_cast<int32_t>(T);
+}
+
+// lengths[li] = prefix_len + min(n_tokens, w)
+__global__ void cache_lengths_kernel(const CacheView c, int32_t *__restrict__ lengths)
+{
+    const int64_t li = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t n_lists = static_cast<int64_t>(c.n_seqs) * c.n_layers * c.n_heads;
+    if (li < n_lists) lengths[li] = c.prefix_len[li] + min(c.n_tokens[li], c.window);
+}
+
+// Linearises one list (prefix pages, then the window oldest first) into K_out/V_out [capacity][D].
+__global__ void __launch_bounds__(256)
+cache_export_kernel(const CacheView c, int64_t li, uint4 *__restrict__ K_out, uint4 *__restrict__ V_out,
+                    int64_t capacity_rows, int32_t *__restrict__ n_rows)
+{
+    const int32_t n_prefix = c.prefix_len[li];
+    const int32_t n = c.n_tokens[li];
+    const int32_t n_win = min(n, c.window);
+    const int64_t total = static_cast<int64_t>(n_prefix) + n_win;
+    if (threadIdx.x == 0 && blockIdx.x == 0) *n_rows = static_cast<int32_t>(total);
+    const int64_t rows = total < capacity_rows ? total : capacity_rows;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < rows * c.row_units;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int64_t r = i / c.row_units;
+        const int u = static_cast<int>(i % c.row_units);
+        int64_t src;
+        const uint4 *ksrc, *vsrc;
+        if (r < n_prefix) {
+            const int32_t page = c.page_table[li * c.max_pages + r / c.page_tokens];
+            src = (static_cast<int64_t>(page) * c.page_tokens + r % c.page_tokens) * c.row_units + u;
+            ksrc = c.k_pool;
+            vsrc = c.v_pool;
+        } else {
+            const int64_t pos = static_cast<int64_t>(n) - n_win + (r - n_prefix);
+            src = (li * c.window + pos % c.window) * c.row_units + u;
+            ksrc = c.k_ring;
+            vsrc = c.v_ring;
+        }
+        K_out[i] = ksrc[src];
+        V_out[i] = vsrc[src];
+    }
+}
+
+}  // namespace kvzap

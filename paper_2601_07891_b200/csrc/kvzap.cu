@@ -11,6 +11,7 @@
 #include <new>
 #include <vector>
 
+#include "decode_kernels.cuh"
 #include "prune_kernels.cuh"
 #include "score_kernel.cuh"
 
@@ -46,6 +47,7 @@ struct kvzap_ctx {
     uint32_t *maskbits = nullptr;    // [H][max_words]
     int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
     int32_t *seqbase = nullptr;      // [H][max_seqs + 1]
+    int32_t *list_page0 = nullptr;   // [max_seqs * H] first page of each list (paged output)
     int32_t *status_dev = nullptr;
     int32_t *status_host = nullptr;  // pinned
     int64_t launches = 0;
@@ -161,6 +163,7 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->maskbits);
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
+    cudaFree(ctx->list_page0);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
@@ -190,7 +193,7 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 // scores [n_layers][n_tokens][H]; maskbits != nullptr fuses the threshold/window test.
 static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
-                                 float tau, int32_t w, cudaStream_t stream)
+                                 float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t tiles_per_layer = (n_tokens + kTileM - 1) / kTileM;
@@ -227,6 +230,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.cu_seqlens = cu_seqlens;
     p.n_seqs = n_seqs;
     p.window = w;
+    p.window_keep = window_keep;
     p.tau = tau;
     p.status = ctx->status_dev;
     const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
@@ -254,7 +258,7 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const void *K, const void 
         ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
         scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
                                             n_tokens, ctx->blockprefix, ctx->seqbase, lengths, 0, 0, 0, 0, nullptr,
-                                            nullptr, nullptr, ctx->status_dev);
+                                            nullptr, nullptr, nullptr, ctx->status_dev);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
@@ -404,6 +408,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * ctx->max_words * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
     CREATE_CUDA(cudaMallocHost(&ctx->status_host, sizeof(int32_t)));
@@ -499,7 +504,7 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     {
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
         mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
-                                                                         cu_seqlens, n_seqs, tau, w, ctx->maskbits,
+                                                                         cu_seqlens, n_seqs, tau, w, 1, ctx->maskbits,
                                                                          n_blocks * 4);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
@@ -731,10 +736,10 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
     // that this call reads is first written by it; only the status word must start at zero.
     KVZAP_CUDA(nullptr, cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
     mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, n_kv_heads, cu_seqlens, n_seqs,
-                                                                     tau, w, maskbits, n_words);
+                                                                     tau, w, 1, maskbits, n_words);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
-                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, status);
+                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(n_kv_heads));
     compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
@@ -744,3 +749,312 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
     KVZAP_CUDA(nullptr, cudaGetLastError());
     return KVZAP_OK;
 }
+
+// ---------------------------------------------------------------------------
+// Paged output and the decode-time cache.
+struct kvzap_cache {
+    kvzap_ctx *ctx = nullptr;
+    kvzap::CacheView v;
+    float *scores = nullptr;        // [L][B][H] scratch when the caller does not want the scores
+    int64_t n_lists = 0;
+};
+
+namespace kvzap {
+
+static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const void *K, const void *V, const int32_t *cu_seqlens,
+                                            int32_t n_seqs, int64_t n_tokens, void *K_pool, void *V_pool,
+                                            int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
+                                            int32_t *page_table, int32_t max_pages, int32_t *lengths,
+                                            int32_t *n_pages_used, cudaStream_t stream,
+                                            int32_t *page_cursor = nullptr)
+{
+    const kvzap_config &c = ctx->cfg;
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    const int64_t n_words = n_blocks * 4;
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
+        scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
+                                            n_tokens, ctx->blockprefix, ctx->seqbase, lengths, page_tokens, first_page,
+                                            n_pages_pool, max_pages, ctx->list_page0, page_table, n_pages_used,
+                                            page_cursor, ctx->status_dev);
+    }
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
+        compact_kernel<true><<<grid, kCompactThreads, 0, stream>>>(
+            static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_pool),
+            static_cast<uint4 *>(V_pool), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
+            n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, page_tokens, ctx->list_page0);
+    }
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 2;
+    return KVZAP_OK;
+}
+
+static kvzap_status check_paged_args(kvzap_ctx *ctx, const void *K, const void *V, const void *K_pool,
+                                     const void *V_pool, int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
+                                     const int32_t *page_table, int32_t max_pages, const int32_t *lengths,
+                                     const int32_t *n_pages_used, int32_t w)
+{
+    if (!K || !V || !K_pool || !V_pool || !page_table || !lengths || !n_pages_used)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "paged: K, V, pools, page_table, lengths, n_pages_used must not be NULL");
+    if (!aligned16(K) || !aligned16(V) || !aligned16(K_pool) || !aligned16(V_pool))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "paged: K/V and pool pointers must be 16-byte aligned");
+    if (page_tokens < 1 || max_pages < 1 || n_pages_pool < 0 || first_page < 0)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "paged: page_tokens, max_pages_per_list >= 1; n_pages_pool, first_page >= 0");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    return KVZAP_OK;
+}
+
+}  // namespace kvzap
+
+extern "C" {
+
+kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                       int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                       int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                       int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                       void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!lengths || !n_pages_used) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths / n_pages_used is NULL");
+    DeviceGuard guard(ctx->cfg.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * ctx->cfg.n_kv_heads, stream));
+        KVZAP_CUDA(ctx, cudaMemsetAsync(n_pages_used, 0, sizeof(int32_t), stream));
+        return KVZAP_OK;
+    }
+    st = check_paged_args(ctx, K, V, K_pool, V_pool, n_pages_pool, page_tokens, first_page, page_table,
+                          max_pages_per_list, lengths, n_pages_used, w);
+    if (st != KVZAP_OK) return st;
+    if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
+        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
+                                                                         cu_seqlens, n_seqs, tau, w, 1, ctx->maskbits,
+                                                                         n_blocks * 4);
+    }
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return launch_compaction_paged(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
+                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
+}
+
+kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                       int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                       int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                       int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                       float *scores_out, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (!lengths || !n_pages_used) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths / n_pages_used is NULL");
+    DeviceGuard guard(ctx->cfg.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * ctx->cfg.n_kv_heads, stream));
+        KVZAP_CUDA(ctx, cudaMemsetAsync(n_pages_used, 0, sizeof(int32_t), stream));
+        return KVZAP_OK;
+    }
+    st = check_paged_args(ctx, K, V, K_pool, V_pool, n_pages_pool, page_tokens, first_page, page_table,
+                          max_pages_per_list, lengths, n_pages_used, w);
+    if (st != KVZAP_OK) return st;
+    if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
+    if (st != KVZAP_OK) return st;
+    return launch_compaction_paged(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
+                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
+}
+
+kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seqs, int32_t window,
+                                int32_t page_tokens, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                int32_t max_pages_per_list)
+{
+    if (!ctx || !out) return KVZAP_ERR_INVALID_ARG;
+    *out = nullptr;
+    const kvzap_config &c = ctx->cfg;
+    if (n_seqs < 1 || n_seqs > c.max_tokens)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "cache: n_seqs %d outside 1..max_tokens", n_seqs);
+    if (window < 0 || page_tokens < 1 || max_pages_per_list < 1 || n_pages_pool < 0)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "cache: window >= 0, page_tokens >= 1, max_pages_per_list >= 1 required");
+    if (!K_pool || !V_pool || !aligned16(K_pool) || !aligned16(V_pool))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "cache: pools must be non-NULL and 16-byte aligned");
+    DeviceGuard guard(c.device);
+    kvzap_cache *cache = new (std::nothrow) kvzap_cache();
+    if (!cache) return fail(ctx, KVZAP_ERR_CUDA, "out of host memory");
+    cache->ctx = ctx;
+    cache->n_lists = static_cast<int64_t>(n_seqs) * c.n_layers * c.n_kv_heads;
+    CacheView &v = cache->v;
+    memset(&v, 0, sizeof v);
+    v.n_seqs = n_seqs; v.n_layers = c.n_layers; v.n_heads = c.n_kv_heads; v.row_units = c.head_dim / 8;
+    v.window = window; v.page_tokens = page_tokens; v.max_pages = max_pages_per_list; v.n_pages_pool = n_pages_pool;
+    v.k_pool = static_cast<uint4 *>(K_pool); v.v_pool = static_cast<uint4 *>(V_pool);
+    const size_t ring_bytes = static_cast<size_t>(cache->n_lists) * (window > 0 ? window : 1) * c.head_dim * 2;
+    const size_t n = static_cast<size_t>(cache->n_lists);
+    cudaError_t e = cudaSuccess;
+    auto alloc = [&](void **p, size_t bytes, bool zero) {
+        if (e != cudaSuccess) return;
+        e = cudaMalloc(p, bytes);
+        if (e == cudaSuccess && zero) e = cudaMemset(*p, 0, bytes);
+    };
+    alloc(reinterpret_cast<void **>(&v.k_ring), ring_bytes, false);
+    alloc(reinterpret_cast<void **>(&v.v_ring), ring_bytes, false);
+    alloc(reinterpret_cast<void **>(&v.score_ring), sizeof(float) * n * (window > 0 ? window : 1), true);
+    alloc(reinterpret_cast<void **>(&v.n_tokens), sizeof(int32_t) * n, true);
+    alloc(reinterpret_cast<void **>(&v.prefix_len), sizeof(int32_t) * n, true);
+    alloc(reinterpret_cast<void **>(&v.page_table), sizeof(int32_t) * n * max_pages_per_list, true);
+    alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
+    alloc(reinterpret_cast<void **>(&cache->scores), sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
+          false);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        fail(ctx, KVZAP_ERR_CUDA, "cache allocation failed: %s", cudaGetErrorString(e));
+        kvzap_cache_destroy(cache);
+        return KVZAP_ERR_CUDA;
+    }
+    *out = cache;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
+{
+    if (!cache) return KVZAP_OK;
+    DeviceGuard guard(cache->ctx->cfg.device);
+    cudaDeviceSynchronize();
+    cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
+    cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
+    cudaFree(cache->v.page_cursor); cudaFree(cache->scores);
+    delete cache;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                               const void *hidden, const void *K_new, const void *V_new, float tau,
+                               float *scores_out, void *stream_)
+{
+    if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "decode: layer range [%d, %d) invalid", layer_begin, layer_end);
+    for (int l = layer_begin; l < layer_end; ++l)
+        if (!ctx->layer_set[l]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", l);
+    if (!hidden || !K_new || !V_new || !aligned16(hidden) || !aligned16(K_new) || !aligned16(V_new))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "decode: hidden, K_new, V_new must be non-NULL, 16-byte aligned");
+    DeviceGuard guard(c.device);
+    const int n_layers = layer_end - layer_begin;
+    float *scores = scores_out ? scores_out : cache->scores;
+    kvzap_status st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
+                                   0.0f, 0, stream);
+    if (st != KVZAP_OK) return st;
+    const int64_t n_groups = static_cast<int64_t>(n_layers) * cache->v.n_seqs * c.n_kv_heads;
+    const int64_t threads = n_groups * 16;
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_DECODE_UPDATE, stream);
+        decode_update_kernel<<<static_cast<unsigned>((threads + kDecodeThreads - 1) / kDecodeThreads), kDecodeThreads, 0,
+                               stream>>>(cache->v, layer_begin, n_layers, scores, static_cast<const uint4 *>(K_new),
+                                         static_cast<const uint4 *>(V_new), tau, ctx->status_dev);
+    }
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream_)
+{
+    if (!cache || !lengths) return KVZAP_ERR_INVALID_ARG;
+    DeviceGuard guard(cache->ctx->cfg.device);
+    cache_lengths_kernel<<<static_cast<unsigned>((cache->n_lists + 255) / 256), 256, 0,
+                           static_cast<cudaStream_t>(stream_)>>>(cache->v, lengths);
+    KVZAP_CUDA(cache->ctx, cudaGetLastError());
+    cache->ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_cache_export(kvzap_cache *cache, int32_t seq, int32_t layer, int32_t head, void *K_out, void *V_out,
+                                int64_t capacity_rows, int32_t *n_rows, void *stream_)
+{
+    if (!cache || !K_out || !V_out || !n_rows || capacity_rows < 0) return KVZAP_ERR_INVALID_ARG;
+    const CacheView &v = cache->v;
+    if (seq < 0 || seq >= v.n_seqs || layer < 0 || layer >= v.n_layers || head < 0 || head >= v.n_heads)
+        return fail(cache->ctx, KVZAP_ERR_INVALID_ARG, "export: (seq, layer, head) out of range");
+    DeviceGuard guard(cache->ctx->cfg.device);
+    const int64_t li = (static_cast<int64_t>(seq) * v.n_layers + layer) * v.n_heads + head;
+    cache_export_kernel<<<64, 256, 0, static_cast<cudaStream_t>(stream_)>>>(v, li, static_cast<uint4 *>(K_out),
+                                                                         static_cast<uint4 *>(V_out), capacity_rows,
+                                                                         n_rows);
+    KVZAP_CUDA(cache->ctx, cudaGetLastError());
+    cache->ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, const int32_t *page_table,
+                                int32_t next_free_page, void *stream_)
+{
+    if (!cache || !prefix_len || !page_table || next_free_page < 0) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    kvzap_ctx *ctx = cache->ctx;
+    DeviceGuard guard(ctx->cfg.device);
+    const size_t n = static_cast<size_t>(cache->n_lists);
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.prefix_len, prefix_len, sizeof(int32_t) * n, cudaMemcpyDeviceToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.page_table, page_table, sizeof(int32_t) * n * cache->v.max_pages,
+                                    cudaMemcpyDeviceToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.n_tokens, 0, sizeof(int32_t) * n, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.page_cursor, &next_free_page, sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, int32_t seq, const void *hidden,
+                                    const void *K, const void *V, int64_t n_tokens, float tau, float *scores_out,
+                                    void *stream_)
+{
+    if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    const CacheView &v = cache->v;
+    if (layer < 0 || layer >= c.n_layers || seq < 0 || seq >= v.n_seqs)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache: layer %d / seq %d out of range", layer, seq);
+    kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (n_tokens == 0) return KVZAP_OK;
+    if (!hidden || !K || !V || !scores_out || !aligned16(hidden) || !aligned16(K) || !aligned16(V))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache: hidden, K, V, scores_out must be non-NULL, aligned");
+    DeviceGuard guard(c.device);
+    const int64_t li0 = (static_cast<int64_t>(seq) * v.n_layers + layer) * v.n_heads;
+    // mask = threshold only, the window's tokens left out: they go to the ring below
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, nullptr, 1, tau, v.window, stream, 0);
+    if (st != KVZAP_OK) return st;
+    st = launch_compaction_paged(ctx, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
+                                 v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
+                                 v.page_cursor);
+    if (st != KVZAP_OK) return st;
+    if (v.window > 0) {
+        const int64_t n_win = n_tokens < v.window ? n_tokens : v.window;
+        const unsigned gx = static_cast<unsigned>((n_win * v.row_units + 255) / 256);
+        ring_fill_kernel<<<dim3(gx, static_cast<unsigned>(v.n_heads)), 256, 0, stream>>>(
+            v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens);
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    } else {
+        // no window: only the token count is kept
+        std::vector<int32_t> nt(v.n_heads, static_cast<int32_t>(n_tokens));
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(v.n_tokens + li0, nt.data(), sizeof(int32_t) * v.n_heads, cudaMemcpyHostToDevice,
+                                        stream));
+        KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
+    }
+    return KVZAP_OK;
+}
+
+}  // extern "C"

@@ -23,7 +23,7 @@ constexpr int kBlockTokens = 128;     // tokens per mask block = 4 words (same a
 // One warp per 32 tokens; 4 warps per CTA = one 128-token block.
 __global__ void __launch_bounds__(128)
 mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
-            const int32_t *__restrict__ cu_seqlens, int n_seqs, float tau, int window,
+            const int32_t *__restrict__ cu_seqlens, int n_seqs, float tau, int window, int window_keep,
             uint32_t *__restrict__ maskbits, int64_t n_words)
 {
     const int lane = threadIdx.x & 31;
@@ -54,7 +54,7 @@ mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
     uint32_t my_word = 0;
 #pragma unroll
     for (int h = 0; h < kMaxHeads; ++h) {
-        const bool keep = valid && (in_window || s[h] >= tau);
+        const bool keep = valid && (in_window ? window_keep != 0 : s[h] >= tau);
         const uint32_t w = __ballot_sync(0xffffffffu, keep);
         if (lane == h) my_word = w;
     }
@@ -94,8 +94,11 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             int32_t *__restrict__ blockprefix, int32_t *__restrict__ seqbase, int32_t *__restrict__ lengths,
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
-            int32_t *__restrict__ status)
+            int32_t *__restrict__ page_cursor, int32_t *__restrict__ status)
 {
+    // page_cursor != nullptr: the first page comes from (and the pages used are added to) a device-side
+    // allocator cursor instead of the first_page argument
+    if (page_tokens > 0 && page_cursor != nullptr) first_page = *page_cursor;
     __shared__ int32_t warp_sums[32];
     __shared__ int32_t carry_s;
     __shared__ int32_t fail_s;
@@ -183,10 +186,16 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + used > n_pages_pool;
     if (fail) {
         for (int idx = tid; idx < n_lists; idx += 1024) list_page0[idx] = -1;
-        if (tid == 0) { atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */); *n_pages_used = 0; }
+        if (tid == 0) {
+            atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+            if (n_pages_used != nullptr) *n_pages_used = 0;
+        }
         return;
     }
-    if (tid == 0) *n_pages_used = used;
+    if (tid == 0) {
+        if (n_pages_used != nullptr) *n_pages_used = used;
+        if (page_cursor != nullptr) *page_cursor = first_page + used;
+    }
     for (int idx = tid; idx < n_lists; idx += 1024) {
         const int32_t p0 = list_page0[idx];
         const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens;

@@ -56,6 +56,7 @@ struct ScoreParams {
     const int32_t *cu_seqlens;   // [n_seqs + 1] or nullptr (one sequence)
     int32_t n_seqs;
     int32_t window;
+    int32_t window_keep;  // 1: tokens inside the window are kept (Algorithm 1); 0: they are left out of the mask
     float tau;
     int32_t *status;      // device status word
 };
@@ -379,7 +380,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         uint32_t my_word = 0;
 #pragma unroll
                         for (int h = 0; h < kMaxHeads; ++h) {
-                            const bool keep = valid && (in_window || s[h] >= p.tau);
+                            const bool keep = valid && (in_window ? p.window_keep != 0 : s[h] >= p.tau);
                             const uint32_t word = __ballot_sync(0xffffffffu, keep);
                             if (lane == h) my_word = word;
                         }
