@@ -96,7 +96,7 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer,
                                const void *W2, const float *b2, void *stream);
 
 /*
- * Surrogate scoring (Method, "KVzap"; Algorithm 1, first line): maps each
+ * Surrogate scoring (Method, "KVzap"; Algorithm 1, the scoring step): maps each
  * hidden state h_t to H scores, independently per position.
  *   Linear: scores[t,h] = b1[h] + sum_k hidden[t,k] W1[h,k]
  *   MLP:    scores[t,h] = b2[h] + sum_j GELU(b1[j] + sum_k hidden[t,k] W1[j,k]) W2[h,j]
@@ -109,7 +109,7 @@ kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int6
 
 /*
  * Threshold + sliding window + per-(sequence, head) ordered compaction
- * (Algorithm 1, lines 2-4; Method, "KVzap": pairs whose score falls below tau
+ * (Algorithm 1, the steps after scoring; Method, "KVzap": pairs whose score falls below tau
  * are discarded, the most recent w tokens are kept).
  *   keep[b,h,t] = (t >= T_b - w) || (scores[t,h] >= tau)        (fp32 compare; NaN is not kept)
  * with t counted inside sequence b of length T_b.  w = 0 protects nothing;

@@ -1,5 +1,5 @@
 // Threshold/window mask, per-head prefix sums and ordered K/V compaction
-// (Algorithm 1, lines 2-4).  Everything here is integer / byte work and must
+// (Algorithm 1: the window, threshold and gather steps).  Everything here is integer / byte work and must
 // be bit-exact.
 //
 // Data flow (all on one stream, no CTA ever waits for another):
