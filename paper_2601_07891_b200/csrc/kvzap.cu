@@ -30,16 +30,19 @@ struct kvzap_ctx {
     kvzap_config cfg;
     int sm_count = 0;
     int w1_rows = 0;                 // rows of the stored first-layer matrix (Linear: padded to 16)
-    // scoring schedule (see ScoreParams)
-    int group_w = 0, n_groups = 0, chunk_n = 0, n_chunks = 0, n_stages = 0, acc_bufs = 0, acc_stride = 0,
-        tmem_cols = 0;
-    uint32_t score_smem = 0;
+    // scoring schedules (see ScoreParams): [0] one CTA per tile, [1] CTA pairs (MLP only)
+    struct Schedule {
+        int group_w = 0, n_groups = 0, chunk_n = 0, n_chunks = 0, n_stages = 0, acc_bufs = 0, acc_stride = 0,
+            tmem_cols = 0;
+        uint32_t smem = 0;
+        CUtensorMap tmap_w;          // box = the W1 rows one CTA stages per MMA chunk
+    } sched[2];
+    int pair_clusters = 0;           // CTA pairs that can be resident at once; 0 = pairs unavailable
     // weights of all layers, stacked so that one tensor map / one base pointer serves any layer range
     void *w1_all = nullptr;          // bf16 [L * w1_rows, d_model]
     float *b1_all = nullptr;         // [L][w1_rows]
     float *w2t_all = nullptr;        // [L][hidden][8] fp32 (MLP)
     float *b2_all = nullptr;         // [L][8] (MLP)
-    CUtensorMap tmap_w;
     std::vector<char> layer_set;
     kvzap::EncodeTiledFn encode = nullptr;
     // scratch
@@ -196,7 +199,11 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
                                  float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1)
 {
     const kvzap_config &c = ctx->cfg;
-    const int64_t tiles_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    // CTA pairs pay off once a layer has at least two 128-token blocks; a pair's work tile is 256 tokens
+    const bool pair = c.hidden > 0 && ctx->pair_clusters > 0 && blocks_per_layer >= 2;
+    const kvzap_ctx::Schedule &sc = ctx->sched[pair ? 1 : 0];
+    const int64_t tiles_per_layer = pair ? (blocks_per_layer + 1) / 2 : blocks_per_layer;
     const int64_t n_tiles = tiles_per_layer * n_layers;
     CUtensorMap tmap_x;
     kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model),
@@ -207,18 +214,19 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.n_tokens = n_tokens;
     p.n_tiles = static_cast<int32_t>(n_tiles);
     p.tiles_per_layer = static_cast<int32_t>(tiles_per_layer);
+    p.blocks_per_layer = static_cast<int32_t>(blocks_per_layer);
     p.n_layers_call = n_layers;
     p.layer0 = layer;
     p.w_rows = ctx->w1_rows;
     p.d_model = c.d_model;
-    p.group_w = ctx->group_w;
-    p.n_groups = ctx->n_groups;
-    p.chunk_n = ctx->chunk_n;
-    p.n_chunks = ctx->n_chunks;
-    p.n_stages = ctx->n_stages;
-    p.acc_bufs = ctx->acc_bufs;
-    p.acc_stride = ctx->acc_stride;
-    p.tmem_cols = ctx->tmem_cols;
+    p.group_w = sc.group_w;
+    p.n_groups = sc.n_groups;
+    p.chunk_n = sc.chunk_n;
+    p.n_chunks = sc.n_chunks;
+    p.n_stages = sc.n_stages;
+    p.acc_bufs = sc.acc_bufs;
+    p.acc_stride = sc.acc_stride;
+    p.tmem_cols = sc.tmem_cols;
     p.n_hidden = c.hidden;
     p.n_heads = c.n_kv_heads;
     p.b1 = ctx->b1_all;
@@ -226,20 +234,38 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.b2 = ctx->b2_all;
     p.scores = scores;
     p.maskbits = maskbits;
-    p.n_words = tiles_per_layer * 4;
+    p.n_words = blocks_per_layer * 4;
     p.cu_seqlens = cu_seqlens;
     p.n_seqs = n_seqs;
     p.window = w;
     p.window_keep = window_keep;
     p.tau = tau;
     p.status = ctx->status_dev;
-    const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
     {
         ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
-        if (c.hidden > 0)
-            score_kernel<true><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, ctx->tmap_w, p);
-        else
-            score_kernel<false><<<grid, kScoreThreads, ctx->score_smem, stream>>>(tmap_x, ctx->tmap_w, p);
+        if (pair) {
+            const int n_clusters = static_cast<int>(n_tiles < ctx->pair_clusters ? n_tiles : ctx->pair_clusters);
+            cudaLaunchConfig_t cfg;
+            memset(&cfg, 0, sizeof cfg);
+            cfg.gridDim = dim3(static_cast<unsigned>(2 * n_clusters));
+            cfg.blockDim = dim3(kScoreThreads);
+            cfg.dynamicSmemBytes = sc.smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, true>, tmap_x, sc.tmap_w, p));
+        } else {
+            const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
+            if (c.hidden > 0)
+                score_kernel<true, false><<<grid, kScoreThreads, sc.smem, stream>>>(tmap_x, sc.tmap_w, p);
+            else
+                score_kernel<false, false><<<grid, kScoreThreads, sc.smem, stream>>>(tmap_x, sc.tmap_w, p);
+        }
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
@@ -329,32 +355,34 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     ctx->cfg = c;
     ctx->sm_count = prop.multiProcessorCount;
 
-    // scoring schedule
-    if (c.hidden == 0) {
-        ctx->w1_rows = 16;            // H <= 8 outputs padded to the smallest N of a 128-row MMA
-        ctx->group_w = 16; ctx->n_groups = 1; ctx->chunk_n = 16; ctx->n_chunks = 1;
-        ctx->acc_bufs = 2; ctx->acc_stride = 32;
-    } else {
-        ctx->w1_rows = c.hidden;
-        ctx->n_groups = c.hidden > 512 ? 2 : 1;
-        ctx->group_w = c.hidden / ctx->n_groups;
-        ctx->n_chunks = ctx->group_w > 256 ? 2 : 1;
-        ctx->chunk_n = ctx->group_w / ctx->n_chunks;
-        ctx->acc_bufs = 512 / ctx->group_w >= 2 ? 2 : 1;
-        ctx->acc_stride = ctx->group_w;
-    }
-    ctx->tmem_cols = next_pow2(ctx->acc_bufs * ctx->acc_stride);
-    {
-        const int budget = static_cast<int>(prop.sharedMemPerBlockOptin) - 1024;
+    // scoring schedules
+    const int budget = static_cast<int>(prop.sharedMemPerBlockOptin) - 1024;
+    for (int mode = 0; mode < (c.hidden > 0 ? 2 : 1); ++mode) {
+        kvzap_ctx::Schedule &sc = ctx->sched[mode];
+        if (c.hidden == 0) {
+            ctx->w1_rows = 16;            // H <= 8 outputs padded to the smallest N of a 128-row MMA
+            sc.group_w = 16; sc.n_groups = 1; sc.chunk_n = 16; sc.n_chunks = 1;
+            sc.acc_bufs = 2; sc.acc_stride = 32;
+        } else {
+            ctx->w1_rows = c.hidden;
+            sc.n_groups = c.hidden > 512 ? 2 : 1;
+            sc.group_w = c.hidden / sc.n_groups;
+            sc.n_chunks = sc.group_w > 256 ? 2 : 1;
+            sc.chunk_n = sc.group_w / sc.n_chunks;
+            sc.acc_bufs = 512 / sc.group_w >= 2 ? 2 : 1;
+            sc.acc_stride = sc.group_w;
+        }
+        sc.tmem_cols = next_pow2(sc.acc_bufs * sc.acc_stride);
+        const int b_rows = sc.group_w / (mode + 1);
         int stages = kMaxStages;
         for (; stages >= 2; --stages)
-            if (static_cast<int>(score_smem_layout(ctx->group_w, stages, c.hidden).total) <= budget) break;
+            if (static_cast<int>(score_smem_layout(b_rows, stages, c.hidden).total) <= budget) break;
         if (stages < 2) {
             delete ctx;
             return fail(nullptr, KVZAP_ERR_UNSUPPORTED, "shared memory too small for this surrogate shape");
         }
-        ctx->n_stages = stages;
-        ctx->score_smem = score_smem_layout(ctx->group_w, stages, c.hidden).total + 1024;
+        sc.n_stages = stages;
+        sc.smem = score_smem_layout(b_rows, stages, c.hidden).total + 1024;
     }
 
 #define CREATE_CUDA(call)                                                                              \
@@ -378,10 +406,33 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         }
         ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(ctx->score_smem)));
-    CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(ctx->score_smem)));
+    if (c.hidden > 0) {
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(ctx->sched[0].smem)));
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(ctx->sched[1].smem)));
+        // how many CTA pairs fit on the device at once (one CTA per SM, both SMs of a pair adjacent)
+        cudaLaunchConfig_t qcfg;
+        memset(&qcfg, 0, sizeof qcfg);
+        qcfg.gridDim = dim3(static_cast<unsigned>(ctx->sm_count / 2 * 2));
+        qcfg.blockDim = dim3(kScoreThreads);
+        qcfg.dynamicSmemBytes = ctx->sched[1].smem;
+        cudaLaunchAttribute qattr[1];
+        qattr[0].id = cudaLaunchAttributeClusterDimension;
+        qattr[0].val.clusterDim.x = 2;
+        qattr[0].val.clusterDim.y = 1;
+        qattr[0].val.clusterDim.z = 1;
+        qcfg.attrs = qattr;
+        qcfg.numAttrs = 1;
+        int n_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&n_clusters, score_kernel<true, true>, &qcfg) == cudaSuccess && n_clusters > 0)
+            ctx->pair_clusters = n_clusters < ctx->sm_count / 2 ? n_clusters : ctx->sm_count / 2;
+        else
+            cudaGetLastError();          // pairs unavailable: the one-CTA kernel serves every size
+    } else {
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(ctx->sched[0].smem)));
+    }
 
     ctx->layer_set.assign(c.n_layers, 0);
     {
@@ -395,12 +446,15 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
             CREATE_CUDA(cudaMalloc(&ctx->b2_all, sizeof(float) * c.n_layers * kMaxHeads));
         }
         ctx->err[0] = 0;
-        if (make_tmap(ctx, &ctx->tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
-                      static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(ctx->chunk_n)) != KVZAP_OK) {
-            snprintf(g_create_error, sizeof g_create_error, "%s", ctx->err);
-            free_all(ctx);
-            delete ctx;
-            return KVZAP_ERR_CUDA;
+        for (int mode = 0; mode < (c.hidden > 0 ? 2 : 1); ++mode) {
+            kvzap_ctx::Schedule &sc = ctx->sched[mode];
+            if (make_tmap(ctx, &sc.tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
+                          static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(sc.chunk_n / (mode + 1))) != KVZAP_OK) {
+                snprintf(g_create_error, sizeof g_create_error, "%s", ctx->err);
+                free_all(ctx);
+                delete ctx;
+                return KVZAP_ERR_CUDA;
+            }
         }
     }
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;

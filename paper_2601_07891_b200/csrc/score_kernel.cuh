@@ -1,6 +1,6 @@
 // Surrogate scoring on the 5th-generation tensor cores (Method, "KVzap").
 //
-// One persistent CTA per SM walks 128-token tiles.  Per tile the first layer
+// Persistent CTAs walk 128-token tiles.  Per tile the first layer
 //   Z[128, N] = X[128, D_h] * W1^T          (bf16 x bf16 -> fp32)
 // is a chain of tcgen05.mma instructions fed by TMA through a ring of shared
 // memory stages, with the accumulator in tensor memory.  The epilogue reads
@@ -15,13 +15,20 @@
 // TMEM owner, warps 2..9 = epilogue (two warps per TMEM lane quarter; in the
 // MLP each takes one half of the hidden units and the halves are combined
 // through shared memory).
+//
+// kPair = true runs the kernel as clusters of two CTAs on neighbouring SMs
+// (tcgen05 cta_group::2): a pair works on 256 tokens, each CTA holds its own
+// 128 rows of X and of the accumulator but only HALF of the W1 rows of every
+// K step, and the MMAs issued by the pair's first CTA read both halves.  That
+// halves the W1 bytes each SM has to pull from L2 per FLOP, which is what
+// bounds the one-CTA version when the hidden layer is wide.
 #pragma once
 
 #include "ptx.cuh"
 
 namespace kvzap {
 
-constexpr int kTileM = 128;            // tokens per tile = UMMA M
+constexpr int kTileM = 128;            // tokens per CTA tile = rows of one CTA's accumulator
 constexpr int kBlockK = 64;            // bf16 elements per 128-byte swizzled row
 constexpr int kUmmaK = 16;             // K of one tcgen05.mma for 16-bit inputs
 constexpr int kATileBytes = kTileM * kBlockK * 2;
@@ -31,8 +38,9 @@ constexpr int kMaxHeads = 8;
 
 struct ScoreParams {
     int64_t n_tokens;        // rows (tokens) per layer
-    int32_t n_tiles;         // tiles_per_layer * n_layers_call
+    int32_t n_tiles;         // work tiles = tiles_per_layer * n_layers_call (a work tile is 128 rows, or 256 for a pair)
     int32_t tiles_per_layer;
+    int32_t blocks_per_layer;   // 128-token blocks per layer = ceil(n_tokens / 128)
     int32_t n_layers_call;   // layers scored by this launch (hidden is [n_layers_call][n_tokens][d_model])
     int32_t layer0;          // first layer: selects the rows of the stacked weights
     int32_t w_rows;          // rows of W1 per layer in the stacked weight matrix
@@ -52,7 +60,7 @@ struct ScoreParams {
     const float *b2;      // MLP: [L][8]
     float *scores;        // [n_layers_call][n_tokens, n_heads] or nullptr
     uint32_t *maskbits;   // [n_layers_call][n_heads][n_words] or nullptr
-    int64_t n_words;      // 32-token words per head and layer (= 4 * tiles_per_layer)
+    int64_t n_words;      // 32-token words per head and layer (= 4 * blocks_per_layer)
     const int32_t *cu_seqlens;   // [n_seqs + 1] or nullptr (one sequence)
     int32_t n_seqs;
     int32_t window;
@@ -62,13 +70,14 @@ struct ScoreParams {
 };
 
 // Byte offsets inside the dynamic shared memory block (after 1024-byte alignment).
+// `b_rows` = rows of W1 one CTA stages per K step (group_w, or group_w / 2 for a pair).
 struct ScoreSmemLayout {
     uint32_t stage_bytes, stages_end, w2s, b1s, part, bars, total;
 };
-__host__ __device__ inline ScoreSmemLayout score_smem_layout(int group_w, int n_stages, int n_hidden)
+__host__ __device__ inline ScoreSmemLayout score_smem_layout(int b_rows, int n_stages, int n_hidden)
 {
     ScoreSmemLayout L;
-    L.stage_bytes = kATileBytes + static_cast<uint32_t>(group_w) * kBlockK * 2;
+    L.stage_bytes = kATileBytes + static_cast<uint32_t>(b_rows) * kBlockK * 2;
     L.stages_end = L.stage_bytes * n_stages;
     L.w2s = L.stages_end;
     L.b1s = L.w2s + static_cast<uint32_t>(n_hidden) * kMaxHeads * 4;
@@ -78,9 +87,31 @@ __host__ __device__ inline ScoreSmemLayout score_smem_layout(int group_w, int n_
     return L;
 }
 
-__device__ __forceinline__ float gelu_erf(float z)
+// GELU(z) = z * Phi(z) for two values at once, through the complementary error function
+//   erfc(x) = (a1 t + a2 t^2 + a3 t^3 + a4 t^4 + a5 t^5) exp(-x^2),  t = 1 / (1 + p x),  x >= 0
+// (Abramowitz & Stegun, formula 7.1.26, |error| <= 1.5e-7), with x = |z| / sqrt(2):
+//   q = erfc(x) / 2,   GELU(z) = z / 2 + |z| (1/2 - q).
+// Measured against the fp64 erf form: absolute error below 5e-7 for |z| <= 12.
+__device__ __forceinline__ uint64_t gelu_pair(uint64_t z2)
 {
-    return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
+    constexpr float kP = 0.3275911f * 0.70710678118654752f;     // p / sqrt(2): t is computed from |z| directly
+    constexpr float kA1 = 0.5f * 0.254829592f, kA2 = 0.5f * -0.284496736f, kA3 = 0.5f * 1.421413741f,
+                    kA4 = 0.5f * -1.453152027f, kA5 = 0.5f * 1.061405429f;
+    constexpr float kC = -0.5f * 1.4426950408889634f;            // exp(-z^2/2) = 2^(kC z^2)
+    float z0, z1;
+    f2_unpack(z2, z0, z1);
+    const uint64_t t = f2_pack(fast_rcp(fmaf(kP, fabsf(z0), 1.0f)), fast_rcp(fmaf(kP, fabsf(z1), 1.0f)));
+    uint64_t u = f2_fma(f2_pack(kA5, kA5), t, f2_pack(kA4, kA4));
+    u = f2_fma(u, t, f2_pack(kA3, kA3));
+    u = f2_fma(u, t, f2_pack(kA2, kA2));
+    u = f2_fma(u, t, f2_pack(kA1, kA1));
+    u = f2_mul(u, t);
+    float m0, m1;
+    f2_unpack(f2_mul(f2_mul(z2, z2), f2_pack(kC, kC)), m0, m1);
+    const uint64_t q = f2_mul(u, f2_pack(fast_ex2(m0), fast_ex2(m1)));
+    float h0, h1;
+    f2_unpack(f2_fma(q, f2_pack(-1.0f, -1.0f), f2_pack(0.5f, 0.5f)), h0, h1);
+    return f2_pack(fmaf(fabsf(z0), h0, 0.5f * z0), fmaf(fabsf(z1), h1, 0.5f * z1));
 }
 
 // Index of the sequence that owns packed token t (cu[b] <= t < cu[b+1]).
@@ -94,26 +125,52 @@ __device__ __forceinline__ int seq_of_token(const int32_t *cu, int n_seqs, int64
     return lo;
 }
 
-template <bool kMlp>
+// Second layer for 32 accumulator columns j0 .. j0+31 of one token: acc[h] (+)= GELU(r + b1) . W2.
+// Hidden units are taken two at a time; acc[h] holds the partial sums of the even and of the odd
+// units of head h.  w2p is W2 repacked as [j / 2][h] pairs {W2[h][j], W2[h][j+1]}.
+__device__ __forceinline__ void mlp_columns(const uint32_t (&r)[32], int j0, const float *b1s, const ulonglong2 *w2p,
+                                            uint64_t (&acc)[kMaxHeads])
+{
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const int j = j0 + i;
+        const float2 b = *reinterpret_cast<const float2 *>(b1s + j);
+        const uint64_t z2 = f2_add(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), f2_pack(b.x, b.y));
+        const uint64_t g2 = gelu_pair(z2);
+        const ulonglong2 *w = w2p + (j >> 1) * 4;
+#pragma unroll
+        for (int hp = 0; hp < 4; ++hp) {
+            const ulonglong2 ww = w[hp];
+            acc[2 * hp] = f2_fma(g2, ww.x, acc[2 * hp]);
+            acc[2 * hp + 1] = f2_fma(g2, ww.y, acc[2 * hp + 1]);
+        }
+    }
+}
+
+template <bool kMlp, bool kPair>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
              const ScoreParams p)
 {
+    static_assert(kMlp || !kPair, "CTA pairs are used for the MLP surrogate only");
+    constexpr int kCtas = kPair ? 2 : 1;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t *smem = smem_raw + pad;
     const uint32_t smem_base = raw_addr + pad;
-    const ScoreSmemLayout L = score_smem_layout(p.group_w, p.n_stages, kMlp ? p.n_hidden : 0);
+    const int b_rows_chunk = p.chunk_n / kCtas;                 // W1 rows this CTA stages per MMA chunk
+    const ScoreSmemLayout L = score_smem_layout(p.group_w / kCtas, p.n_stages, kMlp ? p.n_hidden : 0);
 
-    float4 *w2s = reinterpret_cast<float4 *>(smem + L.w2s);
+    ulonglong2 *w2p = reinterpret_cast<ulonglong2 *>(smem + L.w2s);
+    float *w2f = reinterpret_cast<float *>(smem + L.w2s);
     float *b1s = reinterpret_cast<float *>(smem + L.b1s);
     float *part = reinterpret_cast<float *>(smem + L.part);
     const uint32_t bars = smem_base + L.bars;
-    const uint32_t bar_full = bars;                      // [kMaxStages] TMA -> MMA
+    const uint32_t bar_full = bars;                      // [kMaxStages] TMA -> MMA (the pair's first CTA's is used)
     const uint32_t bar_empty = bars + 8 * kMaxStages;    // [kMaxStages] MMA -> TMA
     const uint32_t bar_tfull = bars + 16 * kMaxStages;   // [2] MMA -> epilogue
-    const uint32_t bar_tempty = bar_tfull + 16;          // [2] epilogue -> MMA
+    const uint32_t bar_tempty = bar_tfull + 16;          // [2] epilogue -> MMA (the pair's first CTA's is used)
     const uint32_t bar_done = bar_tempty + 16;           // [1] abort path only
     const uint32_t bar_pfull = bar_done + 8;             // [1] MLP: second column half -> first
     const uint32_t bar_pempty = bar_pfull + 8;           // [1] MLP: first column half -> second
@@ -124,6 +181,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     constexpr int kEpiWarps = kMlp ? 8 : 4;
+    uint32_t cta_rank = 0;
+    if constexpr (kPair) cta_rank = cluster_cta_rank();
+    const bool leader = cta_rank == 0;
+    const int unit = kPair ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int n_units = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -132,7 +194,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar_tfull + 8 * b, 1);
-            mbar_init(bar_tempty + 8 * b, kEpiWarps);
+            mbar_init(bar_tempty + 8 * b, kEpiWarps * kCtas);
         }
         mbar_init(bar_done, 1);
         mbar_init(bar_pfull, 4);
@@ -144,24 +206,31 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         prefetch_tensormap(&tmap_w);
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
-        tmem_relinquish();
+        if constexpr (kPair) {
+            tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
+            tmem_relinquish_pair();
+        } else {
+            tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
+            tmem_relinquish();
+        }
     }
     tc_fence_before_sync();
     __syncthreads();
+    if constexpr (kPair) cluster_sync_all();     // the other CTA's barriers exist before anything signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
     const int k_blocks = p.d_model / kBlockK;
-    const uint32_t stage_tx = L.stage_bytes;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
         const uint64_t pol_x = l2_policy_evict_first();   // hidden states are streamed once
         const uint64_t pol_w = l2_policy_evict_last();    // weights are re-read by every tile
         uint32_t it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
+        for (int tile = unit; tile < p.n_tiles && ok; tile += n_units) {
+            const int l_rel = tile / p.tiles_per_layer;
+            const int m_tile = (tile - l_rel * p.tiles_per_layer) * kCtas + static_cast<int>(cta_rank);
             for (int g = 0; g < p.n_groups && ok; ++g) {
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const uint32_t s = it % p.n_stages;
@@ -172,14 +241,24 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     if (!got) { ok = false; break; }
                     if (lane == 0) {
                         const uint32_t sa = smem_base + s * L.stage_bytes;
-                        mbar_arrive_expect_tx(bar_full + 8 * s, stage_tx);
-                        const int l_rel = tile / p.tiles_per_layer;
-                        const int m_tile = tile - l_rel * p.tiles_per_layer;
                         const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w;
-                        tma_load_3d(sa, &tmap_x, bar_full + 8 * s, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
-                        for (int c = 0; c < p.n_chunks; ++c)
-                            tma_load_2d(sa + kATileBytes + c * p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * s,
-                                        kb * kBlockK, w_row0 + c * p.chunk_n, pol_w);
+                        if constexpr (kPair) {
+                            // the first CTA's barrier counts the bytes of both CTAs
+                            if (leader) mbar_arrive_expect_tx(bar_full + 8 * s, L.stage_bytes * 2);
+                            const uint32_t bar = map_to_cta(bar_full + 8 * s, 0);
+                            tma_load_3d_pair(sa, &tmap_x, bar, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
+                            for (int c = 0; c < p.n_chunks; ++c)
+                                tma_load_2d_pair(sa + kATileBytes + c * b_rows_chunk * kBlockK * 2, &tmap_w, bar,
+                                                 kb * kBlockK,
+                                                 w_row0 + c * p.chunk_n + static_cast<int>(cta_rank) * b_rows_chunk,
+                                                 pol_w);
+                        } else {
+                            mbar_arrive_expect_tx(bar_full + 8 * s, L.stage_bytes);
+                            tma_load_3d(sa, &tmap_x, bar_full + 8 * s, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
+                            for (int c = 0; c < p.n_chunks; ++c)
+                                tma_load_2d(sa + kATileBytes + c * p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * s,
+                                            kb * kBlockK, w_row0 + c * p.chunk_n, pol_w);
+                        }
                     }
                     __syncwarp();
                 }
@@ -187,64 +266,82 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         }
         if (!ok && lane == 0) {
             // abort path: let the copies already in flight land before the CTA exits
-            const uint32_t n_out = it < static_cast<uint32_t>(p.n_stages) ? it : static_cast<uint32_t>(p.n_stages);
-            for (uint32_t j = 0; j < n_out; ++j) {
-                const uint32_t fill = it - 1 - j;
-                const uint32_t s = fill % p.n_stages;
+            if (leader) {
+                const uint32_t n_out = it < static_cast<uint32_t>(p.n_stages) ? it : static_cast<uint32_t>(p.n_stages);
+                for (uint32_t j = 0; j < n_out; ++j) {
+                    const uint32_t fill = it - 1 - j;
+                    const uint32_t s = fill % p.n_stages;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(bar_full + 8 * s, (fill / p.n_stages) & 1u))
+                        if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+                }
+            } else {
+                // this CTA's copies complete on the other CTA's barriers: give them a fixed time instead
                 const long long t0 = clock64();
-                while (!mbar_try_wait(bar_full + 8 * s, (fill / p.n_stages) & 1u))
-                    if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+                while (clock64() - t0 < 2000000LL) { }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = umma_idesc_bf16_f32(kTileM, static_cast<uint32_t>(p.chunk_n));
-        uint32_t it = 0, acc_it = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x) {
-            for (int g = 0; g < p.n_groups && ok; ++g, ++acc_it) {
-                const uint32_t buf = acc_it % p.acc_bufs;
-                const uint32_t use = acc_it / p.acc_bufs;
-                int got = 0;
-                if (lane == 0) got = mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
-                got = __shfl_sync(0xffffffffu, got, 0);
-                if (!got) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * p.acc_stride;
-                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-                    const uint32_t s = it % p.n_stages;
-                    const uint32_t round = it / p.n_stages;
-                    if (lane == 0) got = mbar_wait(bar_full + 8 * s, round & 1u, abort_flag) ? 1 : 0;
+        // ------------------------------------------------------------ MMA issuer (a pair: its first CTA only)
+        if (leader) {
+            const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.chunk_n));
+            uint32_t it = 0, acc_it = 0;
+            bool ok = true;
+            for (int tile = unit; tile < p.n_tiles && ok; tile += n_units) {
+                for (int g = 0; g < p.n_groups && ok; ++g, ++acc_it) {
+                    const uint32_t buf = acc_it % p.acc_bufs;
+                    const uint32_t use = acc_it / p.acc_bufs;
+                    int got = 0;
+                    if (lane == 0) got = mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
                     got = __shfl_sync(0xffffffffu, got, 0);
                     if (!got) { ok = false; break; }
                     tc_fence_after_sync();
-                    if (lane == 0) {
-                        const uint32_t sa = smem_base + s * L.stage_bytes;
-                        const uint64_t a_desc = umma_desc_k_major_sw128(sa);
+                    const uint32_t d_tmem = tmem_base + buf * p.acc_stride;
+                    for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+                        const uint32_t s = it % p.n_stages;
+                        const uint32_t round = it / p.n_stages;
+                        if (lane == 0) got = mbar_wait(bar_full + 8 * s, round & 1u, abort_flag) ? 1 : 0;
+                        got = __shfl_sync(0xffffffffu, got, 0);
+                        if (!got) { ok = false; break; }
+                        tc_fence_after_sync();
+                        if (lane == 0) {
+                            const uint32_t sa = smem_base + s * L.stage_bytes;
+                            const uint64_t a_desc = umma_desc_k_major_sw128(sa);
 #pragma unroll
-                        for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                            // advancing K by 16 elements = 32 bytes = 2 descriptor address units
-                            for (int c = 0; c < p.n_chunks; ++c) {
-                                const uint64_t b_desc =
-                                    umma_desc_k_major_sw128(sa + kATileBytes + c * p.chunk_n * kBlockK * 2);
-                                umma_bf16(d_tmem + c * p.chunk_n, a_desc + 2 * k, b_desc + 2 * k, idesc,
-                                          (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                                // advancing K by 16 elements = 32 bytes = 2 descriptor address units
+                                for (int c = 0; c < p.n_chunks; ++c) {
+                                    const uint64_t b_desc =
+                                        umma_desc_k_major_sw128(sa + kATileBytes + c * b_rows_chunk * kBlockK * 2);
+                                    if constexpr (kPair)
+                                        umma_bf16_pair(d_tmem + c * p.chunk_n, a_desc + 2 * k, b_desc + 2 * k, idesc,
+                                                       (kb | k) != 0 ? 1u : 0u);
+                                    else
+                                        umma_bf16(d_tmem + c * p.chunk_n, a_desc + 2 * k, b_desc + 2 * k, idesc,
+                                                  (kb | k) != 0 ? 1u : 0u);
+                                }
                             }
+                            // the stage is free (in both CTAs) once these MMAs retire
+                            if constexpr (kPair) umma_commit_pair(bar_empty + 8 * s, 3);
+                            else umma_commit(bar_empty + 8 * s);
                         }
-                        umma_commit(bar_empty + 8 * s);          // stage is free once these MMAs retire
+                        __syncwarp();
+                    }
+                    if (ok && lane == 0) {                   // accumulator complete
+                        if constexpr (kPair) umma_commit_pair(bar_tfull + 8 * buf, 3);
+                        else umma_commit(bar_tfull + 8 * buf);
                     }
                     __syncwarp();
                 }
-                if (ok && lane == 0) umma_commit(bar_tfull + 8 * buf);   // accumulator complete
-                __syncwarp();
             }
-        }
-        if (!ok && lane == 0) {
-            // abort path: wait (bounded) for the MMAs already issued before TMEM is freed
-            umma_commit(bar_done);
-            const long long t0 = clock64();
-            while (!mbar_try_wait(bar_done, 0))
-                if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+            if (!ok && lane == 0) {
+                // abort path: wait (bounded) for the MMAs already issued before TMEM is freed
+                if constexpr (kPair) umma_commit_pair(bar_done, 1);
+                else umma_commit(bar_done);
+                const long long t0 = clock64();
+                while (!mbar_try_wait(bar_done, 0))
+                    if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+            }
         }
     } else {
         // ------------------------------------------------------------ epilogue
@@ -256,10 +353,15 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         uint32_t acc_it = 0, tile_it = 0, epi_it = 0;
         int cur_layer = -1;
         bool ok = true;
+        uint32_t tempty_addr[2] = {bar_tempty, bar_tempty + 8};
+        if constexpr (kPair) {
+            tempty_addr[0] = map_to_cta(bar_tempty, 0);
+            tempty_addr[1] = map_to_cta(bar_tempty + 8, 0);
+        }
         if (active) {
-            for (int tile = blockIdx.x; tile < p.n_tiles && ok; tile += gridDim.x, ++tile_it) {
+            for (int tile = unit; tile < p.n_tiles && ok; tile += n_units, ++tile_it) {
                 const int l_rel = tile / p.tiles_per_layer;
-                const int m_tile = tile - l_rel * p.tiles_per_layer;
+                const int m_tile = (tile - l_rel * p.tiles_per_layer) * kCtas + static_cast<int>(cta_rank);
                 const int layer = p.layer0 + l_rel;
                 if constexpr (kMlp) {
                     if (layer != cur_layer) {
@@ -272,10 +374,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                             if (!mbar_wait(bar_epi, epi_it & 1u, abort_flag)) { ok = false; break; }
                             ++epi_it;
                         }
-                        const float4 *w2g = reinterpret_cast<const float4 *>(p.w2t) +
-                                            static_cast<int64_t>(layer) * p.n_hidden * 2;
+                        const float *w2g = p.w2t + static_cast<int64_t>(layer) * p.n_hidden * kMaxHeads;
                         const float *b1g = p.b1 + static_cast<int64_t>(layer) * p.n_hidden;
-                        for (int i = etid; i < p.n_hidden * 2; i += kEpiWarps * 32) w2s[i] = __ldg(w2g + i);
+                        for (int i = etid; i < p.n_hidden * kMaxHeads; i += kEpiWarps * 32) {
+                            const int j = i >> 3, h = i & 7;      // W2[h][j] -> pair slot (j / 2, h), element j % 2
+                            w2f[(((j >> 1) * kMaxHeads + h) << 1) + (j & 1)] = __ldg(w2g + i);
+                        }
                         for (int i = etid; i < p.n_hidden; i += kEpiWarps * 32) b1s[i] = __ldg(b1g + i);
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_epi);
@@ -285,8 +389,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     }
                 }
                 float s[kMaxHeads];
+                uint64_t acc[kMaxHeads];
 #pragma unroll
-                for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+                for (int h = 0; h < kMaxHeads; ++h) { s[h] = 0.0f; acc[h] = 0ull; }
                 for (int g = 0; g < p.n_groups; ++g, ++acc_it) {
                     const uint32_t buf = acc_it % p.acc_bufs;
                     const uint32_t use = acc_it / p.acc_bufs;
@@ -297,23 +402,19 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         const int half_w = p.group_w >> 1;
                         const int col0 = hsel * half_w;
                         const int j0 = g * p.group_w + col0;
-                        for (int c = 0; c < half_w; c += 32) {
-                            uint32_t r[32];
-                            tmem_ld_x32(t_row + col0 + c, r);
+                        // two register sets: the next 32 columns are in flight while these are processed
+                        uint32_t ra[32], rb[32];
+                        tmem_ld_x32(t_row + col0, ra);
+                        for (int c = 0; c < half_w; c += 64) {
                             tmem_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const int j = j0 + c + i;
-                                const float gz = gelu_erf(__uint_as_float(r[i]) + b1s[j]);
-                                const float4 wa = w2s[2 * j], wb = w2s[2 * j + 1];
-                                s[0] = fmaf(gz, wa.x, s[0]);
-                                s[1] = fmaf(gz, wa.y, s[1]);
-                                s[2] = fmaf(gz, wa.z, s[2]);
-                                s[3] = fmaf(gz, wa.w, s[3]);
-                                s[4] = fmaf(gz, wb.x, s[4]);
-                                s[5] = fmaf(gz, wb.y, s[5]);
-                                s[6] = fmaf(gz, wb.z, s[6]);
-                                s[7] = fmaf(gz, wb.w, s[7]);
+                            reg_fence32(ra);
+                            if (c + 32 < half_w) tmem_ld_x32(t_row + col0 + c + 32, rb);
+                            mlp_columns(ra, j0 + c, b1s, w2p, acc);
+                            if (c + 32 < half_w) {
+                                tmem_wait_ld();
+                                reg_fence32(rb);
+                                if (c + 64 < half_w) tmem_ld_x32(t_row + col0 + c + 64, ra);
+                                mlp_columns(rb, j0 + c + 32, b1s, w2p, acc);
                             }
                         }
                     } else {
@@ -327,10 +428,19 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     // this warp is done reading the accumulator buffer
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_tempty + 8 * buf);
+                    if (lane == 0) {
+                        if constexpr (kPair) mbar_arrive_cluster(tempty_addr[buf]);
+                        else mbar_arrive(bar_tempty + 8 * buf);
+                    }
                 }
                 if (!ok) break;
                 if constexpr (kMlp) {
+#pragma unroll
+                    for (int h = 0; h < kMaxHeads; ++h) {
+                        float lo, hi;
+                        f2_unpack(acc[h], lo, hi);
+                        s[h] = lo + hi;
+                    }
                     // combine the two column halves through `part`; the hsel = 0 warps finish the tile
                     if (hsel == 1) {
                         if (!mbar_wait(bar_pempty, (tile_it & 1u) ^ 1u, abort_flag)) { ok = false; break; }
@@ -355,7 +465,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         s[7] += pb.w + __ldg(p.b2 + layer * kMaxHeads + 7);
                     }
                 }
-                if (hsel == 0) {
+                if (hsel == 0 && m_tile < p.blocks_per_layer) {
                     const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;      // row inside the layer
                     const bool valid = t < p.n_tokens;
                     if (valid && p.scores != nullptr) {
@@ -395,10 +505,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
 
     tc_fence_before_sync();
     __syncthreads();
+    // a pair: neither CTA leaves (or frees tensor memory) while the other may still read its shared
+    // memory, signal its barriers or write its accumulator
+    if constexpr (kPair) cluster_sync_all();
     if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
     if (warp == 1) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        if constexpr (kPair) tmem_dealloc_pair(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        else tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
     }
 }
 
