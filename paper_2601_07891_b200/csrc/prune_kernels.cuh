@@ -287,4 +287,140 @@ compact_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *
     }
 }
 
+// ---------------------------------------------------------------------------
+// Dense-ragged compaction without a separate scan pass.  Grid (chunks, H): a CTA owns
+// `blocks_per_cta` consecutive 128-token blocks of one head.  It first counts, straight from the
+// mask words, the rows kept before its first block (and before the start of the sequence that is
+// in progress there), then walks its blocks keeping a running count, so that every kept row's
+// slot in its (sequence, head) list is known without any other CTA's help.  lengths[b,h] is
+// written by the thread that handles the last token of sequence b; empty sequences by chunk 0.
+constexpr int kDenseThreads = 256;
+
+// bits of the block's four words below in-block position r (0..128)
+__device__ __forceinline__ int popc_below(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, int r)
+{
+    int n = 0;
+    const uint32_t w[4] = {w0, w1, w2, w3};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int lo = i * 32;
+        if (r >= lo + 32) n += __popc(w[i]);
+        else if (r > lo) n += __popc(w[i] & ((1u << (r - lo)) - 1u));
+    }
+    return n;
+}
+
+__global__ void __launch_bounds__(kDenseThreads)
+compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ K_out,
+                     uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
+                     int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
+                     int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths)
+{
+    __shared__ int32_t src_tok[kBlockTokens];
+    __shared__ int64_t dst_row[kBlockTokens];
+    __shared__ int32_t red[2][kDenseThreads / 32];
+    __shared__ int32_t base_next_s;
+    const int h = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t blk0 = static_cast<int64_t>(blockIdx.x) * blocks_per_cta;
+    const int64_t blk1 = blk0 + blocks_per_cta < n_blocks ? blk0 + blocks_per_cta : n_blocks;
+    const bool multi = cu_seqlens != nullptr && n_seqs > 1;
+    const uint32_t *words = maskbits + static_cast<int64_t>(h) * n_words;
+
+    if (blockIdx.x == 0 && cu_seqlens != nullptr)         // empty sequences have no last token to write for them
+        for (int b = tid; b < n_seqs; b += kDenseThreads)
+            if (cu_seqlens[b + 1] == cu_seqlens[b]) lengths[b * n_heads + h] = 0;
+    if (blk0 >= n_blocks) return;
+
+    // rows kept before this CTA's first token, and before the start of the sequence in progress there
+    const int64_t t0 = blk0 * kBlockTokens;
+    int64_t s0 = 0;
+    if (multi) s0 = cu_seqlens[seq_of_token(cu_seqlens, n_seqs, t0)];
+    int32_t total = 0, before_s0 = 0;
+    for (int64_t i = tid; i < blk0 * 4; i += kDenseThreads) {
+        const uint32_t w = words[i];
+        const int c = __popc(w);
+        total += c;
+        const int64_t lo = i * 32;
+        if (lo + 32 <= s0) before_s0 += c;
+        else if (lo < s0) before_s0 += __popc(w & ((1u << static_cast<int>(s0 - lo)) - 1u));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+        before_s0 += __shfl_xor_sync(0xffffffffu, before_s0, o);
+    }
+    if (lane == 0) { red[0][warp] = total; red[1][warp] = before_s0; }
+    __syncthreads();
+    int32_t running = 0, base_cur = 0;       // kept before the current block / before the sequence in progress at its start
+#pragma unroll
+    for (int i = 0; i < kDenseThreads / 32; ++i) { running += red[0][i]; base_cur += red[1][i]; }
+
+    const int group = tid >> 4, gl = tid & 15;
+    constexpr int kGroups = kDenseThreads / 16;
+    for (int64_t blk = blk0; blk < blk1; ++blk) {
+        const uint4 wv = *reinterpret_cast<const uint4 *>(words + blk * 4);
+        const uint32_t w0 = wv.x, w1 = wv.y, w2 = wv.z, w3 = wv.w;
+        const int cnt = __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
+        const int64_t blk_start = blk * kBlockTokens;
+        if (tid < kBlockTokens) {
+            const int64_t t = blk_start + tid;
+            if (t < n_tokens) {
+                int b = 0;
+                int64_t s = 0, e = n_tokens;
+                if (multi) {
+                    b = seq_of_token(cu_seqlens, n_seqs, t);
+                    s = cu_seqlens[b];
+                    e = cu_seqlens[b + 1];
+                }
+                // kept rows before the start of this token's sequence
+                const int32_t base = s >= blk_start ? running + popc_below(w0, w1, w2, w3, static_cast<int>(s - blk_start))
+                                                    : base_cur;
+                const int r = popc_below(w0, w1, w2, w3, tid);
+                const uint32_t w = tid < 32 ? w0 : tid < 64 ? w1 : tid < 96 ? w2 : w3;
+                const bool keep = (w >> (tid & 31)) & 1u;
+                if (keep) {
+                    src_tok[r] = tid;
+                    dst_row[r] = static_cast<int64_t>(h) * n_tokens + s + (running + r - base);
+                }
+                if (t + 1 == e) lengths[b * n_heads + h] = running + r + (keep ? 1 : 0) - base;
+                if (tid == kBlockTokens - 1 || t + 1 == n_tokens) {
+                    // base of the sequence in progress at the next block's first token
+                    int32_t nb = base;
+                    if (multi && t + 1 == e) nb = running + cnt;      // a new sequence starts exactly there
+                    base_next_s = nb;
+                }
+            }
+        }
+        __syncthreads();
+        const int64_t head_row0 = static_cast<int64_t>(h) * n_tokens + blk_start;
+        for (int i0 = group; i0 < cnt; i0 += kGroups * kRowsInFlight) {
+            for (int u0 = gl; u0 < row_units; u0 += 16) {
+                uint4 kv[kRowsInFlight], vv[kRowsInFlight];
+#pragma unroll
+                for (int j = 0; j < kRowsInFlight; ++j) {
+                    const int i = i0 + j * kGroups;
+                    if (i < cnt) {
+                        const int64_t src = (head_row0 + src_tok[i]) * row_units + u0;
+                        kv[j] = __ldg(K + src);
+                        vv[j] = __ldg(V + src);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < kRowsInFlight; ++j) {
+                    const int i = i0 + j * kGroups;
+                    if (i < cnt) {
+                        const int64_t d = dst_row[i] * row_units + u0;
+                        K_out[d] = kv[j];
+                        V_out[d] = vv[j];
+                    }
+                }
+            }
+        }
+        running += cnt;
+        base_cur = base_next_s;
+        __syncthreads();
+    }
+}
+
 }  // namespace kvzap

@@ -147,6 +147,28 @@ __device__ __forceinline__ void mlp_columns(const uint32_t (&r)[32], int j0, con
     }
 }
 
+// Issues the MMAs of one 64-element K block: kBlockK / kUmmaK steps times kChunks accumulator chunks,
+// fully unrolled, descriptors formed by adding constants to the low word (the start-address field).
+// a_lo / b_lo: low descriptor words of the stage's A tile and first B chunk; `first` = this is the
+// first K block of the accumulation (its first step overwrites the accumulator).
+template <bool kPair, int kChunks>
+__device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                              uint32_t b_chunk_step, uint32_t chunk_n, uint32_t idesc, bool first)
+{
+#pragma unroll
+    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+#pragma unroll
+        for (int c = 0; c < kChunks; ++c) {
+            // advancing K by 16 elements = 32 bytes = 2 units of the 16-byte address field
+            const uint64_t a_desc = (static_cast<uint64_t>(desc_hi) << 32) | (a_lo + 2 * k);
+            const uint64_t b_desc = (static_cast<uint64_t>(desc_hi) << 32) | (b_lo + c * b_chunk_step + 2 * k);
+            const uint32_t acc = (k != 0 || !first) ? 1u : 0u;
+            if constexpr (kPair) umma_bf16_pair(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+            else umma_bf16(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+        }
+    }
+}
+
 template <bool kMlp, bool kPair>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -235,11 +257,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                 for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                     const uint32_t s = it % p.n_stages;
                     const uint32_t round = it / p.n_stages;
-                    int got = 0;
-                    if (lane == 0) got = mbar_wait(bar_empty + 8 * s, (round & 1u) ^ 1u, abort_flag) ? 1 : 0;
-                    got = __shfl_sync(0xffffffffu, got, 0);
-                    if (!got) { ok = false; break; }
-                    if (lane == 0) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, (round & 1u) ^ 1u, abort_flag))) {
+                        ok = false;
+                        break;
+                    }
+                    if (elect_one()) {
                         const uint32_t sa = smem_base + s * L.stage_bytes;
                         const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w;
                         if constexpr (kPair) {
@@ -285,56 +307,54 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         // ------------------------------------------------------------ MMA issuer (a pair: its first CTA only)
         if (leader) {
             const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.chunk_n));
+            // operand descriptors: constant high word, low word = (address >> 4) | fixed fields
+            const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
+            const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
+            const uint32_t desc_lo0 = static_cast<uint32_t>(desc0);
+            const uint32_t b_chunk_step = static_cast<uint32_t>(b_rows_chunk * kBlockK * 2) >> 4;
             uint32_t it = 0, acc_it = 0;
             bool ok = true;
             for (int tile = unit; tile < p.n_tiles && ok; tile += n_units) {
                 for (int g = 0; g < p.n_groups && ok; ++g, ++acc_it) {
                     const uint32_t buf = acc_it % p.acc_bufs;
                     const uint32_t use = acc_it / p.acc_bufs;
-                    int got = 0;
-                    if (lane == 0) got = mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag) ? 1 : 0;
-                    got = __shfl_sync(0xffffffffu, got, 0);
-                    if (!got) { ok = false; break; }
+                    // every lane waits (no broadcast needed afterwards); one elected lane issues
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar_tempty + 8 * buf, (use & 1u) ^ 1u, abort_flag))) {
+                        ok = false;
+                        break;
+                    }
                     tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + buf * p.acc_stride;
                     for (int kb = 0; kb < k_blocks; ++kb, ++it) {
                         const uint32_t s = it % p.n_stages;
                         const uint32_t round = it / p.n_stages;
-                        if (lane == 0) got = mbar_wait(bar_full + 8 * s, round & 1u, abort_flag) ? 1 : 0;
-                        got = __shfl_sync(0xffffffffu, got, 0);
-                        if (!got) { ok = false; break; }
+                        if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, round & 1u, abort_flag))) {
+                            ok = false;
+                            break;
+                        }
                         tc_fence_after_sync();
-                        if (lane == 0) {
-                            const uint32_t sa = smem_base + s * L.stage_bytes;
-                            const uint64_t a_desc = umma_desc_k_major_sw128(sa);
-#pragma unroll
-                            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                                // advancing K by 16 elements = 32 bytes = 2 descriptor address units
-                                for (int c = 0; c < p.n_chunks; ++c) {
-                                    const uint64_t b_desc =
-                                        umma_desc_k_major_sw128(sa + kATileBytes + c * b_rows_chunk * kBlockK * 2);
-                                    if constexpr (kPair)
-                                        umma_bf16_pair(d_tmem + c * p.chunk_n, a_desc + 2 * k, b_desc + 2 * k, idesc,
-                                                       (kb | k) != 0 ? 1u : 0u);
-                                    else
-                                        umma_bf16(d_tmem + c * p.chunk_n, a_desc + 2 * k, b_desc + 2 * k, idesc,
-                                                  (kb | k) != 0 ? 1u : 0u);
-                                }
-                            }
+                        if (elect_one()) {
+                            const uint32_t a_lo = desc_lo0 + ((s * L.stage_bytes) >> 4);
+                            const uint32_t b_lo = a_lo + (kATileBytes >> 4);
+                            if (p.n_chunks == 1)
+                                issue_k_block<kPair, 1>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
+                            else
+                                issue_k_block<kPair, 2>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
                             // the stage is free (in both CTAs) once these MMAs retire
                             if constexpr (kPair) umma_commit_pair(bar_empty + 8 * s, 3);
                             else umma_commit(bar_empty + 8 * s);
                         }
                         __syncwarp();
                     }
-                    if (ok && lane == 0) {                   // accumulator complete
+                    if (ok && elect_one()) {                 // accumulator complete
                         if constexpr (kPair) umma_commit_pair(bar_tfull + 8 * buf, 3);
                         else umma_commit(bar_tfull + 8 * buf);
                     }
                     __syncwarp();
                 }
             }
-            if (!ok && lane == 0) {
+            __syncwarp();
+            if (!ok && elect_one()) {
                 // abort path: wait (bounded) for the MMAs already issued before TMEM is freed
                 if constexpr (kPair) umma_commit_pair(bar_done, 1);
                 else umma_commit(bar_done);
