@@ -24,6 +24,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 static char g_create_error[512] = "";
 
+// Mask slices used in rotation.  A scoring kernel may start while the compaction of the call before it
+// is still running (see launch_score); that compaction reads the previous slice, never the current one.
+constexpr int kMaskRing = 4;
+
 }  // namespace kvzap
 
 struct kvzap_ctx {
@@ -47,7 +51,10 @@ struct kvzap_ctx {
     kvzap::EncodeTiledFn encode = nullptr;
     // scratch
     int64_t max_blocks = 0, max_words = 0;
-    uint32_t *maskbits = nullptr;    // [H][max_words]
+    uint32_t *maskbits = nullptr;    // [kMaskRing][H][max_words]: consecutive calls use different slices
+    uint64_t mask_turn = 0;
+    const void *last_scores = nullptr;   // scores buffer of the previous scoring launch, and its size
+    size_t last_scores_bytes = 0;
     int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
     int32_t *seqbase = nullptr;      // [H][max_seqs + 1]
     int32_t *list_page0 = nullptr;   // [max_seqs * H] first page of each list (paged output)
@@ -192,12 +199,55 @@ static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seq
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+static uint32_t *next_mask_slice(kvzap_ctx *ctx)
+{
+    uint32_t *m = ctx->maskbits + (ctx->mask_turn % kMaskRing) * ctx->max_words * ctx->cfg.n_kv_heads;
+    ctx->mask_turn += 1;
+    return m;
+}
+
+// Fills a launch configuration; `early` adds the attribute that lets the kernel start before the
+// kernel ahead of it in the stream has finished (programmatic dependent launch), `cluster` > 1 the
+// cluster dimension.  `attrs` must have room for two attributes.
+static void make_launch(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attrs, dim3 grid, dim3 block, size_t smem,
+                        cudaStream_t stream, bool early, int cluster)
+{
+    memset(cfg, 0, sizeof *cfg);
+    cfg->gridDim = grid;
+    cfg->blockDim = block;
+    cfg->dynamicSmemBytes = smem;
+    cfg->stream = stream;
+    int n = 0;
+    if (cluster > 1) {
+        attrs[n].id = cudaLaunchAttributeClusterDimension;
+        attrs[n].val.clusterDim.x = static_cast<unsigned>(cluster);
+        attrs[n].val.clusterDim.y = 1;
+        attrs[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    if (early) {
+        attrs[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attrs[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg->attrs = attrs;
+    cfg->numAttrs = static_cast<unsigned>(n);
+}
+
 // Launches the scoring kernel over layers [layer, layer + n_layers); hidden is [n_layers][n_tokens][d_model],
 // scores [n_layers][n_tokens][H]; maskbits != nullptr fuses the threshold/window test.
 static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
                                  float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1)
 {
+    // Early start.  When the grid fills the machine (one CTA per SM), this kernel is allowed to start
+    // while the kernels ahead of it in the stream -- the previous call's scoring kernel finishing its
+    // last tiles, and its compaction -- are still running: its CTAs take the SMs as they become free.
+    // That is safe because (a) it reads only hidden states and weights, which none of this library's
+    // kernels write, (b) every scoring CTA waits for the kernel ahead of it before it exits, so a
+    // free SM implies that everything two launches back has completed, and the mask slice written
+    // here was last read at least kMaskRing launches back, (c) the scores buffer is checked below.
+    // A smaller grid is launched the ordinary way.
     const kvzap_config &c = ctx->cfg;
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
     // CTA pairs pay off once a layer has at least two 128-token blocks; a pair's work tile is 256 tokens
@@ -241,30 +291,32 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.window_keep = window_keep;
     p.tau = tau;
     p.status = ctx->status_dev;
+    const size_t scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
+    bool scores_clash = false;           // the previous launch may still be writing the same buffer
+    if (scores && ctx->last_scores) {
+        const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
+        scores_clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + scores_bytes;
+    }
+    ctx->last_scores = scores;
+    ctx->last_scores_bytes = scores_bytes;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
         if (pair) {
             const int n_clusters = static_cast<int>(n_tiles < ctx->pair_clusters ? n_tiles : ctx->pair_clusters);
-            cudaLaunchConfig_t cfg;
-            memset(&cfg, 0, sizeof cfg);
-            cfg.gridDim = dim3(static_cast<unsigned>(2 * n_clusters));
-            cfg.blockDim = dim3(kScoreThreads);
-            cfg.dynamicSmemBytes = sc.smem;
-            cfg.stream = stream;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeClusterDimension;
-            attr[0].val.clusterDim.x = 2;
-            attr[0].val.clusterDim.y = 1;
-            attr[0].val.clusterDim.z = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
+            const bool early = !ctx->profiling && !scores_clash && 2 * n_clusters >= ctx->sm_count / 2 * 2;
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(2 * n_clusters)), dim3(kScoreThreads), sc.smem, stream,
+                        early, 2);
             KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, true>, tmap_x, sc.tmap_w, p));
         } else {
             const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
+            const bool early = !ctx->profiling && !scores_clash && grid >= ctx->sm_count;
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid)), dim3(kScoreThreads), sc.smem, stream, early, 1);
             if (c.hidden > 0)
-                score_kernel<true, false><<<grid, kScoreThreads, sc.smem, stream>>>(tmap_x, sc.tmap_w, p);
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, false>, tmap_x, sc.tmap_w, p));
             else
-                score_kernel<false, false><<<grid, kScoreThreads, sc.smem, stream>>>(tmap_x, sc.tmap_w, p);
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<false, false>, tmap_x, sc.tmap_w, p));
         }
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
@@ -272,31 +324,34 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     return KVZAP_OK;
 }
 
-// scan + compaction over mask words already in ctx->maskbits
-static kvzap_status launch_compaction(kvzap_ctx *ctx, const void *K, const void *V, const int32_t *cu_seqlens,
-                                      int32_t n_seqs, int64_t n_tokens, void *K_out, void *V_out, int32_t *lengths,
-                                      cudaStream_t stream)
+// Dense-ragged compaction over the mask words in `mask` (one kernel, no scan pass).
+static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, void *K_out,
+                                      void *V_out, int32_t *lengths, cudaStream_t stream)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     const int64_t n_words = n_blocks * 4;
-    {
-        ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
-        scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
-                                            n_tokens, ctx->blockprefix, ctx->seqbase, lengths, 0, 0, 0, 0, nullptr,
-                                            nullptr, nullptr, nullptr, ctx->status_dev);
-    }
-    KVZAP_CUDA(ctx, cudaGetLastError());
-    const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
+    // A grid that is resident all at once, next to the scoring kernel's CTAs: the MLP scoring kernel
+    // leaves registers for two of these CTAs per SM, the Linear one for several.
+    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (c.hidden > 0 ? 2 : 6);
+    int64_t chunks = max_ctas / c.n_kv_heads;
+    if (chunks < 1) chunks = 1;
+    if (chunks > n_blocks) chunks = n_blocks;
+    const int blocks_per_cta = static_cast<int>((n_blocks + chunks - 1) / chunks);
+    chunks = (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
-        compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
-            static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
-            static_cast<uint4 *>(V_out), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
-            n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, 0, nullptr);
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(chunks), static_cast<unsigned>(c.n_kv_heads)),
+                    dim3(kDenseThreads), 0, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel, static_cast<const uint4 *>(K),
+                                           static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
+                                           static_cast<uint4 *>(V_out), mask, n_words, n_blocks, blocks_per_cta,
+                                           cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths));
     }
-    KVZAP_CUDA(ctx, cudaGetLastError());
-    ctx->launches += 2;
+    ctx->launches += 1;
     return KVZAP_OK;
 }
 
@@ -434,6 +489,20 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
                                          static_cast<int>(ctx->sched[0].smem)));
     }
 
+    // Kernels share an SM only if they ask for the same split of the L1 / shared-memory array; the
+    // scoring kernels need the largest shared-memory split, so the compaction asks for it too.
+    CREATE_CUDA(cudaFuncSetAttribute(compact_dense_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    if (c.hidden > 0) {
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    } else {
+        CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    }
+
     ctx->layer_set.assign(c.n_layers, 0);
     {
         const size_t w1_bytes = static_cast<size_t>(c.n_layers) * ctx->w1_rows * c.d_model * 2;
@@ -459,7 +528,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     }
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
     ctx->max_words = ctx->max_blocks * 4;
-    CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * ctx->max_words * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * kMaskRing * ctx->max_words * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
@@ -555,15 +624,16 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     if (st != KVZAP_OK) return st;
     if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    uint32_t *mask = next_mask_slice(ctx);
     {
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
         mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
-                                                                         cu_seqlens, n_seqs, tau, w, 1, ctx->maskbits,
+                                                                         cu_seqlens, n_seqs, tau, w, 1, mask,
                                                                          n_blocks * 4);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
-    return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
 }
 
 kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
@@ -586,9 +656,10 @@ kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidd
     st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
     if (st != KVZAP_OK) return st;
     if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
-    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
+    uint32_t *mask = next_mask_slice(ctx);
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
-    return launch_compaction(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
 }
 
 kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
@@ -815,7 +886,8 @@ struct kvzap_cache {
 
 namespace kvzap {
 
-static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const void *K, const void *V, const int32_t *cu_seqlens,
+static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
+                                            const int32_t *cu_seqlens,
                                             int32_t n_seqs, int64_t n_tokens, void *K_pool, void *V_pool,
                                             int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
                                             int32_t *page_table, int32_t max_pages, int32_t *lengths,
@@ -827,7 +899,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const void *K, const
     const int64_t n_words = n_blocks * 4;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
-        scan_kernel<<<1, 1024, 0, stream>>>(ctx->maskbits, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
+        scan_kernel<<<1, 1024, 0, stream>>>(mask, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
                                             n_tokens, ctx->blockprefix, ctx->seqbase, lengths, page_tokens, first_page,
                                             n_pages_pool, max_pages, ctx->list_page0, page_table, n_pages_used,
                                             page_cursor, ctx->status_dev);
@@ -838,7 +910,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const void *K, const
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
         compact_kernel<true><<<grid, kCompactThreads, 0, stream>>>(
             static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_pool),
-            static_cast<uint4 *>(V_pool), ctx->maskbits, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
+            static_cast<uint4 *>(V_pool), mask, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
             n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, page_tokens, ctx->list_page0);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
@@ -888,15 +960,16 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
     if (st != KVZAP_OK) return st;
     if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    uint32_t *mask = next_mask_slice(ctx);
     {
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
         mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
-                                                                         cu_seqlens, n_seqs, tau, w, 1, ctx->maskbits,
+                                                                         cu_seqlens, n_seqs, tau, w, 1, mask,
                                                                          n_blocks * 4);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
-    return launch_compaction_paged(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
+    return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
                                    first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
 }
 
@@ -924,9 +997,10 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
                           max_pages_per_list, lengths, n_pages_used, w);
     if (st != KVZAP_OK) return st;
     if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
-    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, cu_seqlens, n_seqs, tau, w, stream);
+    uint32_t *mask = next_mask_slice(ctx);
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
-    return launch_compaction_paged(ctx, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
+    return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
                                    first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
 }
 
@@ -1088,9 +1162,10 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     DeviceGuard guard(c.device);
     const int64_t li0 = (static_cast<int64_t>(seq) * v.n_layers + layer) * v.n_heads;
     // mask = threshold only, the window's tokens left out: they go to the ring below
-    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, ctx->maskbits, nullptr, 1, tau, v.window, stream, 0);
+    uint32_t *mask = next_mask_slice(ctx);
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, nullptr, 1, tau, v.window, stream, 0);
     if (st != KVZAP_OK) return st;
-    st = launch_compaction_paged(ctx, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
+    st = launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
                                  v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
                                  v.page_cursor);
     if (st != KVZAP_OK) return st;

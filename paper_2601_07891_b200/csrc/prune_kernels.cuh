@@ -294,7 +294,7 @@ compact_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *
 // in progress there), then walks its blocks keeping a running count, so that every kept row's
 // slot in its (sequence, head) list is known without any other CTA's help.  lengths[b,h] is
 // written by the thread that handles the last token of sequence b; empty sequences by chunk 0.
-constexpr int kDenseThreads = 256;
+constexpr int kDenseThreads = 128;     // = kBlockTokens: one thread ranks one token; small enough to sit beside a scoring CTA
 
 // bits of the block's four words below in-block position r (0..128)
 __device__ __forceinline__ int popc_below(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, int r)
@@ -326,6 +326,11 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     const int64_t blk1 = blk0 + blocks_per_cta < n_blocks ? blk0 + blocks_per_cta : n_blocks;
     const bool multi = cu_seqlens != nullptr && n_seqs > 1;
     const uint32_t *words = maskbits + static_cast<int64_t>(h) * n_words;
+
+    // This grid is small enough to be resident all at once: the next kernel in the stream may be
+    // placed as soon as it is; the mask itself is read only after the kernel ahead has completed.
+    griddep_launch_dependents();
+    griddep_wait();
 
     if (blockIdx.x == 0 && cu_seqlens != nullptr)         // empty sequences have no last token to write for them
         for (int b = tid; b < n_seqs; b += kDenseThreads)

@@ -214,6 +214,16 @@ __device__ __forceinline__ void reg_fence32(uint32_t (&r)[32])
                  : "memory");
 }
 
+__device__ __forceinline__ void reg_fence16(uint32_t (&r)[16])
+{
+    asm volatile(""
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                   "+r"(r[15])
+                 :
+                 : "memory");
+}
+
 // Shared-memory operand descriptor for a K-major bf16 tile whose rows are 128 bytes
 // (64 elements) wide, written by TMA with the 128-byte swizzle; the tile base is
 // 1024-byte aligned and 8-row groups follow each other every 1024 bytes.
@@ -235,6 +245,20 @@ __host__ __device__ __forceinline__ uint32_t umma_idesc_bf16_f32(uint32_t M, uin
            | (1u << 10)         // B bf16
            | ((N >> 3) << 17)   // N / 8
            | ((M >> 4) << 24);  // M / 16
+}
+
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start once every CTA
+// of the kernel before it in the stream has executed griddep_launch_dependents() (or exited);
+// griddep_wait() then blocks until that earlier kernel has completed and its writes are visible.
+// Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void griddep_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void griddep_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ---------------------------------------------------------------- CTA pairs (cluster of two)

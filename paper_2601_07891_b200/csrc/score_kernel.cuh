@@ -125,14 +125,15 @@ __device__ __forceinline__ int seq_of_token(const int32_t *cu, int n_seqs, int64
     return lo;
 }
 
-// Second layer for 32 accumulator columns j0 .. j0+31 of one token: acc[h] (+)= GELU(r + b1) . W2.
+// Second layer for kCols accumulator columns j0 .. j0+kCols-1 of one token: acc[h] (+)= GELU(r + b1) . W2.
 // Hidden units are taken two at a time; acc[h] holds the partial sums of the even and of the odd
 // units of head h.  w2p is W2 repacked as [j / 2][h] pairs {W2[h][j], W2[h][j+1]}.
-__device__ __forceinline__ void mlp_columns(const uint32_t (&r)[32], int j0, const float *b1s, const ulonglong2 *w2p,
+template <int kCols>
+__device__ __forceinline__ void mlp_columns(const uint32_t (&r)[kCols], int j0, const float *b1s, const ulonglong2 *w2p,
                                             uint64_t (&acc)[kMaxHeads])
 {
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
+    for (int i = 0; i < kCols; i += 2) {
         const int j = j0 + i;
         const float2 b = *reinterpret_cast<const float2 *>(b1s + j);
         const uint64_t z2 = f2_add(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), f2_pack(b.x, b.y));
@@ -169,8 +170,11 @@ __device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint32_t a_lo, ui
     }
 }
 
+// At most 128 registers per thread: the register file is split over the SM's four schedulers, three
+// of this kernel's ten warps share one of them, and a warp of the compaction kernel must still fit
+// beside them for the two kernels to run on the same SM at the same time.
 template <bool kMlp, bool kPair>
-__global__ void __launch_bounds__(kScoreThreads, 1)
+__global__ void __maxnreg__(128)
 score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
              const ScoreParams p)
 {
@@ -200,6 +204,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 72);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 76);
 
+    // Let the kernel behind this one in the stream (the compaction) be placed right away; it waits
+    // for this kernel's results itself.
+    griddep_launch_dependents();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     constexpr int kEpiWarps = kMlp ? 8 : 4;
@@ -422,20 +429,18 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         const int half_w = p.group_w >> 1;
                         const int col0 = hsel * half_w;
                         const int j0 = g * p.group_w + col0;
-                        // two register sets: the next 32 columns are in flight while these are processed
-                        uint32_t ra[32], rb[32];
-                        tmem_ld_x32(t_row + col0, ra);
-                        for (int c = 0; c < half_w; c += 64) {
+                        // two register sets: the next 16 columns are in flight while these are processed
+                        uint32_t ra[16], rb[16];
+                        tmem_ld_x16(t_row + col0, ra);
+                        for (int c = 0; c < half_w; c += 32) {
                             tmem_wait_ld();
-                            reg_fence32(ra);
-                            if (c + 32 < half_w) tmem_ld_x32(t_row + col0 + c + 32, rb);
-                            mlp_columns(ra, j0 + c, b1s, w2p, acc);
-                            if (c + 32 < half_w) {
-                                tmem_wait_ld();
-                                reg_fence32(rb);
-                                if (c + 64 < half_w) tmem_ld_x32(t_row + col0 + c + 64, ra);
-                                mlp_columns(rb, j0 + c + 32, b1s, w2p, acc);
-                            }
+                            reg_fence16(ra);
+                            tmem_ld_x16(t_row + col0 + c + 16, rb);
+                            mlp_columns<16>(ra, j0 + c, b1s, w2p, acc);
+                            tmem_wait_ld();
+                            reg_fence16(rb);
+                            if (c + 32 < half_w) tmem_ld_x16(t_row + col0 + c + 32, ra);
+                            mlp_columns<16>(rb, j0 + c + 16, b1s, w2p, acc);
                         }
                     } else {
                         uint32_t r[16];
@@ -529,6 +534,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     // memory, signal its barriers or write its accumulator
     if constexpr (kPair) cluster_sync_all();
     if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+    // If this kernel was allowed to start before the one ahead of it had finished, no CTA leaves
+    // before that kernel is complete: kernels then still complete in stream order, and a CTA of the
+    // next scoring kernel that finds this SM free knows that everything two launches back is done.
+    if (threadIdx.x == 0) griddep_wait();
     if (warp == 1) {
         tc_fence_after_sync();
         if constexpr (kPair) tmem_dealloc_pair(tmem_base, static_cast<uint32_t>(p.tmem_cols));
