@@ -53,6 +53,8 @@ struct kvzap_ctx {
     int64_t max_blocks = 0, max_words = 0;
     uint32_t *maskbits = nullptr;    // [kMaskRing][H][max_words]: consecutive calls use different slices
     uint64_t mask_turn = 0;
+    int32_t *tile_counters = nullptr;    // [kMaskRing] work-tile counters of the scoring launches, used in rotation
+    uint64_t score_turn = 0;
     const void *last_scores = nullptr;   // scores buffer of the previous scoring launch, and its size
     size_t last_scores_bytes = 0;
     int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
@@ -171,6 +173,7 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->w2t_all);
     cudaFree(ctx->b2_all);
     cudaFree(ctx->maskbits);
+    cudaFree(ctx->tile_counters);
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
     cudaFree(ctx->list_page0);
@@ -291,6 +294,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.window_keep = window_keep;
     p.tau = tau;
     p.status = ctx->status_dev;
+    // every launch finds its counter at zero: it was cleared by the launch before the previous one
+    p.tile_counter = ctx->tile_counters + ctx->score_turn % kMaskRing;
+    p.tile_counter_reset = ctx->tile_counters + (ctx->score_turn + 2) % kMaskRing;
+    ctx->score_turn += 1;
     const size_t scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
     bool scores_clash = false;           // the previous launch may still be writing the same buffer
     if (scores && ctx->last_scores) {
@@ -532,6 +539,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->tile_counters, sizeof(int32_t) * kMaskRing));
+    CREATE_CUDA(cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
     CREATE_CUDA(cudaMallocHost(&ctx->status_host, sizeof(int32_t)));
@@ -672,6 +681,9 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
     const int32_t v = *ctx->status_host;
     if (v == 0) return KVZAP_OK;
+    // a scoring kernel that gave up may have left its work-tile counter in an unknown state
+    cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing, stream);
+    cudaStreamSynchronize(stream);
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
 }

@@ -67,6 +67,8 @@ struct ScoreParams {
     int32_t window_keep;  // 1: tokens inside the window are kept (Algorithm 1); 0: they are left out of the mask
     float tau;
     int32_t *status;      // device status word
+    int32_t *tile_counter;        // work tiles handed out beyond the first one of every CTA (or pair); starts at 0
+    int32_t *tile_counter_reset;  // the counter of the launch after next: set to 0 by this launch
 };
 
 // Byte offsets inside the dynamic shared memory block (after 1024-byte alignment).
@@ -83,7 +85,7 @@ __host__ __device__ inline ScoreSmemLayout score_smem_layout(int b_rows, int n_s
     L.b1s = L.w2s + static_cast<uint32_t>(n_hidden) * kMaxHeads * 4;
     L.part = L.b1s + static_cast<uint32_t>(n_hidden) * 4;
     L.bars = L.part + kTileM * kMaxHeads * 4;
-    L.total = L.bars + 256;
+    L.total = L.bars + 512;
     return L;
 }
 
@@ -203,6 +205,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     const uint32_t bar_epi = bar_pempty + 8;             // [1] MLP: all epilogue warps (weight reload)
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 72);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 76);
+    // Work tiles are handed out at run time (see the producer warp): a ring of tile numbers with its own
+    // full / empty barriers carries them to the other warps of the CTA (and of the pair's second CTA).
+    constexpr uint32_t kSchedSlots = 4;
+    const uint32_t bar_sfull = bars + 16 * kMaxStages + 80;      // [kSchedSlots] scheduler -> consumers
+    const uint32_t bar_sempty = bar_sfull + 8 * kSchedSlots;     // [kSchedSlots] consumers -> scheduler (first CTA's)
+    volatile int32_t *tile_ring = reinterpret_cast<volatile int32_t *>(smem + L.bars + 16 * kMaxStages + 80 + 16 * kSchedSlots);
+    const uint32_t tile_ring_addr = bars + 16 * kMaxStages + 80 + 16 * kSchedSlots;
 
     // Let the kernel behind this one in the stream (the compaction) be placed right away; it waits
     // for this kernel's results itself.
@@ -229,6 +238,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         mbar_init(bar_pfull, 4);
         mbar_init(bar_pempty, 4);
         mbar_init(bar_epi, kEpiWarps);
+        // consumers of a tile number: the second CTA's producer warp, the MMA warp, every epilogue warp
+        for (uint32_t i = 0; i < kSchedSlots; ++i) {
+            mbar_init(bar_sfull + 8 * i, 1);
+            mbar_init(bar_sempty + 8 * i, (kCtas - 1) + 1 + kEpiWarps * kCtas);
+        }
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
@@ -250,14 +264,56 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
 
     const int k_blocks = p.d_model / kBlockK;
+    if (blockIdx.x == 0 && threadIdx.x == 0) *p.tile_counter_reset = 0;
+
+    // The seq-th work tile of this CTA (pair), as published by the scheduler; -1 if the kernel is
+    // aborting.  Called by all lanes of a warp; values >= p.n_tiles mean "no more work".
+    uint32_t sempty_addr = bar_sempty;
+    if constexpr (kPair) sempty_addr = map_to_cta(bar_sempty, 0);
+    auto sched_get = [&](uint32_t seq) -> int {
+        const uint32_t slot = seq % kSchedSlots;
+        if (!__all_sync(0xffffffffu, mbar_wait_cluster(bar_sfull + 8 * slot, (seq / kSchedSlots) & 1u, abort_flag)))
+            return -1;
+        const int t = tile_ring[slot];
+        __syncwarp();
+        if (lane == 0) {
+            if constexpr (kPair) mbar_arrive_cluster(sempty_addr + 8 * slot);
+            else mbar_arrive(bar_sempty + 8 * slot);
+        }
+        return t;
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
         const uint64_t pol_x = l2_policy_evict_first();   // hidden states are streamed once
         const uint64_t pol_w = l2_policy_evict_last();    // weights are re-read by every tile
-        uint32_t it = 0;
+        uint32_t it = 0, seq = 0;
         bool ok = true;
-        for (int tile = unit; tile < p.n_tiles && ok; tile += n_units) {
+        // The first CTA's producer warp is also the scheduler: every CTA (pair) starts with the tile of
+        // its own index and takes further ones from a global counter, so that CTAs that start early
+        // (on SMs the previous launch left first) end up with more tiles than those that start late.
+        auto publish = [&](uint32_t q, int t) -> bool {
+            const uint32_t slot = q % kSchedSlots;
+            if (q >= kSchedSlots &&
+                !__all_sync(0xffffffffu, mbar_wait_cluster(bar_sempty + 8 * slot, ((q / kSchedSlots) & 1u) ^ 1u, abort_flag)))
+                return false;
+            if (lane == 0) {
+                tile_ring[slot] = t;
+                mbar_arrive(bar_sfull + 8 * slot);
+                if constexpr (kPair) {
+                    st_shared_cluster_u32(map_to_cta(tile_ring_addr + 4 * slot, 1), static_cast<uint32_t>(t));
+                    mbar_arrive_cluster(map_to_cta(bar_sfull + 8 * slot, 1));
+                }
+            }
+            __syncwarp();
+            return true;
+        };
+        int tile = unit;
+        if (leader) ok = publish(0, tile);
+        else tile = sched_get(0);
+        while (ok && tile >= 0 && tile < p.n_tiles) {
+            int tile_next = 0;
+            if (leader && lane == 0) tile_next = n_units + atomicAdd(p.tile_counter, 1);   // used after this tile's loads
             const int l_rel = tile / p.tiles_per_layer;
             const int m_tile = (tile - l_rel * p.tiles_per_layer) * kCtas + static_cast<int>(cta_rank);
             for (int g = 0; g < p.n_groups && ok; ++g) {
@@ -292,7 +348,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     __syncwarp();
                 }
             }
+            if (!ok) break;
+            ++seq;
+            if (leader) {
+                tile_next = __shfl_sync(0xffffffffu, tile_next, 0);
+                ok = publish(seq, tile_next);
+                tile = tile_next;
+            } else {
+                tile = sched_get(seq);
+            }
         }
+        if (tile < 0) ok = false;
         if (!ok && lane == 0) {
             // abort path: let the copies already in flight land before the CTA exits
             if (leader) {
@@ -321,7 +387,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             const uint32_t b_chunk_step = static_cast<uint32_t>(b_rows_chunk * kBlockK * 2) >> 4;
             uint32_t it = 0, acc_it = 0;
             bool ok = true;
-            for (int tile = unit; tile < p.n_tiles && ok; tile += n_units) {
+            for (uint32_t seq = 0; ok; ++seq) {
+                const int tile = sched_get(seq);
+                if (tile < 0) { ok = false; break; }
+                if (tile >= p.n_tiles) break;
                 for (int g = 0; g < p.n_groups && ok; ++g, ++acc_it) {
                     const uint32_t buf = acc_it % p.acc_bufs;
                     const uint32_t use = acc_it / p.acc_bufs;
@@ -386,7 +455,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             tempty_addr[1] = map_to_cta(bar_tempty + 8, 0);
         }
         if (active) {
-            for (int tile = unit; tile < p.n_tiles && ok; tile += n_units, ++tile_it) {
+            for (uint32_t seq = 0; ok; ++seq, ++tile_it) {
+                const int tile = sched_get(seq);
+                if (tile < 0) { ok = false; break; }
+                if (tile >= p.n_tiles) break;
                 const int l_rel = tile / p.tiles_per_layer;
                 const int m_tile = (tile - l_rel * p.tiles_per_layer) * kCtas + static_cast<int>(cta_rank);
                 const int layer = p.layer0 + l_rel;
