@@ -287,7 +287,13 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
         const uint64_t pol_x = l2_policy_evict_first();   // hidden states are streamed once
         const uint64_t pol_w = l2_policy_evict_last();    // weights are re-read by every tile
+        uint32_t full0_cluster = bar_full;                // the pair's first CTA's full barriers
+        if constexpr (kPair) full0_cluster = map_to_cta(bar_full, 0);
+        // Ring position kept incrementally (stage index, its shared-memory address, the parity to wait
+        // for): the loop body is a chain of dependent instructions in one warp, so every one counts.
         uint32_t it = 0, seq = 0;
+        uint32_t st = 0, st_par = 1, st_addr = smem_base;       // empty barriers: the first pass is free
+        const bool elected = elect_one();
         bool ok = true;
         // The first CTA's producer warp is also the scheduler: every CTA (pair) starts with the tile of
         // its own index and takes further ones from a global counter, so that CTAs that start early
@@ -316,36 +322,37 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             if (leader && lane == 0) tile_next = n_units + atomicAdd(p.tile_counter, 1);   // used after this tile's loads
             const int l_rel = tile / p.tiles_per_layer;
             const int m_tile = (tile - l_rel * p.tiles_per_layer) * kCtas + static_cast<int>(cta_rank);
+            const int row0 = m_tile * kTileM;
             for (int g = 0; g < p.n_groups && ok; ++g) {
-                for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-                    const uint32_t s = it % p.n_stages;
-                    const uint32_t round = it / p.n_stages;
-                    if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * s, (round & 1u) ^ 1u, abort_flag))) {
+                const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w + static_cast<int>(cta_rank) * b_rows_chunk;
+                for (int kx = 0; kx < p.d_model; kx += kBlockK, ++it) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
                         ok = false;
                         break;
                     }
-                    if (elect_one()) {
-                        const uint32_t sa = smem_base + s * L.stage_bytes;
-                        const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w;
+                    if (elected) {
+                        const uint32_t sa = st_addr;
                         if constexpr (kPair) {
                             // the first CTA's barrier counts the bytes of both CTAs
-                            if (leader) mbar_arrive_expect_tx(bar_full + 8 * s, L.stage_bytes * 2);
-                            const uint32_t bar = map_to_cta(bar_full + 8 * s, 0);
-                            tma_load_3d_pair(sa, &tmap_x, bar, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
-                            for (int c = 0; c < p.n_chunks; ++c)
-                                tma_load_2d_pair(sa + kATileBytes + c * b_rows_chunk * kBlockK * 2, &tmap_w, bar,
-                                                 kb * kBlockK,
-                                                 w_row0 + c * p.chunk_n + static_cast<int>(cta_rank) * b_rows_chunk,
-                                                 pol_w);
+                            if (leader) mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes * 2);
+                            const uint32_t bar = full0_cluster + 8 * st;
+                            tma_load_3d_pair(sa, &tmap_x, bar, kx, row0, l_rel, pol_x);
+                            tma_load_2d_pair(sa + kATileBytes, &tmap_w, bar, kx, w_row0, pol_w);
+                            if (p.n_chunks == 2)
+                                tma_load_2d_pair(sa + kATileBytes + b_rows_chunk * kBlockK * 2, &tmap_w, bar, kx,
+                                                 w_row0 + p.chunk_n, pol_w);
                         } else {
-                            mbar_arrive_expect_tx(bar_full + 8 * s, L.stage_bytes);
-                            tma_load_3d(sa, &tmap_x, bar_full + 8 * s, kb * kBlockK, m_tile * kTileM, l_rel, pol_x);
-                            for (int c = 0; c < p.n_chunks; ++c)
-                                tma_load_2d(sa + kATileBytes + c * p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * s,
-                                            kb * kBlockK, w_row0 + c * p.chunk_n, pol_w);
+                            mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes);
+                            tma_load_3d(sa, &tmap_x, bar_full + 8 * st, kx, row0, l_rel, pol_x);
+                            tma_load_2d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, kx, w_row0, pol_w);
+                            if (p.n_chunks == 2)
+                                tma_load_2d(sa + kATileBytes + p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * st, kx,
+                                            w_row0 + p.chunk_n, pol_w);
                         }
                     }
                     __syncwarp();
+                    st_addr += L.stage_bytes;
+                    if (++st == static_cast<uint32_t>(p.n_stages)) { st = 0; st_par ^= 1u; st_addr = smem_base; }
                 }
             }
             if (!ok) break;
@@ -385,7 +392,10 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
             const uint32_t desc_lo0 = static_cast<uint32_t>(desc0);
             const uint32_t b_chunk_step = static_cast<uint32_t>(b_rows_chunk * kBlockK * 2) >> 4;
-            uint32_t it = 0, acc_it = 0;
+            const uint32_t stage_units = L.stage_bytes >> 4;
+            const bool elected = elect_one();               // the same lane issues every MMA and commit
+            uint32_t acc_it = 0;
+            uint32_t st = 0, st_par = 0, a_lo = desc_lo0;    // ring position, kept incrementally
             bool ok = true;
             for (uint32_t seq = 0; ok; ++seq) {
                 const int tile = sched_get(seq);
@@ -401,28 +411,27 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     }
                     tc_fence_after_sync();
                     const uint32_t d_tmem = tmem_base + buf * p.acc_stride;
-                    for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-                        const uint32_t s = it % p.n_stages;
-                        const uint32_t round = it / p.n_stages;
-                        if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, round & 1u, abort_flag))) {
+                    for (int kb = 0; kb < k_blocks; ++kb) {
+                        if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * st, st_par, abort_flag))) {
                             ok = false;
                             break;
                         }
                         tc_fence_after_sync();
-                        if (elect_one()) {
-                            const uint32_t a_lo = desc_lo0 + ((s * L.stage_bytes) >> 4);
+                        if (elected) {
                             const uint32_t b_lo = a_lo + (kATileBytes >> 4);
                             if (p.n_chunks == 1)
                                 issue_k_block<kPair, 1>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
                             else
                                 issue_k_block<kPair, 2>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
                             // the stage is free (in both CTAs) once these MMAs retire
-                            if constexpr (kPair) umma_commit_pair(bar_empty + 8 * s, 3);
-                            else umma_commit(bar_empty + 8 * s);
+                            if constexpr (kPair) umma_commit_pair(bar_empty + 8 * st, 3);
+                            else umma_commit(bar_empty + 8 * st);
                         }
                         __syncwarp();
+                        a_lo += stage_units;
+                        if (++st == static_cast<uint32_t>(p.n_stages)) { st = 0; st_par ^= 1u; a_lo = desc_lo0; }
                     }
-                    if (ok && elect_one()) {                 // accumulator complete
+                    if (ok && elected) {                     // accumulator complete
                         if constexpr (kPair) umma_commit_pair(bar_tfull + 8 * buf, 3);
                         else umma_commit(bar_tfull + 8 * buf);
                     }
@@ -430,7 +439,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                 }
             }
             __syncwarp();
-            if (!ok && elect_one()) {
+            if (!ok && elected) {
                 // abort path: wait (bounded) for the MMAs already issued before TMEM is freed
                 if constexpr (kPair) umma_commit_pair(bar_done, 1);
                 else umma_commit(bar_done);
