@@ -39,6 +39,11 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
                      const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, float tau,
                      int32_t *__restrict__ status)
 {
+    // Launched so that it may run beside the scoring kernel ahead of it in the stream: with a window, the
+    // fate of the token leaving it depends only on its BUFFERED score, so all row traffic (old row to
+    // its page, new rows into the ring) happens at once and only the new scores wait for that kernel.
+    griddep_launch_dependents();
+    if (c.window <= 0) griddep_wait();                   // no window: the new score decides now
     const int gl = threadIdx.x & 15;
     const int64_t group = (static_cast<int64_t>(blockIdx.x) * kDecodeThreads + threadIdx.x) >> 4;
     const int64_t n_groups = static_cast<int64_t>(n_layers_call) * c.n_seqs * c.n_heads;
@@ -51,7 +56,6 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
     const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
     const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
     const int32_t n = c.n_tokens[li];
-    const float s_new = scores[src_row];
 
     // which row (if any) moves to the prefix now
     bool append = false;
@@ -66,7 +70,7 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
             app_v = c.v_ring + (li * c.window + slot) * c.row_units;
         }
     } else {
-        append = s_new >= tau;
+        append = scores[src_row] >= tau;
         app_k = K_new + src_row * c.row_units;
         app_v = V_new + src_row * c.row_units;
     }
@@ -100,17 +104,19 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
         }
         if (gl == 0) c.prefix_len[li] = idx + 1;
     }
-    if (!live) return;
-    if (c.window > 0) {
+    if (live && c.window > 0) {
         // each lane overwrites exactly the 16-byte units it read above, so no lane races another
         const int64_t ring = (li * c.window + slot) * c.row_units;
         for (int u = gl; u < c.row_units; u += 16) {
             c.k_ring[ring + u] = K_new[src_row * c.row_units + u];
             c.v_ring[ring + u] = V_new[src_row * c.row_units + u];
         }
-        if (gl == 0) c.score_ring[li * c.window + slot] = s_new;
     }
-    if (gl == 0) c.n_tokens[li] = n + 1;
+    if (live && gl == 0) c.n_tokens[li] = n + 1;
+    if (c.window > 0) {
+        griddep_wait();                                  // every thread: the scoring kernel's output is needed only here
+        if (live && gl == 0) c.score_ring[li * c.window + slot] = scores[src_row];
+    }
 }
 
 // After a prompt's prefix has been compacted: copies the last min(T, w) tokens of the prompt (rows of

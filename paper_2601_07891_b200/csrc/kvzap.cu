@@ -14,6 +14,7 @@
 #include "decode_kernels.cuh"
 #include "prune_kernels.cuh"
 #include "score_kernel.cuh"
+#include "score_split_kernel.cuh"
 
 namespace kvzap {
 
@@ -42,6 +43,10 @@ struct kvzap_ctx {
         CUtensorMap tmap_w;          // box = the W1 rows one CTA stages per MMA chunk
     } sched[2];
     int pair_clusters = 0;           // CTA pairs that can be resident at once; 0 = pairs unavailable
+    // few-token scoring (decode): clusters of split_n CTAs share a tile, each takes hidden / split_n units
+    int split_n = 0, split_stages = 0, split_tmem_cols = 0;
+    uint32_t split_smem = 0;
+    CUtensorMap split_tmap_w;
     // weights of all layers, stacked so that one tensor map / one base pointer serves any layer range
     void *w1_all = nullptr;          // bf16 [L * w1_rows, d_model]
     float *b1_all = nullptr;         // [L][w1_rows]
@@ -118,6 +123,39 @@ static kvzap_status make_tmap(kvzap_ctx *ctx, CUtensorMap *map, const void *base
                     static_cast<int>(r), static_cast<unsigned long long>(rows), static_cast<unsigned long long>(cols),
                     box_rows);
     return KVZAP_OK;
+}
+
+// Tensor map over the context's copy of the first-layer weights, stored K block by K block:
+// [k_blocks][rows_total][64] bf16, so that the `box_rows` x 64 tile a CTA stages per K step is one
+// contiguous piece of memory (a decode step reads every weight byte from HBM exactly once; contiguous
+// tiles keep those reads inside open DRAM pages).  Box = box_rows rows of one K block, 128-byte swizzle.
+static kvzap_status make_tmap_w(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows_total,
+                                uint64_t k_blocks, uint32_t box_rows)
+{
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(kBlockK), rows_total, k_blocks};
+    const cuuint64_t strides[2] = {kBlockK * 2, kBlockK * 2 * rows_total};
+    const cuuint32_t box[3] = {static_cast<cuuint32_t>(kBlockK), box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box,
+                                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, KVZAP_ERR_CUDA, "cuTensorMapEncodeTiled (weights) failed with code %d (rows=%llu box_rows=%u)",
+                    static_cast<int>(r), static_cast<unsigned long long>(rows_total), box_rows);
+    return KVZAP_OK;
+}
+
+// W1 [rows, d_model] bf16 (row-major) -> rows row0 .. row0+rows-1 of the K-blocked copy
+// dst [d_model / 64][rows_total][64]; one thread moves 8 elements (16 bytes).
+__global__ void pack_w1_kernel(const uint4 *__restrict__ W1, int rows, int d_model, int64_t rows_total, int64_t row0,
+                               uint4 *__restrict__ dst)
+{
+    const int units_per_row = d_model / 8;
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<int64_t>(rows) * units_per_row) return;
+    const int r = static_cast<int>(idx / units_per_row), u = static_cast<int>(idx % units_per_row);
+    const int kb = u / (kBlockK / 8), xu = u % (kBlockK / 8);
+    dst[(static_cast<int64_t>(kb) * rows_total + row0 + r) * (kBlockK / 8) + xu] = W1[idx];
 }
 
 // W2 [H, hidden] bf16 -> w2t [hidden][8] fp32 (zero for heads >= H); b2 -> [8] fp32.
@@ -253,6 +291,55 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // A smaller grid is launched the ordinary way.
     const kvzap_config &c = ctx->cfg;
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    // Few tiles (a decode step: one tile per layer): split every tile's hidden units over a cluster, so
+    // that the launch fills the machine and every CTA reads only its own slice of W1.
+    if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n <= ctx->sm_count) {
+        CUtensorMap tmap_x;
+        kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens),
+                                    static_cast<uint64_t>(c.d_model), kTileM, static_cast<uint64_t>(n_layers));
+        if (st != KVZAP_OK) return st;
+        ScoreParams p;
+        memset(&p, 0, sizeof p);
+        p.n_tokens = n_tokens;
+        p.n_tiles = static_cast<int32_t>(blocks_per_layer * n_layers);
+        p.tiles_per_layer = static_cast<int32_t>(blocks_per_layer);
+        p.blocks_per_layer = static_cast<int32_t>(blocks_per_layer);
+        p.n_layers_call = n_layers;
+        p.layer0 = layer;
+        p.w_rows = ctx->w1_rows;
+        p.d_model = c.d_model;
+        p.group_w = p.chunk_n = c.hidden / ctx->split_n;
+        p.n_groups = p.n_chunks = 1;
+        p.n_stages = ctx->split_stages;
+        p.acc_bufs = 1;
+        p.tmem_cols = ctx->split_tmem_cols;
+        p.n_hidden = c.hidden;
+        p.n_heads = c.n_kv_heads;
+        p.b1 = ctx->b1_all;
+        p.w2t = ctx->w2t_all;
+        p.b2 = ctx->b2_all;
+        p.scores = scores;
+        p.maskbits = maskbits;
+        p.n_words = blocks_per_layer * 4;
+        p.cu_seqlens = cu_seqlens;
+        p.n_seqs = n_seqs;
+        p.window = w;
+        p.window_keep = window_keep;
+        p.tau = tau;
+        p.status = ctx->status_dev;
+        ctx->last_scores = scores;
+        ctx->last_scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
+        {
+            ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attrs[2];
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * ctx->split_n)), dim3(kScoreThreads),
+                        ctx->split_smem, stream, false, ctx->split_n);
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n));
+        }
+        ctx->launches += 1;
+        return KVZAP_OK;
+    }
     // CTA pairs pay off once a layer has at least two 128-token blocks; a pair's work tile is 256 tokens
     const bool pair = c.hidden > 0 && ctx->pair_clusters > 0 && blocks_per_layer >= 2;
     const kvzap_ctx::Schedule &sc = ctx->sched[pair ? 1 : 0];
@@ -500,6 +587,11 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     // scoring kernels need the largest shared-memory split, so the compaction asks for it too.
     CREATE_CUDA(cudaFuncSetAttribute(compact_dense_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    CREATE_CUDA(cudaFuncSetAttribute(decode_update_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    if (c.hidden > 0)
+        CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         static_cast<int>(cudaSharedmemCarveoutMaxShared)));
     if (c.hidden > 0) {
         CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          static_cast<int>(cudaSharedmemCarveoutMaxShared)));
@@ -524,13 +616,30 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         ctx->err[0] = 0;
         for (int mode = 0; mode < (c.hidden > 0 ? 2 : 1); ++mode) {
             kvzap_ctx::Schedule &sc = ctx->sched[mode];
-            if (make_tmap(ctx, &sc.tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
-                          static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(sc.chunk_n / (mode + 1))) != KVZAP_OK) {
+            if (make_tmap_w(ctx, &sc.tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
+                            static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(sc.chunk_n / (mode + 1))) != KVZAP_OK) {
                 snprintf(g_create_error, sizeof g_create_error, "%s", ctx->err);
                 free_all(ctx);
                 delete ctx;
                 return KVZAP_ERR_CUDA;
             }
+        }
+    }
+    if (c.hidden > 0) {
+        // few-token schedule: four CTAs per tile
+        const int n_split = 4, ns = c.hidden / n_split;
+        int stages = kMaxStages;
+        for (; stages >= 2; --stages)
+            if (static_cast<int>(split_smem_layout(ns, stages, n_split).total) <= budget) break;
+        if (stages >= 2 && ns % 16 == 0 && ns <= 256) {
+            ctx->split_stages = stages;
+            ctx->split_smem = split_smem_layout(ns, stages, n_split).total + 1024;
+            ctx->split_tmem_cols = next_pow2(ns);
+            CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(ctx->split_smem)));
+            if (make_tmap_w(ctx, &ctx->split_tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
+                            static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns)) == KVZAP_OK)
+                ctx->split_n = n_split;
         }
     }
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -577,10 +686,16 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, co
     if (c.hidden > 0 && !W2) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-MLP needs W2");
     DeviceGuard guard(c.device);
     const int rows = c.hidden > 0 ? c.hidden : c.n_kv_heads;
-    char *w1_dst = static_cast<char *>(ctx->w1_all) + static_cast<size_t>(layer) * ctx->w1_rows * c.d_model * 2;
+    if (!aligned16(W1)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "W1 must be 16-byte aligned");
     float *b1_dst = ctx->b1_all + static_cast<size_t>(layer) * ctx->w1_rows;
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(w1_dst, W1, static_cast<size_t>(rows) * c.d_model * 2, cudaMemcpyDeviceToDevice,
-                                    stream));
+    {
+        const int64_t units = static_cast<int64_t>(rows) * (c.d_model / 8);
+        pack_w1_kernel<<<static_cast<unsigned>((units + 255) / 256), 256, 0, stream>>>(
+            static_cast<const uint4 *>(W1), rows, c.d_model, static_cast<int64_t>(c.n_layers) * ctx->w1_rows,
+            static_cast<int64_t>(layer) * ctx->w1_rows, static_cast<uint4 *>(ctx->w1_all));
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    }
     if (b1)
         KVZAP_CUDA(ctx, cudaMemcpyAsync(b1_dst, b1, sizeof(float) * rows, cudaMemcpyDeviceToDevice, stream));
     else
@@ -1101,11 +1216,14 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
     const int64_t threads = n_groups * 16;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_DECODE_UPDATE, stream);
-        decode_update_kernel<<<static_cast<unsigned>((threads + kDecodeThreads - 1) / kDecodeThreads), kDecodeThreads, 0,
-                               stream>>>(cache->v, layer_begin, n_layers, scores, static_cast<const uint4 *>(K_new),
-                                         static_cast<const uint4 *>(V_new), tau, ctx->status_dev);
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>((threads + kDecodeThreads - 1) / kDecodeThreads)),
+                    dim3(kDecodeThreads), 0, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, decode_update_kernel, cache->v, layer_begin, n_layers,
+                                           static_cast<const float *>(scores), static_cast<const uint4 *>(K_new),
+                                           static_cast<const uint4 *>(V_new), tau, ctx->status_dev));
     }
-    KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
     return KVZAP_OK;
 }

@@ -55,6 +55,7 @@ struct ScoreParams {
     int32_t tmem_cols;    // allocation, power of two >= 32
     int32_t n_hidden;     // MLP hidden width (0 for Linear)
     int32_t n_heads;
+    // W1 (through the tensor map): K-blocked copy [d_model / 64][L * w_rows][64], see make_tmap_w
     const float *b1;      // stacked over all layers: MLP [L][n_hidden]; Linear [L][16] (zero padded)
     const float *w2t;     // MLP: [L][n_hidden][8] fp32, heads beyond n_heads are zero
     const float *b2;      // MLP: [L][8]
@@ -325,7 +326,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             const int row0 = m_tile * kTileM;
             for (int g = 0; g < p.n_groups && ok; ++g) {
                 const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w + static_cast<int>(cta_rank) * b_rows_chunk;
-                for (int kx = 0; kx < p.d_model; kx += kBlockK, ++it) {
+                for (int kx = 0, kb = 0; kx < p.d_model; kx += kBlockK, ++kb, ++it) {
                     if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
                         ok = false;
                         break;
@@ -337,17 +338,17 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                             if (leader) mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes * 2);
                             const uint32_t bar = full0_cluster + 8 * st;
                             tma_load_3d_pair(sa, &tmap_x, bar, kx, row0, l_rel, pol_x);
-                            tma_load_2d_pair(sa + kATileBytes, &tmap_w, bar, kx, w_row0, pol_w);
+                            tma_load_3d_pair(sa + kATileBytes, &tmap_w, bar, 0, w_row0, kb, pol_w);
                             if (p.n_chunks == 2)
-                                tma_load_2d_pair(sa + kATileBytes + b_rows_chunk * kBlockK * 2, &tmap_w, bar, kx,
-                                                 w_row0 + p.chunk_n, pol_w);
+                                tma_load_3d_pair(sa + kATileBytes + b_rows_chunk * kBlockK * 2, &tmap_w, bar, 0,
+                                                 w_row0 + p.chunk_n, kb, pol_w);
                         } else {
                             mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes);
                             tma_load_3d(sa, &tmap_x, bar_full + 8 * st, kx, row0, l_rel, pol_x);
-                            tma_load_2d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, kx, w_row0, pol_w);
+                            tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row0, kb, pol_w);
                             if (p.n_chunks == 2)
-                                tma_load_2d(sa + kATileBytes + p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * st, kx,
-                                            w_row0 + p.chunk_n, pol_w);
+                                tma_load_3d(sa + kATileBytes + p.chunk_n * kBlockK * 2, &tmap_w, bar_full + 8 * st, 0,
+                                            w_row0 + p.chunk_n, kb, pol_w);
                         }
                     }
                     __syncwarp();
@@ -618,7 +619,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     // If this kernel was allowed to start before the one ahead of it had finished, no CTA leaves
     // before that kernel is complete: kernels then still complete in stream order, and a CTA of the
     // next scoring kernel that finds this SM free knows that everything two launches back is done.
-    if (threadIdx.x == 0) griddep_wait();
+    griddep_wait();      // every thread executes it: a wait by some threads only was seen not to hold the others' CTA back
     if (warp == 1) {
         tc_fence_after_sync();
         if constexpr (kPair) tmem_dealloc_pair(tmem_base, static_cast<uint32_t>(p.tmem_cols));

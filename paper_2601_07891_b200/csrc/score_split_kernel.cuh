@@ -1,0 +1,286 @@
+// MLP surrogate scoring for FEW tokens per layer (the decode step: one new token per sequence,
+// Method, "KVzap" and the caption of Algorithm 1), where one 128-token tile per layer would leave
+// most SMs idle and every byte of W1 has to come from HBM.
+//
+// A cluster of n_split CTAs shares one 128-token tile: CTA j computes the hidden units
+// [j * Ns, (j + 1) * Ns), Ns = hidden / n_split, over the whole K range (its slice of W1 is read
+// exactly once, the X tile once per CTA, from L2 after the first), applies bias + GELU and its part
+// of the second layer, and sends its 8 partial sums per token to the cluster's first CTA through
+// distributed shared memory.  After one cluster barrier that CTA adds the parts and b2 and writes the
+// scores (and, if asked for, the keep bits).  36 layers x 4 CTAs fill the machine.
+//
+// Warp roles as in score_kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..9
+// epilogue (TMEM lane quarter = warp % 4; the two warps of a quarter take alternate 16-column chunks).
+#pragma once
+
+#include "score_kernel.cuh"
+
+namespace kvzap {
+
+struct SplitSmemLayout {
+    uint32_t stage_bytes, stages_end, w2s, b1s, part, xpart, bars, total;
+};
+__host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stages, int n_split)
+{
+    SplitSmemLayout L;
+    L.stage_bytes = kATileBytes + static_cast<uint32_t>(ns) * kBlockK * 2;
+    L.stages_end = L.stage_bytes * n_stages;
+    L.w2s = L.stages_end;
+    L.b1s = L.w2s + static_cast<uint32_t>(ns) * kMaxHeads * 4;
+    L.part = L.b1s + static_cast<uint32_t>(ns) * 4;
+    L.xpart = L.part + kTileM * kMaxHeads * 4;
+    L.bars = L.xpart + static_cast<uint32_t>(n_split) * kTileM * kMaxHeads * 4;
+    L.total = L.bars + 256;
+    return L;
+}
+
+// p.group_w = p.chunk_n = Ns; p.n_groups = p.n_chunks = 1; p.acc_bufs = 1; p.n_tiles = 128-token
+// tiles over all layers of the call; gridDim.x = n_split * p.n_tiles, cluster dimension n_split.
+__global__ void __maxnreg__(128)
+score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                   const ScoreParams p, const int n_split)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t *smem = smem_raw + pad;
+    const uint32_t smem_base = raw_addr + pad;
+    const int ns = p.chunk_n;
+    const SplitSmemLayout L = split_smem_layout(ns, p.n_stages, n_split);
+
+    ulonglong2 *w2p = reinterpret_cast<ulonglong2 *>(smem + L.w2s);
+    float *w2f = reinterpret_cast<float *>(smem + L.w2s);
+    float *b1s = reinterpret_cast<float *>(smem + L.b1s);
+    float *part = reinterpret_cast<float *>(smem + L.part);
+    float *xpart = reinterpret_cast<float *>(smem + L.xpart);
+    const uint32_t bars = smem_base + L.bars;
+    const uint32_t bar_full = bars;                      // [kMaxStages] TMA -> MMA
+    const uint32_t bar_empty = bars + 8 * kMaxStages;    // [kMaxStages] MMA -> TMA
+    const uint32_t bar_tfull = bars + 16 * kMaxStages;   // MMA -> epilogue
+    const uint32_t bar_done = bar_tfull + 8;             // abort path only
+    const uint32_t bar_pfull = bar_done + 8;             // second warp of a lane quarter -> first
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 32);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 36);
+
+    griddep_launch_dependents();
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();            // which slice of the hidden units
+    const int tile = static_cast<int>(blockIdx.x) / n_split;
+    const int l_rel = tile / p.tiles_per_layer;
+    const int m_tile = tile - l_rel * p.tiles_per_layer;
+    const int layer = p.layer0 + l_rel;
+    const int j_first = static_cast<int>(rank) * ns;     // first hidden unit of this CTA
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_tfull, 1);
+        mbar_init(bar_done, 1);
+        mbar_init(bar_pfull, 4);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const int k_blocks = p.d_model / kBlockK;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        const uint64_t pol_x = l2_policy_evict_last();    // the other CTAs of the cluster read the same X tile
+        const uint64_t pol_w = l2_policy_evict_first();   // every W1 byte is read once per step
+        const bool elected = elect_one();
+        const int w_row = layer * p.w_rows + j_first;
+        const int row0 = m_tile * kTileM;
+        uint32_t st = 0, st_par = 1, sa = smem_base;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
+                ok = false;
+                break;
+            }
+            if (elected) {
+                mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes);
+                tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row, kb, pol_w);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, kb * kBlockK, row0, l_rel, pol_x);
+            }
+            __syncwarp();
+            sa += L.stage_bytes;
+            if (++st == static_cast<uint32_t>(p.n_stages)) { st = 0; st_par ^= 1u; sa = smem_base; }
+        }
+        if (!ok && lane == 0) {
+            // abort path: give the copies already in flight a fixed time to land before the CTA exits
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000LL) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        const uint32_t idesc = umma_idesc_bf16_f32(kTileM, static_cast<uint32_t>(ns));
+        const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
+        const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
+        const uint32_t desc_lo0 = static_cast<uint32_t>(desc0);
+        const uint32_t stage_units = L.stage_bytes >> 4;
+        const bool elected = elect_one();
+        uint32_t st = 0, st_par = 0, a_lo = desc_lo0;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * st, st_par, abort_flag))) {
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            if (elected) {
+                issue_k_block<false, 1>(tmem_base, a_lo, a_lo + (kATileBytes >> 4), desc_hi, 0, 0, idesc, kb == 0);
+                umma_commit(bar_empty + 8 * st);
+            }
+            __syncwarp();
+            a_lo += stage_units;
+            if (++st == static_cast<uint32_t>(p.n_stages)) { st = 0; st_par ^= 1u; a_lo = desc_lo0; }
+        }
+        if (ok && elected) umma_commit(bar_tfull);
+        __syncwarp();
+        if (!ok && elected) {
+            umma_commit(bar_done);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_done, 0))
+                if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue: partial second layer
+        const int ew = warp - 2;
+        const int q = warp & 3;
+        const int hsel = ew >> 2;
+        const int row = q * 32 + lane;
+        const int etid = threadIdx.x - 64;
+        // this CTA's slice of b1 and W2 (pairs of hidden units, see mlp_columns)
+        const float *w2g = p.w2t + (static_cast<int64_t>(layer) * p.n_hidden + j_first) * kMaxHeads;
+        const float *b1g = p.b1 + static_cast<int64_t>(layer) * p.n_hidden + j_first;
+        for (int i = etid; i < ns * kMaxHeads; i += 256) {
+            const int j = i >> 3, h = i & 7;
+            w2f[(((j >> 1) * kMaxHeads + h) << 1) + (j & 1)] = __ldg(w2g + i);
+        }
+        for (int i = etid; i < ns; i += 256) b1s[i] = __ldg(b1g + i);
+        named_barrier_sync(1, 256);
+        bool ok = mbar_wait(bar_tfull, 0, abort_flag);
+        uint64_t acc[kMaxHeads];
+#pragma unroll
+        for (int h = 0; h < kMaxHeads; ++h) acc[h] = 0ull;
+        if (ok) {
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+            // the first warp of a lane quarter takes the 16-column chunks 0, 2, 4, ..., the second the odd ones
+            const int n16 = ns >> 4;
+            uint32_t ra[16], rb[16];
+            int c = hsel;
+            if (c < n16) tmem_ld_x16(t_row + c * 16, ra);
+            while (c < n16) {
+                tmem_wait_ld();
+                reg_fence16(ra);
+                if (c + 2 < n16) tmem_ld_x16(t_row + (c + 2) * 16, rb);
+                mlp_columns<16>(ra, c * 16, b1s, w2p, acc);
+                c += 2;
+                if (c < n16) {
+                    tmem_wait_ld();
+                    reg_fence16(rb);
+                    if (c + 2 < n16) tmem_ld_x16(t_row + (c + 2) * 16, ra);
+                    mlp_columns<16>(rb, c * 16, b1s, w2p, acc);
+                    c += 2;
+                }
+            }
+        }
+        float s[kMaxHeads];
+#pragma unroll
+        for (int h = 0; h < kMaxHeads; ++h) {
+            float lo, hi;
+            f2_unpack(acc[h], lo, hi);
+            s[h] = lo + hi;
+        }
+        if (hsel == 1) {
+            float4 *dst = reinterpret_cast<float4 *>(part + row * kMaxHeads);
+            dst[0] = make_float4(s[0], s[1], s[2], s[3]);
+            dst[1] = make_float4(s[4], s[5], s[6], s[7]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_pfull);
+        } else {
+            ok = mbar_wait(bar_pfull, 0, abort_flag) && ok;
+            const float4 *src = reinterpret_cast<const float4 *>(part + row * kMaxHeads);
+            const float4 pa = src[0], pb = src[1];
+            s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
+            s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
+            // hand this CTA's partial sums to the cluster's first CTA: xpart[rank][row][8]
+            const uint32_t dst = map_to_cta(smem_base + L.xpart + (rank * kTileM + row) * kMaxHeads * 4, 0);
+            st_shared_cluster_v4(dst, s[0], s[1], s[2], s[3]);
+            st_shared_cluster_v4(dst + 16, s[4], s[5], s[6], s[7]);
+        }
+    }
+
+    tc_fence_before_sync();
+    // every thread of every CTA of the cluster arrives here (all waits above are bounded); after it the
+    // partial sums of all CTAs are visible in the first CTA's shared memory
+    cluster_sync_all();
+    if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    }
+    if (rank != 0 || warp < 2 || warp >= 6 || m_tile >= p.blocks_per_layer) return;
+
+    // ------------------------------------------------------------ first CTA: total, scores, keep bits
+    {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        float s[kMaxHeads];
+#pragma unroll
+        for (int h = 0; h < kMaxHeads; ++h) s[h] = __ldg(p.b2 + layer * kMaxHeads + h);
+        for (int r = 0; r < n_split; ++r) {
+            const float4 *src = reinterpret_cast<const float4 *>(xpart + (r * kTileM + row) * kMaxHeads);
+            const float4 pa = src[0], pb = src[1];
+            s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
+            s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
+        }
+        const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;
+        const bool valid = t < p.n_tokens;
+        if (valid && p.scores != nullptr) {
+            float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
+            if (p.n_heads == kMaxHeads) {
+                reinterpret_cast<float4 *>(dst)[0] = make_float4(s[0], s[1], s[2], s[3]);
+                reinterpret_cast<float4 *>(dst)[1] = make_float4(s[4], s[5], s[6], s[7]);
+            } else {
+#pragma unroll
+                for (int h = 0; h < kMaxHeads; ++h)
+                    if (h < p.n_heads) dst[h] = s[h];
+            }
+        }
+        if (p.maskbits != nullptr) {
+            bool in_window = false;
+            if (valid) {
+                int64_t seq_end = p.n_tokens;
+                if (p.cu_seqlens != nullptr && p.n_seqs > 1)
+                    seq_end = __ldg(p.cu_seqlens + seq_of_token(p.cu_seqlens, p.n_seqs, t) + 1);
+                in_window = t >= seq_end - static_cast<int64_t>(p.window);
+            }
+            uint32_t my_word = 0;
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) {
+                const bool keep = valid && (in_window ? p.window_keep != 0 : s[h] >= p.tau);
+                const uint32_t word = __ballot_sync(0xffffffffu, keep);
+                if (lane == h) my_word = word;
+            }
+            if (lane < p.n_heads)
+                p.maskbits[(static_cast<int64_t>(l_rel) * p.n_heads + lane) * p.n_words +
+                           static_cast<int64_t>(m_tile) * 4 + q] = my_word;
+        }
+    }
+}
+
+}  // namespace kvzap
