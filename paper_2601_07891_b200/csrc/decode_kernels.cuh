@@ -31,91 +31,130 @@ struct CacheView {
 };
 
 constexpr int kDecodeThreads = 256;
+constexpr int kDecodeLanes = 8;        // lanes that share one list (a 256-byte row = two 16-byte units per lane)
 
-// 16 lanes per list; lists of layers [layer0, layer0 + n_layers_call).
-// scores [n_layers_call][B][H] fp32, K_new/V_new [n_layers_call][B][H][D] bf16.
+// kDecodeLanes lanes per list; lists of layers [layer0, layer0 + n_layers_call); the grid walks the lists
+// with a grid stride.  scores [n_layers_call][B][H] fp32, K_new/V_new [n_layers_call][B][H][D] bf16.
+//
+// The kernel is launched so that it may be placed while the scoring kernel ahead of it in the stream
+// is still running.  With a window, the fate of the token that leaves it depends only on its
+// BUFFERED score, so the row traffic (old row to its page, new rows into the ring) needs nothing
+// from that kernel and only the new scores wait for it.  `wait_first` != 0 makes the whole kernel
+// wait instead: required when the scoring kernel itself was started before the previous step's
+// update had finished (two updates must never touch the cache at the same time).
 __global__ void __launch_bounds__(kDecodeThreads)
 decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const float *__restrict__ scores,
                      const uint4 *__restrict__ K_new, const uint4 *__restrict__ V_new, float tau,
-                     int32_t *__restrict__ status)
+                     int32_t *__restrict__ status, int wait_first)
 {
-    // Launched so that it may run beside the scoring kernel ahead of it in the stream: with a window, the
-    // fate of the token leaving it depends only on its BUFFERED score, so all row traffic (old row to
-    // its page, new rows into the ring) happens at once and only the new scores wait for that kernel.
     griddep_launch_dependents();
-    if (c.window <= 0) griddep_wait();                   // no window: the new score decides now
-    const int gl = threadIdx.x & 15;
-    const int64_t group = (static_cast<int64_t>(blockIdx.x) * kDecodeThreads + threadIdx.x) >> 4;
+    const bool rows_first = c.window > 0 && wait_first == 0;
+    if (!rows_first) griddep_wait();                     // every thread executes the wait
+    const int gl = threadIdx.x % kDecodeLanes;
     const int64_t n_groups = static_cast<int64_t>(n_layers_call) * c.n_seqs * c.n_heads;
-    const bool live = group < n_groups;
-    // every lane of the warp runs the whole body (the shuffles below need all 32 lanes)
-    const int64_t g = live ? group : 0;
-    const int l_rel = static_cast<int>(g / (static_cast<int64_t>(c.n_seqs) * c.n_heads));
-    const int rem = static_cast<int>(g - static_cast<int64_t>(l_rel) * c.n_seqs * c.n_heads);
-    const int b = rem / c.n_heads, h = rem % c.n_heads;
-    const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
-    const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
-    const int32_t n = c.n_tokens[li];
+    const int64_t group0 = (static_cast<int64_t>(blockIdx.x) * kDecodeThreads + threadIdx.x) / kDecodeLanes;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * (kDecodeThreads / kDecodeLanes);
+    const int64_t n_iter = (n_groups + stride - 1) / stride;       // the same for every thread
+    for (int64_t it = 0; it < n_iter; ++it) {
+        const int64_t group = group0 + it * stride;
+        const bool live = group < n_groups;
+        // every lane of the warp runs the whole body (the shuffles below need all 32 lanes)
+        const int64_t g = live ? group : 0;
+        const int l_rel = static_cast<int>(g / (static_cast<int64_t>(c.n_seqs) * c.n_heads));
+        const int rem = static_cast<int>(g - static_cast<int64_t>(l_rel) * c.n_seqs * c.n_heads);
+        const int b = rem / c.n_heads, h = rem % c.n_heads;
+        const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
+        const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+        const int32_t n = c.n_tokens[li];
 
-    // which row (if any) moves to the prefix now
-    bool append = false;
-    const uint4 *app_k = nullptr, *app_v = nullptr;
-    int slot = 0;
-    if (c.window > 0) {
-        slot = n % c.window;
-        if (n >= c.window) {
-            const float s_old = c.score_ring[li * c.window + slot];
-            append = s_old >= tau;
-            app_k = c.k_ring + (li * c.window + slot) * c.row_units;
-            app_v = c.v_ring + (li * c.window + slot) * c.row_units;
-        }
-    } else {
-        append = scores[src_row] >= tau;
-        app_k = K_new + src_row * c.row_units;
-        app_v = V_new + src_row * c.row_units;
-    }
-    append = append && live;
-
-    // page for the appended row: lane 0 of the group allocates when the row opens a new page
-    const int32_t idx = c.prefix_len[li];
-    const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
-    int32_t page = -1;
-    if (append && gl == 0) {
-        if (page_i >= c.max_pages) {
-            atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
-        } else if (in_page == 0) {
-            const int32_t got = atomicAdd(c.page_cursor, 1);
-            if (got >= c.n_pages_pool) {
-                atomicCAS(status, 0, 4);
-            } else {
-                page = got;
-                c.page_table[li * c.max_pages + page_i] = got;
+        // which row (if any) moves to the prefix now
+        bool append = false;
+        const uint4 *app_k = nullptr, *app_v = nullptr;
+        int slot = 0;
+        if (c.window > 0) {
+            slot = n % c.window;
+            if (n >= c.window) {
+                const float s_old = c.score_ring[li * c.window + slot];
+                append = s_old >= tau;
+                app_k = c.k_ring + (li * c.window + slot) * c.row_units;
+                app_v = c.v_ring + (li * c.window + slot) * c.row_units;
             }
         } else {
-            page = c.page_table[li * c.max_pages + page_i];
+            append = scores[src_row] >= tau;
+            app_k = K_new + src_row * c.row_units;
+            app_v = V_new + src_row * c.row_units;
+        }
+        append = append && live;
+
+        // page for the appended row: lane 0 of the group allocates when the row opens a new page
+        const int32_t idx = c.prefix_len[li];
+        const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
+        int32_t page = -1;
+        if (append && gl == 0) {
+            if (page_i >= c.max_pages) {
+                atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+            } else if (in_page == 0) {
+                const int32_t got = atomicAdd(c.page_cursor, 1);
+                if (got >= c.n_pages_pool) {
+                    atomicCAS(status, 0, 4);
+                } else {
+                    page = got;
+                    c.page_table[li * c.max_pages + page_i] = got;
+                }
+            } else {
+                page = c.page_table[li * c.max_pages + page_i];
+            }
+        }
+        page = __shfl_sync(0xffffffffu, page, 0, kDecodeLanes);
+        if (append && page >= 0) {
+            const int64_t dst = (static_cast<int64_t>(page) * c.page_tokens + in_page) * c.row_units;
+            for (int u = gl; u < c.row_units; u += 2 * kDecodeLanes) {       // all loads of a pass before its stores
+                const int u2 = u + kDecodeLanes;
+                const bool two = u2 < c.row_units;
+                const uint4 ka = app_k[u], va = app_v[u];
+                uint4 kb = ka, vb = va;
+                if (two) { kb = app_k[u2]; vb = app_v[u2]; }
+                c.k_pool[dst + u] = ka;
+                c.v_pool[dst + u] = va;
+                if (two) { c.k_pool[dst + u2] = kb; c.v_pool[dst + u2] = vb; }
+            }
+            if (gl == 0) c.prefix_len[li] = idx + 1;
+        }
+        if (live && c.window > 0) {
+            // each lane overwrites exactly the 16-byte units it read above, so no lane races another
+            const int64_t ring = (li * c.window + slot) * c.row_units;
+            const uint4 *kn = K_new + src_row * c.row_units, *vn = V_new + src_row * c.row_units;
+            for (int u = gl; u < c.row_units; u += 2 * kDecodeLanes) {
+                const int u2 = u + kDecodeLanes;
+                const bool two = u2 < c.row_units;
+                const uint4 ka = __ldg(kn + u), va = __ldg(vn + u);
+                uint4 kb = ka, vb = va;
+                if (two) { kb = __ldg(kn + u2); vb = __ldg(vn + u2); }
+                c.k_ring[ring + u] = ka;
+                c.v_ring[ring + u] = va;
+                if (two) { c.k_ring[ring + u2] = kb; c.v_ring[ring + u2] = vb; }
+            }
+        }
+        if (live && gl == 0) {
+            c.n_tokens[li] = n + 1;
+            if (c.window > 0 && !rows_first) c.score_ring[li * c.window + slot] = scores[src_row];
         }
     }
-    page = __shfl_sync(0xffffffffu, page, 0, 16);
-    if (append && page >= 0) {
-        const int64_t dst = (static_cast<int64_t>(page) * c.page_tokens + in_page) * c.row_units;
-        for (int u = gl; u < c.row_units; u += 16) {
-            c.k_pool[dst + u] = app_k[u];
-            c.v_pool[dst + u] = app_v[u];
+    if (rows_first) {
+        griddep_wait();                                  // every thread; the scoring kernel's output is needed only here
+        if (gl == 0) {
+            for (int64_t it = 0; it < n_iter; ++it) {
+                const int64_t group = group0 + it * stride;
+                if (group >= n_groups) break;
+                const int l_rel = static_cast<int>(group / (static_cast<int64_t>(c.n_seqs) * c.n_heads));
+                const int rem = static_cast<int>(group - static_cast<int64_t>(l_rel) * c.n_seqs * c.n_heads);
+                const int b = rem / c.n_heads, h = rem % c.n_heads;
+                const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
+                const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+                const int slot = (c.n_tokens[li] - 1) % c.window;      // the slot this thread filled above
+                c.score_ring[li * c.window + slot] = scores[src_row];
+            }
         }
-        if (gl == 0) c.prefix_len[li] = idx + 1;
-    }
-    if (live && c.window > 0) {
-        // each lane overwrites exactly the 16-byte units it read above, so no lane races another
-        const int64_t ring = (li * c.window + slot) * c.row_units;
-        for (int u = gl; u < c.row_units; u += 16) {
-            c.k_ring[ring + u] = K_new[src_row * c.row_units + u];
-            c.v_ring[ring + u] = V_new[src_row * c.row_units + u];
-        }
-    }
-    if (live && gl == 0) c.n_tokens[li] = n + 1;
-    if (c.window > 0) {
-        griddep_wait();                                  // every thread: the scoring kernel's output is needed only here
-        if (live && gl == 0) c.score_ring[li * c.window + slot] = scores[src_row];
     }
 }
 

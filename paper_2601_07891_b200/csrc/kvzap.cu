@@ -44,7 +44,7 @@ struct kvzap_ctx {
     } sched[2];
     int pair_clusters = 0;           // CTA pairs that can be resident at once; 0 = pairs unavailable
     // few-token scoring (decode): clusters of split_n CTAs share a tile, each takes hidden / split_n units
-    int split_n = 0, split_stages = 0, split_tmem_cols = 0;
+    int split_n = 0, split_k = 1, split_stages = 0, split_tmem_cols = 0;   // cluster = split_n * split_k CTAs
     uint32_t split_smem = 0;
     CUtensorMap split_tmap_w;
     // weights of all layers, stacked so that one tensor map / one base pointer serves any layer range
@@ -60,6 +60,7 @@ struct kvzap_ctx {
     uint64_t mask_turn = 0;
     int32_t *tile_counters = nullptr;    // [kMaskRing] work-tile counters of the scoring launches, used in rotation
     uint64_t score_turn = 0;
+    bool last_score_early = false;       // the last scoring launch was allowed to start early
     const void *last_scores = nullptr;   // scores buffer of the previous scoring launch, and its size
     size_t last_scores_bytes = 0;
     int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
@@ -293,7 +294,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
     // Few tiles (a decode step: one tile per layer): split every tile's hidden units over a cluster, so
     // that the launch fills the machine and every CTA reads only its own slice of W1.
-    if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n <= ctx->sm_count) {
+    if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count) {
         CUtensorMap tmap_x;
         kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens),
                                     static_cast<uint64_t>(c.d_model), kTileM, static_cast<uint64_t>(n_layers));
@@ -327,15 +328,27 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         p.window_keep = window_keep;
         p.tau = tau;
         p.status = ctx->status_dev;
+        // Early start (consecutive decode steps): this kernel reads only hidden states and weights; the one
+        // thing it may not do is write a scores buffer that the kernels of the previous call still read.
+        const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
+        bool clash = false;
+        if (scores && ctx->last_scores) {
+            const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
+            clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes;
+        }
         ctx->last_scores = scores;
-        ctx->last_scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
+        ctx->last_scores_bytes = sbytes;
+        const int n_ctas = ctx->split_n * ctx->split_k;
+        const bool early = !ctx->profiling && !clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count;
+        ctx->last_score_early = early;
         {
             ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attrs[2];
-            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * ctx->split_n)), dim3(kScoreThreads),
-                        ctx->split_smem, stream, false, ctx->split_n);
-            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n));
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * n_ctas)), dim3(kScoreThreads),
+                        ctx->split_smem, stream, early, n_ctas);
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n,
+                                               ctx->split_k));
         }
         ctx->launches += 1;
         return KVZAP_OK;
@@ -393,6 +406,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     }
     ctx->last_scores = scores;
     ctx->last_scores_bytes = scores_bytes;
+    ctx->last_score_early = false;       // (only the decode step's update kernel looks at this)
     {
         ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
         cudaLaunchConfig_t cfg;
@@ -443,7 +457,8 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
         KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel, static_cast<const uint4 *>(K),
                                            static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
                                            static_cast<uint4 *>(V_out), mask, n_words, n_blocks, blocks_per_cta,
-                                           cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths));
+                                           cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths, 0,
+                                           static_cast<const int32_t *>(nullptr)));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -626,20 +641,24 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         }
     }
     if (c.hidden > 0) {
-        // few-token schedule: four CTAs per tile
-        const int n_split = 4, ns = c.hidden / n_split;
+        // few-token schedule: four CTAs per tile.  2 x 2 (two slices of hidden units, two halves of K) when
+        // a slice of hidden / 2 units fits one MMA and the K blocks divide evenly, else four slices.
+        const bool two_by_two = c.hidden / 2 <= 256 && (c.hidden / 4) % 16 == 0 && (c.d_model / kBlockK) % 2 == 0;
+        const int n_split = two_by_two ? 2 : 4, k_split = two_by_two ? 2 : 1, ns = c.hidden / n_split;
         int stages = kMaxStages;
         for (; stages >= 2; --stages)
-            if (static_cast<int>(split_smem_layout(ns, stages, n_split).total) <= budget) break;
+            if (static_cast<int>(split_smem_layout(ns, stages, 4).total) <= budget) break;
         if (stages >= 2 && ns % 16 == 0 && ns <= 256) {
             ctx->split_stages = stages;
-            ctx->split_smem = split_smem_layout(ns, stages, n_split).total + 1024;
+            ctx->split_smem = split_smem_layout(ns, stages, 4).total + 1024;
             ctx->split_tmem_cols = next_pow2(ns);
             CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(ctx->split_smem)));
             if (make_tmap_w(ctx, &ctx->split_tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
-                            static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns)) == KVZAP_OK)
+                            static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns)) == KVZAP_OK) {
                 ctx->split_n = n_split;
+                ctx->split_k = k_split;
+            }
         }
     }
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1009,6 +1028,7 @@ struct kvzap_cache {
     kvzap::CacheView v;
     float *scores = nullptr;        // [L][B][H] scratch when the caller does not want the scores
     int64_t n_lists = 0;
+    int step_parity = 0;
 };
 
 namespace kvzap {
@@ -1024,23 +1044,36 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     const int64_t n_words = n_blocks * 4;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attrs[2];
     {
+        // lengths and the first page of every list (the only step that needs all lists at once)
         ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
-        scan_kernel<<<1, 1024, 0, stream>>>(mask, n_words, n_blocks, c.n_kv_heads, cu_seqlens, n_seqs,
-                                            n_tokens, ctx->blockprefix, ctx->seqbase, lengths, page_tokens, first_page,
-                                            n_pages_pool, max_pages, ctx->list_page0, page_table, n_pages_used,
-                                            page_cursor, ctx->status_dev);
+        make_launch(&cfg, attrs, dim3(1), dim3(1024), 0, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, scan_kernel, mask, n_words, n_blocks, static_cast<int>(c.n_kv_heads),
+                                           cu_seqlens, static_cast<int>(n_seqs), n_tokens, ctx->blockprefix, ctx->seqbase,
+                                           lengths, static_cast<int>(page_tokens), first_page, n_pages_pool,
+                                           static_cast<int>(max_pages), ctx->list_page0, page_table, n_pages_used,
+                                           page_cursor, ctx->status_dev));
     }
-    KVZAP_CUDA(ctx, cudaGetLastError());
-    const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(c.n_kv_heads));
+    // the same resident-at-once grid as the dense-ragged output (see launch_compaction)
+    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (c.hidden > 0 ? 2 : 6);
+    int64_t chunks = max_ctas / c.n_kv_heads;
+    if (chunks < 1) chunks = 1;
+    if (chunks > n_blocks) chunks = n_blocks;
+    const int blocks_per_cta = static_cast<int>((n_blocks + chunks - 1) / chunks);
+    chunks = (n_blocks + blocks_per_cta - 1) / blocks_per_cta;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
-        compact_kernel<true><<<grid, kCompactThreads, 0, stream>>>(
-            static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), static_cast<uint4 *>(K_pool),
-            static_cast<uint4 *>(V_pool), mask, n_words, n_blocks, ctx->blockprefix, ctx->seqbase, cu_seqlens,
-            n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, page_tokens, ctx->list_page0);
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(chunks), static_cast<unsigned>(c.n_kv_heads)),
+                    dim3(kDenseThreads), 0, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel, static_cast<const uint4 *>(K),
+                                           static_cast<const uint4 *>(V), static_cast<uint4 *>(K_pool),
+                                           static_cast<uint4 *>(V_pool), mask, n_words, n_blocks, blocks_per_cta,
+                                           cu_seqlens, static_cast<int>(n_seqs), n_tokens, static_cast<int>(c.n_kv_heads),
+                                           static_cast<int>(c.head_dim / 8), lengths, static_cast<int>(page_tokens),
+                                           static_cast<const int32_t *>(ctx->list_page0)));
     }
-    KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 2;
     return KVZAP_OK;
 }
@@ -1169,7 +1202,8 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.prefix_len), sizeof(int32_t) * n, true);
     alloc(reinterpret_cast<void **>(&v.page_table), sizeof(int32_t) * n * max_pages_per_list, true);
     alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
-    alloc(reinterpret_cast<void **>(&cache->scores), sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
+    // two halves used by alternate steps when the caller does not ask for the scores
+    alloc(reinterpret_cast<void **>(&cache->scores), 2 * sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
           false);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -1208,21 +1242,28 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
         return fail(ctx, KVZAP_ERR_INVALID_ARG, "decode: hidden, K_new, V_new must be non-NULL, 16-byte aligned");
     DeviceGuard guard(c.device);
     const int n_layers = layer_end - layer_begin;
-    float *scores = scores_out ? scores_out : cache->scores;
+    float *scores = scores_out;
+    if (!scores) {
+        scores = cache->scores + (cache->step_parity ? static_cast<size_t>(c.n_layers) * cache->v.n_seqs * c.n_kv_heads : 0);
+        cache->step_parity ^= 1;
+    }
     kvzap_status st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
                                    0.0f, 0, stream);
     if (st != KVZAP_OK) return st;
     const int64_t n_groups = static_cast<int64_t>(n_layers) * cache->v.n_seqs * c.n_kv_heads;
-    const int64_t threads = n_groups * 16;
+    const int64_t threads = n_groups * kDecodeLanes;
+    // a grid that is resident all at once beside the scoring kernel (one CTA per SM), walking the lists
+    int64_t blocks = (threads + kDecodeThreads - 1) / kDecodeThreads;
+    if (blocks > ctx->sm_count) blocks = ctx->sm_count;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_DECODE_UPDATE, stream);
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attrs[2];
-        make_launch(&cfg, attrs, dim3(static_cast<unsigned>((threads + kDecodeThreads - 1) / kDecodeThreads)),
-                    dim3(kDecodeThreads), 0, stream, !ctx->profiling, 1);
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(blocks)), dim3(kDecodeThreads), 0, stream, !ctx->profiling, 1);
         KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, decode_update_kernel, cache->v, layer_begin, n_layers,
                                            static_cast<const float *>(scores), static_cast<const uint4 *>(K_new),
-                                           static_cast<const uint4 *>(V_new), tau, ctx->status_dev));
+                                           static_cast<const uint4 *>(V_new), tau, ctx->status_dev,
+                                           ctx->last_score_early ? 1 : 0));
     }
     ctx->launches += 1;
     return KVZAP_OK;

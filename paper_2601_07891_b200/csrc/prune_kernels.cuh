@@ -96,6 +96,9 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
             int32_t *__restrict__ page_cursor, int32_t *__restrict__ status)
 {
+    // may be placed before the kernel that writes the mask has finished; waits for it here
+    griddep_launch_dependents();
+    griddep_wait();
     // page_cursor != nullptr: the first page comes from (and the pages used are added to) a device-side
     // allocator cursor instead of the first_page argument
     if (page_tokens > 0 && page_cursor != nullptr) first_page = *page_cursor;
@@ -314,8 +317,12 @@ __global__ void __launch_bounds__(kDenseThreads)
 compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ K_out,
                      uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
-                     int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths)
+                     int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths, int page_tokens,
+                     const int32_t *__restrict__ list_page0)
 {
+    // page_tokens > 0: paged output.  K_out / V_out are the page pools, list (b,h) starts at page
+    // list_page0[b * H + h] (-1 = nothing may be written), and lengths come from the scan kernel.
+    const bool paged = page_tokens > 0;
     __shared__ int32_t src_tok[kBlockTokens];
     __shared__ int64_t dst_row[kBlockTokens];
     __shared__ int32_t red[2][kDenseThreads / 32];
@@ -332,7 +339,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     griddep_launch_dependents();
     griddep_wait();
 
-    if (blockIdx.x == 0 && cu_seqlens != nullptr)         // empty sequences have no last token to write for them
+    if (blockIdx.x == 0 && cu_seqlens != nullptr && !paged)   // empty sequences have no last token to write for them
         for (int b = tid; b < n_seqs; b += kDenseThreads)
             if (cu_seqlens[b + 1] == cu_seqlens[b]) lengths[b * n_heads + h] = 0;
     if (blk0 >= n_blocks) return;
@@ -386,9 +393,15 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                 const bool keep = (w >> (tid & 31)) & 1u;
                 if (keep) {
                     src_tok[r] = tid;
-                    dst_row[r] = static_cast<int64_t>(h) * n_tokens + s + (running + r - base);
+                    const int64_t n = running + r - base;                  // rank inside list (b,h)
+                    if (paged) {
+                        const int32_t p0 = list_page0[b * n_heads + h];
+                        dst_row[r] = p0 < 0 ? -1 : (static_cast<int64_t>(p0) + n / page_tokens) * page_tokens + n % page_tokens;
+                    } else {
+                        dst_row[r] = static_cast<int64_t>(h) * n_tokens + s + n;
+                    }
                 }
-                if (t + 1 == e) lengths[b * n_heads + h] = running + r + (keep ? 1 : 0) - base;
+                if (t + 1 == e && !paged) lengths[b * n_heads + h] = running + r + (keep ? 1 : 0) - base;
                 if (tid == kBlockTokens - 1 || t + 1 == n_tokens) {
                     // base of the sequence in progress at the next block's first token
                     int32_t nb = base;
@@ -414,7 +427,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
 #pragma unroll
                 for (int j = 0; j < kRowsInFlight; ++j) {
                     const int i = i0 + j * kGroups;
-                    if (i < cnt) {
+                    if (i < cnt && dst_row[i] >= 0) {
                         const int64_t d = dst_row[i] * row_units + u0;
                         K_out[d] = kv[j];
                         V_out[d] = vv[j];

@@ -9,6 +9,12 @@
 // distributed shared memory.  After one cluster barrier that CTA adds the parts and b2 and writes the
 // scores (and, if asked for, the keep bits).  36 layers x 4 CTAs fill the machine.
 //
+// With k_split = 2 the cluster is 2 x 2: two CTAs share a slice of hidden units and each runs half of
+// the K range, so an X tile is read by two CTAs instead of four (the launch is bound by the bytes the
+// SMs pull through L2).  The two partial pre-activation tiles are combined before the GELU: each CTA
+// sends the half of its accumulator that its partner owns through distributed shared memory (into
+// the partner's pipeline stages, idle by then), and finishes the columns it owns itself.
+//
 // Warp roles as in score_kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..9
 // epilogue (TMEM lane quarter = warp % 4; the two warps of a quarter take alternate 16-column chunks).
 #pragma once
@@ -34,11 +40,12 @@ __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stage
     return L;
 }
 
-// p.group_w = p.chunk_n = Ns; p.n_groups = p.n_chunks = 1; p.acc_bufs = 1; p.n_tiles = 128-token
-// tiles over all layers of the call; gridDim.x = n_split * p.n_tiles, cluster dimension n_split.
+// p.group_w = p.chunk_n = Ns (the MMA's N); p.n_chunks = 1; p.acc_bufs = 1; p.n_tiles = 128-token tiles
+// over all layers of the call; cluster dimension n_split * k_split, gridDim.x = cluster size * p.n_tiles.
+// A CTA ends up owning Ns / k_split hidden units: xpart and the W2 / b1 slices are sized for those.
 __global__ void __maxnreg__(128)
 score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                   const ScoreParams p, const int n_split)
+                   const ScoreParams p, const int n_split, const int k_split)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -46,7 +53,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     uint8_t *smem = smem_raw + pad;
     const uint32_t smem_base = raw_addr + pad;
     const int ns = p.chunk_n;
-    const SplitSmemLayout L = split_smem_layout(ns, p.n_stages, n_split);
+    const int n_ctas = n_split * k_split;
+    const SplitSmemLayout L = split_smem_layout(ns, p.n_stages, n_ctas);
 
     ulonglong2 *w2p = reinterpret_cast<ulonglong2 *>(smem + L.w2s);
     float *w2f = reinterpret_cast<float *>(smem + L.w2s);
@@ -65,12 +73,16 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     griddep_launch_dependents();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_cta_rank();            // which slice of the hidden units
-    const int tile = static_cast<int>(blockIdx.x) / n_split;
+    const uint32_t rank = cluster_cta_rank();
+    const int nh = static_cast<int>(rank) % n_split;     // which slice of the hidden units
+    const int kh = static_cast<int>(rank) / n_split;     // which part of the K range
+    const int tile = static_cast<int>(blockIdx.x) / n_ctas;
     const int l_rel = tile / p.tiles_per_layer;
     const int m_tile = tile - l_rel * p.tiles_per_layer;
     const int layer = p.layer0 + l_rel;
-    const int j_first = static_cast<int>(rank) * ns;     // first hidden unit of this CTA
+    const int own_n = ns / k_split;                      // accumulator columns this CTA finishes
+    const int own_c0 = kh * own_n;                       // the first of them
+    const int j_first = nh * ns + own_c0;                // = first hidden unit of this CTA
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) {
@@ -93,14 +105,15 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int k_blocks = p.d_model / kBlockK;
+    const int k_blocks = p.d_model / kBlockK / k_split;  // K blocks of this CTA
+    const int kb_first = kh * k_blocks;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         const uint64_t pol_x = l2_policy_evict_last();    // the other CTAs of the cluster read the same X tile
         const uint64_t pol_w = l2_policy_evict_first();   // every W1 byte is read once per step
         const bool elected = elect_one();
-        const int w_row = layer * p.w_rows + j_first;
+        const int w_row = layer * p.w_rows + nh * ns;
         const int row0 = m_tile * kTileM;
         uint32_t st = 0, st_par = 1, sa = smem_base;
         bool ok = true;
@@ -111,8 +124,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
             if (elected) {
                 mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes);
-                tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row, kb, pol_w);
-                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, kb * kBlockK, row0, l_rel, pol_x);
+                tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row, kb_first + kb, pol_w);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, (kb_first + kb) * kBlockK, row0, l_rel, pol_x);
             }
             __syncwarp();
             sa += L.stage_bytes;
@@ -155,44 +168,92 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             while (!mbar_try_wait(bar_done, 0))
                 if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
         }
-    } else {
-        // ------------------------------------------------------------ epilogue: partial second layer
-        const int ew = warp - 2;
-        const int q = warp & 3;
-        const int hsel = ew >> 2;
-        const int row = q * 32 + lane;
-        const int etid = threadIdx.x - 64;
+    }
+
+    // ------------------------------------------------------------ epilogue (warps 2..9)
+    const bool epi = warp >= 2;
+    const int q = warp & 3;                 // TMEM lane quarter
+    const int hsel = (warp - 2) >> 2;       // which of the two warps of that quarter
+    const int row = q * 32 + lane;
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+    bool ok = true;
+    if (epi) {
         // this CTA's slice of b1 and W2 (pairs of hidden units, see mlp_columns)
+        const int etid = threadIdx.x - 64;
         const float *w2g = p.w2t + (static_cast<int64_t>(layer) * p.n_hidden + j_first) * kMaxHeads;
         const float *b1g = p.b1 + static_cast<int64_t>(layer) * p.n_hidden + j_first;
-        for (int i = etid; i < ns * kMaxHeads; i += 256) {
+        for (int i = etid; i < own_n * kMaxHeads; i += 256) {
             const int j = i >> 3, h = i & 7;
             w2f[(((j >> 1) * kMaxHeads + h) << 1) + (j & 1)] = __ldg(w2g + i);
         }
-        for (int i = etid; i < ns; i += 256) b1s[i] = __ldg(b1g + i);
+        for (int i = etid; i < own_n; i += 256) b1s[i] = __ldg(b1g + i);
         named_barrier_sync(1, 256);
-        bool ok = mbar_wait(bar_tfull, 0, abort_flag);
+        ok = mbar_wait(bar_tfull, 0, abort_flag);
+        tc_fence_after_sync();
+    }
+    const int n16 = own_n >> 4;             // 16-column chunks this CTA owns (and as many it sends away)
+    float4 *recv = reinterpret_cast<float4 *>(smem);          // [own_n / 4][128 rows] float4, over the idle stages
+    if (k_split == 2) {
+        // every CTA's MMAs are complete once all have passed this barrier: the stages may be overwritten
+        tc_fence_before_sync();
+        cluster_sync_all();
+        if (epi && ok) {
+            const uint32_t partner = rank ^ static_cast<uint32_t>(n_split);
+            const int send_c0 = (1 - kh) * own_n;               // the columns the partner owns
+            const uint32_t dst0 = map_to_cta(smem_base, partner);
+            for (int c = hsel; c < n16; c += 2) {
+                uint32_t r[16];
+                tmem_ld_x16(t_row + send_c0 + c * 16, r);
+                tmem_wait_ld();
+                reg_fence16(r);
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    st_shared_cluster_v4(dst0 + (static_cast<uint32_t>(c * 4 + i) * kTileM + row) * 16,
+                                         __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                         __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            }
+        }
+        cluster_sync_all();                                     // the partner's half has arrived
+    }
+    if (epi) {
         uint64_t acc[kMaxHeads];
 #pragma unroll
         for (int h = 0; h < kMaxHeads; ++h) acc[h] = 0ull;
         if (ok) {
-            tc_fence_after_sync();
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
             // the first warp of a lane quarter takes the 16-column chunks 0, 2, 4, ..., the second the odd ones
-            const int n16 = ns >> 4;
             uint32_t ra[16], rb[16];
             int c = hsel;
-            if (c < n16) tmem_ld_x16(t_row + c * 16, ra);
+            if (c < n16) tmem_ld_x16(t_row + own_c0 + c * 16, ra);
             while (c < n16) {
                 tmem_wait_ld();
                 reg_fence16(ra);
-                if (c + 2 < n16) tmem_ld_x16(t_row + (c + 2) * 16, rb);
+                if (c + 2 < n16) tmem_ld_x16(t_row + own_c0 + (c + 2) * 16, rb);
+                if (k_split == 2) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float4 o = recv[(c * 4 + i) * kTileM + row];
+                        ra[4 * i] = __float_as_uint(__uint_as_float(ra[4 * i]) + o.x);
+                        ra[4 * i + 1] = __float_as_uint(__uint_as_float(ra[4 * i + 1]) + o.y);
+                        ra[4 * i + 2] = __float_as_uint(__uint_as_float(ra[4 * i + 2]) + o.z);
+                        ra[4 * i + 3] = __float_as_uint(__uint_as_float(ra[4 * i + 3]) + o.w);
+                    }
+                }
                 mlp_columns<16>(ra, c * 16, b1s, w2p, acc);
                 c += 2;
                 if (c < n16) {
                     tmem_wait_ld();
                     reg_fence16(rb);
-                    if (c + 2 < n16) tmem_ld_x16(t_row + (c + 2) * 16, ra);
+                    if (c + 2 < n16) tmem_ld_x16(t_row + own_c0 + (c + 2) * 16, ra);
+                    if (k_split == 2) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const float4 o = recv[(c * 4 + i) * kTileM + row];
+                            rb[4 * i] = __float_as_uint(__uint_as_float(rb[4 * i]) + o.x);
+                            rb[4 * i + 1] = __float_as_uint(__uint_as_float(rb[4 * i + 1]) + o.y);
+                            rb[4 * i + 2] = __float_as_uint(__uint_as_float(rb[4 * i + 2]) + o.z);
+                            rb[4 * i + 3] = __float_as_uint(__uint_as_float(rb[4 * i + 3]) + o.w);
+                        }
+                    }
                     mlp_columns<16>(rb, c * 16, b1s, w2p, acc);
                     c += 2;
                 }
@@ -212,7 +273,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_pfull);
         } else {
-            ok = mbar_wait(bar_pfull, 0, abort_flag) && ok;
+            mbar_wait(bar_pfull, 0, abort_flag);
             const float4 *src = reinterpret_cast<const float4 *>(part + row * kMaxHeads);
             const float4 pa = src[0], pb = src[1];
             s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
@@ -233,16 +294,17 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
     }
+    // If this launch was allowed to start before the kernel ahead of it had finished (consecutive decode
+    // steps), it still completes after it: every thread waits here.
+    griddep_wait();
     if (rank != 0 || warp < 2 || warp >= 6 || m_tile >= p.blocks_per_layer) return;
 
     // ------------------------------------------------------------ first CTA: total, scores, keep bits
     {
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
         float s[kMaxHeads];
 #pragma unroll
         for (int h = 0; h < kMaxHeads; ++h) s[h] = __ldg(p.b2 + layer * kMaxHeads + h);
-        for (int r = 0; r < n_split; ++r) {
+        for (int r = 0; r < n_ctas; ++r) {
             const float4 *src = reinterpret_cast<const float4 *>(xpart + (r * kTileM + row) * kMaxHeads);
             const float4 pa = src[0], pb = src[1];
             s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
