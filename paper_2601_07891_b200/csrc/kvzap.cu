@@ -280,8 +280,10 @@ static void make_launch(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attrs, dim
 // scores [n_layers][n_tokens][H]; maskbits != nullptr fuses the threshold/window test.
 static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
-                                 float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1)
+                                 float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1,
+                                 const DecodeFuse *fuse = nullptr, bool *fused = nullptr)
 {
+    if (fused) *fused = false;
     // Early start.  When the grid fills the machine (one CTA per SM), this kernel is allowed to start
     // while the kernels ahead of it in the stream -- the previous call's scoring kernel finishing its
     // last tiles, and its compaction -- are still running: its CTAs take the SMs as they become free.
@@ -339,7 +341,16 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         ctx->last_scores = scores;
         ctx->last_scores_bytes = sbytes;
         const int n_ctas = ctx->split_n * ctx->split_k;
-        const bool early = !ctx->profiling && !clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count;
+        // only the fused decode step is started early: its clusters order themselves through `done`
+        DecodeFuse f;
+        memset(&f, 0, sizeof f);
+        const bool fuse_ok = fuse != nullptr && !ctx->profiling && n_ctas == 4;
+        if (fuse_ok) {
+            f = *fuse;
+            f.enabled = 1;
+            if (fused) *fused = true;
+        }
+        const bool early = fuse_ok && !clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count;
         ctx->last_score_early = early;
         {
             ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
@@ -348,7 +359,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * n_ctas)), dim3(kScoreThreads),
                         ctx->split_smem, stream, early, n_ctas);
             KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n,
-                                               ctx->split_k));
+                                               ctx->split_k, f));
         }
         ctx->launches += 1;
         return KVZAP_OK;
@@ -647,7 +658,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         const int n_split = two_by_two ? 2 : 4, k_split = two_by_two ? 2 : 1, ns = c.hidden / n_split;
         int stages = kMaxStages;
         for (; stages >= 2; --stages)
-            if (static_cast<int>(split_smem_layout(ns, stages, 4).total) <= budget) break;
+            if (static_cast<int>(split_smem_layout(ns, stages, 4).total) <= budget - 4096) break;   // 4 KB static
         if (stages >= 2 && ns % 16 == 0 && ns <= 256) {
             ctx->split_stages = stages;
             ctx->split_smem = split_smem_layout(ns, stages, 4).total + 1024;
@@ -1029,6 +1040,9 @@ struct kvzap_cache {
     float *scores = nullptr;        // [L][B][H] scratch when the caller does not want the scores
     int64_t n_lists = 0;
     int step_parity = 0;
+    // fused decode steps: per-cluster count of completed steps on the device, and the host's view of it
+    int32_t *done = nullptr;             // [n_layers * ceil(n_seqs / 128)]
+    std::vector<int32_t> steps_done;     // per layer
 };
 
 namespace kvzap {
@@ -1202,6 +1216,9 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.prefix_len), sizeof(int32_t) * n, true);
     alloc(reinterpret_cast<void **>(&v.page_table), sizeof(int32_t) * n * max_pages_per_list, true);
     alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
+    alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
+          true);
+    cache->steps_done.assign(c.n_layers, 0);
     // two halves used by alternate steps when the caller does not ask for the scores
     alloc(reinterpret_cast<void **>(&cache->scores), 2 * sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
           false);
@@ -1222,7 +1239,7 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     cudaDeviceSynchronize();
     cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
     cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
-    cudaFree(cache->v.page_cursor); cudaFree(cache->scores);
+    cudaFree(cache->v.page_cursor); cudaFree(cache->scores); cudaFree(cache->done);
     delete cache;
     return KVZAP_OK;
 }
@@ -1247,14 +1264,33 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
         scores = cache->scores + (cache->step_parity ? static_cast<size_t>(c.n_layers) * cache->v.n_seqs * c.n_kv_heads : 0);
         cache->step_parity ^= 1;
     }
+    // The whole step in one launch when the few-token scoring kernel applies: the cache update runs in
+    // its idle warps.  Needs a window (else the new score decides at once) and every layer of the range
+    // at the same step count.
+    DecodeFuse fuse;
+    memset(&fuse, 0, sizeof fuse);
+    bool can_fuse = cache->v.window > 0 && c.hidden > 0;
+    for (int l = layer_begin; l < layer_end && can_fuse; ++l)
+        can_fuse = cache->steps_done[l] == cache->steps_done[layer_begin];
+    if (can_fuse) {
+        fuse.expect = cache->steps_done[layer_begin];
+        fuse.c = cache->v;
+        fuse.K_new = static_cast<const uint4 *>(K_new);
+        fuse.V_new = static_cast<const uint4 *>(V_new);
+        fuse.tau = tau;
+        fuse.done = cache->done;
+    }
+    bool fused = false;
     kvzap_status st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
-                                   0.0f, 0, stream);
+                                   0.0f, 0, stream, 1, can_fuse ? &fuse : nullptr, &fused);
     if (st != KVZAP_OK) return st;
+    if (fused) {
+        for (int l = layer_begin; l < layer_end; ++l) cache->steps_done[l] += 1;
+        return KVZAP_OK;
+    }
     const int64_t n_groups = static_cast<int64_t>(n_layers) * cache->v.n_seqs * c.n_kv_heads;
     const int64_t threads = n_groups * kDecodeLanes;
-    // a grid that is resident all at once beside the scoring kernel (one CTA per SM), walking the lists
     int64_t blocks = (threads + kDecodeThreads - 1) / kDecodeThreads;
-    if (blocks > ctx->sm_count) blocks = ctx->sm_count;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_DECODE_UPDATE, stream);
         cudaLaunchConfig_t cfg;

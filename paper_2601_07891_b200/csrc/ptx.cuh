@@ -247,6 +247,18 @@ __host__ __device__ __forceinline__ uint32_t umma_idesc_bf16_f32(uint32_t M, uin
            | ((M >> 4) << 24);  // M / 16
 }
 
+// ---------------------------------------------------------------- flags in global memory
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t *p)
+{
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int32_t *p, int32_t v)
+{
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
 // ---------------------------------------------------------------- programmatic dependent launch
 // A kernel launched with the programmatic-stream-serialization attribute may start once every CTA
 // of the kernel before it in the stream has executed griddep_launch_dependents() (or exited);

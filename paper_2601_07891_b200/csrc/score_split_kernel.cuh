@@ -19,9 +19,26 @@
 // epilogue (TMEM lane quarter = warp % 4; the two warps of a quarter take alternate 16-column chunks).
 #pragma once
 
+#include "decode_kernels.cuh"
 #include "score_kernel.cuh"
 
 namespace kvzap {
+
+// Decode step fused into the scoring launch (enabled != 0): while the MMAs run, the epilogue warps
+// of a cluster do the cache update of the cluster's own lists -- 128 sequences x H heads of one layer,
+// a quarter per CTA -- exactly as decode_update_kernel does (the token that leaves the window is
+// judged by its buffered score, so nothing here needs the new scores); the cluster's first CTA puts
+// the new scores into the score buffer at the very end.  Consecutive steps may overlap in time
+// (the next launch starts as SMs become free): `done[cluster]` counts the steps a cluster has
+// completed, and a cluster touches the cache only after its predecessor has published `expect`.
+struct DecodeFuse {
+    int32_t enabled;
+    int32_t expect;
+    CacheView c;
+    const uint4 *K_new, *V_new;     // [n_layers_call][B][H][D] bf16
+    float tau;
+    int32_t *done;                  // [n_layers * tiles_per_layer]
+};
 
 struct SplitSmemLayout {
     uint32_t stage_bytes, stages_end, w2s, b1s, part, xpart, bars, total;
@@ -45,8 +62,10 @@ __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stage
 // A CTA ends up owning Ns / k_split hidden units: xpart and the W2 / b1 slices are sized for those.
 __global__ void __maxnreg__(128)
 score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                   const ScoreParams p, const int n_split, const int k_split)
+                   const ScoreParams p, const int n_split, const int k_split, const DecodeFuse f)
 {
+    __shared__ int64_t fuse_dst[256];       // fused decode step: page row of the evicted token (-1 = dropped)
+    __shared__ int64_t fuse_ring[256];      //                     ring row of the list's current slot (-1 = no list)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
@@ -188,6 +207,74 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
         for (int i = etid; i < own_n; i += 256) b1s[i] = __ldg(b1g + i);
         named_barrier_sync(1, 256);
+        if (f.enabled) {
+            // ---- the cache update of this CTA's lists, under the MMAs
+            const CacheView &c = f.c;
+            const int cid = layer * p.tiles_per_layer + m_tile;
+            if (etid == 0) {
+                const long long t0 = clock64();
+                while (ld_acquire_gpu(f.done + cid) != f.expect) {
+                    if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES) { *abort_flag = 1; break; }
+                }
+            }
+            named_barrier_sync(1, 256);
+            const bool go = *abort_flag == 0;
+            const int rows_per_cta = kTileM / n_ctas;
+            // one thread per list: which row leaves, where it goes, which slot the new token takes
+            {
+                const int b_loc = static_cast<int>(rank) * rows_per_cta + etid / kMaxHeads, h = etid % kMaxHeads;
+                const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
+                int64_t dst = -1, ring = -1;
+                if (go && etid < rows_per_cta * kMaxHeads && b < c.n_seqs && h < c.n_heads) {
+                    const int64_t li = (b * c.n_layers + layer) * c.n_heads + h;
+                    const int32_t n = __ldcg(c.n_tokens + li);
+                    const int slot = n % c.window;
+                    ring = li * c.window + slot;
+                    if (n >= c.window && __ldcg(c.score_ring + ring) >= f.tau) {
+                        const int32_t idx = __ldcg(c.prefix_len + li);
+                        const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
+                        int32_t page = -1;
+                        if (page_i >= c.max_pages) {
+                            atomicCAS(p.status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+                        } else if (in_page == 0) {
+                            const int32_t got = atomicAdd(c.page_cursor, 1);
+                            if (got >= c.n_pages_pool) atomicCAS(p.status, 0, 4);
+                            else { page = got; c.page_table[li * c.max_pages + page_i] = got; }
+                        } else {
+                            page = __ldcg(c.page_table + li * c.max_pages + page_i);
+                        }
+                        if (page >= 0) {
+                            dst = static_cast<int64_t>(page) * c.page_tokens + in_page;
+                            c.prefix_len[li] = idx + 1;
+                        }
+                    }
+                    c.n_tokens[li] = n + 1;
+                }
+                fuse_dst[etid] = dst;
+                fuse_ring[etid] = ring;
+            }
+            named_barrier_sync(1, 256);
+            // rows: 16 lanes per list, every lane loads (old row, new row) before it stores
+            {
+                const int grp = etid >> 4, l16 = etid & 15;
+                for (int j = grp; j < rows_per_cta * kMaxHeads; j += 16) {
+                    const int64_t ring = fuse_ring[j], dst = fuse_dst[j];
+                    if (ring < 0) continue;
+                    const int b_loc = static_cast<int>(rank) * rows_per_cta + j / kMaxHeads, h = j % kMaxHeads;
+                    const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
+                    const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+                    for (int u = l16; u < c.row_units; u += 16) {
+                        uint4 ko = make_uint4(0, 0, 0, 0), vo = ko;
+                        if (dst >= 0) { ko = __ldcg(c.k_ring + ring * c.row_units + u); vo = __ldcg(c.v_ring + ring * c.row_units + u); }
+                        const uint4 kn = __ldg(f.K_new + src_row * c.row_units + u);
+                        const uint4 vn = __ldg(f.V_new + src_row * c.row_units + u);
+                        if (dst >= 0) { c.k_pool[dst * c.row_units + u] = ko; c.v_pool[dst * c.row_units + u] = vo; }
+                        c.k_ring[ring * c.row_units + u] = kn;
+                        c.v_ring[ring * c.row_units + u] = vn;
+                    }
+                }
+            }
+        }
         ok = mbar_wait(bar_tfull, 0, abort_flag);
         tc_fence_after_sync();
     }
@@ -312,6 +399,23 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
         const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;
         const bool valid = t < p.n_tokens;
+        if (f.enabled) {
+            // the new token's scores go into the slot it took (n_tokens was advanced by the list's CTA)
+            const CacheView &c = f.c;
+            if (valid && *abort_flag == 0) {
+#pragma unroll
+                for (int h = 0; h < kMaxHeads; ++h) {
+                    if (h < c.n_heads) {
+                        const int64_t li = (t * c.n_layers + layer) * c.n_heads + h;
+                        const int slot = (__ldcg(c.n_tokens + li) - 1) % c.window;
+                        c.score_ring[li * c.window + slot] = s[h];
+                    }
+                }
+            }
+            __threadfence();
+            named_barrier_sync(2, 128);
+            if (threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + layer * p.tiles_per_layer + m_tile, f.expect + 1);
+        }
         if (valid && p.scores != nullptr) {
             float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
             if (p.n_heads == kMaxHeads) {

@@ -142,8 +142,10 @@ def test_config4_qwen3_32b_mlp_128k_paged_one_layer(binding, oracle):
 
 def test_config5_decode_b128_all_layers(binding, oracle):
     """36 layers x 128 sequences, w = 128, 16-token pages, 132 steps so that tokens leave the window.
-    Scores: compared with the oracle on a few (step, layer) pairs.  Evictions and list contents: the
-    decode oracle replays the GPU's own scores for a sample of lists."""
+    All steps are enqueued back to back with no host synchronisation in between and with a different
+    scores buffer per step -- the launch configuration bench.py times, in which consecutive steps
+    overlap on the GPU.  Scores: compared with the oracle on a few (step, layer) pairs.  Evictions and
+    list contents: the decode oracle replays the GPU's own scores for a sample of lists."""
     wl = W["qwen3_8b_decode_b128"]
     L, B, H, D, w, P = wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     n_steps = w + 4
@@ -160,39 +162,51 @@ def test_config5_decode_b128_all_layers(binding, oracle):
     cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, 4)
     rng = np.random.default_rng(5)
     sample_lists = [(int(rng.integers(B)), int(rng.integers(L)), int(rng.integers(H))) for _ in range(48)]
-    sample_lists += [(0, 0, 0), (B - 1, L - 1, H - 1)]
-    dec = oracle.DecodeOracle(B, L, H, D, w)          # only the sampled lists are fed
+    sample_lists += [(0, 0, 0), (B - 1, L - 1, H - 1), (31, 3, 7), (32, 3, 0), (127, 0, 0)]
+    sample_lists = sorted(set(sample_lists))
     check_steps = {0: [0, L - 1], w: [17], n_steps - 1: [5]}
+    Xs, Ks, Vs = [], [], []
     for step in range(n_steps):
-        X = synth.hidden_states(L * B, wl.d_model, 9000 + step, "cuda").view(L, B, wl.d_model)
+        Xs.append(synth.hidden_states(L * B, wl.d_model, 9000 + step, "cuda").view(L, B, wl.d_model))
         Kn, Vn = synth.keys_values(L * B, H, D, 9500 + step, "cuda")
-        Kn, Vn = Kn.view(L, B, H, D), Vn.view(L, B, H, D)
-        scores = torch.empty(L, B, H, dtype=torch.float32, device="cuda")
-        binding.kvzap_decode_step(ctx.handle, cache, 0, L, X, Kn, Vn, wl.tau, scores)
-        torch.cuda.synchronize()
-        s = scores.cpu().numpy()
-        for l in check_steps.get(step, []):
-            want = oracle.score(synth.bits(X[l]), parity.weights_to_oracle(tuple(t.cpu() for t in weights[l])))
-            assert np.abs(s[l] - want).max() <= parity.SCORE_ATOL
-        Kb, Vb = synth.bits(Kn), synth.bits(Vn)
-        for (b, l, h) in set(sample_lists):
-            # feed one head's list: a one-head view of the oracle's per-(b,l) append
+        Ks.append(Kn.view(L, B, H, D))
+        Vs.append(Vn.view(L, B, H, D))
+    scores_all = torch.empty(n_steps, L, B, H, dtype=torch.float32, device="cuda")
+    torch.cuda.synchronize()
+    for step in range(n_steps):                       # no synchronisation between steps
+        binding.kvzap_decode_step(ctx.handle, cache, 0, L, Xs[step], Ks[step], Vs[step], wl.tau, scores_all[step])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    s_all = scores_all.cpu().numpy()
+    for step, layers in check_steps.items():
+        for l in layers:
+            want = oracle.score(synth.bits(Xs[step][l]), parity.weights_to_oracle(tuple(t.cpu() for t in weights[l])))
+            assert np.abs(s_all[step, l] - want).max() <= parity.SCORE_ATOL
+    dec = oracle.DecodeOracle(B, L, H, D, w)          # only the sampled lists are fed
+    idx_b = torch.tensor([x[0] for x in sample_lists], device="cuda")
+    idx_l = torch.tensor([x[1] for x in sample_lists], device="cuda")
+    idx_h = torch.tensor([x[2] for x in sample_lists], device="cuda")
+    for step in range(n_steps):
+        Kb = synth.bits(Ks[step][idx_l, idx_b, idx_h])         # [n_sample, D]
+        Vb = synth.bits(Vs[step][idx_l, idx_b, idx_h])
+        for i, (b, l, h) in enumerate(sample_lists):
             win = dec.window[b][l][h]
-            pos = step
-            win.append((pos, np.float32(s[l, b, h]), Kb[l, b, h].copy(), Vb[l, b, h].copy()))
+            win.append((step, np.float32(s_all[step, l, b, h]), Kb[i].copy(), Vb[i].copy()))
             if len(win) > w:
                 p_, s_, kr, vr = win.popleft()
                 if s_ >= np.float32(wl.tau):
                     dec.prefix[b][l][h].append((p_, kr, vr))
-    assert ctx.poll_status() == 0
     lengths = torch.zeros(B, L, H, dtype=torch.int32, device="cuda")
     binding.kvzap_cache_lengths(ctx.handle, cache, lengths)
     ln = lengths.cpu().numpy()
     assert (ln >= w).all() and (ln <= n_steps).all()
+    # every list: rows held = window + tokens that left it with a score >= tau (from the GPU's own scores)
+    kept_exit = (s_all[:n_steps - w] >= np.float32(wl.tau)).sum(axis=0)          # [L, B, H]
+    np.testing.assert_array_equal(ln, w + kept_exit.transpose(1, 0, 2))
     K_out = torch.zeros(n_steps, D, dtype=torch.bfloat16, device="cuda")
     V_out = torch.zeros_like(K_out)
     n_rows = torch.zeros(1, dtype=torch.int32, device="cuda")
-    for (b, l, h) in set(sample_lists):
+    for (b, l, h) in sample_lists:
         binding.kvzap_cache_export(ctx.handle, cache, b, l, h, K_out, V_out, n_rows)
         torch.cuda.synchronize()
         n = int(n_rows.item())
