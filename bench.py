@@ -30,7 +30,7 @@ UNIT = "tokens/s/layer"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes); None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 277.6e6}
+NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 277.1e6, "qwen3_8b_decode_b128": 225.5e6}
 
 
 def load_peaks():
@@ -421,7 +421,7 @@ def run_decode(args, wl, env):
     achieved = bytes_layer * L / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
-                "kernel": "decode step (score_kernel + decode_update_kernel)", "peak_source": peak_src,
+                "kernel": "score_split_kernel (scoring + cache update in one launch)", "peak_source": peak_src,
                 "kernel_ms": ms_per_step, "algorithmic_bytes_per_step": bytes_layer * L}
     config = {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
               "n_kv_heads": H, "head_dim": D, "n_layers": L, "batch": B, "tau": wl.tau, "window": w, "page_tokens": P,

@@ -20,6 +20,20 @@
  *     Calls enqueue work on it and return without synchronising.  A context
  *     must not be used from two streams at the same time: its scratch is
  *     shared by all calls.
+ *   - Work of consecutive calls on one stream may overlap on the GPU: the kernels
+ *     are launched so that a scoring kernel can start on SMs that the previous
+ *     call's kernels have already left, and the compaction of one call runs
+ *     beside the scoring kernel of the next.  This is invisible to stream
+ *     order: every output of a call is complete before any later operation on
+ *     the stream (a copy, another library's kernel, an event) starts.  Two
+ *     rules follow for the caller.  (1) Inputs of a call (hidden states,
+ *     weights, K, V) must be complete in stream order before the PREVIOUS
+ *     kvzap call on that stream was enqueued, or be produced by an ordinary
+ *     kernel or copy enqueued between the two calls (which then separates
+ *     them); a producer that itself signals "dependents may start" before it
+ *     has finished must not sit directly ahead of a kvzap call.  (2) Passing
+ *     the same scores buffer to two consecutive calls is allowed; the library
+ *     then launches the second call's scoring kernel without overlap.
  *   - Errors the host can see (bad argument, unsupported shape) return at once
  *     and launch nothing.  Conditions only the device can see set a status
  *     word that kvzap_poll_status() reads; kernels never trap and every
@@ -84,7 +98,7 @@ const char *kvzap_last_error(const kvzap_ctx *ctx);
 /*
  * Installs one layer's surrogate (Method, "KVzap": a linear layer or a
  * two-layer MLP; Appendix B: W1 in R^{D_h x D_h/8}, W2 in R^{D_h/8 x H}).
- * Matrices are bf16, stored [out, in] row-major; biases are fp32, NULL = zero.
+ * Matrices are bf16, stored [out, in] row-major, 16-byte aligned; biases are fp32, NULL = zero.
  *   KVzap-Linear (cfg.hidden == 0): W1 [H, d_model], b1 [H]; W2 and b2 must be NULL.
  *   KVzap-MLP:                      W1 [hidden, d_model], b1 [hidden],
  *                                   W2 [H, hidden],       b2 [H].
@@ -223,6 +237,11 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache);
  *   scores_out   [layer_end-layer_begin, n_seqs, H] fp32 or NULL
  * A full pool or page table drops the row that needed the page and sets the
  * status word to KVZAP_ERR_OOM_PAGES.
+ * With the MLP surrogate, window > 0 and at most 128 sequences per 128-token
+ * tile of a few-layer-by-few-tile launch (the usual decode shape), the whole
+ * step is ONE kernel launch: the cache update runs in the scoring kernel's
+ * otherwise idle warps, and consecutive steps overlap on the GPU when their
+ * scores_out buffers differ (or are NULL).
  */
 kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
                                const void *hidden, const void *K_new, const void *V_new, float tau,
