@@ -440,25 +440,32 @@ def run_decode(args, wl, env):
     return line
 
 
-def run_ours(args, wl):
+def make_env(backend="nccl"):
+    """Process-group plumbing of the N > 1 run: replicas only, so all it carries is the barrier around the
+    timed region and the maximum over ranks of the timed duration.  `backend="gloo"` runs the same code
+    on CPU tensors (used by the multi-process CPU test)."""
     import torch
     import torch.distributed as dist
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
+    on_gpu = backend == "nccl"
+    dev = torch.device("cuda", local_rank) if on_gpu else torch.device("cpu")
+    if on_gpu:
+        torch.cuda.set_device(local_rank)
     if world > 1:
-        # replicas only: the path needs no exchange; the process group carries the barrier and the max
-        dist.init_process_group("nccl", device_id=dev)
+        # the path needs no exchange between ranks: no collective moves any data of the method
+        if on_gpu:
+            dist.init_process_group(backend, device_id=dev)
+        else:
+            dist.init_process_group(backend)
 
     def barrier():
         if world > 1:
             dist.barrier()
-        torch.cuda.synchronize()
+        if on_gpu:
+            torch.cuda.synchronize()
 
     def max_over_ranks(ms):
         if world > 1:
@@ -467,7 +474,20 @@ def run_ours(args, wl):
             return float(t.item())
         return ms
 
-    env = {"dev": dev, "rank": rank, "world": world, "barrier": barrier, "max_over_ranks": max_over_ranks}
+    def close():
+        if world > 1:
+            dist.destroy_process_group()
+
+    return {"dev": dev, "rank": rank, "world": world, "barrier": barrier, "max_over_ranks": max_over_ranks,
+            "close": close}
+
+
+def run_ours(args, wl):
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    env = make_env("nccl")
+    rank, world = env["rank"], env["world"]
     line = run_decode(args, wl, env) if wl.decode_steps > 0 else run_prefill(args, wl, env)
     if rank == 0 and world == 1 and not args.skip_cpu and wl.decode_steps == 0:
         # the oracle on the host cores, bounded sample
@@ -477,8 +497,7 @@ def run_ours(args, wl):
                                 "sample": "one layer, first %d tokens: scoring + mask + compaction (%.1f s)" % (n_sample, dt)}
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    env["close"]()
 
 
 def main():
