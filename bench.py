@@ -193,11 +193,15 @@ def run_prefill(args, wl, env):
     # needed); beyond ~60 GB the layers rotate over fewer input sets (weights stay distinct per layer)
     per_layer_bytes = n_tokens * wl.d_model * 2 + 4 * H * n_tokens * D * 2
     n_sets = L if L * per_layer_bytes <= 60e9 else max(2, int(60e9 // per_layer_bytes))
+    # a small workload (config 1: 56 MB per layer) would otherwise run out of the 126 MB L2: rotate over
+    # enough input/output sets that 2.5 x L2 lies between two uses of the same buffer
+    n_sets = max(n_sets, int(-(-2.5 * 126e6 // per_layer_bytes)))
     Xs, Ks, Vs, Kos, Vos, lens, scs, tabs, used = [], [], [], [], [], [], [], [], []
     max_pages = (T // P + 2) if P else 0
     pool_pages = (H * B * (T // P + 2)) // 2 if P else 0       # room for half of all rows per layer set
     for l in range(L):
         ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
+    for l in range(max(L, n_sets)):
         lens.append(torch.zeros(B, H, dtype=torch.int32, device=dev))
         if l >= n_sets:
             for lst in (Xs, Ks, Vs, Kos, Vos, scs, tabs, used):
@@ -221,14 +225,20 @@ def run_prefill(args, wl, env):
         scs.append(torch.empty(n_tokens, H, dtype=torch.float32, device=dev))
     torch.cuda.synchronize()
 
+    n_bufs = len(Xs)
+    turn = [0]
+
     def step():
         for l in range(L):
+            i = (turn[0] + l) % n_bufs          # layer l's buffers; with more sets than layers they rotate per step
             if P:
-                binding.kvzap_prefill_fused_paged(ctx.handle, l, Xs[l], Ks[l], Vs[l], cu, B, wl.tau, wl.window,
-                                                  Kos[l], Vos[l], P, 0, tabs[l], lens[l], used[l], scs[l])
+                binding.kvzap_prefill_fused_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau, wl.window,
+                                                  Kos[i], Vos[i], P, 0, tabs[i], lens[i], used[i], scs[i])
             else:
-                binding.kvzap_prefill_fused(ctx.handle, l, Xs[l], Ks[l], Vs[l], cu, B, wl.tau, wl.window,
-                                            Kos[l], Vos[l], lens[l], scs[l])
+                binding.kvzap_prefill_fused(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau, wl.window,
+                                            Kos[i], Vos[i], lens[i], scs[i])
+        if n_bufs > L:
+            turn[0] += L
 
     n_warm = args.warmup if args.layers > 0 else max(args.warmup, 3)
     for _ in range(n_warm):
@@ -255,21 +265,27 @@ def run_prefill(args, wl, env):
     value = world * n_tokens / (layer_ms * 1e-3)
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during the timed region")
-    kept_rows = float(sum(int(x.sum().item()) for x in lens)) / L          # kept (head, token) rows per layer
+    kept_rows = float(sum(int(x.sum().item()) for x in lens[:n_bufs])) / n_bufs   # kept (head, token) rows per layer
 
     # The two kernels of a layer, each timed alone with CUDA events around a loop of launches through
     # the public calls (scoring only; mask + compaction on the scores just computed).
     sync = torch.cuda.synchronize
     n_rep = max(1, min(args.steps, 5))
-    score_ms = _timed(lambda: [binding.kvzap_score(ctx.handle, l, Xs[l], scs[l]) for l in range(L)], n_rep, sync) / L
+    def score_only():
+        for l in range(L):
+            i = (turn[0] + l) % n_bufs
+            binding.kvzap_score(ctx.handle, l, Xs[i], scs[i])
+        if n_bufs > L:
+            turn[0] += L
+    score_ms = _timed(score_only, n_rep, sync) / L
     if P:
         prune = lambda: [binding.kvzap_prune_prefill_paged(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
                                                            Kos[l], Vos[l], P, 0, tabs[l], lens[l], used[l])
-                         for l in range(L)]
+                         for l in range(n_bufs)]
     else:
         prune = lambda: [binding.kvzap_prune_prefill(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
-                                                     Kos[l], Vos[l], lens[l]) for l in range(L)]
-    prune_ms = _timed(prune, n_rep, sync) / L
+                                                     Kos[l], Vos[l], lens[l]) for l in range(n_bufs)]
+    prune_ms = _timed(prune, n_rep, sync) / n_bufs
 
     peaks, peak_src = load_peaks()
     flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer = _roofline_times(wl, n_tokens, kept_rows, peaks)
@@ -299,8 +315,9 @@ def run_prefill(args, wl, env):
              "kept_fraction": kept_rows / (H * n_tokens)}
     config = {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
               "n_kv_heads": H, "head_dim": D, "n_layers": L, "batch": B, "seq_len": T, "tau": wl.tau,
-              "window": wl.window, "page_tokens": P, "input_sets": n_sets,
-              "l2": "inputs larger than L2 (distinct resident buffers per layer)",
+              "window": wl.window, "page_tokens": P, "input_sets": n_bufs,
+              "l2": "inputs larger than L2 (distinct resident buffers per layer; small workloads rotate over "
+                    "enough sets that 2.5 x L2 lies between two uses of a buffer)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

@@ -80,7 +80,7 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
                 app_v = c.v_ring + (li * c.window + slot) * c.row_units;
             }
         } else {
-            append = scores[src_row] >= tau;
+            append = __ldcg(scores + src_row) >= tau;
             app_k = K_new + src_row * c.row_units;
             app_v = V_new + src_row * c.row_units;
         }
@@ -137,7 +137,7 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
         }
         if (live && gl == 0) {
             c.n_tokens[li] = n + 1;
-            if (c.window > 0 && !rows_first) c.score_ring[li * c.window + slot] = scores[src_row];
+            if (c.window > 0 && !rows_first) c.score_ring[li * c.window + slot] = __ldcg(scores + src_row);
         }
     }
     if (rows_first) {
@@ -152,7 +152,7 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
                 const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
                 const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
                 const int slot = (c.n_tokens[li] - 1) % c.window;      // the slot this thread filled above
-                c.score_ring[li * c.window + slot] = scores[src_row];
+                c.score_ring[li * c.window + slot] = __ldcg(scores + src_row);
             }
         }
     }

@@ -291,7 +291,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // kernels write, (b) every scoring CTA waits for the kernel ahead of it before it exits, so a
     // free SM implies that everything two launches back has completed, and the mask slice written
     // here was last read at least kMaskRing launches back, (c) the scores buffer is checked below.
-    // A smaller grid is launched the ordinary way.
+    // A smaller grid (or a scores buffer shared with the previous call) is started early as well, but
+    // its epilogue waits for the kernel ahead before its first store (wait_before_write): loads and
+    // MMAs of several small calls then overlap, and nothing is written while an earlier call may
+    // still use it.
     const kvzap_config &c = ctx->cfg;
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
     // Few tiles (a decode step: one tile per layer): split every tile's hidden units over a cluster, so
@@ -424,13 +427,15 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         cudaLaunchAttribute attrs[2];
         if (pair) {
             const int n_clusters = static_cast<int>(n_tiles < ctx->pair_clusters ? n_tiles : ctx->pair_clusters);
-            const bool early = !ctx->profiling && !scores_clash && 2 * n_clusters >= ctx->sm_count / 2 * 2;
+            const bool early = !ctx->profiling;
+            p.wait_before_write = (scores_clash || 2 * n_clusters < ctx->sm_count / 2 * 2) ? 1 : 0;
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(2 * n_clusters)), dim3(kScoreThreads), sc.smem, stream,
                         early, 2);
             KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, true>, tmap_x, sc.tmap_w, p));
         } else {
             const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
-            const bool early = !ctx->profiling && !scores_clash && grid >= ctx->sm_count;
+            const bool early = !ctx->profiling;
+            p.wait_before_write = (scores_clash || grid < ctx->sm_count) ? 1 : 0;
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid)), dim3(kScoreThreads), sc.smem, stream, early, 1);
             if (c.hidden > 0)
                 KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, false>, tmap_x, sc.tmap_w, p));

@@ -73,8 +73,8 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
         const int r = static_cast<int>(t - blk * kBlockTokens);       // 0..127 bits of this block
         for (int i = 0; i < 4; ++i) {
             const int lo = i * 32;
-            if (r >= lo + 32) n += __popc(w[i]);
-            else if (r > lo) n += __popc(w[i] & ((1u << (r - lo)) - 1u));
+            if (r >= lo + 32) n += __popc(__ldcg(w + i));
+            else if (r > lo) n += __popc(__ldcg(w + i) & ((1u << (r - lo)) - 1u));
         }
     }
     return n;
@@ -138,7 +138,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             const int64_t blk = base + tid;
             int32_t cnt = 0;
             if (blk < n_blocks) {
-                const uint4 w = *reinterpret_cast<const uint4 *>(maskbits + static_cast<int64_t>(h) * n_words + blk * 4);
+                const uint4 w = __ldcg(reinterpret_cast<const uint4 *>(maskbits + static_cast<int64_t>(h) * n_words + blk * 4));
                 cnt = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
             }
             int32_t total;
@@ -350,7 +350,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     if (multi) s0 = cu_seqlens[seq_of_token(cu_seqlens, n_seqs, t0)];
     int32_t total = 0, before_s0 = 0;
     for (int64_t i = tid; i < blk0 * 4; i += kDenseThreads) {
-        const uint32_t w = words[i];
+        const uint32_t w = __ldcg(words + i);     // not a read-only-data load: it must stay behind griddep_wait()
         const int c = __popc(w);
         total += c;
         const int64_t lo = i * 32;
@@ -371,7 +371,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     const int group = tid >> 4, gl = tid & 15;
     constexpr int kGroups = kDenseThreads / 16;
     for (int64_t blk = blk0; blk < blk1; ++blk) {
-        const uint4 wv = *reinterpret_cast<const uint4 *>(words + blk * 4);
+        const uint4 wv = __ldcg(reinterpret_cast<const uint4 *>(words + blk * 4));
         const uint32_t w0 = wv.x, w1 = wv.y, w2 = wv.z, w3 = wv.w;
         const int cnt = __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
         const int64_t blk_start = blk * kBlockTokens;

@@ -68,6 +68,7 @@ struct ScoreParams {
     int32_t window_keep;  // 1: tokens inside the window are kept (Algorithm 1); 0: they are left out of the mask
     float tau;
     int32_t *status;      // device status word
+    int32_t wait_before_write;    // 1: the epilogue waits for the kernel ahead in the stream before its first store
     int32_t *tile_counter;        // work tiles handed out beyond the first one of every CTA (or pair); starts at 0
     int32_t *tile_counter_reset;  // the counter of the launch after next: set to 0 by this launch
 };
@@ -458,6 +459,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
         const bool active = kMlp || hsel == 0;
         uint32_t acc_it = 0, tile_it = 0, epi_it = 0;
         int cur_layer = -1;
+        bool waited = false;
         bool ok = true;
         uint32_t tempty_addr[2] = {bar_tempty, bar_tempty + 8};
         if constexpr (kPair) {
@@ -573,6 +575,12 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                     }
                 }
                 if (hsel == 0 && m_tile < p.blocks_per_layer) {
+                    if (p.wait_before_write && !waited) {
+                        // started early on a machine that was not full: the buffers written below may still
+                        // be in use by the calls before this one until the kernel ahead has completed
+                        griddep_wait();
+                        waited = true;
+                    }
                     const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;      // row inside the layer
                     const bool valid = t < p.n_tokens;
                     if (valid && p.scores != nullptr) {
