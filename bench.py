@@ -227,16 +227,21 @@ def run_prefill(args, wl, env):
 
     n_bufs = len(Xs)
     turn = [0]
+    # the calls of a step, marshalled once (same entry points, same arguments every step)
+    calls = {}
+    for l in range(L):
+        for i in (range(n_bufs) if n_bufs > L else [l]):
+            if P:
+                calls[(l, i)] = binding.prepare_prefill_fused_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
+                                                                    wl.window, Kos[i], Vos[i], P, 0, tabs[i], lens[i],
+                                                                    used[i], scs[i])
+            else:
+                calls[(l, i)] = binding.prepare_prefill_fused(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
+                                                              wl.window, Kos[i], Vos[i], lens[i], scs[i])
 
     def step():
         for l in range(L):
-            i = (turn[0] + l) % n_bufs          # layer l's buffers; with more sets than layers they rotate per step
-            if P:
-                binding.kvzap_prefill_fused_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau, wl.window,
-                                                  Kos[i], Vos[i], P, 0, tabs[i], lens[i], used[i], scs[i])
-            else:
-                binding.kvzap_prefill_fused(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau, wl.window,
-                                            Kos[i], Vos[i], lens[i], scs[i])
+            calls[(l, (turn[0] + l) % n_bufs)]()   # layer l's buffers; with more sets than layers they rotate per step
         if n_bufs > L:
             turn[0] += L
 
@@ -395,11 +400,12 @@ def run_decode(args, wl, env):
     scores = [torch.empty(L, B, H, dtype=torch.float32, device=dev) for _ in range(n_sets)]
     it = [0]
 
+    dcalls = [binding.prepare_decode_step(ctx.handle, cache, 0, L, Xs[i], KVs[i][0].view(L, B, H, D),
+                                          KVs[i][1].view(L, B, H, D), wl.tau, scores[i]) for i in range(n_sets)]
+
     def step():
-        i = it[0] % n_sets
+        dcalls[it[0] % n_sets]()
         it[0] += 1
-        binding.kvzap_decode_step(ctx.handle, cache, 0, L, Xs[i], KVs[i][0].view(L, B, H, D), KVs[i][1].view(L, B, H, D),
-                                  wl.tau, scores[i])
 
     for _ in range(w):                # fill the window: from here on every step decides one token per list
         step()

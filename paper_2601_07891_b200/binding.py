@@ -244,6 +244,50 @@ def kvzap_cache_import(handle, cache, prefix_len, page_table, next_free_page, st
                                              _stream(stream)))
 
 
+class PreparedCall:
+    """One C entry point with its arguments marshalled once.  For loops that repeat the same call on the
+    same buffers (a benchmark step, a serving loop with fixed buffers): calling it costs one ctypes
+    call instead of re-wrapping a dozen tensors.  The tensors are kept alive by the object; the
+    stream is the one current when it was prepared (or the one given)."""
+
+    __slots__ = ("_fn", "_args", "_handle", "_keep")
+
+    def __init__(self, name, handle, args, keep):
+        self._fn = getattr(load(), name)
+        self._args = args
+        self._handle = handle
+        self._keep = keep
+
+    def __call__(self):
+        st = self._fn(*self._args)
+        if st != KVZAP_OK:
+            _check(self._handle, st)
+
+
+def prepare_prefill_fused(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                          scores_out=None, stream=None) -> PreparedCall:
+    """kvzap_prefill_fused with pre-marshalled arguments (see PreparedCall)."""
+    args = (handle, layer, _ptr(hidden), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_out),
+            _ptr(V_out), _ptr(lengths), _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_prefill_fused", handle, args, (hidden, K, V, cu_seqlens, K_out, V_out, lengths, scores_out))
+
+
+def prepare_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                                first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None) -> PreparedCall:
+    args = (handle, layer, _ptr(hidden), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_pool),
+            _ptr(V_pool), K_pool.shape[0], page_tokens, first_page, _ptr(page_table), page_table.shape[1], _ptr(lengths),
+            _ptr(n_pages_used), _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_prefill_fused_paged", handle, args,
+                        (hidden, K, V, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used, scores_out))
+
+
+def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None,
+                        stream=None) -> PreparedCall:
+    args = (handle, cache, layer_begin, layer_end, _ptr(hidden), _ptr(K_new), _ptr(V_new), tau, _ptr(scores_out),
+            _stream(stream))
+    return PreparedCall("kvzap_decode_step", handle, args, (hidden, K_new, V_new, scores_out))
+
+
 KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3, "decode_update": 4}
 
 

@@ -69,6 +69,10 @@ struct kvzap_ctx {
     int32_t *status_dev = nullptr;
     int32_t *status_host = nullptr;  // pinned
     int64_t launches = 0;
+    // tensor maps of recently used hidden-state buffers (encoding one costs about as much as a launch)
+    struct TmapEntry { const void *base; int64_t rows; int32_t slabs; CUtensorMap map; };
+    std::vector<TmapEntry> tmap_cache;
+    size_t tmap_next = 0;
     // optional per-kernel timing (kvzap_set_profiling)
     bool profiling = false;
     struct ProfRec { int kind; cudaEvent_t start, stop; };
@@ -194,14 +198,18 @@ struct ProfScope {
 
 struct DeviceGuard {
     int prev = -1;
-    bool ok = true;
+    bool ok = true, changed = false;
     explicit DeviceGuard(int dev)
     {
-        ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+        ok = cudaGetDevice(&prev) == cudaSuccess;
+        if (ok && prev != dev) {           // the usual case (already current) costs one query
+            ok = cudaSetDevice(dev) == cudaSuccess;
+            changed = true;
+        }
     }
     ~DeviceGuard()
     {
-        if (prev >= 0) cudaSetDevice(prev);
+        if (changed && prev >= 0) cudaSetDevice(prev);
     }
 };
 
@@ -240,6 +248,24 @@ static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seq
 }
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Tensor map of hidden states [slabs][rows][d_model] (box 128 x 64), from a small cache keyed by the
+// buffer's address and shape.
+static kvzap_status hidden_tmap(kvzap_ctx *ctx, CUtensorMap *out, const void *base, int64_t rows, int32_t slabs)
+{
+    for (const auto &e : ctx->tmap_cache)
+        if (e.base == base && e.rows == rows && e.slabs == slabs) { *out = e.map; return KVZAP_OK; }
+    kvzap_ctx::TmapEntry e;
+    e.base = base; e.rows = rows; e.slabs = slabs;
+    kvzap_status st = make_tmap(ctx, &e.map, base, static_cast<uint64_t>(rows), static_cast<uint64_t>(ctx->cfg.d_model),
+                                kTileM, static_cast<uint64_t>(slabs));
+    if (st != KVZAP_OK) return st;
+    constexpr size_t kEntries = 128;
+    if (ctx->tmap_cache.size() < kEntries) ctx->tmap_cache.push_back(e);
+    else { ctx->tmap_cache[ctx->tmap_next] = e; ctx->tmap_next = (ctx->tmap_next + 1) % kEntries; }
+    *out = e.map;
+    return KVZAP_OK;
+}
 
 static uint32_t *next_mask_slice(kvzap_ctx *ctx)
 {
@@ -301,8 +327,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // that the launch fills the machine and every CTA reads only its own slice of W1.
     if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count) {
         CUtensorMap tmap_x;
-        kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens),
-                                    static_cast<uint64_t>(c.d_model), kTileM, static_cast<uint64_t>(n_layers));
+        kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
         if (st != KVZAP_OK) return st;
         ScoreParams p;
         memset(&p, 0, sizeof p);
@@ -373,8 +398,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     const int64_t tiles_per_layer = pair ? (blocks_per_layer + 1) / 2 : blocks_per_layer;
     const int64_t n_tiles = tiles_per_layer * n_layers;
     CUtensorMap tmap_x;
-    kvzap_status st = make_tmap(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model),
-                                kTileM, static_cast<uint64_t>(n_layers));
+    kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
     if (st != KVZAP_OK) return st;
     ScoreParams p;
     memset(&p, 0, sizeof p);
