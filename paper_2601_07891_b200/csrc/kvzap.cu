@@ -475,14 +475,16 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
 // Dense-ragged compaction over the mask words in `mask` (one kernel, no scan pass).
 static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, void *K_out,
-                                      void *V_out, int32_t *lengths, cudaStream_t stream)
+                                      void *V_out, int32_t *lengths, cudaStream_t stream, bool beside_scoring = true)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     const int64_t n_words = n_blocks * 4;
     // A grid that is resident all at once, next to the scoring kernel's CTAs: the MLP scoring kernel
     // leaves registers for two of these CTAs per SM, the Linear one for several.
-    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (c.hidden > 0 ? 2 : 6);
+    // On its own (kvzap_prune_prefill) the kernel fills every SM instead: eight CTAs each.
+    const int per_sm = !beside_scoring ? 8 : (c.hidden > 0 ? 2 : 6);
+    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * per_sm;
     int64_t chunks = max_ctas / c.n_kv_heads;
     if (chunks < 1) chunks = 1;
     if (chunks > n_blocks) chunks = n_blocks;
@@ -816,7 +818,7 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
-    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
 }
 
 kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
