@@ -1,0 +1,84 @@
+"""Calls enqueued back to back, without host synchronisation, give the same bits as calls made one
+at a time.
+
+Consecutive calls overlap on the GPU (a scoring kernel starts while the previous call's kernels are
+still running, the compaction runs beside the next scoring kernel).  These tests run the same fused
+prefill calls both ways on the same inputs -- several buffer sets in rotation, and also with ONE
+scores buffer shared by all calls -- and compare every output bit for bit.  Shapes cover a grid
+that fills the machine (CTA pairs and one-CTA tiles) and grids far smaller than it.
+"""
+import pytest
+import torch
+
+from paper_2601_07891_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2601_07891_b200 import binding as b
+    b.load()
+    return b
+
+
+def _make_sets(n_sets, T, d_model, H, D, seed):
+    sets = []
+    for i in range(n_sets):
+        X = synth.hidden_states(T, d_model, seed + i, "cuda")
+        K, V = synth.keys_values(H, T, D, seed + 100 + i, "cuda")
+        sets.append({"X": X, "K": K, "V": V})
+    return sets
+
+
+def _outputs(T, H, D):
+    return {"Ko": torch.full((H, T, D), -3.0, dtype=torch.bfloat16, device="cuda"),
+            "Vo": torch.full((H, T, D), -3.0, dtype=torch.bfloat16, device="cuda"),
+            "len": torch.full((1, H), -1, dtype=torch.int32, device="cuda"),
+            "sc": torch.full((T, H), float("nan"), dtype=torch.float32, device="cuda")}
+
+
+@pytest.mark.parametrize("d_model,hidden,T,n_layers", [
+    (256, 128, 74 * 256 + 77, 2),      # MLP, CTA pairs, grid = all SMs
+    (256, 0, 150 * 128 + 5, 1),        # Linear, one-CTA tiles, grid = all SMs
+    (512, 256, 700, 3),                # MLP, a few pair tiles
+    (1024, 0, 4096, 1),                # Linear, 32 tiles
+    (256, 64, 100, 2),                 # MLP, one tile: the few-token kernel
+])
+@pytest.mark.parametrize("shared_scores", [False, True])
+def test_back_to_back_calls_equal_synchronous_calls(binding, d_model, hidden, T, n_layers, shared_scores):
+    H, D, tau, w, n_sets, n_calls = 8, 64, 0.2, 32, 3, 12
+    ctx = binding.Kvzap(d_model, hidden, H, D, n_layers, T)
+    for l in range(n_layers):
+        wts = (synth.mlp_weights(d_model, hidden, H, 40 + l, "cuda", 0.3) if hidden
+               else synth.linear_weights(d_model, H, 40 + l, "cuda", 0.3))
+        ctx.set_weights(l, *wts)
+    sets = _make_sets(n_sets, T, d_model, H, D, seed=7)
+    one_sc = torch.empty(T, H, dtype=torch.float32, device="cuda")
+
+    def run(sync_each):
+        outs = [_outputs(T, H, D) for _ in range(n_sets)]
+        last = {}
+        for c in range(n_calls):
+            i, l = c % n_sets, c % n_layers
+            o = outs[i]
+            sc = one_sc if shared_scores else o["sc"]
+            binding.kvzap_prefill_fused(ctx.handle, l, sets[i]["X"], sets[i]["K"], sets[i]["V"], None, 1, tau, w,
+                                        o["Ko"], o["Vo"], o["len"], sc)
+            last[i] = l
+            if sync_each:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        return outs
+
+    ref = run(True)
+    got = run(False)
+    for a, b in zip(ref, got):
+        assert torch.equal(a["len"], b["len"])
+        assert int(a["len"].min()) >= min(w, T)
+        assert torch.equal(a["Ko"].view(torch.int16), b["Ko"].view(torch.int16))
+        assert torch.equal(a["Vo"].view(torch.int16), b["Vo"].view(torch.int16))
+        if not shared_scores:
+            assert torch.equal(a["sc"].view(torch.int32), b["sc"].view(torch.int32))
+    ctx.close()
