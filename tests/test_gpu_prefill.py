@@ -46,7 +46,8 @@ def test_linear_scores_match_oracle(binding, oracle, T):
 
 
 @pytest.mark.parametrize("d_model,hidden,T", [(256, 64, 300), (512, 128, 129), (256, 256, 257), (256, 512, 520),
-                                              (256, 640, 200), (128, 1024, 131), (4096, 512, 260), (5120, 640, 130)])
+                                              (256, 640, 200), (128, 1024, 131), (4096, 512, 260), (5120, 640, 130),
+                                              (1024, 512, 700), (512, 384, 1000), (2048, 1024, 300)])
 def test_mlp_scores_match_oracle(binding, oracle, d_model, hidden, T):
     H = 8
     ctx = _make_ctx(binding, d_model, hidden, H, 128, max_tokens=1024)
