@@ -287,7 +287,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (both CTAs of a pair)
-        const uint64_t pol_x = l2_policy_evict_first();   // hidden states are streamed once
+        const uint64_t pol_x1 = l2_policy_evict_first();  // hidden states are streamed once ...
+        const uint64_t pol_xn = l2_policy_evict_normal(); // ... unless a second pass over K follows (hidden > 512)
         const uint64_t pol_w = l2_policy_evict_last();    // weights are re-read by every tile
         uint32_t full0_cluster = bar_full;                // the pair's first CTA's full barriers
         if constexpr (kPair) full0_cluster = map_to_cta(bar_full, 0);
@@ -327,7 +328,14 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
             const int row0 = m_tile * kTileM;
             for (int g = 0; g < p.n_groups && ok; ++g) {
                 const int w_row0 = (p.layer0 + l_rel) * p.w_rows + g * p.group_w + static_cast<int>(cta_rank) * b_rows_chunk;
-                for (int kx = 0, kb = 0; kx < p.d_model; kx += kBlockK, ++kb, ++it) {
+                // Two passes over K: the second walks the K blocks backwards, so that it starts with the X
+                // blocks the first pass loaded last (still in L2; all CTAs together have more X in flight
+                // than L2 holds, walking forwards again every block would come from HBM a second time).
+                const bool backwards = (g & 1) != 0;
+                const uint64_t pol_x = (g + 1 < p.n_groups) ? pol_xn : pol_x1;
+                for (int i = 0; i < k_blocks; ++i, ++it) {
+                    const int kb = backwards ? k_blocks - 1 - i : i;
+                    const int kx = kb * kBlockK;
                     if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
                         ok = false;
                         break;
