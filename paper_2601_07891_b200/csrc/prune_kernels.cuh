@@ -3,13 +3,17 @@
 // be bit-exact.
 //
 // Data flow (all on one stream, no CTA ever waits for another):
-//   mask words  [H][n_words]   one keep bit per (head, packed token), 32 tokens per word,
-//                              written either by the scoring epilogue or by mask_kernel
-//   scan_kernel                per head: exclusive prefix of the kept count over 128-token
-//                              blocks; kept count before each sequence start; lengths[b,h]
-//   compact_kernel             one CTA per (128-token block, head): ranks its kept rows with
-//                              popc over the mask words and copies whole K and V rows with
-//                              16-byte accesses to their slot in the (b,h) list
+//   mask words  [H][n_words]    one keep bit per (head, packed token), 32 tokens per word,
+//                               written either by the scoring epilogue or by mask_kernel
+//   compact_dense_kernel        the compaction of every entry point that has a context: a CTA owns a
+//                               run of 128-token blocks of one head, counts the rows kept before them
+//                               straight from the mask words, ranks its kept rows with popc and copies
+//                               whole K and V rows with 16-byte accesses to their slot in the (b,h)
+//                               list (dense-ragged) or in the list's pages (paged)
+//   scan_kernel                 paged output only: lengths[b,h] and the first page of every list
+//                               (an exclusive scan over all lists, the one step that needs them all)
+//   compact_kernel              the older one-CTA-per-(block, head) compaction behind scan_kernel's
+//                               block prefix; still used by the allocation-free entry point
 #pragma once
 
 #include "score_kernel.cuh"

@@ -22,6 +22,12 @@
 // K step, and the MMAs issued by the pair's first CTA read both halves.  That
 // halves the W1 bytes each SM has to pull from L2 per FLOP, which is what
 // bounds the one-CTA version when the hidden layer is wide.
+//
+// Work tiles are handed out at run time (first tile = the CTA's or pair's own index, further ones from
+// a global counter), and the kernel cooperates with the launches around it: it lets the kernel behind
+// it in the stream be placed at once, may itself be started before the kernel ahead has finished
+// (it reads nothing that kernel writes) and in that case waits for it before it exits -- or, when the
+// grid does not fill the machine, before its first store.  The host side explains why that is safe.
 #pragma once
 
 #include "ptx.cuh"
