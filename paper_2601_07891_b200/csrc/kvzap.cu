@@ -59,6 +59,8 @@ struct kvzap_ctx {
     uint32_t *maskbits = nullptr;    // [kMaskRing][H][max_words]: consecutive calls use different slices
     uint64_t mask_turn = 0;
     int32_t *tile_counters = nullptr;    // [kMaskRing] work-tile counters of the scoring launches, used in rotation
+    float *split_part = nullptr;         // few-token kernel: [sm_count tiles][4 slices][128][8] partial scores
+    uint32_t *split_arrive = nullptr;    //                   [sm_count] arrival counts per tile
     uint64_t score_turn = 0;
     bool last_score_early = false;       // the last scoring launch was allowed to start early
     const void *last_scores = nullptr;   // scores buffer of the previous scoring launch, and its size
@@ -221,6 +223,8 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->b2_all);
     cudaFree(ctx->maskbits);
     cudaFree(ctx->tile_counters);
+    cudaFree(ctx->split_part);
+    cudaFree(ctx->split_arrive);
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
     cudaFree(ctx->list_page0);
@@ -323,8 +327,8 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // still use it.
     const kvzap_config &c = ctx->cfg;
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
-    // Few tiles (a decode step: one tile per layer): split every tile's hidden units over a cluster, so
-    // that the launch fills the machine and every CTA reads only its own slice of W1.
+    // Few tiles (a decode step: one tile per layer): split every tile's hidden units (and K range) over
+    // several CTAs, so that the launch fills the machine and every CTA reads only its own part of W1.
     if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count) {
         CUtensorMap tmap_x;
         kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
@@ -358,6 +362,8 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         p.window_keep = window_keep;
         p.tau = tau;
         p.status = ctx->status_dev;
+        p.split_part = ctx->split_part;
+        p.split_arrive = ctx->split_arrive;
         // Early start (consecutive decode steps): this kernel reads only hidden states and weights; the one
         // thing it may not do is write a scores buffer that the kernels of the previous call still read.
         const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
@@ -385,7 +391,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attrs[2];
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * n_ctas)), dim3(kScoreThreads),
-                        ctx->split_smem, stream, early, n_ctas);
+                        ctx->split_smem, stream, early, ctx->split_k);
             KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n,
                                                ctx->split_k, f));
         }
@@ -711,6 +717,11 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->tile_counters, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing));
+    if (ctx->split_n > 0) {
+        CREATE_CUDA(cudaMalloc(&ctx->split_part, sizeof(float) * static_cast<size_t>(ctx->sm_count) * 4 * kTileM * kMaxHeads));
+        CREATE_CUDA(cudaMalloc(&ctx->split_arrive, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
+        CREATE_CUDA(cudaMemset(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
+    }
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
     CREATE_CUDA(cudaMallocHost(&ctx->status_host, sizeof(int32_t)));
@@ -859,6 +870,7 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     if (v == 0) return KVZAP_OK;
     // a scoring kernel that gave up may have left its work-tile counter in an unknown state
     cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing, stream);
+    if (ctx->split_arrive) cudaMemsetAsync(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
     cudaStreamSynchronize(stream);
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
@@ -1072,7 +1084,7 @@ struct kvzap_cache {
     int64_t n_lists = 0;
     int step_parity = 0;
     // fused decode steps: per-cluster count of completed steps on the device, and the host's view of it
-    int32_t *done = nullptr;             // [n_layers * ceil(n_seqs / 128)]
+    int32_t *done = nullptr;             // [n_layers * ceil(n_seqs / 128)][4]: one per cluster of the fused step
     std::vector<int32_t> steps_done;     // per layer
 };
 
@@ -1247,7 +1259,7 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.prefix_len), sizeof(int32_t) * n, true);
     alloc(reinterpret_cast<void **>(&v.page_table), sizeof(int32_t) * n * max_pages_per_list, true);
     alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
-    alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
+    alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * 4 * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
           true);
     cache->steps_done.assign(c.n_layers, 0);
     // two halves used by alternate steps when the caller does not ask for the scores

@@ -77,6 +77,9 @@ struct ScoreParams {
     int32_t wait_before_write;    // 1: the epilogue waits for the kernel ahead in the stream before its first store
     int32_t *tile_counter;        // work tiles handed out beyond the first one of every CTA (or pair); starts at 0
     int32_t *tile_counter_reset;  // the counter of the launch after next: set to 0 by this launch
+    // few-token kernel only: the clusters of one tile combine their partial scores through global memory
+    float *split_part;            // [n_tiles][n_split][128][8]
+    uint32_t *split_arrive;       // [n_tiles] arrivals so far, over all launches (never reset in normal use)
 };
 
 // Byte offsets inside the dynamic shared memory block (after 1024-byte alignment).

@@ -2,18 +2,20 @@
 // Method, "KVzap" and the caption of Algorithm 1), where one 128-token tile per layer would leave
 // most SMs idle and every byte of W1 has to come from HBM.
 //
-// A cluster of n_split CTAs shares one 128-token tile: CTA j computes the hidden units
-// [j * Ns, (j + 1) * Ns), Ns = hidden / n_split, over the whole K range (its slice of W1 is read
-// exactly once, the X tile once per CTA, from L2 after the first), applies bias + GELU and its part
-// of the second layer, and sends its 8 partial sums per token to the cluster's first CTA through
-// distributed shared memory.  After one cluster barrier that CTA adds the parts and b2 and writes the
-// scores (and, if asked for, the keep bits).  36 layers x 4 CTAs fill the machine.
+// n_split * k_split CTAs share one 128-token tile.  The hidden units are cut into n_split slices of
+// Ns = hidden / n_split; a slice is computed by a cluster of k_split CTAs (1 or 2).  With k_split = 2
+// each CTA of the pair runs half of the K range (so an X tile is read by two CTAs per slice and every
+// byte of W1 exactly once), and the two partial pre-activation tiles are combined before the GELU:
+// each CTA sends the half of its accumulator that its partner owns through distributed shared memory
+// (into the partner's pipeline stages, idle by then) and finishes the columns it owns itself: bias,
+// GELU, its part of the second layer.  The 8 partial sums per token go to the pair's first CTA
+// (distributed shared memory, one cluster barrier).
 //
-// With k_split = 2 the cluster is 2 x 2: two CTAs share a slice of hidden units and each runs half of
-// the K range, so an X tile is read by two CTAs instead of four (the launch is bound by the bytes the
-// SMs pull through L2).  The two partial pre-activation tiles are combined before the GELU: each CTA
-// sends the half of its accumulator that its partner owns through distributed shared memory (into
-// the partner's pipeline stages, idle by then), and finishes the columns it owns itself.
+// The slices of a tile meet in global memory: the first CTA of every cluster stores its 128 x 8 partial
+// sums and counts itself in; the cluster that arrives last adds the parts in slice order (so the sum
+// does not depend on who was last) plus b2 and writes the scores (and, if asked for, the keep bits).
+// Clusters are kept this small on purpose: 36 layers x 2 slices x 2 CTAs fill the machine at once,
+// whereas clusters of four do not all find four free SMs in one GPC and leave a second wave.
 //
 // Warp roles as in score_kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..9
 // epilogue (TMEM lane quarter = warp % 4; the two warps of a quarter take alternate 16-column chunks).
@@ -28,16 +30,17 @@ namespace kvzap {
 // of a cluster do the cache update of the cluster's own lists -- 128 sequences x H heads of one layer,
 // a quarter per CTA -- exactly as decode_update_kernel does (the token that leaves the window is
 // judged by its buffered score, so nothing here needs the new scores); the cluster's first CTA puts
-// the new scores into the score buffer at the very end.  Consecutive steps may overlap in time
-// (the next launch starts as SMs become free): `done[cluster]` counts the steps a cluster has
-// completed, and a cluster touches the cache only after its predecessor has published `expect`.
+// the new scores into the score buffer at the very end (the last cluster of the tile to arrive).
+// Consecutive steps may overlap in time (the next launch starts as SMs become free): `done[cluster]`
+// counts the steps a cluster has completed, and a cluster touches the cache only after all clusters of
+// its tile have published `expect` for the step before.
 struct DecodeFuse {
     int32_t enabled;
     int32_t expect;
     CacheView c;
     const uint4 *K_new, *V_new;     // [n_layers_call][B][H][D] bf16
     float tau;
-    int32_t *done;                  // [n_layers * tiles_per_layer]
+    int32_t *done;                  // [n_layers * tiles_per_layer][n_split]
 };
 
 struct SplitSmemLayout {
@@ -58,7 +61,7 @@ __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stage
 }
 
 // p.group_w = p.chunk_n = Ns (the MMA's N); p.n_chunks = 1; p.acc_bufs = 1; p.n_tiles = 128-token tiles
-// over all layers of the call; cluster dimension n_split * k_split, gridDim.x = cluster size * p.n_tiles.
+// over all layers of the call; cluster dimension k_split, gridDim.x = n_split * k_split * p.n_tiles.
 // A CTA ends up owning Ns / k_split hidden units: xpart and the W2 / b1 slices are sized for those.
 __global__ void __maxnreg__(128)
 score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -88,13 +91,15 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const uint32_t bar_pfull = bar_done + 8;             // second warp of a lane quarter -> first
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + L.bars + 16 * kMaxStages + 32);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 36);
+    volatile int *last_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 40);
 
     griddep_launch_dependents();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_cta_rank();
-    const int nh = static_cast<int>(rank) % n_split;     // which slice of the hidden units
-    const int kh = static_cast<int>(rank) / n_split;     // which part of the K range
+    const uint32_t rank = cluster_cta_rank();            // 0 .. k_split - 1
+    const int kh = static_cast<int>(rank);               // which part of the K range
+    const int nh = (static_cast<int>(blockIdx.x) / k_split) % n_split;   // which slice of the hidden units
+    const int pos = nh * k_split + kh;                   // this CTA among the n_ctas of its tile
     const int tile = static_cast<int>(blockIdx.x) / n_ctas;
     const int l_rel = tile / p.tiles_per_layer;
     const int m_tile = tile - l_rel * p.tiles_per_layer;
@@ -211,9 +216,9 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             // ---- the cache update of this CTA's lists, under the MMAs
             const CacheView &c = f.c;
             const int cid = layer * p.tiles_per_layer + m_tile;
-            if (etid == 0) {
+            if (etid < n_split) {
                 const long long t0 = clock64();
-                while (ld_acquire_gpu(f.done + cid) != f.expect) {
+                while (ld_acquire_gpu(f.done + cid * n_split + etid) != f.expect) {
                     if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES) { *abort_flag = 1; break; }
                 }
             }
@@ -222,17 +227,23 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const int rows_per_cta = kTileM / n_ctas;
             // one thread per list: which row leaves, where it goes, which slot the new token takes
             {
-                const int b_loc = static_cast<int>(rank) * rows_per_cta + etid / kMaxHeads, h = etid % kMaxHeads;
+                const int b_loc = pos * rows_per_cta + etid / kMaxHeads, h = etid % kMaxHeads;
                 const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
                 int64_t dst = -1, ring = -1;
                 if (go && etid < rows_per_cta * kMaxHeads && b < c.n_seqs && h < c.n_heads) {
                     const int64_t li = (b * c.n_layers + layer) * c.n_heads + h;
+                    // two round trips to memory instead of four: both counters first, then the score of
+                    // the slot's old token and the page the prefix ends in, whether or not it will be needed
                     const int32_t n = __ldcg(c.n_tokens + li);
+                    const int32_t idx = __ldcg(c.prefix_len + li);
                     const int slot = n % c.window;
                     ring = li * c.window + slot;
-                    if (n >= c.window && __ldcg(c.score_ring + ring) >= f.tau) {
-                        const int32_t idx = __ldcg(c.prefix_len + li);
-                        const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
+                    const int page_i = idx / c.page_tokens, in_page = idx % c.page_tokens;
+                    const bool full = n >= c.window;
+                    const float s_old = full ? __ldcg(c.score_ring + ring) : 0.0f;
+                    const int32_t page_old =
+                        full && in_page != 0 && page_i < c.max_pages ? __ldcg(c.page_table + li * c.max_pages + page_i) : -1;
+                    if (full && s_old >= f.tau) {
                         int32_t page = -1;
                         if (page_i >= c.max_pages) {
                             atomicCAS(p.status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
@@ -241,7 +252,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                             if (got >= c.n_pages_pool) atomicCAS(p.status, 0, 4);
                             else { page = got; c.page_table[li * c.max_pages + page_i] = got; }
                         } else {
-                            page = __ldcg(c.page_table + li * c.max_pages + page_i);
+                            page = page_old;
                         }
                         if (page >= 0) {
                             dst = static_cast<int64_t>(page) * c.page_tokens + in_page;
@@ -254,23 +265,49 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 fuse_ring[etid] = ring;
             }
             named_barrier_sync(1, 256);
-            // rows: 16 lanes per list, every lane loads (old row, new row) before it stores
+            // rows: 16 lanes per list, kLists lists at a time; a lane loads the (old row, new row) pairs of all
+            // of them before it stores any of them, so that their round trips to memory overlap
             {
+                constexpr int kLists = 2;
                 const int grp = etid >> 4, l16 = etid & 15;
-                for (int j = grp; j < rows_per_cta * kMaxHeads; j += 16) {
-                    const int64_t ring = fuse_ring[j], dst = fuse_dst[j];
-                    if (ring < 0) continue;
-                    const int b_loc = static_cast<int>(rank) * rows_per_cta + j / kMaxHeads, h = j % kMaxHeads;
-                    const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
-                    const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+                const int n_lists = rows_per_cta * kMaxHeads;
+                for (int j0 = grp; j0 < n_lists; j0 += 16 * kLists) {
+                    int64_t ring[kLists], dst[kLists], src[kLists];
+#pragma unroll
+                    for (int i = 0; i < kLists; ++i) {
+                        const int j = j0 + 16 * i;
+                        ring[i] = j < n_lists ? fuse_ring[j] : -1;
+                        dst[i] = j < n_lists ? fuse_dst[j] : -1;
+                        const int b_loc = pos * rows_per_cta + j / kMaxHeads, h = j % kMaxHeads;
+                        const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
+                        src[i] = ((static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h) * c.row_units;
+                        ring[i] *= c.row_units;           // stays negative where there is no list
+                        dst[i] *= c.row_units;
+                    }
                     for (int u = l16; u < c.row_units; u += 16) {
-                        uint4 ko = make_uint4(0, 0, 0, 0), vo = ko;
-                        if (dst >= 0) { ko = __ldcg(c.k_ring + ring * c.row_units + u); vo = __ldcg(c.v_ring + ring * c.row_units + u); }
-                        const uint4 kn = __ldg(f.K_new + src_row * c.row_units + u);
-                        const uint4 vn = __ldg(f.V_new + src_row * c.row_units + u);
-                        if (dst >= 0) { c.k_pool[dst * c.row_units + u] = ko; c.v_pool[dst * c.row_units + u] = vo; }
-                        c.k_ring[ring * c.row_units + u] = kn;
-                        c.v_ring[ring * c.row_units + u] = vn;
+                        uint4 ko[kLists], vo[kLists], kn[kLists], vn[kLists];
+#pragma unroll
+                        for (int i = 0; i < kLists; ++i) {
+                            if (ring[i] >= 0 && dst[i] >= 0) {
+                                ko[i] = __ldcg(c.k_ring + ring[i] + u);
+                                vo[i] = __ldcg(c.v_ring + ring[i] + u);
+                            }
+                            if (ring[i] >= 0) {
+                                kn[i] = __ldg(f.K_new + src[i] + u);
+                                vn[i] = __ldg(f.V_new + src[i] + u);
+                            }
+                        }
+#pragma unroll
+                        for (int i = 0; i < kLists; ++i) {
+                            if (ring[i] >= 0 && dst[i] >= 0) {
+                                c.k_pool[dst[i] + u] = ko[i];
+                                c.v_pool[dst[i] + u] = vo[i];
+                            }
+                            if (ring[i] >= 0) {
+                                c.k_ring[ring[i] + u] = kn[i];
+                                c.v_ring[ring[i] + u] = vn[i];
+                            }
+                        }
                     }
                 }
             }
@@ -285,7 +322,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         tc_fence_before_sync();
         cluster_sync_all();
         if (epi && ok) {
-            const uint32_t partner = rank ^ static_cast<uint32_t>(n_split);
+            const uint32_t partner = rank ^ 1u;
             const int send_c0 = (1 - kh) * own_n;               // the columns the partner owns
             const uint32_t dst0 = map_to_cta(smem_base, partner);
             for (int c = hsel; c < n16; c += 2) {
@@ -365,7 +402,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const float4 pa = src[0], pb = src[1];
             s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
             s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
-            // hand this CTA's partial sums to the cluster's first CTA: xpart[rank][row][8]
+            // hand this CTA's partial sums to its cluster's first CTA: xpart[rank][row][8]
             const uint32_t dst = map_to_cta(smem_base + L.xpart + (rank * kTileM + row) * kMaxHeads * 4, 0);
             st_shared_cluster_v4(dst, s[0], s[1], s[2], s[3]);
             st_shared_cluster_v4(dst + 16, s[4], s[5], s[6], s[7]);
@@ -386,17 +423,47 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     griddep_wait();
     if (rank != 0 || warp < 2 || warp >= 6 || m_tile >= p.blocks_per_layer) return;
 
-    // ------------------------------------------------------------ first CTA: total, scores, keep bits
+    // ------------------------------------------------------------ first CTA of the cluster: the slice's sums
     {
         float s[kMaxHeads];
 #pragma unroll
-        for (int h = 0; h < kMaxHeads; ++h) s[h] = __ldg(p.b2 + layer * kMaxHeads + h);
-        for (int r = 0; r < n_ctas; ++r) {
+        for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+        for (int r = 0; r < k_split; ++r) {
             const float4 *src = reinterpret_cast<const float4 *>(xpart + (r * kTileM + row) * kMaxHeads);
             const float4 pa = src[0], pb = src[1];
             s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
             s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
         }
+        const int32_t done_i = (layer * p.tiles_per_layer + m_tile) * n_split + nh;
+        if (n_split > 1) {
+            // the slices meet in global memory; whoever arrives last finishes the tile
+            float4 *mine = reinterpret_cast<float4 *>(p.split_part + ((static_cast<int64_t>(tile) * n_split + nh) * kTileM + row) * kMaxHeads);
+            __stcg(mine, make_float4(s[0], s[1], s[2], s[3]));
+            __stcg(mine + 1, make_float4(s[4], s[5], s[6], s[7]));
+            __threadfence();
+            named_barrier_sync(2, 128);
+            if (threadIdx.x == 64) {
+                const uint32_t before = atomicAdd(p.split_arrive + tile, 1u);
+                *last_flag = (before + 1u) % static_cast<uint32_t>(n_split) == 0u ? 1 : 0;
+                __threadfence();
+            }
+            named_barrier_sync(2, 128);
+            if (*last_flag == 0) {
+                // not the last: this cluster's part of the cache update is complete, say so and leave
+                if (f.enabled && threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, f.expect + 1);
+                return;
+            }
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+            for (int r = 0; r < n_split; ++r) {
+                const float4 *src = reinterpret_cast<const float4 *>(p.split_part + ((static_cast<int64_t>(tile) * n_split + r) * kTileM + row) * kMaxHeads);
+                const float4 pa = __ldcg(src), pb = __ldcg(src + 1);
+                s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
+                s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < kMaxHeads; ++h) s[h] += __ldg(p.b2 + layer * kMaxHeads + h);
         const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;
         const bool valid = t < p.n_tokens;
         if (f.enabled) {
@@ -414,7 +481,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
             __threadfence();
             named_barrier_sync(2, 128);
-            if (threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + layer * p.tiles_per_layer + m_tile, f.expect + 1);
+            if (threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, f.expect + 1);
         }
         if (valid && p.scores != nullptr) {
             float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
