@@ -208,6 +208,33 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
                                        float *scores_out, void *stream);
 
 /*
+ * Pruning on the write side (Discussion, "Implementation Challenges": the
+ * surrogate needs only hidden states, so pruning can run before attention).
+ * Same operation and outputs as kvzap_prefill_fused / kvzap_prefill_fused_paged,
+ * but K and V are taken as the key/value projection leaves them, one token
+ * after the other:
+ *   K_proj, V_proj [n_tokens, H, D] bf16 (device, 16-byte aligned, caller-owned)
+ * so a caller never has to build the dense head-major cache [H, n_tokens, D]:
+ * rows that are dropped are never read, rows that are kept are read once and
+ * written once, straight into list (b,h).  All other arguments, the outputs,
+ * the empty-input behaviour and the errors are those of the calls named above.
+ */
+kvzap_status kvzap_prefill_write(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                 const void *K_proj, const void *V_proj,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                 float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths,
+                                 float *scores_out, void *stream);
+kvzap_status kvzap_prefill_write_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                       const void *K_proj, const void *V_proj,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                       float tau, int32_t w,
+                                       void *K_pool, void *V_pool, int64_t n_pages_pool, int32_t page_tokens,
+                                       int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
+                                       int32_t *lengths, int32_t *n_pages_used,
+                                       float *scores_out, void *stream);
+
+/*
  * Decode-time cache (caption of Algorithm 1: decoding is like prefilling but
  * needs a buffer of scores to enforce the sliding window; contributions:
  * delayed eviction with a sliding window).  One list per (sequence, layer, KV

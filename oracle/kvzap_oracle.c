@@ -258,6 +258,79 @@ int kvzap_oracle_compact_paged(const uint16_t *K, const uint16_t *V, const uint8
 }
 
 /*
+ * The same two compactions with K and V given as the key/value projection
+ * writes them, [T_total, H, D] (Discussion, "Implementation Challenges":
+ * the surrogate needs only hidden states, so pruning may run before
+ * attention, i.e. before a head-major cache exists).  Row (t,h) of the input
+ * is at element (t*H + h)*D; outputs, lengths and page numbering are exactly
+ * those of kvzap_oracle_compact / kvzap_oracle_compact_paged.
+ */
+void kvzap_oracle_compact_write(const uint16_t *K_proj, const uint16_t *V_proj, const uint8_t *keep,
+                                const int32_t *cu_seqlens, int B, int H, int D,
+                                uint16_t *K_out, uint16_t *V_out, int32_t *lengths)
+{
+    const int64_t T_total = cu_seqlens[B];
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int64_t n = 0;
+            for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t) {
+                if (!keep[(int64_t)h * T_total + t]) continue;
+                const uint16_t *k_row = K_proj + (t * H + h) * (int64_t)D;
+                const uint16_t *v_row = V_proj + (t * H + h) * (int64_t)D;
+                uint16_t *k_dst = K_out + ((int64_t)h * T_total + cu_seqlens[b] + n) * D;
+                uint16_t *v_dst = V_out + ((int64_t)h * T_total + cu_seqlens[b] + n) * D;
+                for (int d = 0; d < D; ++d) {
+                    k_dst[d] = k_row[d];
+                    v_dst[d] = v_row[d];
+                }
+                ++n;
+            }
+            lengths[b * H + h] = (int32_t)n;
+        }
+}
+
+int kvzap_oracle_compact_write_paged(const uint16_t *K_proj, const uint16_t *V_proj, const uint8_t *keep,
+                                     const int32_t *cu_seqlens, int B, int H, int D,
+                                     int page_tokens, int32_t first_page, int64_t n_pages_pool,
+                                     int max_pages_per_list,
+                                     uint16_t *K_pool, uint16_t *V_pool, int32_t *page_table,
+                                     int32_t *lengths, int32_t *n_pages_used)
+{
+    const int64_t T_total = cu_seqlens[B];
+    int64_t pages = 0;
+    for (int list = 0; list < B * H; ++list) {
+        const int b = list / H, h = list % H;
+        int64_t n = 0;
+        for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t)
+            if (keep[(int64_t)h * T_total + t]) ++n;
+        lengths[list] = (int32_t)n;
+        const int64_t need = (n + page_tokens - 1) / page_tokens;
+        if (need > max_pages_per_list) return -1;
+        pages += need;
+    }
+    if ((int64_t)first_page + pages > n_pages_pool) return -1;
+    int64_t next_page = first_page;            /* first page of the list being filled */
+    for (int list = 0; list < B * H; ++list) {
+        const int b = list / H, h = list % H;
+        int64_t n = 0;
+        for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t) {
+            if (!keep[(int64_t)h * T_total + t]) continue;
+            const int64_t page = next_page + n / page_tokens;
+            if (n % page_tokens == 0) page_table[(int64_t)list * max_pages_per_list + n / page_tokens] = (int32_t)page;
+            const int64_t slot = page * page_tokens + n % page_tokens;
+            for (int d = 0; d < D; ++d) {
+                K_pool[slot * D + d] = K_proj[(t * H + h) * (int64_t)D + d];
+                V_pool[slot * D + d] = V_proj[(t * H + h) * (int64_t)D + d];
+            }
+            ++n;
+        }
+        next_page += (n + page_tokens - 1) / page_tokens;
+    }
+    *n_pages_used = (int32_t)pages;
+    return 0;
+}
+
+/*
  * Closed forms of Appendix B (per token, per layer).
  *   C        = 4 D_h (H_Q D + H D) + 6 D_h D_int      linear-projection FLOPs of a layer
  *   C_MLP    = 2 D_h (D_h/8) + 2 (D_h/8) H = D_h/4 (D_h + H)

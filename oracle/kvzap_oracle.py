@@ -50,6 +50,7 @@ def lib():
         L.kvzap_oracle_gelu.argtypes = [ctypes.c_double]
         L.kvzap_oracle_score_mlp.restype = ctypes.c_int
         L.kvzap_oracle_compact_paged.restype = ctypes.c_int
+        L.kvzap_oracle_compact_write_paged.restype = ctypes.c_int
         for name in ("layer_flops", "mlp_flops", "linear_flops"):
             getattr(L, "kvzap_oracle_" + name).restype = ctypes.c_double
         L.kvzap_oracle_layer_flops.argtypes = [ctypes.c_int] * 5
@@ -187,6 +188,54 @@ def compact_paged(K, V, keep, page_tokens, n_pages_pool, max_pages_per_list,
     used = ctypes.c_int32(0)
     rc = lib().kvzap_oracle_compact_paged(
         _c(K, ctypes.c_uint16), _c(V, ctypes.c_uint16), _c(keep, ctypes.c_uint8),
+        _c(cu, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
+        ctypes.c_int(page_tokens), ctypes.c_int32(first_page), ctypes.c_int64(n_pages_pool),
+        ctypes.c_int(max_pages_per_list),
+        _c(K_pool, ctypes.c_uint16), _c(V_pool, ctypes.c_uint16), _c(table, ctypes.c_int32),
+        _c(lengths, ctypes.c_int32), ctypes.byref(used))
+    if rc != 0:
+        raise ValueError("page pool or page table too small")
+    return K_pool, V_pool, table, lengths, int(used.value)
+
+
+def compact_write(K_proj, V_proj, keep, cu_seqlens=None, fill=0):
+    """Write-side compaction: K_proj,V_proj [T_total,H,D] bf16 bits, keep [H,T_total]
+    -> (K_out, V_out [H,T_total,D], lengths[B,H])."""
+    K_proj = _u16(K_proj, 3)
+    V_proj = _u16(V_proj, 3)
+    T_total, H, D = K_proj.shape
+    assert V_proj.shape == K_proj.shape
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    assert keep.shape == (H, T_total)
+    cu = _cu(cu_seqlens, T_total)
+    B = len(cu) - 1
+    K_out = np.full((H, T_total, D), fill, dtype=np.uint16)
+    V_out = np.full((H, T_total, D), fill, dtype=np.uint16)
+    lengths = np.zeros((B, H), dtype=np.int32)
+    lib().kvzap_oracle_compact_write(
+        _c(K_proj, ctypes.c_uint16), _c(V_proj, ctypes.c_uint16), _c(keep, ctypes.c_uint8),
+        _c(cu, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
+        _c(K_out, ctypes.c_uint16), _c(V_out, ctypes.c_uint16), _c(lengths, ctypes.c_int32))
+    return K_out, V_out, lengths
+
+
+def compact_write_paged(K_proj, V_proj, keep, page_tokens, n_pages_pool, max_pages_per_list,
+                        cu_seqlens=None, first_page=0, fill=0):
+    """Write-side compaction into pages -> (K_pool, V_pool, page_table, lengths, n_pages_used)."""
+    K_proj = _u16(K_proj, 3)
+    V_proj = _u16(V_proj, 3)
+    T_total, H, D = K_proj.shape
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    assert keep.shape == (H, T_total)
+    cu = _cu(cu_seqlens, T_total)
+    B = len(cu) - 1
+    K_pool = np.full((n_pages_pool, page_tokens, D), fill, dtype=np.uint16)
+    V_pool = np.full((n_pages_pool, page_tokens, D), fill, dtype=np.uint16)
+    table = np.full((B * H, max_pages_per_list), -1, dtype=np.int32)
+    lengths = np.zeros((B, H), dtype=np.int32)
+    used = ctypes.c_int32(0)
+    rc = lib().kvzap_oracle_compact_write_paged(
+        _c(K_proj, ctypes.c_uint16), _c(V_proj, ctypes.c_uint16), _c(keep, ctypes.c_uint8),
         _c(cu, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(D),
         ctypes.c_int(page_tokens), ctypes.c_int32(first_page), ctypes.c_int64(n_pages_pool),
         ctypes.c_int(max_pages_per_list),

@@ -56,6 +56,9 @@ SIGNATURES = {
                                          _vp, _i32, _vp, _vp, _vp]),
     "kvzap_prefill_fused_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
                                          _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_write_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
+                                         _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_cache_create": (_i32, [_vp, ctypes.POINTER(_vp), _i32, _i32, _i32, _vp, _vp, _i64, _i32]),
     "kvzap_cache_destroy": (_i32, [_vp]),
     "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
@@ -209,6 +212,28 @@ def kvzap_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, t
         _ptr(scores_out) if nz else None, _stream(stream)))
 
 
+def kvzap_prefill_write(handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                        scores_out=None, stream=None):
+    """K_proj, V_proj [n_tokens, H, D]: the projection's own layout."""
+    n_tokens = K_proj.shape[0]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_write(
+        handle, layer, _ptr(hidden) if nz else None, _ptr(K_proj) if nz else None, _ptr(V_proj) if nz else None,
+        _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
+        _ptr(lengths), _ptr(scores_out) if nz else None, _stream(stream)))
+
+
+def kvzap_prefill_write_paged(handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_pool, V_pool,
+                              page_tokens, first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None):
+    n_tokens = K_proj.shape[0]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_write_paged(
+        handle, layer, _ptr(hidden) if nz else None, _ptr(K_proj) if nz else None, _ptr(V_proj) if nz else None,
+        _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens,
+        first_page, _ptr(page_table), page_table.shape[1], _ptr(lengths), _ptr(n_pages_used),
+        _ptr(scores_out) if nz else None, _stream(stream)))
+
+
 def kvzap_cache_create(handle, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list):
     cache = ctypes.c_void_p()
     _check(handle, load().kvzap_cache_create(handle, ctypes.byref(cache), n_seqs, window, page_tokens, _ptr(K_pool),
@@ -279,6 +304,24 @@ def prepare_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs,
             _ptr(n_pages_used), _ptr(scores_out), _stream(stream))
     return PreparedCall("kvzap_prefill_fused_paged", handle, args,
                         (hidden, K, V, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used, scores_out))
+
+
+def prepare_prefill_write(handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                          scores_out=None, stream=None) -> PreparedCall:
+    args = (handle, layer, _ptr(hidden), _ptr(K_proj), _ptr(V_proj), _ptr(cu_seqlens), n_seqs, K_proj.shape[0], tau, w,
+            _ptr(K_out), _ptr(V_out), _ptr(lengths), _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_prefill_write", handle, args,
+                        (hidden, K_proj, V_proj, cu_seqlens, K_out, V_out, lengths, scores_out))
+
+
+def prepare_prefill_write_paged(handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_pool, V_pool,
+                                page_tokens, first_page, page_table, lengths, n_pages_used, scores_out=None,
+                                stream=None) -> PreparedCall:
+    args = (handle, layer, _ptr(hidden), _ptr(K_proj), _ptr(V_proj), _ptr(cu_seqlens), n_seqs, K_proj.shape[0], tau, w,
+            _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens, first_page, _ptr(page_table), page_table.shape[1],
+            _ptr(lengths), _ptr(n_pages_used), _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_prefill_write_paged", handle, args,
+                        (hidden, K_proj, V_proj, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used, scores_out))
 
 
 def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None,

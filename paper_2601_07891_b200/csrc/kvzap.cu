@@ -481,7 +481,8 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
 // Dense-ragged compaction over the mask words in `mask` (one kernel, no scan pass).
 static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, void *K_out,
-                                      void *V_out, int32_t *lengths, cudaStream_t stream, bool beside_scoring = true)
+                                      void *V_out, int32_t *lengths, cudaStream_t stream, bool beside_scoring = true,
+                                      bool tok_major = false)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -506,7 +507,9 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
                                            static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
                                            static_cast<uint4 *>(V_out), mask, n_words, n_blocks, blocks_per_cta,
                                            cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths, 0,
-                                           static_cast<const int32_t *>(nullptr)));
+                                           static_cast<const int32_t *>(nullptr),
+                                           tok_major ? int64_t{1} : n_tokens,
+                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1}));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -832,9 +835,11 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
 }
 
-kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
-                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
-                                 void *K_out, void *V_out, int32_t *lengths, float *scores_out, void *stream_)
+// tok_major: K and V are [n_tokens][H][D] (the K/V projection's output) instead of [H][n_tokens][D]
+static kvzap_status prefill_fused_impl(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                       int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
+                                       void *stream_, bool tok_major)
 {
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -855,7 +860,24 @@ kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidd
     uint32_t *mask = next_mask_slice(ctx);
     st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
-    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream);
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, true, tok_major);
+}
+
+kvzap_status kvzap_prefill_fused(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                 const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
+                                 void *K_out, void *V_out, int32_t *lengths, float *scores_out, void *stream_)
+{
+    return prefill_fused_impl(ctx, layer, hidden, K, V, cu_seqlens, n_seqs, n_tokens, tau, w, K_out, V_out, lengths,
+                              scores_out, stream_, false);
+}
+
+kvzap_status kvzap_prefill_write(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K_proj,
+                                 const void *V_proj, const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                 float tau, int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
+                                 void *stream_)
+{
+    return prefill_fused_impl(ctx, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, n_tokens, tau, w, K_out, V_out,
+                              lengths, scores_out, stream_, true);
 }
 
 kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
@@ -1096,7 +1118,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                             int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
                                             int32_t *page_table, int32_t max_pages, int32_t *lengths,
                                             int32_t *n_pages_used, cudaStream_t stream,
-                                            int32_t *page_cursor = nullptr)
+                                            int32_t *page_cursor = nullptr, bool tok_major = false)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1129,7 +1151,9 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            static_cast<uint4 *>(V_pool), mask, n_words, n_blocks, blocks_per_cta,
                                            cu_seqlens, static_cast<int>(n_seqs), n_tokens, static_cast<int>(c.n_kv_heads),
                                            static_cast<int>(c.head_dim / 8), lengths, static_cast<int>(page_tokens),
-                                           static_cast<const int32_t *>(ctx->list_page0)));
+                                           static_cast<const int32_t *>(ctx->list_page0),
+                                           tok_major ? int64_t{1} : n_tokens,
+                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1}));
     }
     ctx->launches += 2;
     return KVZAP_OK;
@@ -1190,12 +1214,12 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
                                    first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
 }
 
-kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
-                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
-                                       int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
-                                       int32_t page_tokens, int32_t first_page, int32_t *page_table,
-                                       int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
-                                       float *scores_out, void *stream_)
+static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K,
+                                             const void *V, const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                             float tau, int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                             int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                             int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                             float *scores_out, void *stream_, bool tok_major)
 {
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -1218,7 +1242,32 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
     st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
     return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
-                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
+                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream, nullptr,
+                                   tok_major);
+}
+
+kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                       int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                       int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                       int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                       float *scores_out, void *stream_)
+{
+    return prefill_fused_paged_impl(ctx, layer, hidden, K, V, cu_seqlens, n_seqs, n_tokens, tau, w, K_pool, V_pool,
+                                    n_pages_pool, page_tokens, first_page, page_table, max_pages_per_list, lengths,
+                                    n_pages_used, scores_out, stream_, false);
+}
+
+kvzap_status kvzap_prefill_write_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K_proj,
+                                       const void *V_proj, const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                       float tau, int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
+                                       int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                       int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                       float *scores_out, void *stream_)
+{
+    return prefill_fused_paged_impl(ctx, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, n_tokens, tau, w, K_pool,
+                                    V_pool, n_pages_pool, page_tokens, first_page, page_table, max_pages_per_list,
+                                    lengths, n_pages_used, scores_out, stream_, true);
 }
 
 kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seqs, int32_t window,

@@ -322,8 +322,10 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                      uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
                      int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths, int page_tokens,
-                     const int32_t *__restrict__ list_page0)
+                     const int32_t *__restrict__ list_page0, int64_t in_stride_h, int64_t in_stride_t)
 {
+    // Row (h, t) of the inputs starts at row index h * in_stride_h + t * in_stride_t: (n_tokens, 1) for
+    // the head-major cache layout [H][T][D], (1, H) for the K/V projection's own output [T][H][D].
     // page_tokens > 0: paged output.  K_out / V_out are the page pools, list (b,h) starts at page
     // list_page0[b * H + h] (-1 = nothing may be written), and lengths come from the scan kernel.
     const bool paged = page_tokens > 0;
@@ -415,7 +417,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
             }
         }
         __syncthreads();
-        const int64_t head_row0 = static_cast<int64_t>(h) * n_tokens + blk_start;
+        const int64_t head_row0 = static_cast<int64_t>(h) * in_stride_h + blk_start * in_stride_t;
         for (int i0 = group; i0 < cnt; i0 += kGroups * kRowsInFlight) {
             for (int u0 = gl; u0 < row_units; u0 += 16) {
                 uint4 kv[kRowsInFlight], vv[kRowsInFlight];
@@ -423,7 +425,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                 for (int j = 0; j < kRowsInFlight; ++j) {
                     const int i = i0 + j * kGroups;
                     if (i < cnt) {
-                        const int64_t src = (head_row0 + src_tok[i]) * row_units + u0;
+                        const int64_t src = (head_row0 + src_tok[i] * in_stride_t) * row_units + u0;
                         kv[j] = __ldg(K + src);
                         vv[j] = __ldg(V + src);
                     }

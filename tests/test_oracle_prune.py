@@ -231,3 +231,69 @@ def test_decode_prefill_then_steps_equals_longer_prefill(oracle):
         _pos, Kd, Vd = dec.logical(0, 0, h)
         np.testing.assert_array_equal(Kd, Kc[h, :lengths[0, h]])
         np.testing.assert_array_equal(Vd, Vc[h, :lengths[0, h]])
+
+
+# ---------------------------------------------------------------------------
+# Write-side pruning (Discussion, "Implementation Challenges"): K and V arrive as
+# the projection wrote them, [T, H, D].
+
+
+def test_write_side_compaction_is_the_ordered_gather_of_projection_rows(oracle):
+    rng = np.random.default_rng(40)
+    lens = [50, 0, 3, 120]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    H, T, D = 3, int(cu[-1]), 8
+    K, V = _tagged_kv(H, T, D)
+    K_proj = np.ascontiguousarray(K.transpose(1, 0, 2))      # [T, H, D]
+    V_proj = np.ascontiguousarray(V.transpose(1, 0, 2))
+    keep = (rng.random((H, T)) < 0.4).astype(np.uint8)
+    K_out, V_out, lengths = oracle.compact_write(K_proj, V_proj, keep, cu, fill=0xDEAD)
+    for b in range(len(lens)):
+        for h in range(H):
+            idx = cu[b] + np.flatnonzero(keep[h, cu[b]:cu[b + 1]])       # explicit index list
+            n = len(idx)
+            assert lengths[b, h] == n
+            np.testing.assert_array_equal(K_out[h, cu[b]:cu[b] + n], K_proj[idx, h])
+            np.testing.assert_array_equal(V_out[h, cu[b]:cu[b] + n], V_proj[idx, h])
+            assert (K_out[h, cu[b]:cu[b] + n, 0] == h).all()             # rows of head h only
+            assert np.all(np.diff(K_out[h, cu[b]:cu[b] + n, 1].astype(np.int64)) > 0)   # token order
+            assert (K_out[h, cu[b] + n:cu[b + 1]] == 0xDEAD).all()
+            assert (V_out[h, cu[b] + n:cu[b + 1]] == 0xDEAD).all()
+    # keeping everything is the transposition [T,H,D] -> [H,T,D]
+    K_all, V_all, len_all = oracle.compact_write(K_proj, V_proj, np.ones((H, T), np.uint8), cu)
+    np.testing.assert_array_equal(K_all, K)
+    np.testing.assert_array_equal(V_all, V)
+    np.testing.assert_array_equal(len_all, np.repeat(np.array(lens)[:, None], H, 1))
+
+
+def test_write_side_paged_compaction_pages_and_rows(oracle):
+    rng = np.random.default_rng(41)
+    lens = [37, 64, 5]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    H, T, D, P = 3, int(cu[-1]), 8, 16
+    K, V = _tagged_kv(H, T, D)
+    K_proj = np.ascontiguousarray(K.transpose(1, 0, 2))
+    V_proj = np.ascontiguousarray(V.transpose(1, 0, 2))
+    keep = (rng.random((H, T)) < 0.6).astype(np.uint8)
+    Kp, Vp, table, lengths, used = oracle.compact_write_paged(K_proj, V_proj, keep, P, n_pages_pool=40,
+                                                              max_pages_per_list=5, cu_seqlens=cu, first_page=2,
+                                                              fill=0x1111)
+    cursor = 2
+    for b in range(len(lens)):
+        for h in range(H):
+            idx = cu[b] + np.flatnonzero(keep[h, cu[b]:cu[b + 1]])
+            n, need = len(idx), -(-len(idx) // P)
+            assert lengths[b, h] == n
+            pages = table[b * H + h]
+            np.testing.assert_array_equal(pages[:need], np.arange(cursor, cursor + need))   # (b,h) order, contiguous
+            assert (pages[need:] == -1).all()
+            np.testing.assert_array_equal(Kp[pages[:need]].reshape(-1, D)[:n], K_proj[idx, h])
+            np.testing.assert_array_equal(Vp[pages[:need]].reshape(-1, D)[:n], V_proj[idx, h])
+            cursor += need
+    assert used == cursor - 2
+    assert (Kp[:2] == 0x1111).all() and (Kp[cursor:] == 0x1111).all()
+    with pytest.raises(ValueError):
+        oracle.compact_write_paged(K_proj, V_proj, keep, P, n_pages_pool=used + 1, max_pages_per_list=5,
+                                   cu_seqlens=cu, first_page=2)
+    with pytest.raises(ValueError):
+        oracle.compact_write_paged(K_proj, V_proj, keep, P, n_pages_pool=40, max_pages_per_list=1, cu_seqlens=cu)
