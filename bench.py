@@ -186,6 +186,7 @@ def run_prefill(args, wl, env):
         L = min(L, args.layers)          # small case for profiler captures; reported in config.n_layers
     n_tokens = B * T
     H, D, P = wl.n_kv_heads, wl.head_dim, wl.page_tokens
+    proj = args.kv_layout == "proj"
     ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=dev.index)
     cu = torch.from_numpy(synth.cu_seqlens([T] * B)).to(dev) if B > 1 else None
 
@@ -210,6 +211,9 @@ def run_prefill(args, wl, env):
         seed = 1000 * args.workload_index + l + 100000 * rank
         Xs.append(synth.hidden_states(n_tokens, wl.d_model, seed, dev, wl.token_scale_sigma))
         K, V = synth.keys_values(H, n_tokens, D, seed + 500, dev)
+        if proj:
+            # write-side pruning: the same draws, laid out as the K/V projection writes them, [T, H, D]
+            K, V = K.transpose(0, 1).contiguous(), V.transpose(0, 1).contiguous()
         Ks.append(K)
         Vs.append(V)
         if P:
@@ -218,8 +222,8 @@ def run_prefill(args, wl, env):
             tabs.append(torch.zeros(B * H, max_pages, dtype=torch.int32, device=dev))
             used.append(torch.zeros(1, dtype=torch.int32, device=dev))
         else:
-            Kos.append(torch.empty_like(K))
-            Vos.append(torch.empty_like(V))
+            Kos.append(torch.empty(H, n_tokens, D, dtype=torch.bfloat16, device=dev))
+            Vos.append(torch.empty(H, n_tokens, D, dtype=torch.bfloat16, device=dev))
             tabs.append(None)
             used.append(None)
         scs.append(torch.empty(n_tokens, H, dtype=torch.float32, device=dev))
@@ -231,13 +235,14 @@ def run_prefill(args, wl, env):
     calls = {}
     for l in range(L):
         for i in (range(n_bufs) if n_bufs > L else [l]):
+            prep_paged = binding.prepare_prefill_write_paged if proj else binding.prepare_prefill_fused_paged
+            prep_dense = binding.prepare_prefill_write if proj else binding.prepare_prefill_fused
             if P:
-                calls[(l, i)] = binding.prepare_prefill_fused_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
-                                                                    wl.window, Kos[i], Vos[i], P, 0, tabs[i], lens[i],
-                                                                    used[i], scs[i])
+                calls[(l, i)] = prep_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
+                                           wl.window, Kos[i], Vos[i], P, 0, tabs[i], lens[i], used[i], scs[i])
             else:
-                calls[(l, i)] = binding.prepare_prefill_fused(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
-                                                              wl.window, Kos[i], Vos[i], lens[i], scs[i])
+                calls[(l, i)] = prep_dense(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
+                                           wl.window, Kos[i], Vos[i], lens[i], scs[i])
 
     def step():
         for l in range(L):
@@ -283,14 +288,16 @@ def run_prefill(args, wl, env):
         if n_bufs > L:
             turn[0] += L
     score_ms = _timed(score_only, n_rep, sync) / L
-    if P:
+    if proj:
+        prune = None          # the two-call route exists for the head-major layout only
+    elif P:
         prune = lambda: [binding.kvzap_prune_prefill_paged(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
                                                            Kos[l], Vos[l], P, 0, tabs[l], lens[l], used[l])
                          for l in range(n_bufs)]
     else:
         prune = lambda: [binding.kvzap_prune_prefill(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
                                                      Kos[l], Vos[l], lens[l]) for l in range(n_bufs)]
-    prune_ms = _timed(prune, n_rep, sync) / n_bufs
+    prune_ms = _timed(prune, n_rep, sync) / n_bufs if prune else None
 
     peaks, peak_src = load_peaks()
     flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer = _roofline_times(wl, n_tokens, kept_rows, peaks)
@@ -316,11 +323,12 @@ def run_prefill(args, wl, env):
     extra = {"layer_ms": layer_ms, "layer_roofline_ms": t_roof_layer * 1e3,
              "layer_frac_of_roofline": t_roof_layer * 1e3 / layer_ms,
              "score_alone_ms": score_ms, "mask_plus_compaction_alone_ms": prune_ms,
-             "compaction_alone_GBps": compact_bytes / (prune_ms * 1e-3) / 1e9,
+             "compaction_alone_GBps": compact_bytes / (prune_ms * 1e-3) / 1e9 if prune_ms else None,
              "kept_fraction": kept_rows / (H * n_tokens)}
     config = {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
               "n_kv_heads": H, "head_dim": D, "n_layers": L, "batch": B, "seq_len": T, "tau": wl.tau,
               "window": wl.window, "page_tokens": P, "input_sets": n_bufs,
+              "kv_layout": "[T,H,D] as the projection writes it (write-side pruning)" if proj else "[H,T,D]",
               "l2": "inputs larger than L2 (distinct resident buffers per layer; small workloads rotate over "
                     "enough sets that 2.5 x L2 lies between two uses of a buffer)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
@@ -329,7 +337,7 @@ def run_prefill(args, wl, env):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
             "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
 
-    if rank == 0 and world == 1 and not args.skip_e2e and not P:
+    if rank == 0 and world == 1 and not args.skip_e2e and not P and not proj:
         # end to end through the host-buffer entry point: H2D of the layer's inputs and D2H of its
         # result happen inside the timed region; host inputs rotate over a few pinned layer sets
         n_h = min(L, 2)
@@ -538,6 +546,8 @@ def main():
     ap.add_argument("--workload", default="qwen3_8b_prefill_32k", choices=list(synth.WORKLOAD_ORDER))
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (small case for profiling)")
+    ap.add_argument("--kv-layout", default="heads", choices=["heads", "proj"],
+                    help="prefill workloads: K/V as [H,T,D] (default) or as the projection writes them, [T,H,D]")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=32768,

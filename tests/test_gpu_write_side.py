@@ -133,3 +133,36 @@ def test_write_side_empty_input_and_argument_errors(binding):
     with pytest.raises(binding.KvzapError):
         binding.kvzap_prefill_write(ctx.handle, 3, X, Kp, Kp, None, 1, 0.0, 4, out, out, lengths)      # layer out of range
     ctx.close()
+
+
+def test_write_side_at_config3_size(binding, oracle):
+    """Four sequences of 16k tokens, Linear surrogate, K/V as [T,H,D]: everything checked in full."""
+    wl = synth.WORKLOADS["llama31_8b_prefill_4x16k"]
+    B, T = wl.batch, wl.seq_len
+    n_tokens, H, D, tau = B * T, wl.n_kv_heads, wl.head_dim, wl.tau
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, 1, n_tokens, max_seqs=B)
+    weights = synth.surrogate_weights(wl, 2, "cuda")
+    ctx.set_weights(0, *weights)
+    X = synth.hidden_states(n_tokens, wl.d_model, 77, "cuda", wl.token_scale_sigma)
+    K, V = synth.keys_values(H, n_tokens, D, 78, "cuda")
+    K_proj, V_proj = K.transpose(0, 1).contiguous(), V.transpose(0, 1).contiguous()
+    del K, V
+    cu = synth.cu_seqlens([T] * B)
+    K_out = parity.poison_like(torch.empty(H, n_tokens, D, dtype=torch.bfloat16, device="cuda"))
+    V_out = parity.poison_like(K_out)
+    lengths = torch.zeros(B, H, dtype=torch.int32, device="cuda")
+    scores = torch.empty(n_tokens, H, dtype=torch.float32, device="cuda")
+    binding.kvzap_prefill_write(ctx.handle, 0, X, K_proj, V_proj, torch.from_numpy(cu).cuda(), B, tau, wl.window,
+                                K_out, V_out, lengths, scores)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    want, _ = parity.check_scores(oracle, scores, X.cpu(), tuple(w.cpu() if w is not None else None for w in weights))
+    s = scores.cpu().numpy()
+    keep = parity.check_mask_band(oracle, s, want, tau, wl.window, cu)
+    K_ref, V_ref, len_ref = oracle.compact_write(synth.bits(K_proj.cpu()), synth.bits(V_proj.cpu()), keep, cu,
+                                                 fill=parity.POISON)
+    np.testing.assert_array_equal(lengths.cpu().numpy(), len_ref)
+    np.testing.assert_array_equal(synth.bits(K_out.cpu()), K_ref)
+    np.testing.assert_array_equal(synth.bits(V_out.cpu()), V_ref)
+    assert (len_ref >= wl.window).all()
+    ctx.close()
