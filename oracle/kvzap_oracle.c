@@ -331,6 +331,54 @@ int kvzap_oracle_compact_write_paged(const uint16_t *K_proj, const uint16_t *V_p
 }
 
 /*
+ * The consumer of the pruned cache: attention of ONE new token over ONE
+ * (sequence, layer, KV head) list of whatever length pruning left
+ * (Criterion 3 of the introduction and Discussion, "Implementation
+ * Challenges": per-head lengths differ, so the attention kernel must take
+ * variable-length lists).  The paper prints no formula of its own; this is
+ * the ordinary scaled dot-product softmax attention it refers to:
+ *   a[g,i]  = scale * sum_d q[g,d] * K[i,d]
+ *   p[g,i]  = exp(a[g,i]) / sum_j exp(a[g,j])
+ *   out[g]  = sum_i p[g,i] * V[i]
+ * for the G query heads g that share the KV head (grouped-query attention).
+ * q [G,D] bf16, K,V [n,D] bf16 (the list's rows, any order: the result does
+ * not depend on it), out [G,D] fp32 (one rounding from double).  n = 0 gives
+ * zeros.  The largest a[g,.] is subtracted before exp, which changes nothing
+ * mathematically and keeps exp in range.  Returns 0, or -1 without memory.
+ */
+int kvzap_oracle_attention(const uint16_t *q, int G, const uint16_t *K, const uint16_t *V,
+                           int64_t n, int D, double scale, float *out)
+{
+    double *a = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *acc = (double *)malloc(sizeof(double) * (size_t)D);
+    if (!a || !acc) { free(a); free(acc); return -1; }
+    for (int g = 0; g < G; ++g) {
+        double a_max = -INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += bf16_to_double(q[(int64_t)g * D + d]) * bf16_to_double(K[i * D + d]);
+            a[i] = scale * dot;
+            if (a[i] > a_max) a_max = a[i];
+        }
+        double denom = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            a[i] = exp(a[i] - a_max);
+            denom += a[i];
+        }
+        for (int d = 0; d < D; ++d) acc[d] = 0.0;
+        for (int64_t i = 0; i < n; ++i)
+            for (int d = 0; d < D; ++d)
+                acc[d] += a[i] * bf16_to_double(V[i * D + d]);
+        for (int d = 0; d < D; ++d)
+            out[(int64_t)g * D + d] = n > 0 ? (float)(acc[d] / denom) : 0.0f;
+    }
+    free(a);
+    free(acc);
+    return 0;
+}
+
+/*
  * Closed forms of Appendix B (per token, per layer).
  *   C        = 4 D_h (H_Q D + H D) + 6 D_h D_int      linear-projection FLOPs of a layer
  *   C_MLP    = 2 D_h (D_h/8) + 2 (D_h/8) H = D_h/4 (D_h + H)

@@ -51,6 +51,7 @@ def lib():
         L.kvzap_oracle_score_mlp.restype = ctypes.c_int
         L.kvzap_oracle_compact_paged.restype = ctypes.c_int
         L.kvzap_oracle_compact_write_paged.restype = ctypes.c_int
+        L.kvzap_oracle_attention.restype = ctypes.c_int
         for name in ("layer_flops", "mlp_flops", "linear_flops"):
             getattr(L, "kvzap_oracle_" + name).restype = ctypes.c_double
         L.kvzap_oracle_layer_flops.argtypes = [ctypes.c_int] * 5
@@ -244,6 +245,22 @@ def compact_write_paged(K_proj, V_proj, keep, page_tokens, n_pages_pool, max_pag
     if rc != 0:
         raise ValueError("page pool or page table too small")
     return K_pool, V_pool, table, lengths, int(used.value)
+
+
+def attention(q, K, V, scale):
+    """One new token's attention over one pruned list: q [G,D], K,V [n,D] bf16 bits -> out [G,D] fp32."""
+    q = _u16(q, 2)
+    G, D = q.shape
+    K = np.ascontiguousarray(K, dtype=np.uint16).reshape(-1, D)
+    V = np.ascontiguousarray(V, dtype=np.uint16).reshape(-1, D)
+    assert K.shape == V.shape
+    out = np.zeros((G, D), dtype=np.float32)
+    rc = lib().kvzap_oracle_attention(_c(q, ctypes.c_uint16), ctypes.c_int(G), _c(K, ctypes.c_uint16),
+                                      _c(V, ctypes.c_uint16), ctypes.c_int64(K.shape[0]), ctypes.c_int(D),
+                                      ctypes.c_double(scale), _c(out, ctypes.c_float))
+    if rc != 0:
+        raise MemoryError("oracle attention: out of memory")
+    return out
 
 
 def prune_prefill(X, weights, K, V, tau, w, cu_seqlens=None):
