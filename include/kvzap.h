@@ -274,6 +274,30 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
                                const void *hidden, const void *K_new, const void *V_new, float tau,
                                float *scores_out, void *stream);
 
+/*
+ * Attention of the newest token over the pruned cache (Introduction, Criterion 3;
+ * Discussion, "Implementation Challenges": lists of different lengths per head
+ * need an attention kernel that takes variable-length paged lists).  For every
+ * sequence b, layer l in [layer_begin, layer_end) and query head j, with KV head
+ * h = j / G, G = n_q_heads / H (grouped-query attention, consecutive query heads
+ * share a KV head):
+ *   O[l,b,j] = sum_i softmax_i(scale * Q[l,b,j] . K_i) V_i
+ * over all rows i list (b,l,h) holds at the time of the call: its paged prefix
+ * and the valid slots of its window (the row appended by the latest
+ * kvzap_decode_step included).  The order of a list's rows does not matter.
+ *   Q, O  [layer_end - layer_begin, n_seqs, n_q_heads, D] bf16 (device, 16-byte aligned)
+ *   scale >= 0, usually 1 / sqrt(D)
+ * An empty list gives zeros.  Arithmetic: bf16 products with fp32 accumulation,
+ * softmax in fp32, probabilities rounded to bf16 for the second product, one
+ * rounding of O to bf16.  Reads the cache only; one kernel launch, ordered on
+ * the stream after the decode steps enqueued before it.
+ * KVZAP_ERR_UNSUPPORTED unless D is 64 or 128, page_tokens and window are
+ * multiples of 16, and 1 <= G <= 8.  A bounded wait that runs out sets the
+ * status word to KVZAP_ERR_TIMEOUT and zeros the affected outputs.
+ */
+kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                    const void *Q, int32_t n_q_heads, float scale, void *O, void *stream);
+
 /* lengths [n_seqs, L, H] int32 (device): rows currently held by each list (prefix + window). */
 kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream);
 
@@ -312,7 +336,7 @@ kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, c
 
 /* Kernel identifiers for kvzap_get_profile. */
 enum { KVZAP_KERNEL_SCORE = 0, KVZAP_KERNEL_MASK = 1, KVZAP_KERNEL_SCAN = 2, KVZAP_KERNEL_COMPACT = 3,
-       KVZAP_KERNEL_DECODE_UPDATE = 4 };
+       KVZAP_KERNEL_DECODE_UPDATE = 4, KVZAP_KERNEL_ATTENTION = 5 };
 
 /*
  * Per-kernel timing with CUDA events on the launching stream (a measurement

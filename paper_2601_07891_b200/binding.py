@@ -62,6 +62,7 @@ SIGNATURES = {
     "kvzap_cache_create": (_i32, [_vp, ctypes.POINTER(_vp), _i32, _i32, _i32, _vp, _vp, _i64, _i32]),
     "kvzap_cache_destroy": (_i32, [_vp]),
     "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
+    "kvzap_decode_attention": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
     "kvzap_cache_lengths": (_i32, [_vp, _vp, _vp]),
     "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
     "kvzap_prefill_to_cache": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
@@ -324,6 +325,17 @@ def prepare_prefill_write_paged(handle, layer, hidden, K_proj, V_proj, cu_seqlen
                         (hidden, K_proj, V_proj, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used, scores_out))
 
 
+def kvzap_decode_attention(handle, cache, layer_begin, layer_end, Q, scale, O, stream=None):
+    """Q, O [layer_end - layer_begin, n_seqs, n_q_heads, D] bf16 on the device."""
+    _check(handle, load().kvzap_decode_attention(handle, cache, layer_begin, layer_end, _ptr(Q), Q.shape[2], scale,
+                                                 _ptr(O), _stream(stream)))
+
+
+def prepare_decode_attention(handle, cache, layer_begin, layer_end, Q, scale, O, stream=None) -> PreparedCall:
+    args = (handle, cache, layer_begin, layer_end, _ptr(Q), Q.shape[2], scale, _ptr(O), _stream(stream))
+    return PreparedCall("kvzap_decode_attention", handle, args, (Q, O))
+
+
 def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None,
                         stream=None) -> PreparedCall:
     args = (handle, cache, layer_begin, layer_end, _ptr(hidden), _ptr(K_new), _ptr(V_new), tau, _ptr(scores_out),
@@ -331,7 +343,7 @@ def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_
     return PreparedCall("kvzap_decode_step", handle, args, (hidden, K_new, V_new, scores_out))
 
 
-KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3, "decode_update": 4}
+KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3, "decode_update": 4, "attention": 5}
 
 
 def kvzap_set_profiling(handle, enable):

@@ -1,0 +1,278 @@
+// Attention of the new token over the pruned cache (Introduction, Criterion 3; Discussion,
+// "Implementation Challenges": per-head list lengths differ, so the attention kernel has to take
+// variable-length lists).  One CTA per (sequence, layer, KV head) list; the G query heads that share
+// the KV head (grouped-query attention) are processed together, so every K and V row is read from
+// HBM exactly once per step.  The kernel is bound by those reads.
+//
+// A list is its paged prefix (prefix_len rows in pages of page_tokens rows) plus the valid slots of
+// its window ring; softmax attention does not depend on the order of the rows, so the two parts are
+// simply walked one after the other in tiles of 16 rows.  Warp w of the CTA takes tiles w, w + W,
+// w + 2W, ... with its own online-softmax state and its own ring of shared-memory stages: lane 0
+// issues the TMA loads of a tile (K and V, 128-byte swizzle, two 64-element halves per row when
+// D = 128) onto the stage's mbarrier, the warp waits for it, and nothing is shared between warps
+// until the end, when the partial (max, sum, output) triples are merged through shared memory.
+//
+// Math per tile, on the warp-level tensor-core path (the work is HBM-bound; 16-row MMAs are enough):
+//   S[16 x 16]  = Q[16 x D] K^T      m16n8k16, Q rows 0..G-1 real, the rest zero
+//   P           = exp2(S * scale * log2(e) - running max), rows beyond the list's end masked
+//   O[16 x D]  += P[16 x 16] V
+// Rows of a partly filled tile that lie past the end are excluded from the softmax, and their V
+// rows are zeroed in shared memory first (stale pool memory may hold NaN bit patterns).
+#pragma once
+
+#include "decode_kernels.cuh"
+#include "ptx.cuh"
+
+namespace kvzap {
+
+constexpr int kAttnWarps = 4;
+constexpr int kAttnStages = 3;
+constexpr int kAttnTileRows = 16;
+constexpr int kAttnThreads = kAttnWarps * 32;
+constexpr int kAttnMaxGroup = 8;                 // query heads per KV head (rows 0..7 of the 16-row MMA)
+constexpr uint32_t kAttnHalfBytes = kAttnTileRows * 128;   // 16 rows x 64 bf16
+
+struct AttnParams {
+    CacheView c;
+    int32_t layer0, n_layers_call;
+    int32_t group;              // G = query heads per KV head, 1..8
+    float scale_log2e;          // softmax scale times log2(e)
+    const uint16_t *q;          // [n_layers_call][B][H * G][D] bf16
+    uint16_t *out;              // same shape
+    int32_t *status;
+};
+
+__host__ __device__ constexpr uint32_t attn_stage_bytes(int head_dim) { return 2u * (head_dim / 64) * kAttnHalfBytes; }
+__host__ __device__ constexpr uint32_t attn_smem_bytes(int head_dim)
+{
+    return kAttnWarps * kAttnStages * attn_stage_bytes(head_dim) + 1024u /* alignment */ + 256u /* barriers */;
+}
+
+template <int kD>
+__global__ void __launch_bounds__(kAttnThreads)
+decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_constant__ CUtensorMap tmap_vpool,
+                   const __grid_constant__ CUtensorMap tmap_kring, const __grid_constant__ CUtensorMap tmap_vring,
+                   const AttnParams p)
+{
+    constexpr int kHalves = kD / 64;
+    constexpr uint32_t kStageBytes = attn_stage_bytes(kD);
+    constexpr int kNTiles = kD / 8;              // 8-column tiles of the output
+    extern __shared__ uint8_t attn_smem_raw[];
+    const uint32_t raw_addr = smem_u32(attn_smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t *smem = attn_smem_raw + pad;
+    const uint32_t smem_base = raw_addr + pad;
+    const uint32_t bars = smem_base + kAttnWarps * kAttnStages * kStageBytes;      // [warp][stage] mbarriers
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kAttnWarps * kAttnStages * kStageBytes + 8 * kAttnWarps * kAttnStages);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const CacheView &c = p.c;
+    const int H = c.n_heads, B = c.n_seqs;
+    const int list = blockIdx.x;
+    const int h = list % H, b = (list / H) % B, l_rel = list / (H * B);
+    const int layer = p.layer0 + l_rel;
+    const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer) * H + h;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kAttnWarps * kAttnStages; ++i) mbar_init(bars + 8 * i, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_kpool);
+        prefetch_tensormap(&tmap_vpool);
+        prefetch_tensormap(&tmap_kring);
+        prefetch_tensormap(&tmap_vring);
+    }
+    __syncthreads();
+
+    const int32_t n_total = __ldcg(c.n_tokens + li);
+    const int32_t n_prefix = __ldcg(c.prefix_len + li);
+    const int32_t n_ring = c.window > 0 ? (n_total < c.window ? n_total : c.window) : 0;
+    const int tiles_per_page = c.page_tokens / kAttnTileRows;
+    const int n_pt = (n_prefix + kAttnTileRows - 1) / kAttnTileRows;
+    const int n_rt = (n_ring + kAttnTileRows - 1) / kAttnTileRows;
+    const int n_tiles = n_pt + n_rt;
+    const int32_t *pages = c.page_table + li * c.max_pages;
+
+    // the query rows of this KV head as A fragments: row g = lane / 4 (real for g < G), two packed
+    // elements at columns 16 ks + 2 (lane % 4) and the same + 8
+    const int g = lane >> 2, qc = (lane & 3) * 2;
+    const int Hq = H * p.group;
+    uint32_t qa[kD / 16][2];
+    {
+        const uint16_t *qrow = p.q + ((static_cast<int64_t>(l_rel) * B + b) * Hq + h * p.group + g) * kD;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+            qa[ks][0] = qa[ks][1] = 0u;
+            if (g < p.group) {
+                qa[ks][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + qc));
+                qa[ks][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + qc));
+            }
+        }
+    }
+
+    float o[kNTiles][4];
+#pragma unroll
+    for (int i = 0; i < kNTiles; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
+    float m_run = -INFINITY, l_run = 0.0f;
+
+    const uint32_t my_stages = smem_base + warp * kAttnStages * kStageBytes;
+    const uint32_t my_bars = bars + 8 * warp * kAttnStages;
+    const uint64_t policy = l2_policy_evict_first();
+
+    // first row (in its tensor map) of tile t of this list; needs the page number for prefix tiles
+    auto tile_row = [&](int t) -> int32_t {
+        if (t < n_pt) {
+            const int32_t page = __ldcg(pages + t / tiles_per_page);
+            return page * c.page_tokens + (t % tiles_per_page) * kAttnTileRows;
+        }
+        return static_cast<int32_t>(li * c.window) + (t - n_pt) * kAttnTileRows;
+    };
+    auto issue = [&](int t, int32_t row, int stage) {
+        const uint32_t dst = my_stages + stage * kStageBytes;
+        const uint32_t bar = my_bars + 8 * stage;
+        const bool prefix = t < n_pt;
+        mbar_arrive_expect_tx(bar, kStageBytes);
+#pragma unroll
+        for (int hf = 0; hf < kHalves; ++hf) {
+            tma_load_2d(dst + hf * kAttnHalfBytes, prefix ? &tmap_kpool : &tmap_kring, bar, hf * 64, row, policy);
+            tma_load_2d(dst + (kHalves + hf) * kAttnHalfBytes, prefix ? &tmap_vpool : &tmap_vring, bar, hf * 64, row, policy);
+        }
+    };
+
+    // prologue: fill the stages; row_next belongs to the first tile not yet issued
+    int t_issue = warp;
+    for (int s = 0; s < kAttnStages && t_issue < n_tiles; ++s, t_issue += kAttnWarps) {
+        const int32_t row = tile_row(t_issue);
+        if (lane == 0) issue(t_issue, row, s);
+    }
+    int32_t row_next = t_issue < n_tiles ? tile_row(t_issue) : 0;
+
+    bool ok = true;
+    int stage = 0;
+    uint32_t parity = 0;
+    for (int t = warp; t < n_tiles; t += kAttnWarps) {
+        if (!__all_sync(0xffffffffu, mbar_wait(my_bars + 8 * stage, parity, abort_flag))) {
+            ok = false;
+            break;
+        }
+        const uint32_t sK = my_stages + stage * kStageBytes;
+        const uint32_t sV = sK + kHalves * kAttnHalfBytes;
+        const int valid = t < n_pt ? n_prefix - t * kAttnTileRows : n_ring - (t - n_pt) * kAttnTileRows;   // >= 1
+        if (valid < kAttnTileRows) {
+            // zero the V rows past the end of the list
+            const int n_units = (kAttnTileRows - valid) * kHalves * 8;
+            for (int i = lane; i < n_units; i += 32) {
+                const int r = valid + i / (kHalves * 8), rem = i % (kHalves * 8);
+                *reinterpret_cast<uint4 *>(smem + (sV - smem_base) + (rem >> 3) * kAttnHalfBytes + r * 128 + ((rem & 7) << 4)) =
+                    make_uint4(0u, 0u, 0u, 0u);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+        }
+
+        // ---- S = Q K^T: two 8-row column tiles
+        float s0[4] = {0.0f, 0.0f, 0.0f, 0.0f}, s1[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        {
+            const int mi = lane >> 3, r8 = lane & 7;
+            const int krow = (mi >> 1) * 8 + r8;
+#pragma unroll
+            for (int ks = 0; ks < kD / 16; ++ks) {
+                const int chunk = 2 * ks + (mi & 1);
+                const uint32_t addr = sK + (chunk >> 3) * kAttnHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4);
+                uint32_t k0, k1, k2, k3;
+                ldmatrix_x4(addr, k0, k1, k2, k3);
+                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, k0, k1);
+                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, k2, k3);
+            }
+        }
+        // ---- online softmax for row g: this lane holds columns qc, qc + 1 of both column tiles
+        float v00 = s0[0] * p.scale_log2e, v01 = s0[1] * p.scale_log2e;
+        float v10 = s1[0] * p.scale_log2e, v11 = s1[1] * p.scale_log2e;
+        if (valid < kAttnTileRows) {
+            if (qc >= valid) v00 = -INFINITY;
+            if (qc + 1 >= valid) v01 = -INFINITY;
+            if (8 + qc >= valid) v10 = -INFINITY;
+            if (9 + qc >= valid) v11 = -INFINITY;
+        }
+        float mx = fmaxf(fmaxf(v00, v01), fmaxf(v10, v11));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);             // finite: row 0 of a tile is always valid
+        const float alpha = fast_ex2(m_run - m_new);      // 0 on the first tile
+        const float p00 = fast_ex2(v00 - m_new), p01 = fast_ex2(v01 - m_new);
+        const float p10 = fast_ex2(v10 - m_new), p11 = fast_ex2(v11 - m_new);
+        l_run = l_run * alpha + ((p00 + p01) + (p10 + p11));
+        m_run = m_new;
+#pragma unroll
+        for (int i = 0; i < kNTiles; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
+        const uint32_t pa0 = pack_bf16x2(p00, p01), pa2 = pack_bf16x2(p10, p11);
+
+        // ---- O += P V: two 8-column output tiles per ldmatrix
+        {
+            const int mi = lane >> 3, r8 = lane & 7;
+            const int krow = (mi & 1) * 8 + r8;
+#pragma unroll
+            for (int ndp = 0; ndp < kD / 16; ++ndp) {
+                const int chunk = 2 * ndp + (mi >> 1);
+                const uint32_t addr = sV + (chunk >> 3) * kAttnHalfBytes + krow * 128 + (((chunk & 7) ^ (krow & 7)) << 4);
+                uint32_t v0, v1, v2, v3;
+                ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+                mma_bf16_16816(o[2 * ndp], pa0, 0u, pa2, 0u, v0, v1);
+                mma_bf16_16816(o[2 * ndp + 1], pa0, 0u, pa2, 0u, v2, v3);
+            }
+        }
+        __syncwarp();                                     // all lanes are done with this stage
+        if (t_issue < n_tiles) {
+            if (lane == 0) issue(t_issue, row_next, stage);
+            t_issue += kAttnWarps;
+            row_next = t_issue < n_tiles ? tile_row(t_issue) : 0;
+        }
+        if (++stage == kAttnStages) { stage = 0; parity ^= 1u; }
+    }
+    if (!ok) {
+        // a wait ran out: report it, give the copies already in flight a fixed time to land, merge nothing
+        if (lane == 0) {
+            atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000LL) { }
+        }
+        __syncwarp();
+    }
+
+    // ---- merge the warps' partial results: [warp] { m[8], l[8], O[8][kD] } in the warp's own stages
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    {
+        float *mine = reinterpret_cast<float *>(smem + warp * kAttnStages * kStageBytes);
+        if ((lane & 3) == 0) { mine[g] = m_run; mine[8 + g] = l_run; }
+#pragma unroll
+        for (int i = 0; i < kNTiles; ++i) {
+            mine[16 + g * kD + i * 8 + qc] = o[i][0];
+            mine[16 + g * kD + i * 8 + qc + 1] = o[i][1];
+        }
+    }
+    __syncthreads();
+    const bool failed = *abort_flag != 0;
+    for (int idx = threadIdx.x; idx < p.group * kD; idx += kAttnThreads) {
+        const int gq = idx / kD, d = idx % kD;
+        float m_all = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kAttnWarps; ++w)
+            m_all = fmaxf(m_all, reinterpret_cast<const float *>(smem + w * kAttnStages * kStageBytes)[gq]);
+        float num = 0.0f, den = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kAttnWarps; ++w) {
+            const float *part = reinterpret_cast<const float *>(smem + w * kAttnStages * kStageBytes);
+            const float f = fast_ex2(part[gq] - m_all);   // 0 for a warp that saw no tile
+            if (part[gq] > -INFINITY) {
+                num += part[16 + gq * kD + d] * f;
+                den += part[8 + gq] * f;
+            }
+        }
+        const float r = (den > 0.0f && !failed) ? num / den : 0.0f;      // an empty list gives zeros
+        p.out[((static_cast<int64_t>(l_rel) * B + b) * Hq + h * p.group + gq) * kD + d] =
+            static_cast<uint16_t>(pack_bf16x2(r, 0.0f) & 0xffffu);
+    }
+}
+
+}  // namespace kvzap

@@ -11,6 +11,7 @@
 #include <new>
 #include <vector>
 
+#include "attn_kernel.cuh"
 #include "decode_kernels.cuh"
 #include "prune_kernels.cuh"
 #include "score_kernel.cuh"
@@ -1108,6 +1109,9 @@ struct kvzap_cache {
     // fused decode steps: per-cluster count of completed steps on the device, and the host's view of it
     int32_t *done = nullptr;             // [n_layers * ceil(n_seqs / 128)][4]: one per cluster of the fused step
     std::vector<int32_t> steps_done;     // per layer
+    // attention over the cache: tensor maps of the page pools and of the window rings (built on first use)
+    CUtensorMap tm_kpool, tm_vpool, tm_kring, tm_vring;
+    int attn_state = 0;                  // 0 not built yet, 1 ready, -1 this cache's geometry is not supported
 };
 
 namespace kvzap {
@@ -1392,6 +1396,77 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
                                            static_cast<const float *>(scores), static_cast<const uint4 *>(K_new),
                                            static_cast<const uint4 *>(V_new), tau, ctx->status_dev,
                                            ctx->last_score_early ? 1 : 0));
+    }
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                    const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_)
+{
+    if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    const CacheView &v = cache->v;
+    if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "attention: layer range [%d, %d) invalid", layer_begin, layer_end);
+    if (!Q || !O || !aligned16(Q) || !aligned16(O))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "attention: Q and O must be non-NULL and 16-byte aligned");
+    if (n_q_heads < c.n_kv_heads || n_q_heads % c.n_kv_heads != 0 || n_q_heads / c.n_kv_heads > kAttnMaxGroup)
+        return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: n_q_heads must be 1..%d times the number of KV heads",
+                    kAttnMaxGroup);
+    if (!(scale == scale) || scale < 0.0f) return fail(ctx, KVZAP_ERR_INVALID_ARG, "attention: scale must be >= 0");
+    DeviceGuard guard(c.device);
+    if (cache->attn_state == 0) {
+        // tiles of 16 rows: pages and the window must be whole numbers of them; rows of 64 or 128 elements
+        const int64_t pool_rows = v.n_pages_pool * v.page_tokens;
+        const int64_t ring_rows = cache->n_lists * (v.window > 0 ? v.window : 1);
+        const bool ok = (c.head_dim == 64 || c.head_dim == 128) && v.page_tokens % kAttnTileRows == 0 &&
+                        v.window % kAttnTileRows == 0 && pool_rows < (int64_t{1} << 31) && ring_rows < (int64_t{1} << 31) &&
+                        pool_rows >= kAttnTileRows;
+        cache->attn_state = -1;
+        if (ok) {
+            const void *kring = v.window > 0 ? static_cast<const void *>(v.k_ring) : static_cast<const void *>(v.k_pool);
+            const void *vring = v.window > 0 ? static_cast<const void *>(v.v_ring) : static_cast<const void *>(v.v_pool);
+            const uint64_t rr = v.window > 0 ? static_cast<uint64_t>(ring_rows) : static_cast<uint64_t>(pool_rows);
+            if (make_tmap(ctx, &cache->tm_kpool, v.k_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                make_tmap(ctx, &cache->tm_vpool, v.v_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                make_tmap(ctx, &cache->tm_kring, kring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                make_tmap(ctx, &cache->tm_vring, vring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK) {
+                cudaError_t e = c.head_dim == 128
+                    ? cudaFuncSetAttribute(decode_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(attn_smem_bytes(128)))
+                    : cudaFuncSetAttribute(decode_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(attn_smem_bytes(64)));
+                if (e == cudaSuccess) cache->attn_state = 1;
+            }
+        }
+    }
+    if (cache->attn_state != 1)
+        return fail(ctx, KVZAP_ERR_UNSUPPORTED,
+                    "attention needs head_dim 64 or 128, page_tokens and window multiples of %d, fewer than 2^31 rows",
+                    kAttnTileRows);
+    AttnParams p;
+    memset(&p, 0, sizeof p);
+    p.c = v;
+    p.layer0 = layer_begin;
+    p.n_layers_call = layer_end - layer_begin;
+    p.group = n_q_heads / c.n_kv_heads;
+    p.scale_log2e = scale * 1.4426950408889634f;
+    p.q = static_cast<const uint16_t *>(Q);
+    p.out = static_cast<uint16_t *>(O);
+    p.status = ctx->status_dev;
+    const int64_t n_ctas = static_cast<int64_t>(p.n_layers_call) * v.n_seqs * v.n_heads;
+    if (n_ctas > 0x7fffffffLL) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: too many lists for one launch");
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_ATTENTION, stream);
+        if (c.head_dim == 128)
+            decode_attn_kernel<128><<<static_cast<unsigned>(n_ctas), kAttnThreads, attn_smem_bytes(128), stream>>>(
+                cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+        else
+            decode_attn_kernel<64><<<static_cast<unsigned>(n_ctas), kAttnThreads, attn_smem_bytes(64), stream>>>(
+                cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+        KVZAP_CUDA(ctx, cudaGetLastError());
     }
     ctx->launches += 1;
     return KVZAP_OK;
