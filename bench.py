@@ -475,6 +475,90 @@ def run_decode(args, wl, env):
     return line
 
 
+def run_attention(args, wl, env):
+    """The consumer of the pruned cache (not part of the pruning metric; run with --attention): the new
+    token's attention over every list of a few layers of the decode workload, lists fully backed by memory.
+    One step = one kvzap_decode_attention call over those layers."""
+    import numpy as np
+    import torch
+    from paper_2601_07891_b200 import binding, synth
+    dev, rank, world, barrier = env["dev"], env["rank"], env["world"], env["barrier"]
+    B, H, D, w, P = wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
+    L = args.layers if args.layers > 0 else 4
+    G = 4                                             # 32 query heads over 8 KV heads
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index)
+    for l in range(L):
+        ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
+    n_lists = B * L * H
+    # pre-pruned lists: a sequence of prefix_min..prefix_max tokens of which every (layer, head) kept 15-35 %
+    rng = np.random.default_rng(777 + rank)
+    seq_len = rng.integers(wl.prefix_min, wl.prefix_max + 1, size=B)
+    kept = rng.uniform(0.15, 0.35, size=(B, L, H))
+    prefix = np.maximum(1, (seq_len[:, None, None] * kept)).astype(np.int32).reshape(-1)      # list index (b, l, h)
+    grow_pages = (w + 16) // P + 2
+    pages_of = (prefix + P - 1) // P + grow_pages
+    first = np.concatenate([[0], np.cumsum(pages_of)[:-1]]).astype(np.int64)
+    n_pool = int(pages_of.sum())
+    max_pages = int(pages_of.max())
+    K_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
+    V_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
+    table = torch.from_numpy((first[:, None] + np.arange(max_pages)[None, :]).astype(np.int32)).to(dev)
+    cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
+    # imported page tables are private to each list (contiguous runs); growth pages come from each run's tail
+    binding.kvzap_cache_import(ctx.handle, cache, torch.from_numpy(prefix).to(dev), table, n_pool)
+    Xd = synth.hidden_states(L * B, wl.d_model, 1, dev).view(L, B, wl.d_model)
+    Kn, Vn = synth.keys_values(L * B, H, D, 2, dev)
+    for _ in range(w + 3):            # fill every window; tau = +inf keeps the prefixes as imported
+        binding.kvzap_decode_step(ctx.handle, cache, 0, L, Xd, Kn.view(L, B, H, D), Vn.view(L, B, H, D), float("inf"), None)
+    lengths = torch.zeros(B, L, H, dtype=torch.int32, device=dev)
+    binding.kvzap_cache_lengths(ctx.handle, cache, lengths)
+    torch.cuda.synchronize()
+    if ctx.poll_status() != 0:
+        raise RuntimeError("device status word set while the cache was filled")
+    rows = float(lengths.sum().item())
+    Qs = [synth.hidden_states(L * B * H * G, D, 50 + i, dev).view(L, B, H * G, D) for i in range(3)]
+    Os = [torch.empty_like(q) for q in Qs]
+    calls = [binding.prepare_decode_attention(ctx.handle, cache, 0, L, Qs[i], 1.0 / D ** 0.5, Os[i]) for i in range(3)]
+    n_warm, steps = max(args.warmup, 3), min(args.steps, 30)
+    for i in range(n_warm):
+        calls[i % 3]()
+    barrier()
+    sampler = ClockSampler(dev.index)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count()
+    sampler.start()
+    barrier()
+    e0.record()
+    for i in range(steps):
+        calls[i % 3]()
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = env["max_over_ranks"](e0.elapsed_time(e1)) / steps
+    if ctx.poll_status() != 0:
+        raise RuntimeError("device status word set during the timed region")
+    peaks, peak_src = load_peaks()
+    alg_bytes = rows * 2 * D * 2 + 2 * L * B * H * G * D * 2        # every K and V row once; Q read, O written
+    achieved = alg_bytes / (ms * 1e-3) / 1e9
+    line = {"metric": "decode attention over the pruned cache, sequences/sec per layer", "value": world * B / (ms * 1e-3 / L),
+            "unit": "sequences/s/layer", "n_gpus": world, "steps": steps, "warmup": n_warm, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name + " / attention", "n_kv_heads": H, "n_q_heads": H * G, "head_dim": D,
+                       "n_layers": L, "batch": B, "window": w, "page_tokens": P,
+                       "sequence_len": [wl.prefix_min, wl.prefix_max], "kept_fraction": [0.15, 0.35],
+                       "rows_per_list_mean": rows / n_lists,
+                       "l2": "the lists read by one call (%.1f GB) exceed L2" % (rows * 2 * D * 2 / 1e9),
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "clocks": clocks, "gpu_launches": int(ctx.launch_count() - launches0),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name + "/attention"),
+                         "kernel": "decode_attn_kernel", "peak_source": peak_src, "kernel_ms": ms,
+                         "algorithmic_bytes_per_step": alg_bytes}}
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
+    return line
+
+
 def make_env(backend="nccl"):
     """Process-group plumbing of the N > 1 run: replicas only, so all it carries is the barrier around the
     timed region and the maximum over ranks of the timed duration.  `backend="gloo"` runs the same code
@@ -523,7 +607,12 @@ def run_ours(args, wl):
         raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
     env = make_env("nccl")
     rank, world = env["rank"], env["world"]
-    line = run_decode(args, wl, env) if wl.decode_steps > 0 else run_prefill(args, wl, env)
+    if args.attention:
+        if wl.decode_steps == 0:
+            raise SystemExit("--attention goes with the decode workload")
+        line = run_attention(args, wl, env)
+    else:
+        line = run_decode(args, wl, env) if wl.decode_steps > 0 else run_prefill(args, wl, env)
     if rank == 0 and world == 1 and not args.skip_cpu and wl.decode_steps == 0:
         # the oracle on the host cores, bounded sample
         n_sample = min(wl.batch * wl.seq_len, args.ref_tokens)
@@ -548,6 +637,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (small case for profiling)")
     ap.add_argument("--kv-layout", default="heads", choices=["heads", "proj"],
                     help="prefill workloads: K/V as [H,T,D] (default) or as the projection writes them, [T,H,D]")
+    ap.add_argument("--attention", action="store_true",
+                    help="decode workload: time the attention over the pruned cache instead of the pruning step")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=32768,

@@ -166,3 +166,58 @@ def test_attention_empty_cache_and_argument_errors(binding):
         binding.kvzap_decode_attention(ctx.handle, cache7, 0, 1, Q, 0.1, O)
     binding.kvzap_cache_destroy(cache7)
     ctx.close()
+
+
+def test_attention_at_bench_size_sampled_lists(binding, oracle):
+    """128 sequences x 8 KV heads with lists of 1k..8k pruned rows plus a full window of 128, the
+    launch shape bench.py --attention times (one layer): sampled lists against the oracle."""
+    d_model, H, D, P, w, B, G = 256, 8, 128, 16, 128, 128, 4
+    ctx = binding.Kvzap(d_model, 0, H, D, 1, max_tokens=B)
+    W, bias = synth.linear_weights(d_model, H, 3)
+    ctx.set_weights(0, parity.dev(W), parity.dev(bias))
+    n_lists = B * H
+    rng = np.random.default_rng(99)
+    prefix = rng.integers(1000, 8001, size=n_lists).astype(np.int32)
+    prefix[:4] = [1, 15, 16, 17]                      # ragged first tiles
+    pages_of = (prefix + P - 1) // P
+    first = np.concatenate([[0], np.cumsum(pages_of)[:-1]]).astype(np.int64)
+    n_pool, max_pages = int(pages_of.sum()), int(pages_of.max())
+    Kp, Vp = synth.keys_values(1, n_pool * P, D, seed=123, device="cuda")          # [1, rows, D]
+    K_pool, V_pool = Kp.view(n_pool, P, D), Vp.view(n_pool, P, D)
+    # rows past a list's end inside its last page must not matter: overwrite them with NaN
+    last_fill = prefix - (pages_of - 1) * P
+    for li in range(0, n_lists, 37):
+        pg = int(first[li] + pages_of[li] - 1)
+        K_pool[pg, int(last_fill[li]):] = float("nan")
+        V_pool[pg, int(last_fill[li]):] = float("nan")
+    table = torch.from_numpy((first[:, None] + np.arange(max_pages)[None, :]).astype(np.int32)).cuda()
+    cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
+    binding.kvzap_cache_import(ctx.handle, cache, torch.from_numpy(prefix).cuda(), table, n_pool)
+    n_steps = w + 3
+    new_rows = []
+    for step in range(n_steps):
+        X = parity.dev(synth.hidden_states(B, d_model, seed=600 + step)).view(1, B, d_model)
+        Kn, Vn = synth.keys_values(B, H, D, seed=700 + step)                       # [B, H, D]
+        new_rows.append((synth.bits(Kn), synth.bits(Vn)))
+        binding.kvzap_decode_step(ctx.handle, cache, 0, 1, X, parity.dev(Kn).view(1, B, H, D),
+                                  parity.dev(Vn).view(1, B, H, D), float("inf"), None)    # nothing joins the prefix
+    Q = synth.hidden_states(B * H * G, D, seed=8).view(1, B, H * G, D)
+    O = torch.zeros(1, B, H * G, D, dtype=torch.bfloat16, device="cuda")
+    scale = 1.0 / np.sqrt(D)
+    binding.kvzap_decode_attention(ctx.handle, cache, 0, 1, parity.dev(Q), scale, O)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got = O.float().cpu().numpy()[0]
+    assert np.isfinite(got).all()
+    Qb = synth.bits(Q)[0]
+    Kp_bits, Vp_bits = synth.bits(K_pool.cpu()).reshape(-1, D), synth.bits(V_pool.cpu()).reshape(-1, D)
+    sample = sorted(set([0, 1, 2, 3, 37, 74, n_lists - 1] + rng.integers(0, n_lists, 20).tolist()))
+    for li in sample:
+        b, h = li // H, li % H                         # one layer: list index = b * H + h
+        r0 = int(first[li]) * P
+        Kd = np.concatenate([Kp_bits[r0:r0 + int(prefix[li])]] + [new_rows[s][0][b, h][None] for s in range(n_steps - w, n_steps)])
+        Vd = np.concatenate([Vp_bits[r0:r0 + int(prefix[li])]] + [new_rows[s][1][b, h][None] for s in range(n_steps - w, n_steps)])
+        want = oracle.attention(Qb[b, h * G:(h + 1) * G], Kd, Vd, scale)
+        assert np.abs(got[b, h * G:(h + 1) * G] - want).max() <= ATTN_ATOL, li
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
