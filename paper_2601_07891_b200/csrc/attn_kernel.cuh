@@ -11,6 +11,10 @@
 // issues the TMA loads of a tile (K and V, 128-byte swizzle, two 64-element halves per row when
 // D = 128) onto the stage's mbarrier, the warp waits for it, and nothing is shared between warps
 // until the end, when the partial (max, sum, output) triples are merged through shared memory.
+// When a call has too few lists to keep every SM busy to the end (one layer of a moderate batch, or
+// a few long sequences), each list is cut into n_parts equal runs of tiles, one CTA each; the parts
+// leave their triples in global memory and the part that arrives last (a counter per list) merges
+// them in part order, so the result does not depend on which one that was.
 //
 // Math per tile, on the warp-level tensor-core path (the work is HBM-bound; 16-row MMAs are enough):
 //   S[16 x 16]  = Q[16 x D] K^T      m16n8k16, Q rows 0..G-1 real, the rest zero
@@ -40,6 +44,9 @@ struct AttnParams {
     const uint16_t *q;          // [n_layers_call][B][H * G][D] bf16
     uint16_t *out;              // same shape
     int32_t *status;
+    int32_t n_parts;            // CTAs per list (1 = the CTA writes the output itself)
+    float *part_scratch;        // n_parts > 1: [list][part] { m[8], l[8], O[8][D] }
+    uint32_t *part_arrive;      // n_parts > 1: [list] parts that have stored their triple; back to 0 after the launch
 };
 
 __host__ __device__ constexpr uint32_t attn_stage_bytes(int head_dim) { return 2u * (head_dim / 64) * kAttnHalfBytes; }
@@ -68,7 +75,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const CacheView &c = p.c;
     const int H = c.n_heads, B = c.n_seqs;
-    const int list = blockIdx.x;
+    const int list = blockIdx.x / p.n_parts, part = blockIdx.x % p.n_parts;
     const int h = list % H, b = (list / H) % B, l_rel = list / (H * B);
     const int layer = p.layer0 + l_rel;
     const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer) * H + h;
@@ -90,7 +97,10 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     const int tiles_per_page = c.page_tokens / kAttnTileRows;
     const int n_pt = (n_prefix + kAttnTileRows - 1) / kAttnTileRows;
     const int n_rt = (n_ring + kAttnTileRows - 1) / kAttnTileRows;
-    const int n_tiles = n_pt + n_rt;
+    const int n_tiles_list = n_pt + n_rt;
+    // this CTA's run of the list's tiles
+    const int t_begin = static_cast<int>(static_cast<int64_t>(n_tiles_list) * part / p.n_parts);
+    const int n_tiles = static_cast<int>(static_cast<int64_t>(n_tiles_list) * (part + 1) / p.n_parts);
     const int32_t *pages = c.page_table + li * c.max_pages;
 
     // the query rows of this KV head as A fragments: row g = lane / 4 (real for g < G), two packed
@@ -140,7 +150,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     };
 
     // prologue: fill the stages; row_next belongs to the first tile not yet issued
-    int t_issue = warp;
+    int t_issue = t_begin + warp;
     for (int s = 0; s < kAttnStages && t_issue < n_tiles; ++s, t_issue += kAttnWarps) {
         const int32_t row = tile_row(t_issue);
         if (lane == 0) issue(t_issue, row, s);
@@ -150,7 +160,7 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     bool ok = true;
     int stage = 0;
     uint32_t parity = 0;
-    for (int t = warp; t < n_tiles; t += kAttnWarps) {
+    for (int t = t_begin + warp; t < n_tiles; t += kAttnWarps) {
         if (!__all_sync(0xffffffffu, mbar_wait(my_bars + 8 * stage, parity, abort_flag))) {
             ok = false;
             break;
@@ -253,6 +263,8 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     }
     __syncthreads();
     const bool failed = *abort_flag != 0;
+    const int64_t out_row0 = (static_cast<int64_t>(l_rel) * B + b) * Hq + h * p.group;
+    float *unit = p.n_parts > 1 ? p.part_scratch + (static_cast<int64_t>(list) * p.n_parts + part) * (16 + kAttnMaxGroup * kD) : nullptr;
     for (int idx = threadIdx.x; idx < p.group * kD; idx += kAttnThreads) {
         const int gq = idx / kD, d = idx % kD;
         float m_all = -INFINITY;
@@ -262,16 +274,55 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         float num = 0.0f, den = 0.0f;
 #pragma unroll
         for (int w = 0; w < kAttnWarps; ++w) {
-            const float *part = reinterpret_cast<const float *>(smem + w * kAttnStages * kStageBytes);
-            const float f = fast_ex2(part[gq] - m_all);   // 0 for a warp that saw no tile
-            if (part[gq] > -INFINITY) {
-                num += part[16 + gq * kD + d] * f;
-                den += part[8 + gq] * f;
+            const float *wp = reinterpret_cast<const float *>(smem + w * kAttnStages * kStageBytes);
+            if (wp[gq] > -INFINITY) {                       // a warp that saw no tile contributes nothing
+                const float f = fast_ex2(wp[gq] - m_all);
+                num += wp[16 + gq * kD + d] * f;
+                den += wp[8 + gq] * f;
             }
         }
-        const float r = (den > 0.0f && !failed) ? num / den : 0.0f;      // an empty list gives zeros
-        p.out[((static_cast<int64_t>(l_rel) * B + b) * Hq + h * p.group + gq) * kD + d] =
-            static_cast<uint16_t>(pack_bf16x2(r, 0.0f) & 0xffffu);
+        if (p.n_parts == 1) {
+            const float r = (den > 0.0f && !failed) ? num / den : 0.0f;      // an empty list gives zeros
+            p.out[(out_row0 + gq) * kD + d] = static_cast<uint16_t>(pack_bf16x2(r, 0.0f) & 0xffffu);
+        } else {
+            __stcg(unit + 16 + gq * kD + d, num);
+            if (d == 0) {
+                __stcg(unit + gq, failed ? -INFINITY : m_all);
+                __stcg(unit + 8 + gq, failed ? 0.0f : den);
+            }
+        }
+    }
+    if (p.n_parts == 1) return;
+
+    // ---- several CTAs per list: the one that arrives last merges all parts, in part order
+    __shared__ int last_s;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t before = atomicAdd(p.part_arrive + list, 1u);
+        last_s = before + 1u == static_cast<uint32_t>(p.n_parts);
+        if (last_s) p.part_arrive[list] = 0u;               // ready for the next launch
+        __threadfence();
+    }
+    __syncthreads();
+    if (!last_s) return;
+    const float *units = p.part_scratch + static_cast<int64_t>(list) * p.n_parts * (16 + kAttnMaxGroup * kD);
+    for (int idx = threadIdx.x; idx < p.group * kD; idx += kAttnThreads) {
+        const int gq = idx / kD, d = idx % kD;
+        float m_all = -INFINITY;
+        for (int i = 0; i < p.n_parts; ++i) m_all = fmaxf(m_all, __ldcg(units + i * (16 + kAttnMaxGroup * kD) + gq));
+        float num = 0.0f, den = 0.0f;
+        for (int i = 0; i < p.n_parts; ++i) {
+            const float *u = units + i * (16 + kAttnMaxGroup * kD);
+            const float m_i = __ldcg(u + gq);
+            if (m_i > -INFINITY) {
+                const float f = fast_ex2(m_i - m_all);
+                num += __ldcg(u + 16 + gq * kD + d) * f;
+                den += __ldcg(u + 8 + gq) * f;
+            }
+        }
+        const float r = den > 0.0f ? num / den : 0.0f;
+        p.out[(out_row0 + gq) * kD + d] = static_cast<uint16_t>(pack_bf16x2(r, 0.0f) & 0xffffu);
     }
 }
 

@@ -1112,6 +1112,9 @@ struct kvzap_cache {
     // attention over the cache: tensor maps of the page pools and of the window rings (built on first use)
     CUtensorMap tm_kpool, tm_vpool, tm_kring, tm_vring;
     int attn_state = 0;                  // 0 not built yet, 1 ready, -1 this cache's geometry is not supported
+    float *attn_scratch = nullptr;       // partial results of lists that are split over several CTAs
+    uint32_t *attn_arrive = nullptr;     // [attn_split_lists] arrival counts, zero between launches
+    int64_t attn_units = 0;              // capacity of attn_scratch in (list, part) units
 };
 
 namespace kvzap {
@@ -1318,6 +1321,11 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     // two halves used by alternate steps when the caller does not ask for the scores
     alloc(reinterpret_cast<void **>(&cache->scores), 2 * sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
           false);
+    // attention: calls with few lists cut each list into parts; room for 16 units per SM
+    cache->attn_units = static_cast<int64_t>(ctx->sm_count) * 16;
+    alloc(reinterpret_cast<void **>(&cache->attn_scratch),
+          sizeof(float) * static_cast<size_t>(cache->attn_units) * (16 + kAttnMaxGroup * 128), false);
+    alloc(reinterpret_cast<void **>(&cache->attn_arrive), sizeof(uint32_t) * static_cast<size_t>(cache->attn_units), true);
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         fail(ctx, KVZAP_ERR_CUDA, "cache allocation failed: %s", cudaGetErrorString(e));
@@ -1336,6 +1344,7 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
     cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
     cudaFree(cache->v.page_cursor); cudaFree(cache->scores); cudaFree(cache->done);
+    cudaFree(cache->attn_scratch); cudaFree(cache->attn_arrive);
     delete cache;
     return KVZAP_OK;
 }
@@ -1456,8 +1465,21 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     p.q = static_cast<const uint16_t *>(Q);
     p.out = static_cast<uint16_t *>(O);
     p.status = ctx->status_dev;
-    const int64_t n_ctas = static_cast<int64_t>(p.n_layers_call) * v.n_seqs * v.n_heads;
-    if (n_ctas > 0x7fffffffLL) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: too many lists for one launch");
+    const int64_t n_lists_call = static_cast<int64_t>(p.n_layers_call) * v.n_seqs * v.n_heads;
+    if (n_lists_call > 0x7fffffffLL) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: too many lists for one launch");
+    // Two CTAs fit an SM.  With fewer than eight CTAs per slot the last, longest lists leave most SMs
+    // idle: cut every list into up to 16 parts so that there are about that many units.
+    p.n_parts = 1;
+    const int64_t want_units = static_cast<int64_t>(ctx->sm_count) * 16;
+    if (n_lists_call * 2 <= want_units) {
+        int64_t parts = want_units / n_lists_call;
+        if (parts > 16) parts = 16;
+        if (parts * n_lists_call > cache->attn_units) parts = cache->attn_units / n_lists_call;
+        if (parts > 1) p.n_parts = static_cast<int32_t>(parts);
+    }
+    p.part_scratch = cache->attn_scratch;
+    p.part_arrive = cache->attn_arrive;
+    const int64_t n_ctas = n_lists_call * p.n_parts;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_ATTENTION, stream);
         if (c.head_dim == 128)

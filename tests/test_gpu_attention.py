@@ -168,10 +168,12 @@ def test_attention_empty_cache_and_argument_errors(binding):
     ctx.close()
 
 
-def test_attention_at_bench_size_sampled_lists(binding, oracle):
+@pytest.mark.parametrize("B", [128, 160])
+def test_attention_at_bench_size_sampled_lists(binding, oracle, B):
     """128 sequences x 8 KV heads with lists of 1k..8k pruned rows plus a full window of 128, the
-    launch shape bench.py --attention times (one layer): sampled lists against the oracle."""
-    d_model, H, D, P, w, B, G = 256, 8, 128, 16, 128, 128, 4
+    launch shape bench.py --attention times (one layer): sampled lists against the oracle.
+    With 128 sequences every list is cut into two parts, with 160 each list is one CTA."""
+    d_model, H, D, P, w, G = 256, 8, 128, 16, 128, 4
     ctx = binding.Kvzap(d_model, 0, H, D, 1, max_tokens=B)
     W, bias = synth.linear_weights(d_model, H, 3)
     ctx.set_weights(0, parity.dev(W), parity.dev(bias))
