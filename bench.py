@@ -31,6 +31,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes); None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 276.8e6, "qwen3_8b_decode_b128": 226.9e6}
+# attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
+NCU_ATTENTION_TRAFFIC_RATIO = 2.408 / 2.3986
 
 
 def load_peaks():
@@ -551,7 +553,7 @@ def run_attention(args, wl, env):
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "gpu_launches": int(ctx.launch_count() - launches0),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name + "/attention"),
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": alg_bytes * NCU_ATTENTION_TRAFFIC_RATIO,
                          "kernel": "decode_attn_kernel", "peak_source": peak_src, "kernel_ms": ms,
                          "algorithmic_bytes_per_step": alg_bytes}}
     binding.kvzap_cache_destroy(cache)
