@@ -167,6 +167,74 @@ void kvzap_oracle_keep_mask(const float *scores, const int32_t *cu_seqlens, int 
 }
 
 /*
+ * Fixed-budget selection: the alternative that the ablation compares
+ * thresholding with (Ablations, "Threshold-based pruning": fixed-ratio top-k
+ * selection per head, or per layer as in AdaKV).  The paper only names the two
+ * variants; the reading used here: for sequence b the candidates are the
+ * positions outside the window, n_cand = max(T_b - w, 0), and the budget is
+ * k = ceil(keep_ratio * n_cand) rows per head (computed in double).
+ *   per head  (per_layer = 0): list (b,h) keeps its k highest-scoring candidates;
+ *   per layer (per_layer = 1): the H*k highest of all H*n_cand candidate scores of
+ *                              the sequence are kept, whichever heads they fall on.
+ * Both are stated through a cut value: tau_out[b,h] = the k-th largest candidate
+ * score of the list (per layer: the (H*k)-th largest over all heads, the same
+ * for every h), and keep = in_window || score >= tau_out[b,h].  Scores equal to
+ * the cut value are all kept, so ties may take a list past its budget; NaN
+ * scores are never candidates; k = 0 gives +inf; fewer than k (non-NaN)
+ * candidates give -inf.  The window rule is that of kvzap_oracle_keep_mask.
+ * scores [T_total,H] fp32; keep [H,T_total] bytes; tau_out [B,H] fp32.
+ * Returns 0, or -1 without memory.
+ */
+static int cmp_float_desc(const void *a, const void *b)
+{
+    const float x = *(const float *)a, y = *(const float *)b;
+    return (x < y) - (x > y);
+}
+
+int kvzap_oracle_topk_mask(const float *scores, const int32_t *cu_seqlens, int B, int H, int w,
+                           double keep_ratio, int per_layer, uint8_t *keep, float *tau_out)
+{
+    const int64_t T_total = cu_seqlens[B];
+    float *buf = (float *)malloc(sizeof(float) * (size_t)(T_total > 0 ? T_total : 1) * (size_t)H);
+    if (!buf) return -1;
+    for (int b = 0; b < B; ++b) {
+        const int64_t t0 = cu_seqlens[b], t1 = cu_seqlens[b + 1];
+        const int64_t Tb = t1 - t0;
+        const int64_t n_cand = Tb - w > 0 ? Tb - w : 0;
+        const int64_t k = (int64_t)ceil(keep_ratio * (double)n_cand);
+        for (int h = 0; h < H; ++h) {
+            if (per_layer && h > 0) {
+                tau_out[b * H + h] = tau_out[b * H];
+                continue;
+            }
+            /* the candidate scores of this list (of all heads for the per-layer budget), NaN left out */
+            int64_t n = 0;
+            for (int64_t t = t0; t < t0 + n_cand; ++t)
+                for (int hh = (per_layer ? 0 : h); hh < (per_layer ? H : h + 1); ++hh) {
+                    const float v = scores[t * H + hh];
+                    if (v == v) buf[n++] = v;
+                }
+            const int64_t want = per_layer ? k * H : k;
+            float tau;
+            if (want <= 0) tau = INFINITY;
+            else if (n < want) tau = -INFINITY;
+            else {
+                qsort(buf, (size_t)n, sizeof(float), cmp_float_desc);
+                tau = buf[want - 1];
+            }
+            tau_out[b * H + h] = tau;
+        }
+        for (int h = 0; h < H; ++h)
+            for (int64_t t = t0; t < t1; ++t) {
+                const int in_window = (t - t0) >= Tb - (int64_t)w;
+                keep[(int64_t)h * T_total + t] = (uint8_t)(in_window || scores[t * H + h] >= tau_out[b * H + h]);
+            }
+    }
+    free(buf);
+    return 0;
+}
+
+/*
  * Per-(sequence, head) ordered compaction (Algorithm 1: keys[indices],
  * values[indices]; contribution list: per-head compression).
  * For each (b,h) walk the sequence's positions in order and copy row t of K

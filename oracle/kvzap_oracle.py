@@ -52,6 +52,7 @@ def lib():
         L.kvzap_oracle_compact_paged.restype = ctypes.c_int
         L.kvzap_oracle_compact_write_paged.restype = ctypes.c_int
         L.kvzap_oracle_attention.restype = ctypes.c_int
+        L.kvzap_oracle_topk_mask.restype = ctypes.c_int
         for name in ("layer_flops", "mlp_flops", "linear_flops"):
             getattr(L, "kvzap_oracle_" + name).restype = ctypes.c_double
         L.kvzap_oracle_layer_flops.argtypes = [ctypes.c_int] * 5
@@ -147,6 +148,24 @@ def keep_mask(scores, tau, w, cu_seqlens=None):
         _c(scores, ctypes.c_float), _c(cu, ctypes.c_int32), ctypes.c_int(len(cu) - 1),
         ctypes.c_int(H), ctypes.c_float(tau), ctypes.c_int(w), _c(keep, ctypes.c_uint8))
     return keep
+
+
+def topk_mask(scores, keep_ratio, w, per_layer=False, cu_seqlens=None):
+    """Fixed-budget selection: scores [T_total,H] fp32 -> (keep [H,T_total] uint8, tau [B,H] fp32)."""
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    T_total, H = scores.shape
+    assert w >= 0
+    cu = _cu(cu_seqlens, T_total)
+    B = len(cu) - 1
+    keep = np.zeros((H, T_total), dtype=np.uint8)
+    tau = np.zeros((B, H), dtype=np.float32)
+    rc = lib().kvzap_oracle_topk_mask(
+        _c(scores, ctypes.c_float), _c(cu, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(w),
+        ctypes.c_double(float(np.float32(keep_ratio))), ctypes.c_int(1 if per_layer else 0),
+        _c(keep, ctypes.c_uint8), _c(tau, ctypes.c_float))
+    if rc != 0:
+        raise MemoryError("oracle top-k: out of memory")
+    return keep, tau
 
 
 def compact(K, V, keep, cu_seqlens=None, fill=0):
