@@ -208,6 +208,29 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
                                        float *scores_out, void *stream);
 
 /*
+ * Fixed-budget selection instead of a threshold (Ablations, "Threshold-based
+ * pruning": the top-k alternatives the paper compares thresholding with, per
+ * head or per layer as in AdaKV).  For sequence b the candidates are the
+ * positions outside the window, n_cand = max(T_b - w, 0), and the budget is
+ * k = ceil(keep_ratio * n_cand) rows per head:
+ *   per_layer = 0: list (b,h) keeps its k highest-scoring candidates;
+ *   per_layer = 1: the H*k highest of all candidate scores of sequence b are kept,
+ *                  whichever heads they fall on (heads share one budget).
+ * The call finds the cut value tau[b,h] (the k-th largest candidate score; per
+ * layer the (H*k)-th largest over all heads, the same for every h) and then
+ * prunes exactly as kvzap_prune_prefill does with that threshold for list (b,h):
+ * scores equal to the cut value are all kept (ties may exceed the budget), NaN
+ * scores are never candidates, k = 0 gives tau = +inf, fewer than k candidates
+ * that are numbers give tau = -inf.  The window is always kept.
+ *   keep_ratio in [0, 1];  tau_out [n_seqs, H] fp32 (device) or NULL: the cut values used
+ * Other arguments, outputs and errors as kvzap_prune_prefill.
+ */
+kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                      float keep_ratio, int32_t w, int32_t per_layer,
+                                      void *K_out, void *V_out, int32_t *lengths, float *tau_out, void *stream);
+
+/*
  * Pruning on the write side (Discussion, "Implementation Challenges": the
  * surrogate needs only hidden states, so pruning can run before attention).
  * Same operation and outputs as kvzap_prefill_fused / kvzap_prefill_fused_paged,

@@ -56,6 +56,7 @@ SIGNATURES = {
                                          _vp, _i32, _vp, _vp, _vp]),
     "kvzap_prefill_fused_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
                                          _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prune_prefill_topk": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_write_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
                                          _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
@@ -211,6 +212,16 @@ def kvzap_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, t
         _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens,
         first_page, _ptr(page_table), page_table.shape[1], _ptr(lengths), _ptr(n_pages_used),
         _ptr(scores_out) if nz else None, _stream(stream)))
+
+
+def kvzap_prune_prefill_topk(handle, K, V, scores, cu_seqlens, n_seqs, keep_ratio, w, per_layer, K_out, V_out, lengths,
+                             tau_out=None, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prune_prefill_topk(
+        handle, _ptr(K) if nz else None, _ptr(V) if nz else None, _ptr(scores) if nz else None, _ptr(cu_seqlens),
+        n_seqs, n_tokens, keep_ratio, w, 1 if per_layer else 0, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
+        _ptr(lengths), _ptr(tau_out), _stream(stream)))
 
 
 def kvzap_prefill_write(handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,

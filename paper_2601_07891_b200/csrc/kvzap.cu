@@ -16,6 +16,7 @@
 #include "prune_kernels.cuh"
 #include "score_kernel.cuh"
 #include "score_split_kernel.cuh"
+#include "select_kernels.cuh"
 
 namespace kvzap {
 
@@ -60,6 +61,8 @@ struct kvzap_ctx {
     uint32_t *maskbits = nullptr;    // [kMaskRing][H][max_words]: consecutive calls use different slices
     uint64_t mask_turn = 0;
     int32_t *tile_counters = nullptr;    // [kMaskRing] work-tile counters of the scoring launches, used in rotation
+    uint32_t *select_hist = nullptr;     // fixed-budget selection: [4 passes][max_seqs][H][256] histograms
+    float *select_tau = nullptr;         //                         [max_seqs][H] cut values when the caller wants none
     float *split_part = nullptr;         // few-token kernel: [sm_count tiles][4 slices][128][8] partial scores
     uint32_t *split_arrive = nullptr;    //                   [sm_count] arrival counts per tile
     uint64_t score_turn = 0;
@@ -225,6 +228,8 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->maskbits);
     cudaFree(ctx->tile_counters);
     cudaFree(ctx->split_part);
+    cudaFree(ctx->select_hist);
+    cudaFree(ctx->select_tau);
     cudaFree(ctx->split_arrive);
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
@@ -721,6 +726,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->tile_counters, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing));
+    CREATE_CUDA(cudaMalloc(&ctx->select_hist, sizeof(uint32_t) * 4 * static_cast<size_t>(c.max_seqs) * c.n_kv_heads * 256));
+    CREATE_CUDA(cudaMalloc(&ctx->select_tau, sizeof(float) * static_cast<size_t>(c.max_seqs) * c.n_kv_heads));
     if (ctx->split_n > 0) {
         CREATE_CUDA(cudaMalloc(&ctx->split_part, sizeof(float) * static_cast<size_t>(ctx->sm_count) * 4 * kTileM * kMaxHeads));
         CREATE_CUDA(cudaMalloc(&ctx->split_arrive, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
@@ -829,10 +836,53 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
         mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
                                                                          cu_seqlens, n_seqs, tau, w, 1, mask,
-                                                                         n_blocks * 4);
+                                                                         n_blocks * 4, nullptr);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
+}
+
+kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float keep_ratio,
+                                      int32_t w, int32_t per_layer, void *K_out, void *V_out, int32_t *lengths,
+                                      float *tau_out, void *stream_)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    if (!(keep_ratio >= 0.0f && keep_ratio <= 1.0f)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "keep_ratio outside [0, 1]");
+    const kvzap_config &c = ctx->cfg;
+    DeviceGuard guard(c.device);
+    float *tau_list = tau_out ? tau_out : ctx->select_tau;
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * c.n_kv_heads, stream));
+        return KVZAP_OK;
+    }
+    st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
+    if (st != KVZAP_OK) return st;
+    if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
+    const int n_sel = per_layer ? 1 : c.n_kv_heads;
+    KVZAP_CUDA(ctx, cudaMemsetAsync(ctx->select_hist, 0, sizeof(uint32_t) * 4 * static_cast<size_t>(n_seqs) * n_sel * 256, stream));
+    const dim3 grid(static_cast<unsigned>((n_tokens + kSelectThreads - 1) / kSelectThreads), static_cast<unsigned>(n_seqs));
+    for (int pass = 0; pass < 4; ++pass)
+        select_hist_kernel<<<grid, kSelectThreads, 0, stream>>>(scores, n_tokens, c.n_kv_heads, cu_seqlens, n_seqs, w,
+                                                                keep_ratio, per_layer ? 1 : 0, pass, ctx->select_hist);
+    select_finish_kernel<<<static_cast<unsigned>(n_seqs), kSelectThreads, 0, stream>>>(
+        n_tokens, c.n_kv_heads, cu_seqlens, n_seqs, w, keep_ratio, per_layer ? 1 : 0, ctx->select_hist, tau_list,
+        ctx->status_dev);
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    uint32_t *mask = next_mask_slice(ctx);
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
+        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, c.n_kv_heads, cu_seqlens, n_seqs,
+                                                                         0.0f, w, 1, mask, n_blocks * 4, tau_list);
+    }
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 6;
     return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
 }
 
@@ -1084,7 +1134,7 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
     // that this call reads is first written by it; only the status word must start at zero.
     KVZAP_CUDA(nullptr, cudaMemsetAsync(status, 0, sizeof(int32_t), stream));
     mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, n_kv_heads, cu_seqlens, n_seqs,
-                                                                     tau, w, 1, maskbits, n_words);
+                                                                     tau, w, 1, maskbits, n_words, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
                                         blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status);
@@ -1213,7 +1263,7 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
         mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
                                                                          cu_seqlens, n_seqs, tau, w, 1, mask,
-                                                                         n_blocks * 4);
+                                                                         n_blocks * 4, nullptr);
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;

@@ -25,18 +25,19 @@ constexpr int kBlockTokens = 128;     // tokens per mask block = 4 words (same a
 // ---------------------------------------------------------------------------
 // keep[h,t] = in_window(t) || scores[t,h] >= tau, as 32-token ballot words.
 // One warp per 32 tokens; 4 warps per CTA = one 128-token block.
+// tau_list != nullptr: a threshold per list, tau_list[b * n_heads + h] (fixed-budget selection), instead of tau.
 __global__ void __launch_bounds__(128)
 mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
             const int32_t *__restrict__ cu_seqlens, int n_seqs, float tau, int window, int window_keep,
-            uint32_t *__restrict__ maskbits, int64_t n_words)
+            uint32_t *__restrict__ maskbits, int64_t n_words, const float *__restrict__ tau_list)
 {
     const int lane = threadIdx.x & 31;
     const int64_t word = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
     const int64_t t = word * 32 + lane;
     const bool valid = t < n_tokens;
-    float s[kMaxHeads];
+    float s[kMaxHeads], tau_h[kMaxHeads];
 #pragma unroll
-    for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+    for (int h = 0; h < kMaxHeads; ++h) { s[h] = 0.0f; tau_h[h] = tau; }
     bool in_window = false;
     if (valid) {
         const float *src = scores + t * n_heads;
@@ -51,14 +52,23 @@ mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
                 if (h < n_heads) s[h] = __ldg(src + h);
         }
         int64_t seq_end = n_tokens;
-        if (cu_seqlens != nullptr && n_seqs > 1)
-            seq_end = __ldg(cu_seqlens + seq_of_token(cu_seqlens, n_seqs, t) + 1);
+        int b = 0;
+        if (cu_seqlens != nullptr && n_seqs > 1) {
+            b = seq_of_token(cu_seqlens, n_seqs, t);
+            seq_end = __ldg(cu_seqlens + b + 1);
+        }
         in_window = t >= seq_end - static_cast<int64_t>(window);
+        if (tau_list != nullptr) {
+            // thresholds written by the kernel ahead in the stream: plain loads
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h)
+                if (h < n_heads) tau_h[h] = tau_list[b * n_heads + h];
+        }
     }
     uint32_t my_word = 0;
 #pragma unroll
     for (int h = 0; h < kMaxHeads; ++h) {
-        const bool keep = valid && (in_window ? window_keep != 0 : s[h] >= tau);
+        const bool keep = valid && (in_window ? window_keep != 0 : s[h] >= tau_h[h]);
         const uint32_t w = __ballot_sync(0xffffffffu, keep);
         if (lane == h) my_word = w;
     }
