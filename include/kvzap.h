@@ -341,7 +341,12 @@ kvzap_status kvzap_cache_export(kvzap_cache *cache, int32_t seq, int32_t layer, 
  * prefill(T) followed by k decode steps equals prefill(T + k).
  *   hidden [n_tokens, d_model] bf16, K, V [H, n_tokens, D] bf16 (one sequence)
  *   scores_out [n_tokens, H] fp32 (device) -- required, it also serves as scratch
- * The lists must be empty (fresh cache) when this is called.
+ * Chunked prefill: the lists need not be empty.  Called again with the next
+ * chunk of the same prompt (or after decode steps), the call first decides the
+ * tokens of the present window that the chunk pushes out, by their buffered
+ * scores, then appends the chunk as described above; prefill in chunks of any
+ * lengths equals one prefill of the whole prompt (the score buffer carries the
+ * window across chunk boundaries).
  */
 kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, int32_t seq,
                                     const void *hidden, const void *K, const void *V, int64_t n_tokens,

@@ -158,27 +158,86 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
     }
 }
 
-// After a prompt's prefix has been compacted: copies the last min(T, w) tokens of the prompt (rows of
-// K, V [H][T][D], scores [T][H]) into the window rings of lists li0 .. li0+H-1 and sets n_tokens = T.
+// A further chunk of m prompt tokens is about to be appended to lists li0 .. li0+H-1 (chunked
+// prefill): the tokens of the present window that it pushes out are decided here by their buffered
+// scores, oldest first, and the kept ones appended to the list's paged prefix (pages from the
+// cache's cursor), exactly as m decode steps would have done.  One warp per list; n_tokens is left
+// as it is (tokens_add_kernel advances it once the chunk's own rows are in place).
+__global__ void __launch_bounds__(32)
+chunk_evict_kernel(const CacheView c, int64_t li0, int64_t m, float tau, int32_t *__restrict__ status)
+{
+    const int64_t li = li0 + blockIdx.x;
+    const int lane = threadIdx.x;
+    const int64_t n_old = c.n_tokens[li];
+    const int64_t in_ring = n_old < c.window ? n_old : c.window;
+    const int64_t first = n_old - in_ring;                         // oldest position still in the window
+    int64_t exit_end = n_old + m - c.window;                       // positions below it leave the window
+    if (exit_end > n_old) exit_end = n_old;
+    const int64_t n_exit = exit_end > first ? exit_end - first : 0;
+    int64_t len = c.prefix_len[li];
+    int32_t *table = c.page_table + li * c.max_pages;
+    for (int64_t base = 0; base < n_exit; base += 32) {
+        const int64_t pos = first + base + lane;
+        const bool valid = base + lane < n_exit;
+        const int64_t slot = li * c.window + pos % c.window;
+        const bool keep = valid && c.score_ring[slot] >= tau;
+        const uint32_t kept = __ballot_sync(0xffffffffu, keep);
+        const int cnt = __popc(kept);
+        const int64_t have = (len + c.page_tokens - 1) / c.page_tokens;
+        const int64_t want = (len + cnt + c.page_tokens - 1) / c.page_tokens;
+        int ok = 1;
+        if (lane == 0 && want > have) {
+            if (want > c.max_pages) ok = 0;
+            else {
+                const int32_t got = atomicAdd(c.page_cursor, static_cast<int32_t>(want - have));
+                if (static_cast<int64_t>(got) + (want - have) > c.n_pages_pool) ok = 0;
+                else for (int64_t i = have; i < want; ++i) table[i] = got + static_cast<int32_t>(i - have);
+            }
+            if (!ok) atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;                                            // what was appended so far stays valid
+        __syncwarp();
+        if (keep) {
+            const int64_t nn = len + __popc(kept & ((1u << lane) - 1u));
+            const int64_t page = *(volatile int32_t *)(table + nn / c.page_tokens);
+            const int64_t dst = (page * c.page_tokens + nn % c.page_tokens) * c.row_units;
+            for (int u = 0; u < c.row_units; ++u) {
+                c.k_pool[dst + u] = c.k_ring[slot * c.row_units + u];
+                c.v_pool[dst + u] = c.v_ring[slot * c.row_units + u];
+            }
+        }
+        len += cnt;
+    }
+    if (lane == 0) c.prefix_len[li] = static_cast<int32_t>(len);
+}
+
+// The last min(m, w) tokens of a chunk of m (rows of K, V [H][m][D], scores [m][H]) go into the window
+// rings of lists li0 .. li0+H-1 at the slots of their absolute positions n_tokens + chunk index.
 __global__ void __launch_bounds__(256)
-ring_fill_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
-                 const uint4 *__restrict__ V, int64_t T)
+ring_append_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
+                   const uint4 *__restrict__ V, int64_t m)
 {
     const int h = blockIdx.y;
     const int64_t li = li0 + h;
-    const int64_t n_win = T < c.window ? T : c.window;
+    const int64_t n_old = c.n_tokens[li];
+    const int64_t n_win = m < c.window ? m : c.window;
     for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_win * c.row_units;
          i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
         const int64_t j = i / c.row_units;
         const int u = static_cast<int>(i % c.row_units);
-        const int64_t pos = T - n_win + j;
-        const int64_t dst = (li * c.window + pos % c.window) * c.row_units + u;
-        const int64_t src = (static_cast<int64_t>(h) * T + pos) * c.row_units + u;
-        c.k_ring[dst] = K[src];
-        c.v_ring[dst] = V[src];
-        if (u == 0) c.score_ring[li * c.window + pos % c.window] = scores[pos * c.n_heads + h];
+        const int64_t ci = m - n_win + j;                      // index inside the chunk
+        const int64_t slot = li * c.window + (n_old + ci) % c.window;
+        const int64_t src = (static_cast<int64_t>(h) * m + ci) * c.row_units + u;
+        c.k_ring[slot * c.row_units + u] = K[src];
+        c.v_ring[slot * c.row_units + u] = V[src];
+        if (u == 0) c.score_ring[slot] = scores[ci * c.n_heads + h];
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) c.n_tokens[li] = static_cast<int32_t>(T);
+}
+
+__global__ void tokens_add_kernel(const CacheView c, int64_t li0, int64_t m)
+{
+    if (threadIdx.x < c.n_heads) c.n_tokens[li0 + threadIdx.x] += static_cast<int32_t>(m);
 }
 
 // lengths[li] = prefix_len + min(n_tokens, w)

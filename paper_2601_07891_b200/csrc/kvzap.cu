@@ -72,6 +72,8 @@ struct kvzap_ctx {
     int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
     int32_t *seqbase = nullptr;      // [H][max_seqs + 1]
     int32_t *list_page0 = nullptr;   // [max_seqs * H] first page of each list (paged output)
+    int32_t *list_base = nullptr;    // [max_seqs * H] appending to lists: rows each list held before
+    int32_t *list_tail = nullptr;    // [max_seqs * H]                     and the page of its last row
     int32_t *status_dev = nullptr;
     int32_t *status_host = nullptr;  // pinned
     int64_t launches = 0;
@@ -234,6 +236,8 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->blockprefix);
     cudaFree(ctx->seqbase);
     cudaFree(ctx->list_page0);
+    cudaFree(ctx->list_base);
+    cudaFree(ctx->list_tail);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
@@ -515,7 +519,8 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
                                            cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths, 0,
                                            static_cast<const int32_t *>(nullptr),
                                            tok_major ? int64_t{1} : n_tokens,
-                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1}));
+                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
+                                           static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr)));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -724,6 +729,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->list_base, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
+    CREATE_CUDA(cudaMalloc(&ctx->list_tail, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->tile_counters, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMalloc(&ctx->select_hist, sizeof(uint32_t) * 4 * static_cast<size_t>(c.max_seqs) * c.n_kv_heads * 256));
@@ -1137,7 +1144,7 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
                                                                      tau, w, 1, maskbits, n_words, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
-                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status);
+                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status, 0, nullptr, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(n_kv_heads));
     compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
@@ -1175,7 +1182,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                             int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
                                             int32_t *page_table, int32_t max_pages, int32_t *lengths,
                                             int32_t *n_pages_used, cudaStream_t stream,
-                                            int32_t *page_cursor = nullptr, bool tok_major = false)
+                                            int32_t *page_cursor = nullptr, bool tok_major = false, bool append = false)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1190,7 +1197,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            cu_seqlens, static_cast<int>(n_seqs), n_tokens, ctx->blockprefix, ctx->seqbase,
                                            lengths, static_cast<int>(page_tokens), first_page, n_pages_pool,
                                            static_cast<int>(max_pages), ctx->list_page0, page_table, n_pages_used,
-                                           page_cursor, ctx->status_dev));
+                                           page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, ctx->list_tail));
     }
     // the same resident-at-once grid as the dense-ragged output (see launch_compaction)
     const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (c.hidden > 0 ? 2 : 6);
@@ -1210,7 +1217,9 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            static_cast<int>(c.head_dim / 8), lengths, static_cast<int>(page_tokens),
                                            static_cast<const int32_t *>(ctx->list_page0),
                                            tok_major ? int64_t{1} : n_tokens,
-                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1}));
+                                           tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
+                                           static_cast<const int32_t *>(append ? ctx->list_base : nullptr),
+                                           static_cast<const int32_t *>(append ? ctx->list_tail : nullptr)));
     }
     ctx->launches += 2;
     return KVZAP_OK;
@@ -1607,28 +1616,33 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
         return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache: hidden, K, V, scores_out must be non-NULL, aligned");
     DeviceGuard guard(c.device);
     const int64_t li0 = (static_cast<int64_t>(seq) * v.n_layers + layer) * v.n_heads;
-    // mask = threshold only, the window's tokens left out: they go to the ring below
+    // The lists may already hold earlier chunks of the prompt.  First the tokens of the present window
+    // that this chunk pushes out are decided by their buffered scores (as decode steps would have done).
+    if (v.window > 0) {
+        chunk_evict_kernel<<<static_cast<unsigned>(v.n_heads), 32, 0, stream>>>(v, li0, n_tokens, tau, ctx->status_dev);
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    }
+    // Then the chunk itself.  mask = threshold only, the chunk's last `window` tokens left out: they go
+    // to the ring below; the kept ones are appended behind what the lists hold.
     uint32_t *mask = next_mask_slice(ctx);
     st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, nullptr, 1, tau, v.window, stream, 0);
     if (st != KVZAP_OK) return st;
     st = launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
                                  v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
-                                 v.page_cursor);
+                                 v.page_cursor, false, true);
     if (st != KVZAP_OK) return st;
     if (v.window > 0) {
         const int64_t n_win = n_tokens < v.window ? n_tokens : v.window;
         const unsigned gx = static_cast<unsigned>((n_win * v.row_units + 255) / 256);
-        ring_fill_kernel<<<dim3(gx, static_cast<unsigned>(v.n_heads)), 256, 0, stream>>>(
+        ring_append_kernel<<<dim3(gx, static_cast<unsigned>(v.n_heads)), 256, 0, stream>>>(
             v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens);
         KVZAP_CUDA(ctx, cudaGetLastError());
         ctx->launches += 1;
-    } else {
-        // no window: only the token count is kept
-        std::vector<int32_t> nt(v.n_heads, static_cast<int32_t>(n_tokens));
-        KVZAP_CUDA(ctx, cudaMemcpyAsync(v.n_tokens + li0, nt.data(), sizeof(int32_t) * v.n_heads, cudaMemcpyHostToDevice,
-                                        stream));
-        KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
     }
+    tokens_add_kernel<<<1, 32, 0, stream>>>(v, li0, n_tokens);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
     return KVZAP_OK;
 }
 

@@ -102,13 +102,18 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
 // [n_seqs*H][max_pages] its page numbers; *n_pages_used the total.  A pool or
 // table that is too small sets the status word and marks every list with
 // list_page0 = -1 so that the compaction writes nothing.
+// append != 0 (paged only): the lists already hold lengths[] rows in the pages their tables name; the
+// kept rows are added behind them.  lengths becomes old + kept (unchanged on failure), only the pages
+// beyond the old ones are assigned (list_page0 = the first of them, table entries appended), and
+// list_base / list_tail receive the old length and the page that holds the old tail (-1 if none).
 __global__ void __launch_bounds__(1024)
 scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
             const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens,
             int32_t *__restrict__ blockprefix, int32_t *__restrict__ seqbase, int32_t *__restrict__ lengths,
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
-            int32_t *__restrict__ page_cursor, int32_t *__restrict__ status)
+            int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
+            int32_t *__restrict__ list_base, int32_t *__restrict__ list_tail)
 {
     // may be placed before the kernel that writes the mask has finished; waits for it here
     griddep_launch_dependents();
@@ -175,7 +180,9 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     __syncthreads();
     for (int idx = tid; idx < n_heads * n_seqs; idx += 1024) {
         const int b = idx / n_heads, h = idx % n_heads;
-        lengths[idx] = seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
+        const int32_t old = append ? lengths[idx] : 0;
+        if (append) list_base[idx] = old;
+        lengths[idx] = old + seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
     }
     if (page_tokens <= 0) return;
 
@@ -190,6 +197,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         if (idx < n_lists) {
             need = (lengths[idx] + page_tokens - 1) / page_tokens;
             if (need > max_pages) fail_s = 1;
+            if (append) need -= (list_base[idx] + page_tokens - 1) / page_tokens;     // pages the list already owns
         }
         int32_t total;
         const int32_t incl = block_scan(need, total);
@@ -202,7 +210,10 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     const int32_t used = carry_s;
     const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + used > n_pages_pool;
     if (fail) {
-        for (int idx = tid; idx < n_lists; idx += 1024) list_page0[idx] = -1;
+        for (int idx = tid; idx < n_lists; idx += 1024) {
+            list_page0[idx] = -1;
+            if (append) lengths[idx] = list_base[idx];
+        }
         if (tid == 0) {
             atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
             if (n_pages_used != nullptr) *n_pages_used = 0;
@@ -215,8 +226,10 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     }
     for (int idx = tid; idx < n_lists; idx += 1024) {
         const int32_t p0 = list_page0[idx];
-        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens;
-        for (int32_t i = 0; i < need; ++i) page_table[static_cast<int64_t>(idx) * max_pages + i] = p0 + i;
+        const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
+        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
+        if (append) list_tail[idx] = have > 0 ? page_table[static_cast<int64_t>(idx) * max_pages + have - 1] : -1;
+        for (int32_t i = 0; i < need; ++i) page_table[static_cast<int64_t>(idx) * max_pages + have + i] = p0 + i;
     }
 }
 
@@ -332,8 +345,12 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                      uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
                      int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths, int page_tokens,
-                     const int32_t *__restrict__ list_page0, int64_t in_stride_h, int64_t in_stride_t)
+                     const int32_t *__restrict__ list_page0, int64_t in_stride_h, int64_t in_stride_t,
+                     const int32_t *__restrict__ list_base, const int32_t *__restrict__ list_tail)
 {
+    // list_base != nullptr (paged): list (b,h) already holds list_base[] rows, the last of them in page
+    // list_tail[]; kept rows go behind them, first into that page's free slots, then into the pages
+    // from list_page0 on.
     // Row (h, t) of the inputs starts at row index h * in_stride_h + t * in_stride_t: (n_tokens, 1) for
     // the head-major cache layout [H][T][D], (1, H) for the K/V projection's own output [T][H][D].
     // page_tokens > 0: paged output.  K_out / V_out are the page pools, list (b,h) starts at page
@@ -412,7 +429,15 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                     const int64_t n = running + r - base;                  // rank inside list (b,h)
                     if (paged) {
                         const int32_t p0 = list_page0[b * n_heads + h];
-                        dst_row[r] = p0 < 0 ? -1 : (static_cast<int64_t>(p0) + n / page_tokens) * page_tokens + n % page_tokens;
+                        if (list_base == nullptr) {
+                            dst_row[r] = p0 < 0 ? -1 : (static_cast<int64_t>(p0) + n / page_tokens) * page_tokens + n % page_tokens;
+                        } else {
+                            const int64_t base = list_base[b * n_heads + h];
+                            const int64_t have = (base + page_tokens - 1) / page_tokens;
+                            const int64_t nn = base + n, q = nn / page_tokens;
+                            const int64_t page = q < have ? list_tail[b * n_heads + h] : p0 + (q - have);
+                            dst_row[r] = p0 < 0 ? -1 : page * page_tokens + nn % page_tokens;
+                        }
                     } else {
                         dst_row[r] = static_cast<int64_t>(h) * n_tokens + s + n;
                     }

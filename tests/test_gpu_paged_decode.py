@@ -227,3 +227,57 @@ def test_decode_pool_exhaustion_sets_status(binding):
     assert ctx.poll_status() == 4
     binding.kvzap_cache_destroy(cache)
     ctx.close()
+
+
+@pytest.mark.parametrize("chunks,w,P", [([300, 5, 200, 17, 129], 16, 8), ([100, 100, 100], 128, 16), ([64, 1, 1, 300], 0, 4),
+                                        ([3, 2, 700, 40], 32, 16)])
+def test_chunked_prefill_equals_one_prefill(binding, oracle, chunks, w, P):
+    """Prefill in chunks of any lengths (then a few decode steps) == prefill of the whole sequence:
+    the score buffer carries the window across chunk boundaries."""
+    d_model, hidden, H, D, tau, k = 256, 128, 8, 64, 0.2, 7
+    T0 = sum(chunks)
+    ctx = binding.Kvzap(d_model, hidden, H, D, 1, max_tokens=max(max(chunks), 128))
+    wts = _weights(d_model, hidden, H, seed=T0)
+    ctx.set_weights(0, *[parity.dev(x) for x in wts])
+    X = synth.hidden_states(T0 + k, d_model, seed=T0 + 1)
+    K, V = synth.keys_values(H, T0 + k, D, seed=T0 + 2)
+    n_pool = H * ((T0 + k) // P + 2) + 8
+    K_pool = torch.zeros(n_pool, P, D, dtype=torch.bfloat16, device="cuda")
+    V_pool = torch.zeros_like(K_pool)
+    cache = binding.kvzap_cache_create(ctx.handle, 1, w, P, K_pool, V_pool, (T0 + k) // P + 2)
+    scores_all = torch.empty(T0 + k, H, dtype=torch.float32, device="cuda")
+    t = 0
+    for m in chunks:
+        binding.kvzap_prefill_to_cache(ctx.handle, cache, 0, 0, parity.dev(X[t:t + m]), parity.dev(K[:, t:t + m].contiguous()),
+                                       parity.dev(V[:, t:t + m].contiguous()), tau, scores_all[t:t + m])
+        t += m
+        if t in (chunks[0], T0):             # check at a chunk boundary and at the end of the prompt
+            torch.cuda.synchronize()
+            assert ctx.poll_status() == 0
+            s = scores_all[:t].cpu().numpy()
+            keep = oracle.keep_mask(s, tau, w)
+            Kc, Vc, ln = oracle.compact(synth.bits(K[:, :t]), synth.bits(V[:, :t]), keep)
+            for h in range(H):
+                Kg, Vg, n = _export(binding, ctx, cache, 0, 0, h, T0 + k, D)
+                assert n == ln[0, h]
+                np.testing.assert_array_equal(Kg, Kc[h, :n])
+                np.testing.assert_array_equal(Vg, Vc[h, :n])
+    for t in range(T0, T0 + k):
+        binding.kvzap_decode_step(ctx.handle, cache, 0, 1, parity.dev(X[t:t + 1]).view(1, 1, d_model),
+                                  parity.dev(K[:, t].contiguous()).view(1, 1, H, D),
+                                  parity.dev(V[:, t].contiguous()).view(1, 1, H, D), tau, scores_all[t:t + 1].view(1, 1, H))
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    s = scores_all.cpu().numpy()
+    want = oracle.score(synth.bits(X), parity.weights_to_oracle(wts))
+    assert np.abs(s - want).max() <= parity.SCORE_ATOL
+    keep = oracle.keep_mask(s, tau, w)
+    Kc, Vc, ln = oracle.compact(synth.bits(K), synth.bits(V), keep)
+    tables = []
+    for h in range(H):
+        Kg, Vg, n = _export(binding, ctx, cache, 0, 0, h, T0 + k, D)
+        assert n == ln[0, h]
+        np.testing.assert_array_equal(Kg, Kc[h, :n])
+        np.testing.assert_array_equal(Vg, Vc[h, :n])
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
