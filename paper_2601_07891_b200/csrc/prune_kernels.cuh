@@ -340,7 +340,11 @@ __device__ __forceinline__ int popc_below(uint32_t w0, uint32_t w1, uint32_t w2,
     return n;
 }
 
-__global__ void __launch_bounds__(kDenseThreads)
+// At most 64 registers per thread (eight CTAs per SM by registers): two of these CTAs then fit into the
+// register-file quarters that the MLP scoring kernel's ten warps leave free, so the compaction of layer
+// l runs beside the scoring of layer l + 1 at full width; at 72 registers only one fits and the layer
+// period of the fused path grows by ~10 us.
+__global__ void __launch_bounds__(kDenseThreads, 8)
 compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ K_out,
                      uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
