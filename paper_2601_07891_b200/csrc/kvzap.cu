@@ -1182,7 +1182,8 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                             int64_t n_pages_pool, int32_t page_tokens, int32_t first_page,
                                             int32_t *page_table, int32_t max_pages, int32_t *lengths,
                                             int32_t *n_pages_used, cudaStream_t stream,
-                                            int32_t *page_cursor = nullptr, bool tok_major = false, bool append = false)
+                                            int32_t *page_cursor = nullptr, bool tok_major = false, bool append = false,
+                                            bool beside_scoring = true)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1200,7 +1201,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, ctx->list_tail));
     }
     // the same resident-at-once grid as the dense-ragged output (see launch_compaction)
-    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (c.hidden > 0 ? 2 : 6);
+    const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (!beside_scoring ? 8 : (c.hidden > 0 ? 2 : 6));
     int64_t chunks = max_ctas / c.n_kv_heads;
     if (chunks < 1) chunks = 1;
     if (chunks > n_blocks) chunks = n_blocks;
@@ -1277,7 +1278,8 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
     return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
-                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream);
+                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream, nullptr,
+                                   false, false, false);
 }
 
 static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K,
