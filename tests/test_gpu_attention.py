@@ -223,3 +223,56 @@ def test_attention_at_bench_size_sampled_lists(binding, oracle, B):
         assert np.abs(got[b, h * G:(h + 1) * G] - want).max() <= ATTN_ATOL, li
     binding.kvzap_cache_destroy(cache)
     ctx.close()
+
+
+def test_decode_loop_step_then_attention_enqueued_back_to_back(binding, oracle):
+    """The serving loop: decode step, attention, decode step, attention, ... all enqueued without a
+    host synchronisation in between.  Every attention call must see exactly the cache its own step
+    left (the next step, which may start early, must not disturb it)."""
+    d_model, hidden, H, D, w, P, B, L, G, tau, n_steps = 256, 128, 8, 64, 16, 16, 6, 2, 4, 0.0, 70
+    ctx = binding.Kvzap(d_model, hidden, H, D, L, max_tokens=128, max_seqs=1)
+    all_w = []
+    for l in range(L):
+        wts = _weights(d_model, hidden, H, seed=90 + l)
+        all_w.append(wts)
+        ctx.set_weights(l, *[parity.dev(x) for x in wts])
+    max_pages = n_steps // P + 2
+    n_pool = B * L * H * max_pages
+    K_pool, V_pool = _poisoned_pool(n_pool, P, D), _poisoned_pool(n_pool, P, D)
+    cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
+    scale = 1.0 / np.sqrt(D)
+    Xs, Ks, Vs, Qs, Os, Ss = [], [], [], [], [], []
+    for step in range(n_steps):
+        Xs.append(parity.dev(synth.hidden_states(L * B, d_model, seed=100 + step).view(L, B, d_model)))
+        Kn, Vn = synth.keys_values(L * B, H, D, seed=300 + step)
+        Ks.append(parity.dev(Kn.view(L, B, H, D)))
+        Vs.append(parity.dev(Vn.view(L, B, H, D)))
+        Qs.append(parity.dev(synth.hidden_states(L * B * H * G, D, seed=500 + step).view(L, B, H * G, D)))
+        Os.append(torch.zeros(L, B, H * G, D, dtype=torch.bfloat16, device="cuda"))
+        Ss.append(torch.empty(L, B, H, dtype=torch.float32, device="cuda"))
+    torch.cuda.synchronize()
+    for step in range(n_steps):
+        binding.kvzap_decode_step(ctx.handle, cache, 0, L, Xs[step], Ks[step], Vs[step], tau, Ss[step])
+        binding.kvzap_decode_attention(ctx.handle, cache, 0, L, Qs[step], scale, Os[step])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    dec = oracle.DecodeOracle(B, L, H, D, w)
+    worst = 0.0
+    for step in range(n_steps):
+        s = Ss[step].cpu().numpy()
+        Kb, Vb = synth.bits(Ks[step].cpu()), synth.bits(Vs[step].cpu())
+        for l in range(L):
+            for b in range(B):
+                dec.append(b, l, s[l, b], Kb[l, b], Vb[l, b], tau)
+        if step % 3 == 0 or step > n_steps - 4:
+            got = Os[step].float().cpu().numpy()
+            Qb = synth.bits(Qs[step].cpu())
+            for l in range(L):
+                for b in range(B):
+                    for h in range(H):
+                        _pos, Kd, Vd = dec.logical(b, l, h)
+                        want = oracle.attention(Qb[l, b, h * G:(h + 1) * G], Kd, Vd, scale)
+                        worst = max(worst, float(np.abs(got[l, b, h * G:(h + 1) * G] - want).max()))
+    assert worst <= ATTN_ATOL, worst
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
