@@ -15,6 +15,7 @@
 #include "decode_kernels.cuh"
 #include "prune_kernels.cuh"
 #include "score_kernel.cuh"
+#include "score_linear_split_kernel.cuh"
 #include "score_split_kernel.cuh"
 #include "select_kernels.cuh"
 
@@ -37,6 +38,7 @@ struct kvzap_ctx {
     kvzap_config cfg;
     int sm_count = 0;
     int w1_rows = 0;                 // rows of the stored first-layer matrix (Linear: padded to 16)
+    bool lin_split_ok = false;       // KVzap-Linear: the four-CTAs-per-tile kernel for short inputs can be used
     // scoring schedules (see ScoreParams): [0] one CTA per tile, [1] CTA pairs (MLP only)
     struct Schedule {
         int group_w = 0, n_groups = 0, chunk_n = 0, n_chunks = 0, n_stages = 0, acc_bufs = 0, acc_stride = 0,
@@ -408,6 +410,61 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         ctx->launches += 1;
         return KVZAP_OK;
     }
+    // KVzap-Linear on few tiles (a short prompt, or a decode step): four CTAs share a tile, each a quarter
+    // of the K range.  The kernel writes only after it has waited for the kernel ahead, so it may always
+    // be placed early.
+    if (c.hidden == 0 && ctx->lin_split_ok && blocks_per_layer * n_layers * kLinSplit <= ctx->sm_count) {
+        CUtensorMap tmap_x;
+        kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
+        if (st != KVZAP_OK) return st;
+        ScoreParams p;
+        memset(&p, 0, sizeof p);
+        p.n_tokens = n_tokens;
+        p.n_tiles = static_cast<int32_t>(blocks_per_layer * n_layers);
+        p.tiles_per_layer = static_cast<int32_t>(blocks_per_layer);
+        p.blocks_per_layer = static_cast<int32_t>(blocks_per_layer);
+        p.n_layers_call = n_layers;
+        p.layer0 = layer;
+        p.w_rows = ctx->w1_rows;
+        p.d_model = c.d_model;
+        p.n_heads = c.n_kv_heads;
+        p.b1 = ctx->b1_all;
+        p.scores = scores;
+        p.maskbits = maskbits;
+        p.n_words = blocks_per_layer * 4;
+        p.cu_seqlens = cu_seqlens;
+        p.n_seqs = n_seqs;
+        p.window = w;
+        p.window_keep = window_keep;
+        p.tau = tau;
+        p.status = ctx->status_dev;
+        const bool early = !ctx->profiling;
+        // Writing before the kernel ahead has completed is safe only if (a) the scores buffer is not the
+        // previous call's, and (b) the launch takes more than half of the SMs (one CTA each): then its
+        // CTAs find room only as CTAs of the previous scoring launch exit, which they do after the
+        // compaction two launches back has completed -- so the mask slice written here, last read
+        // kMaskRing launches back, is free.
+        const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
+        bool clash = false;
+        if (scores && ctx->last_scores) {
+            const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
+            clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes;
+        }
+        p.wait_before_write = (clash || p.n_tiles * kLinSplit * 2 <= ctx->sm_count) ? 1 : 0;
+        ctx->last_score_early = early;
+        ctx->last_scores = scores;
+        ctx->last_scores_bytes = sbytes;
+        {
+            ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
+            cudaLaunchConfig_t cfg;
+            cudaLaunchAttribute attrs[2];
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * kLinSplit)), dim3(kLinThreads), kLinSmemBytes,
+                        stream, early, kLinSplit);
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_linear_split_kernel, tmap_x, ctx->sched[0].tmap_w, p));
+        }
+        ctx->launches += 1;
+        return KVZAP_OK;
+    }
     // CTA pairs pay off once a layer has at least two 128-token blocks; a pair's work tile is 256 tokens
     const bool pair = c.hidden > 0 && ctx->pair_clusters > 0 && blocks_per_layer >= 2;
     const kvzap_ctx::Schedule &sc = ctx->sched[pair ? 1 : 0];
@@ -677,6 +734,13 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     } else {
         CREATE_CUDA(cudaFuncSetAttribute(score_kernel<false, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+        if ((c.d_model / kBlockK) % kLinSplit == 0 && static_cast<int>(kLinSmemBytes) <= budget + 1024) {
+            CREATE_CUDA(cudaFuncSetAttribute(score_linear_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(kLinSmemBytes)));
+            CREATE_CUDA(cudaFuncSetAttribute(score_linear_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+            ctx->lin_split_ok = true;
+        }
     }
 
     ctx->layer_set.assign(c.n_layers, 0);

@@ -1,0 +1,225 @@
+// KVzap-Linear scoring (Method, "KVzap": one linear map from the hidden state to H scores) for SHORT
+// inputs: a prompt of a few thousand tokens gives only a few dozen 128-token tiles, and with one CTA
+// per tile most SMs would idle while each busy one streams a whole 1 MB tile of hidden states at the
+// rate a single SM can pull (the launch then takes ~20 us however fast HBM is).  Here a cluster of
+// kLinSplit CTAs shares a tile: CTA r runs the K blocks [r, r+1) * d_model / kLinSplit of the product
+// (its quarter of the X tile, its quarter of W), the partial 128 x 8 sums of the others go to the
+// cluster's first CTA through distributed shared memory, and after one cluster barrier that CTA adds
+// them in rank order plus the bias and writes scores and keep bits.
+//
+// Warp roles as in score_kernel: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5
+// epilogue (TMEM lane quarter = warp % 4).  The kernel may be placed before the kernel ahead of it in
+// the stream has finished: it reads only hidden states and weights, every thread waits for that
+// kernel before it exits, and with p.wait_before_write set nothing is written before that wait either
+// (the host sets it unless the mask slice and the scores buffer written here are known to be free).
+#pragma once
+
+#include "score_kernel.cuh"
+
+namespace kvzap {
+
+constexpr int kLinSplit = 4;
+constexpr int kLinStages = 8;
+constexpr int kLinThreads = 192;          // producer warp, MMA warp, four epilogue warps
+constexpr uint32_t kLinBTileBytes = 16 * kBlockK * 2;                 // 16 weight rows (H <= 8, padded) of one K block
+constexpr uint32_t kLinStageBytes = kATileBytes + kLinBTileBytes;    // 18 KB, a multiple of 1024
+constexpr uint32_t kLinXpartOff = kLinStages * kLinStageBytes;        // [kLinSplit - 1][128][8] fp32
+constexpr uint32_t kLinBarsOff = kLinXpartOff + (kLinSplit - 1) * kTileM * kMaxHeads * 4;
+constexpr uint32_t kLinSmemBytes = kLinBarsOff + 256 + 1024;          // + barriers + alignment slack
+
+// gridDim.x = kLinSplit * p.n_tiles (cluster dimension kLinSplit); p.n_tiles = 128-token tiles over all
+// layers of the call, p.tiles_per_layer of them per layer; d_model / 64 divisible by kLinSplit.
+__global__ void __launch_bounds__(kLinThreads)
+score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                          const ScoreParams p)
+{
+    extern __shared__ uint8_t lin_smem_raw[];
+    const uint32_t raw_addr = smem_u32(lin_smem_raw);
+    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    uint8_t *smem = lin_smem_raw + pad;
+    const uint32_t smem_base = raw_addr + pad;
+    float *xpart = reinterpret_cast<float *>(smem + kLinXpartOff);
+    const uint32_t bars = smem_base + kLinBarsOff;
+    const uint32_t bar_full = bars;                       // [kLinStages] TMA -> MMA
+    const uint32_t bar_empty = bars + 8 * kLinStages;     // [kLinStages] MMA -> TMA
+    const uint32_t bar_tfull = bars + 16 * kLinStages;    // MMA -> epilogue
+    const uint32_t bar_done = bar_tfull + 8;              // abort path only
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kLinBarsOff + 16 * kLinStages + 16);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kLinBarsOff + 16 * kLinStages + 20);
+
+    griddep_launch_dependents();
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();
+    const int tile = static_cast<int>(blockIdx.x) / kLinSplit;
+    const int l_rel = tile / p.tiles_per_layer;
+    const int m_tile = tile - l_rel * p.tiles_per_layer;
+    const int layer = p.layer0 + l_rel;
+    constexpr uint32_t kTmemCols = 32;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kLinStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        mbar_init(bar_tfull, 1);
+        mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_x);
+        prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const int k_blocks = p.d_model / kBlockK / kLinSplit;      // K blocks of this CTA
+    const int kb_first = static_cast<int>(rank) * k_blocks;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        const uint64_t pol_x = l2_policy_evict_first();    // every byte of X is read once
+        const uint64_t pol_w = l2_policy_evict_last();     // the weights are shared by all tiles of the layer
+        const bool elected = elect_one();
+        const int w_row = layer * p.w_rows;
+        const int row0 = m_tile * kTileM;
+        uint32_t st = 0, st_par = 1, sa = smem_base;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
+                ok = false;
+                break;
+            }
+            if (elected) {
+                mbar_arrive_expect_tx(bar_full + 8 * st, kLinStageBytes);
+                tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row, kb_first + kb, pol_w);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, (kb_first + kb) * kBlockK, row0, l_rel, pol_x);
+            }
+            __syncwarp();
+            sa += kLinStageBytes;
+            if (++st == kLinStages) { st = 0; st_par ^= 1u; sa = smem_base; }
+        }
+        if (!ok && lane == 0) {
+            // abort path: give the copies already in flight a fixed time to land before the CTA exits
+            const long long t0 = clock64();
+            while (clock64() - t0 < 2000000LL) { }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        const uint32_t idesc = umma_idesc_bf16_f32(kTileM, 16);
+        const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
+        const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
+        const uint32_t desc_lo0 = static_cast<uint32_t>(desc0);
+        const bool elected = elect_one();
+        uint32_t st = 0, st_par = 0, a_lo = desc_lo0;
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * st, st_par, abort_flag))) {
+                ok = false;
+                break;
+            }
+            tc_fence_after_sync();
+            if (elected) {
+                issue_k_block<false, 1>(tmem_base, a_lo, a_lo + (kATileBytes >> 4), desc_hi, 0, 0, idesc, kb == 0);
+                umma_commit(bar_empty + 8 * st);
+            }
+            __syncwarp();
+            a_lo += kLinStageBytes >> 4;
+            if (++st == kLinStages) { st = 0; st_par ^= 1u; a_lo = desc_lo0; }
+        }
+        if (ok && elected) umma_commit(bar_tfull);
+        __syncwarp();
+        if (!ok && elected) {
+            umma_commit(bar_done);
+            const long long t0 = clock64();
+            while (!mbar_try_wait(bar_done, 0))
+                if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES / 16) break;
+        }
+    }
+
+    // ------------------------------------------------------------ epilogue (warps 2..5): one thread per token
+    const bool epi = warp >= 2;
+    const int q = warp & 3;                 // TMEM lane quarter
+    const int row = q * 32 + lane;
+    float s[kMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kMaxHeads; ++h) s[h] = 0.0f;
+    if (epi) {
+        if (mbar_wait(bar_tfull, 0, abort_flag)) {
+            tc_fence_after_sync();
+            uint32_t r[16];
+            tmem_ld_x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16), r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) s[h] = __uint_as_float(r[h]);
+        }
+        if (rank != 0) {
+            // the partial sums of this CTA's K range go to the first CTA: xpart[rank - 1][row][8]
+            const uint32_t dst = map_to_cta(smem_base + kLinXpartOff + ((rank - 1) * kTileM + row) * kMaxHeads * 4, 0);
+            st_shared_cluster_v4(dst, s[0], s[1], s[2], s[3]);
+            st_shared_cluster_v4(dst + 16, s[4], s[5], s[6], s[7]);
+        }
+    }
+    tc_fence_before_sync();
+    // every thread of every CTA of the cluster arrives here (all waits above are bounded)
+    cluster_sync_all();
+    if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+    // nothing has been written so far
+    if (p.wait_before_write || rank != 0 || !epi) {
+        griddep_wait();                     // from here on the kernel ahead in the stream has completed
+        if (rank != 0 || !epi) return;
+    }
+
+    // ------------------------------------------------------------ first CTA: total, scores, keep bits
+#pragma unroll
+    for (int r = 0; r < kLinSplit - 1; ++r) {
+        const float4 *src = reinterpret_cast<const float4 *>(xpart + (r * kTileM + row) * kMaxHeads);
+        const float4 pa = src[0], pb = src[1];
+        s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
+        s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
+    }
+#pragma unroll
+    for (int h = 0; h < kMaxHeads; ++h) s[h] += __ldg(p.b1 + layer * p.w_rows + h);
+    const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;
+    const bool valid = t < p.n_tokens;
+    if (valid && p.scores != nullptr) {
+        float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
+        if (p.n_heads == kMaxHeads) {
+            reinterpret_cast<float4 *>(dst)[0] = make_float4(s[0], s[1], s[2], s[3]);
+            reinterpret_cast<float4 *>(dst)[1] = make_float4(s[4], s[5], s[6], s[7]);
+        } else {
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h)
+                if (h < p.n_heads) dst[h] = s[h];
+        }
+    }
+    if (p.maskbits != nullptr) {
+        bool in_window = false;
+        if (valid) {
+            int64_t seq_end = p.n_tokens;
+            if (p.cu_seqlens != nullptr && p.n_seqs > 1)
+                seq_end = __ldg(p.cu_seqlens + seq_of_token(p.cu_seqlens, p.n_seqs, t) + 1);
+            in_window = t >= seq_end - static_cast<int64_t>(p.window);
+        }
+        uint32_t my_word = 0;
+#pragma unroll
+        for (int h = 0; h < kMaxHeads; ++h) {
+            const bool keep = valid && (in_window ? p.window_keep != 0 : s[h] >= p.tau);
+            const uint32_t word = __ballot_sync(0xffffffffu, keep);
+            if (lane == h) my_word = word;
+        }
+        if (lane < p.n_heads)
+            p.maskbits[(static_cast<int64_t>(l_rel) * p.n_heads + lane) * p.n_words + static_cast<int64_t>(m_tile) * 4 + q] = my_word;
+    }
+    griddep_wait();                         // this kernel still completes after the one ahead of it
+}
+
+}  // namespace kvzap
