@@ -568,9 +568,12 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attrs[2];
+        // a short input (one block per CTA, a grid that is resident at once anyway): CTAs of 256 threads
+        const bool short_input = blocks_per_cta == 1 && chunks * c.n_kv_heads <= 4 * static_cast<int64_t>(ctx->sm_count);
         make_launch(&cfg, attrs, dim3(static_cast<unsigned>(chunks), static_cast<unsigned>(c.n_kv_heads)),
-                    dim3(kDenseThreads), 0, stream, !ctx->profiling, 1);
-        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel, static_cast<const uint4 *>(K),
+                    dim3(short_input ? kDenseThreadsShort : kDenseThreads), 0, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, short_input ? compact_dense_kernel<kDenseThreadsShort> : compact_dense_kernel<kDenseThreads>,
+                                           static_cast<const uint4 *>(K),
                                            static_cast<const uint4 *>(V), static_cast<uint4 *>(K_out),
                                            static_cast<uint4 *>(V_out), mask, n_words, n_blocks, blocks_per_cta,
                                            cu_seqlens, n_seqs, n_tokens, c.n_kv_heads, c.head_dim / 8, lengths, 0,
@@ -719,7 +722,9 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
 
     // Kernels share an SM only if they ask for the same split of the L1 / shared-memory array; the
     // scoring kernels need the largest shared-memory split, so the compaction asks for it too.
-    CREATE_CUDA(cudaFuncSetAttribute(compact_dense_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+    CREATE_CUDA(cudaFuncSetAttribute(compact_dense_kernel<kDenseThreads>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+    CREATE_CUDA(cudaFuncSetAttribute(compact_dense_kernel<kDenseThreadsShort>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      static_cast<int>(cudaSharedmemCarveoutMaxShared)));
     CREATE_CUDA(cudaFuncSetAttribute(decode_update_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      static_cast<int>(cudaSharedmemCarveoutMaxShared)));
@@ -1275,7 +1280,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
         make_launch(&cfg, attrs, dim3(static_cast<unsigned>(chunks), static_cast<unsigned>(c.n_kv_heads)),
                     dim3(kDenseThreads), 0, stream, !ctx->profiling, 1);
-        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel, static_cast<const uint4 *>(K),
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, compact_dense_kernel<kDenseThreads>, static_cast<const uint4 *>(K),
                                            static_cast<const uint4 *>(V), static_cast<uint4 *>(K_pool),
                                            static_cast<uint4 *>(V_pool), mask, n_words, n_blocks, blocks_per_cta,
                                            cu_seqlens, static_cast<int>(n_seqs), n_tokens, static_cast<int>(c.n_kv_heads),

@@ -325,6 +325,7 @@ compact_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *
 // slot in its (sequence, head) list is known without any other CTA's help.  lengths[b,h] is
 // written by the thread that handles the last token of sequence b; empty sequences by chunk 0.
 constexpr int kDenseThreads = 128;     // = kBlockTokens: one thread ranks one token; small enough to sit beside a scoring CTA
+constexpr int kDenseThreadsShort = 256; // short inputs (one block per CTA): twice the rows in flight, one round of row loads
 
 // bits of the block's four words below in-block position r (0..128)
 __device__ __forceinline__ int popc_below(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3, int r)
@@ -340,11 +341,13 @@ __device__ __forceinline__ int popc_below(uint32_t w0, uint32_t w1, uint32_t w2,
     return n;
 }
 
-// At most 64 registers per thread (eight CTAs per SM by registers): two of these CTAs then fit into the
+// kThreads = 128, or 256 for short inputs (one block per CTA: all kept rows of the block in flight at once).
+// At most 64 registers per thread (eight 128-thread CTAs per SM by registers): two of these CTAs then fit into the
 // register-file quarters that the MLP scoring kernel's ten warps leave free, so the compaction of layer
 // l runs beside the scoring of layer l + 1 at full width; at 72 registers only one fits and the layer
 // period of the fused path grows by ~10 us.
-__global__ void __launch_bounds__(kDenseThreads, 8)
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
 compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, uint4 *__restrict__ K_out,
                      uint4 *__restrict__ V_out, const uint32_t *__restrict__ maskbits, int64_t n_words,
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
@@ -362,7 +365,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     const bool paged = page_tokens > 0;
     __shared__ int32_t src_tok[kBlockTokens];
     __shared__ int64_t dst_row[kBlockTokens];
-    __shared__ int32_t red[2][kDenseThreads / 32];
+    __shared__ int32_t red[2][kThreads / 32];
     __shared__ int32_t base_next_s;
     const int h = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -377,7 +380,7 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     griddep_wait();
 
     if (blockIdx.x == 0 && cu_seqlens != nullptr && !paged)   // empty sequences have no last token to write for them
-        for (int b = tid; b < n_seqs; b += kDenseThreads)
+        for (int b = tid; b < n_seqs; b += kThreads)
             if (cu_seqlens[b + 1] == cu_seqlens[b]) lengths[b * n_heads + h] = 0;
     if (blk0 >= n_blocks) return;
 
@@ -386,7 +389,9 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     int64_t s0 = 0;
     if (multi) s0 = cu_seqlens[seq_of_token(cu_seqlens, n_seqs, t0)];
     int32_t total = 0, before_s0 = 0;
-    for (int64_t i = tid; i < blk0 * 4; i += kDenseThreads) {
+    // the first block's own words are fetched together with the words before it (one round trip, not two)
+    uint4 wv_next = __ldcg(reinterpret_cast<const uint4 *>(words + blk0 * 4));
+    for (int64_t i = tid; i < blk0 * 4; i += kThreads) {
         const uint32_t w = __ldcg(words + i);     // not a read-only-data load: it must stay behind griddep_wait()
         const int c = __popc(w);
         total += c;
@@ -403,12 +408,13 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
     __syncthreads();
     int32_t running = 0, base_cur = 0;       // kept before the current block / before the sequence in progress at its start
 #pragma unroll
-    for (int i = 0; i < kDenseThreads / 32; ++i) { running += red[0][i]; base_cur += red[1][i]; }
+    for (int i = 0; i < kThreads / 32; ++i) { running += red[0][i]; base_cur += red[1][i]; }
 
     const int group = tid >> 4, gl = tid & 15;
-    constexpr int kGroups = kDenseThreads / 16;
+    constexpr int kGroups = kThreads / 16;
     for (int64_t blk = blk0; blk < blk1; ++blk) {
-        const uint4 wv = __ldcg(reinterpret_cast<const uint4 *>(words + blk * 4));
+        const uint4 wv = wv_next;
+        if (blk + 1 < blk1) wv_next = __ldcg(reinterpret_cast<const uint4 *>(words + (blk + 1) * 4));
         const uint32_t w0 = wv.x, w1 = wv.y, w2 = wv.z, w3 = wv.w;
         const int cnt = __popc(w0) + __popc(w1) + __popc(w2) + __popc(w3);
         const int64_t blk_start = blk * kBlockTokens;
