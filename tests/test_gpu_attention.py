@@ -276,3 +276,39 @@ def test_decode_loop_step_then_attention_enqueued_back_to_back(binding, oracle):
     assert worst <= ATTN_ATOL, worst
     binding.kvzap_cache_destroy(cache)
     ctx.close()
+
+
+def test_attention_without_window_and_with_one_row(binding, oracle):
+    """w = 0 (nothing but the paged prefix) and lists of a single row."""
+    d_model, H, D, P, G = 256, 8, 64, 16, 2
+    ctx = binding.Kvzap(d_model, 0, H, D, 1, max_tokens=128)
+    W, b = synth.linear_weights(d_model, H, 1)
+    ctx.set_weights(0, parity.dev(W), parity.dev(b))
+    K_pool, V_pool = _poisoned_pool(64, P, D), _poisoned_pool(64, P, D)
+    cache = binding.kvzap_cache_create(ctx.handle, 2, 0, P, K_pool, V_pool, 4)
+    dec = oracle.DecodeOracle(2, 1, H, D, 0)
+    Q = synth.hidden_states(2 * H * G, D, seed=3).view(1, 2, H * G, D)
+    O = torch.full((1, 2, H * G, D), 5.0, dtype=torch.bfloat16, device="cuda")
+    for step in range(3):
+        X = synth.hidden_states(2, d_model, seed=20 + step).view(1, 2, d_model)
+        Kn, Vn = synth.keys_values(2, H, D, seed=30 + step)
+        sc = torch.empty(1, 2, H, dtype=torch.float32, device="cuda")
+        tau = float("-inf") if step == 0 else float("inf")         # the first token stays, later ones are dropped at once
+        binding.kvzap_decode_step(ctx.handle, cache, 0, 1, parity.dev(X), parity.dev(Kn).view(1, 2, H, D),
+                                  parity.dev(Vn).view(1, 2, H, D), tau, sc)
+        torch.cuda.synchronize()
+        s = sc.cpu().numpy()
+        for bb in range(2):
+            dec.append(bb, 0, s[0, bb], synth.bits(Kn)[bb], synth.bits(Vn)[bb], tau)
+    binding.kvzap_decode_attention(ctx.handle, cache, 0, 1, parity.dev(Q), 0.125, O)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got = O.float().cpu().numpy()[0]
+    for bb in range(2):
+        for h in range(H):
+            _pos, Kd, Vd = dec.logical(bb, 0, h)
+            assert len(Kd) == 1
+            want = oracle.attention(synth.bits(Q)[0, bb, h * G:(h + 1) * G], Kd, Vd, 0.125)
+            assert np.abs(got[bb, h * G:(h + 1) * G] - want).max() <= ATTN_ATOL
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()

@@ -281,3 +281,33 @@ def test_chunked_prefill_equals_one_prefill(binding, oracle, chunks, w, P):
         np.testing.assert_array_equal(Vg, Vc[h, :n])
     binding.kvzap_cache_destroy(cache)
     ctx.close()
+
+
+def test_chunked_prefill_pool_exhaustion_sets_status(binding):
+    """A second chunk that needs more pages than the pool has left: the status word reports it, the
+    lengths stay what fits, nothing crashes, and the context keeps working."""
+    d_model, H, D, w, P = 256, 8, 64, 8, 4
+    ctx = binding.Kvzap(d_model, 0, H, D, 1, max_tokens=256)
+    W, b = synth.linear_weights(d_model, H, 1)
+    ctx.set_weights(0, parity.dev(W), parity.dev(b))
+    n_pool = H * 6                                      # 24 rows per list
+    K_pool = torch.zeros(n_pool, P, D, dtype=torch.bfloat16, device="cuda")
+    V_pool = torch.zeros_like(K_pool)
+    cache = binding.kvzap_cache_create(ctx.handle, 1, w, P, K_pool, V_pool, 64)
+    lengths = torch.zeros(1, 1, H, dtype=torch.int32, device="cuda")
+    for i, m in enumerate([20, 200]):                    # tau = -inf keeps everything: 12 rows, then 200 more
+        X = parity.dev(synth.hidden_states(m, d_model, seed=i))
+        Kn, Vn = synth.keys_values(H, m, D, seed=10 + i)
+        sc = torch.empty(m, H, dtype=torch.float32, device="cuda")
+        binding.kvzap_prefill_to_cache(ctx.handle, cache, 0, 0, X, parity.dev(Kn), parity.dev(Vn), float("-inf"), sc)
+        torch.cuda.synchronize()
+        st = ctx.poll_status()
+        binding.kvzap_cache_lengths(ctx.handle, cache, lengths)
+        torch.cuda.synchronize()
+        if i == 0:
+            assert st == 0 and (lengths == 20).all()
+        else:
+            assert st == 4                               # KVZAP_ERR_OOM_PAGES
+            assert (lengths <= n_pool // H * P + w).all()
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
