@@ -447,8 +447,80 @@ class Kvzap:
                             scores_out, stream)
         return K_out, V_out, lengths
 
+    def prefill_write(self, layer, hidden, K_proj, V_proj, tau, w, cu_seqlens=None, K_out=None, V_out=None, lengths=None,
+                      scores_out=None, stream=None):
+        """Write-side pruning: K_proj, V_proj [T, H, D] as the projection leaves them -> per-head lists [H, T, D]."""
+        n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        T = K_proj.shape[0]
+        if tuple(K_proj.shape[1:]) != (self.n_kv_heads, self.head_dim) or K_proj.shape != V_proj.shape or \
+                K_proj.dtype != torch.bfloat16:
+            raise ValueError("K_proj/V_proj must be bf16 [T, %d, %d]" % (self.n_kv_heads, self.head_dim))
+        if hidden.shape != (T, self.d_model) or hidden.dtype != torch.bfloat16:
+            raise ValueError("hidden must be bf16 [%d, %d], got %s" % (T, self.d_model, tuple(hidden.shape)))
+        if K_out is None:
+            K_out = torch.empty(self.n_kv_heads, T, self.head_dim, dtype=torch.bfloat16, device=self.device)
+        if V_out is None:
+            V_out = torch.empty_like(K_out)
+        if lengths is None:
+            lengths = torch.empty(n_seqs, self.n_kv_heads, dtype=torch.int32, device=self.device)
+        kvzap_prefill_write(self.handle, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                            scores_out, stream)
+        return K_out, V_out, lengths
+
+    def prune_prefill_topk(self, K, V, scores, keep_ratio, w, per_layer=False, cu_seqlens=None, K_out=None, V_out=None,
+                           lengths=None, tau_out=None, stream=None):
+        """Fixed-budget selection (top-k per head, or per layer) instead of a threshold."""
+        n_seqs = 1 if cu_seqlens is None else cu_seqlens.numel() - 1
+        self._check_shapes(K, V, scores=scores)
+        K_out, V_out, lengths = self._outputs(K, n_seqs, K_out, V_out, lengths)
+        kvzap_prune_prefill_topk(self.handle, K, V, scores, cu_seqlens, n_seqs, keep_ratio, w, per_layer, K_out, V_out,
+                                 lengths, tau_out, stream)
+        return K_out, V_out, lengths
+
+    def create_cache(self, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list) -> "KvzapCache":
+        return KvzapCache(self, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list)
+
     def poll_status(self, stream=None) -> int:
         return kvzap_poll_status(self.handle, stream)
 
     def launch_count(self) -> int:
         return kvzap_launch_count(self.handle)
+
+
+class KvzapCache:
+    """The decode-time cache of one context (window ring + paged prefix per (sequence, layer, head) list).
+    The page pools stay the caller's tensors; the object keeps them alive."""
+
+    def __init__(self, ctx: Kvzap, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list):
+        self.ctx, self.n_seqs, self.window, self.page_tokens = ctx, n_seqs, window, page_tokens
+        self._pools = (K_pool, V_pool)
+        self.handle = kvzap_cache_create(ctx.handle, n_seqs, window, page_tokens, K_pool, V_pool, max_pages_per_list)
+
+    def close(self):
+        if self.handle is not None:
+            kvzap_cache_destroy(self.handle)
+            self.handle = None
+
+    def prefill(self, layer, seq, hidden, K, V, tau, scores_out=None, stream=None):
+        """One prompt, or the next chunk of it, for one layer (chunks of any lengths give the same lists)."""
+        if scores_out is None:
+            scores_out = torch.empty(K.shape[1], self.ctx.n_kv_heads, dtype=torch.float32, device=self.ctx.device)
+        kvzap_prefill_to_cache(self.ctx.handle, self.handle, layer, seq, hidden, K, V, tau, scores_out, stream)
+        return scores_out
+
+    def decode_step(self, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None, stream=None):
+        kvzap_decode_step(self.ctx.handle, self.handle, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out, stream)
+
+    def attention(self, layer_begin, layer_end, Q, scale=None, out=None, stream=None):
+        """The newest token's attention over the pruned lists: Q [L, B, H_q, D] -> O of the same shape."""
+        if out is None:
+            out = torch.empty_like(Q)
+        if scale is None:
+            scale = 1.0 / float(self.ctx.head_dim) ** 0.5
+        kvzap_decode_attention(self.ctx.handle, self.handle, layer_begin, layer_end, Q, scale, out, stream)
+        return out
+
+    def lengths(self, stream=None):
+        out = torch.empty(self.n_seqs, self.ctx.n_layers, self.ctx.n_kv_heads, dtype=torch.int32, device=self.ctx.device)
+        kvzap_cache_lengths(self.ctx.handle, self.handle, out, stream)
+        return out
