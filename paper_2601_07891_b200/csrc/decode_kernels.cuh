@@ -158,83 +158,143 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
     }
 }
 
-// A further chunk of m prompt tokens is about to be appended to lists li0 .. li0+H-1 (chunked
-// prefill): the tokens of the present window that it pushes out are decided here by their buffered
-// scores, oldest first, and the kept ones appended to the list's paged prefix (pages from the
-// cache's cursor), exactly as m decode steps would have done.  One warp per list; n_tokens is left
-// as it is (tokens_add_kernel advances it once the chunk's own rows are in place).
-__global__ void __launch_bounds__(32)
-chunk_evict_kernel(const CacheView c, int64_t li0, int64_t m, float tau, int32_t *__restrict__ status)
+// Chunked prefill, the window side of one chunk of m prompt tokens appended to lists li0 .. li0+H-1
+// (one CTA per list), after the chunk has been scored:
+//   1. the tokens of the present window that the chunk pushes out (positions below n_old + m - w) are
+//      decided by their buffered scores, oldest first, and the kept ones appended to the list's paged
+//      prefix (pages from the cache's cursor) -- what m decode steps would have done;
+//   2. the chunk's last min(m, w) tokens (rows of K, V [H][m][D], scores [m][H]) take the ring slots of
+//      their absolute positions n_old + chunk index;
+//   3. n_tokens advances by m.
+// The chunk's own tokens before its last w are appended to the prefix afterwards by the compaction.
+__global__ void __launch_bounds__(256)
+chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
+                  const uint4 *__restrict__ V, int64_t m, float tau, int32_t *__restrict__ status)
 {
-    const int64_t li = li0 + blockIdx.x;
-    const int lane = threadIdx.x;
+    __shared__ int64_t exit_src[128];       // ring row of an exiting token
+    __shared__ int64_t exit_dst[128];       // its pool row, -1 = dropped
+    __shared__ int64_t len_s;
+    __shared__ int ok_s;
+    const int h = blockIdx.x;
+    const int64_t li = li0 + h;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t n_old = c.n_tokens[li];
     const int64_t in_ring = n_old < c.window ? n_old : c.window;
     const int64_t first = n_old - in_ring;                         // oldest position still in the window
     int64_t exit_end = n_old + m - c.window;                       // positions below it leave the window
     if (exit_end > n_old) exit_end = n_old;
     const int64_t n_exit = exit_end > first ? exit_end - first : 0;
-    int64_t len = c.prefix_len[li];
     int32_t *table = c.page_table + li * c.max_pages;
-    for (int64_t base = 0; base < n_exit; base += 32) {
-        const int64_t pos = first + base + lane;
-        const bool valid = base + lane < n_exit;
-        const int64_t slot = li * c.window + pos % c.window;
-        const bool keep = valid && c.score_ring[slot] >= tau;
-        const uint32_t kept = __ballot_sync(0xffffffffu, keep);
-        const int cnt = __popc(kept);
-        const int64_t have = (len + c.page_tokens - 1) / c.page_tokens;
-        const int64_t want = (len + cnt + c.page_tokens - 1) / c.page_tokens;
-        int ok = 1;
-        if (lane == 0 && want > have) {
-            if (want > c.max_pages) ok = 0;
-            else {
-                const int32_t got = atomicAdd(c.page_cursor, static_cast<int32_t>(want - have));
-                if (static_cast<int64_t>(got) + (want - have) > c.n_pages_pool) ok = 0;
-                else for (int64_t i = have; i < want; ++i) table[i] = got + static_cast<int32_t>(i - have);
+    if (tid == 0) { len_s = c.prefix_len[li]; ok_s = 1; }
+    __syncthreads();
+    for (int64_t base = 0; base < n_exit && ok_s; base += 128) {
+        if (warp == 0) {
+            int64_t len = len_s;
+            for (int i = lane; i < 128; i += 32) exit_dst[i] = -1;     // nothing is copied unless it is decided below
+            float sc4[4];                                              // the buffered scores of the batch, loaded together
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t pos = first + base + 32 * j + lane;
+                sc4[j] = base + 32 * j + lane < n_exit ? c.score_ring[li * c.window + pos % c.window] : 0.0f;
             }
-            if (!ok) atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+            __syncwarp();
+#pragma unroll
+            for (int sub = 0; sub < 128; sub += 32) {
+                if (base + sub >= n_exit) break;
+                const int64_t pos = first + base + sub + lane;
+                const bool valid = base + sub + lane < n_exit;
+                const int64_t slot = li * c.window + pos % c.window;
+                const bool keep = valid && sc4[sub >> 5] >= tau;
+                const uint32_t kept = __ballot_sync(0xffffffffu, keep);
+                const int cnt = __popc(kept);
+                const int64_t have = (len + c.page_tokens - 1) / c.page_tokens;
+                const int64_t want = (len + cnt + c.page_tokens - 1) / c.page_tokens;
+                int ok = 1;
+                if (lane == 0 && want > have) {
+                    if (want > c.max_pages) ok = 0;
+                    else {
+                        const int32_t got = atomicAdd(c.page_cursor, static_cast<int32_t>(want - have));
+                        if (static_cast<int64_t>(got) + (want - have) > c.n_pages_pool) ok = 0;
+                        else for (int64_t i = have; i < want; ++i) table[i] = got + static_cast<int32_t>(i - have);
+                    }
+                    if (!ok) atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                __syncwarp();
+                if (valid) {
+                    int64_t dst = -1;
+                    if (keep && ok) {
+                        const int64_t nn = len + __popc(kept & ((1u << lane) - 1u));
+                        const int64_t page = *(volatile int32_t *)(table + nn / c.page_tokens);
+                        dst = page * c.page_tokens + nn % c.page_tokens;
+                    }
+                    exit_src[sub + lane] = slot;
+                    exit_dst[sub + lane] = dst;
+                }
+                if (!ok) { if (lane == 0) ok_s = 0; break; }       // what was appended so far stays valid
+                len += cnt;
+            }
+            if (lane == 0) len_s = len;
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;                                            // what was appended so far stays valid
-        __syncwarp();
-        if (keep) {
-            const int64_t nn = len + __popc(kept & ((1u << lane) - 1u));
-            const int64_t page = *(volatile int32_t *)(table + nn / c.page_tokens);
-            const int64_t dst = (page * c.page_tokens + nn % c.page_tokens) * c.row_units;
-            for (int u = 0; u < c.row_units; ++u) {
-                c.k_pool[dst + u] = c.k_ring[slot * c.row_units + u];
-                c.v_pool[dst + u] = c.v_ring[slot * c.row_units + u];
+        __syncthreads();
+        // rows of this batch of exits: 16 lanes per row
+        const int64_t n_batch = n_exit - base < 128 ? n_exit - base : 128;
+        for (int64_t i0 = tid >> 4; i0 < n_batch; i0 += 64) {     // four rows per lane group in flight
+            for (int u = tid & 15; u < c.row_units; u += 16) {
+                uint4 kr[4], vr[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t i = i0 + 16 * j;
+                    if (i < n_batch && exit_dst[i] >= 0) {
+                        kr[j] = c.k_ring[exit_src[i] * c.row_units + u];
+                        vr[j] = c.v_ring[exit_src[i] * c.row_units + u];
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t i = i0 + 16 * j;
+                    if (i < n_batch && exit_dst[i] >= 0) {
+                        c.k_pool[exit_dst[i] * c.row_units + u] = kr[j];
+                        c.v_pool[exit_dst[i] * c.row_units + u] = vr[j];
+                    }
+                }
             }
         }
-        len += cnt;
+        __syncthreads();
     }
-    if (lane == 0) c.prefix_len[li] = static_cast<int32_t>(len);
-}
-
-// The last min(m, w) tokens of a chunk of m (rows of K, V [H][m][D], scores [m][H]) go into the window
-// rings of lists li0 .. li0+H-1 at the slots of their absolute positions n_tokens + chunk index.
-__global__ void __launch_bounds__(256)
-ring_append_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
-                   const uint4 *__restrict__ V, int64_t m)
-{
-    const int h = blockIdx.y;
-    const int64_t li = li0 + h;
-    const int64_t n_old = c.n_tokens[li];
+    // the chunk's last min(m, w) tokens into the ring (the slots they take were read above)
     const int64_t n_win = m < c.window ? m : c.window;
-    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_win * c.row_units;
-         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-        const int64_t j = i / c.row_units;
-        const int u = static_cast<int>(i % c.row_units);
-        const int64_t ci = m - n_win + j;                      // index inside the chunk
-        const int64_t slot = li * c.window + (n_old + ci) % c.window;
-        const int64_t src = (static_cast<int64_t>(h) * m + ci) * c.row_units + u;
-        c.k_ring[slot * c.row_units + u] = K[src];
-        c.v_ring[slot * c.row_units + u] = V[src];
-        if (u == 0) c.score_ring[slot] = scores[ci * c.n_heads + h];
+    for (int64_t i0 = tid; i0 < n_win * c.row_units; i0 += 4 * 256) {     // four units per thread in flight
+        uint4 kr[4], vr[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t i = i0 + 256 * j;
+            if (i < n_win * c.row_units) {
+                const int64_t src = (static_cast<int64_t>(h) * m + m - n_win + i / c.row_units) * c.row_units + i % c.row_units;
+                kr[j] = __ldg(K + src);
+                vr[j] = __ldg(V + src);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t i = i0 + 256 * j;
+            if (i < n_win * c.row_units) {
+                const int64_t ci = m - n_win + i / c.row_units;        // index inside the chunk
+                const int u = static_cast<int>(i % c.row_units);
+                const int64_t slot = li * c.window + (n_old + ci) % c.window;
+                c.k_ring[slot * c.row_units + u] = kr[j];
+                c.v_ring[slot * c.row_units + u] = vr[j];
+                if (u == 0) c.score_ring[slot] = scores[ci * c.n_heads + h];
+            }
+        }
+    }
+    if (tid == 0) {
+        c.prefix_len[li] = static_cast<int32_t>(len_s);
+        c.n_tokens[li] = static_cast<int32_t>(n_old + m);
     }
 }
 
+// no window: only the token count advances
 __global__ void tokens_add_kernel(const CacheView c, int64_t li0, int64_t m)
 {
     if (threadIdx.x < c.n_heads) c.n_tokens[li0 + threadIdx.x] += static_cast<int32_t>(m);

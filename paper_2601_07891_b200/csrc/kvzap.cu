@@ -71,8 +71,6 @@ struct kvzap_ctx {
     bool last_score_early = false;       // the last scoring launch was allowed to start early
     const void *last_scores = nullptr;   // scores buffer of the previous scoring launch, and its size
     size_t last_scores_bytes = 0;
-    int32_t *blockprefix = nullptr;  // [H][max_blocks + 1]
-    int32_t *seqbase = nullptr;      // [H][max_seqs + 1]
     int32_t *list_page0 = nullptr;   // [max_seqs * H] first page of each list (paged output)
     int32_t *list_base = nullptr;    // [max_seqs * H] appending to lists: rows each list held before
     int32_t *list_tail = nullptr;    // [max_seqs * H]                     and the page of its last row
@@ -235,8 +233,6 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->select_hist);
     cudaFree(ctx->select_tau);
     cudaFree(ctx->split_arrive);
-    cudaFree(ctx->blockprefix);
-    cudaFree(ctx->seqbase);
     cudaFree(ctx->list_page0);
     cudaFree(ctx->list_base);
     cudaFree(ctx->list_tail);
@@ -795,8 +791,6 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
     ctx->max_words = ctx->max_blocks * 4;
     CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * kMaskRing * ctx->max_words * c.n_kv_heads));
-    CREATE_CUDA(cudaMalloc(&ctx->blockprefix, sizeof(int32_t) * (ctx->max_blocks + 1) * c.n_kv_heads));
-    CREATE_CUDA(cudaMalloc(&ctx->seqbase, sizeof(int32_t) * (static_cast<int64_t>(c.max_seqs) + 1) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_base, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_tail, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
@@ -1264,7 +1258,8 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
         ProfScope prof(ctx, KVZAP_KERNEL_SCAN, stream);
         make_launch(&cfg, attrs, dim3(1), dim3(1024), 0, stream, !ctx->profiling, 1);
         KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, scan_kernel, mask, n_words, n_blocks, static_cast<int>(c.n_kv_heads),
-                                           cu_seqlens, static_cast<int>(n_seqs), n_tokens, ctx->blockprefix, ctx->seqbase,
+                                           cu_seqlens, static_cast<int>(n_seqs), n_tokens, static_cast<int32_t *>(nullptr),
+                                           static_cast<int32_t *>(nullptr),
                                            lengths, static_cast<int>(page_tokens), first_page, n_pages_pool,
                                            static_cast<int>(max_pages), ctx->list_page0, page_table, n_pages_used,
                                            page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, ctx->list_tail));
@@ -1687,34 +1682,24 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
         return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache: hidden, K, V, scores_out must be non-NULL, aligned");
     DeviceGuard guard(c.device);
     const int64_t li0 = (static_cast<int64_t>(seq) * v.n_layers + layer) * v.n_heads;
-    // The lists may already hold earlier chunks of the prompt.  First the tokens of the present window
-    // that this chunk pushes out are decided by their buffered scores (as decode steps would have done).
-    if (v.window > 0) {
-        chunk_evict_kernel<<<static_cast<unsigned>(v.n_heads), 32, 0, stream>>>(v, li0, n_tokens, tau, ctx->status_dev);
-        KVZAP_CUDA(ctx, cudaGetLastError());
-        ctx->launches += 1;
-    }
-    // Then the chunk itself.  mask = threshold only, the chunk's last `window` tokens left out: they go
-    // to the ring below; the kept ones are appended behind what the lists hold.
+    // The lists may already hold earlier chunks of the prompt.  Scoring first (mask = threshold only, the
+    // chunk's last `window` tokens left out: they go to the ring); then the window side -- the tokens the
+    // chunk pushes out of the present window are decided by their buffered scores and appended to the
+    // prefix, the chunk's last tokens take their ring slots; then the chunk's kept tokens are appended
+    // behind what the lists hold by then.
     uint32_t *mask = next_mask_slice(ctx);
     st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, nullptr, 1, tau, v.window, stream, 0);
     if (st != KVZAP_OK) return st;
-    st = launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
-                                 v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
-                                 v.page_cursor, false, true);
-    if (st != KVZAP_OK) return st;
-    if (v.window > 0) {
-        const int64_t n_win = n_tokens < v.window ? n_tokens : v.window;
-        const unsigned gx = static_cast<unsigned>((n_win * v.row_units + 255) / 256);
-        ring_append_kernel<<<dim3(gx, static_cast<unsigned>(v.n_heads)), 256, 0, stream>>>(
-            v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens);
-        KVZAP_CUDA(ctx, cudaGetLastError());
-        ctx->launches += 1;
-    }
-    tokens_add_kernel<<<1, 32, 0, stream>>>(v, li0, n_tokens);
+    if (v.window > 0)
+        chunk_ring_kernel<<<static_cast<unsigned>(v.n_heads), 256, 0, stream>>>(
+            v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens, tau, ctx->status_dev);
+    else
+        tokens_add_kernel<<<1, 32, 0, stream>>>(v, li0, n_tokens);
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
-    return KVZAP_OK;
+    return launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
+                                   v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
+                                   v.page_cursor, false, true);
 }
 
 }  // extern "C"

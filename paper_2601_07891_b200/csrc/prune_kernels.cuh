@@ -95,8 +95,9 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
 }
 
 // ---------------------------------------------------------------------------
-// One CTA of 1024 threads.  blockprefix [H][n_blocks+1], seqbase [H][n_seqs+1],
-// lengths [n_seqs][H].  Paged output (page_tokens > 0): list (b,h) gets
+// One CTA of 1024 threads.  blockprefix [H][n_blocks+1], seqbase [H][n_seqs+1] (both nullptr when only the
+// lengths and the page assignment are wanted: the lists are then counted directly), lengths [n_seqs][H].
+// Paged output (page_tokens > 0): list (b,h) gets
 // ceil(len/page_tokens) pages numbered contiguously from first_page in (b,h)
 // order; list_page0 [n_seqs*H] receives each list's first page and page_table
 // [n_seqs*H][max_pages] its page numbers; *n_pages_used the total.  A pool or
@@ -150,6 +151,43 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         return x + (warp > 0 ? warp_sums[warp - 1] : 0);
     };
 
+    if (blockprefix == nullptr) {
+        // Only the lengths are wanted (the compaction counts its own prefixes): every list's kept rows are
+        // counted straight from the mask words of its token range, a group of threads per list.
+        const int n_lists_all = n_heads * n_seqs;
+        int per_list = 1024;
+        while (per_list > 32 && 1024 / per_list < n_lists_all) per_list >>= 1;
+        const int n_groups = 1024 / per_list, grp = tid / per_list, gt = tid % per_list;
+        __shared__ int32_t group_sum[32];
+        for (int idx0 = 0; idx0 < n_lists_all; idx0 += n_groups) {
+            if (tid < 32) group_sum[tid] = 0;
+            __syncthreads();
+            const int idx = idx0 + grp;
+            int32_t cnt = 0;
+            if (idx < n_lists_all) {
+                const int b = idx / n_heads, h = idx % n_heads;
+                const int64_t t_lo = cu_seqlens != nullptr ? static_cast<int64_t>(cu_seqlens[b]) : 0;
+                const int64_t t_hi = cu_seqlens != nullptr ? static_cast<int64_t>(cu_seqlens[b + 1]) : n_tokens;
+                const uint32_t *wh = maskbits + static_cast<int64_t>(h) * n_words;
+                for (int64_t wi = t_lo / 32 + gt; wi * 32 < t_hi; wi += per_list) {
+                    uint32_t w = __ldcg(wh + wi);
+                    if (wi * 32 < t_lo) w &= ~0u << static_cast<int>(t_lo - wi * 32);               // bits below the sequence
+                    if (wi * 32 + 32 > t_hi) w &= (1u << static_cast<int>(t_hi - wi * 32)) - 1u;    // bits above it
+                    cnt += __popc(w);
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+            if (lane == 0 && cnt) atomicAdd(&group_sum[grp], cnt);
+            __syncthreads();
+            if (gt == 0 && idx < n_lists_all) {
+                const int32_t old = append ? lengths[idx] : 0;
+                if (append) list_base[idx] = old;
+                lengths[idx] = old + group_sum[grp];
+            }
+            __syncthreads();
+        }
+    } else {
     for (int h = 0; h < n_heads; ++h) {
         if (tid == 0) carry_s = 0;
         __syncthreads();
@@ -183,6 +221,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         const int32_t old = append ? lengths[idx] : 0;
         if (append) list_base[idx] = old;
         lengths[idx] = old + seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
+    }
     }
     if (page_tokens <= 0) return;
 
@@ -224,12 +263,13 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         if (n_pages_used != nullptr) *n_pages_used = used;
         if (page_cursor != nullptr) *page_cursor = first_page + used;
     }
-    for (int idx = tid; idx < n_lists; idx += 1024) {
+    __syncthreads();      // list_page0 and lengths of all lists are final
+    for (int idx = warp; idx < n_lists; idx += 32) {            // a warp per list
         const int32_t p0 = list_page0[idx];
         const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
         const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
-        if (append) list_tail[idx] = have > 0 ? page_table[static_cast<int64_t>(idx) * max_pages + have - 1] : -1;
-        for (int32_t i = 0; i < need; ++i) page_table[static_cast<int64_t>(idx) * max_pages + have + i] = p0 + i;
+        if (append && lane == 0) list_tail[idx] = have > 0 ? page_table[static_cast<int64_t>(idx) * max_pages + have - 1] : -1;
+        for (int32_t i = lane; i < need; i += 32) page_table[static_cast<int64_t>(idx) * max_pages + have + i] = p0 + i;
     }
 }
 
