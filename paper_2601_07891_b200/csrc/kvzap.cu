@@ -51,6 +51,12 @@ struct kvzap_ctx {
     int split_n = 0, split_k = 1, split_stages = 0, split_tmem_cols = 0;   // cluster = split_n * split_k CTAs
     uint32_t split_smem = 0;
     CUtensorMap split_tmap_w;
+    // the same kernel with eight CTAs per tile (4 slices x 2 halves of K) for launches of even fewer tiles
+    // (a short prompt or a chunk of one): set when the shape allows it
+    int wide_n = 0, wide_k = 1, wide_stages = 0, wide_tmem_cols = 0;
+    uint32_t wide_smem = 0;
+    CUtensorMap wide_tmap_w;
+    uint32_t *wide_arrive = nullptr;     // its own arrival counts (the count per tile is taken modulo the slices)
     // weights of all layers, stacked so that one tensor map / one base pointer serves any layer range
     void *w1_all = nullptr;          // bf16 [L * w1_rows, d_model]
     float *b1_all = nullptr;         // [L][w1_rows]
@@ -233,6 +239,7 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->select_hist);
     cudaFree(ctx->select_tau);
     cudaFree(ctx->split_arrive);
+    cudaFree(ctx->wide_arrive);
     cudaFree(ctx->list_page0);
     cudaFree(ctx->list_base);
     cudaFree(ctx->list_tail);
@@ -338,6 +345,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // Few tiles (a decode step: one tile per layer): split every tile's hidden units (and K range) over
     // several CTAs, so that the launch fills the machine and every CTA reads only its own part of W1.
     if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count) {
+        // eight CTAs per tile when even those fit (not for the fused decode step, which is laid out for four)
+        const bool wide = ctx->wide_n > 0 && fuse == nullptr &&
+                          blocks_per_layer * n_layers * ctx->wide_n * ctx->wide_k <= ctx->sm_count;
+        const int split_n = wide ? ctx->wide_n : ctx->split_n, split_k = wide ? ctx->wide_k : ctx->split_k;
         CUtensorMap tmap_x;
         kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
         if (st != KVZAP_OK) return st;
@@ -351,11 +362,11 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         p.layer0 = layer;
         p.w_rows = ctx->w1_rows;
         p.d_model = c.d_model;
-        p.group_w = p.chunk_n = c.hidden / ctx->split_n;
+        p.group_w = p.chunk_n = c.hidden / split_n;
         p.n_groups = p.n_chunks = 1;
-        p.n_stages = ctx->split_stages;
+        p.n_stages = wide ? ctx->wide_stages : ctx->split_stages;
         p.acc_bufs = 1;
-        p.tmem_cols = ctx->split_tmem_cols;
+        p.tmem_cols = wide ? ctx->wide_tmem_cols : ctx->split_tmem_cols;
         p.n_hidden = c.hidden;
         p.n_heads = c.n_kv_heads;
         p.b1 = ctx->b1_all;
@@ -371,7 +382,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         p.tau = tau;
         p.status = ctx->status_dev;
         p.split_part = ctx->split_part;
-        p.split_arrive = ctx->split_arrive;
+        p.split_arrive = wide ? ctx->wide_arrive : ctx->split_arrive;
         // Early start (consecutive decode steps): this kernel reads only hidden states and weights; the one
         // thing it may not do is write a scores buffer that the kernels of the previous call still read.
         const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
@@ -382,7 +393,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         }
         ctx->last_scores = scores;
         ctx->last_scores_bytes = sbytes;
-        const int n_ctas = ctx->split_n * ctx->split_k;
+        const int n_ctas = split_n * split_k;
         // only the fused decode step is started early: its clusters order themselves through `done`
         DecodeFuse f;
         memset(&f, 0, sizeof f);
@@ -399,9 +410,9 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attrs[2];
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * n_ctas)), dim3(kScoreThreads),
-                        ctx->split_smem, stream, early, ctx->split_k);
-            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, ctx->split_tmap_w, p, ctx->split_n,
-                                               ctx->split_k, f));
+                        wide ? ctx->wide_smem : ctx->split_smem, stream, early, split_k);
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, wide ? ctx->wide_tmap_w : ctx->split_tmap_w, p,
+                                               split_n, split_k, f));
         }
         ctx->launches += 1;
         return KVZAP_OK;
@@ -787,6 +798,26 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
                 ctx->split_k = k_split;
             }
         }
+        // 4 x 2: slices of hidden / 4 units, each CTA finishing hidden / 8 of them
+        const int ns8 = c.hidden / 4;
+        if (ctx->split_n > 0 && c.hidden % 128 == 0 && ns8 <= 256 && (c.d_model / kBlockK) % 2 == 0) {
+            int st8 = kMaxStages;
+            for (; st8 >= 2; --st8)
+                if (static_cast<int>(split_smem_layout(ns8, st8, 8).total) <= budget - 4096) break;
+            if (st8 >= 2) {
+                ctx->wide_stages = st8;
+                ctx->wide_smem = split_smem_layout(ns8, st8, 8).total + 1024;
+                ctx->wide_tmem_cols = next_pow2(ns8);
+                if (ctx->wide_smem > ctx->split_smem)
+                    CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     static_cast<int>(ctx->wide_smem)));
+                if (make_tmap_w(ctx, &ctx->wide_tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
+                                static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns8)) == KVZAP_OK) {
+                    ctx->wide_n = 4;
+                    ctx->wide_k = 2;
+                }
+            }
+        }
     }
     ctx->max_blocks = (c.max_tokens + kBlockTokens - 1) / kBlockTokens;
     ctx->max_words = ctx->max_blocks * 4;
@@ -802,6 +833,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         CREATE_CUDA(cudaMalloc(&ctx->split_part, sizeof(float) * static_cast<size_t>(ctx->sm_count) * 4 * kTileM * kMaxHeads));
         CREATE_CUDA(cudaMalloc(&ctx->split_arrive, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
         CREATE_CUDA(cudaMemset(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
+        CREATE_CUDA(cudaMalloc(&ctx->wide_arrive, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
+        CREATE_CUDA(cudaMemset(ctx->wide_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
     }
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
@@ -1014,6 +1047,7 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     // a scoring kernel that gave up may have left its work-tile counter in an unknown state
     cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing, stream);
     if (ctx->split_arrive) cudaMemsetAsync(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
+    if (ctx->wide_arrive) cudaMemsetAsync(ctx->wide_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
     cudaStreamSynchronize(stream);
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
