@@ -82,3 +82,44 @@ def test_back_to_back_calls_equal_synchronous_calls(binding, d_model, hidden, T,
         if not shared_scores:
             assert torch.equal(a["sc"].view(torch.int32), b["sc"].view(torch.int32))
     ctx.close()
+
+
+def test_two_contexts_on_two_streams_do_not_disturb_each_other(binding):
+    """An MLP context and a Linear context, each on its own stream, calls interleaved from the host:
+    every output equals what the same context gives when it runs alone and synchronously."""
+    H, D, tau, w, T = 8, 64, 0.1, 16, 3000
+    cfgs = [(512, 256), (256, 0)]
+    ctxs, sets = [], []
+    for d_model, hidden in cfgs:
+        ctx = binding.Kvzap(d_model, hidden, H, D, 1, T)
+        wts = (synth.mlp_weights(d_model, hidden, H, 3, "cuda", 0.3) if hidden
+               else synth.linear_weights(d_model, H, 3, "cuda", 0.3))
+        ctx.set_weights(0, *wts)
+        ctxs.append(ctx)
+        sets.append(_make_sets(3, T, d_model, H, D, seed=50 + hidden))
+    torch.cuda.synchronize()
+
+    def run(concurrent):
+        outs = [[_outputs(T, H, D) for _ in range(6)] for _ in ctxs]
+        streams = [torch.cuda.Stream() for _ in ctxs] if concurrent else [None, None]
+        for i in range(6):
+            for c, ctx in enumerate(ctxs):
+                s, o = sets[c][i % 3], outs[c][i]
+                binding.kvzap_prefill_fused(ctx.handle, 0, s["X"], s["K"], s["V"], None, 1, tau, w, o["Ko"], o["Vo"],
+                                            o["len"], o["sc"], stream=streams[c])
+                if not concurrent:
+                    torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        return outs
+
+    alone = run(False)
+    both = run(True)
+    for c in range(2):
+        assert ctxs[c].poll_status() == 0
+        for i in range(6):
+            for key in ("len", "sc"):
+                assert torch.equal(alone[c][i][key], both[c][i][key]), (c, i, key)
+            for key in ("Ko", "Vo"):
+                assert torch.equal(alone[c][i][key].view(torch.int16), both[c][i][key].view(torch.int16)), (c, i, key)
+    for ctx in ctxs:
+        ctx.close()
