@@ -47,6 +47,33 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def live_gemm_tflops(dev, seconds=1.5):
+    """cuBLAS bf16 GEMM (8192^3) looped for `seconds` on this GPU, right after the timed region: the
+    same kind of number as MEASURED_PEAKS.json's bf16_tflops_sustained, but of this GPU in its present
+    power and thermal state.  Measurement aid only; nothing of the hot path runs through it."""
+    import torch
+    n = 8192
+    a = torch.randn(n, n, dtype=torch.bfloat16, device=dev)
+    b = torch.randn(n, n, dtype=torch.bfloat16, device=dev)
+    c = torch.empty(n, n, dtype=torch.bfloat16, device=dev)
+    for _ in range(3):
+        torch.matmul(a, b, out=c)
+    torch.cuda.synchronize()
+    per = 2.0 * n ** 3
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps, done, t_total, last = 40, 0, 0.0, 0.0
+    while t_total < seconds * 1e3:
+        e0.record()
+        for _ in range(reps):
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        last = e0.elapsed_time(e1)
+        t_total += last
+        done += reps
+    return per * reps / (last * 1e-3) / 1e12          # the last block of launches: the settled rate
+
+
 def surrogate_flops_per_token(wl):
     """Algorithmic FLOPs per token per layer (Appendix B): 2 D_h N1 + 2 N1 H, or 2 D_h H."""
     if wl.surrogate == "mlp":
@@ -312,6 +339,11 @@ def run_prefill(args, wl, env):
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
                     "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
                     "alone_achieved": flops / (score_ms * 1e-3) / 1e12}
+        if not args.skip_live_peak:
+            # the GPUs of the pool settle at different clocks under the power cap: the same loop on this one, now
+            live = live_gemm_tflops(dev)
+            roofline["live_cublas_bf16_tflops_sustained"] = live
+            roofline["frac_of_live_cublas"] = achieved / live
     else:
         achieved = score_bytes / (layer_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -641,6 +673,8 @@ def main():
                     help="prefill workloads: K/V as [H,T,D] (default) or as the projection writes them, [T,H,D]")
     ap.add_argument("--attention", action="store_true",
                     help="decode workload: time the attention over the pruned cache instead of the pruning step")
+    ap.add_argument("--skip-live-peak", action="store_true",
+                    help="tensor-bound workloads: do not run the cuBLAS loop that measures this GPU's sustained rate")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--ref-tokens", type=int, default=32768,
