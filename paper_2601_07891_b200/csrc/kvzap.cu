@@ -344,11 +344,16 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
     // Few tiles (a decode step: one tile per layer): split every tile's hidden units (and K range) over
     // several CTAs, so that the launch fills the machine and every CTA reads only its own part of W1.
-    if (ctx->split_n > 0 && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count) {
+    // ... and with the K split left out (two CTAs per tile, each a slice of the hidden units over the whole K
+    // range) the same kernel serves launches of up to half as many tiles as there are SMs, where CTA pairs
+    // would leave most SMs idle.
+    const bool slices_only = ctx->split_n == 2 && ctx->split_k == 2 && fuse == nullptr &&
+                             blocks_per_layer * n_layers * 4 > ctx->sm_count && blocks_per_layer * n_layers * 2 <= ctx->sm_count;
+    if (ctx->split_n > 0 && (slices_only || blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count)) {
         // eight CTAs per tile when even those fit (not for the fused decode step, which is laid out for four)
         const bool wide = ctx->wide_n > 0 && fuse == nullptr &&
                           blocks_per_layer * n_layers * ctx->wide_n * ctx->wide_k <= ctx->sm_count;
-        const int split_n = wide ? ctx->wide_n : ctx->split_n, split_k = wide ? ctx->wide_k : ctx->split_k;
+        const int split_n = wide ? ctx->wide_n : ctx->split_n, split_k = wide ? ctx->wide_k : (slices_only ? 1 : ctx->split_k);
         CUtensorMap tmap_x;
         kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
         if (st != KVZAP_OK) return st;

@@ -47,10 +47,14 @@ def test_linear_scores_match_oracle(binding, oracle, T):
 
 @pytest.mark.parametrize("d_model,hidden,T", [(256, 64, 300), (512, 128, 129), (256, 256, 257), (256, 512, 520),
                                               (256, 640, 200), (128, 1024, 131), (4096, 512, 260), (5120, 640, 130),
-                                              (1024, 512, 700), (512, 384, 1000), (2048, 1024, 300)])
+                                              (1024, 512, 700), (512, 384, 1000), (2048, 1024, 300),
+                                              # 47 and 71 tiles: two CTAs per tile, one per half of the hidden units
+                                              (256, 128, 6000), (512, 256, 9000),
+                                              # 12 tiles of an MLP whose width allows eight CTAs per tile
+                                              (512, 256, 1500)])
 def test_mlp_scores_match_oracle(binding, oracle, d_model, hidden, T):
     H = 8
-    ctx = _make_ctx(binding, d_model, hidden, H, 128, max_tokens=1024)
+    ctx = _make_ctx(binding, d_model, hidden, H, 128, max_tokens=max(1024, T))
     weights = _weights(d_model, hidden, H, seed=hidden + T)
     ctx.set_weights(0, *[parity.dev(w) for w in weights])
     X = synth.hidden_states(T, d_model, seed=7 * T)
@@ -133,7 +137,7 @@ def test_fused_linear_single_sequence(binding, oracle, T, w, tau):
         assert (lengths == T).all()
 
 
-@pytest.mark.parametrize("hidden,T", [(64, 300), (512, 600), (640, 257)])
+@pytest.mark.parametrize("hidden,T", [(64, 300), (512, 600), (640, 257), (128, 7000)])
 def test_fused_mlp_single_sequence(binding, oracle, hidden, T):
     _run_fused(binding, oracle, 256, hidden, 8, 128, [T], 0.2, 128, seed=hidden)
 
