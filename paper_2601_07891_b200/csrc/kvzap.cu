@@ -4,9 +4,11 @@
 
 #include <cuda.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -190,6 +192,19 @@ __global__ void pack_w2_kernel(const uint16_t *__restrict__ W2, const float *__r
     }
     if (idx < kMaxHeads) b2p[idx] = (b2 != nullptr && idx < n_heads) ? b2[idx] : 0.0f;
 }
+
+// NVTX range around a public call, for timelines; off unless the environment has KVZAP_NVTX=1 when the
+// library is first used (the header-only NVTX does nothing without a tool attached).
+static bool nvtx_enabled()
+{
+    static const bool on = [] { const char *v = getenv("KVZAP_NVTX"); return v != nullptr && v[0] == '1'; }();
+    return on;
+}
+struct NvtxRange {
+    bool on;
+    explicit NvtxRange(const char *name) : on(nvtx_enabled()) { if (on) nvtxRangePushA(name); }
+    ~NvtxRange() { if (on) nvtxRangePop(); }
+};
 
 // Brackets one kernel launch with events when profiling is on.
 struct ProfScope {
@@ -868,6 +883,7 @@ int64_t kvzap_launch_count(const kvzap_ctx *ctx) { return ctx ? ctx->launches : 
 kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, const float *b1, const void *W2,
                                const float *b2, void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_set_weights");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
@@ -907,6 +923,7 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, co
 kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens, float *scores,
                          void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_score");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
@@ -924,6 +941,7 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
                                  const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
                                  void *K_out, void *V_out, int32_t *lengths, void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_prune_prefill");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -956,6 +974,7 @@ kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void 
                                       int32_t w, int32_t per_layer, void *K_out, void *V_out, int32_t *lengths,
                                       float *tau_out, void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_prune_prefill_topk");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -1000,6 +1019,7 @@ static kvzap_status prefill_fused_impl(kvzap_ctx *ctx, int32_t layer, const void
                                        int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
                                        void *stream_, bool tok_major)
 {
+    NvtxRange nvtx_range("kvzap_prefill_fused / kvzap_prefill_write");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -1092,6 +1112,7 @@ kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void 
                                       int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
                                       void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_prefill_fused_host");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
@@ -1355,6 +1376,7 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
                                        int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
                                        void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_prune_prefill_paged");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -1392,6 +1414,7 @@ static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, cons
                                              int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
                                              float *scores_out, void *stream_, bool tok_major)
 {
+    NvtxRange nvtx_range("kvzap_prefill_fused_paged / kvzap_prefill_write_paged");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -1517,6 +1540,7 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
                                const void *hidden, const void *K_new, const void *V_new, float tau,
                                float *scores_out, void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_decode_step");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
@@ -1577,6 +1601,7 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
 kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
                                     const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_decode_attention");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
@@ -1707,6 +1732,7 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
                                     const void *K, const void *V, int64_t n_tokens, float tau, float *scores_out,
                                     void *stream_)
 {
+    NvtxRange nvtx_range("kvzap_prefill_to_cache");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
