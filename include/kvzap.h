@@ -321,6 +321,15 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
 kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
                                     const void *Q, int32_t n_q_heads, float scale, void *O, void *stream);
 
+/*
+ * A sequence has ended: all lists (seq, *, *) become empty and their pages go back to the cache's
+ * allocator, which hands released pages out again (to any list) before it touches never-used pages
+ * of the pool.  The slot `seq` can then take a new prompt (kvzap_prefill_to_cache) or start decoding
+ * from nothing.  Enqueued on the stream like every other call; the paper does not discuss this, it is
+ * bookkeeping a serving loop needs around the method.
+ */
+kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stream);
+
 /* lengths [n_seqs, L, H] int32 (device): rows currently held by each list (prefix + window). */
 kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream);
 

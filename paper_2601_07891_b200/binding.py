@@ -64,6 +64,7 @@ SIGNATURES = {
     "kvzap_cache_destroy": (_i32, [_vp]),
     "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "kvzap_decode_attention": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
+    "kvzap_cache_release_seq": (_i32, [_vp, _i32, _vp]),
     "kvzap_cache_lengths": (_i32, [_vp, _vp, _vp]),
     "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
     "kvzap_prefill_to_cache": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
@@ -260,6 +261,10 @@ def kvzap_cache_destroy(cache):
 def kvzap_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None, stream=None):
     _check(handle, load().kvzap_decode_step(handle, cache, layer_begin, layer_end, _ptr(hidden), _ptr(K_new),
                                             _ptr(V_new), tau, _ptr(scores_out), _stream(stream)))
+
+
+def kvzap_cache_release_seq(handle, cache, seq, stream=None):
+    _check(handle, load().kvzap_cache_release_seq(cache, seq, _stream(stream)))
 
 
 def kvzap_cache_lengths(handle, cache, lengths, stream=None):
@@ -519,6 +524,10 @@ class KvzapCache:
             scale = 1.0 / float(self.ctx.head_dim) ** 0.5
         kvzap_decode_attention(self.ctx.handle, self.handle, layer_begin, layer_end, Q, scale, out, stream)
         return out
+
+    def release_seq(self, seq, stream=None):
+        """The sequence in slot `seq` has ended: its lists become empty and its pages are handed out again."""
+        kvzap_cache_release_seq(self.ctx.handle, self.handle, seq, stream)
 
     def lengths(self, stream=None):
         out = torch.empty(self.n_seqs, self.ctx.n_layers, self.ctx.n_kv_heads, dtype=torch.int32, device=self.ctx.device)

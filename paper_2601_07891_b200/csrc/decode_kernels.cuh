@@ -28,7 +28,28 @@ struct CacheView {
     float *score_ring;
     int32_t *n_tokens, *prefix_len, *page_table, *page_cursor;
     uint4 *k_pool, *v_pool;
+    // pages given back by released sequences: a stack; a new page is taken from it before the cursor moves on
+    int32_t *free_stack;      // [n_pages_pool]
+    int32_t *free_top;        // entries on the stack
 };
+
+// One more page for a list: a released one if the stack has any, else the next never-used page of the
+// pool; -1 (and the status word) when neither is left.  Kernels that take pages never release any, so the
+// stack only shrinks while they run: an index handed out by the atomic below is stable.
+__device__ __forceinline__ int32_t cache_take_page(const CacheView &c, int32_t *status)
+{
+    if (__ldcg(c.free_top) > 0) {                       // the usual case, an empty stack, costs one load
+        const int32_t top = atomicSub(c.free_top, 1);
+        if (top > 0) return c.free_stack[top - 1];
+        atomicAdd(c.free_top, 1);                       // someone else took the last one
+    }
+    const int32_t got = atomicAdd(c.page_cursor, 1);
+    if (got >= c.n_pages_pool) {
+        atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+        return -1;
+    }
+    return got;
+}
 
 constexpr int kDecodeThreads = 256;
 constexpr int kDecodeLanes = 8;        // lanes that share one list (a 256-byte row = two 16-byte units per lane)
@@ -94,13 +115,8 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
             if (page_i >= c.max_pages) {
                 atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
             } else if (in_page == 0) {
-                const int32_t got = atomicAdd(c.page_cursor, 1);
-                if (got >= c.n_pages_pool) {
-                    atomicCAS(status, 0, 4);
-                } else {
-                    page = got;
-                    c.page_table[li * c.max_pages + page_i] = got;
-                }
+                page = cache_take_page(c, status);
+                if (page >= 0) c.page_table[li * c.max_pages + page_i] = page;
             } else {
                 page = c.page_table[li * c.max_pages + page_i];
             }
@@ -211,13 +227,16 @@ chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scor
                 const int64_t want = (len + cnt + c.page_tokens - 1) / c.page_tokens;
                 int ok = 1;
                 if (lane == 0 && want > have) {
-                    if (want > c.max_pages) ok = 0;
-                    else {
-                        const int32_t got = atomicAdd(c.page_cursor, static_cast<int32_t>(want - have));
-                        if (static_cast<int64_t>(got) + (want - have) > c.n_pages_pool) ok = 0;
-                        else for (int64_t i = have; i < want; ++i) table[i] = got + static_cast<int32_t>(i - have);
+                    if (want > c.max_pages) {
+                        ok = 0;
+                        atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+                    } else {
+                        for (int64_t i = have; i < want && ok; ++i) {
+                            const int32_t page = cache_take_page(c, status);
+                            if (page < 0) ok = 0;
+                            else table[i] = page;
+                        }
                     }
-                    if (!ok) atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 __syncwarp();
@@ -291,6 +310,26 @@ chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scor
     if (tid == 0) {
         c.prefix_len[li] = static_cast<int32_t>(len_s);
         c.n_tokens[li] = static_cast<int32_t>(n_old + m);
+    }
+}
+
+// A sequence has ended: the pages of all its lists (L x H of them, one warp each) go onto the stack of
+// released pages and the lists become empty.  Runs alone on the stream (it is the one kernel that adds
+// to the stack).
+__global__ void __launch_bounds__(32)
+release_seq_kernel(const CacheView c, int32_t seq)
+{
+    const int64_t li = static_cast<int64_t>(seq) * c.n_layers * c.n_heads + blockIdx.x;
+    const int lane = threadIdx.x;
+    const int32_t n_pages = (c.prefix_len[li] + c.page_tokens - 1) / c.page_tokens;
+    int32_t base = 0;
+    if (lane == 0 && n_pages > 0) base = atomicAdd(c.free_top, n_pages);
+    base = __shfl_sync(0xffffffffu, base, 0);
+    for (int32_t i = lane; i < n_pages; i += 32) c.free_stack[base + i] = c.page_table[li * c.max_pages + i];
+    __syncwarp();
+    if (lane == 0) {
+        c.prefix_len[li] = 0;
+        c.n_tokens[li] = 0;
     }
 }
 

@@ -81,7 +81,6 @@ struct kvzap_ctx {
     size_t last_scores_bytes = 0;
     int32_t *list_page0 = nullptr;   // [max_seqs * H] first page of each list (paged output)
     int32_t *list_base = nullptr;    // [max_seqs * H] appending to lists: rows each list held before
-    int32_t *list_tail = nullptr;    // [max_seqs * H]                     and the page of its last row
     int32_t *status_dev = nullptr;
     int32_t *status_host = nullptr;  // pinned
     int64_t launches = 0;
@@ -257,7 +256,6 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->wide_arrive);
     cudaFree(ctx->list_page0);
     cudaFree(ctx->list_base);
-    cudaFree(ctx->list_tail);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
@@ -607,7 +605,7 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
                                            static_cast<const int32_t *>(nullptr),
                                            tok_major ? int64_t{1} : n_tokens,
                                            tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
-                                           static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr)));
+                                           static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr), 0));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -844,7 +842,6 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaMalloc(&ctx->maskbits, sizeof(uint32_t) * kMaskRing * ctx->max_words * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_page0, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->list_base, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
-    CREATE_CUDA(cudaMalloc(&ctx->list_tail, sizeof(int32_t) * static_cast<int64_t>(c.max_seqs) * c.n_kv_heads));
     CREATE_CUDA(cudaMalloc(&ctx->tile_counters, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMemset(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing));
     CREATE_CUDA(cudaMalloc(&ctx->select_hist, sizeof(uint32_t) * 4 * static_cast<size_t>(c.max_seqs) * c.n_kv_heads * 256));
@@ -1267,7 +1264,7 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
                                                                      tau, w, 1, maskbits, n_words, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
-                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status, 0, nullptr, nullptr);
+                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status, 0, nullptr, nullptr, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(n_kv_heads));
     compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
@@ -1306,7 +1303,8 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                             int32_t *page_table, int32_t max_pages, int32_t *lengths,
                                             int32_t *n_pages_used, cudaStream_t stream,
                                             int32_t *page_cursor = nullptr, bool tok_major = false, bool append = false,
-                                            bool beside_scoring = true)
+                                            bool beside_scoring = true, const int32_t *free_stack = nullptr,
+                                            int32_t *free_top = nullptr)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1322,7 +1320,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            static_cast<int32_t *>(nullptr),
                                            lengths, static_cast<int>(page_tokens), first_page, n_pages_pool,
                                            static_cast<int>(max_pages), ctx->list_page0, page_table, n_pages_used,
-                                           page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, ctx->list_tail));
+                                           page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, free_stack, free_top));
     }
     // the same resident-at-once grid as the dense-ragged output (see launch_compaction)
     const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (!beside_scoring ? 8 : (c.hidden > 0 ? 2 : 6));
@@ -1344,7 +1342,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            tok_major ? int64_t{1} : n_tokens,
                                            tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
                                            static_cast<const int32_t *>(append ? ctx->list_base : nullptr),
-                                           static_cast<const int32_t *>(append ? ctx->list_tail : nullptr)));
+                                           static_cast<const int32_t *>(page_table), static_cast<int>(max_pages)));
     }
     ctx->launches += 2;
     return KVZAP_OK;
@@ -1502,6 +1500,8 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.prefix_len), sizeof(int32_t) * n, true);
     alloc(reinterpret_cast<void **>(&v.page_table), sizeof(int32_t) * n * max_pages_per_list, true);
     alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
+    alloc(reinterpret_cast<void **>(&v.free_stack), sizeof(int32_t) * static_cast<size_t>(n_pages_pool > 0 ? n_pages_pool : 1), false);
+    alloc(reinterpret_cast<void **>(&v.free_top), sizeof(int32_t), true);
     alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * 4 * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
           true);
     cache->steps_done.assign(c.n_layers, 0);
@@ -1531,6 +1531,7 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
     cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
     cudaFree(cache->v.page_cursor); cudaFree(cache->scores); cudaFree(cache->done);
+    cudaFree(cache->v.free_stack); cudaFree(cache->v.free_top);
     cudaFree(cache->attn_scratch); cudaFree(cache->attn_arrive);
     delete cache;
     return KVZAP_OK;
@@ -1683,6 +1684,19 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     return KVZAP_OK;
 }
 
+kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stream_)
+{
+    if (!cache) return KVZAP_ERR_INVALID_ARG;
+    kvzap_ctx *ctx = cache->ctx;
+    if (seq < 0 || seq >= cache->v.n_seqs) return fail(ctx, KVZAP_ERR_INVALID_ARG, "release: seq %d out of range", seq);
+    DeviceGuard guard(ctx->cfg.device);
+    release_seq_kernel<<<static_cast<unsigned>(cache->v.n_layers * cache->v.n_heads), 32, 0,
+                         static_cast<cudaStream_t>(stream_)>>>(cache->v, seq);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
 kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream_)
 {
     if (!cache || !lengths) return KVZAP_ERR_INVALID_ARG;
@@ -1724,6 +1738,7 @@ kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, c
                                     cudaMemcpyDeviceToDevice, stream));
     KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.n_tokens, 0, sizeof(int32_t) * n, stream));
     KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.page_cursor, &next_free_page, sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.free_top, 0, sizeof(int32_t), stream));
     KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
     return KVZAP_OK;
 }
@@ -1764,7 +1779,7 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     ctx->launches += 1;
     return launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
                                    v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
-                                   v.page_cursor, false, true);
+                                   v.page_cursor, false, true, true, v.free_stack, v.free_top);
 }
 
 }  // extern "C"

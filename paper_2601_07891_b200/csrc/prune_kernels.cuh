@@ -105,8 +105,11 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
 // list_page0 = -1 so that the compaction writes nothing.
 // append != 0 (paged only): the lists already hold lengths[] rows in the pages their tables name; the
 // kept rows are added behind them.  lengths becomes old + kept (unchanged on failure), only the pages
-// beyond the old ones are assigned (list_page0 = the first of them, table entries appended), and
-// list_base / list_tail receive the old length and the page that holds the old tail (-1 if none).
+// beyond the old ones are assigned and entered into the table, and list_base receives the old length.
+// With a cursor (a cache's allocator) the new pages are taken from the stack of released pages first
+// (free_stack / free_top, may be nullptr), then from the cursor: the pages of a list are then not
+// consecutive numbers and the compaction finds them through the table; list_page0 is the ordinal of
+// the list's first new page among the pages this call assigns (plus first_page), or -1.
 __global__ void __launch_bounds__(1024)
 scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
             const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens,
@@ -114,7 +117,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
             int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
-            int32_t *__restrict__ list_base, int32_t *__restrict__ list_tail)
+            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top)
 {
     // may be placed before the kernel that writes the mask has finished; waits for it here
     griddep_launch_dependents();
@@ -247,7 +250,13 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         __syncthreads();
     }
     const int32_t used = carry_s;
-    const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + used > n_pages_pool;
+    int32_t n_free = 0;
+    if (page_cursor != nullptr && free_top != nullptr) {
+        n_free = *free_top;
+        if (n_free < 0) n_free = 0;
+    }
+    const int32_t from_stack = used < n_free ? used : n_free;
+    const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + (used - from_stack) > n_pages_pool;
     if (fail) {
         for (int idx = tid; idx < n_lists; idx += 1024) {
             list_page0[idx] = -1;
@@ -259,17 +268,22 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         }
         return;
     }
+    __syncthreads();      // every thread has read the cursor and the stack height
     if (tid == 0) {
         if (n_pages_used != nullptr) *n_pages_used = used;
-        if (page_cursor != nullptr) *page_cursor = first_page + used;
+        if (page_cursor != nullptr) *page_cursor = first_page + used - from_stack;
+        if (from_stack > 0) *free_top = n_free - from_stack;
     }
     __syncthreads();      // list_page0 and lengths of all lists are final
     for (int idx = warp; idx < n_lists; idx += 32) {            // a warp per list
         const int32_t p0 = list_page0[idx];
         const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
         const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
-        if (append && lane == 0) list_tail[idx] = have > 0 ? page_table[static_cast<int64_t>(idx) * max_pages + have - 1] : -1;
-        for (int32_t i = lane; i < need; i += 32) page_table[static_cast<int64_t>(idx) * max_pages + have + i] = p0 + i;
+        for (int32_t i = lane; i < need; i += 32) {
+            const int32_t j = p0 - first_page + i;            // ordinal among the pages assigned by this call
+            page_table[static_cast<int64_t>(idx) * max_pages + have + i] =
+                j < from_stack ? free_stack[n_free - 1 - j] : first_page + (j - from_stack);
+        }
     }
 }
 
@@ -393,11 +407,10 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
                      int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths, int page_tokens,
                      const int32_t *__restrict__ list_page0, int64_t in_stride_h, int64_t in_stride_t,
-                     const int32_t *__restrict__ list_base, const int32_t *__restrict__ list_tail)
+                     const int32_t *__restrict__ list_base, const int32_t *__restrict__ page_table, int max_pages)
 {
-    // list_base != nullptr (paged): list (b,h) already holds list_base[] rows, the last of them in page
-    // list_tail[]; kept rows go behind them, first into that page's free slots, then into the pages
-    // from list_page0 on.
+    // list_base != nullptr (paged): list (b,h) already holds list_base[] rows; kept rows go behind them,
+    // into the pages that page_table [list][max_pages] names (the scan has entered the new ones).
     // Row (h, t) of the inputs starts at row index h * in_stride_h + t * in_stride_t: (n_tokens, 1) for
     // the head-major cache layout [H][T][D], (1, H) for the K/V projection's own output [T][H][D].
     // page_tokens > 0: paged output.  K_out / V_out are the page pools, list (b,h) starts at page
@@ -482,11 +495,13 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                         if (list_base == nullptr) {
                             dst_row[r] = p0 < 0 ? -1 : (static_cast<int64_t>(p0) + n / page_tokens) * page_tokens + n % page_tokens;
                         } else {
-                            const int64_t base = list_base[b * n_heads + h];
-                            const int64_t have = (base + page_tokens - 1) / page_tokens;
-                            const int64_t nn = base + n, q = nn / page_tokens;
-                            const int64_t page = q < have ? list_tail[b * n_heads + h] : p0 + (q - have);
-                            dst_row[r] = p0 < 0 ? -1 : page * page_tokens + nn % page_tokens;
+                            const int64_t nn = list_base[b * n_heads + h] + n;
+                            if (p0 < 0) {
+                                dst_row[r] = -1;
+                            } else {
+                                const int64_t page = __ldcg(page_table + static_cast<int64_t>(b * n_heads + h) * max_pages + nn / page_tokens);
+                                dst_row[r] = page * page_tokens + nn % page_tokens;
+                            }
                         }
                     } else {
                         dst_row[r] = static_cast<int64_t>(h) * n_tokens + s + n;

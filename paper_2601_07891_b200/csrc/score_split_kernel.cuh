@@ -248,9 +248,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         if (page_i >= c.max_pages) {
                             atomicCAS(p.status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
                         } else if (in_page == 0) {
-                            const int32_t got = atomicAdd(c.page_cursor, 1);
-                            if (got >= c.n_pages_pool) atomicCAS(p.status, 0, 4);
-                            else { page = got; c.page_table[li * c.max_pages + page_i] = got; }
+                            page = cache_take_page(c, p.status);
+                            if (page >= 0) c.page_table[li * c.max_pages + page_i] = page;
                         } else {
                             page = page_old;
                         }

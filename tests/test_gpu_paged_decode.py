@@ -311,3 +311,75 @@ def test_chunked_prefill_pool_exhaustion_sets_status(binding):
             assert (lengths <= n_pool // H * P + w).all()
     binding.kvzap_cache_destroy(cache)
     ctx.close()
+
+
+def test_release_seq_hands_its_pages_out_again(binding, oracle):
+    """A sequence ends, its slot takes a new prompt: the pool is sized so that this only fits if the
+    released pages are reused; every list of both slots is compared with the oracle before and after."""
+    d_model, hidden, H, D, L, w, P, tau = 256, 128, 8, 64, 2, 16, 16, float("-inf")       # keep everything: pages = rows / 16
+    ctx = binding.Kvzap(d_model, hidden, H, D, L, max_tokens=512)
+    weights = [_weights(d_model, hidden, H, seed=80 + l) for l in range(L)]
+    for l in range(L):
+        ctx.set_weights(l, *[parity.dev(x) for x in weights[l]])
+    n_pool = 900                                    # 400 + 300 rows first, then 500 more in slot 0: 1216 pages without reuse
+    K_pool = torch.full((n_pool, P, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    V_pool = torch.full_like(K_pool, float("nan"))
+    cache = ctx.create_cache(2, w, P, K_pool, V_pool, 40)
+    decs = [oracle.DecodeOracle(1, L, H, D, w), oracle.DecodeOracle(1, L, H, D, w)]
+    seed = [1000]
+
+    def prefill(slot, chunks):
+        for m in chunks:
+            for l in range(L):
+                seed[0] += 1
+                X = synth.hidden_states(m, d_model, seed=seed[0])
+                K, V = synth.keys_values(H, m, D, seed=seed[0] + 5000)
+                s = cache.prefill(l, slot, parity.dev(X), parity.dev(K), parity.dev(V), tau).cpu().numpy()
+                Kb, Vb = synth.bits(K), synth.bits(V)
+                for t in range(m):
+                    decs[slot].append(0, l, s[t], Kb[:, t], Vb[:, t], tau)
+
+    def decode(n_steps):
+        for _ in range(n_steps):
+            seed[0] += 1
+            X = synth.hidden_states(L * 2, d_model, seed=seed[0]).view(L, 2, d_model)
+            Kn, Vn = synth.keys_values(L * 2, H, D, seed=seed[0] + 5000)
+            Kn, Vn = Kn.view(L, 2, H, D), Vn.view(L, 2, H, D)
+            sc = torch.empty(L, 2, H, dtype=torch.float32, device="cuda")
+            cache.decode_step(0, L, parity.dev(X), parity.dev(Kn), parity.dev(Vn), tau, sc)
+            s = sc.cpu().numpy()
+            for l in range(L):
+                for slot in range(2):
+                    decs[slot].append(0, l, s[l, slot], synth.bits(Kn)[l, slot], synth.bits(Vn)[l, slot], tau)
+
+    def check():
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        for slot in range(2):
+            for l in range(L):
+                for h in range(H):
+                    _pos, Kd, Vd = decs[slot].logical(0, l, h)
+                    Kg, Vg, n = _export(binding, ctx, cache.handle, slot, l, h, 700, D)
+                    assert n == len(Kd)
+                    np.testing.assert_array_equal(Kg, Kd)
+                    np.testing.assert_array_equal(Vg, Vd)
+
+    prefill(0, [250, 150])
+    prefill(1, [300])
+    decode(5)
+    check()
+    cache.release_seq(0)
+    decs[0] = oracle.DecodeOracle(1, L, H, D, w)
+    ln = cache.lengths().cpu().numpy()
+    assert (ln[0] == 0).all() and (ln[1] == 305).all()
+    prefill(0, [200, 300])                           # needs the released pages
+    decode(7)
+    check()
+    # and once more, to see pages go round a second time
+    cache.release_seq(1)
+    decs[1] = oracle.DecodeOracle(1, L, H, D, w)
+    prefill(1, [120])
+    decode(20)                                       # single pages taken by decode steps from the stack as well
+    check()
+    cache.close()
+    ctx.close()
