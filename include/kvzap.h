@@ -324,8 +324,9 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
 /*
  * A sequence has ended: all lists (seq, *, *) become empty and their pages go back to the cache's
  * allocator, which hands released pages out again (to any list) before it touches never-used pages
- * of the pool.  The slot `seq` can then take a new prompt (kvzap_prefill_to_cache) or start decoding
- * from nothing.  Enqueued on the stream like every other call; the paper does not discuss this, it is
+ * of the pool.  Until the slot is given a new prompt (kvzap_prefill_to_cache) decode steps leave its
+ * lists alone (its rows of hidden, K_new, V_new are ignored, its scores still computed) and attention over
+ * it gives zeros.  Enqueued on the stream like every other call; the paper does not discuss this, it is
  * bookkeeping a serving loop needs around the method.
  */
 kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stream);

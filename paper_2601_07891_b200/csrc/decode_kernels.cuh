@@ -31,6 +31,9 @@ struct CacheView {
     // pages given back by released sequences: a stack; a new page is taken from it before the cursor moves on
     int32_t *free_stack;      // [n_pages_pool]
     int32_t *free_top;        // entries on the stack
+    // 0 for a slot whose sequence has been released and that has not been given a new prompt: decode steps
+    // leave its lists alone
+    uint8_t *active;          // [n_seqs]
 };
 
 // One more page for a list: a released one if the stack has any, else the next never-used page of the
@@ -78,15 +81,16 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
     const int64_t n_iter = (n_groups + stride - 1) / stride;       // the same for every thread
     for (int64_t it = 0; it < n_iter; ++it) {
         const int64_t group = group0 + it * stride;
-        const bool live = group < n_groups;
+        const bool in_range = group < n_groups;
         // every lane of the warp runs the whole body (the shuffles below need all 32 lanes)
-        const int64_t g = live ? group : 0;
+        const int64_t g = in_range ? group : 0;
         const int l_rel = static_cast<int>(g / (static_cast<int64_t>(c.n_seqs) * c.n_heads));
         const int rem = static_cast<int>(g - static_cast<int64_t>(l_rel) * c.n_seqs * c.n_heads);
         const int b = rem / c.n_heads, h = rem % c.n_heads;
         const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
         const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
         const int32_t n = c.n_tokens[li];
+        const bool live = in_range && c.active[b] != 0;
 
         // which row (if any) moves to the prefix now
         bool append = false;
@@ -167,6 +171,7 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
                 const int b = rem / c.n_heads, h = rem % c.n_heads;
                 const int64_t li = (static_cast<int64_t>(b) * c.n_layers + layer0 + l_rel) * c.n_heads + h;
                 const int64_t src_row = (static_cast<int64_t>(l_rel) * c.n_seqs + b) * c.n_heads + h;
+                if (c.active[b] == 0) continue;
                 const int slot = (c.n_tokens[li] - 1) % c.window;      // the slot this thread filled above
                 c.score_ring[li * c.window + slot] = __ldcg(scores + src_row);
             }
@@ -310,6 +315,7 @@ chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scor
     if (tid == 0) {
         c.prefix_len[li] = static_cast<int32_t>(len_s);
         c.n_tokens[li] = static_cast<int32_t>(n_old + m);
+        if (h == 0) c.active[li / (static_cast<int64_t>(c.n_layers) * c.n_heads)] = 1;     // the slot holds a sequence again
     }
 }
 
@@ -330,6 +336,7 @@ release_seq_kernel(const CacheView c, int32_t seq)
     if (lane == 0) {
         c.prefix_len[li] = 0;
         c.n_tokens[li] = 0;
+        if (blockIdx.x == 0) c.active[seq] = 0;
     }
 }
 
@@ -337,6 +344,7 @@ release_seq_kernel(const CacheView c, int32_t seq)
 __global__ void tokens_add_kernel(const CacheView c, int64_t li0, int64_t m)
 {
     if (threadIdx.x < c.n_heads) c.n_tokens[li0 + threadIdx.x] += static_cast<int32_t>(m);
+    if (threadIdx.x == 0) c.active[li0 / (static_cast<int64_t>(c.n_layers) * c.n_heads)] = 1;
 }
 
 // lengths[li] = prefix_len + min(n_tokens, w)

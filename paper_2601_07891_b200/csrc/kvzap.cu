@@ -1502,6 +1502,8 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.page_cursor), sizeof(int32_t), true);
     alloc(reinterpret_cast<void **>(&v.free_stack), sizeof(int32_t) * static_cast<size_t>(n_pages_pool > 0 ? n_pages_pool : 1), false);
     alloc(reinterpret_cast<void **>(&v.free_top), sizeof(int32_t), true);
+    alloc(reinterpret_cast<void **>(&v.active), static_cast<size_t>(n_seqs), false);
+    if (e == cudaSuccess) e = cudaMemset(v.active, 1, static_cast<size_t>(n_seqs));      // every slot takes part until released
     alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * 4 * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
           true);
     cache->steps_done.assign(c.n_layers, 0);
@@ -1531,7 +1533,7 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
     cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
     cudaFree(cache->v.page_cursor); cudaFree(cache->scores); cudaFree(cache->done);
-    cudaFree(cache->v.free_stack); cudaFree(cache->v.free_top);
+    cudaFree(cache->v.free_stack); cudaFree(cache->v.free_top); cudaFree(cache->v.active);
     cudaFree(cache->attn_scratch); cudaFree(cache->attn_arrive);
     delete cache;
     return KVZAP_OK;
@@ -1739,6 +1741,7 @@ kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, c
     KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.n_tokens, 0, sizeof(int32_t) * n, stream));
     KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.page_cursor, &next_free_page, sizeof(int32_t), cudaMemcpyHostToDevice, stream));
     KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.free_top, 0, sizeof(int32_t), stream));
+    KVZAP_CUDA(ctx, cudaMemsetAsync(cache->v.active, 1, static_cast<size_t>(cache->v.n_seqs), stream));
     KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
     return KVZAP_OK;
 }

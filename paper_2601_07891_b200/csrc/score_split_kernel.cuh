@@ -230,7 +230,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 const int b_loc = pos * rows_per_cta + etid / kMaxHeads, h = etid % kMaxHeads;
                 const int64_t b = static_cast<int64_t>(m_tile) * kTileM + b_loc;
                 int64_t dst = -1, ring = -1;
-                if (go && etid < rows_per_cta * kMaxHeads && b < c.n_seqs && h < c.n_heads) {
+                if (go && etid < rows_per_cta * kMaxHeads && b < c.n_seqs && h < c.n_heads && c.active[b] != 0) {
                     const int64_t li = (b * c.n_layers + layer) * c.n_heads + h;
                     // two round trips to memory instead of four: both counters first, then the score of
                     // the slot's old token and the page the prefix ends in, whether or not it will be needed
@@ -471,7 +471,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             if (valid && *abort_flag == 0) {
 #pragma unroll
                 for (int h = 0; h < kMaxHeads; ++h) {
-                    if (h < c.n_heads) {
+                    if (h < c.n_heads && c.active[t] != 0) {
                         const int64_t li = (t * c.n_layers + layer) * c.n_heads + h;
                         const int slot = (__ldcg(c.n_tokens + li) - 1) % c.window;
                         c.score_ring[li * c.window + slot] = s[h];

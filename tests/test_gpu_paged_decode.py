@@ -339,7 +339,7 @@ def test_release_seq_hands_its_pages_out_again(binding, oracle):
                 for t in range(m):
                     decs[slot].append(0, l, s[t], Kb[:, t], Vb[:, t], tau)
 
-    def decode(n_steps):
+    def decode(n_steps, slots=(0, 1)):
         for _ in range(n_steps):
             seed[0] += 1
             X = synth.hidden_states(L * 2, d_model, seed=seed[0]).view(L, 2, d_model)
@@ -349,7 +349,7 @@ def test_release_seq_hands_its_pages_out_again(binding, oracle):
             cache.decode_step(0, L, parity.dev(X), parity.dev(Kn), parity.dev(Vn), tau, sc)
             s = sc.cpu().numpy()
             for l in range(L):
-                for slot in range(2):
+                for slot in slots:
                     decs[slot].append(0, l, s[l, slot], synth.bits(Kn)[l, slot], synth.bits(Vn)[l, slot], tau)
 
     def check():
@@ -372,7 +372,11 @@ def test_release_seq_hands_its_pages_out_again(binding, oracle):
     decs[0] = oracle.DecodeOracle(1, L, H, D, w)
     ln = cache.lengths().cpu().numpy()
     assert (ln[0] == 0).all() and (ln[1] == 305).all()
-    prefill(0, [200, 300])                           # needs the released pages
+    decode(3, slots=(1,))                            # the released slot takes no part in decode steps
+    ln = cache.lengths().cpu().numpy()
+    assert (ln[0] == 0).all() and (ln[1] == 308).all()
+    check()
+    prefill(0, [200, 300])                           # needs the released pages; the slot takes part again
     decode(7)
     check()
     # and once more, to see pages go round a second time
