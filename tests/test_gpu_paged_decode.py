@@ -313,10 +313,11 @@ def test_chunked_prefill_pool_exhaustion_sets_status(binding):
     ctx.close()
 
 
-def test_release_seq_hands_its_pages_out_again(binding, oracle):
+@pytest.mark.parametrize("hidden", [128, 0])        # the one-launch decode step, and the scoring + update pair of launches
+def test_release_seq_hands_its_pages_out_again(binding, oracle, hidden):
     """A sequence ends, its slot takes a new prompt: the pool is sized so that this only fits if the
     released pages are reused; every list of both slots is compared with the oracle before and after."""
-    d_model, hidden, H, D, L, w, P, tau = 256, 128, 8, 64, 2, 16, 16, float("-inf")       # keep everything: pages = rows / 16
+    d_model, H, D, L, w, P, tau = 256, 8, 64, 2, 16, 16, float("-inf")       # keep everything: pages = rows / 16
     ctx = binding.Kvzap(d_model, hidden, H, D, L, max_tokens=512)
     weights = [_weights(d_model, hidden, H, seed=80 + l) for l in range(L)]
     for l in range(L):
