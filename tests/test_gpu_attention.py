@@ -97,7 +97,7 @@ def test_attention_after_decode_steps(binding, oracle, hidden, w, P, B, L, D, G)
     ctx.close()
 
 
-@pytest.mark.parametrize("T0,w,D", [(1500, 128, 128), (700, 16, 64)])
+@pytest.mark.parametrize("T0,w,D", [(1500, 128, 128), (700, 16, 64), (900, 256, 128)])
 def test_attention_after_prefill_to_cache(binding, oracle, T0, w, D):
     """Long lists: many tiles per warp, so every pipeline stage is reused several times."""
     d_model, hidden, H, tau, P, G, k = 256, 128, 8, 0.0, 16, 4, 5

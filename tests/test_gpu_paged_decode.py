@@ -230,7 +230,7 @@ def test_decode_pool_exhaustion_sets_status(binding):
 
 
 @pytest.mark.parametrize("chunks,w,P", [([300, 5, 200, 17, 129], 16, 8), ([100, 100, 100], 128, 16), ([64, 1, 1, 300], 0, 4),
-                                        ([3, 2, 700, 40], 32, 16)])
+                                        ([3, 2, 700, 40], 32, 16), ([300, 700, 50, 290], 256, 16)])
 def test_chunked_prefill_equals_one_prefill(binding, oracle, chunks, w, P):
     """Prefill in chunks of any lengths (then a few decode steps) == prefill of the whole sequence:
     the score buffer carries the window across chunk boundaries."""
