@@ -992,18 +992,27 @@ kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void 
     const int n_sel = per_layer ? 1 : c.n_kv_heads;
     KVZAP_CUDA(ctx, cudaMemsetAsync(ctx->select_hist, 0, sizeof(uint32_t) * 4 * static_cast<size_t>(n_seqs) * n_sel * 256, stream));
     const dim3 grid(static_cast<unsigned>((n_tokens + kSelectThreads - 1) / kSelectThreads), static_cast<unsigned>(n_seqs));
-    for (int pass = 0; pass < 4; ++pass)
-        select_hist_kernel<<<grid, kSelectThreads, 0, stream>>>(scores, n_tokens, c.n_kv_heads, cu_seqlens, n_seqs, w,
-                                                                keep_ratio, per_layer ? 1 : 0, pass, ctx->select_hist);
-    select_finish_kernel<<<static_cast<unsigned>(n_seqs), kSelectThreads, 0, stream>>>(
-        n_tokens, c.n_kv_heads, cu_seqlens, n_seqs, w, keep_ratio, per_layer ? 1 : 0, ctx->select_hist, tau_list,
-        ctx->status_dev);
+    const bool early = !ctx->profiling;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attrs[2];
+    for (int pass = 0; pass < 4; ++pass) {
+        make_launch(&cfg, attrs, grid, dim3(kSelectThreads), 0, stream, early, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, select_hist_kernel, scores, n_tokens, static_cast<int>(c.n_kv_heads), cu_seqlens,
+                                           static_cast<int>(n_seqs), static_cast<int>(w), keep_ratio, per_layer ? 1 : 0, pass,
+                                           ctx->select_hist));
+    }
+    make_launch(&cfg, attrs, dim3(static_cast<unsigned>(n_seqs)), dim3(kSelectThreads), 0, stream, early, 1);
+    KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, select_finish_kernel, n_tokens, static_cast<int>(c.n_kv_heads), cu_seqlens,
+                                       static_cast<int>(n_seqs), static_cast<int>(w), keep_ratio, per_layer ? 1 : 0,
+                                       static_cast<const uint32_t *>(ctx->select_hist), tau_list, ctx->status_dev));
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
     uint32_t *mask = next_mask_slice(ctx);
     {
         ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
-        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, c.n_kv_heads, cu_seqlens, n_seqs,
-                                                                         0.0f, w, 1, mask, n_blocks * 4, tau_list);
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(n_blocks)), dim3(128), 0, stream, early, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, mask_kernel, scores, n_tokens, static_cast<int>(c.n_kv_heads), cu_seqlens,
+                                           static_cast<int>(n_seqs), 0.0f, static_cast<int>(w), 1, mask, n_blocks * 4,
+                                           static_cast<const float *>(tau_list)));
     }
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 6;

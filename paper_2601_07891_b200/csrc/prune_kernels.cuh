@@ -31,6 +31,9 @@ mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
             const int32_t *__restrict__ cu_seqlens, int n_seqs, float tau, int window, int window_keep,
             uint32_t *__restrict__ maskbits, int64_t n_words, const float *__restrict__ tau_list)
 {
+    // may be queued with early start behind the kernels that produce the per-list thresholds
+    griddep_launch_dependents();
+    griddep_wait();
     const int lane = threadIdx.x & 31;
     const int64_t word = static_cast<int64_t>(blockIdx.x) * 4 + (threadIdx.x >> 5);
     const int64_t t = word * 32 + lane;
@@ -62,7 +65,7 @@ mask_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_heads,
             // thresholds written by the kernel ahead in the stream: plain loads
 #pragma unroll
             for (int h = 0; h < kMaxHeads; ++h)
-                if (h < n_heads) tau_h[h] = tau_list[b * n_heads + h];
+                if (h < n_heads) tau_h[h] = __ldcg(tau_list + b * n_heads + h);
         }
     }
     uint32_t my_word = 0;

@@ -101,6 +101,10 @@ select_hist_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_hea
     __shared__ uint32_t sh[kMaxHeads][256];
     __shared__ uint32_t s_prefix[kMaxHeads];
     __shared__ int s_dead[kMaxHeads];
+    // the launches of one selection are queued with early start: each lets the next be placed at once and
+    // waits here, every thread, for the one ahead (its histograms, or the scores) to be complete
+    griddep_launch_dependents();
+    griddep_wait();
     const int b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t t0 = cu_seqlens ? cu_seqlens[b] : 0, t1 = cu_seqlens ? cu_seqlens[b + 1] : n_tokens;
     const int64_t n_cand = t1 - t0 - window > 0 ? t1 - t0 - window : 0;
@@ -121,7 +125,7 @@ select_hist_kernel(const float *__restrict__ scores, int64_t n_tokens, int n_hea
         const float *row = scores + (t0 + c0 + tid) * n_heads;
         for (int h = 0; h < n_heads; ++h) {
             const int hs = per_layer ? 0 : h;
-            const float v = __ldg(row + h);
+            const float v = __ldcg(row + h);
             if (s_dead[hs] || v != v) continue;
             const uint32_t key = score_key(v);
             if (pass == 0 || (key >> (32 - 8 * pass)) == s_prefix[hs])
@@ -142,6 +146,8 @@ select_finish_kernel(int64_t n_tokens, int n_heads, const int32_t *__restrict__ 
                      float keep_ratio, int per_layer, const uint32_t *__restrict__ hist, float *__restrict__ tau_list,
                      int32_t *__restrict__ status)
 {
+    griddep_launch_dependents();
+    griddep_wait();
     const int b = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t t0 = cu_seqlens ? cu_seqlens[b] : 0, t1 = cu_seqlens ? cu_seqlens[b + 1] : n_tokens;
     const int64_t n_cand = t1 - t0 - window > 0 ? t1 - t0 - window : 0;
