@@ -143,3 +143,37 @@ def test_planted_mistake_fails_a_pin(build_dir, name, pins, old, new):
             pytest.skip("widening helper is written differently")
     mod = _load_variant(build_dir, name, old, new)
     assert _failures(mod, pins), "no pin noticed the planted mistake '%s'" % name
+
+
+# ---------------------------------------------------------------------------
+# The decode oracle is Python: mistakes are planted by replacing one line of its source text.
+
+DECODE_MUTANTS = [
+    ("decode_window_one_too_long", "            if len(win) > self.w:", "            if len(win) > self.w + 1:"),
+    ("decode_strict_compare", "                if s >= tau32:          # NaN compares false -> dropped", "                if s > tau32:"),
+    ("decode_judges_the_new_score", "                if s >= tau32:          # NaN compares false -> dropped",
+     "                if np.float32(scores_h[h]) >= tau32:"),
+    ("decode_newest_leaves_first", "                p, s, kr, vr = win.popleft()", "                p, s, kr, vr = win.pop()"),
+    ("decode_shared_heads", "            win = self.window[b][l][h]", "            win = self.window[b][l][0]"),
+]
+
+
+def _load_python_variant(name, old, new):
+    path = os.path.join(_ORACLE_DIR, "kvzap_oracle.py")
+    src = open(path).read()
+    assert src.count(old) == 1, "mutation site not found exactly once: %r" % old
+    src = src.replace(old, new)
+    spec = importlib.util.spec_from_file_location("kvzap_oracle_" + name, path)
+    mod = importlib.util.module_from_spec(spec)
+    exec(compile(src, path, "exec"), mod.__dict__)
+    return mod
+
+
+DECODE_PINS = [p for p in PRUNE if "decode" in p[0] or "prefill_then" in p[0] or "score_buffer" in p[0]]
+
+
+@pytest.mark.parametrize("name,old,new", DECODE_MUTANTS, ids=[m[0] for m in DECODE_MUTANTS])
+def test_planted_mistake_in_the_decode_oracle_fails_a_pin(name, old, new):
+    assert len(DECODE_PINS) >= 3
+    mod = _load_python_variant(name, old, new)
+    assert _failures(mod, DECODE_PINS), "no pin noticed the planted mistake '%s'" % name
