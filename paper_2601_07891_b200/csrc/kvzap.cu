@@ -421,7 +421,11 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             f.enabled = 1;
             if (fused) *fused = true;
         }
-        const bool early = fuse_ok && !clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count;
+        // The fused decode step touches the cache before it has waited for the kernel ahead (its clusters
+        // order themselves through `done`), so it is started early only with a grid of at least half the
+        // SMs and its own scores buffer.  Without the fused part the kernel reads nothing but hidden states
+        // and weights until every thread has waited, and writes only after: it may always start early.
+        const bool early = !ctx->profiling && (fuse_ok ? (!clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count) : true);
         ctx->last_score_early = early;
         {
             ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
