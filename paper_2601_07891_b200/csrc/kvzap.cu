@@ -412,7 +412,6 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         ctx->last_scores = scores;
         ctx->last_scores_bytes = sbytes;
         const int n_ctas = split_n * split_k;
-        // only the fused decode step is started early: its clusters order themselves through `done`
         DecodeFuse f;
         memset(&f, 0, sizeof f);
         const bool fuse_ok = fuse != nullptr && !ctx->profiling && n_ctas == 4;
