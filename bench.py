@@ -504,6 +504,37 @@ def run_decode(args, wl, env):
             "gpu_launches": int(gpu_launches), "roofline": roofline,
             "breakdown": {"layer_us": ms_per_step * 1e3 / L, "layer_roofline_us": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
                           "kept_fraction_of_exiting_tokens": kept_exit}}
+    if rank == 0 and world == 1 and not args.skip_e2e:
+        # End to end: the step's inputs start in pinned host memory and its scores end there; the copies
+        # (torch, on the stream of the call) are inside the timed region.
+        hX = [x.cpu().pin_memory() for x in Xs[:2]]
+        hK = [kv[0].cpu().pin_memory() for kv in KVs[:2]]
+        hV = [kv[1].cpu().pin_memory() for kv in KVs[:2]]
+        hS = [torch.empty(L, B, H, dtype=torch.float32).pin_memory() for _ in range(2)]
+        dX, dK, dV = torch.empty_like(Xs[0]), torch.empty_like(KVs[0][0]), torch.empty_like(KVs[0][1])
+        dS = torch.empty(L, B, H, dtype=torch.float32, device=dev)
+
+        def e2e_step(i):
+            dX.copy_(hX[i % 2], non_blocking=True)
+            dK.copy_(hK[i % 2], non_blocking=True)
+            dV.copy_(hV[i % 2], non_blocking=True)
+            binding.kvzap_decode_step(ctx.handle, cache, 0, L, dX, dK.view(L, B, H, D), dV.view(L, B, H, D), wl.tau, dS)
+            hS[i % 2].copy_(dS, non_blocking=True)
+
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        n_e2e = max(args.e2e_steps, 10)
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        e2e_ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        h2d = hX[0].numel() * 2 + hK[0].numel() * 2 + hV[0].numel() * 2
+        line["e2e"] = {"value": B / (e2e_ms * 1e-3 / L), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                       "d2h_bytes_per_step": int(hS[0].numel() * 4), "ms_per_step": e2e_ms, "steps": n_e2e,
+                       "note": "kvzap_decode_step with the step's hidden states and new K/V rows copied from pinned host "
+                               "memory and the scores copied back, inside the timed region"}
     binding.kvzap_cache_destroy(cache)
     ctx.close()
     return line
