@@ -121,6 +121,27 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         prefetch_tensormap(&tmap_x);
         prefetch_tensormap(&tmap_w);
     }
+    const int k_blocks = p.d_model / kBlockK / k_split;  // K blocks of this CTA
+    const int kb_first = kh * k_blocks;
+    const uint64_t pol_x = l2_policy_evict_last();        // the other CTAs of the cluster read the same X tile
+    const uint64_t pol_w = l2_policy_evict_first();       // every W1 byte is read once per step
+    const int w_row = layer * p.w_rows + nh * ns;
+    const int row0 = m_tile * kTileM;
+    const int n_pre = k_blocks < p.n_stages ? k_blocks : p.n_stages;
+    if (warp == 0) {
+        // The first loads go out before the CTA-wide barrier below (TMEM allocation, the other warps): the
+        // stages are empty and their barriers were initialised by this warp's lane 0 just above.
+        __syncwarp();
+        if (elect_one()) {
+            for (int kb = 0; kb < n_pre; ++kb) {
+                const uint32_t sa = smem_base + kb * L.stage_bytes;
+                mbar_arrive_expect_tx(bar_full + 8 * kb, L.stage_bytes);
+                tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * kb, 0, w_row, kb_first + kb, pol_w);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * kb, (kb_first + kb) * kBlockK, row0, l_rel, pol_x);
+            }
+        }
+        __syncwarp();
+    }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), static_cast<uint32_t>(p.tmem_cols));
         tmem_relinquish();
@@ -129,19 +150,15 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int k_blocks = p.d_model / kBlockK / k_split;  // K blocks of this CTA
-    const int kb_first = kh * k_blocks;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
-        const uint64_t pol_x = l2_policy_evict_last();    // the other CTAs of the cluster read the same X tile
-        const uint64_t pol_w = l2_policy_evict_first();   // every W1 byte is read once per step
+        // ------------------------------------------------------------ TMA producer (from the stage after those)
         const bool elected = elect_one();
-        const int w_row = layer * p.w_rows + nh * ns;
-        const int row0 = m_tile * kTileM;
-        uint32_t st = 0, st_par = 1, sa = smem_base;
+        uint32_t st = n_pre == p.n_stages ? 0u : static_cast<uint32_t>(n_pre);
+        uint32_t st_par = n_pre == p.n_stages ? 0u : 1u;
+        uint32_t sa = smem_base + st * L.stage_bytes;
         bool ok = true;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = n_pre; kb < k_blocks; ++kb) {
             if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
                 ok = false;
                 break;
