@@ -30,7 +30,7 @@ UNIT = "tokens/s/layer"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (bytes); None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 276.8e6, "qwen3_8b_decode_b128": 227.1e6}
+NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 276.8e6, "qwen3_8b_decode_b128": 227.9e6}
 # attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
 NCU_ATTENTION_TRAFFIC_RATIO = 2.408 / 2.3986
 
