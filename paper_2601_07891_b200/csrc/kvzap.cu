@@ -1672,12 +1672,24 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     const int64_t n_lists_call = static_cast<int64_t>(p.n_layers_call) * v.n_seqs * v.n_heads;
     if (n_lists_call > 0x7fffffffLL) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: too many lists for one launch");
     // Two CTAs fit an SM.  With fewer than eight CTAs per slot the last, longest lists leave most SMs
-    // idle: cut every list into up to 16 parts so that there are about that many units.
+    // idle: cut every list into parts so that there are about that many units -- up to 16 parts, or up
+    // to 64 when a handful of long lists (a single sequence) is all there is, but never parts shorter
+    // than about a thousand rows of the longest list the cache can hold.
     p.n_parts = 1;
     const int64_t want_units = static_cast<int64_t>(ctx->sm_count) * 16;
     if (n_lists_call * 2 <= want_units) {
         int64_t parts = want_units / n_lists_call;
-        if (parts > 16) parts = 16;
+        const int64_t cap = n_lists_call * 16 < 2 * static_cast<int64_t>(ctx->sm_count) ? 64 : 16;
+        if (parts > cap) parts = cap;
+        const int64_t max_rows = static_cast<int64_t>(v.max_pages) * v.page_tokens + v.window;
+        if (parts > 16 && parts > (max_rows + 1023) / 1024) parts = (max_rows + 1023) / 1024 > 16 ? (max_rows + 1023) / 1024 : 16;
+        // fewer lists than resident CTA slots: one full wave of equal parts (a second, partly filled wave
+        // would cost as much as the first)
+        const int64_t slots = 2 * static_cast<int64_t>(ctx->sm_count);
+        if (n_lists_call < slots) {
+            parts = slots / n_lists_call;
+            if (parts > 64) parts = 64;
+        }
         if (parts * n_lists_call > cache->attn_units) parts = cache->attn_units / n_lists_call;
         if (parts > 1) p.n_parts = static_cast<int32_t>(parts);
     }
