@@ -307,18 +307,34 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     __syncthreads();
     if (!last_s) return;
     const float *units = p.part_scratch + static_cast<int64_t>(list) * p.n_parts * (16 + kAttnMaxGroup * kD);
+    constexpr int kBatch = 8;               // parts whose values are loaded together (independent loads in flight)
+    constexpr int kUnit = 16 + kAttnMaxGroup * kD;
     for (int idx = threadIdx.x; idx < p.group * kD; idx += kAttnThreads) {
         const int gq = idx / kD, d = idx % kD;
         float m_all = -INFINITY;
-        for (int i = 0; i < p.n_parts; ++i) m_all = fmaxf(m_all, __ldcg(units + i * (16 + kAttnMaxGroup * kD) + gq));
+        for (int i0 = 0; i0 < p.n_parts; i0 += kBatch) {
+            float mv[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) mv[j] = i0 + j < p.n_parts ? __ldcg(units + (i0 + j) * kUnit + gq) : -INFINITY;
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) m_all = fmaxf(m_all, mv[j]);
+        }
         float num = 0.0f, den = 0.0f;
-        for (int i = 0; i < p.n_parts; ++i) {
-            const float *u = units + i * (16 + kAttnMaxGroup * kD);
-            const float m_i = __ldcg(u + gq);
-            if (m_i > -INFINITY) {
-                const float f = fast_ex2(m_i - m_all);
-                num += __ldcg(u + 16 + gq * kD + d) * f;
-                den += __ldcg(u + 8 + gq) * f;
+        for (int i0 = 0; i0 < p.n_parts; i0 += kBatch) {
+            float mv[kBatch], nv[kBatch], dv[kBatch];
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                const bool in = i0 + j < p.n_parts;
+                const float *u = units + (i0 + j) * kUnit;
+                mv[j] = in ? __ldcg(u + gq) : -INFINITY;
+                nv[j] = in ? __ldcg(u + 16 + gq * kD + d) : 0.0f;      // a part without tiles stored zeros
+                dv[j] = in ? __ldcg(u + 8 + gq) : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {                          // summed in part order
+                const float f = mv[j] > -INFINITY ? fast_ex2(mv[j] - m_all) : 0.0f;
+                num += nv[j] * f;
+                den += dv[j] * f;
             }
         }
         const float r = den > 0.0f ? num / den : 0.0f;
