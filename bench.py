@@ -32,7 +32,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # capture summarised under profiles/ (bytes); None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 276.8e6, "qwen3_8b_decode_b128": 227.9e6}
 # attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
-NCU_ATTENTION_TRAFFIC_RATIO = 2.408 / 2.3986
+NCU_ATTENTION_TRAFFIC_RATIO = 2.409 / 2.3986
 
 
 def load_peaks():
