@@ -1522,8 +1522,8 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     // two halves used by alternate steps when the caller does not ask for the scores
     alloc(reinterpret_cast<void **>(&cache->scores), 2 * sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
           false);
-    // attention: calls with few lists cut each list into parts; room for 16 units per SM
-    cache->attn_units = static_cast<int64_t>(ctx->sm_count) * 16;
+    // attention: calls with few lists cut each list into parts; room for 32 units per SM
+    cache->attn_units = static_cast<int64_t>(ctx->sm_count) * 32;
     alloc(reinterpret_cast<void **>(&cache->attn_scratch),
           sizeof(float) * static_cast<size_t>(cache->attn_units) * (16 + kAttnMaxGroup * 128), false);
     alloc(reinterpret_cast<void **>(&cache->attn_arrive), sizeof(uint32_t) * static_cast<size_t>(cache->attn_units), true);
@@ -1671,12 +1671,12 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     p.status = ctx->status_dev;
     const int64_t n_lists_call = static_cast<int64_t>(p.n_layers_call) * v.n_seqs * v.n_heads;
     if (n_lists_call > 0x7fffffffLL) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "attention: too many lists for one launch");
-    // Two CTAs fit an SM.  With fewer than eight CTAs per slot the last, longest lists leave most SMs
+    // Two CTAs fit an SM.  With fewer than sixteen CTAs per slot the last, longest lists leave most SMs
     // idle: cut every list into parts so that there are about that many units -- up to 16 parts, or up
     // to 64 when a handful of long lists (a single sequence) is all there is, but never parts shorter
     // than about a thousand rows of the longest list the cache can hold.
     p.n_parts = 1;
-    const int64_t want_units = static_cast<int64_t>(ctx->sm_count) * 16;
+    const int64_t want_units = static_cast<int64_t>(ctx->sm_count) * 32;
     if (n_lists_call * 2 <= want_units) {
         int64_t parts = want_units / n_lists_call;
         const int64_t cap = n_lists_call * 16 < 2 * static_cast<int64_t>(ctx->sm_count) ? 64 : 16;

@@ -168,18 +168,18 @@ def test_attention_empty_cache_and_argument_errors(binding):
     ctx.close()
 
 
-@pytest.mark.parametrize("B", [128, 160])
-def test_attention_at_bench_size_sampled_lists(binding, oracle, B):
+@pytest.mark.parametrize("B,lo,hi", [(128, 1000, 8000), (300, 200, 2000)])
+def test_attention_at_bench_size_sampled_lists(binding, oracle, B, lo, hi):
     """128 sequences x 8 KV heads with lists of 1k..8k pruned rows plus a full window of 128, the
     launch shape bench.py --attention times (one layer): sampled lists against the oracle.
-    With 128 sequences every list is cut into two parts, with 160 each list is one CTA."""
+    With 128 sequences every list is cut into parts, with 300 (2400 lists) each list is one CTA."""
     d_model, H, D, P, w, G = 256, 8, 128, 16, 128, 4
     ctx = binding.Kvzap(d_model, 0, H, D, 1, max_tokens=B)
     W, bias = synth.linear_weights(d_model, H, 3)
     ctx.set_weights(0, parity.dev(W), parity.dev(bias))
     n_lists = B * H
     rng = np.random.default_rng(99)
-    prefix = rng.integers(1000, 8001, size=n_lists).astype(np.int32)
+    prefix = rng.integers(lo, hi + 1, size=n_lists).astype(np.int32)
     prefix[:4] = [1, 15, 16, 17]                      # ragged first tiles
     pages_of = (prefix + P - 1) // P
     first = np.concatenate([[0], np.cumsum(pages_of)[:-1]]).astype(np.int64)
