@@ -216,7 +216,7 @@ def run_prefill(args, wl, env):
     n_tokens = B * T
     H, D, P = wl.n_kv_heads, wl.head_dim, wl.page_tokens
     proj = args.kv_layout == "proj"
-    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=dev.index)
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=dev.index, trusted_producers=True)
     cu = torch.from_numpy(synth.cu_seqlens([T] * B)).to(dev) if B > 1 else None
 
     # resident inputs, one set per layer while they fit (every layer's inputs exceed L2, so no flush is
@@ -415,7 +415,7 @@ def run_decode(args, wl, env):
     L, B, H, D, w, P = wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     if args.layers > 0:
         L = min(L, args.layers)
-    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index)
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index, trusted_producers=True)
     for l in range(L):
         ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
     n_lists = B * L * H
@@ -551,7 +551,7 @@ def run_attention(args, wl, env):
     B, H, D, w, P = wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     L = args.layers if args.layers > 0 else 4
     G = 4                                             # 32 query heads over 8 KV heads
-    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index)
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index, trusted_producers=True)
     for l in range(L):
         ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
     n_lists = B * L * H

@@ -25,15 +25,19 @@
  *     call's kernels have already left, and the compaction of one call runs
  *     beside the scoring kernel of the next.  This is invisible to stream
  *     order: every output of a call is complete before any later operation on
- *     the stream (a copy, another library's kernel, an event) starts.  Two
- *     rules follow for the caller.  (1) Inputs of a call (hidden states,
- *     weights, K, V) must be complete in stream order before the PREVIOUS
- *     kvzap call on that stream was enqueued, or be produced by an ordinary
- *     kernel or copy enqueued between the two calls (which then separates
- *     them); a producer that itself signals "dependents may start" before it
- *     has finished must not sit directly ahead of a kvzap call.  (2) Passing
- *     the same scores buffer to two consecutive calls is allowed; the library
- *     then launches the second call's scoring kernel without overlap.
+ *     the stream (a copy, another library's kernel, an event) starts.
+ *     By default a call's first kernel still waits, before it reads any caller
+ *     data, until everything ahead of it in the stream has completed; so any
+ *     producer of the inputs is safe, including library kernels that signal
+ *     "dependents may start" before their last store (only launch latency is
+ *     overlapped then).  KVZAP_FLAG_TRUSTED_PRODUCERS in kvzap_config.flags
+ *     drops that wait and gives the full overlap; the caller then guarantees:
+ *     (1) inputs of a call (hidden states, K, V) are complete in stream order
+ *     before the PREVIOUS kvzap call on that stream was enqueued, or are
+ *     produced by an ordinary kernel or copy enqueued between the two calls
+ *     that does not itself signal early.  (2) Passing the same scores buffer
+ *     to two consecutive calls is allowed in either mode; the library then
+ *     launches the second call's scoring kernel without overlap of its stores.
  *   - Errors the host can see (bad argument, unsupported shape) return at once
  *     and launch nothing.  Conditions only the device can see set a status
  *     word that kvzap_poll_status() reads; kernels never trap and every
@@ -80,8 +84,12 @@ typedef struct {
     int32_t device;       /* CUDA device ordinal                                                */
     int64_t max_tokens;   /* largest n_tokens any call will pass (sizes the scratch)            */
     int32_t max_seqs;     /* largest number of sequences in one call (>= 1)                     */
-    int32_t reserved;     /* set to 0                                                           */
+    int32_t flags;        /* 0, or KVZAP_FLAG_* values or-ed together                           */
 } kvzap_config;
+
+/* The caller vouches for whatever produces the inputs of its calls (see "Work of consecutive calls"
+ * above): kernels of a call may read caller data before the work ahead in the stream has completed. */
+#define KVZAP_FLAG_TRUSTED_PRODUCERS 1
 
 /* Creates a context on cfg->device (allocates weights storage and scratch with
  * cudaMalloc; synchronous).  *out is NULL on failure. */
@@ -372,6 +380,16 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
 kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, const int32_t *page_table,
                                 int32_t next_free_page, void *stream);
 
+/*
+ * The inverse of kvzap_cache_import, a snapshot of the prefix bookkeeping: copies prefix_len
+ * [n_seqs*L*H] and page_table [n_seqs*L*H, max_pages_per_list] (device int32, list order (seq, layer,
+ * head)) out of the cache and writes the allocator's cursor -- the first pool page never handed out --
+ * to *next_free_page (device).  Entries of a list's table row beyond ceil(prefix_len / page_tokens)
+ * are meaningless.  Enqueued on `stream`; used by the tests to check that no page is owned twice.
+ */
+kvzap_status kvzap_cache_snapshot(kvzap_cache *cache, int32_t *prefix_len, int32_t *page_table,
+                                  int32_t *next_free_page, void *stream);
+
 /* Kernel identifiers for kvzap_get_profile. */
 enum { KVZAP_KERNEL_SCORE = 0, KVZAP_KERNEL_MASK = 1, KVZAP_KERNEL_SCAN = 2, KVZAP_KERNEL_COMPACT = 3,
        KVZAP_KERNEL_DECODE_UPDATE = 4, KVZAP_KERNEL_ATTENTION = 5 };
@@ -430,6 +448,27 @@ kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V, const flo
  * since the last poll (KVZAP_ERR_TIMEOUT, KVZAP_ERR_OOM_PAGES).
  */
 kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream);
+
+/*
+ * Failure detection (the paper has no counterpart).  Waits on flags in global memory that another
+ * CTA or an earlier launch sets -- the step counters that order consecutive fused decode steps, the
+ * per-tile counts of the one-launch prefill of short prompts -- give up after `cycles` SM clock cycles
+ * (default about one second), set the status word to KVZAP_ERR_TIMEOUT and return without touching
+ * the cache, the lengths or the compacted rows (a scores buffer may hold unfinished values).
+ * kvzap_set_wait_limit changes that bound for later calls on the context (cycles >= 1000).  Waits on hardware barriers inside a CTA keep their compile-time bound.
+ * After a polled KVZAP_ERR_TIMEOUT the step counters of every cache of the context are cleared, so
+ * the next decode step starts from a consistent state; steps that were in flight when the wait ran
+ * out did nothing.
+ */
+kvzap_status kvzap_set_wait_limit(kvzap_ctx *ctx, int64_t cycles);
+
+/*
+ * Test aid: adds `delta` to the host's count of fused decode steps completed on every layer of the
+ * cache, WITHOUT telling the device.  The next fused step then waits for a step that never ran, its
+ * bounded wait runs out, and the status word reads KVZAP_ERR_TIMEOUT: the one way to see that path
+ * without a fault.  Never call it in production code.
+ */
+kvzap_status kvzap_cache_debug_skew_steps(kvzap_cache *cache, int32_t delta);
 
 /* Number of kernels the library has launched through this context since it was
  * created (for launch accounting in benchmarks). */

@@ -35,7 +35,7 @@ class KvzapError(RuntimeError):
 class KvzapConfig(ctypes.Structure):
     _fields_ = [("d_model", ctypes.c_int32), ("hidden", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
                 ("head_dim", ctypes.c_int32), ("n_layers", ctypes.c_int32), ("device", ctypes.c_int32),
-                ("max_tokens", ctypes.c_int64), ("max_seqs", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("max_tokens", ctypes.c_int64), ("max_seqs", ctypes.c_int32), ("flags", ctypes.c_int32)]
 
 
 _vp, _i32, _i64, _f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
@@ -69,6 +69,9 @@ SIGNATURES = {
     "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
     "kvzap_prefill_to_cache": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
     "kvzap_cache_import": (_i32, [_vp, _vp, _vp, _i32, _vp]),
+    "kvzap_cache_snapshot": (_i32, [_vp, _vp, _vp, _vp, _vp]),
+    "kvzap_set_wait_limit": (_i32, [_vp, _i64]),
+    "kvzap_cache_debug_skew_steps": (_i32, [_vp, _i32]),
     "kvzap_set_profiling": (_i32, [_vp, _i32]),
     "kvzap_get_profile": (_i32, [_vp, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64)]),
     "kvzap_poll_status": (_i32, [_vp, _vp]),
@@ -121,8 +124,11 @@ def _check(handle, st):
         raise KvzapError(st, msg.decode() if msg else "")
 
 
-def kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0):
-    cfg = KvzapConfig(d_model, hidden, n_kv_heads, head_dim, n_layers, device, max_tokens, max_seqs, 0)
+FLAG_TRUSTED_PRODUCERS = 1
+
+
+def kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0, flags=0):
+    cfg = KvzapConfig(d_model, hidden, n_kv_heads, head_dim, n_layers, device, max_tokens, max_seqs, flags)
     handle = ctypes.c_void_p()
     st = load().kvzap_create(ctypes.byref(handle), ctypes.byref(cfg))
     _check(None, st)
@@ -286,6 +292,11 @@ def kvzap_cache_import(handle, cache, prefix_len, page_table, next_free_page, st
                                              _stream(stream)))
 
 
+def kvzap_cache_snapshot(handle, cache, prefix_len, page_table, next_free_page, stream=None):
+    _check(handle, load().kvzap_cache_snapshot(cache, _ptr(prefix_len), _ptr(page_table), _ptr(next_free_page),
+                                               _stream(stream)))
+
+
 class PreparedCall:
     """One C entry point with its arguments marshalled once.  For loops that repeat the same call on the
     same buffers (a benchmark step, a serving loop with fixed buffers): calling it costs one ctypes
@@ -374,6 +385,15 @@ def kvzap_get_profile(handle, kernel):
     return float(ms.value), int(n.value)
 
 
+def kvzap_set_wait_limit(handle, cycles):
+    _check(handle, load().kvzap_set_wait_limit(handle, cycles))
+
+
+def kvzap_cache_debug_skew_steps(cache, delta):
+    """Test aid: makes the next fused decode step wait for a step that never ran (see the header)."""
+    _check(None, load().kvzap_cache_debug_skew_steps(cache, delta))
+
+
 def kvzap_poll_status(handle, stream=None) -> int:
     return int(load().kvzap_poll_status(handle, _stream(stream)))
 
@@ -385,11 +405,16 @@ def kvzap_launch_count(handle) -> int:
 class Kvzap:
     """Owns one context; allocates outputs with torch; same calls as the C ABI."""
 
-    def __init__(self, d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0):
+    def __init__(self, d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs=1, device=0,
+                 trusted_producers=False):
+        """trusted_producers: the caller vouches that the inputs of every call are complete before the
+        previous call on the stream was enqueued (KVZAP_FLAG_TRUSTED_PRODUCERS): full overlap of
+        consecutive calls.  Off, a call's first kernel waits for the work ahead of it in the stream."""
         self.d_model, self.hidden, self.n_kv_heads, self.head_dim = d_model, hidden, n_kv_heads, head_dim
         self.n_layers, self.max_tokens, self.max_seqs = n_layers, max_tokens, max_seqs
         self.device = torch.device("cuda", device)
-        self.handle = kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs, device)
+        self.handle = kvzap_create(d_model, hidden, n_kv_heads, head_dim, n_layers, max_tokens, max_seqs, device,
+                                   FLAG_TRUSTED_PRODUCERS if trusted_producers else 0)
 
     def close(self):
         if self.handle is not None:

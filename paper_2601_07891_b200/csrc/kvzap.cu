@@ -97,6 +97,17 @@ struct kvzap_ctx {
     float *stage_scores = nullptr;
     int32_t *stage_lengths = nullptr, *stage_cu = nullptr;
     int32_t *lengths_pinned = nullptr;
+    // kvzap_config.flags & KVZAP_FLAG_TRUSTED_PRODUCERS: kernels may read caller data before the work ahead of
+    // them in the stream has completed
+    bool trusted = false;
+    int64_t wait_limit = KVZAP_WAIT_LIMIT_CYCLES;   // bound of the waits on flags in global memory
+    // Every public call that enqueues work takes the next number.  A fused decode step may start before the
+    // kernel ahead of it has finished only when that kernel is the fused step of the call just before, on
+    // the same cache: those two order their cache accesses through the step counters, nothing else does.
+    uint64_t op_seq = 0, fused_seq = 0;
+    const kvzap_cache *fused_cache = nullptr;
+    std::vector<kvzap_cache *> caches;              // caches created on this context (their step counters are
+                                                    // cleared when a timeout has been polled)
     char err[512] = "";
 };
 
@@ -118,6 +129,12 @@ static kvzap_status fail(kvzap_ctx *ctx, kvzap_status st, const char *fmt, ...)
         if (e_ != cudaSuccess)                                                                       \
             return kvzap::fail(ctx, KVZAP_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
     } while (0)
+
+// Numbers a public call (see kvzap_ctx::op_seq).
+static inline void begin_op(kvzap_ctx *ctx) { ctx->op_seq += 1; }
+
+// Clears the fused decode step's counters (device and host view) of every cache of the context.
+static void reset_step_counters(kvzap_ctx *ctx, cudaStream_t stream);
 
 static int next_pow2(int v)
 {
@@ -339,7 +356,7 @@ static void make_launch(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attrs, dim
 static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
                                  float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1,
-                                 const DecodeFuse *fuse = nullptr, bool *fused = nullptr)
+                                 const DecodeFuse *fuse = nullptr, bool *fused = nullptr, bool fuse_chain = false)
 {
     if (fused) *fused = false;
     // Early start.  When the grid fills the machine (one CTA per SM), this kernel is allowed to start
@@ -420,11 +437,16 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             f.enabled = 1;
             if (fused) *fused = true;
         }
-        // The fused decode step touches the cache before it has waited for the kernel ahead (its clusters
-        // order themselves through `done`), so it is started early only with a grid of at least half the
-        // SMs and its own scores buffer.  Without the fused part the kernel reads nothing but hidden states
-        // and weights until every thread has waited, and writes only after: it may always start early.
-        const bool early = !ctx->profiling && (fuse_ok ? (!clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count) : true);
+        // The fused decode step touches the cache (counters, page allocator, rows) before it has waited for
+        // the kernel ahead; its clusters order themselves through `done`, which covers earlier fused steps
+        // only.  So it is started early only directly behind the fused step of the previous call on the
+        // same cache (fuse_chain) -- never behind a prompt chunk's page assignment, a release or an export,
+        // whose kernels it would race with -- and with a grid of at least half the SMs and its own scores
+        // buffer.  Without the fused part the kernel reads nothing but hidden states and weights until
+        // every thread has waited, and writes only after: it may always start early.
+        const bool early = !ctx->profiling &&
+                           (fuse_ok ? (fuse_chain && !clash && p.n_tiles * n_ctas * 2 >= ctx->sm_count) : true);
+        p.wait_before_load = ctx->trusted ? 0 : 1;
         ctx->last_score_early = early;
         {
             ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
@@ -466,6 +488,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         p.window_keep = window_keep;
         p.tau = tau;
         p.status = ctx->status_dev;
+        p.wait_before_load = ctx->trusted ? 0 : 1;
         const bool early = !ctx->profiling;
         // Writing before the kernel ahead has completed is safe only if (a) the scores buffer is not the
         // previous call's, and (b) the launch takes more than half of the SMs (one CTA each): then its
@@ -533,6 +556,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.window_keep = window_keep;
     p.tau = tau;
     p.status = ctx->status_dev;
+    p.wait_before_load = ctx->trusted ? 0 : 1;
     // every launch finds its counter at zero: it was cleared by the launch before the previous one
     p.tile_counter = ctx->tile_counters + ctx->score_turn % kMaskRing;
     p.tile_counter_reset = ctx->tile_counters + (ctx->score_turn + 2) % kMaskRing;
@@ -651,6 +675,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         return fail(nullptr, KVZAP_ERR_INVALID_ARG, "max_tokens out of range (1..2^30)");
     if (c.max_seqs < 1 || c.max_seqs > (1 << 20))
         return fail(nullptr, KVZAP_ERR_INVALID_ARG, "max_seqs out of range (1..2^20)");
+    if (c.flags & ~KVZAP_FLAG_TRUSTED_PRODUCERS)
+        return fail(nullptr, KVZAP_ERR_INVALID_ARG, "flags 0x%x: unknown bits set", static_cast<unsigned>(c.flags));
 
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || c.device < 0 || c.device >= n_dev)
@@ -667,6 +693,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     kvzap_ctx *ctx = new (std::nothrow) kvzap_ctx();
     if (!ctx) return fail(nullptr, KVZAP_ERR_CUDA, "out of host memory");
     ctx->cfg = c;
+    ctx->trusted = (c.flags & KVZAP_FLAG_TRUSTED_PRODUCERS) != 0;
     ctx->sm_count = prop.multiProcessorCount;
 
     // scoring schedules
@@ -885,6 +912,7 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, co
 {
     NvtxRange nvtx_range("kvzap_set_weights");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
     if (layer < 0 || layer >= c.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
@@ -925,6 +953,7 @@ kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int6
 {
     NvtxRange nvtx_range("kvzap_score");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
     if (st != KVZAP_OK) return st;
@@ -943,6 +972,7 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
 {
     NvtxRange nvtx_range("kvzap_prune_prefill");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
     if (st != KVZAP_OK) return st;
@@ -976,6 +1006,7 @@ kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void 
 {
     NvtxRange nvtx_range("kvzap_prune_prefill_topk");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
     if (st != KVZAP_OK) return st;
@@ -1030,6 +1061,7 @@ static kvzap_status prefill_fused_impl(kvzap_ctx *ctx, int32_t layer, const void
 {
     NvtxRange nvtx_range("kvzap_prefill_fused / kvzap_prefill_write");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -1082,9 +1114,18 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing, stream);
     if (ctx->split_arrive) cudaMemsetAsync(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
     if (ctx->wide_arrive) cudaMemsetAsync(ctx->wide_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
+    if (v == KVZAP_ERR_TIMEOUT) reset_step_counters(ctx, stream);
     cudaStreamSynchronize(stream);
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
+}
+
+kvzap_status kvzap_set_wait_limit(kvzap_ctx *ctx, int64_t cycles)
+{
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    if (cycles < 1000) return fail(ctx, KVZAP_ERR_INVALID_ARG, "wait limit %lld: need at least 1000 cycles", static_cast<long long>(cycles));
+    ctx->wait_limit = cycles;
+    return KVZAP_OK;
 }
 
 kvzap_status kvzap_set_profiling(kvzap_ctx *ctx, int32_t enable)
@@ -1123,6 +1164,7 @@ kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void 
 {
     NvtxRange nvtx_range("kvzap_prefill_fused_host");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -1308,6 +1350,16 @@ struct kvzap_cache {
 
 namespace kvzap {
 
+static void reset_step_counters(kvzap_ctx *ctx, cudaStream_t stream)
+{
+    for (kvzap_cache *cache : ctx->caches) {
+        const size_t n = 4 * static_cast<size_t>(ctx->cfg.n_layers) * ((cache->v.n_seqs + 127) / 128);
+        cudaMemsetAsync(cache->done, 0, sizeof(int32_t) * n, stream);
+        cache->steps_done.assign(ctx->cfg.n_layers, 0);
+    }
+    ctx->fused_cache = nullptr;
+}
+
 static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
                                             const int32_t *cu_seqlens,
                                             int32_t n_seqs, int64_t n_tokens, void *K_pool, void *V_pool,
@@ -1388,6 +1440,7 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
 {
     NvtxRange nvtx_range("kvzap_prune_prefill_paged");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
     if (st != KVZAP_OK) return st;
@@ -1426,6 +1479,7 @@ static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, cons
 {
     NvtxRange nvtx_range("kvzap_prefill_fused_paged / kvzap_prefill_write_paged");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
@@ -1533,7 +1587,15 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
         kvzap_cache_destroy(cache);
         return KVZAP_ERR_CUDA;
     }
+    ctx->caches.push_back(cache);
     *out = cache;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_cache_debug_skew_steps(kvzap_cache *cache, int32_t delta)
+{
+    if (!cache) return KVZAP_ERR_INVALID_ARG;
+    for (auto &n : cache->steps_done) n += delta;
     return KVZAP_OK;
 }
 
@@ -1542,6 +1604,12 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     if (!cache) return KVZAP_OK;
     DeviceGuard guard(cache->ctx->cfg.device);
     cudaDeviceSynchronize();
+    {
+        auto &list = cache->ctx->caches;
+        for (size_t i = 0; i < list.size(); ++i)
+            if (list[i] == cache) { list.erase(list.begin() + static_cast<long>(i)); break; }
+        if (cache->ctx->fused_cache == cache) cache->ctx->fused_cache = nullptr;
+    }
     cudaFree(cache->v.k_ring); cudaFree(cache->v.v_ring); cudaFree(cache->v.score_ring);
     cudaFree(cache->v.n_tokens); cudaFree(cache->v.prefix_len); cudaFree(cache->v.page_table);
     cudaFree(cache->v.page_cursor); cudaFree(cache->scores); cudaFree(cache->done);
@@ -1557,6 +1625,7 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
 {
     NvtxRange nvtx_range("kvzap_decode_step");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
     if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end)
@@ -1587,13 +1656,18 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
         fuse.V_new = static_cast<const uint4 *>(V_new);
         fuse.tau = tau;
         fuse.done = cache->done;
+        fuse.wait_limit = ctx->wait_limit;
     }
     bool fused = false;
+    // the call just before this one was a fused step on this cache: the two may overlap
+    const bool chain = ctx->fused_cache == cache && ctx->fused_seq + 1 == ctx->op_seq;
     kvzap_status st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
-                                   0.0f, 0, stream, 1, can_fuse ? &fuse : nullptr, &fused);
+                                   0.0f, 0, stream, 1, can_fuse ? &fuse : nullptr, &fused, chain);
     if (st != KVZAP_OK) return st;
     if (fused) {
         for (int l = layer_begin; l < layer_end; ++l) cache->steps_done[l] += 1;
+        ctx->fused_cache = cache;
+        ctx->fused_seq = ctx->op_seq;
         return KVZAP_OK;
     }
     const int64_t n_groups = static_cast<int64_t>(n_layers) * cache->v.n_seqs * c.n_kv_heads;
@@ -1618,6 +1692,7 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
 {
     NvtxRange nvtx_range("kvzap_decode_attention");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
     const CacheView &v = cache->v;
@@ -1714,6 +1789,7 @@ kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stre
 {
     if (!cache) return KVZAP_ERR_INVALID_ARG;
     kvzap_ctx *ctx = cache->ctx;
+    begin_op(ctx);
     if (seq < 0 || seq >= cache->v.n_seqs) return fail(ctx, KVZAP_ERR_INVALID_ARG, "release: seq %d out of range", seq);
     DeviceGuard guard(ctx->cfg.device);
     release_seq_kernel<<<static_cast<unsigned>(cache->v.n_layers * cache->v.n_heads), 32, 0,
@@ -1726,6 +1802,7 @@ kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stre
 kvzap_status kvzap_cache_lengths(kvzap_cache *cache, int32_t *lengths, void *stream_)
 {
     if (!cache || !lengths) return KVZAP_ERR_INVALID_ARG;
+    begin_op(cache->ctx);
     DeviceGuard guard(cache->ctx->cfg.device);
     cache_lengths_kernel<<<static_cast<unsigned>((cache->n_lists + 255) / 256), 256, 0,
                            static_cast<cudaStream_t>(stream_)>>>(cache->v, lengths);
@@ -1738,6 +1815,7 @@ kvzap_status kvzap_cache_export(kvzap_cache *cache, int32_t seq, int32_t layer, 
                                 int64_t capacity_rows, int32_t *n_rows, void *stream_)
 {
     if (!cache || !K_out || !V_out || !n_rows || capacity_rows < 0) return KVZAP_ERR_INVALID_ARG;
+    begin_op(cache->ctx);
     const CacheView &v = cache->v;
     if (seq < 0 || seq >= v.n_seqs || layer < 0 || layer >= v.n_layers || head < 0 || head >= v.n_heads)
         return fail(cache->ctx, KVZAP_ERR_INVALID_ARG, "export: (seq, layer, head) out of range");
@@ -1757,6 +1835,7 @@ kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, c
     if (!cache || !prefix_len || !page_table || next_free_page < 0) return KVZAP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     kvzap_ctx *ctx = cache->ctx;
+    begin_op(ctx);
     DeviceGuard guard(ctx->cfg.device);
     const size_t n = static_cast<size_t>(cache->n_lists);
     KVZAP_CUDA(ctx, cudaMemcpyAsync(cache->v.prefix_len, prefix_len, sizeof(int32_t) * n, cudaMemcpyDeviceToDevice, stream));
@@ -1770,12 +1849,29 @@ kvzap_status kvzap_cache_import(kvzap_cache *cache, const int32_t *prefix_len, c
     return KVZAP_OK;
 }
 
+kvzap_status kvzap_cache_snapshot(kvzap_cache *cache, int32_t *prefix_len, int32_t *page_table, int32_t *next_free_page,
+                                  void *stream_)
+{
+    if (!cache || !prefix_len || !page_table || !next_free_page) return KVZAP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    kvzap_ctx *ctx = cache->ctx;
+    begin_op(ctx);
+    DeviceGuard guard(ctx->cfg.device);
+    const size_t n = static_cast<size_t>(cache->n_lists);
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(prefix_len, cache->v.prefix_len, sizeof(int32_t) * n, cudaMemcpyDeviceToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(page_table, cache->v.page_table, sizeof(int32_t) * n * cache->v.max_pages,
+                                    cudaMemcpyDeviceToDevice, stream));
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(next_free_page, cache->v.page_cursor, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream));
+    return KVZAP_OK;
+}
+
 kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, int32_t seq, const void *hidden,
                                     const void *K, const void *V, int64_t n_tokens, float tau, float *scores_out,
                                     void *stream_)
 {
     NvtxRange nvtx_range("kvzap_prefill_to_cache");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const kvzap_config &c = ctx->cfg;
     const CacheView &v = cache->v;

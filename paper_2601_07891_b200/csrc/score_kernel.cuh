@@ -75,6 +75,7 @@ struct ScoreParams {
     float tau;
     int32_t *status;      // device status word
     int32_t wait_before_write;    // 1: the epilogue waits for the kernel ahead in the stream before its first store
+    int32_t wait_before_load;     // 1: every thread waits for the work ahead in the stream before caller data is read
     int32_t *tile_counter;        // work tiles handed out beyond the first one of every CTA (or pair); starts at 0
     int32_t *tile_counter_reset;  // the counter of the launch after next: set to 0 by this launch
     // few-token kernel only: the clusters of one tile combine their partial scores through global memory
@@ -273,6 +274,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     if constexpr (kPair) cluster_sync_all();     // the other CTA's barriers exist before anything signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // The set-up above overlaps the tail of the work ahead in the stream either way; unless the caller
+    // vouches for the producers of its inputs, nothing of them is read before that work has completed.
+    if (p.wait_before_load) griddep_wait();
 
     const int k_blocks = p.d_model / kBlockK;
     if (blockIdx.x == 0 && threadIdx.x == 0) *p.tile_counter_reset = 0;

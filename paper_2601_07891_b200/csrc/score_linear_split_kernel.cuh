@@ -48,6 +48,7 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kLinBarsOff + 16 * kLinStages + 20);
 
     griddep_launch_dependents();
+    if (p.wait_before_load) griddep_wait();     // caller data is read only after the work ahead in the stream is complete
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();

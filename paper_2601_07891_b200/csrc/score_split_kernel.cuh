@@ -41,6 +41,7 @@ struct DecodeFuse {
     const uint4 *K_new, *V_new;     // [n_layers_call][B][H][D] bf16
     float tau;
     int32_t *done;                  // [n_layers * tiles_per_layer][n_split]
+    int64_t wait_limit;             // cycles a cluster waits for the step before to be published
 };
 
 struct SplitSmemLayout {
@@ -94,6 +95,9 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     volatile int *last_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 40);
 
     griddep_launch_dependents();
+    // unless the caller vouches for the producers of its inputs, nothing of them is read before the work
+    // ahead in the stream has completed (every thread waits: the loads below are issued by several warps)
+    if (p.wait_before_load) griddep_wait();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();            // 0 .. k_split - 1
@@ -236,7 +240,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             if (etid < n_split) {
                 const long long t0 = clock64();
                 while (ld_acquire_gpu(f.done + cid * n_split + etid) != f.expect) {
-                    if (clock64() - t0 > KVZAP_WAIT_LIMIT_CYCLES) { *abort_flag = 1; break; }
+                    if (clock64() - t0 > f.wait_limit) { *abort_flag = 1; break; }
                 }
             }
             named_barrier_sync(1, 256);

@@ -36,7 +36,7 @@ def _prefill_case(binding, oracle, wl, layer, tau, sample=None, seed_shift=0):
     dev = "cuda"
     B, T = wl.batch, wl.seq_len
     n_tokens, H, D = B * T, wl.n_kv_heads, wl.head_dim
-    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, 1, n_tokens, max_seqs=B)
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, 1, n_tokens, max_seqs=B, trusted_producers=True)
     weights = synth.surrogate_weights(wl, layer, dev)
     ctx.set_weights(0, *weights)
     X = synth.hidden_states(n_tokens, wl.d_model, 31 + layer + seed_shift, dev, wl.token_scale_sigma)
@@ -149,7 +149,7 @@ def test_config5_decode_b128_all_layers(binding, oracle):
     wl = W["qwen3_8b_decode_b128"]
     L, B, H, D, w, P = wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     n_steps = w + 4
-    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B)
+    ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, trusted_producers=True)
     weights = []
     for l in range(L):
         wts = synth.surrogate_weights(wl, l, "cuda")

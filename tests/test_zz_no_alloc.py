@@ -10,11 +10,12 @@ import pytest
 import torch
 
 from paper_2601_07891_b200 import synth
+from tests import parity
 
 pytestmark = pytest.mark.gpu
 
 
-def _one_round(binding, ctx, seq_lens, tau, w, seed, D=128, H=8):
+def _one_round(binding, ctx, oracle, seq_lens, tau, w, seed, D=128, H=8):
     T = int(sum(seq_lens))
     B = len(seq_lens)
     g = torch.Generator().manual_seed(seed)
@@ -22,7 +23,7 @@ def _one_round(binding, ctx, seq_lens, tau, w, seed, D=128, H=8):
     K, V = synth.keys_values(H, T, D, seed)
     K, V = K.cuda(), V.cuda()
     cu = torch.from_numpy(synth.cu_seqlens(seq_lens)).cuda() if B > 1 else None
-    poison = lambda: torch.full((H, T, D), -3.0, dtype=torch.bfloat16, device="cuda")
+    poison = lambda: parity.poison_like(K)
     # existing entry point (context scratch from cudaMalloc)
     K_ref, V_ref = poison(), poison()
     len_ref = torch.full((B, H), -1, dtype=torch.int32, device="cuda")
@@ -36,17 +37,20 @@ def _one_round(binding, ctx, seq_lens, tau, w, seed, D=128, H=8):
     assert int(len_ref.sum()) > 0
     assert torch.equal(K_new.view(torch.int16), K_ref.view(torch.int16))      # bit-exact, poison rows included
     assert torch.equal(V_new.view(torch.int16), V_ref.view(torch.int16))
+    # and against the oracle's mask + ordered gather of the same scores (rows past the lengths keep their poison)
+    cu_np = synth.cu_seqlens(seq_lens) if B > 1 else None
+    parity.check_compaction(oracle, K.cpu(), V.cpu(), scores.cpu().numpy(), tau, w, cu_np, K_new.cpu(), V_new.cpu(), len_new)
 
 
-def test_noalloc_matches_context_entry_point_two_calls_in_a_row():
+def test_noalloc_matches_context_entry_point_two_calls_in_a_row(oracle):
     from paper_2601_07891_b200 import binding
     binding.load()
     ctx = binding.Kvzap(256, 0, 8, 128, 1, max_tokens=8192, max_seqs=8)
-    _one_round(binding, ctx, [5000, 1, 0, 2999], 0.43, 128, seed=1)      # 8000 tokens, several blocks, ragged
-    _one_round(binding, ctx, [333], -0.2, 16, seed=2)                    # smaller: stale scratch must not matter
+    _one_round(binding, ctx, oracle, [5000, 1, 0, 2999], 0.43, 128, seed=1)      # 8000 tokens, several blocks, ragged
+    _one_round(binding, ctx, oracle, [333], -0.2, 16, seed=2)                    # smaller: stale scratch must not matter
     ctx.close()
     ctx = binding.Kvzap(256, 0, 3, 64, 1, max_tokens=2048, max_seqs=2)   # other shape parameters
-    _one_round(binding, ctx, [700, 700], 0.9, 0, seed=3, D=64, H=3)
+    _one_round(binding, ctx, oracle, [700, 700], 0.9, 0, seed=3, D=64, H=3)
     ctx.close()
 
 
