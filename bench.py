@@ -319,13 +319,14 @@ def run_prefill(args, wl, env):
     score_ms = _timed(score_only, n_rep, sync) / L
     if proj:
         prune = None          # the two-call route exists for the head-major layout only
-    elif P:
-        prune = lambda: [binding.kvzap_prune_prefill_paged(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
-                                                           Kos[l], Vos[l], P, 0, tabs[l], lens[l], used[l])
-                         for l in range(n_bufs)]
     else:
-        prune = lambda: [binding.kvzap_prune_prefill(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
-                                                     Kos[l], Vos[l], lens[l]) for l in range(n_bufs)]
+        if P:
+            pcalls = [binding.prepare_prune_prefill_paged(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
+                                                          Kos[l], Vos[l], P, 0, tabs[l], lens[l], used[l]) for l in range(n_bufs)]
+        else:
+            pcalls = [binding.prepare_prune_prefill(ctx.handle, Ks[l], Vs[l], scs[l], cu, B, wl.tau, wl.window,
+                                                    Kos[l], Vos[l], lens[l]) for l in range(n_bufs)]
+        prune = lambda: [pc() for pc in pcalls]
     prune_ms = _timed(prune, n_rep, sync) / n_bufs if prune else None
 
     peaks, peak_src = load_peaks()

@@ -325,6 +325,21 @@ def prepare_prefill_fused(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, 
     return PreparedCall("kvzap_prefill_fused", handle, args, (hidden, K, V, cu_seqlens, K_out, V_out, lengths, scores_out))
 
 
+def prepare_prune_prefill(handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths, stream=None) -> PreparedCall:
+    args = (handle, _ptr(K), _ptr(V), _ptr(scores), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_out), _ptr(V_out),
+            _ptr(lengths), _stream(stream))
+    return PreparedCall("kvzap_prune_prefill", handle, args, (K, V, scores, cu_seqlens, K_out, V_out, lengths))
+
+
+def prepare_prune_prefill_paged(handle, K, V, scores, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens, first_page,
+                                page_table, lengths, n_pages_used, stream=None) -> PreparedCall:
+    args = (handle, _ptr(K), _ptr(V), _ptr(scores), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_pool), _ptr(V_pool),
+            K_pool.shape[0], page_tokens, first_page, _ptr(page_table), page_table.shape[1], _ptr(lengths),
+            _ptr(n_pages_used), _stream(stream))
+    return PreparedCall("kvzap_prune_prefill_paged", handle, args,
+                        (K, V, scores, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used))
+
+
 def prepare_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
                                 first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None) -> PreparedCall:
     args = (handle, layer, _ptr(hidden), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_pool),

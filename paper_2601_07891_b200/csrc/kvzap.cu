@@ -16,6 +16,7 @@
 #include "attn_kernel.cuh"
 #include "decode_kernels.cuh"
 #include "prune_kernels.cuh"
+#include "prune_onepass_kernel.cuh"
 #include "score_kernel.cuh"
 #include "score_linear_split_kernel.cuh"
 #include "score_split_kernel.cuh"
@@ -108,6 +109,24 @@ struct kvzap_ctx {
     const kvzap_cache *fused_cache = nullptr;
     std::vector<kvzap_cache *> caches;              // caches created on this context (their step counters are
                                                     // cleared when a timeout has been polled)
+    // one-launch pruning (kvzap_prune_prefill and its paged / fixed-budget forms): kOpRing scratch sets in rotation
+    int op_capacity = 0;                 // CTAs of prune_onepass_kernel the device holds at once
+    uint32_t *op_mask = nullptr;         // [kOpRing][H][max_words]
+    uint64_t *op_counts = nullptr;       // [kOpRing][op_capacity][8]
+    int32_t *op_len_acc = nullptr;       // [kOpRing][max_seqs * H], zero between calls
+    uint32_t *op_arrive = nullptr;       // [kOpRing]
+    int32_t *op_scan_flag = nullptr;     // [kOpRing]
+    int32_t *op_page0 = nullptr;         // [kOpRing][max_seqs * H]
+    uint64_t op_turn = 0;
+    int32_t op_epoch = 0;
+    int op_chain = 0;                    // launches of that kernel in a row that did not wait for the work ahead
+    uint64_t op_last_seq = 0;            // number (op_seq) of the last call that launched it
+    // Caller memory read or written by the launches of that kernel since the last one that waited for all
+    // work ahead of it: these launches may still be running.  Another one is started without such a wait
+    // only directly behind them and only if it conflicts with none of these ranges; the scoring kernels
+    // consult the list before they write a scores buffer early.
+    struct Range { const char *p; size_t n; bool w; };
+    std::vector<Range> pending;
     char err[512] = "";
 };
 
@@ -132,6 +151,25 @@ static kvzap_status fail(kvzap_ctx *ctx, kvzap_status st, const char *fmt, ...)
 
 // Numbers a public call (see kvzap_ctx::op_seq).
 static inline void begin_op(kvzap_ctx *ctx) { ctx->op_seq += 1; }
+
+// ---- what the kernels in flight may still touch (see kvzap_ctx::pending)
+constexpr size_t kMaxPending = 96;
+static inline void note_range(kvzap_ctx *ctx, const void *p, size_t n, bool write)
+{
+    if (p != nullptr && n > 0) ctx->pending.push_back({static_cast<const char *>(p), n, write});
+}
+// true if [p, p + n) overlaps a pending range in a conflicting way (a write on either side)
+static inline bool hazard(const kvzap_ctx *ctx, const void *p, size_t n, bool write)
+{
+    if (p == nullptr || n == 0) return false;
+    if (ctx->pending.size() > kMaxPending) return true;
+    const char *a = static_cast<const char *>(p);
+    for (const auto &r : ctx->pending)
+        if ((write || r.w) && a < r.p + r.n && r.p < a + n) return true;
+    return false;
+}
+// everything enqueued so far is complete before whatever is enqueued next starts
+static inline void serial_point(kvzap_ctx *ctx) { ctx->pending.clear(); ctx->op_chain = 0; }
 
 // Clears the fused decode step's counters (device and host view) of every cache of the context.
 static void reset_step_counters(kvzap_ctx *ctx, cudaStream_t stream);
@@ -273,6 +311,8 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->wide_arrive);
     cudaFree(ctx->list_page0);
     cudaFree(ctx->list_base);
+    cudaFree(ctx->op_mask); cudaFree(ctx->op_counts); cudaFree(ctx->op_len_acc);
+    cudaFree(ctx->op_arrive); cudaFree(ctx->op_scan_flag); cudaFree(ctx->op_page0);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
@@ -372,6 +412,9 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // still use it.
     const kvzap_config &c = ctx->cfg;
     const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    // the scores buffer may still be in use by a kernel of an earlier call that has not completed
+    const bool scores_busy = scores != nullptr &&
+                             hazard(ctx, scores, sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads, true);
     // Few tiles (a decode step: one tile per layer): split every tile's hidden units (and K range) over
     // several CTAs, so that the launch fills the machine and every CTA reads only its own part of W1.
     // ... and with the K split left out (two CTAs per tile, each a slice of the hidden units over the whole K
@@ -421,10 +464,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         // Early start (consecutive decode steps): this kernel reads only hidden states and weights; the one
         // thing it may not do is write a scores buffer that the kernels of the previous call still read.
         const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
-        bool clash = false;
+        bool clash = scores_busy;
         if (scores && ctx->last_scores) {
             const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
-            clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes;
+            clash = clash || (a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes);
         }
         ctx->last_scores = scores;
         ctx->last_scores_bytes = sbytes;
@@ -496,10 +539,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         // compaction two launches back has completed -- so the mask slice written here, last read
         // kMaskRing launches back, is free.
         const size_t sbytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
-        bool clash = false;
+        bool clash = scores_busy;
         if (scores && ctx->last_scores) {
             const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
-            clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes;
+            clash = clash || (a0 < b0 + ctx->last_scores_bytes && b0 < a0 + sbytes);
         }
         p.wait_before_write = (clash || p.n_tiles * kLinSplit * 2 <= ctx->sm_count) ? 1 : 0;
         ctx->last_score_early = early;
@@ -562,10 +605,10 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     p.tile_counter_reset = ctx->tile_counters + (ctx->score_turn + 2) % kMaskRing;
     ctx->score_turn += 1;
     const size_t scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_layers) * n_tokens * c.n_kv_heads : 0;
-    bool scores_clash = false;           // the previous launch may still be writing the same buffer
+    bool scores_clash = scores_busy;     // the previous launch may still be writing the same buffer
     if (scores && ctx->last_scores) {
         const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
-        scores_clash = a0 < b0 + ctx->last_scores_bytes && b0 < a0 + scores_bytes;
+        scores_clash = scores_clash || (a0 < b0 + ctx->last_scores_bytes && b0 < a0 + scores_bytes);
     }
     ctx->last_scores = scores;
     ctx->last_scores_bytes = scores_bytes;
@@ -633,6 +676,102 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
                                            tok_major ? int64_t{1} : n_tokens,
                                            tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
                                            static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr), 0));
+    }
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
+// Threshold / window mask, counts, prefix sums and the ordered gather in one launch (prune_onepass_kernel),
+// dense-ragged (page_tokens == 0) or paged.  tau_list != nullptr: a threshold per list, written by the
+// kernel ahead in the stream.
+static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, const float *tau_list, float tau, int32_t w,
+                                         const void *K, const void *V, const int32_t *cu_seqlens, int32_t n_seqs,
+                                         int64_t n_tokens, void *K_out, void *V_out, int32_t *lengths, int32_t page_tokens,
+                                         int32_t first_page, int64_t n_pages_pool, int32_t max_pages, int32_t *page_table,
+                                         int32_t *n_pages_used, cudaStream_t stream)
+{
+    const kvzap_config &c = ctx->cfg;
+    if (page_tokens > 0 && n_pages_pool * page_tokens >= 0xffffffffLL)
+        return fail(ctx, KVZAP_ERR_UNSUPPORTED, "paged pruning: the pool must hold fewer than 2^32 - 1 rows");
+    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
+    int64_t grid = n_blocks < ctx->op_capacity ? n_blocks : ctx->op_capacity;
+    const int64_t per_cta = (n_blocks + grid - 1) / grid;
+    grid = (n_blocks + per_cta - 1) / per_cta;
+    const int set = static_cast<int>(ctx->op_turn % kOpRing);
+    ctx->op_turn += 1;
+    ctx->op_epoch = ctx->op_epoch == 0x7fffffff ? 1 : ctx->op_epoch + 1;
+    const size_t n_lists = static_cast<size_t>(n_seqs) * c.n_kv_heads;
+    const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * c.head_dim * 2;
+    const size_t out_bytes = page_tokens > 0 ? static_cast<size_t>(n_pages_pool) * page_tokens * c.head_dim * 2 : kv_bytes;
+    const size_t sc_bytes = sizeof(float) * static_cast<size_t>(n_tokens) * c.n_kv_heads;
+    // Started before the work ahead of it has completed only on a context that trusts its producers,
+    // directly behind another launch of this kernel (whose memory is on the pending list, and whose scratch
+    // set is a different one for kOpRing - 2 launches in a row), and when it conflicts with none of them.
+    bool wait_first = !ctx->trusted || ctx->profiling || tau_list != nullptr || ctx->op_last_seq + 1 != ctx->op_seq ||
+                      ctx->op_chain >= kOpRing - 2;
+    if (!wait_first)
+        wait_first = hazard(ctx, scores, sc_bytes, false) || hazard(ctx, K, kv_bytes, false) || hazard(ctx, V, kv_bytes, false) ||
+                     hazard(ctx, cu_seqlens, sizeof(int32_t) * (n_seqs + 1), false) ||
+                     hazard(ctx, K_out, out_bytes, true) || hazard(ctx, V_out, out_bytes, true) ||
+                     hazard(ctx, lengths, sizeof(int32_t) * n_lists, true) ||
+                     hazard(ctx, page_table, sizeof(int32_t) * n_lists * max_pages, true) ||
+                     hazard(ctx, n_pages_used, sizeof(int32_t), true);
+    if (wait_first) serial_point(ctx);
+    else ctx->op_chain += 1;
+    ctx->op_last_seq = ctx->op_seq;
+    note_range(ctx, scores, sc_bytes, false);
+    note_range(ctx, K, kv_bytes, false);
+    note_range(ctx, V, kv_bytes, false);
+    note_range(ctx, K_out, out_bytes, true);
+    note_range(ctx, V_out, out_bytes, true);
+    note_range(ctx, lengths, sizeof(int32_t) * n_lists, true);
+    if (page_tokens > 0) {
+        note_range(ctx, page_table, sizeof(int32_t) * n_lists * max_pages, true);
+        note_range(ctx, n_pages_used, sizeof(int32_t), true);
+    }
+    PruneParams p;
+    memset(&p, 0, sizeof p);
+    p.scores = scores;
+    p.tau_list = tau_list;
+    p.tau = tau;
+    p.window = w;
+    p.n_tokens = n_tokens;
+    p.n_blocks = n_blocks;
+    p.n_words = n_blocks * 4;
+    p.n_heads = c.n_kv_heads;
+    p.n_seqs = n_seqs;
+    p.cu_seqlens = cu_seqlens;
+    p.blocks_per_cta = static_cast<int32_t>(per_cta);
+    p.K = static_cast<const uint4 *>(K);
+    p.V = static_cast<const uint4 *>(V);
+    p.K_out = static_cast<uint4 *>(K_out);
+    p.V_out = static_cast<uint4 *>(V_out);
+    p.in_stride_h = n_tokens;
+    p.in_stride_t = 1;
+    p.row_units = c.head_dim / 8;
+    p.lengths = lengths;
+    p.page_tokens = page_tokens;
+    p.first_page = first_page;
+    p.max_pages = max_pages;
+    p.n_pages_pool = n_pages_pool;
+    p.list_page0 = ctx->op_page0 + static_cast<size_t>(set) * c.max_seqs * c.n_kv_heads;
+    p.page_table = page_table;
+    p.n_pages_used = n_pages_used;
+    p.status = ctx->status_dev;
+    p.maskbits = ctx->op_mask + static_cast<size_t>(set) * ctx->max_words * c.n_kv_heads;
+    p.cta_counts = ctx->op_counts + static_cast<size_t>(set) * ctx->op_capacity * kMaxHeads;
+    p.len_acc = ctx->op_len_acc + static_cast<size_t>(set) * c.max_seqs * c.n_kv_heads;
+    p.arrive = ctx->op_arrive + set;
+    p.scan_flag = ctx->op_scan_flag + set;
+    p.epoch = ctx->op_epoch;
+    p.wait_limit = ctx->wait_limit;
+    p.wait_first = wait_first ? 1 : 0;
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid)), dim3(kOpThreads), kOpDynSmem, stream, !ctx->profiling, 1);
+        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, prune_onepass_kernel<kOpRows>, p));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -883,6 +1022,31 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         CREATE_CUDA(cudaMalloc(&ctx->wide_arrive, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
         CREATE_CUDA(cudaMemset(ctx->wide_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count)));
     }
+    {
+        // one-launch pruning: a grid never larger than what the device holds at once (its CTAs wait for one another)
+        // No shared-memory carve-out is asked for: with the largest one (which the compaction that runs beside
+        // a scoring kernel needs) the L1 that is left holds too few lines in flight, and this kernel alone moved
+        // rows at 2.4 TB/s instead of 4.9.
+        CREATE_CUDA(cudaFuncSetAttribute(prune_onepass_kernel<kOpRows>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(kOpDynSmem)));
+        int per_sm = 0;
+        CREATE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, prune_onepass_kernel<kOpRows>, kOpThreads, kOpDynSmem));
+        if (per_sm < 1) per_sm = 1;
+        // half of what fits: the next call's kernel then finds room beside this one
+        ctx->op_capacity = per_sm * ctx->sm_count / 2;
+        if (ctx->op_capacity < 1) ctx->op_capacity = 1;
+        const size_t cap = static_cast<size_t>(ctx->op_capacity);
+        CREATE_CUDA(cudaMalloc(&ctx->op_mask, sizeof(uint32_t) * kOpRing * ctx->max_words * c.n_kv_heads));
+        CREATE_CUDA(cudaMalloc(&ctx->op_counts, sizeof(uint64_t) * kOpRing * cap * kMaxHeads));
+        CREATE_CUDA(cudaMemset(ctx->op_counts, 0, sizeof(uint64_t) * kOpRing * cap * kMaxHeads));
+        CREATE_CUDA(cudaMalloc(&ctx->op_len_acc, sizeof(int32_t) * kOpRing * static_cast<size_t>(c.max_seqs) * c.n_kv_heads));
+        CREATE_CUDA(cudaMemset(ctx->op_len_acc, 0, sizeof(int32_t) * kOpRing * static_cast<size_t>(c.max_seqs) * c.n_kv_heads));
+        CREATE_CUDA(cudaMalloc(&ctx->op_arrive, sizeof(uint32_t) * kOpRing));
+        CREATE_CUDA(cudaMemset(ctx->op_arrive, 0, sizeof(uint32_t) * kOpRing));
+        CREATE_CUDA(cudaMalloc(&ctx->op_scan_flag, sizeof(int32_t) * kOpRing));
+        CREATE_CUDA(cudaMemset(ctx->op_scan_flag, 0, sizeof(int32_t) * kOpRing));
+        CREATE_CUDA(cudaMalloc(&ctx->op_page0, sizeof(int32_t) * kOpRing * static_cast<size_t>(c.max_seqs) * c.n_kv_heads));
+    }
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
     CREATE_CUDA(cudaMallocHost(&ctx->status_host, sizeof(int32_t)));
@@ -986,17 +1150,8 @@ kvzap_status kvzap_prune_prefill(kvzap_ctx *ctx, const void *K, const void *V, c
     st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
     if (st != KVZAP_OK) return st;
     if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
-    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-    uint32_t *mask = next_mask_slice(ctx);
-    {
-        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
-        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
-                                                                         cu_seqlens, n_seqs, tau, w, 1, mask,
-                                                                         n_blocks * 4, nullptr);
-    }
-    KVZAP_CUDA(ctx, cudaGetLastError());
-    ctx->launches += 1;
-    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
+    return launch_prune_onepass(ctx, scores, nullptr, tau, w, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, 0, 0,
+                                0, 0, nullptr, nullptr, stream);
 }
 
 kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void *V, const float *scores,
@@ -1039,18 +1194,11 @@ kvzap_status kvzap_prune_prefill_topk(kvzap_ctx *ctx, const void *K, const void 
     KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, select_finish_kernel, n_tokens, static_cast<int>(c.n_kv_heads), cu_seqlens,
                                        static_cast<int>(n_seqs), static_cast<int>(w), keep_ratio, per_layer ? 1 : 0,
                                        static_cast<const uint32_t *>(ctx->select_hist), tau_list, ctx->status_dev));
-    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-    uint32_t *mask = next_mask_slice(ctx);
-    {
-        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
-        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(n_blocks)), dim3(128), 0, stream, early, 1);
-        KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, mask_kernel, scores, n_tokens, static_cast<int>(c.n_kv_heads), cu_seqlens,
-                                           static_cast<int>(n_seqs), 0.0f, static_cast<int>(w), 1, mask, n_blocks * 4,
-                                           static_cast<const float *>(tau_list)));
-    }
     KVZAP_CUDA(ctx, cudaGetLastError());
-    ctx->launches += 6;
-    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, false);
+    ctx->launches += 5;
+    // the same mask + compaction launch as kvzap_prune_prefill, with the cut values as per-list thresholds
+    return launch_prune_onepass(ctx, scores, tau_list, 0.0f, w, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, 0,
+                                0, 0, 0, nullptr, nullptr, stream);
 }
 
 // tok_major: K and V are [n_tokens][H][D] (the K/V projection's output) instead of [H][n_tokens][D]
@@ -1114,7 +1262,12 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)
     cudaMemsetAsync(ctx->tile_counters, 0, sizeof(int32_t) * kMaskRing, stream);
     if (ctx->split_arrive) cudaMemsetAsync(ctx->split_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
     if (ctx->wide_arrive) cudaMemsetAsync(ctx->wide_arrive, 0, sizeof(uint32_t) * static_cast<size_t>(ctx->sm_count), stream);
-    if (v == KVZAP_ERR_TIMEOUT) reset_step_counters(ctx, stream);
+    if (v == KVZAP_ERR_TIMEOUT) {
+        reset_step_counters(ctx, stream);
+        // a one-launch pruning call that gave up may have left its list-length sums and arrival count behind
+        cudaMemsetAsync(ctx->op_len_acc, 0, sizeof(int32_t) * kOpRing * static_cast<size_t>(ctx->cfg.max_seqs) * ctx->cfg.n_kv_heads, stream);
+        cudaMemsetAsync(ctx->op_arrive, 0, sizeof(uint32_t) * kOpRing, stream);
+    }
     cudaStreamSynchronize(stream);
     fail(ctx, static_cast<kvzap_status>(v), "device-side condition %d recorded", v);
     return static_cast<kvzap_status>(v);
@@ -1455,19 +1608,8 @@ kvzap_status kvzap_prune_prefill_paged(kvzap_ctx *ctx, const void *K, const void
                           max_pages_per_list, lengths, n_pages_used, w);
     if (st != KVZAP_OK) return st;
     if (!scores) return fail(ctx, KVZAP_ERR_INVALID_ARG, "scores is NULL");
-    const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-    uint32_t *mask = next_mask_slice(ctx);
-    {
-        ProfScope prof(ctx, KVZAP_KERNEL_MASK, stream);
-        mask_kernel<<<static_cast<unsigned>(n_blocks), 128, 0, stream>>>(scores, n_tokens, ctx->cfg.n_kv_heads,
-                                                                         cu_seqlens, n_seqs, tau, w, 1, mask,
-                                                                         n_blocks * 4, nullptr);
-    }
-    KVZAP_CUDA(ctx, cudaGetLastError());
-    ctx->launches += 1;
-    return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
-                                   first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream, nullptr,
-                                   false, false, false);
+    return launch_prune_onepass(ctx, scores, nullptr, tau, w, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, lengths,
+                                page_tokens, first_page, n_pages_pool, max_pages_per_list, page_table, n_pages_used, stream);
 }
 
 static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K,

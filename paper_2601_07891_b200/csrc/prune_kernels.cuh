@@ -98,7 +98,111 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
 }
 
 // ---------------------------------------------------------------------------
-// One CTA of 1024 threads.  blockprefix [H][n_blocks+1], seqbase [H][n_seqs+1] (both nullptr when only the
+// Page assignment of the paged output, by all NT threads of one CTA: list idx (= b * n_heads + h) needs
+// ceil(lengths[idx] / page_tokens) pages (less those it owns already when appending); list_page0 receives the
+// exclusive scan of the needs plus first_page, *n_pages_used the total; a pool or table that is too small
+// sets the status word, marks every list with list_page0 = -1 and (append) restores the old lengths.
+// fill_table != 0: the page numbers are also entered into page_table here; otherwise the caller does
+// that (fill_page_table), e.g. spread over many CTAs.  Arguments as scan_lists.
+template <int NT>
+__device__ __forceinline__ void
+assign_pages(int n_heads, int n_seqs, int32_t *__restrict__ lengths, int page_tokens, int32_t first_page,
+             int64_t n_pages_pool, int max_pages, int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table,
+             int32_t *__restrict__ n_pages_used, int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
+             int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top,
+             int fill_table)
+{
+    __shared__ int32_t warp_sums[32];
+    __shared__ int32_t carry_s;
+    __shared__ int32_t fail_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    auto block_scan = [&](int32_t v, int32_t &total) -> int32_t {   // inclusive scan over the CTA
+        int32_t x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int32_t y = __shfl_up_sync(0xffffffffu, x, o);
+            if (lane >= o) x += y;
+        }
+        __syncthreads();
+        if (lane == 31) warp_sums[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            int32_t w = lane < NT / 32 ? warp_sums[lane] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int32_t y = __shfl_up_sync(0xffffffffu, w, o);
+                if (lane >= o) w += y;
+            }
+            warp_sums[lane] = w;
+        }
+        __syncthreads();
+        total = warp_sums[31];
+        return x + (warp > 0 ? warp_sums[warp - 1] : 0);
+    };
+    // paged output: exclusive scan of the per-list page counts in (b,h) order
+    __syncthreads();
+    if (tid == 0) { carry_s = 0; fail_s = 0; }
+    __syncthreads();
+    const int n_lists = n_heads * n_seqs;
+    for (int base = 0; base < n_lists; base += NT) {
+        const int idx = base + tid;
+        int32_t need = 0;
+        if (idx < n_lists) {
+            need = (lengths[idx] + page_tokens - 1) / page_tokens;
+            if (need > max_pages) fail_s = 1;
+            if (append) need -= (list_base[idx] + page_tokens - 1) / page_tokens;     // pages the list already owns
+        }
+        int32_t total;
+        const int32_t incl = block_scan(need, total);
+        const int32_t carry = carry_s;
+        if (idx < n_lists) list_page0[idx] = first_page + carry + incl - need;
+        __syncthreads();
+        if (tid == 0) carry_s = carry + total;
+        __syncthreads();
+    }
+    const int32_t used = carry_s;
+    int32_t n_free = 0;
+    if (page_cursor != nullptr && free_top != nullptr) {
+        n_free = *free_top;
+        if (n_free < 0) n_free = 0;
+    }
+    const int32_t from_stack = used < n_free ? used : n_free;
+    const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + (used - from_stack) > n_pages_pool;
+    if (fail) {
+        for (int idx = tid; idx < n_lists; idx += NT) {
+            list_page0[idx] = -1;
+            if (append) lengths[idx] = list_base[idx];
+        }
+        if (tid == 0) {
+            atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
+            if (n_pages_used != nullptr) *n_pages_used = 0;
+        }
+        return;
+    }
+    __syncthreads();      // every thread has read the cursor and the stack height
+    if (tid == 0) {
+        if (n_pages_used != nullptr) *n_pages_used = used;
+        if (page_cursor != nullptr) *page_cursor = first_page + used - from_stack;
+        if (from_stack > 0) *free_top = n_free - from_stack;
+    }
+    __syncthreads();      // list_page0 and lengths of all lists are final
+    if (!fill_table) return;
+    for (int idx = warp; idx < n_lists; idx += NT / 32) {            // a warp per list
+        const int32_t p0 = list_page0[idx];
+        const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
+        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
+        for (int32_t i = lane; i < need; i += 32) {
+            const int32_t j = p0 - first_page + i;            // ordinal among the pages assigned by this call
+            page_table[static_cast<int64_t>(idx) * max_pages + have + i] =
+                j < from_stack ? free_stack[n_free - 1 - j] : first_page + (j - from_stack);
+        }
+    }
+}
+
+
+
+// ---------------------------------------------------------------------------
+// One CTA of NT threads (all of them call it).  blockprefix [H][n_blocks+1], seqbase [H][n_seqs+1] (both nullptr when only the
 // lengths and the page assignment are wanted: the lists are then counted directly), lengths [n_seqs][H].
 // Paged output (page_tokens > 0): list (b,h) gets
 // ceil(len/page_tokens) pages numbered contiguously from first_page in (b,h)
@@ -113,8 +217,9 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
 // (free_stack / free_top, may be nullptr), then from the cursor: the pages of a list are then not
 // consecutive numbers and the compaction finds them through the table; list_page0 is the ordinal of
 // the list's first new page among the pages this call assigns (plus first_page), or -1.
-__global__ void __launch_bounds__(1024)
-scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
+template <int NT>
+__device__ __forceinline__ void
+scan_lists(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
             const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens,
             int32_t *__restrict__ blockprefix, int32_t *__restrict__ seqbase, int32_t *__restrict__ lengths,
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
@@ -122,15 +227,11 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
             int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top)
 {
-    // may be placed before the kernel that writes the mask has finished; waits for it here
-    griddep_launch_dependents();
-    griddep_wait();
     // page_cursor != nullptr: the first page comes from (and the pages used are added to) a device-side
     // allocator cursor instead of the first_page argument
     if (page_tokens > 0 && page_cursor != nullptr) first_page = *page_cursor;
     __shared__ int32_t warp_sums[32];
     __shared__ int32_t carry_s;
-    __shared__ int32_t fail_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     auto block_scan = [&](int32_t v, int32_t &total) -> int32_t {   // inclusive scan over the CTA
@@ -144,7 +245,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         if (lane == 31) warp_sums[warp] = x;
         __syncthreads();
         if (warp == 0) {
-            int32_t w = warp_sums[lane];
+            int32_t w = lane < NT / 32 ? warp_sums[lane] : 0;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const int32_t y = __shfl_up_sync(0xffffffffu, w, o);
@@ -161,9 +262,9 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
         // Only the lengths are wanted (the compaction counts its own prefixes): every list's kept rows are
         // counted straight from the mask words of its token range, a group of threads per list.
         const int n_lists_all = n_heads * n_seqs;
-        int per_list = 1024;
-        while (per_list > 32 && 1024 / per_list < n_lists_all) per_list >>= 1;
-        const int n_groups = 1024 / per_list, grp = tid / per_list, gt = tid % per_list;
+        int per_list = NT;
+        while (per_list > 32 && NT / per_list < n_lists_all) per_list >>= 1;
+        const int n_groups = NT / per_list, grp = tid / per_list, gt = tid % per_list;
         __shared__ int32_t group_sum[32];
         for (int idx0 = 0; idx0 < n_lists_all; idx0 += n_groups) {
             if (tid < 32) group_sum[tid] = 0;
@@ -197,7 +298,7 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     for (int h = 0; h < n_heads; ++h) {
         if (tid == 0) carry_s = 0;
         __syncthreads();
-        for (int64_t base = 0; base < n_blocks; base += 1024) {
+        for (int64_t base = 0; base < n_blocks; base += NT) {
             const int64_t blk = base + tid;
             int32_t cnt = 0;
             if (blk < n_blocks) {
@@ -216,13 +317,13 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     }
     __syncthreads();      // blockprefix written by this CTA is visible to it from here on
 
-    for (int idx = tid; idx < n_heads * (n_seqs + 1); idx += 1024) {
+    for (int idx = tid; idx < n_heads * (n_seqs + 1); idx += NT) {
         const int h = idx / (n_seqs + 1), b = idx % (n_seqs + 1);
         const int64_t t = cu_seqlens != nullptr ? static_cast<int64_t>(cu_seqlens[b]) : (b == 0 ? 0 : n_tokens);
         seqbase[idx] = kept_before(maskbits, n_words, blockprefix, n_blocks, h, t);
     }
     __syncthreads();
-    for (int idx = tid; idx < n_heads * n_seqs; idx += 1024) {
+    for (int idx = tid; idx < n_heads * n_seqs; idx += NT) {
         const int b = idx / n_heads, h = idx % n_heads;
         const int32_t old = append ? lengths[idx] : 0;
         if (append) list_base[idx] = old;
@@ -230,64 +331,28 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
     }
     }
     if (page_tokens <= 0) return;
+    __syncthreads();
+    assign_pages<NT>(n_heads, n_seqs, lengths, page_tokens, first_page, n_pages_pool, max_pages, list_page0, page_table,
+                     n_pages_used, page_cursor, status, append, list_base, free_stack, free_top, 1);
+}
 
-    // paged output: exclusive scan of the per-list page counts in (b,h) order
-    __syncthreads();
-    if (tid == 0) { carry_s = 0; fail_s = 0; }
-    __syncthreads();
-    const int n_lists = n_heads * n_seqs;
-    for (int base = 0; base < n_lists; base += 1024) {
-        const int idx = base + tid;
-        int32_t need = 0;
-        if (idx < n_lists) {
-            need = (lengths[idx] + page_tokens - 1) / page_tokens;
-            if (need > max_pages) fail_s = 1;
-            if (append) need -= (list_base[idx] + page_tokens - 1) / page_tokens;     // pages the list already owns
-        }
-        int32_t total;
-        const int32_t incl = block_scan(need, total);
-        const int32_t carry = carry_s;
-        if (idx < n_lists) list_page0[idx] = first_page + carry + incl - need;
-        __syncthreads();
-        if (tid == 0) carry_s = carry + total;
-        __syncthreads();
-    }
-    const int32_t used = carry_s;
-    int32_t n_free = 0;
-    if (page_cursor != nullptr && free_top != nullptr) {
-        n_free = *free_top;
-        if (n_free < 0) n_free = 0;
-    }
-    const int32_t from_stack = used < n_free ? used : n_free;
-    const bool fail = fail_s != 0 || static_cast<int64_t>(first_page) + (used - from_stack) > n_pages_pool;
-    if (fail) {
-        for (int idx = tid; idx < n_lists; idx += 1024) {
-            list_page0[idx] = -1;
-            if (append) lengths[idx] = list_base[idx];
-        }
-        if (tid == 0) {
-            atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
-            if (n_pages_used != nullptr) *n_pages_used = 0;
-        }
-        return;
-    }
-    __syncthreads();      // every thread has read the cursor and the stack height
-    if (tid == 0) {
-        if (n_pages_used != nullptr) *n_pages_used = used;
-        if (page_cursor != nullptr) *page_cursor = first_page + used - from_stack;
-        if (from_stack > 0) *free_top = n_free - from_stack;
-    }
-    __syncthreads();      // list_page0 and lengths of all lists are final
-    for (int idx = warp; idx < n_lists; idx += 32) {            // a warp per list
-        const int32_t p0 = list_page0[idx];
-        const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
-        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
-        for (int32_t i = lane; i < need; i += 32) {
-            const int32_t j = p0 - first_page + i;            // ordinal among the pages assigned by this call
-            page_table[static_cast<int64_t>(idx) * max_pages + have + i] =
-                j < from_stack ? free_stack[n_free - 1 - j] : first_page + (j - from_stack);
-        }
-    }
+// The page assignment as a kernel of its own: one CTA of 1024 threads (behind the fused scoring kernels
+// and for appending to a cache's lists).
+__global__ void __launch_bounds__(1024)
+scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blocks, int n_heads,
+            const int32_t *__restrict__ cu_seqlens, int n_seqs, int64_t n_tokens,
+            int32_t *__restrict__ blockprefix, int32_t *__restrict__ seqbase, int32_t *__restrict__ lengths,
+            int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
+            int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
+            int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
+            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top)
+{
+    // may be placed before the kernel that writes the mask has finished; waits for it here
+    griddep_launch_dependents();
+    griddep_wait();
+    scan_lists<1024>(maskbits, n_words, n_blocks, n_heads, cu_seqlens, n_seqs, n_tokens, blockprefix, seqbase, lengths,
+                     page_tokens, first_page, n_pages_pool, max_pages, list_page0, page_table, n_pages_used, page_cursor,
+                     status, append, list_base, free_stack, free_top);
 }
 
 // ---------------------------------------------------------------------------

@@ -224,3 +224,55 @@ def test_larger_tau_keeps_a_subset_on_the_gpu(binding, oracle):
                 assert kept[h] <= prev[h]
         prev = kept
     ctx.close()
+
+
+@pytest.mark.parametrize("seq_lens,H,D,P", [
+    ([131072 + 77], 8, 128, 0),                         # more blocks than CTAs: several blocks per CTA
+    ([40000, 1, 0, 50011, 129, 30000], 8, 64, 0),       # sequences that start inside a CTA's run of blocks
+    ([131072 + 77], 8, 128, 16),                        # the same, paged: the last CTA to arrive assigns the pages
+    ([40000, 1, 0, 50011, 129, 30000], 5, 64, 16),
+    ([2600000, 17], 2, 8, 0),                           # more than 32 blocks per CTA: mask words re-read from memory
+    ([2600000, 17], 2, 8, 5),
+])
+def test_prune_prefill_one_launch_many_blocks_per_cta(binding, oracle, seq_lens, H, D, P):
+    """kvzap_prune_prefill / _paged on given scores at sizes where a CTA of the one-launch kernel owns
+    several (and more than 32) blocks and sequences begin in the middle of a CTA's run; lengths, rows,
+    page tables and untouched memory bit for bit against the oracle's mask and ordered gather."""
+    T, B, tau, w = int(sum(seq_lens)), len(seq_lens), 0.43, 128
+    ctx = binding.Kvzap(256, 0, H, D, 1, T, max_seqs=B, trusted_producers=True)
+    g = torch.Generator(device="cuda").manual_seed(T % 1000 + H)
+    scores = torch.randn(T, H, generator=g, device="cuda")
+    K, V = synth.keys_values(H, T, D, seed=3, device="cuda")
+    cu = synth.cu_seqlens(seq_lens)
+    cu_dev = torch.from_numpy(cu).cuda() if B > 1 else None
+    cu_arg = cu if B > 1 else None
+    s_np = scores.cpu().numpy()
+    for rep in range(2):                                # twice in a row: the second launch starts under the first
+        if P == 0:
+            K_out, V_out = parity.poison_like(K), parity.poison_like(V)
+            lengths = torch.full((B, H), -1, dtype=torch.int32, device="cuda")
+            binding.kvzap_prune_prefill(ctx.handle, K, V, scores, cu_dev, B, tau, w, K_out, V_out, lengths)
+        else:
+            n_pool, max_pages, first_page = H * (T // P + B + 1) // 2 + 7, max(seq_lens) // P + 2, 3
+            K_pool = torch.full((n_pool, P, D), -5.0, dtype=torch.bfloat16, device="cuda")
+            V_pool = torch.full((n_pool, P, D), -5.0, dtype=torch.bfloat16, device="cuda")
+            table = torch.full((B * H, max_pages), -1, dtype=torch.int32, device="cuda")
+            lengths = torch.zeros(B, H, dtype=torch.int32, device="cuda")
+            used = torch.zeros(1, dtype=torch.int32, device="cuda")
+            binding.kvzap_prune_prefill_paged(ctx.handle, K, V, scores, cu_dev, B, tau, w, K_pool, V_pool, P, first_page,
+                                              table, lengths, used)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    if P == 0:
+        parity.check_compaction(oracle, K.cpu(), V.cpu(), s_np, tau, w, cu_arg, K_out.cpu(), V_out.cpu(), lengths)
+    else:
+        keep = oracle.keep_mask(s_np, tau, w, cu_arg)
+        fill = int(synth.bits(torch.tensor([-5.0], dtype=torch.bfloat16))[0])
+        Kp, Vp, tab, ln, n_used = oracle.compact_paged(synth.bits(K), synth.bits(V), keep, P, n_pool, max_pages,
+                                                       cu_seqlens=cu_arg, first_page=first_page, fill=fill)
+        np.testing.assert_array_equal(lengths.cpu().numpy(), ln)
+        assert int(used.item()) == n_used
+        np.testing.assert_array_equal(table.cpu().numpy(), tab)
+        np.testing.assert_array_equal(synth.bits(K_pool), Kp)
+        np.testing.assert_array_equal(synth.bits(V_pool), Vp)
+    ctx.close()
