@@ -8,7 +8,10 @@ layer = B*T / (step time / n_layers).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
 
-Prints ONE JSON line.  ``--impl reference`` times the CPU oracle (as it
+Prints ONE JSON line.  Without ``--workload`` the line is that of the largest
+single-GPU workload (Qwen3-32B shape, 128k tokens, 64 layers, paged output) and
+carries, under ``configs``, a short record of each of the other four workloads
+measured in the same process.  ``--impl reference`` times the CPU oracle (as it
 stands) on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -28,9 +31,13 @@ if ROOT not in sys.path:
 METRIC = "tokens pruned/sec per layer"
 UNIT = "tokens/s/layer"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (bytes); None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {"qwen3_8b_prefill_32k": 276.8e6, "qwen3_8b_decode_b128": 227.9e6}
+HEADLINE = "qwen3_32b_prefill_128k_paged"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, taken from the ncu
+# capture summarised in the named file under profiles/ (bytes per launch; not measured in this run).
+NCU_TRAFFIC = {
+    "qwen3_8b_prefill_32k": (276.8e6, "profiles/score_kernel_mlp_qwen3_8b_prefill_32k.md"),
+    "qwen3_8b_decode_b128": (227.9e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
+}
 # attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
 NCU_ATTENTION_TRAFFIC_RATIO = 2.409 / 2.3986
 
@@ -72,6 +79,14 @@ def live_gemm_tflops(dev, seconds=1.5):
         t_total += last
         done += reps
     return per * reps / (last * 1e-3) / 1e12          # the last block of launches: the settled rate
+
+
+def pick_tensor_peak(peaks, clocks):
+    """Which measured cuBLAS figure the timed region is compared with: the burst one when the region ran
+    at (nearly) full SM clock with no power cap seen, the sustained one otherwise."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    burst = bool(mhz and mx and mhz >= 0.95 * mx and "sw_power_cap" not in clocks.get("reasons", []))
+    return ("burst", peaks["bf16_tflops"]) if burst else ("sustained", peaks["bf16_tflops_sustained"])
 
 
 def surrogate_flops_per_token(wl):
@@ -182,10 +197,10 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
-def _roofline_times(wl, n_tokens, kept_rows, peaks):
+def _roofline_times(wl, n_tokens, kept_rows, peaks, tensor_peak):
     """(tensor time, HBM time of the scoring kernel's bytes, HBM time of all algorithmic bytes) of one layer, seconds."""
     flops = surrogate_flops_per_token(wl) * n_tokens
-    t_tensor = flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_tensor = flops / (tensor_peak * 1e12)
     score_bytes = n_tokens * wl.d_model * 2 + n_tokens * wl.n_kv_heads * 4
     t_hbm_score = score_bytes / (peaks["hbm_gbs"] * 1e9)
     t_hbm_layer = algorithmic_bytes_per_layer(wl, n_tokens, kept_rows) / (peaks["hbm_gbs"] * 1e9)
@@ -205,8 +220,9 @@ def _timed(fn, n, stream_sync):
     return e0.elapsed_time(e1) / n
 
 
-def run_prefill(args, wl, env):
-    """Prefill workloads: one step = the fused hot path (scoring, mask, compaction) over every layer."""
+def run_prefill(args, wl, env, sub=False):
+    """Prefill workloads: one step = the fused hot path (scoring, mask, compaction) over every layer.
+    sub: a short record for the `configs` list (no end-to-end leg, no live cuBLAS loop)."""
     import torch
     from paper_2601_07891_b200 import binding, synth
     dev, rank, world, barrier = env["dev"], env["rank"], env["world"], env["barrier"]
@@ -222,7 +238,7 @@ def run_prefill(args, wl, env):
     # resident inputs, one set per layer while they fit (every layer's inputs exceed L2, so no flush is
     # needed); beyond ~60 GB the layers rotate over fewer input sets (weights stay distinct per layer)
     per_layer_bytes = n_tokens * wl.d_model * 2 + 4 * H * n_tokens * D * 2
-    n_sets = L if L * per_layer_bytes <= 60e9 else max(2, int(60e9 // per_layer_bytes))
+    n_sets = L if L * per_layer_bytes <= 60e9 else max(2, int(40e9 // per_layer_bytes))
     # a small workload (config 1: 56 MB per layer) would otherwise run out of the 126 MB L2: rotate over
     # enough input/output sets that 2.5 x L2 lies between two uses of the same buffer
     n_sets = max(n_sets, int(-(-2.5 * 126e6 // per_layer_bytes)))
@@ -286,20 +302,24 @@ def run_prefill(args, wl, env):
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during warm-up")
 
+    n_steps = args.steps
+    if sub:
+        # enough steps that the region is not a burst: at least ~0.3 s for the tensor-bound workloads
+        n_steps = max(args.steps, 100 if wl.surrogate == "mlp" else 20, 2000 if L == 1 else 0)
     sampler = ClockSampler(dev.index)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = ctx.launch_count()
     sampler.start()
     barrier()
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(n_steps):
         step()
     e1.record()
     barrier()
     clocks = sampler.stop()
     total_ms = env["max_over_ranks"](e0.elapsed_time(e1))
     gpu_launches = ctx.launch_count() - launches0
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / n_steps
     layer_ms = ms_per_step / L
     value = world * n_tokens / (layer_ms * 1e-3)
     if ctx.poll_status() != 0:
@@ -309,7 +329,7 @@ def run_prefill(args, wl, env):
     # The two kernels of a layer, each timed alone with CUDA events around a loop of launches through
     # the public calls (scoring only; mask + compaction on the scores just computed).
     sync = torch.cuda.synchronize
-    n_rep = max(1, min(args.steps, 5))
+    n_rep = max(1, min(n_steps, 5))
     def score_only():
         for l in range(L):
             i = (turn[0] + l) % n_bufs
@@ -330,17 +350,22 @@ def run_prefill(args, wl, env):
     prune_ms = _timed(prune, n_rep, sync) / n_bufs if prune else None
 
     peaks, peak_src = load_peaks()
-    flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer = _roofline_times(wl, n_tokens, kept_rows, peaks)
+    peak_kind, tensor_peak = pick_tensor_peak(peaks, clocks)
+    flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer = _roofline_times(wl, n_tokens, kept_rows, peaks, tensor_peak)
     # Dominant kernel = the scoring kernel.  Its launch duration inside the timed region cannot be
     # separated from the compaction that runs beside it, so the layer period (step time / layers) is
     # used: an upper bound of the kernel's own duration.  `alone_ms` is the same kernel in a loop of
     # scoring-only launches.
     if t_tensor >= t_hbm_score:
         achieved = flops / (layer_ms * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"],
-                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops_sustained"],
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": tensor_peak,
+                    "unit": "TFLOP/s", "frac": achieved / tensor_peak,
+                    "peak_kind": peak_kind + " cuBLAS bf16 figure, chosen from this run's clock record (burst: median SM "
+                                             "clock within 5 % of max and no sw_power_cap sample)",
+                    "frac_of_burst": achieved / peaks["bf16_tflops"],
+                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                     "alone_achieved": flops / (score_ms * 1e-3) / 1e12}
-        if not args.skip_live_peak:
+        if not args.skip_live_peak and not sub:
             # the GPUs of the pool settle at different clocks under the power cap: the same loop on this one, now
             live = live_gemm_tflops(dev)
             roofline["live_cublas_bf16_tflops_sustained"] = live
@@ -349,7 +374,10 @@ def run_prefill(args, wl, env):
         achieved = score_bytes / (layer_ms * 1e-3) / 1e9
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "alone_achieved": score_bytes / (score_ms * 1e-3) / 1e9}
-    roofline.update({"traffic": NCU_TRAFFIC_BYTES.get(wl.name), "kernel": "score_kernel", "peak_source": peak_src,
+    traffic = NCU_TRAFFIC.get(wl.name) if args.layers == 0 and not proj else None
+    roofline.update({"traffic": traffic[0] if traffic else None,
+                     "traffic_source": (traffic[1] + " (ncu capture, not measured in this run)") if traffic else None,
+                     "kernel": "score_kernel", "peak_source": peak_src,
                      "kernel_ms": layer_ms, "alone_ms": score_ms,
                      "note": "kernel_ms = layer period in the timed region (compaction overlaps the next "
                              "layer's scoring kernel); alone_ms = scoring-only launches back to back"})
@@ -367,28 +395,37 @@ def run_prefill(args, wl, env):
               "l2": "inputs larger than L2 (distinct resident buffers per layer; small workloads rotate over "
                     "enough sets that 2.5 x L2 lies between two uses of a buffer)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps,
             "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
             "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
 
-    if rank == 0 and world == 1 and not args.skip_e2e and not P and not proj:
-        # end to end through the host-buffer entry point: H2D of the layer's inputs and D2H of its
-        # result happen inside the timed region; host inputs rotate over a few pinned layer sets
+    if rank == 0 and world == 1 and not args.skip_e2e and not proj and not sub:
+        # End to end through the host-buffer entry point: one call per step takes every layer's inputs from
+        # pinned host memory and leaves every layer's result there; the copies happen inside the call (layer
+        # l + 1 is copied in while layer l is computed and copied out).  Host inputs rotate over two layer sets.
         n_h = min(L, 2)
         hX = [Xs[i].cpu().pin_memory() for i in range(n_h)]
         hK = [Ks[i].cpu().pin_memory() for i in range(n_h)]
         hV = [Vs[i].cpu().pin_memory() for i in range(n_h)]
-        hKo, hVo = torch.empty_like(hK[0]).pin_memory(), torch.empty_like(hV[0]).pin_memory()
-        hlen = torch.zeros(B, H, dtype=torch.int32).pin_memory()
+        if P:
+            hKo = torch.empty(pool_pages, P, D, dtype=torch.bfloat16).pin_memory()
+            hVo = torch.empty(pool_pages, P, D, dtype=torch.bfloat16).pin_memory()
+            htab = torch.zeros(B * H, max_pages, dtype=torch.int32).pin_memory()
+            hused = torch.zeros(1, dtype=torch.int32).pin_memory()
+        else:
+            hKo, hVo = torch.empty_like(hK[0]).pin_memory(), torch.empty_like(hV[0]).pin_memory()
+            htab = hused = None
+        hlen = [torch.zeros(B, H, dtype=torch.int32).pin_memory() for _ in range(L)]
         hcu = torch.from_numpy(synth.cu_seqlens([T] * B)) if B > 1 else None
         e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        lists = dict(hidden=[hX[l % n_h] for l in range(L)], K=[hK[l % n_h] for l in range(L)],
+                     V=[hV[l % n_h] for l in range(L)], K_out=[hKo] * L, V_out=[hVo] * L)
 
         def e2e_step():
-            for l in range(L):
-                i = l % n_h
-                binding.kvzap_prefill_fused_host(ctx.handle, l, hX[i], hK[i], hV[i], hcu, B, wl.tau, wl.window,
-                                                 hKo, hVo, hlen, None)
+            binding.kvzap_prefill_layers_host(ctx.handle, 0, lists["hidden"], lists["K"], lists["V"], hcu, B, wl.tau, wl.window,
+                                              lists["K_out"], lists["V_out"], hlen, None, page_tokens=P,
+                                              page_table=[htab] * L if P else None, n_pages_used=[hused] * L if P else None)
         e2e_step()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -396,17 +433,31 @@ def run_prefill(args, wl, env):
             e2e_step()
         torch.cuda.synchronize()
         e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-        h2d = L * (n_tokens * wl.d_model * 2 + 2 * H * n_tokens * D * 2 + (4 * (B + 1) if B > 1 else 0))
-        d2h = int(L * (kept_rows * 2 * D * 2 + B * H * 4))
+        # the rate of a plain pinned-host-to-device copy of one layer's hidden states on this machine, for comparison
+        t0 = time.perf_counter()
+        for _ in range(3):
+            Xs[0].copy_(hX[0], non_blocking=True)
+        torch.cuda.synchronize()
+        h2d_rate = 3 * hX[0].numel() * 2 / (time.perf_counter() - t0) / 1e9
+        h2d = L * (n_tokens * wl.d_model * 2 + 2 * H * n_tokens * D * 2 + (B * H * max_pages * 4 if P else 0)) + \
+            (4 * (B + 1) if B > 1 else 0)
+        kept_e2e = float(sum(int(x.sum()) for x in hlen)) / L
+        if P:
+            d2h = int(L * (int(hused.item()) * P * 2 * D * 2 + B * H * max_pages * 4 + B * H * 4 + 4))
+        else:
+            d2h = int(L * (kept_e2e * 2 * D * 2 + B * H * 4))
         line["e2e"] = {"value": n_tokens / (e2e_ms * 1e-3 / L), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                       "note": "kvzap_prefill_fused_host: pinned host buffers, copies inside the timed region"}
-        del hX, hK, hV, hKo, hVo
+                       "h2d_GBps_achieved": h2d / (e2e_ms * 1e-3) / 1e9, "h2d_GBps_plain_copy": h2d_rate,
+                       "frac_of_plain_h2d_copy": h2d / (e2e_ms * 1e-3) / 1e9 / h2d_rate,
+                       "note": "kvzap_prefill_layers_host, all layers in one call: pinned host buffers, copies inside the "
+                               "timed region and overlapped with the kernels of the neighbouring layers"}
+        del hX, hK, hV, hKo, hVo, lists
     ctx.close()
     return line
 
 
-def run_decode(args, wl, env):
+def run_decode(args, wl, env, sub=False):
     """Decode workload: one step = one decode step (score the new token of every sequence with every
     layer's surrogate, append, decide the token leaving the window) over all layers."""
     import numpy as np
@@ -420,7 +471,8 @@ def run_decode(args, wl, env):
     for l in range(L):
         ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
     n_lists = B * L * H
-    total_steps = w + max(args.warmup, 3) + args.steps + 8
+    n_steps = max(args.steps, 1000) if sub else args.steps
+    total_steps = w + max(args.warmup, 3) + n_steps + 8 + (max(args.e2e_steps, 10) + 3 if not args.skip_e2e and not sub else 0)
     # Pre-pruned caches: per-list prefix lengths uniform in [prefix_min, prefix_max].  Decoding never
     # reads a list's earlier pages, so only each list's last (partly filled) page and the pages it can
     # grow into are backed by memory; lengths and page tables carry the full logical sizes.
@@ -466,19 +518,19 @@ def run_decode(args, wl, env):
     sampler.start()
     barrier()
     e0.record()
-    for _ in range(args.steps):
+    for _ in range(n_steps):
         step()
     e1.record()
     barrier()
     clocks = sampler.stop()
     total_ms = env["max_over_ranks"](e0.elapsed_time(e1))
     gpu_launches = ctx.launch_count() - launches0
-    ms_per_step = total_ms / args.steps
+    ms_per_step = total_ms / n_steps
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during the timed region")
     len1 = torch.zeros_like(len0)
     binding.kvzap_cache_lengths(ctx.handle, cache, len1)
-    kept_exit = float((len1 - len0).sum().item()) / (args.steps * n_lists)     # fraction of exiting tokens kept
+    kept_exit = float((len1 - len0).sum().item()) / (n_steps * n_lists)     # fraction of exiting tokens kept
     value = world * B / (ms_per_step * 1e-3 / L)
 
     peaks, peak_src = load_peaks()
@@ -490,7 +542,10 @@ def run_decode(args, wl, env):
                    + kept_exit * B * H * 2 * row * 2)                  # kept exiting rows: window -> page
     achieved = bytes_layer * L / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(wl.name),
+                "frac": achieved / peaks["hbm_gbs"],
+                "traffic": NCU_TRAFFIC[wl.name][0] if wl.name in NCU_TRAFFIC and args.layers == 0 else None,
+                "traffic_source": (NCU_TRAFFIC[wl.name][1] + " (ncu capture, not measured in this run)")
+                if wl.name in NCU_TRAFFIC and args.layers == 0 else None,
                 "kernel": "score_split_kernel (scoring + cache update in one launch)", "peak_source": peak_src,
                 "kernel_ms": ms_per_step, "algorithmic_bytes_per_step": bytes_layer * L}
     config = {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
@@ -499,13 +554,14 @@ def run_decode(args, wl, env):
               "l2": "weights of all layers (151 MB) exceed L2; per-step inputs rotate over %d sets" % n_sets,
               "backing": "only each list's last page and growth pages are backed (decode never reads earlier pages)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": n_warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
             "gpu_launches": int(gpu_launches), "roofline": roofline,
             "breakdown": {"layer_us": ms_per_step * 1e3 / L, "layer_roofline_us": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
+                          "layer_frac_of_roofline": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e3 / (ms_per_step / L),
                           "kept_fraction_of_exiting_tokens": kept_exit}}
-    if rank == 0 and world == 1 and not args.skip_e2e:
+    if rank == 0 and world == 1 and not args.skip_e2e and not sub:
         # End to end: the step's inputs start in pinned host memory and its scores end there; the copies
         # (torch, on the stream of the call) are inside the timed region.
         hX = [x.cpu().pin_memory() for x in Xs[:2]]
@@ -667,8 +723,29 @@ def make_env(backend="nccl"):
             "close": close}
 
 
-def run_ours(args, wl):
+def summarise(line):
+    """The short record of one workload for the headline line's `configs` list."""
+    bd, rf = line["breakdown"], line["roofline"]
+    rec = {"workload": line["config"]["workload"], "value": line["value"], "unit": line["unit"], "steps": line["steps"],
+           "ms_per_step": line["ms_per_step"], "layer_frac_of_roofline": bd.get("layer_frac_of_roofline"),
+           "roofline_bound": rf["bound"], "roofline_frac": rf["frac"], "clocks": line["clocks"],
+           "gpu_launches": line["gpu_launches"]}
+    if "layer_ms" in bd:
+        rec.update({"ms_per_layer": bd["layer_ms"], "layer_roofline_ms": bd["layer_roofline_ms"],
+                    "kept_fraction": bd["kept_fraction"], "compaction_alone_GBps": bd.get("compaction_alone_GBps")})
+        if rf["bound"] == "tensor":
+            rec.update({"peak_kind": rf["peak_kind"].split(" ")[0], "frac_of_burst": rf["frac_of_burst"],
+                        "frac_of_sustained": rf["frac_of_sustained"]})
+    else:
+        rec.update({"ms_per_layer": bd["layer_us"] * 1e-3, "layer_roofline_ms": bd["layer_roofline_us"] * 1e-3,
+                    "kept_fraction_of_exiting_tokens": bd["kept_fraction_of_exiting_tokens"]})
+    return rec
+
+
+def run_ours(args, wl, with_configs):
+    import gc
     import torch
+    from paper_2601_07891_b200 import synth
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
     env = make_env("nccl")
@@ -686,6 +763,23 @@ def run_ours(args, wl):
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": "%d layer(s), first %d tokens of each: scoring + mask + compaction (%.1f s)"
                                           % (n_l, n_sample, dt)}
+    if with_configs and world == 1 and not args.attention:
+        # the other workloads, each in full, in the same process (short records; the headline is the line itself)
+        records = []
+        for idx, name in enumerate(synth.WORKLOAD_ORDER):
+            if name == wl.name:
+                continue
+            gc.collect()
+            torch.cuda.empty_cache()
+            sub_wl = synth.WORKLOADS[name]
+            saved = args.workload_index
+            args.workload_index = idx + 1
+            try:
+                sub = run_decode(args, sub_wl, env, sub=True) if sub_wl.decode_steps > 0 else run_prefill(args, sub_wl, env, sub=True)
+                records.append(summarise(sub))
+            finally:
+                args.workload_index = saved
+        line["configs"] = records
     if rank == 0:
         print(json.dumps(line), flush=True)
     env["close"]()
@@ -698,7 +792,9 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="qwen3_8b_prefill_32k", choices=list(synth.WORKLOAD_ORDER))
+    ap.add_argument("--workload", default=None, choices=list(synth.WORKLOAD_ORDER),
+                    help="one workload only (default: the largest, %s, plus short records of the other four)" % HEADLINE)
+    ap.add_argument("--no-configs", action="store_true", help="default run: leave the other four workloads out")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (small case for profiling)")
     ap.add_argument("--kv-layout", default="heads", choices=["heads", "proj"],
@@ -712,6 +808,9 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=32768,
                     help="tokens of one layer the CPU oracle is timed on (bounded sample)")
     args = ap.parse_args()
+    with_configs = args.workload is None and not args.no_configs and args.layers == 0
+    if args.workload is None:
+        args.workload = HEADLINE
     args.workload_index = synth.WORKLOAD_ORDER.index(args.workload) + 1
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
@@ -719,7 +818,7 @@ def main():
             args.ref_tokens = min(args.ref_tokens, 4096)     # keep the whole run within minutes
         run_reference(args, wl)
     else:
-        run_ours(args, wl)
+        run_ours(args, wl, with_configs)
 
 
 if __name__ == "__main__":

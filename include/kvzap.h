@@ -181,6 +181,29 @@ kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void 
                                       float *scores_out, void *stream);
 
 /*
+ * The same for a run of layers, with the copies overlapped: while layer l is scored and compacted and its
+ * kept rows travel back, layer l + 1 is already being copied in (two staging sets, a copy stream in each
+ * direction; kernels on `stream`).  hidden, K, V, K_out, V_out, lengths, scores_out (NULL, or entries NULL,
+ * when the scores are not wanted) are HOST arrays of layer_end - layer_begin HOST pointers, one per layer,
+ * each with the shapes of kvzap_prefill_fused_host; cu_seqlens is shared by all layers.
+ * page_tokens == 0: dense-ragged output as above.  page_tokens > 0: paged output as
+ * kvzap_prefill_fused_paged -- K_out[i] / V_out[i] are the host page pools [n_pages_pool, page_tokens, D] of
+ * layer i, first_page (host int32 [n_layers], NULL = all 0), page_table[i] (host int32
+ * [n_seqs*H, max_pages_per_list]) and n_pages_used[i] (host int32 [1]) as there; only the pages a layer
+ * used are copied back.  Pinned host memory is needed for the overlap (pageable memory works, serially).
+ * Returns after every layer's results are in host memory.
+ */
+kvzap_status kvzap_prefill_layers_host(kvzap_ctx *ctx, int32_t layer_begin, int32_t layer_end,
+                                       const void *const *hidden, const void *const *K, const void *const *V,
+                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                       float tau, int32_t w,
+                                       void *const *K_out, void *const *V_out, int32_t *const *lengths,
+                                       float *const *scores_out,
+                                       int32_t page_tokens, int64_t n_pages_pool, const int32_t *first_page,
+                                       int32_t *const *page_table, int32_t max_pages_per_list,
+                                       int32_t *const *n_pages_used, void *stream);
+
+/*
  * Paged output of the same pruning (Discussion, "Implementation Challenges":
  * per-head lengths differ, so the pruned cache needs paged kernels with
  * variable-length blocks; the paper fixes no page format, this one is ours).
@@ -214,6 +237,17 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
                                        int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
                                        int32_t *lengths, int32_t *n_pages_used,
                                        float *scores_out, void *stream);
+
+/* kvzap_prefill_fused_paged for HOST tensors (every pointer, the pools, the page table and n_pages_used
+ * included, is a host pointer); see kvzap_prefill_fused_host and kvzap_prefill_layers_host. */
+kvzap_status kvzap_prefill_fused_paged_host(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                            const void *K, const void *V,
+                                            const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                            float tau, int32_t w,
+                                            void *K_pool, void *V_pool, int64_t n_pages_pool, int32_t page_tokens,
+                                            int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
+                                            int32_t *lengths, int32_t *n_pages_used,
+                                            float *scores_out, void *stream);
 
 /*
  * Fixed-budget selection instead of a threshold (Ablations, "Threshold-based

@@ -51,6 +51,10 @@ SIGNATURES = {
     "kvzap_prefill_fused": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_fused_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp,
                                         _vp]),
+    "kvzap_prefill_layers_host": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp,
+                                         _i32, _i64, _vp, _vp, _i32, _vp, _vp]),
+    "kvzap_prefill_fused_paged_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
+                                              _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _f32, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32, _i32,
                                          _vp, _i32, _vp, _vp, _vp]),
@@ -182,6 +186,46 @@ def kvzap_prefill_fused_host(handle, layer, hidden, K, V, cu_seqlens, n_seqs, ta
     _check(handle, load().kvzap_prefill_fused_host(
         handle, layer, _hptr(hidden), _hptr(K), _hptr(V), _hptr(cu_seqlens), n_seqs, n_tokens, tau, w,
         _hptr(K_out), _hptr(V_out), _hptr(lengths), _hptr(scores_out), _stream(stream)))
+
+
+def _hptr_array(tensors):
+    """A C array of host pointers (NULL for None entries); returns (array, keep-alive list)."""
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        if t is not None:
+            assert not t.is_cuda and t.is_contiguous(), "host entry point takes contiguous CPU tensors"
+            arr[i] = t.data_ptr()
+    return arr
+
+
+def kvzap_prefill_layers_host(handle, layer_begin, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                              scores_out=None, page_tokens=0, first_page=None, page_table=None, n_pages_used=None,
+                              stream=None):
+    """Lists of HOST tensors, one entry per layer of [layer_begin, layer_begin + len(hidden)); paged output when
+    page_tokens > 0 (K_out / V_out are then the host pools, first_page a list of ints or None)."""
+    n = len(hidden)
+    n_tokens = K[0].shape[1]
+    args = [_hptr_array(x) for x in (hidden, K, V)]
+    outs = [_hptr_array(x) for x in (K_out, V_out, lengths)]
+    sc = _hptr_array(scores_out) if scores_out is not None else None
+    if page_tokens > 0:
+        fp = (ctypes.c_int32 * n)(*(first_page if first_page is not None else [0] * n))
+        tab, used = _hptr_array(page_table), _hptr_array(n_pages_used)
+        n_pool, max_pages = K_out[0].shape[0], page_table[0].shape[1]
+    else:
+        fp, tab, used, n_pool, max_pages = None, None, None, 0, 0
+    _check(handle, load().kvzap_prefill_layers_host(
+        handle, layer_begin, layer_begin + n, args[0], args[1], args[2], _hptr(cu_seqlens), n_seqs, n_tokens, tau, w,
+        outs[0], outs[1], outs[2], sc, page_tokens, n_pool, fp, tab, max_pages, used, _stream(stream)))
+
+
+def kvzap_prefill_fused_paged_host(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                                   first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None):
+    """All tensors are HOST tensors, the pools, the page table and n_pages_used included."""
+    _check(handle, load().kvzap_prefill_fused_paged_host(
+        handle, layer, _hptr(hidden), _hptr(K), _hptr(V), _hptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _hptr(K_pool),
+        _hptr(V_pool), K_pool.shape[0], page_tokens, first_page, _hptr(page_table), page_table.shape[1], _hptr(lengths),
+        _hptr(n_pages_used), _hptr(scores_out), _stream(stream)))
 
 
 NOALLOC_MAX_TOKENS = 131072

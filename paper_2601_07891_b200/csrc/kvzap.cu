@@ -94,10 +94,17 @@ struct kvzap_ctx {
     struct ProfRec { int kind; cudaEvent_t start, stop; };
     std::vector<ProfRec> prof;
     // device staging for the host-buffer entry point (allocated on first use)
-    void *stage_x = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_ko = nullptr, *stage_vo = nullptr;
-    float *stage_scores = nullptr;
-    int32_t *stage_lengths = nullptr, *stage_cu = nullptr;
-    int32_t *lengths_pinned = nullptr;
+    // two sets, used by alternate layers: layer l + 1 is copied in while layer l is computed and copied out
+    struct HostStage {
+        void *x = nullptr, *k = nullptr, *v = nullptr, *ko = nullptr, *vo = nullptr;
+        float *scores = nullptr;
+        int32_t *lengths = nullptr, *table = nullptr, *used = nullptr;   // device
+        int32_t *lengths_pinned = nullptr;                               // host, lengths followed by the page count
+        size_t out_bytes = 0, table_ints = 0;
+        cudaEvent_t copied_in = nullptr, computed = nullptr;
+    } stage[2];
+    int32_t *stage_cu = nullptr;
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
     // kvzap_config.flags & KVZAP_FLAG_TRUSTED_PRODUCERS: kernels may read caller data before the work ahead of
     // them in the stream has completed
     bool trusted = false;
@@ -117,6 +124,7 @@ struct kvzap_ctx {
     uint32_t *op_arrive = nullptr;       // [kOpRing]
     int32_t *op_scan_flag = nullptr;     // [kOpRing]
     int32_t *op_page0 = nullptr;         // [kOpRing][max_seqs * H]
+    uint64_t *lin_counts = nullptr;      // [kOpRing][kLinMaxTiles][8]: tile counts of the scoring launch that also compacts
     uint64_t op_turn = 0;
     int32_t op_epoch = 0;
     int op_chain = 0;                    // launches of that kernel in a row that did not wait for the work ahead
@@ -312,15 +320,21 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->list_page0);
     cudaFree(ctx->list_base);
     cudaFree(ctx->op_mask); cudaFree(ctx->op_counts); cudaFree(ctx->op_len_acc);
-    cudaFree(ctx->op_arrive); cudaFree(ctx->op_scan_flag); cudaFree(ctx->op_page0);
+    cudaFree(ctx->op_arrive); cudaFree(ctx->op_scan_flag); cudaFree(ctx->op_page0); cudaFree(ctx->lin_counts);
     cudaFree(ctx->status_dev);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     for (auto &r : ctx->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     ctx->prof.clear();
-    cudaFree(ctx->stage_x); cudaFree(ctx->stage_k); cudaFree(ctx->stage_v);
-    cudaFree(ctx->stage_ko); cudaFree(ctx->stage_vo); cudaFree(ctx->stage_scores);
-    cudaFree(ctx->stage_lengths); cudaFree(ctx->stage_cu);
-    if (ctx->lengths_pinned) cudaFreeHost(ctx->lengths_pinned);
+    for (auto &g : ctx->stage) {
+        cudaFree(g.x); cudaFree(g.k); cudaFree(g.v); cudaFree(g.ko); cudaFree(g.vo); cudaFree(g.scores);
+        cudaFree(g.lengths); cudaFree(g.table); cudaFree(g.used);
+        if (g.lengths_pinned) cudaFreeHost(g.lengths_pinned);
+        if (g.copied_in) cudaEventDestroy(g.copied_in);
+        if (g.computed) cudaEventDestroy(g.computed);
+    }
+    cudaFree(ctx->stage_cu);
+    if (ctx->h2d_stream) cudaStreamDestroy(ctx->h2d_stream);
+    if (ctx->d2h_stream) cudaStreamDestroy(ctx->d2h_stream);
 }
 
 static kvzap_status check_common(kvzap_ctx *ctx, int64_t n_tokens, int32_t n_seqs, const int32_t *cu_seqlens)
@@ -391,14 +405,25 @@ static void make_launch(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attrs, dim
     cfg->numAttrs = static_cast<unsigned>(n);
 }
 
+// What the compaction of a fused call works on; given to launch_score so that a launch which can do the
+// compaction itself (KVzap-Linear, a short single sequence) does it.
+struct CompactArgs {
+    const void *K, *V;
+    void *K_out, *V_out;
+    int32_t *lengths;
+    bool tok_major;
+};
+
 // Launches the scoring kernel over layers [layer, layer + n_layers); hidden is [n_layers][n_tokens][d_model],
 // scores [n_layers][n_tokens][H]; maskbits != nullptr fuses the threshold/window test.
 static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers, const void *hidden, int64_t n_tokens,
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
                                  float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1,
-                                 const DecodeFuse *fuse = nullptr, bool *fused = nullptr, bool fuse_chain = false)
+                                 const DecodeFuse *fuse = nullptr, bool *fused = nullptr, bool fuse_chain = false,
+                                 const CompactArgs *compact = nullptr, bool *compacted = nullptr)
 {
     if (fused) *fused = false;
+    if (compacted) *compacted = false;
     // Early start.  When the grid fills the machine (one CTA per SM), this kernel is allowed to start
     // while the kernels ahead of it in the stream -- the previous call's scoring kernel finishing its
     // last tiles, and its compaction -- are still running: its CTAs take the SMs as they become free.
@@ -548,13 +573,61 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         ctx->last_score_early = early;
         ctx->last_scores = scores;
         ctx->last_scores_bytes = sbytes;
+        // Scoring and compaction in one launch: one layer, one sequence, the window kept, few enough tiles.
+        LinCompact fc;
+        memset(&fc, 0, sizeof fc);
+        uint32_t smem = kLinSmemBytes;
+        if (compact != nullptr && n_layers == 1 && n_seqs == 1 && maskbits != nullptr && window_keep == 1 &&
+            p.n_tiles <= kLinMaxTiles && c.head_dim * 2 <= 2048) {
+            const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * c.head_dim * 2;
+            const int set = static_cast<int>(ctx->op_turn % kOpRing);
+            ctx->op_turn += 1;
+            ctx->op_epoch = ctx->op_epoch == 0x7fffffff ? 1 : ctx->op_epoch + 1;
+            // the same rule as for the one-launch pruning kernel: rows and counts are written before the work
+            // ahead has completed only directly behind launches whose memory is on the pending list and does
+            // not conflict
+            bool wait_first = !ctx->trusted || ctx->profiling || ctx->op_last_seq + 1 != ctx->op_seq || ctx->op_chain >= kOpRing - 2 ||
+                              clash;
+            if (!wait_first)
+                wait_first = hazard(ctx, hidden, static_cast<size_t>(n_tokens) * c.d_model * 2, false) ||
+                             hazard(ctx, compact->K, kv_bytes, false) || hazard(ctx, compact->V, kv_bytes, false) ||
+                             hazard(ctx, compact->K_out, kv_bytes, true) || hazard(ctx, compact->V_out, kv_bytes, true) ||
+                             hazard(ctx, compact->lengths, sizeof(int32_t) * c.n_kv_heads, true);
+            if (wait_first) serial_point(ctx);
+            else ctx->op_chain += 1;
+            ctx->op_last_seq = ctx->op_seq;
+            note_range(ctx, hidden, static_cast<size_t>(n_tokens) * c.d_model * 2, false);
+            note_range(ctx, scores, sbytes, true);
+            note_range(ctx, compact->K, kv_bytes, false);
+            note_range(ctx, compact->V, kv_bytes, false);
+            note_range(ctx, compact->K_out, kv_bytes, true);
+            note_range(ctx, compact->V_out, kv_bytes, true);
+            note_range(ctx, compact->lengths, sizeof(int32_t) * c.n_kv_heads, true);
+            fc.enabled = 1;
+            fc.row_bytes = c.head_dim * 2;
+            fc.K = static_cast<const char *>(compact->K);
+            fc.V = static_cast<const char *>(compact->V);
+            fc.K_out = static_cast<char *>(compact->K_out);
+            fc.V_out = static_cast<char *>(compact->V_out);
+            fc.in_stride_h = compact->tok_major ? 1 : n_tokens;
+            fc.in_stride_t = compact->tok_major ? c.n_kv_heads : 1;
+            fc.lengths = compact->lengths;
+            fc.tile_counts = ctx->lin_counts + static_cast<size_t>(set) * kLinMaxTiles * kMaxHeads;
+            fc.epoch = ctx->op_epoch;
+            fc.n_stages = kLinStagesCompact;
+            fc.wait_limit = ctx->wait_limit;
+            p.wait_before_write = wait_first ? 1 : 0;
+            p.maskbits = nullptr;
+            smem = lin_smem_bytes(kLinStagesCompact);
+            if (compacted) *compacted = true;
+        }
         {
             ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
             cudaLaunchConfig_t cfg;
             cudaLaunchAttribute attrs[2];
-            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * kLinSplit)), dim3(kLinThreads), kLinSmemBytes,
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * kLinSplit)), dim3(kLinThreads), smem,
                         stream, early, kLinSplit);
-            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_linear_split_kernel, tmap_x, ctx->sched[0].tmap_w, p));
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_linear_split_kernel, tmap_x, ctx->sched[0].tmap_w, p, fc));
         }
         ctx->launches += 1;
         return KVZAP_OK;
@@ -1046,6 +1119,8 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
         CREATE_CUDA(cudaMalloc(&ctx->op_scan_flag, sizeof(int32_t) * kOpRing));
         CREATE_CUDA(cudaMemset(ctx->op_scan_flag, 0, sizeof(int32_t) * kOpRing));
         CREATE_CUDA(cudaMalloc(&ctx->op_page0, sizeof(int32_t) * kOpRing * static_cast<size_t>(c.max_seqs) * c.n_kv_heads));
+        CREATE_CUDA(cudaMalloc(&ctx->lin_counts, sizeof(uint64_t) * kOpRing * kLinMaxTiles * kMaxHeads));
+        CREATE_CUDA(cudaMemset(ctx->lin_counts, 0, sizeof(uint64_t) * kOpRing * kLinMaxTiles * kMaxHeads));
     }
     CREATE_CUDA(cudaMalloc(&ctx->status_dev, sizeof(int32_t)));
     CREATE_CUDA(cudaMemset(ctx->status_dev, 0, sizeof(int32_t)));
@@ -1226,8 +1301,11 @@ static kvzap_status prefill_fused_impl(kvzap_ctx *ctx, int32_t layer, const void
     if (st != KVZAP_OK) return st;
     if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
     uint32_t *mask = next_mask_slice(ctx);
-    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
-    if (st != KVZAP_OK) return st;
+    const CompactArgs compact{K, V, K_out, V_out, lengths, tok_major};
+    bool compacted = false;
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream, 1, nullptr, nullptr,
+                      false, &compact, &compacted);
+    if (st != KVZAP_OK || compacted) return st;
     return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, true, tok_major);
 }
 
@@ -1307,75 +1385,6 @@ kvzap_status kvzap_get_profile(kvzap_ctx *ctx, int32_t kernel, double *total_ms,
     }
     *total_ms = sum;
     *n_launches = n;
-    return KVZAP_OK;
-}
-
-kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
-                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
-                                      int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
-                                      void *stream_)
-{
-    NvtxRange nvtx_range("kvzap_prefill_fused_host");
-    if (!ctx) return KVZAP_ERR_INVALID_ARG;
-    begin_op(ctx);
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const kvzap_config &c = ctx->cfg;
-    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
-    if (st != KVZAP_OK) return st;
-    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
-    if (n_tokens == 0) {
-        memset(lengths, 0, sizeof(int32_t) * n_seqs * c.n_kv_heads);
-        return KVZAP_OK;
-    }
-    if (!hidden || !K || !V || !K_out || !V_out)
-        return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden, K, V, K_out and V_out must not be NULL");
-    DeviceGuard guard(c.device);
-    const size_t row_bytes = static_cast<size_t>(c.head_dim) * 2;
-    const size_t kv_cap = static_cast<size_t>(c.n_kv_heads) * c.max_tokens * row_bytes;
-    if (!ctx->stage_x) {
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_x, static_cast<size_t>(c.max_tokens) * c.d_model * 2));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_k, kv_cap));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_v, kv_cap));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_ko, kv_cap));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_vo, kv_cap));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_scores, sizeof(float) * c.max_tokens * c.n_kv_heads));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_lengths, sizeof(int32_t) * c.max_seqs * c.n_kv_heads));
-        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_cu, sizeof(int32_t) * (static_cast<size_t>(c.max_seqs) + 1)));
-        KVZAP_CUDA(ctx, cudaMallocHost(&ctx->lengths_pinned, sizeof(int32_t) * c.max_seqs * c.n_kv_heads));
-    }
-    const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * row_bytes;
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_x, hidden, static_cast<size_t>(n_tokens) * c.d_model * 2,
-                                    cudaMemcpyHostToDevice, stream));
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_k, K, kv_bytes, cudaMemcpyHostToDevice, stream));
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_v, V, kv_bytes, cudaMemcpyHostToDevice, stream));
-    if (cu_seqlens)
-        KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_cu, cu_seqlens, sizeof(int32_t) * (n_seqs + 1),
-                                        cudaMemcpyHostToDevice, stream));
-    st = kvzap_prefill_fused(ctx, layer, ctx->stage_x, ctx->stage_k, ctx->stage_v, cu_seqlens ? ctx->stage_cu : nullptr,
-                             n_seqs, n_tokens, tau, w, ctx->stage_ko, ctx->stage_vo, ctx->stage_lengths,
-                             scores_out ? ctx->stage_scores : nullptr, stream);
-    if (st != KVZAP_OK) return st;
-    const size_t n_lists = static_cast<size_t>(n_seqs) * c.n_kv_heads;
-    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->lengths_pinned, ctx->stage_lengths, sizeof(int32_t) * n_lists,
-                                    cudaMemcpyDeviceToHost, stream));
-    if (scores_out)
-        KVZAP_CUDA(ctx, cudaMemcpyAsync(scores_out, ctx->stage_scores, sizeof(float) * n_tokens * c.n_kv_heads,
-                                        cudaMemcpyDeviceToHost, stream));
-    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
-    memcpy(lengths, ctx->lengths_pinned, sizeof(int32_t) * n_lists);
-    for (int b = 0; b < n_seqs; ++b) {
-        const int64_t seq_start = cu_seqlens ? cu_seqlens[b] : 0;
-        for (int h = 0; h < c.n_kv_heads; ++h) {
-            const int32_t n = lengths[b * c.n_kv_heads + h];
-            if (n <= 0) continue;
-            const size_t off = (static_cast<size_t>(h) * n_tokens + seq_start) * row_bytes;
-            KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(K_out) + off, static_cast<char *>(ctx->stage_ko) + off,
-                                            n * row_bytes, cudaMemcpyDeviceToHost, stream));
-            KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(V_out) + off, static_cast<char *>(ctx->stage_vo) + off,
-                                            n * row_bytes, cudaMemcpyDeviceToHost, stream));
-        }
-    }
-    KVZAP_CUDA(ctx, cudaStreamSynchronize(stream));
     return KVZAP_OK;
 }
 
@@ -2045,6 +2054,223 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     return launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
                                    v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
                                    v.page_cursor, false, true, true, v.free_stack, v.free_top);
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Host-buffer entry points: Algorithm 1 on tensors that live in host memory, layer after layer, with the
+// copies of neighbouring layers overlapped.
+namespace kvzap {
+
+static kvzap_status host_stage_prepare(kvzap_ctx *ctx, size_t out_bytes, size_t table_ints)
+{
+    const kvzap_config &c = ctx->cfg;
+    const size_t kv_cap = static_cast<size_t>(c.n_kv_heads) * c.max_tokens * c.head_dim * 2;
+    const size_t n_lists = static_cast<size_t>(c.max_seqs) * c.n_kv_heads;
+    if (!ctx->h2d_stream) {
+        KVZAP_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->h2d_stream, cudaStreamNonBlocking));
+        KVZAP_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->d2h_stream, cudaStreamNonBlocking));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->stage_cu, sizeof(int32_t) * (static_cast<size_t>(c.max_seqs) + 1)));
+    }
+    for (auto &g : ctx->stage) {
+        if (!g.x) {
+            KVZAP_CUDA(ctx, cudaMalloc(&g.x, static_cast<size_t>(c.max_tokens) * c.d_model * 2));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.k, kv_cap));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.v, kv_cap));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.scores, sizeof(float) * c.max_tokens * c.n_kv_heads));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.lengths, sizeof(int32_t) * n_lists));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.used, sizeof(int32_t)));
+            KVZAP_CUDA(ctx, cudaMallocHost(&g.lengths_pinned, sizeof(int32_t) * (n_lists + 1)));
+            KVZAP_CUDA(ctx, cudaEventCreateWithFlags(&g.copied_in, cudaEventDisableTiming));
+            KVZAP_CUDA(ctx, cudaEventCreateWithFlags(&g.computed, cudaEventDisableTiming));
+        }
+        if (g.out_bytes < out_bytes) {          // the output staging grows with the largest call seen (page size is a call argument)
+            cudaFree(g.ko); cudaFree(g.vo);
+            g.ko = g.vo = nullptr;
+            g.out_bytes = 0;
+            KVZAP_CUDA(ctx, cudaMalloc(&g.ko, out_bytes));
+            KVZAP_CUDA(ctx, cudaMalloc(&g.vo, out_bytes));
+            g.out_bytes = out_bytes;
+        }
+        if (g.table_ints < table_ints) {
+            cudaFree(g.table);
+            g.table = nullptr;
+            g.table_ints = 0;
+            KVZAP_CUDA(ctx, cudaMalloc(&g.table, sizeof(int32_t) * table_ints));
+            g.table_ints = table_ints;
+        }
+    }
+    return KVZAP_OK;
+}
+
+}  // namespace kvzap
+
+extern "C" {
+
+kvzap_status kvzap_prefill_layers_host(kvzap_ctx *ctx, int32_t layer_begin, int32_t layer_end, const void *const *hidden,
+                                       const void *const *K, const void *const *V, const int32_t *cu_seqlens, int32_t n_seqs,
+                                       int64_t n_tokens, float tau, int32_t w, void *const *K_out, void *const *V_out,
+                                       int32_t *const *lengths, float *const *scores_out, int32_t page_tokens,
+                                       int64_t n_pages_pool, const int32_t *first_page, int32_t *const *page_table,
+                                       int32_t max_pages_per_list, int32_t *const *n_pages_used, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_prefill_layers_host");
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    serial_point(ctx);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: layer range [%d, %d) invalid", layer_begin, layer_end);
+    const int n_layers = layer_end - layer_begin;
+    for (int l = layer_begin; l < layer_end; ++l)
+        if (!ctx->layer_set[l]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", l);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!lengths || w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: lengths is NULL or w negative");
+    const bool paged = page_tokens > 0;
+    if (page_tokens < 0 || (paged && (!page_table || !n_pages_used || max_pages_per_list < 1 || n_pages_pool < 0)))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: paged output needs page_table, n_pages_used, max_pages_per_list >= 1");
+    const size_t n_lists = static_cast<size_t>(n_seqs) * c.n_kv_heads;
+    for (int i = 0; i < n_layers; ++i) {
+        if (!lengths[i]) return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: lengths[%d] is NULL", i);
+        if (paged && (!page_table[i] || !n_pages_used[i])) return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: page_table[%d] / n_pages_used[%d] is NULL", i, i);
+        if (paged && first_page && first_page[i] < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: first_page[%d] negative", i);
+    }
+    if (n_tokens == 0) {
+        for (int i = 0; i < n_layers; ++i) {
+            memset(lengths[i], 0, sizeof(int32_t) * n_lists);
+            if (paged) *n_pages_used[i] = 0;
+        }
+        return KVZAP_OK;
+    }
+    if (!hidden || !K || !V || !K_out || !V_out)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: hidden, K, V, K_out and V_out must not be NULL");
+    for (int i = 0; i < n_layers; ++i)
+        if (!hidden[i] || !K[i] || !V[i] || !K_out[i] || !V_out[i])
+            return fail(ctx, KVZAP_ERR_INVALID_ARG, "host prefill: a tensor pointer of layer %d is NULL", layer_begin + i);
+    DeviceGuard guard(c.device);
+    const size_t row_bytes = static_cast<size_t>(c.head_dim) * 2;
+    const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * row_bytes;
+    const size_t x_bytes = static_cast<size_t>(n_tokens) * c.d_model * 2;
+    const size_t page_bytes = paged ? static_cast<size_t>(page_tokens) * row_bytes : 0;
+    // pages one layer can need at most: every list's rows rounded up to whole pages
+    const size_t stage_pages = paged ? static_cast<size_t>(c.n_kv_heads) * n_tokens / page_tokens + n_lists + 1 : 0;
+    st = host_stage_prepare(ctx, paged ? stage_pages * page_bytes : kv_bytes, paged ? n_lists * max_pages_per_list : 0);
+    if (st != KVZAP_OK) return st;
+    // everything enqueued on the caller's stream so far comes first
+    KVZAP_CUDA(ctx, cudaEventRecord(ctx->stage[0].computed, stream));
+    KVZAP_CUDA(ctx, cudaStreamWaitEvent(ctx->h2d_stream, ctx->stage[0].computed, 0));
+    if (cu_seqlens)
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->stage_cu, cu_seqlens, sizeof(int32_t) * (n_seqs + 1), cudaMemcpyHostToDevice, ctx->h2d_stream));
+    auto copy_in = [&](int i) -> kvzap_status {
+        kvzap_ctx::HostStage &g = ctx->stage[i & 1];
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(g.x, hidden[i], x_bytes, cudaMemcpyHostToDevice, ctx->h2d_stream));
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(g.k, K[i], kv_bytes, cudaMemcpyHostToDevice, ctx->h2d_stream));
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(g.v, V[i], kv_bytes, cudaMemcpyHostToDevice, ctx->h2d_stream));
+        if (paged)      // the caller's table goes in and comes back whole, so that entries no list uses stay as they were
+            KVZAP_CUDA(ctx, cudaMemcpyAsync(g.table, page_table[i], sizeof(int32_t) * n_lists * max_pages_per_list,
+                                            cudaMemcpyHostToDevice, ctx->h2d_stream));
+        KVZAP_CUDA(ctx, cudaEventRecord(g.copied_in, ctx->h2d_stream));
+        return KVZAP_OK;
+    };
+    st = copy_in(0);
+    if (st != KVZAP_OK) return st;
+    const int32_t *cu_dev = cu_seqlens ? ctx->stage_cu : nullptr;
+    for (int i = 0; i < n_layers; ++i) {
+        kvzap_ctx::HostStage &g = ctx->stage[i & 1];
+        // the other set is free: the layer that used it was copied out before the previous iteration ended
+        if (i + 1 < n_layers && (st = copy_in(i + 1)) != KVZAP_OK) return st;
+        KVZAP_CUDA(ctx, cudaStreamWaitEvent(stream, g.copied_in, 0));
+        const bool want_scores = scores_out != nullptr && scores_out[i] != nullptr;
+        const int32_t fp = paged && first_page ? first_page[i] : 0;
+        uint32_t *mask = next_mask_slice(ctx);
+        st = launch_score(ctx, layer_begin + i, 1, g.x, n_tokens, want_scores ? g.scores : nullptr, mask, cu_dev, n_seqs, tau, w, stream);
+        if (st != KVZAP_OK) return st;
+        if (paged) {
+            // the staging pool stands for pages first_page .. of the caller's pool
+            char *kp = static_cast<char *>(g.ko) - static_cast<size_t>(fp) * page_bytes;
+            char *vp = static_cast<char *>(g.vo) - static_cast<size_t>(fp) * page_bytes;
+            st = launch_compaction_paged(ctx, mask, g.k, g.v, cu_dev, n_seqs, n_tokens, kp, vp, n_pages_pool, page_tokens, fp, g.table,
+                                         max_pages_per_list, g.lengths, g.used, stream);
+        } else {
+            st = launch_compaction(ctx, mask, g.k, g.v, cu_dev, n_seqs, n_tokens, g.ko, g.vo, g.lengths, stream);
+        }
+        if (st != KVZAP_OK) return st;
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(g.lengths_pinned, g.lengths, sizeof(int32_t) * n_lists, cudaMemcpyDeviceToHost, stream));
+        if (paged)
+            KVZAP_CUDA(ctx, cudaMemcpyAsync(g.lengths_pinned + n_lists, g.used, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+        KVZAP_CUDA(ctx, cudaEventRecord(g.computed, stream));
+        KVZAP_CUDA(ctx, cudaEventSynchronize(g.computed));
+        memcpy(lengths[i], g.lengths_pinned, sizeof(int32_t) * n_lists);
+        if (want_scores)
+            KVZAP_CUDA(ctx, cudaMemcpyAsync(scores_out[i], g.scores, sizeof(float) * n_tokens * c.n_kv_heads, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+        if (paged) {
+            const int32_t used = g.lengths_pinned[n_lists];
+            *n_pages_used[i] = used;
+            if (used > 0) {
+                // Lists own consecutive pages in list order.  Rows are copied in runs that end where a list's
+                // last page is only partly filled, so that the rows behind a list's end stay as the caller had them.
+                const int64_t row0 = static_cast<int64_t>(fp) * page_tokens;
+                int64_t run_begin = row0, pos = row0;
+                auto copy_rows = [&](int64_t from, int64_t to) -> kvzap_status {
+                    if (to <= from) return KVZAP_OK;
+                    const size_t host_off = static_cast<size_t>(from) * row_bytes, dev_off = static_cast<size_t>(from - row0) * row_bytes;
+                    const size_t n = static_cast<size_t>(to - from) * row_bytes;
+                    KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(K_out[i]) + host_off, static_cast<char *>(g.ko) + dev_off, n, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+                    KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(V_out[i]) + host_off, static_cast<char *>(g.vo) + dev_off, n, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+                    return KVZAP_OK;
+                };
+                for (size_t li = 0; li < n_lists; ++li) {
+                    const int64_t len = g.lengths_pinned[li];
+                    if (len <= 0) continue;
+                    const int64_t n_pages = (len + page_tokens - 1) / page_tokens;
+                    if (len % page_tokens != 0) {
+                        if ((st = copy_rows(run_begin, pos + len)) != KVZAP_OK) return st;
+                        run_begin = pos + n_pages * page_tokens;
+                    }
+                    pos += n_pages * page_tokens;
+                }
+                if ((st = copy_rows(run_begin, pos)) != KVZAP_OK) return st;
+                KVZAP_CUDA(ctx, cudaMemcpyAsync(page_table[i], g.table, sizeof(int32_t) * n_lists * max_pages_per_list, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+            }
+        } else {
+            for (int b = 0; b < n_seqs; ++b) {
+                const int64_t seq_start = cu_seqlens ? cu_seqlens[b] : 0;
+                for (int h = 0; h < c.n_kv_heads; ++h) {
+                    const int32_t n = g.lengths_pinned[b * c.n_kv_heads + h];
+                    if (n <= 0) continue;
+                    const size_t off = (static_cast<size_t>(h) * n_tokens + seq_start) * row_bytes;
+                    KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(K_out[i]) + off, static_cast<char *>(g.ko) + off, n * row_bytes, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+                    KVZAP_CUDA(ctx, cudaMemcpyAsync(static_cast<char *>(V_out[i]) + off, static_cast<char *>(g.vo) + off, n * row_bytes, cudaMemcpyDeviceToHost, ctx->d2h_stream));
+                }
+            }
+        }
+        KVZAP_CUDA(ctx, cudaStreamSynchronize(ctx->d2h_stream));
+    }
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_prefill_fused_host(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                      const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                      int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out,
+                                      void *stream_)
+{
+    return kvzap_prefill_layers_host(ctx, layer, layer + 1, &hidden, &K, &V, cu_seqlens, n_seqs, n_tokens, tau, w, &K_out, &V_out,
+                                     &lengths, &scores_out, 0, 0, nullptr, nullptr, 0, nullptr, stream_);
+}
+
+kvzap_status kvzap_prefill_fused_paged_host(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K, const void *V,
+                                            const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau, int32_t w,
+                                            void *K_pool, void *V_pool, int64_t n_pages_pool, int32_t page_tokens,
+                                            int32_t first_page, int32_t *page_table, int32_t max_pages_per_list,
+                                            int32_t *lengths, int32_t *n_pages_used, float *scores_out, void *stream_)
+{
+    if (page_tokens < 1) return ctx ? kvzap::fail(ctx, KVZAP_ERR_INVALID_ARG, "paged host prefill: page_tokens must be >= 1") : KVZAP_ERR_INVALID_ARG;
+    return kvzap_prefill_layers_host(ctx, layer, layer + 1, &hidden, &K, &V, cu_seqlens, n_seqs, n_tokens, tau, w, &K_pool, &V_pool,
+                                     &lengths, &scores_out, page_tokens, n_pages_pool, &first_page, &page_table,
+                                     max_pages_per_list, &n_pages_used, stream_);
 }
 
 }  // extern "C"

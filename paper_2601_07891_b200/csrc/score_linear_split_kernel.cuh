@@ -14,38 +14,83 @@
 // (the host sets it unless the mask slice and the scores buffer written here are known to be free).
 #pragma once
 
+#include "prune_onepass_kernel.cuh"
 #include "score_kernel.cuh"
 
 namespace kvzap {
 
 constexpr int kLinSplit = 4;
-constexpr int kLinStages = 8;
+constexpr int kLinStages = 8;             // pipeline stages; kLinStagesCompact when the compaction runs in the same launch
+constexpr int kLinStagesCompact = 5;      // (two CTAs then fit an SM, so the next call's launch runs beside this one)
 constexpr int kLinThreads = 192;          // producer warp, MMA warp, four epilogue warps
+constexpr int kLinMaxTiles = 64;          // tiles of a launch that also compacts (its clusters wait for one another)
 constexpr uint32_t kLinBTileBytes = 16 * kBlockK * 2;                 // 16 weight rows (H <= 8, padded) of one K block
 constexpr uint32_t kLinStageBytes = kATileBytes + kLinBTileBytes;    // 18 KB, a multiple of 1024
-constexpr uint32_t kLinXpartOff = kLinStages * kLinStageBytes;        // [kLinSplit - 1][128][8] fp32
-constexpr uint32_t kLinBarsOff = kLinXpartOff + (kLinSplit - 1) * kTileM * kMaxHeads * 4;
-constexpr uint32_t kLinSmemBytes = kLinBarsOff + 256 + 1024;          // + barriers + alignment slack
+// shared memory after the stages: [kLinSplit - 1][128][8] fp32 partial sums, then barriers and flags
+__host__ __device__ constexpr uint32_t lin_xpart_off(int n_stages) { return static_cast<uint32_t>(n_stages) * kLinStageBytes; }
+__host__ __device__ constexpr uint32_t lin_bars_off(int n_stages) { return lin_xpart_off(n_stages) + (kLinSplit - 1) * kTileM * kMaxHeads * 4; }
+__host__ __device__ constexpr uint32_t lin_smem_bytes(int n_stages) { return lin_bars_off(n_stages) + 256 + 1024; }   // + alignment slack
+constexpr uint32_t kLinSmemBytes = lin_smem_bytes(kLinStages);
+
+// The compaction of Algorithm 1 inside the scoring launch (one sequence, dense-ragged output, one layer per
+// launch, a grid that is resident at once): the cluster of a tile publishes the tile's kept count per head,
+// adds up the counts of the tiles before it, and moves its own tile's kept rows -- each of its four CTAs a
+// quarter of the tile's tokens -- with bulk copies through the pipeline stages, which are idle by then.
+struct LinCompact {
+    int32_t enabled;
+    int32_t row_bytes;           // 2 * head_dim, a multiple of 16
+    const char *K, *V;           // row (h, t) at (h * in_stride_h + t * in_stride_t) * row_bytes
+    char *K_out, *V_out;         // [H][n_tokens][D]
+    int64_t in_stride_h, in_stride_t;
+    int32_t *lengths;            // [H]
+    uint64_t *tile_counts;       // [n_tiles][8]: (call number << 32) | rows of head h kept in the tile
+    int32_t epoch;               // the call's number, never 0
+    int32_t n_stages;
+    int64_t wait_limit;
+};
+
+// one row: global -> shared, completion counted on an mbarrier (bytes a multiple of 16, both sides 16-byte aligned)
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// one row: shared -> global, in the thread's current bulk group
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit_and_wait_read()
+{
+    asm volatile("cp.async.bulk.commit_group;\n\tcp.async.bulk.wait_group.read 0;" ::: "memory");
+}
 
 // gridDim.x = kLinSplit * p.n_tiles (cluster dimension kLinSplit); p.n_tiles = 128-token tiles over all
 // layers of the call, p.tiles_per_layer of them per layer; d_model / 64 divisible by kLinSplit.
 __global__ void __launch_bounds__(kLinThreads)
 score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                          const ScoreParams p)
+                          const ScoreParams p, const LinCompact fc)
 {
+    __shared__ uint32_t wt_s[kMaxHeads][4];             // compaction: the tile's keep words (head, quarter of the tile)
+    __shared__ int32_t run_s[kMaxHeads];                //             rows of head h kept before the tile
+    __shared__ int32_t red_s[kLinThreads / 32][kMaxHeads];
+    __shared__ int64_t ent_src_s[kMaxHeads * 32], ent_dst_s[kMaxHeads * 32];     // kept rows of this CTA's quarter (byte offsets)
+    const int n_st = fc.enabled ? fc.n_stages : kLinStages;
     extern __shared__ uint8_t lin_smem_raw[];
     const uint32_t raw_addr = smem_u32(lin_smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
     uint8_t *smem = lin_smem_raw + pad;
     const uint32_t smem_base = raw_addr + pad;
-    float *xpart = reinterpret_cast<float *>(smem + kLinXpartOff);
-    const uint32_t bars = smem_base + kLinBarsOff;
+    const uint32_t xpart_off = lin_xpart_off(n_st), bars_off = lin_bars_off(n_st);
+    float *xpart = reinterpret_cast<float *>(smem + xpart_off);
+    const uint32_t bars = smem_base + bars_off;
     const uint32_t bar_full = bars;                       // [kLinStages] TMA -> MMA
     const uint32_t bar_empty = bars + 8 * kLinStages;     // [kLinStages] MMA -> TMA
     const uint32_t bar_tfull = bars + 16 * kLinStages;    // MMA -> epilogue
     const uint32_t bar_done = bar_tfull + 8;              // abort path only
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + kLinBarsOff + 16 * kLinStages + 16);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kLinBarsOff + 16 * kLinStages + 20);
+    const uint32_t bar_bulk = bar_tfull + 24;             // compaction: rows arriving in the stages
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + bars_off + 16 * kLinStages + 16);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + bars_off + 16 * kLinStages + 20);
 
     griddep_launch_dependents();
     if (p.wait_before_load) griddep_wait();     // caller data is read only after the work ahead in the stream is complete
@@ -65,6 +110,7 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
         }
         mbar_init(bar_tfull, 1);
         mbar_init(bar_done, 1);
+        mbar_init(bar_bulk, kLinThreads);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
@@ -102,7 +148,7 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
             }
             __syncwarp();
             sa += kLinStageBytes;
-            if (++st == kLinStages) { st = 0; st_par ^= 1u; sa = smem_base; }
+            if (++st == static_cast<uint32_t>(n_st)) { st = 0; st_par ^= 1u; sa = smem_base; }
         }
         if (!ok && lane == 0) {
             // abort path: give the copies already in flight a fixed time to land before the CTA exits
@@ -130,7 +176,7 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
             }
             __syncwarp();
             a_lo += kLinStageBytes >> 4;
-            if (++st == kLinStages) { st = 0; st_par ^= 1u; a_lo = desc_lo0; }
+            if (++st == static_cast<uint32_t>(n_st)) { st = 0; st_par ^= 1u; a_lo = desc_lo0; }
         }
         if (ok && elected) umma_commit(bar_tfull);
         __syncwarp();
@@ -160,7 +206,7 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
         }
         if (rank != 0) {
             // the partial sums of this CTA's K range go to the first CTA: xpart[rank - 1][row][8]
-            const uint32_t dst = map_to_cta(smem_base + kLinXpartOff + ((rank - 1) * kTileM + row) * kMaxHeads * 4, 0);
+            const uint32_t dst = map_to_cta(smem_base + xpart_off + ((rank - 1) * kTileM + row) * kMaxHeads * 4, 0);
             st_shared_cluster_v4(dst, s[0], s[1], s[2], s[3]);
             st_shared_cluster_v4(dst + 16, s[4], s[5], s[6], s[7]);
         }
@@ -172,6 +218,152 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
     if (warp == 1) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
+    }
+    // nothing has been written so far
+    if (fc.enabled) {
+        // ------------------------------------------------------------ scoring and compaction in one launch
+        if (p.wait_before_write) griddep_wait();           // every thread: outputs may still be in use by the work ahead
+        const uint32_t wt_addr = smem_u32(&wt_s[0][0]);
+        if (rank == 0 && epi) {
+#pragma unroll
+            for (int r = 0; r < kLinSplit - 1; ++r) {
+                const float4 *src = reinterpret_cast<const float4 *>(xpart + (r * kTileM + row) * kMaxHeads);
+                const float4 pa = src[0], pb = src[1];
+                s[0] += pa.x; s[1] += pa.y; s[2] += pa.z; s[3] += pa.w;
+                s[4] += pb.x; s[5] += pb.y; s[6] += pb.z; s[7] += pb.w;
+            }
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) s[h] += __ldg(p.b1 + layer * p.w_rows + h);
+            const int64_t t = static_cast<int64_t>(m_tile) * kTileM + row;
+            const bool valid = t < p.n_tokens;
+            if (valid && p.scores != nullptr) {
+                float *dst = p.scores + t * p.n_heads;
+                if (p.n_heads == kMaxHeads) {
+                    reinterpret_cast<float4 *>(dst)[0] = make_float4(s[0], s[1], s[2], s[3]);
+                    reinterpret_cast<float4 *>(dst)[1] = make_float4(s[4], s[5], s[6], s[7]);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < kMaxHeads; ++h)
+                        if (h < p.n_heads) dst[h] = s[h];
+                }
+            }
+            const bool in_window = valid && t >= p.n_tokens - static_cast<int64_t>(p.window);      // one sequence
+            uint32_t my_word = 0;
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) {
+                const bool keep = valid && (in_window || s[h] >= p.tau);
+                const uint32_t word = __ballot_sync(0xffffffffu, keep);
+                if (lane == h) my_word = word;
+            }
+            if (lane < kMaxHeads) {
+                if (lane >= p.n_heads || *abort_flag) my_word = 0;      // a pipeline that gave up: nothing is kept, nothing moved
+                // the tile's keep words go to all four CTAs of the cluster
+#pragma unroll
+                for (uint32_t r = 0; r < kLinSplit; ++r)
+                    st_shared_cluster_u32(map_to_cta(wt_addr + (lane * 4 + q) * 4, r), my_word);
+            }
+        }
+        cluster_sync_all();
+        const uint64_t tag = static_cast<uint64_t>(static_cast<uint32_t>(fc.epoch)) << 32;
+        if (rank == 0 && threadIdx.x < kMaxHeads) {
+            const int cnt = __popc(wt_s[threadIdx.x][0]) + __popc(wt_s[threadIdx.x][1]) + __popc(wt_s[threadIdx.x][2]) +
+                            __popc(wt_s[threadIdx.x][3]);
+            st_relaxed_gpu_u64(fc.tile_counts + tile * kMaxHeads + threadIdx.x, tag | static_cast<uint32_t>(cnt));
+        }
+        // rows kept before this tile: the counts of the tiles before it (every CTA of the cluster adds them up itself)
+        {
+            int32_t acc[kMaxHeads];
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) acc[h] = 0;
+            for (int j = threadIdx.x; j < tile; j += kLinThreads) {
+                const uint64_t *e = fc.tile_counts + static_cast<int64_t>(j) * kMaxHeads;
+                ulonglong2 v[4];
+                const long long t_begin = clock64();
+                for (;;) {
+                    bool all = true;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[i] = ld_relaxed_gpu_v2(e + 2 * i);
+                        all = all && (v[i].x >> 32) == (tag >> 32) && (v[i].y >> 32) == (tag >> 32);
+                    }
+                    if (all) break;
+                    if (clock64() - t_begin > fc.wait_limit) { *abort_flag = 2; break; }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[2 * i] += static_cast<int32_t>(static_cast<uint32_t>(v[i].x));
+                    acc[2 * i + 1] += static_cast<int32_t>(static_cast<uint32_t>(v[i].y));
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < kMaxHeads; ++h) acc[h] = __reduce_add_sync(0xffffffffu, acc[h]);
+            if (lane == 0) {
+#pragma unroll
+                for (int h = 0; h < kMaxHeads; ++h) red_s[warp][h] = acc[h];
+            }
+            __syncthreads();
+            if (threadIdx.x < kMaxHeads) {
+                int32_t r = 0;
+#pragma unroll
+                for (int wv = 0; wv < kLinThreads / 32; ++wv) r += red_s[wv][threadIdx.x];
+                run_s[threadIdx.x] = r;
+            }
+            __syncthreads();
+        }
+        if (*abort_flag == 2) {                             // a tile before this one never published: nothing is moved
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+            griddep_wait();
+            return;
+        }
+        // this CTA's quarter of the tile: tokens 32 * rank .. + 31, all heads; its kept rows listed by (head, token)
+        const int64_t t_q0 = static_cast<int64_t>(m_tile) * kTileM + rank * 32;
+        int n_rows = 0;
+        for (int h = 0; h < p.n_heads; ++h) n_rows += __popc(wt_s[h][rank]);
+        for (int pi = threadIdx.x; pi < p.n_heads * 32; pi += kLinThreads) {
+            const int h = pi >> 5, tk = pi & 31;
+            const uint32_t w = wt_s[h][rank];
+            if ((w >> tk) & 1u) {
+                int idx = __popc(w & ((1u << tk) - 1u)), before = 0;
+                for (int hh = 0; hh < h; ++hh) idx += __popc(wt_s[hh][rank]);
+                for (uint32_t qq = 0; qq < rank; ++qq) before += __popc(wt_s[h][qq]);
+                const int64_t n = run_s[h] + before + __popc(w & ((1u << tk) - 1u));          // rank inside head h's list
+                ent_src_s[idx] = (h * fc.in_stride_h + (t_q0 + tk) * fc.in_stride_t) * fc.row_bytes;
+                ent_dst_s[idx] = (static_cast<int64_t>(h) * p.n_tokens + n) * fc.row_bytes;
+            }
+        }
+        if (rank == 0 && m_tile == p.tiles_per_layer - 1 && threadIdx.x < p.n_heads) {
+            const int h = threadIdx.x;
+            fc.lengths[h] = run_s[h] + __popc(wt_s[h][0]) + __popc(wt_s[h][1]) + __popc(wt_s[h][2]) + __popc(wt_s[h][3]);
+        }
+        __syncthreads();
+        // rows travel global -> the idle pipeline stages -> global as bulk copies; as many per round as the stages hold
+        const int cap = static_cast<int>(static_cast<uint32_t>(n_st) * kLinStageBytes / (2u * fc.row_bytes));
+        uint32_t phase = 0;
+        for (int c0 = 0; c0 < n_rows; c0 += cap, phase ^= 1u) {
+            const int n_chunk = n_rows - c0 < cap ? n_rows - c0 : cap;
+            int mine = 0;
+            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) ++mine;
+            if (mine > 0) mbar_arrive_expect_tx(bar_bulk, static_cast<uint32_t>(mine) * 2u * fc.row_bytes);
+            else mbar_arrive(bar_bulk);
+            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) {
+                const uint32_t slot = smem_base + static_cast<uint32_t>(i) * 2u * fc.row_bytes;
+                bulk_load(slot, fc.K + ent_src_s[c0 + i], fc.row_bytes, bar_bulk);
+                bulk_load(slot + fc.row_bytes, fc.V + ent_src_s[c0 + i], fc.row_bytes, bar_bulk);
+            }
+            if (!mbar_wait(bar_bulk, phase, abort_flag)) break;
+            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) {
+                const uint32_t slot = smem_base + static_cast<uint32_t>(i) * 2u * fc.row_bytes;
+                bulk_store(fc.K_out + ent_dst_s[c0 + i], slot, fc.row_bytes);
+                bulk_store(fc.V_out + ent_dst_s[c0 + i], slot + fc.row_bytes, fc.row_bytes);
+            }
+            bulk_commit_and_wait_read();                    // the stages are read before the next round overwrites them
+            __syncthreads();
+        }
+        if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
+        // bulk stores complete before the grid does; this kernel still completes after the one ahead of it
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        griddep_wait();
+        return;
     }
     // nothing has been written so far
     if (p.wait_before_write || rank != 0 || !epi) {
