@@ -767,9 +767,21 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
     if (page_tokens > 0 && n_pages_pool * page_tokens >= 0xffffffffLL)
         return fail(ctx, KVZAP_ERR_UNSUPPORTED, "paged pruning: the pool must hold fewer than 2^32 - 1 rows");
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
-    int64_t grid = n_blocks < ctx->op_capacity ? n_blocks : ctx->op_capacity;
-    const int64_t per_cta = (n_blocks + grid - 1) / grid;
-    grid = (n_blocks + per_cta - 1) / per_cta;
+    // Heads per CTA: as many as still leave a CTA a dozen blocks or more.  The one CTA that holds a sequence's window
+    // keeps all rows of a block where the others keep a quarter or a third; with many blocks per CTA that is a small
+    // surplus, with two or three it would make that CTA the last to finish by far.
+    int heads_per_cta = kMaxHeads, groups = 1;
+    int64_t grid = 1, per_cta = n_blocks;
+    for (int hg = kMaxHeads; hg >= 1; hg >>= 1) {
+        heads_per_cta = hg;
+        groups = (c.n_kv_heads + hg - 1) / hg;
+        grid = ctx->op_capacity / groups;
+        if (grid < 1) grid = 1;
+        if (grid > n_blocks) grid = n_blocks;
+        per_cta = (n_blocks + grid - 1) / grid;
+        grid = (n_blocks + per_cta - 1) / per_cta;
+        if (per_cta >= 12) break;
+    }
     const int set = static_cast<int>(ctx->op_turn % kOpRing);
     ctx->op_turn += 1;
     ctx->op_epoch = ctx->op_epoch == 0x7fffffff ? 1 : ctx->op_epoch + 1;
@@ -815,6 +827,7 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
     p.n_seqs = n_seqs;
     p.cu_seqlens = cu_seqlens;
     p.blocks_per_cta = static_cast<int32_t>(per_cta);
+    p.heads_per_cta = heads_per_cta;
     p.K = static_cast<const uint4 *>(K);
     p.V = static_cast<const uint4 *>(V);
     p.K_out = static_cast<uint4 *>(K_out);
@@ -843,7 +856,8 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
         ProfScope prof(ctx, KVZAP_KERNEL_COMPACT, stream);
         cudaLaunchConfig_t cfg;
         cudaLaunchAttribute attrs[2];
-        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid)), dim3(kOpThreads), kOpDynSmem, stream, !ctx->profiling, 1);
+        make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid), static_cast<unsigned>(groups)), dim3(kOpThreads), kOpDynSmem,
+                    stream, !ctx->profiling, 1);
         KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, prune_onepass_kernel<kOpRows>, p));
     }
     ctx->launches += 1;

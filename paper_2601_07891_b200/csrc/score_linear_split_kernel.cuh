@@ -21,7 +21,8 @@ namespace kvzap {
 
 constexpr int kLinSplit = 4;
 constexpr int kLinStages = 8;             // pipeline stages; kLinStagesCompact when the compaction runs in the same launch
-constexpr int kLinStagesCompact = 5;      // (two CTAs then fit an SM, so the next call's launch runs beside this one)
+constexpr int kLinStagesCompact = 2;      // (four CTAs then fit an SM: the launches of the next calls run beside this one;
+                                          //  measured per call at 4096 tokens: 8.8 us with 2 stages, 9.9 with 3, 9.6 with 5)
 constexpr int kLinThreads = 192;          // producer warp, MMA warp, four epilogue warps
 constexpr int kLinMaxTiles = 64;          // tiles of a launch that also compacts (its clusters wait for one another)
 constexpr uint32_t kLinBTileBytes = 16 * kBlockK * 2;                 // 16 weight rows (H <= 8, padded) of one K block
@@ -35,7 +36,8 @@ constexpr uint32_t kLinSmemBytes = lin_smem_bytes(kLinStages);
 // The compaction of Algorithm 1 inside the scoring launch (one sequence, dense-ragged output, one layer per
 // launch, a grid that is resident at once): the cluster of a tile publishes the tile's kept count per head,
 // adds up the counts of the tiles before it, and moves its own tile's kept rows -- each of its four CTAs a
-// quarter of the tile's tokens -- with bulk copies through the pipeline stages, which are idle by then.
+// quarter of the tile's tokens -- through the pipeline stages, which are idle by then.  (Bulk copies, one
+// per 256-byte row, were tried for that and moved rows at 2.7 TB/s; 16-byte asynchronous copies do 4+.)
 struct LinCompact {
     int32_t enabled;
     int32_t row_bytes;           // 2 * head_dim, a multiple of 16
@@ -48,22 +50,6 @@ struct LinCompact {
     int32_t n_stages;
     int64_t wait_limit;
 };
-
-// one row: global -> shared, completion counted on an mbarrier (bytes a multiple of 16, both sides 16-byte aligned)
-__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-// one row: shared -> global, in the thread's current bulk group
-__device__ __forceinline__ void bulk_store(void *dst, uint32_t smem_src, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit_and_wait_read()
-{
-    asm volatile("cp.async.bulk.commit_group;\n\tcp.async.bulk.wait_group.read 0;" ::: "memory");
-}
 
 // gridDim.x = kLinSplit * p.n_tiles (cluster dimension kLinSplit); p.n_tiles = 128-token tiles over all
 // layers of the call, p.tiles_per_layer of them per layer; d_model / 64 divisible by kLinSplit.
@@ -88,7 +74,6 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
     const uint32_t bar_empty = bars + 8 * kLinStages;     // [kLinStages] MMA -> TMA
     const uint32_t bar_tfull = bars + 16 * kLinStages;    // MMA -> epilogue
     const uint32_t bar_done = bar_tfull + 8;              // abort path only
-    const uint32_t bar_bulk = bar_tfull + 24;             // compaction: rows arriving in the stages
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + bars_off + 16 * kLinStages + 16);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + bars_off + 16 * kLinStages + 20);
 
@@ -110,7 +95,6 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
         }
         mbar_init(bar_tfull, 1);
         mbar_init(bar_done, 1);
-        mbar_init(bar_bulk, kLinThreads);
         *abort_flag = 0;
         fence_mbar_init();
         prefetch_tensormap(&tmap_x);
@@ -336,33 +320,34 @@ score_linear_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __gr
             fc.lengths[h] = run_s[h] + __popc(wt_s[h][0]) + __popc(wt_s[h][1]) + __popc(wt_s[h][2]) + __popc(wt_s[h][3]);
         }
         __syncthreads();
-        // rows travel global -> the idle pipeline stages -> global as bulk copies; as many per round as the stages hold
+        // rows travel global -> the idle pipeline stages -> global; as many per round as the stages hold
         const int cap = static_cast<int>(static_cast<uint32_t>(n_st) * kLinStageBytes / (2u * fc.row_bytes));
-        uint32_t phase = 0;
-        for (int c0 = 0; c0 < n_rows; c0 += cap, phase ^= 1u) {
+        // as asynchronous 16-byte copies into shared memory (they pass by the L1 and the registers, so the rows of
+        // a round are all in flight at once), 16 lanes per row, then ordinary loads from there and stores
+        const int group = threadIdx.x >> 4, gl = threadIdx.x & 15;
+        for (int c0 = 0; c0 < n_rows; c0 += cap) {
             const int n_chunk = n_rows - c0 < cap ? n_rows - c0 : cap;
-            int mine = 0;
-            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) ++mine;
-            if (mine > 0) mbar_arrive_expect_tx(bar_bulk, static_cast<uint32_t>(mine) * 2u * fc.row_bytes);
-            else mbar_arrive(bar_bulk);
-            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) {
+            for (int i = group; i < n_chunk; i += kLinThreads / 16) {
                 const uint32_t slot = smem_base + static_cast<uint32_t>(i) * 2u * fc.row_bytes;
-                bulk_load(slot, fc.K + ent_src_s[c0 + i], fc.row_bytes, bar_bulk);
-                bulk_load(slot + fc.row_bytes, fc.V + ent_src_s[c0 + i], fc.row_bytes, bar_bulk);
+                const int64_t src = ent_src_s[c0 + i];
+                for (uint32_t u = gl * 16u; u < static_cast<uint32_t>(fc.row_bytes); u += 256u) {
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + u), "l"(fc.K + src + u) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + fc.row_bytes + u), "l"(fc.V + src + u) : "memory");
+                }
             }
-            if (!mbar_wait(bar_bulk, phase, abort_flag)) break;
-            for (int i = threadIdx.x; i < n_chunk; i += kLinThreads) {
-                const uint32_t slot = smem_base + static_cast<uint32_t>(i) * 2u * fc.row_bytes;
-                bulk_store(fc.K_out + ent_dst_s[c0 + i], slot, fc.row_bytes);
-                bulk_store(fc.V_out + ent_dst_s[c0 + i], slot + fc.row_bytes, fc.row_bytes);
+            asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+            for (int i = group; i < n_chunk; i += kLinThreads / 16) {
+                const uint8_t *slot = smem + static_cast<uint32_t>(i) * 2u * fc.row_bytes;
+                const int64_t dst = ent_dst_s[c0 + i];
+                for (uint32_t u = gl * 16u; u < static_cast<uint32_t>(fc.row_bytes); u += 256u) {
+                    *reinterpret_cast<uint4 *>(fc.K_out + dst + u) = *reinterpret_cast<const uint4 *>(slot + u);
+                    *reinterpret_cast<uint4 *>(fc.V_out + dst + u) = *reinterpret_cast<const uint4 *>(slot + fc.row_bytes + u);
+                }
             }
-            bulk_commit_and_wait_read();                    // the stages are read before the next round overwrites them
             __syncthreads();
         }
-        if (threadIdx.x == 0 && *abort_flag) atomicCAS(p.status, 0, 5 /* KVZAP_ERR_TIMEOUT */);
-        // bulk stores complete before the grid does; this kernel still completes after the one ahead of it
-        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        griddep_wait();
+        griddep_wait();                                     // this kernel still completes after the one ahead of it
         return;
     }
     // nothing has been written so far
