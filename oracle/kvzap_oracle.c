@@ -473,3 +473,203 @@ int64_t kvzap_oracle_param_count(int Dh, int N1, int H)
     if (N1 == 0) return (int64_t)Dh * H + H;
     return (int64_t)Dh * N1 + N1 + (int64_t)N1 * H + H;
 }
+
+/*
+ * Write plan (Discussion, "Implementation Challenges": since the surrogate
+ * needs only hidden states, pruning can be applied before attention, i.e. before
+ * the keys and values are stored).  Instead of moving rows, the plan tells
+ * whoever produces K and V where each row belongs:
+ *   slot[t,h] = n, the number of kept positions of list (b,h) before t, if keep[h,t]
+ *             = -1 if the pair is dropped
+ * so that writing row t of head h to row cu_seqlens[b] + slot of head h gives
+ * exactly kvzap_oracle_compact's output.  Paged (page_tokens > 0): the page
+ * assignment is that of kvzap_oracle_compact_paged and the slot is the pool row,
+ *   slot[t,h] = (first page of list (b,h) + n / page_tokens) * page_tokens + n % page_tokens.
+ * slot [T_total,H] int32; lengths [B,H]; page_table / n_pages_used as in
+ * kvzap_oracle_compact_paged (ignored when page_tokens == 0).
+ * Returns 0, or -1 if the pool or the table is too small (slot is then all -1).
+ */
+int kvzap_oracle_plan(const uint8_t *keep, const int32_t *cu_seqlens, int B, int H,
+                      int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages_per_list,
+                      int32_t *slot, int32_t *page_table, int32_t *lengths, int32_t *n_pages_used)
+{
+    const int64_t T_total = cu_seqlens[B];
+    for (int64_t i = 0; i < T_total * H; ++i) slot[i] = -1;
+    int64_t pages = 0;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            int64_t n = 0;
+            for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t)
+                n += keep[(int64_t)h * T_total + t] ? 1 : 0;
+            lengths[b * H + h] = (int32_t)n;
+            if (page_tokens > 0) {
+                const int64_t need = (n + page_tokens - 1) / page_tokens;
+                if (need > max_pages_per_list) return -1;
+                pages += need;
+            }
+        }
+    if (page_tokens > 0 && (int64_t)first_page + pages > n_pages_pool) return -1;
+    int64_t cursor = first_page;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H; ++h) {
+            const int list = b * H + h;
+            int64_t n = 0;
+            for (int64_t t = cu_seqlens[b]; t < cu_seqlens[b + 1]; ++t) {
+                if (!keep[(int64_t)h * T_total + t]) continue;
+                if (page_tokens > 0)
+                    slot[t * H + h] = (int32_t)((cursor + n / page_tokens) * page_tokens + n % page_tokens);
+                else
+                    slot[t * H + h] = (int32_t)n;
+                ++n;
+            }
+            if (page_tokens > 0) {
+                const int64_t need = (n + page_tokens - 1) / page_tokens;
+                int32_t *row = page_table + (int64_t)list * max_pages_per_list;
+                for (int64_t i = 0; i < need; ++i) row[i] = (int32_t)(cursor + i);
+                cursor += need;
+            }
+        }
+    if (page_tokens > 0) *n_pages_used = (int32_t)pages;
+    return 0;
+}
+
+/*
+ * 8-bit floating point inputs (Related work, "Quantization": pruning composes
+ * with quantisation of the cache; the paper fixes no format).  The reading
+ * used here is the OCP 8-bit format E4M3 in its finite variant: 1 sign bit,
+ * 4 exponent bits with bias 7, 3 mantissa bits; exponent field 0 holds the
+ * subnormals m/8 * 2^-6; there are no infinities; only S.1111.111 is NaN, so
+ * the largest magnitude is 1.75 * 2^8 = 448.  Exact widening to double:
+ */
+double kvzap_oracle_e4m3_to_double(uint8_t bits)
+{
+    const int sign = bits >> 7, e = (bits >> 3) & 15, m = bits & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/*
+ * KVzap-Linear on quantised inputs: hidden states X8 [T,Dh] and weights W8 [H,Dh]
+ * as E4M3 bytes, with one fp32 scale per token (x_scale [T], NULL = 1) and one
+ * per output row (w_scale [H], NULL = 1) -- the usual per-token / per-channel
+ * scaling; the paper gives none.
+ *   scores[t,h] = b[h] + x_scale[t] * w_scale[h] * sum_k X8[t,k] * W8[h,k]
+ */
+void kvzap_oracle_score_linear_fp8(const uint8_t *X8, const float *x_scale, int64_t T, int Dh,
+                                   const uint8_t *W8, const float *w_scale, const float *b, int H,
+                                   float *scores)
+{
+    int64_t t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < T; ++t) {
+        for (int h = 0; h < H; ++h) {
+            double acc = 0.0;
+            for (int k = 0; k < Dh; ++k)
+                acc += kvzap_oracle_e4m3_to_double(X8[t * Dh + k]) * kvzap_oracle_e4m3_to_double(W8[(int64_t)h * Dh + k]);
+            const double sx = x_scale ? (double)x_scale[t] : 1.0, sw = w_scale ? (double)w_scale[h] : 1.0;
+            scores[t * H + h] = (float)((b ? (double)b[h] : 0.0) + sx * sw * acc);
+        }
+    }
+}
+
+/*
+ * KVzap-MLP on quantised inputs: the first layer as above (X8, W18 [N1,Dh] E4M3,
+ * x_scale [T], w1_scale [N1]); GELU and the second layer (W2 [H,N1] bf16) unchanged.
+ *   z[j] = b1[j] + x_scale[t] * w1_scale[j] * sum_k X8[t,k] * W18[j,k]
+ *   scores[t,h] = b2[h] + sum_j GELU(z[j]) * W2[h,j]
+ * Returns 0, or -1 without memory.
+ */
+int kvzap_oracle_score_mlp_fp8(const uint8_t *X8, const float *x_scale, int64_t T, int Dh,
+                               const uint8_t *W18, const float *w1_scale, const float *b1, int N1,
+                               const uint16_t *W2, const float *b2, int H, float *scores)
+{
+    double *w1 = (double *)malloc(sizeof(double) * (size_t)Dh * (size_t)N1);
+    if (!w1) return -1;
+    for (int j = 0; j < N1; ++j)
+        for (int k = 0; k < Dh; ++k)
+            w1[(size_t)k * N1 + j] = kvzap_oracle_e4m3_to_double(W18[(size_t)j * Dh + k]);
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *z = (double *)malloc(sizeof(double) * (size_t)N1);
+        if (!z) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+            int64_t t;
+#pragma omp for schedule(static)
+            for (t = 0; t < T; ++t) {
+                for (int j = 0; j < N1; ++j) z[j] = 0.0;
+                for (int k = 0; k < Dh; ++k) {
+                    const double x = kvzap_oracle_e4m3_to_double(X8[t * Dh + k]);
+                    const double *row = w1 + (size_t)k * N1;
+                    for (int j = 0; j < N1; ++j) z[j] += x * row[j];
+                }
+                const double sx = x_scale ? (double)x_scale[t] : 1.0;
+                for (int j = 0; j < N1; ++j) {
+                    const double sw = w1_scale ? (double)w1_scale[j] : 1.0;
+                    z[j] = kvzap_oracle_gelu((b1 ? (double)b1[j] : 0.0) + sx * sw * z[j]);
+                }
+                for (int h = 0; h < H; ++h) {
+                    double sum = 0.0;
+                    for (int j = 0; j < N1; ++j) sum += z[j] * bf16_to_double(W2[(size_t)h * N1 + j]);
+                    scores[t * H + h] = (float)((b2 ? (double)b2[h] : 0.0) + sum);
+                }
+            }
+        }
+        free(z);
+    }
+    free(w1);
+    return failed ? -1 : 0;
+}
+
+/*
+ * kvzap_oracle_attention over a list whose rows are stored quantised (Related
+ * work, "Quantization"): K8, V8 [n,D] E4M3 bytes with one fp32 scale per row
+ * (k_scale, v_scale [n], NULL = 1), so that row i stands for k_scale[i] * K8[i]
+ * and v_scale[i] * V8[i]; q [G,D] stays bf16.
+ *   a[g,i] = scale * k_scale[i] * sum_d q[g,d] * K8[i,d]
+ *   out[g] = sum_i softmax_i(a[g,.]) * v_scale[i] * V8[i]
+ * Returns 0, or -1 without memory.
+ */
+int kvzap_oracle_attention_fp8(const uint16_t *q, int G, const uint8_t *K8, const float *k_scale,
+                               const uint8_t *V8, const float *v_scale, int64_t n, int D, double scale,
+                               float *out)
+{
+    double *a = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *acc = (double *)malloc(sizeof(double) * (size_t)D);
+    if (!a || !acc) { free(a); free(acc); return -1; }
+    for (int g = 0; g < G; ++g) {
+        double a_max = -INFINITY;
+        for (int64_t i = 0; i < n; ++i) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += bf16_to_double(q[(int64_t)g * D + d]) * kvzap_oracle_e4m3_to_double(K8[i * D + d]);
+            a[i] = scale * (k_scale ? (double)k_scale[i] : 1.0) * dot;
+            if (a[i] > a_max) a_max = a[i];
+        }
+        double denom = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            a[i] = exp(a[i] - a_max);
+            denom += a[i];
+        }
+        for (int d = 0; d < D; ++d) acc[d] = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            const double sv = v_scale ? (double)v_scale[i] : 1.0;
+            for (int d = 0; d < D; ++d)
+                acc[d] += a[i] * sv * kvzap_oracle_e4m3_to_double(V8[i * D + d]);
+        }
+        for (int d = 0; d < D; ++d) {
+            const double o = n > 0 ? acc[d] / denom : 0.0;
+            out[(int64_t)g * D + d] = (float)o;
+        }
+    }
+    free(a);
+    free(acc);
+    return 0;
+}

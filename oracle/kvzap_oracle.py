@@ -58,6 +58,11 @@ def lib():
         L.kvzap_oracle_layer_flops.argtypes = [ctypes.c_int] * 5
         L.kvzap_oracle_mlp_flops.argtypes = [ctypes.c_int] * 3
         L.kvzap_oracle_linear_flops.argtypes = [ctypes.c_int] * 2
+        L.kvzap_oracle_plan.restype = ctypes.c_int
+        L.kvzap_oracle_e4m3_to_double.restype = ctypes.c_double
+        L.kvzap_oracle_e4m3_to_double.argtypes = [ctypes.c_uint8]
+        L.kvzap_oracle_score_mlp_fp8.restype = ctypes.c_int
+        L.kvzap_oracle_attention_fp8.restype = ctypes.c_int
         L.kvzap_oracle_param_count.restype = ctypes.c_int64
         L.kvzap_oracle_param_count.argtypes = [ctypes.c_int] * 3
         _lib = L
@@ -277,6 +282,89 @@ def attention(q, K, V, scale):
     rc = lib().kvzap_oracle_attention(_c(q, ctypes.c_uint16), ctypes.c_int(G), _c(K, ctypes.c_uint16),
                                       _c(V, ctypes.c_uint16), ctypes.c_int64(K.shape[0]), ctypes.c_int(D),
                                       ctypes.c_double(scale), _c(out, ctypes.c_float))
+    if rc != 0:
+        raise MemoryError("oracle attention: out of memory")
+    return out
+
+
+def plan(keep, cu_seqlens=None, page_tokens=0, n_pages_pool=0, max_pages_per_list=1, first_page=0):
+    """Write plan: keep [H,T_total] -> (slot [T_total,H] int32, lengths [B,H]) for the dense-ragged layout, or
+    (slot, lengths, page_table [B*H,max_pages], n_pages_used) with slot = pool row when page_tokens > 0."""
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    H, T_total = keep.shape
+    cu = _cu(cu_seqlens, T_total)
+    B = len(cu) - 1
+    slot = np.full((T_total, H), -7, dtype=np.int32)
+    lengths = np.zeros((B, H), dtype=np.int32)
+    table = np.full((B * H, max_pages_per_list), -1, dtype=np.int32)
+    used = ctypes.c_int32(0)
+    rc = lib().kvzap_oracle_plan(
+        _c(keep, ctypes.c_uint8), _c(cu, ctypes.c_int32), ctypes.c_int(B), ctypes.c_int(H), ctypes.c_int(page_tokens),
+        ctypes.c_int32(first_page), ctypes.c_int64(n_pages_pool), ctypes.c_int(max_pages_per_list),
+        _c(slot, ctypes.c_int32), _c(table, ctypes.c_int32), _c(lengths, ctypes.c_int32), ctypes.byref(used))
+    if rc != 0:
+        raise ValueError("page pool or page table too small")
+    if page_tokens > 0:
+        return slot, lengths, table, int(used.value)
+    return slot, lengths
+
+
+def e4m3_to_double(bits: int) -> float:
+    """Exact value of one E4M3 byte (finite variant; 0x7f and 0xff are NaN)."""
+    return float(lib().kvzap_oracle_e4m3_to_double(ctypes.c_uint8(int(bits) & 0xFF)))
+
+
+def _u8(a, ndim):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint8 and a.ndim == ndim, (a.dtype, a.shape)
+    return a
+
+
+def score_linear_fp8(X8, x_scale, W8, w_scale, b=None):
+    """X8 [T,Dh], W8 [H,Dh] E4M3 bytes; x_scale [T], w_scale [H] fp32|None -> scores [T,H] fp32."""
+    X8, W8 = _u8(X8, 2), _u8(W8, 2)
+    T, Dh = X8.shape
+    H = W8.shape[0]
+    assert W8.shape[1] == Dh
+    x_scale, w_scale, b = _f32_or_none(x_scale, T), _f32_or_none(w_scale, H), _f32_or_none(b, H)
+    out = np.empty((T, H), dtype=np.float32)
+    lib().kvzap_oracle_score_linear_fp8(
+        _c(X8, ctypes.c_uint8), _c(x_scale, ctypes.c_float), ctypes.c_int64(T), ctypes.c_int(Dh),
+        _c(W8, ctypes.c_uint8), _c(w_scale, ctypes.c_float), _c(b, ctypes.c_float), ctypes.c_int(H), _c(out, ctypes.c_float))
+    return out
+
+
+def score_mlp_fp8(X8, x_scale, W18, w1_scale, b1, W2, b2):
+    """X8 [T,Dh], W18 [N1,Dh] E4M3 bytes with scales [T], [N1]; W2 [H,N1] bf16 bits -> scores [T,H] fp32."""
+    X8, W18, W2 = _u8(X8, 2), _u8(W18, 2), _u16(W2, 2)
+    T, Dh = X8.shape
+    N1, H = W18.shape[0], W2.shape[0]
+    assert W18.shape[1] == Dh and W2.shape[1] == N1
+    x_scale, w1_scale = _f32_or_none(x_scale, T), _f32_or_none(w1_scale, N1)
+    b1, b2 = _f32_or_none(b1, N1), _f32_or_none(b2, H)
+    out = np.empty((T, H), dtype=np.float32)
+    rc = lib().kvzap_oracle_score_mlp_fp8(
+        _c(X8, ctypes.c_uint8), _c(x_scale, ctypes.c_float), ctypes.c_int64(T), ctypes.c_int(Dh),
+        _c(W18, ctypes.c_uint8), _c(w1_scale, ctypes.c_float), _c(b1, ctypes.c_float), ctypes.c_int(N1),
+        _c(W2, ctypes.c_uint16), _c(b2, ctypes.c_float), ctypes.c_int(H), _c(out, ctypes.c_float))
+    if rc != 0:
+        raise MemoryError("oracle scratch allocation failed")
+    return out
+
+
+def attention_fp8(q, K8, k_scale, V8, v_scale, scale):
+    """q [G,D] bf16 bits; K8, V8 [n,D] E4M3 bytes with per-row scales [n] fp32|None -> out [G,D] fp32."""
+    q = _u16(q, 2)
+    G, D = q.shape
+    K8 = np.ascontiguousarray(K8, dtype=np.uint8).reshape(-1, D)
+    V8 = np.ascontiguousarray(V8, dtype=np.uint8).reshape(-1, D)
+    n = K8.shape[0]
+    assert V8.shape == K8.shape
+    k_scale, v_scale = _f32_or_none(k_scale, n), _f32_or_none(v_scale, n)
+    out = np.zeros((G, D), dtype=np.float32)
+    rc = lib().kvzap_oracle_attention_fp8(_c(q, ctypes.c_uint16), ctypes.c_int(G), _c(K8, ctypes.c_uint8),
+                                          _c(k_scale, ctypes.c_float), _c(V8, ctypes.c_uint8), _c(v_scale, ctypes.c_float),
+                                          ctypes.c_int64(n), ctypes.c_int(D), ctypes.c_double(scale), _c(out, ctypes.c_float))
     if rc != 0:
         raise MemoryError("oracle attention: out of memory")
     return out

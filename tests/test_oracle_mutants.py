@@ -12,7 +12,7 @@ import sys
 
 import pytest
 
-from tests import test_oracle_attention, test_oracle_prune, test_oracle_score, test_oracle_topk
+from tests import test_oracle_attention, test_oracle_fp8, test_oracle_plan, test_oracle_prune, test_oracle_score, test_oracle_topk
 
 _ORACLE_DIR = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle")
 
@@ -75,6 +75,8 @@ SCORE = _pins(test_oracle_score)
 PRUNE = _pins(test_oracle_prune)
 TOPK = _pins(test_oracle_topk)
 ATTN = _pins(test_oracle_attention)
+PLAN = _pins(test_oracle_plan)
+FP8 = _pins(test_oracle_fp8)
 
 MUTANTS = [
     # name, pins, text in the source, replacement
@@ -111,6 +113,21 @@ MUTANTS = [
     ("attention_no_scale", ATTN, "a[i] = scale * dot;", "a[i] = dot;"),
     ("attention_keys_for_values", ATTN, "acc[d] += a[i] * bf16_to_double(V[i * D + d]);", "acc[d] += a[i] * bf16_to_double(K[i * D + d]);"),
     ("attention_unnormalised", ATTN, "out[(int64_t)g * D + d] = n > 0 ? (float)(acc[d] / denom) : 0.0f;", "out[(int64_t)g * D + d] = n > 0 ? (float)(acc[d]) : 0.0f;"),
+    ("plan_counts_from_one", PLAN, "slot[t * H + h] = (int32_t)n;", "slot[t * H + h] = (int32_t)(n + 1);"),
+    ("plan_dropped_rows_get_a_slot", PLAN, "if (!keep[(int64_t)h * T_total + t]) continue;\n                if (page_tokens > 0)", "if (page_tokens > 0)"),
+    ("plan_pages_do_not_advance", PLAN, "cursor += need;\n            }\n        }\n    if (page_tokens > 0) *n_pages_used", "cursor += 0;\n            }\n        }\n    if (page_tokens > 0) *n_pages_used"),
+    ("plan_slot_ignores_the_page_offset", PLAN, "slot[t * H + h] = (int32_t)((cursor + n / page_tokens) * page_tokens + n % page_tokens);",
+     "slot[t * H + h] = (int32_t)((cursor + n / page_tokens) * page_tokens);"),
+    ("e4m3_bias_eight", FP8, "else v = ldexp(1.0 + (double)m / 8.0, e - 7);", "else v = ldexp(1.0 + (double)m / 8.0, e - 8);"),
+    ("e4m3_subnormals_as_normals", FP8, "if (e == 0) v = ldexp((double)m / 8.0, -6);", "if (e == 0) v = ldexp(1.0 + (double)m / 8.0, -7);"),
+    ("e4m3_has_infinities", FP8, "if (e == 15 && m == 7) return NAN;", "if (e == 15) return m == 0 ? INFINITY : NAN;"),
+    ("fp8_linear_drops_token_scale", FP8, "const double sx = x_scale ? (double)x_scale[t] : 1.0, sw = w_scale ? (double)w_scale[h] : 1.0;",
+     "const double sx = 1.0, sw = w_scale ? (double)w_scale[h] : 1.0;"),
+    ("fp8_mlp_scales_the_bias_too", FP8, "z[j] = kvzap_oracle_gelu((b1 ? (double)b1[j] : 0.0) + sx * sw * z[j]);",
+     "z[j] = kvzap_oracle_gelu(sx * sw * ((b1 ? (double)b1[j] : 0.0) + z[j]));"),
+    ("fp8_mlp_channel_scale_by_token", FP8, "const double sw = w1_scale ? (double)w1_scale[j] : 1.0;", "const double sw = w1_scale ? (double)w1_scale[j % 2] : 1.0;"),
+    ("fp8_attention_value_scale_dropped", FP8, "const double sv = v_scale ? (double)v_scale[i] : 1.0;", "const double sv = 1.0;"),
+    ("fp8_attention_key_scale_after_softmax", FP8, "a[i] = scale * (k_scale ? (double)k_scale[i] : 1.0) * dot;", "a[i] = scale * dot;"),
     ("attention_shared_query", ATTN, "dot += bf16_to_double(q[(int64_t)g * D + d]) * bf16_to_double(K[i * D + d]);", "dot += bf16_to_double(q[d]) * bf16_to_double(K[i * D + d]);"),
 ]
 
@@ -130,7 +147,7 @@ def build_dir(tmp_path_factory):
 
 def test_unmodified_source_passes_through_this_route(build_dir):
     mod = _load_variant(build_dir, "unmodified")
-    for pins in (SCORE, PRUNE, TOPK, ATTN):
+    for pins in (SCORE, PRUNE, TOPK, ATTN, PLAN, FP8):
         assert len(pins) >= 3
         assert _failures(mod, pins) == []
 
