@@ -300,6 +300,30 @@ kvzap_status kvzap_prefill_write_paged(kvzap_ctx *ctx, int32_t layer, const void
                                        float *scores_out, void *stream);
 
 /*
+ * Pruning on the write side without any copy: a write plan (Discussion, "Implementation Challenges": the
+ * surrogate needs only hidden states, so "pruning could also be applied before attention" -- here, before
+ * the keys and values are stored at all).  Scores the hidden states, applies threshold and window, and
+ * instead of moving rows tells the producer of K and V where every (token, head) pair belongs:
+ *   slot [n_tokens, H] int32 (out): the pair's destination row, or -1 if it is dropped.
+ *     page_tokens == 0: the row inside list (b,h), i.e. the number of kept positions of the list before the
+ *                       token; in the dense-ragged layout of kvzap_prune_prefill the producer writes the pair
+ *                       to row cu_seqlens[b] + slot of head h;
+ *     page_tokens  > 0: the row of the page pools, pages assigned exactly as by kvzap_prune_prefill_paged
+ *                       (page_table, n_pages_used, first_page, n_pages_pool, max_pages_per_list as there;
+ *                       on a pool or table that is too small every slot is -1 and the status word is set).
+ *   lengths [n_seqs, H] int32 (out);  scores_out [n_tokens, H] fp32 or NULL.
+ * A producer that writes each kept row to its slot gets exactly the output of kvzap_prefill_fused
+ * (kvzap_prefill_fused_paged), the dropped rows are never stored, and the library moves no K or V byte.
+ */
+kvzap_status kvzap_prefill_plan(kvzap_ctx *ctx, int32_t layer, const void *hidden,
+                                const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                float tau, int32_t w,
+                                int32_t *slot, int32_t *lengths, float *scores_out,
+                                int32_t page_tokens, int64_t n_pages_pool, int32_t first_page,
+                                int32_t *page_table, int32_t max_pages_per_list, int32_t *n_pages_used,
+                                void *stream);
+
+/*
  * Decode-time cache (caption of Algorithm 1: decoding is like prefilling but
  * needs a buffer of scores to enforce the sliding window; contributions:
  * delayed eviction with a sliding window).  One list per (sequence, layer, KV

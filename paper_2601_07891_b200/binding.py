@@ -55,6 +55,8 @@ SIGNATURES = {
                                          _i32, _i64, _vp, _vp, _i32, _vp, _vp]),
     "kvzap_prefill_fused_paged_host": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
                                               _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_plan": (_i32, [_vp, _i32, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _i32, _i64, _i32, _vp, _i32, _vp,
+                                  _vp]),
     "kvzap_prune_prefill_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _f32, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32, _i32,
                                          _vp, _i32, _vp, _vp, _vp]),
@@ -186,6 +188,17 @@ def kvzap_prefill_fused_host(handle, layer, hidden, K, V, cu_seqlens, n_seqs, ta
     _check(handle, load().kvzap_prefill_fused_host(
         handle, layer, _hptr(hidden), _hptr(K), _hptr(V), _hptr(cu_seqlens), n_seqs, n_tokens, tau, w,
         _hptr(K_out), _hptr(V_out), _hptr(lengths), _hptr(scores_out), _stream(stream)))
+
+
+def kvzap_prefill_plan(handle, layer, hidden, cu_seqlens, n_seqs, tau, w, slot, lengths, scores_out=None, page_tokens=0,
+                       n_pages_pool=0, first_page=0, page_table=None, n_pages_used=None, stream=None):
+    """Write plan: slot [n_tokens, H] int32 receives every pair's destination row (-1 = dropped)."""
+    n_tokens = hidden.shape[0]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_plan(
+        handle, layer, _ptr(hidden) if nz else None, _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(slot) if nz else None,
+        _ptr(lengths), _ptr(scores_out) if nz else None, page_tokens, n_pages_pool, first_page, _ptr(page_table),
+        page_table.shape[1] if page_table is not None else 0, _ptr(n_pages_used), _stream(stream)))
 
 
 def _hptr_array(tensors):

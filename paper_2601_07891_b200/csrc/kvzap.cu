@@ -74,6 +74,7 @@ struct kvzap_ctx {
     int32_t *tile_counters = nullptr;    // [kMaskRing] work-tile counters of the scoring launches, used in rotation
     uint32_t *select_hist = nullptr;     // fixed-budget selection: [4 passes][max_seqs][H][256] histograms
     float *select_tau = nullptr;         //                         [max_seqs][H] cut values when the caller wants none
+    float *plan_scores = nullptr;        // kvzap_prefill_plan without scores_out: [max_tokens][H] (allocated on first use)
     float *split_part = nullptr;         // few-token kernel: [sm_count tiles][4 slices][128][8] partial scores
     uint32_t *split_arrive = nullptr;    //                   [sm_count] arrival counts per tile
     uint64_t score_turn = 0;
@@ -313,6 +314,7 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->maskbits);
     cudaFree(ctx->tile_counters);
     cudaFree(ctx->split_part);
+    cudaFree(ctx->plan_scores);
     cudaFree(ctx->select_hist);
     cudaFree(ctx->select_tau);
     cudaFree(ctx->split_arrive);
@@ -761,7 +763,8 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
                                          const void *K, const void *V, const int32_t *cu_seqlens, int32_t n_seqs,
                                          int64_t n_tokens, void *K_out, void *V_out, int32_t *lengths, int32_t page_tokens,
                                          int32_t first_page, int64_t n_pages_pool, int32_t max_pages, int32_t *page_table,
-                                         int32_t *n_pages_used, cudaStream_t stream)
+                                         int32_t *n_pages_used, cudaStream_t stream, int32_t *slot_out = nullptr,
+                                         bool scores_just_made = false)
 {
     const kvzap_config &c = ctx->cfg;
     if (page_tokens > 0 && n_pages_pool * page_tokens >= 0xffffffffLL)
@@ -792,15 +795,16 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
     // Started before the work ahead of it has completed only on a context that trusts its producers,
     // directly behind another launch of this kernel (whose memory is on the pending list, and whose scratch
     // set is a different one for kOpRing - 2 launches in a row), and when it conflicts with none of them.
-    bool wait_first = !ctx->trusted || ctx->profiling || tau_list != nullptr || ctx->op_last_seq + 1 != ctx->op_seq ||
-                      ctx->op_chain >= kOpRing - 2;
+    bool wait_first = !ctx->trusted || ctx->profiling || tau_list != nullptr || scores_just_made ||
+                      ctx->op_last_seq + 1 != ctx->op_seq || ctx->op_chain >= kOpRing - 2;
     if (!wait_first)
         wait_first = hazard(ctx, scores, sc_bytes, false) || hazard(ctx, K, kv_bytes, false) || hazard(ctx, V, kv_bytes, false) ||
                      hazard(ctx, cu_seqlens, sizeof(int32_t) * (n_seqs + 1), false) ||
                      hazard(ctx, K_out, out_bytes, true) || hazard(ctx, V_out, out_bytes, true) ||
                      hazard(ctx, lengths, sizeof(int32_t) * n_lists, true) ||
                      hazard(ctx, page_table, sizeof(int32_t) * n_lists * max_pages, true) ||
-                     hazard(ctx, n_pages_used, sizeof(int32_t), true);
+                     hazard(ctx, n_pages_used, sizeof(int32_t), true) ||
+                     hazard(ctx, slot_out, sizeof(int32_t) * static_cast<size_t>(n_tokens) * c.n_kv_heads, true);
     if (wait_first) serial_point(ctx);
     else ctx->op_chain += 1;
     ctx->op_last_seq = ctx->op_seq;
@@ -810,6 +814,7 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
     note_range(ctx, K_out, out_bytes, true);
     note_range(ctx, V_out, out_bytes, true);
     note_range(ctx, lengths, sizeof(int32_t) * n_lists, true);
+    note_range(ctx, slot_out, sizeof(int32_t) * static_cast<size_t>(n_tokens) * c.n_kv_heads, true);
     if (page_tokens > 0) {
         note_range(ctx, page_table, sizeof(int32_t) * n_lists * max_pages, true);
         note_range(ctx, n_pages_used, sizeof(int32_t), true);
@@ -836,6 +841,7 @@ static kvzap_status launch_prune_onepass(kvzap_ctx *ctx, const float *scores, co
     p.in_stride_t = 1;
     p.row_units = c.head_dim / 8;
     p.lengths = lengths;
+    p.slot_out = slot_out;
     p.page_tokens = page_tokens;
     p.first_page = first_page;
     p.max_pages = max_pages;
@@ -1338,6 +1344,42 @@ kvzap_status kvzap_prefill_write(kvzap_ctx *ctx, int32_t layer, const void *hidd
 {
     return prefill_fused_impl(ctx, layer, hidden, K_proj, V_proj, cu_seqlens, n_seqs, n_tokens, tau, w, K_out, V_out,
                               lengths, scores_out, stream_, true);
+}
+
+kvzap_status kvzap_prefill_plan(kvzap_ctx *ctx, int32_t layer, const void *hidden, const int32_t *cu_seqlens, int32_t n_seqs,
+                                int64_t n_tokens, float tau, int32_t w, int32_t *slot, int32_t *lengths, float *scores_out,
+                                int32_t page_tokens, int64_t n_pages_pool, int32_t first_page, int32_t *page_table,
+                                int32_t max_pages_per_list, int32_t *n_pages_used, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_prefill_plan");
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (!lengths || w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "plan: lengths is NULL or w negative");
+    const bool paged = page_tokens > 0;
+    if (page_tokens < 0 || (paged && (!page_table || !n_pages_used || max_pages_per_list < 1 || n_pages_pool < 0 || first_page < 0)))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "plan: paged output needs page_table, n_pages_used, max_pages_per_list >= 1, first_page >= 0");
+    DeviceGuard guard(c.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * c.n_kv_heads, stream));
+        if (paged) KVZAP_CUDA(ctx, cudaMemsetAsync(n_pages_used, 0, sizeof(int32_t), stream));
+        return KVZAP_OK;
+    }
+    if (!hidden || !aligned16(hidden) || !slot) return fail(ctx, KVZAP_ERR_INVALID_ARG, "plan: hidden (16-byte aligned) and slot must not be NULL");
+    float *scores = scores_out;
+    if (!scores) {
+        if (!ctx->plan_scores) KVZAP_CUDA(ctx, cudaMalloc(&ctx->plan_scores, sizeof(float) * static_cast<size_t>(c.max_tokens) * c.n_kv_heads));
+        scores = ctx->plan_scores;
+    }
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores, nullptr, nullptr, 1, 0.0f, 0, stream);
+    if (st != KVZAP_OK) return st;
+    return launch_prune_onepass(ctx, scores, nullptr, tau, w, nullptr, nullptr, cu_seqlens, n_seqs, n_tokens, nullptr, nullptr, lengths,
+                                page_tokens, first_page, n_pages_pool, max_pages_per_list, page_table, n_pages_used, stream, slot, true);
 }
 
 kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream_)

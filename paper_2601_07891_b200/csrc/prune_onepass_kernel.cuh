@@ -55,6 +55,8 @@ struct PruneParams {
     int64_t in_stride_h, in_stride_t;
     int32_t row_units;
     int32_t *lengths;
+    int32_t *slot_out;         // write plan [n_tokens][n_heads]: when given, no row is moved; every (token, head) gets its
+                               // destination row (inside its list, or the pool row when paged), -1 when dropped
     // paged output (page_tokens > 0)
     int32_t page_tokens, first_page, max_pages;
     int64_t n_pages_pool;
@@ -443,7 +445,10 @@ prune_onepass_kernel(const PruneParams p)
             const uint32_t wq = tok < 32 ? w.x : tok < 64 ? w.y : tok < 96 ? w.z : w.w;
             const bool keep = (wq >> (tok & 31)) & 1u;
             const bool last = t + 1 == e && !paged;
-            if (!keep && !last) continue;
+            if (!keep && !last) {
+                if (p.slot_out != nullptr) p.slot_out[t * H + h] = -1;
+                continue;
+            }
             const int r = popc_below(w.x, w.y, w.z, w.w, tok);
             int32_t n = runb_s[pi] + r;                       // rank inside list (b,h)
             if (multi) n -= s >= sb_start ? kept_before_local(hh, s) : base_s[h];
@@ -455,13 +460,18 @@ prune_onepass_kernel(const PruneParams p)
                 } else {
                     dst = static_cast<int64_t>(h) * p.n_tokens + s + n;
                 }
-                ent_s[off_s[pi] + r] =
-                    make_longlong2((h * p.in_stride_h + t * p.in_stride_t) * row_bytes, dst < 0 ? -1 : dst * row_bytes);
+                if (p.slot_out != nullptr)
+                    p.slot_out[t * H + h] = static_cast<int32_t>(paged ? dst : n);
+                else
+                    ent_s[off_s[pi] + r] =
+                        make_longlong2((h * p.in_stride_h + t * p.in_stride_t) * row_bytes, dst < 0 ? -1 : dst * row_bytes);
+            } else if (p.slot_out != nullptr) {
+                p.slot_out[t * H + h] = -1;
             }
             if (last) p.lengths[b * H + h] = n + (keep ? 1 : 0);
         }
         __syncthreads();
-        for (int u0 = gl; u0 < p.row_units; u0 += 16) {
+        for (int u0 = gl; u0 < p.row_units && p.slot_out == nullptr; u0 += 16) {
             // two register sets: the loads of one are in flight while the other is stored
             const int64_t lane_off = static_cast<int64_t>(u0) * 16;
             uint4 ka[kRows], va[kRows], kb[kRows], vb[kRows];
