@@ -130,6 +130,32 @@ kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int6
                          float *scores, void *stream);
 
 /*
+ * 8-bit floating point inputs (Related work, "Quantization": pruning composes with quantisation; the paper
+ * fixes no format).  Format used here: OCP E4M3 in its finite variant (1 sign, 4 exponent bits with bias 7, 3
+ * mantissa bits, no infinities, S.1111.111 = NaN), one fp32 scale per token for the hidden states and one per
+ * output row for the first-layer weights -- a value stands for scale * E4M3(byte).  The first layer then runs
+ * on the tensor cores' 8-bit path (twice the bf16 rate, half the bytes per hidden state):
+ *   Linear: scores[t,h] = b1[h] + x_scale[t] * w1_scale[h] * sum_k X8[t,k] W8[h,k]
+ *   MLP:    z[j] = b1[j] + x_scale[t] * w1_scale[j] * sum_k X8[t,k] W8[j,k];  scores as kvzap_score from z
+ * kvzap_set_weights_fp8: W1_e4m3 [rows, d_model] bytes (rows = H or hidden), w1_scale [rows] fp32 (NULL = 1),
+ * b1, W2 (bf16), b2 as in kvzap_set_weights.  A layer holds either kind of weights; the calls of the other
+ * kind return KVZAP_ERR_STATE for it.  d_model must be a multiple of 128 (else KVZAP_ERR_UNSUPPORTED).
+ * kvzap_score_fp8 / kvzap_prefill_fused_fp8: hidden_e4m3 [n_tokens, d_model] bytes (device, 16-byte aligned),
+ * x_scale [n_tokens] fp32 (device, NULL = 1); everything else as kvzap_score / kvzap_prefill_fused (K and V stay
+ * bf16 rows, or any rows of head_dim * 2 bytes: the compaction copies bytes).
+ */
+kvzap_status kvzap_set_weights_fp8(kvzap_ctx *ctx, int32_t layer, const void *W1_e4m3, const float *w1_scale,
+                                   const float *b1, const void *W2, const float *b2, void *stream);
+kvzap_status kvzap_score_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale,
+                             int64_t n_tokens, float *scores, void *stream);
+kvzap_status kvzap_prefill_fused_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale,
+                                     const void *K, const void *V,
+                                     const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens,
+                                     float tau, int32_t w,
+                                     void *K_out, void *V_out, int32_t *lengths,
+                                     float *scores_out, void *stream);
+
+/*
  * Threshold + sliding window + per-(sequence, head) ordered compaction
  * (Algorithm 1, the steps after scoring; Method, "KVzap": pairs whose score falls below tau
  * are discarded, the most recent w tokens are kept).

@@ -57,6 +57,9 @@ SIGNATURES = {
                                               _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_plan": (_i32, [_vp, _i32, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _i32, _i64, _i32, _vp, _i32, _vp,
                                   _vp]),
+    "kvzap_set_weights_fp8": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "kvzap_score_fp8": (_i32, [_vp, _i32, _vp, _vp, _i64, _vp, _vp]),
+    "kvzap_prefill_fused_fp8": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_noalloc": (_i32, [_vp, _vp, _vp, _vp, _i32, _i64, _i32, _i32, _f32, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_paged": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32, _i32,
                                          _vp, _i32, _vp, _vp, _vp]),
@@ -199,6 +202,28 @@ def kvzap_prefill_plan(handle, layer, hidden, cu_seqlens, n_seqs, tau, w, slot, 
         handle, layer, _ptr(hidden) if nz else None, _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(slot) if nz else None,
         _ptr(lengths), _ptr(scores_out) if nz else None, page_tokens, n_pages_pool, first_page, _ptr(page_table),
         page_table.shape[1] if page_table is not None else 0, _ptr(n_pages_used), _stream(stream)))
+
+
+def kvzap_set_weights_fp8(handle, layer, W1_e4m3, w1_scale, b1=None, W2=None, b2=None, stream=None):
+    """W1_e4m3: uint8 tensor [rows, d_model] of E4M3 bytes; w1_scale fp32 [rows] or None."""
+    _check(handle, load().kvzap_set_weights_fp8(handle, layer, _ptr(W1_e4m3), _ptr(w1_scale), _ptr(b1), _ptr(W2), _ptr(b2),
+                                                _stream(stream)))
+
+
+def kvzap_score_fp8(handle, layer, hidden_e4m3, x_scale, scores, stream=None):
+    n_tokens = hidden_e4m3.shape[0]
+    _check(handle, load().kvzap_score_fp8(handle, layer, _ptr(hidden_e4m3) if n_tokens else None, _ptr(x_scale), n_tokens,
+                                          _ptr(scores) if n_tokens else None, _stream(stream)))
+
+
+def kvzap_prefill_fused_fp8(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                            scores_out=None, stream=None):
+    n_tokens = K.shape[1]
+    nz = n_tokens > 0
+    _check(handle, load().kvzap_prefill_fused_fp8(
+        handle, layer, _ptr(hidden_e4m3) if nz else None, _ptr(x_scale), _ptr(K) if nz else None, _ptr(V) if nz else None,
+        _ptr(cu_seqlens), n_seqs, n_tokens, tau, w, _ptr(K_out) if nz else None, _ptr(V_out) if nz else None,
+        _ptr(lengths), _ptr(scores_out) if nz else None, _stream(stream)))
 
 
 def _hptr_array(tensors):

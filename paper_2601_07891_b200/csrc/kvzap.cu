@@ -66,6 +66,12 @@ struct kvzap_ctx {
     float *w2t_all = nullptr;        // [L][hidden][8] fp32 (MLP)
     float *b2_all = nullptr;         // [L][8] (MLP)
     std::vector<char> layer_set;
+    // layers whose first layer was given as E4M3 bytes (kvzap_set_weights_fp8): K-blocked copy with 128 elements
+    // per block, one scale per output row; allocated when the first such layer arrives
+    void *w1_fp8_all = nullptr;      // [d_model / 128][L * w1_rows][128] bytes
+    float *w1_scale_all = nullptr;   // [L][w1_rows]
+    std::vector<char> layer_fp8;
+    CUtensorMap tmap_w8[2];          // boxes as sched[].tmap_w
     kvzap::EncodeTiledFn encode = nullptr;
     // scratch
     int64_t max_blocks = 0, max_words = 0;
@@ -209,6 +215,30 @@ static kvzap_status make_tmap(kvzap_ctx *ctx, CUtensorMap *map, const void *base
     return KVZAP_OK;
 }
 
+// 8-bit tensor map over `slabs` matrices of `rows` x `cols` bytes; box = box_rows rows x 128 bytes, 128-byte swizzle.
+// inner_blocked: the matrix is stored K block by K block, [cols / 128][rows][128] (the weights' copy).
+static kvzap_status make_tmap8(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+                               uint64_t slabs, bool inner_blocked)
+{
+    cuuint64_t dims[3], strides[2];
+    if (inner_blocked) {
+        dims[0] = 128; dims[1] = rows; dims[2] = cols / 128;
+        strides[0] = 128; strides[1] = 128 * rows;
+    } else {
+        dims[0] = cols; dims[1] = rows; dims[2] = slabs ? slabs : 1;
+        strides[0] = cols; strides[1] = cols * rows;
+    }
+    const cuuint32_t box[3] = {128, box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims, strides, box, estr,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, KVZAP_ERR_CUDA, "cuTensorMapEncodeTiled (8-bit) failed with code %d (rows=%llu cols=%llu box_rows=%u)",
+                    static_cast<int>(r), static_cast<unsigned long long>(rows), static_cast<unsigned long long>(cols), box_rows);
+    return KVZAP_OK;
+}
+
 // Tensor map over the context's copy of the first-layer weights, stored K block by K block:
 // [k_blocks][rows_total][64] bf16, so that the `box_rows` x 64 tile a CTA stages per K step is one
 // contiguous piece of memory (a decode step reads every weight byte from HBM exactly once; contiguous
@@ -240,6 +270,25 @@ __global__ void pack_w1_kernel(const uint4 *__restrict__ W1, int rows, int d_mod
     const int r = static_cast<int>(idx / units_per_row), u = static_cast<int>(idx % units_per_row);
     const int kb = u / (kBlockK / 8), xu = u % (kBlockK / 8);
     dst[(static_cast<int64_t>(kb) * rows_total + row0 + r) * (kBlockK / 8) + xu] = W1[idx];
+}
+
+// The same for E4M3 bytes: 128 elements per K block, one thread moves 16 of them (16 bytes).
+__global__ void pack_w1_fp8_kernel(const uint4 *__restrict__ W1, int rows, int d_model, int64_t rows_total, int64_t row0,
+                                   uint4 *__restrict__ dst)
+{
+    const int units_per_row = d_model / 16;
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<int64_t>(rows) * units_per_row) return;
+    const int r = static_cast<int>(idx / units_per_row), u = static_cast<int>(idx % units_per_row);
+    const int kb = u / 8, xu = u % 8;
+    dst[(static_cast<int64_t>(kb) * rows_total + row0 + r) * 8 + xu] = W1[idx];
+}
+
+// out[i] = src ? src[i] : 1 for i < n, 1 (unused rows) up to n_pad
+__global__ void fill_scale_kernel(const float *__restrict__ src, int n, int n_pad, float *__restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_pad) out[i] = (src != nullptr && i < n) ? src[i] : 1.0f;
 }
 
 // W2 [H, hidden] bf16 -> w2t [hidden][8] fp32 (zero for heads >= H); b2 -> [8] fp32.
@@ -311,6 +360,8 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->b1_all);
     cudaFree(ctx->w2t_all);
     cudaFree(ctx->b2_all);
+    cudaFree(ctx->w1_fp8_all);
+    cudaFree(ctx->w1_scale_all);
     cudaFree(ctx->maskbits);
     cudaFree(ctx->tile_counters);
     cudaFree(ctx->split_part);
@@ -715,6 +766,94 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     return KVZAP_OK;
 }
 
+// Scoring with 8-bit inputs: hidden [n_tokens][d_model] E4M3 bytes with one scale per token, the layer's first-layer
+// weights given by kvzap_set_weights_fp8.  Always the persistent kernel (CTA pairs for the MLP from two blocks on);
+// the waits before loads and stores follow the rules of launch_score.
+static kvzap_status launch_score_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden8, const float *x_scale, int64_t n_tokens,
+                                     float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs, float tau,
+                                     int32_t w, cudaStream_t stream)
+{
+    const kvzap_config &c = ctx->cfg;
+    const int64_t blocks_per_layer = (n_tokens + kTileM - 1) / kTileM;
+    const bool pair = c.hidden > 0 && ctx->pair_clusters > 0 && blocks_per_layer >= 2;
+    const kvzap_ctx::Schedule &sc = ctx->sched[pair ? 1 : 0];
+    const int64_t n_tiles = pair ? (blocks_per_layer + 1) / 2 : blocks_per_layer;
+    CUtensorMap tmap_x;
+    kvzap_status st = make_tmap8(ctx, &tmap_x, hidden8, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model), kTileM, 1, false);
+    if (st != KVZAP_OK) return st;
+    ScoreParams p;
+    memset(&p, 0, sizeof p);
+    p.n_tokens = n_tokens;
+    p.n_tiles = static_cast<int32_t>(n_tiles);
+    p.tiles_per_layer = static_cast<int32_t>(n_tiles);
+    p.blocks_per_layer = static_cast<int32_t>(blocks_per_layer);
+    p.n_layers_call = 1;
+    p.layer0 = layer;
+    p.w_rows = ctx->w1_rows;
+    p.d_model = c.d_model;
+    p.group_w = sc.group_w;
+    p.n_groups = sc.n_groups;
+    p.chunk_n = sc.chunk_n;
+    p.n_chunks = sc.n_chunks;
+    p.n_stages = sc.n_stages;
+    p.acc_bufs = sc.acc_bufs;
+    p.acc_stride = sc.acc_stride;
+    p.tmem_cols = sc.tmem_cols;
+    p.n_hidden = c.hidden;
+    p.n_heads = c.n_kv_heads;
+    p.b1 = ctx->b1_all;
+    p.w2t = ctx->w2t_all;
+    p.b2 = ctx->b2_all;
+    p.scores = scores;
+    p.maskbits = maskbits;
+    p.n_words = blocks_per_layer * 4;
+    p.cu_seqlens = cu_seqlens;
+    p.n_seqs = n_seqs;
+    p.window = w;
+    p.window_keep = 1;
+    p.tau = tau;
+    p.status = ctx->status_dev;
+    p.wait_before_load = ctx->trusted ? 0 : 1;
+    p.k_blocks = c.d_model / 128;
+    p.k_elems = 128;
+    p.x_scale = x_scale;
+    p.w1_scale = ctx->w1_scale_all;
+    p.tile_counter = ctx->tile_counters + ctx->score_turn % kMaskRing;
+    p.tile_counter_reset = ctx->tile_counters + (ctx->score_turn + 2) % kMaskRing;
+    ctx->score_turn += 1;
+    const size_t scores_bytes = scores ? sizeof(float) * static_cast<size_t>(n_tokens) * c.n_kv_heads : 0;
+    bool scores_clash = scores != nullptr && hazard(ctx, scores, scores_bytes, true);
+    if (scores && ctx->last_scores) {
+        const char *a0 = reinterpret_cast<const char *>(scores), *b0 = static_cast<const char *>(ctx->last_scores);
+        scores_clash = scores_clash || (a0 < b0 + ctx->last_scores_bytes && b0 < a0 + scores_bytes);
+    }
+    ctx->last_scores = scores;
+    ctx->last_scores_bytes = scores_bytes;
+    ctx->last_score_early = false;
+    {
+        ProfScope prof(ctx, KVZAP_KERNEL_SCORE, stream);
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[2];
+        const bool early = !ctx->profiling;
+        if (pair) {
+            const int n_clusters = static_cast<int>(n_tiles < ctx->pair_clusters ? n_tiles : ctx->pair_clusters);
+            p.wait_before_write = (scores_clash || 2 * n_clusters < ctx->sm_count / 2 * 2) ? 1 : 0;
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(2 * n_clusters)), dim3(kScoreThreads), sc.smem, stream, early, 2);
+            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, true, true>, tmap_x, ctx->tmap_w8[1], p));
+        } else {
+            const int grid = static_cast<int>(n_tiles < ctx->sm_count ? n_tiles : ctx->sm_count);
+            p.wait_before_write = (scores_clash || grid < ctx->sm_count) ? 1 : 0;
+            make_launch(&cfg, attrs, dim3(static_cast<unsigned>(grid)), dim3(kScoreThreads), sc.smem, stream, early, 1);
+            if (c.hidden > 0)
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<true, false, true>, tmap_x, ctx->tmap_w8[0], p));
+            else
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_kernel<false, false, true>, tmap_x, ctx->tmap_w8[0], p));
+        }
+    }
+    ctx->launches += 1;
+    return KVZAP_OK;
+}
+
 // Dense-ragged compaction over the mask words in `mask` (one kernel, no scan pass).
 static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, const void *K, const void *V,
                                       const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, void *K_out,
@@ -1036,6 +1175,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     }
 
     ctx->layer_set.assign(c.n_layers, 0);
+    ctx->layer_fp8.assign(c.n_layers, 0);
     {
         const size_t w1_bytes = static_cast<size_t>(c.n_layers) * ctx->w1_rows * c.d_model * 2;
         CREATE_CUDA(cudaMalloc(&ctx->w1_all, w1_bytes));
@@ -1204,7 +1344,119 @@ kvzap_status kvzap_set_weights(kvzap_ctx *ctx, int32_t layer, const void *W1, co
         ctx->launches += 1;
     }
     ctx->layer_set[layer] = 1;
+    ctx->layer_fp8[layer] = 0;
     return KVZAP_OK;
+}
+
+kvzap_status kvzap_set_weights_fp8(kvzap_ctx *ctx, int32_t layer, const void *W1_e4m3, const float *w1_scale, const float *b1,
+                                   const void *W2, const float *b2, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_set_weights_fp8");
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    serial_point(ctx);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    if (layer < 0 || layer >= c.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    if (c.d_model % 128) return fail(ctx, KVZAP_ERR_UNSUPPORTED, "8-bit inputs need d_model to be a multiple of 128 (is %d)", c.d_model);
+    if (!W1_e4m3 || !aligned16(W1_e4m3)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "W1 must be non-NULL and 16-byte aligned");
+    if (c.hidden == 0 && (W2 || b2)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-Linear takes no W2/b2");
+    if (c.hidden > 0 && !W2) return fail(ctx, KVZAP_ERR_INVALID_ARG, "KVzap-MLP needs W2");
+    DeviceGuard guard(c.device);
+    const int rows = c.hidden > 0 ? c.hidden : c.n_kv_heads;
+    const int64_t rows_total = static_cast<int64_t>(c.n_layers) * ctx->w1_rows;
+    if (!ctx->w1_fp8_all) {
+        const size_t bytes = static_cast<size_t>(rows_total) * c.d_model;
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->w1_fp8_all, bytes));
+        KVZAP_CUDA(ctx, cudaMemsetAsync(ctx->w1_fp8_all, 0, bytes, stream));
+        KVZAP_CUDA(ctx, cudaMalloc(&ctx->w1_scale_all, sizeof(float) * rows_total));
+        for (int mode = 0; mode < (c.hidden > 0 ? 2 : 1); ++mode) {
+            kvzap_status st = make_tmap8(ctx, &ctx->tmap_w8[mode], ctx->w1_fp8_all, static_cast<uint64_t>(rows_total),
+                                         static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(ctx->sched[mode].chunk_n / (mode + 1)), 0, true);
+            if (st != KVZAP_OK) return st;
+        }
+        if (c.hidden > 0) {
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(ctx->sched[0].smem)));
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(ctx->sched[1].smem)));
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<true, false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<true, true, true>, cudaFuncAttributePreferredSharedMemoryCarveout, static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+        } else {
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(ctx->sched[0].smem)));
+            KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<false, false, true>, cudaFuncAttributePreferredSharedMemoryCarveout, static_cast<int>(cudaSharedmemCarveoutMaxShared)));
+        }
+    }
+    {
+        const int64_t units = static_cast<int64_t>(rows) * (c.d_model / 16);
+        pack_w1_fp8_kernel<<<static_cast<unsigned>((units + 255) / 256), 256, 0, stream>>>(
+            static_cast<const uint4 *>(W1_e4m3), rows, c.d_model, rows_total, static_cast<int64_t>(layer) * ctx->w1_rows,
+            static_cast<uint4 *>(ctx->w1_fp8_all));
+        fill_scale_kernel<<<(ctx->w1_rows + 255) / 256, 256, 0, stream>>>(w1_scale, rows, ctx->w1_rows,
+                                                                         ctx->w1_scale_all + static_cast<size_t>(layer) * ctx->w1_rows);
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 2;
+    }
+    float *b1_dst = ctx->b1_all + static_cast<size_t>(layer) * ctx->w1_rows;
+    if (b1)
+        KVZAP_CUDA(ctx, cudaMemcpyAsync(b1_dst, b1, sizeof(float) * rows, cudaMemcpyDeviceToDevice, stream));
+    else
+        KVZAP_CUDA(ctx, cudaMemsetAsync(b1_dst, 0, sizeof(float) * rows, stream));
+    if (c.hidden > 0) {
+        const int n = c.hidden * kMaxHeads;
+        pack_w2_kernel<<<(n + 255) / 256, 256, 0, stream>>>(static_cast<const uint16_t *>(W2), b2, c.n_kv_heads, c.hidden,
+                                                            ctx->w2t_all + static_cast<size_t>(layer) * n,
+                                                            ctx->b2_all + static_cast<size_t>(layer) * kMaxHeads);
+        KVZAP_CUDA(ctx, cudaGetLastError());
+        ctx->launches += 1;
+    }
+    ctx->layer_set[layer] = 0;       // the bf16 entry points refuse this layer from now on
+    ctx->layer_fp8[layer] = 1;
+    return KVZAP_OK;
+}
+
+kvzap_status kvzap_score_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale, int64_t n_tokens,
+                             float *scores, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_score_fp8");
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, 1, nullptr);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_fp8[layer])
+        return fail(ctx, KVZAP_ERR_STATE, "layer %d has no 8-bit weights (kvzap_set_weights_fp8)", layer);
+    if (n_tokens == 0) return KVZAP_OK;
+    if (!hidden_e4m3 || !scores || !aligned16(hidden_e4m3)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden (16-byte aligned) and scores must not be NULL");
+    DeviceGuard guard(ctx->cfg.device);
+    return launch_score_fp8(ctx, layer, hidden_e4m3, x_scale, n_tokens, scores, nullptr, nullptr, 1, 0.0f, 0, static_cast<cudaStream_t>(stream_));
+}
+
+kvzap_status kvzap_prefill_fused_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale, const void *K,
+                                     const void *V, const int32_t *cu_seqlens, int32_t n_seqs, int64_t n_tokens, float tau,
+                                     int32_t w, void *K_out, void *V_out, int32_t *lengths, float *scores_out, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_prefill_fused_fp8");
+    if (!ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_fp8[layer])
+        return fail(ctx, KVZAP_ERR_STATE, "layer %d has no 8-bit weights (kvzap_set_weights_fp8)", layer);
+    if (!lengths) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths is NULL");
+    if (w < 0) return fail(ctx, KVZAP_ERR_INVALID_ARG, "window w is negative");
+    DeviceGuard guard(ctx->cfg.device);
+    if (n_tokens == 0) {
+        KVZAP_CUDA(ctx, cudaMemsetAsync(lengths, 0, sizeof(int32_t) * n_seqs * ctx->cfg.n_kv_heads, stream));
+        return KVZAP_OK;
+    }
+    st = check_prune_args(ctx, K, V, K_out, V_out, lengths, w);
+    if (st != KVZAP_OK) return st;
+    if (!hidden_e4m3 || !aligned16(hidden_e4m3)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
+    uint32_t *mask = next_mask_slice(ctx);
+    st = launch_score_fp8(ctx, layer, hidden_e4m3, x_scale, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
+    if (st != KVZAP_OK) return st;
+    return launch_compaction(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_out, V_out, lengths, stream, true, false);
 }
 
 kvzap_status kvzap_score(kvzap_ctx *ctx, int32_t layer, const void *hidden, int64_t n_tokens, float *scores,

@@ -78,6 +78,12 @@ struct ScoreParams {
     int32_t wait_before_load;     // 1: every thread waits for the work ahead in the stream before caller data is read
     int32_t *tile_counter;        // work tiles handed out beyond the first one of every CTA (or pair); starts at 0
     int32_t *tile_counter_reset;  // the counter of the launch after next: set to 0 by this launch
+    // 8-bit inputs (score_kernel<.., .., true>): hidden states and first-layer weights are E4M3 bytes, a 128-byte
+    // swizzled row then holds 128 elements
+    int32_t k_blocks;             // K blocks per row of X (0: d_model / 64, the bf16 layout)
+    int32_t k_elems;              // elements per K block (0: 64)
+    const float *x_scale;         // [n_layers_call][n_tokens] one scale per token, or nullptr (= 1)
+    const float *w1_scale;        // stacked over all layers [L][w_rows], one scale per first-layer output row
     // few-token kernel only: the clusters of one tile combine their partial scores through global memory
     float *split_part;            // [n_tiles][n_split][128][8]
     uint32_t *split_arrive;       // [n_tiles] arrivals so far, over all launches (never reset in normal use)
@@ -86,7 +92,7 @@ struct ScoreParams {
 // Byte offsets inside the dynamic shared memory block (after 1024-byte alignment).
 // `b_rows` = rows of W1 one CTA stages per K step (group_w, or group_w / 2 for a pair).
 struct ScoreSmemLayout {
-    uint32_t stage_bytes, stages_end, w2s, b1s, part, bars, total;
+    uint32_t stage_bytes, stages_end, w2s, b1s, w1s, part, bars, total;
 };
 __host__ __device__ inline ScoreSmemLayout score_smem_layout(int b_rows, int n_stages, int n_hidden)
 {
@@ -95,7 +101,8 @@ __host__ __device__ inline ScoreSmemLayout score_smem_layout(int b_rows, int n_s
     L.stages_end = L.stage_bytes * n_stages;
     L.w2s = L.stages_end;
     L.b1s = L.w2s + static_cast<uint32_t>(n_hidden) * kMaxHeads * 4;
-    L.part = L.b1s + static_cast<uint32_t>(n_hidden) * 4;
+    L.w1s = L.b1s + static_cast<uint32_t>(n_hidden) * 4;        // first-layer row scales (8-bit inputs)
+    L.part = L.w1s + static_cast<uint32_t>(n_hidden) * 4;
     L.bars = L.part + kTileM * kMaxHeads * 4;
     L.total = L.bars + 512;
     return L;
@@ -162,11 +169,34 @@ __device__ __forceinline__ void mlp_columns(const uint32_t (&r)[kCols], int j0, 
     }
 }
 
+// The same with the pre-activation scaled first: z = r * (scale of the token) * (scale of the hidden unit) + b1.
+template <int kCols>
+__device__ __forceinline__ void mlp_columns_scaled(const uint32_t (&r)[kCols], int j0, const float *b1s, const float *w1s,
+                                                   uint64_t sx2, const ulonglong2 *w2p, uint64_t (&acc)[kMaxHeads])
+{
+#pragma unroll
+    for (int i = 0; i < kCols; i += 2) {
+        const int j = j0 + i;
+        const float2 b = *reinterpret_cast<const float2 *>(b1s + j);
+        const float2 sw = *reinterpret_cast<const float2 *>(w1s + j);
+        const uint64_t z2 = f2_fma(f2_pack(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), f2_mul(f2_pack(sw.x, sw.y), sx2),
+                                   f2_pack(b.x, b.y));
+        const uint64_t g2 = gelu_pair(z2);
+        const ulonglong2 *w = w2p + (j >> 1) * 4;
+#pragma unroll
+        for (int hp = 0; hp < 4; ++hp) {
+            const ulonglong2 ww = w[hp];
+            acc[2 * hp] = f2_fma(g2, ww.x, acc[2 * hp]);
+            acc[2 * hp + 1] = f2_fma(g2, ww.y, acc[2 * hp + 1]);
+        }
+    }
+}
+
 // Issues the MMAs of one 64-element K block: kBlockK / kUmmaK steps times kChunks accumulator chunks,
 // fully unrolled, descriptors formed by adding constants to the low word (the start-address field).
 // a_lo / b_lo: low descriptor words of the stage's A tile and first B chunk; `first` = this is the
 // first K block of the accumulation (its first step overwrites the accumulator).
-template <bool kPair, int kChunks>
+template <bool kPair, int kChunks, bool kFp8 = false>
 __device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
                                               uint32_t b_chunk_step, uint32_t chunk_n, uint32_t idesc, bool first)
 {
@@ -178,8 +208,13 @@ __device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint32_t a_lo, ui
             const uint64_t a_desc = (static_cast<uint64_t>(desc_hi) << 32) | (a_lo + 2 * k);
             const uint64_t b_desc = (static_cast<uint64_t>(desc_hi) << 32) | (b_lo + c * b_chunk_step + 2 * k);
             const uint32_t acc = (k != 0 || !first) ? 1u : 0u;
-            if constexpr (kPair) umma_bf16_pair(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
-            else umma_bf16(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+            if constexpr (kFp8) {
+                if constexpr (kPair) umma_fp8_pair(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+                else umma_fp8(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+            } else {
+                if constexpr (kPair) umma_bf16_pair(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+                else umma_bf16(d_tmem + c * chunk_n, a_desc, b_desc, idesc, acc);
+            }
         }
     }
 }
@@ -187,7 +222,7 @@ __device__ __forceinline__ void issue_k_block(uint32_t d_tmem, uint32_t a_lo, ui
 // At most 128 registers per thread: the register file is split over the SM's four schedulers, three
 // of this kernel's ten warps share one of them, and a warp of the compaction kernel must still fit
 // beside them for the two kernels to run on the same SM at the same time.
-template <bool kMlp, bool kPair>
+template <bool kMlp, bool kPair, bool kFp8 = false>
 __global__ void __maxnreg__(128)
 score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
              const ScoreParams p)
@@ -205,6 +240,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     ulonglong2 *w2p = reinterpret_cast<ulonglong2 *>(smem + L.w2s);
     float *w2f = reinterpret_cast<float *>(smem + L.w2s);
     float *b1s = reinterpret_cast<float *>(smem + L.b1s);
+    float *w1s = reinterpret_cast<float *>(smem + L.w1s);
     float *part = reinterpret_cast<float *>(smem + L.part);
     const uint32_t bars = smem_base + L.bars;
     const uint32_t bar_full = bars;                      // [kMaxStages] TMA -> MMA (the pair's first CTA's is used)
@@ -278,7 +314,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     // vouches for the producers of its inputs, nothing of them is read before that work has completed.
     if (p.wait_before_load) griddep_wait();
 
-    const int k_blocks = p.d_model / kBlockK;
+    const int k_blocks = p.k_blocks > 0 ? p.k_blocks : p.d_model / kBlockK;
+    const int k_elems = p.k_elems > 0 ? p.k_elems : kBlockK;
     if (blockIdx.x == 0 && threadIdx.x == 0) *p.tile_counter_reset = 0;
 
     // The seq-th work tile of this CTA (pair), as published by the scheduler; -1 if the kernel is
@@ -348,7 +385,7 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                 const uint64_t pol_x = (g + 1 < p.n_groups) ? pol_xn : pol_x1;
                 for (int i = 0; i < k_blocks; ++i, ++it) {
                     const int kb = backwards ? k_blocks - 1 - i : i;
-                    const int kx = kb * kBlockK;
+                    const int kx = kb * k_elems;
                     if (!__all_sync(0xffffffffu, mbar_wait(bar_empty + 8 * st, st_par, abort_flag))) {
                         ok = false;
                         break;
@@ -409,7 +446,8 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (a pair: its first CTA only)
         if (leader) {
-            const uint32_t idesc = umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.chunk_n));
+            const uint32_t idesc = kFp8 ? umma_idesc_e4m3_f32(kTileM * kCtas, static_cast<uint32_t>(p.chunk_n))
+                                        : umma_idesc_bf16_f32(kTileM * kCtas, static_cast<uint32_t>(p.chunk_n));
             // operand descriptors: constant high word, low word = (address >> 4) | fixed fields
             const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
             const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
@@ -443,9 +481,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                         if (elected) {
                             const uint32_t b_lo = a_lo + (kATileBytes >> 4);
                             if (p.n_chunks == 1)
-                                issue_k_block<kPair, 1>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
+                                issue_k_block<kPair, 1, kFp8>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
                             else
-                                issue_k_block<kPair, 2>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
+                                issue_k_block<kPair, 2, kFp8>(d_tmem, a_lo, b_lo, desc_hi, b_chunk_step, p.chunk_n, idesc, kb == 0);
                             // the stage is free (in both CTAs) once these MMAs retire
                             if constexpr (kPair) umma_commit_pair(bar_empty + 8 * st, 3);
                             else umma_commit(bar_empty + 8 * st);
@@ -513,6 +551,9 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                             w2f[(((j >> 1) * kMaxHeads + h) << 1) + (j & 1)] = __ldg(w2g + i);
                         }
                         for (int i = etid; i < p.n_hidden; i += kEpiWarps * 32) b1s[i] = __ldg(b1g + i);
+                        if constexpr (kFp8)
+                            for (int i = etid; i < p.n_hidden; i += kEpiWarps * 32)
+                                w1s[i] = __ldg(p.w1_scale + static_cast<int64_t>(layer) * p.n_hidden + i);
                         __syncwarp();
                         if (lane == 0) mbar_arrive(bar_epi);
                         if (!mbar_wait(bar_epi, epi_it & 1u, abort_flag)) { ok = false; break; }
@@ -524,6 +565,11 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                 uint64_t acc[kMaxHeads];
 #pragma unroll
                 for (int h = 0; h < kMaxHeads; ++h) { s[h] = 0.0f; acc[h] = 0ull; }
+                float sx = 1.0f;                               // 8-bit inputs: this token's scale
+                if constexpr (kFp8) {
+                    const int64_t t_row = static_cast<int64_t>(m_tile) * kTileM + row;
+                    if (p.x_scale != nullptr && t_row < p.n_tokens) sx = __ldg(p.x_scale + static_cast<int64_t>(l_rel) * p.n_tokens + t_row);
+                }
                 for (int g = 0; g < p.n_groups; ++g, ++acc_it) {
                     const uint32_t buf = acc_it % p.acc_bufs;
                     const uint32_t use = acc_it / p.acc_bufs;
@@ -541,19 +587,25 @@ score_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__
                             tmem_wait_ld();
                             reg_fence16(ra);
                             tmem_ld_x16(t_row + col0 + c + 16, rb);
-                            mlp_columns<16>(ra, j0 + c, b1s, w2p, acc);
+                            if constexpr (kFp8) mlp_columns_scaled<16>(ra, j0 + c, b1s, w1s, f2_pack(sx, sx), w2p, acc);
+                            else mlp_columns<16>(ra, j0 + c, b1s, w2p, acc);
                             tmem_wait_ld();
                             reg_fence16(rb);
                             if (c + 32 < half_w) tmem_ld_x16(t_row + col0 + c + 32, ra);
-                            mlp_columns<16>(rb, j0 + c + 16, b1s, w2p, acc);
+                            if constexpr (kFp8) mlp_columns_scaled<16>(rb, j0 + c + 16, b1s, w1s, f2_pack(sx, sx), w2p, acc);
+                            else mlp_columns<16>(rb, j0 + c + 16, b1s, w2p, acc);
                         }
                     } else {
                         uint32_t r[16];
                         tmem_ld_x16(t_row, r);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int h = 0; h < kMaxHeads; ++h)
-                            s[h] = __uint_as_float(r[h]) + __ldg(p.b1 + layer * p.w_rows + h);
+                        for (int h = 0; h < kMaxHeads; ++h) {
+                            if constexpr (kFp8)
+                                s[h] = fmaf(__uint_as_float(r[h]), sx * __ldg(p.w1_scale + layer * p.w_rows + h), __ldg(p.b1 + layer * p.w_rows + h));
+                            else
+                                s[h] = __uint_as_float(r[h]) + __ldg(p.b1 + layer * p.w_rows + h);
+                        }
                     }
                     // this warp is done reading the accumulator buffer
                     tc_fence_before_sync();

@@ -128,3 +128,14 @@ def from_bits(a: np.ndarray, device="cpu") -> torch.Tensor:
     """Inverse of :func:`bits`."""
     assert a.dtype == np.uint16
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
+
+
+def quantize_e4m3(x: torch.Tensor, per_row: bool = True):
+    """Input preparation for the 8-bit paths: x [rows, cols] (any float dtype) -> (bytes uint8 [rows, cols] of
+    E4M3 values, scale fp32 [rows]) with x ~ scale[:, None] * E4M3(bytes); the scale maps each row's largest
+    magnitude to 448, the format's largest value.  torch's own conversion does the rounding."""
+    xf = x.to(torch.float32)
+    amax = xf.abs().amax(dim=1) if per_row else xf.abs().max().expand(xf.shape[0])
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax)).to(torch.float32).contiguous()
+    q = (xf / scale[:, None]).to(torch.float8_e4m3fn)
+    return q.view(torch.uint8).contiguous(), scale

@@ -1,0 +1,107 @@
+"""The 8-bit (E4M3) scoring path against the oracle: the first layer on the tensor cores' 8-bit path
+with per-token and per-row scales, then GELU / second layer / mask / compaction as for bf16.
+Tolerance as everywhere: 2e-2 absolute on the scores (E4M3 products are exact in fp32; the
+accumulation order differs), masks equal outside that band, compaction bit-exact given the scores."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_07891_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2601_07891_b200 import binding as b
+    b.load()
+    return b
+
+
+def _fp8_case(d_model, hidden, H, T, seed):
+    X = synth.hidden_states(T, d_model, seed)
+    X8, sx = synth.quantize_e4m3(X)
+    if hidden:
+        W1, b1, W2, b2 = synth.mlp_weights(d_model, hidden, H, seed + 1, "cpu", 0.3)
+    else:
+        W1, b1 = synth.linear_weights(d_model, H, seed + 1, "cpu", 0.3)
+        W2 = b2 = None
+    W18, sw = synth.quantize_e4m3(W1)
+    return X8, sx, W18, sw, b1, W2, b2
+
+
+def _oracle_scores(oracle, case, hidden):
+    X8, sx, W18, sw, b1, W2, b2 = case
+    if hidden:
+        return oracle.score_mlp_fp8(X8.numpy(), sx.numpy(), W18.numpy(), sw.numpy(), b1.numpy(), synth.bits(W2), b2.numpy())
+    return oracle.score_linear_fp8(X8.numpy(), sx.numpy(), W18.numpy(), sw.numpy(), b1.numpy())
+
+
+@pytest.mark.parametrize("d_model,hidden,T", [(256, 0, 1), (256, 0, 300), (1024, 0, 4097), (256, 64, 129), (512, 128, 1000),
+                                              (256, 256, 257), (256, 512, 520), (256, 640, 200), (4096, 512, 260), (5120, 640, 130),
+                                              (1024, 512, 20000)])
+def test_fp8_scores_match_oracle(binding, oracle, d_model, hidden, T):
+    H = 8
+    ctx = binding.Kvzap(d_model, hidden, H, 64, 1, max_tokens=T)
+    case = _fp8_case(d_model, hidden, H, T, seed=T + hidden)
+    X8, sx, W18, sw, b1, W2, b2 = case
+    binding.kvzap_set_weights_fp8(ctx.handle, 0, W18.cuda(), sw.cuda(), b1.cuda(), parity.dev(W2), parity.dev(b2))
+    scores = torch.empty(T, H, dtype=torch.float32, device="cuda")
+    binding.kvzap_score_fp8(ctx.handle, 0, X8.cuda(), sx.cuda(), scores)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    rows = np.arange(T) if T * max(hidden, 8) * d_model < 3e9 else np.unique(np.concatenate([[0, 127, 128, T - 1], np.random.default_rng(0).integers(0, T, 400)]))
+    sub = tuple(t[rows] if i in (0, 1) else t for i, t in enumerate(case))
+    want = _oracle_scores(oracle, sub, hidden)
+    got = scores.cpu().numpy()[rows]
+    assert np.isfinite(got).all()
+    assert np.abs(got - want).max() <= parity.SCORE_ATOL
+    # the bf16 calls refuse a layer that holds 8-bit weights
+    with pytest.raises(binding.KvzapError) as ei:
+        ctx.score(0, torch.zeros(1, d_model, dtype=torch.bfloat16, device="cuda"))
+    assert ei.value.status == 6
+    ctx.close()
+
+
+@pytest.mark.parametrize("seq_lens,hidden", [([700], 0), ([37, 64, 5, 0, 300, 900], 128), ([33000], 256)])
+def test_fp8_fused_prefill_matches_oracle(binding, oracle, seq_lens, hidden):
+    d_model, H, D, tau, w = 512, 8, 64, 0.25, 32
+    T, B = int(sum(seq_lens)), len(seq_lens)
+    ctx = binding.Kvzap(d_model, hidden, H, D, 1, T, max_seqs=B)
+    case = _fp8_case(d_model, hidden, H, T, seed=5 + hidden)
+    X8, sx, W18, sw, b1, W2, b2 = case
+    binding.kvzap_set_weights_fp8(ctx.handle, 0, W18.cuda(), sw.cuda(), b1.cuda(), parity.dev(W2), parity.dev(b2))
+    K, V = synth.keys_values(H, T, D, seed=9)
+    cu = synth.cu_seqlens(seq_lens)
+    cu_dev = torch.from_numpy(cu).cuda() if B > 1 else None
+    cu_arg = cu if B > 1 else None
+    K_out, V_out = parity.poison_like(K).cuda(), parity.poison_like(V).cuda()
+    lengths = torch.full((B, H), -1, dtype=torch.int32, device="cuda")
+    scores = torch.empty(T, H, dtype=torch.float32, device="cuda")
+    binding.kvzap_prefill_fused_fp8(ctx.handle, 0, X8.cuda(), sx.cuda(), parity.dev(K), parity.dev(V), cu_dev, B, tau, w,
+                                    K_out, V_out, lengths, scores)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    want = _oracle_scores(oracle, case, hidden)
+    s = scores.cpu().numpy()
+    assert np.abs(s - want).max() <= parity.SCORE_ATOL
+    parity.check_mask_band(oracle, s, want, tau, w, cu_arg)
+    parity.check_compaction(oracle, K, V, s, tau, w, cu_arg, K_out.cpu(), V_out.cpu(), lengths)
+    ctx.close()
+
+
+def test_fp8_needs_d_model_multiple_of_128_and_its_own_weights(binding):
+    ctx = binding.Kvzap(192, 0, 8, 64, 1, max_tokens=64)
+    W = torch.zeros(8, 192, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.KvzapError) as ei:
+        binding.kvzap_set_weights_fp8(ctx.handle, 0, W, None)
+    assert ei.value.status == 2
+    ctx.close()
+    ctx = binding.Kvzap(256, 0, 8, 64, 1, max_tokens=64)
+    ctx.set_weights(0, *[t.cuda() for t in synth.linear_weights(256, 8, 1)])
+    with pytest.raises(binding.KvzapError) as ei:
+        binding.kvzap_score_fp8(ctx.handle, 0, torch.zeros(4, 256, dtype=torch.uint8, device="cuda"), None,
+                                torch.zeros(4, 8, device="cuda"))
+    assert ei.value.status == 6
+    ctx.close()
