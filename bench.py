@@ -232,6 +232,9 @@ def run_prefill(args, wl, env, sub=False):
     n_tokens = B * T
     H, D, P = wl.n_kv_heads, wl.head_dim, wl.page_tokens
     proj = args.kv_layout == "proj"
+    fp8 = args.fp8 and not sub
+    if fp8 and (wl.page_tokens or proj):
+        raise SystemExit("--fp8 goes with the dense-ragged prefill workloads in the [H,T,D] layout")
     ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=dev.index, trusted_producers=True)
     cu = torch.from_numpy(synth.cu_seqlens([T] * B)).to(dev) if B > 1 else None
 
@@ -246,15 +249,27 @@ def run_prefill(args, wl, env, sub=False):
     max_pages = (T // P + 2) if P else 0
     pool_pages = (H * B * (T // P + 2)) // 2 if P else 0       # room for half of all rows per layer set
     for l in range(L):
-        ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
+        wts = synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index)
+        if fp8:
+            W18, sw = synth.quantize_e4m3(wts[0])
+            binding.kvzap_set_weights_fp8(ctx.handle, l, W18, sw, wts[1], *(wts[2:] if len(wts) == 4 else (None, None)))
+        else:
+            ctx.set_weights(l, *wts)
+    Xscales = []
     for l in range(max(L, n_sets)):
         lens.append(torch.zeros(B, H, dtype=torch.int32, device=dev))
         if l >= n_sets:
-            for lst in (Xs, Ks, Vs, Kos, Vos, scs, tabs, used):
+            for lst in (Xs, Ks, Vs, Kos, Vos, scs, tabs, used, Xscales):
                 lst.append(lst[l % n_sets])
             continue
         seed = 1000 * args.workload_index + l + 100000 * rank
-        Xs.append(synth.hidden_states(n_tokens, wl.d_model, seed, dev, wl.token_scale_sigma))
+        X = synth.hidden_states(n_tokens, wl.d_model, seed, dev, wl.token_scale_sigma)
+        if fp8:
+            X, xs = synth.quantize_e4m3(X)
+            Xscales.append(xs)
+        else:
+            Xscales.append(None)
+        Xs.append(X)
         K, V = synth.keys_values(H, n_tokens, D, seed + 500, dev)
         if proj:
             # write-side pruning: the same draws, laid out as the K/V projection writes them, [T, H, D]
@@ -282,7 +297,10 @@ def run_prefill(args, wl, env, sub=False):
         for i in (range(n_bufs) if n_bufs > L else [l]):
             prep_paged = binding.prepare_prefill_write_paged if proj else binding.prepare_prefill_fused_paged
             prep_dense = binding.prepare_prefill_write if proj else binding.prepare_prefill_fused
-            if P:
+            if fp8:
+                calls[(l, i)] = binding.prepare_prefill_fused_fp8(ctx.handle, l, Xs[i], Xscales[i], Ks[i], Vs[i], cu, B, wl.tau,
+                                                                  wl.window, Kos[i], Vos[i], lens[i], scs[i])
+            elif P:
                 calls[(l, i)] = prep_paged(ctx.handle, l, Xs[i], Ks[i], Vs[i], cu, B, wl.tau,
                                            wl.window, Kos[i], Vos[i], P, 0, tabs[i], lens[i], used[i], scs[i])
             else:
@@ -333,7 +351,10 @@ def run_prefill(args, wl, env, sub=False):
     def score_only():
         for l in range(L):
             i = (turn[0] + l) % n_bufs
-            binding.kvzap_score(ctx.handle, l, Xs[i], scs[i])
+            if fp8:
+                binding.kvzap_score_fp8(ctx.handle, l, Xs[i], Xscales[i], scs[i])
+            else:
+                binding.kvzap_score(ctx.handle, l, Xs[i], scs[i])
         if n_bufs > L:
             turn[0] += L
     score_ms = _timed(score_only, n_rep, sync) / L
@@ -351,7 +372,15 @@ def run_prefill(args, wl, env, sub=False):
 
     peaks, peak_src = load_peaks()
     peak_kind, tensor_peak = pick_tensor_peak(peaks, clocks)
+    if fp8:
+        tensor_peak *= 2.0           # no 8-bit GEMM was measured on this machine: the bf16 figure times the nominal ratio (4.5 / 2.25 PFLOP/s)
+        peak_kind += " x 2 (nominal fp8 : bf16 ratio)"
     flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer = _roofline_times(wl, n_tokens, kept_rows, peaks, tensor_peak)
+    if fp8:
+        # an 8-bit hidden state is half the bytes (plus 4 bytes of scale per token)
+        score_bytes = n_tokens * wl.d_model + n_tokens * 4 + n_tokens * wl.n_kv_heads * 4
+        t_hbm_score = score_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_hbm_layer -= (n_tokens * wl.d_model - n_tokens * 4) / (peaks["hbm_gbs"] * 1e9)
     # Dominant kernel = the scoring kernel.  Its launch duration inside the timed region cannot be
     # separated from the compaction that runs beside it, so the layer period (step time / layers) is
     # used: an upper bound of the kernel's own duration.  `alone_ms` is the same kernel in a loop of
@@ -362,8 +391,8 @@ def run_prefill(args, wl, env, sub=False):
                     "unit": "TFLOP/s", "frac": achieved / tensor_peak,
                     "peak_kind": peak_kind + " cuBLAS bf16 figure, chosen from this run's clock record (burst: median SM "
                                              "clock within 5 % of max and no sw_power_cap sample)",
-                    "frac_of_burst": achieved / peaks["bf16_tflops"],
-                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                    "frac_of_burst": achieved / (peaks["bf16_tflops"] * (2.0 if fp8 else 1.0)),
+                    "frac_of_sustained": achieved / (peaks["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)),
                     "alone_achieved": flops / (score_ms * 1e-3) / 1e12}
         if not args.skip_live_peak and not sub:
             # the GPUs of the pool settle at different clocks under the power cap: the same loop on this one, now
@@ -397,10 +426,10 @@ def run_prefill(args, wl, env, sub=False):
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps,
             "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
-            "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
+            "vs_baseline": None, "dtype": "e4m3 x e4m3 -> f32 (first layer), bf16 K/V" if fp8 else "bf16", "data": "synthetic",
+            "config": config, "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
 
-    if rank == 0 and world == 1 and not args.skip_e2e and not proj and not sub:
+    if rank == 0 and world == 1 and not args.skip_e2e and not proj and not sub and not fp8:
         # End to end through the host-buffer entry point: one call per step takes every layer's inputs from
         # pinned host memory and leaves every layer's result there; the copies happen inside the call (layer
         # l + 1 is copied in while layer l is computed and copied out).  Host inputs rotate over two layer sets.
@@ -756,7 +785,7 @@ def run_ours(args, wl, with_configs):
         line = run_attention(args, wl, env)
     else:
         line = run_decode(args, wl, env) if wl.decode_steps > 0 else run_prefill(args, wl, env)
-    if rank == 0 and world == 1 and not args.skip_cpu and wl.decode_steps == 0:
+    if rank == 0 and world == 1 and not args.skip_cpu and wl.decode_steps == 0 and not args.fp8:
         # the oracle on the host cores, bounded sample
         n_sample = min(wl.batch * wl.seq_len, args.ref_tokens)
         v, dt, threads, n_l = oracle_sample(wl, n_sample, budget_s=12.0)
@@ -799,6 +828,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="run only the first N layers (small case for profiling)")
     ap.add_argument("--kv-layout", default="heads", choices=["heads", "proj"],
                     help="prefill workloads: K/V as [H,T,D] (default) or as the projection writes them, [T,H,D]")
+    ap.add_argument("--fp8", action="store_true",
+                    help="prefill workloads with dense-ragged output: hidden states and first-layer weights as E4M3 bytes with scales")
     ap.add_argument("--attention", action="store_true",
                     help="decode workload: time the attention over the pruned cache instead of the pruning step")
     ap.add_argument("--skip-live-peak", action="store_true",

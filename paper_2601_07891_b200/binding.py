@@ -422,6 +422,14 @@ def prepare_prune_prefill_paged(handle, K, V, scores, cu_seqlens, n_seqs, tau, w
                         (K, V, scores, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used))
 
 
+def prepare_prefill_fused_fp8(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_out, V_out, lengths,
+                              scores_out=None, stream=None) -> PreparedCall:
+    args = (handle, layer, _ptr(hidden_e4m3), _ptr(x_scale), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w,
+            _ptr(K_out), _ptr(V_out), _ptr(lengths), _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_prefill_fused_fp8", handle, args,
+                        (hidden_e4m3, x_scale, K, V, cu_seqlens, K_out, V_out, lengths, scores_out))
+
+
 def prepare_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
                                 first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None) -> PreparedCall:
     args = (handle, layer, _ptr(hidden), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w, _ptr(K_pool),
