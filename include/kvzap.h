@@ -414,6 +414,23 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
                                     const void *Q, int32_t n_q_heads, float scale, void *O, void *stream);
 
 /*
+ * The same attention over a cache whose rows are 8-bit (Related work, "Quantization": quantising the
+ * cache and pruning it compose; the pruning calls move rows as opaque bytes, so only this call has to know
+ * the format).  The context is created with head_dim = (D + 16) / 2, where D = 64 or 128 is the number of
+ * elements per head: a row of head_dim * 2 bytes is D E4M3 codes (1 sign, 4 exponent, 3 mantissa bits, bias 7,
+ * no infinities, S.1111.111 = NaN) followed by a 16-byte trailer, the row's fp32 scale and 12 unused bytes;
+ * the row stands for scale * code.  Whoever writes K_new / V_new (the projection's epilogue) quantises; every
+ * kvzap_* call that moves rows keeps codes and scale together.
+ *   Q, O [layer_end - layer_begin, n_seqs, n_q_heads, D] bf16 (device)
+ * logit_i = scale * k_scale_i * (q . K8_i), out = sum_i softmax(logit)_i * v_scale_i * V8_i, fp32 accumulation,
+ * codes widened exactly, the probabilities times v_scale_i rounded to bf16 for the second product.
+ * Everything else (grouping of query heads, empty lists, released slots, page and window multiples of 16,
+ * bounded waits) as kvzap_decode_attention.  A cache serves one of the two attention calls, not both.
+ */
+kvzap_status kvzap_decode_attention_fp8(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                        const void *Q, int32_t n_q_heads, float scale, void *O, void *stream);
+
+/*
  * A sequence has ended: all lists (seq, *, *) become empty and their pages go back to the cache's
  * allocator, which hands released pages out again (to any list) before it touches never-used pages
  * of the pool.  Until the slot is given a new prompt (kvzap_prefill_to_cache) decode steps leave its

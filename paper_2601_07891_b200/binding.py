@@ -73,6 +73,7 @@ SIGNATURES = {
     "kvzap_cache_destroy": (_i32, [_vp]),
     "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
     "kvzap_decode_attention": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
+    "kvzap_decode_attention_fp8": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
     "kvzap_cache_release_seq": (_i32, [_vp, _i32, _vp]),
     "kvzap_cache_lengths": (_i32, [_vp, _vp, _vp]),
     "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
@@ -466,6 +467,17 @@ def kvzap_decode_attention(handle, cache, layer_begin, layer_end, Q, scale, O, s
 def prepare_decode_attention(handle, cache, layer_begin, layer_end, Q, scale, O, stream=None) -> PreparedCall:
     args = (handle, cache, layer_begin, layer_end, _ptr(Q), Q.shape[2], scale, _ptr(O), _stream(stream))
     return PreparedCall("kvzap_decode_attention", handle, args, (Q, O))
+
+
+def kvzap_decode_attention_fp8(handle, cache, layer_begin, layer_end, Q, scale, O, stream=None):
+    """Cache rows are E4M3 codes + a 16-byte trailer (fp32 scale first); Q, O [layers, n_seqs, n_q_heads, D] bf16."""
+    _check(handle, load().kvzap_decode_attention_fp8(handle, cache, layer_begin, layer_end, _ptr(Q), Q.shape[2], scale,
+                                                     _ptr(O), _stream(stream)))
+
+
+def prepare_decode_attention_fp8(handle, cache, layer_begin, layer_end, Q, scale, O, stream=None) -> PreparedCall:
+    args = (handle, cache, layer_begin, layer_end, _ptr(Q), Q.shape[2], scale, _ptr(O), _stream(stream))
+    return PreparedCall("kvzap_decode_attention_fp8", handle, args, (Q, O))
 
 
 def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_new, tau, scores_out=None,

@@ -22,7 +22,20 @@
 //   O[16 x D]  += P[16 x 16] V
 // Rows of a partly filled tile that lie past the end are excluded from the softmax, and their V
 // rows are zeroed in shared memory first (stale pool memory may hold NaN bit patterns).
+//
+// 8-bit rows (Related work, "Quantization": pruning and quantisation of the cache compose).  A cache whose
+// rows are D E4M3 codes followed by a 16-byte trailer (the row's fp32 scale, then 12 unused bytes) is walked
+// by the same kernel with kFp8 = true: a tile is 16 whole rows brought in by one unswizzled TMA box per
+// K and V, the codes are widened to bf16 in registers (E4M3 -> f16 -> f32 -> bf16, every step exact) and the
+// row scales are applied outside the MMAs: logit = scale * ks_i * (q . K8_i), P is multiplied by vs_i before it
+// is rounded to bf16 for P V8 (the softmax denominator uses the unscaled P).  The MMA's summation index and the
+// output columns may be numbered freely as long as both operands agree, so each lane reads whole 16- or 32-byte
+// pieces of a row: for Q K^T lane (n, c) owns bytes [c D/4, (c+1) D/4) of K rows n and n + 8, k-step ks taking
+// four of them; for P V lane (n', c) owns bytes [n' D/8, (n'+1) D/8) of V rows 2c, 2c+1, 2c+8, 2c+9, output
+// tile i holding column n' D/8 + i.  With rows 144 (or 80) bytes apart these reads have no bank conflicts.
 #pragma once
+
+#include <cuda_fp16.h>
 
 #include "decode_kernels.cuh"
 #include "ptx.cuh"
@@ -49,20 +62,42 @@ struct AttnParams {
     uint32_t *part_arrive;      // n_parts > 1: [list] parts that have stored their triple; back to 0 after the launch
 };
 
-__host__ __device__ constexpr uint32_t attn_stage_bytes(int head_dim) { return 2u * (head_dim / 64) * kAttnHalfBytes; }
-__host__ __device__ constexpr uint32_t attn_smem_bytes(int head_dim)
+constexpr int kAttnTrailerBytes = 16;            // 8-bit rows: fp32 scale + 12 unused bytes behind the codes
+__host__ __device__ constexpr uint32_t attn_stage_bytes(int head_dim, bool fp8 = false)
 {
-    return kAttnWarps * kAttnStages * attn_stage_bytes(head_dim) + 1024u /* alignment */ + 256u /* barriers */;
+    return fp8 ? 2u * kAttnTileRows * (head_dim + kAttnTrailerBytes) : 2u * (head_dim / 64) * kAttnHalfBytes;
+}
+__host__ __device__ constexpr uint32_t attn_smem_bytes(int head_dim, bool fp8 = false)
+{
+    return kAttnWarps * kAttnStages * attn_stage_bytes(head_dim, fp8) + 1024u /* alignment */ + 256u /* barriers */;
 }
 
-template <int kD>
+// four E4M3 codes (a 32-bit word, lowest byte first) -> two packed bf16 pairs; every step is exact
+__device__ __forceinline__ uint32_t f16x2_to_bf16x2(uint32_t h2)
+{
+    const __half2 h = *reinterpret_cast<const __half2 *>(&h2);
+    const float2 f = __half22float2(h);
+    return pack_bf16x2(f.x, f.y);
+}
+__device__ __forceinline__ void e4m3x4_to_bf16(uint32_t w, uint32_t &lo, uint32_t &hi)
+{
+    uint32_t h0, h1;
+    asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(h0), "=r"(h1) : "r"(w));
+    lo = f16x2_to_bf16x2(h0);
+    hi = f16x2_to_bf16x2(h1);
+}
+
+template <int kD, bool kFp8>
 __global__ void __launch_bounds__(kAttnThreads)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_constant__ CUtensorMap tmap_vpool,
                    const __grid_constant__ CUtensorMap tmap_kring, const __grid_constant__ CUtensorMap tmap_vring,
                    const AttnParams p)
 {
     constexpr int kHalves = kD / 64;
-    constexpr uint32_t kStageBytes = attn_stage_bytes(kD);
+    constexpr uint32_t kStageBytes = attn_stage_bytes(kD, kFp8);
+    constexpr int kRowBytes8 = kD + kAttnTrailerBytes;              // 8-bit rows
+    constexpr uint32_t kTileBytes8 = kAttnTileRows * kRowBytes8;
     constexpr int kNTiles = kD / 8;              // 8-column tiles of the output
     extern __shared__ uint8_t attn_smem_raw[];
     const uint32_t raw_addr = smem_u32(attn_smem_raw);
@@ -114,8 +149,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         for (int ks = 0; ks < kD / 16; ++ks) {
             qa[ks][0] = qa[ks][1] = 0u;
             if (g < p.group) {
-                qa[ks][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + qc));
-                qa[ks][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + qc));
+                if constexpr (kFp8) {      // summation index renumbered: this lane's k-step ks covers columns c D/4 + 4 ks ..+3
+                    qa[ks][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + (lane & 3) * (kD / 4) + ks * 4));
+                    qa[ks][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + (lane & 3) * (kD / 4) + ks * 4 + 2));
+                } else {
+                    qa[ks][0] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + qc));
+                    qa[ks][1] = __ldg(reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + qc));
+                }
             }
         }
     }
@@ -142,10 +182,15 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         const uint32_t bar = my_bars + 8 * stage;
         const bool prefix = t < n_pt;
         mbar_arrive_expect_tx(bar, kStageBytes);
+        if constexpr (kFp8) {
+            tma_load_2d(dst, prefix ? &tmap_kpool : &tmap_kring, bar, 0, row, policy);
+            tma_load_2d(dst + kTileBytes8, prefix ? &tmap_vpool : &tmap_vring, bar, 0, row, policy);
+        } else {
 #pragma unroll
-        for (int hf = 0; hf < kHalves; ++hf) {
-            tma_load_2d(dst + hf * kAttnHalfBytes, prefix ? &tmap_kpool : &tmap_kring, bar, hf * 64, row, policy);
-            tma_load_2d(dst + (kHalves + hf) * kAttnHalfBytes, prefix ? &tmap_vpool : &tmap_vring, bar, hf * 64, row, policy);
+            for (int hf = 0; hf < kHalves; ++hf) {
+                tma_load_2d(dst + hf * kAttnHalfBytes, prefix ? &tmap_kpool : &tmap_kring, bar, hf * 64, row, policy);
+                tma_load_2d(dst + (kHalves + hf) * kAttnHalfBytes, prefix ? &tmap_vpool : &tmap_vring, bar, hf * 64, row, policy);
+            }
         }
     };
 
@@ -166,15 +211,21 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
             break;
         }
         const uint32_t sK = my_stages + stage * kStageBytes;
-        const uint32_t sV = sK + kHalves * kAttnHalfBytes;
+        const uint32_t sV = sK + (kFp8 ? kTileBytes8 : kHalves * kAttnHalfBytes);
         const int valid = t < n_pt ? n_prefix - t * kAttnTileRows : n_ring - (t - n_pt) * kAttnTileRows;   // >= 1
         if (valid < kAttnTileRows) {
-            // zero the V rows past the end of the list
-            const int n_units = (kAttnTileRows - valid) * kHalves * 8;
-            for (int i = lane; i < n_units; i += 32) {
-                const int r = valid + i / (kHalves * 8), rem = i % (kHalves * 8);
-                *reinterpret_cast<uint4 *>(smem + (sV - smem_base) + (rem >> 3) * kAttnHalfBytes + r * 128 + ((rem & 7) << 4)) =
-                    make_uint4(0u, 0u, 0u, 0u);
+            // zero the V rows past the end of the list (8-bit rows: codes and scale)
+            if constexpr (kFp8) {
+                const int n_units = (kAttnTileRows - valid) * (kRowBytes8 / 16);
+                for (int i = lane; i < n_units; i += 32)
+                    *reinterpret_cast<uint4 *>(smem + (sV - smem_base) + valid * kRowBytes8 + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+                const int n_units = (kAttnTileRows - valid) * kHalves * 8;
+                for (int i = lane; i < n_units; i += 32) {
+                    const int r = valid + i / (kHalves * 8), rem = i % (kHalves * 8);
+                    *reinterpret_cast<uint4 *>(smem + (sV - smem_base) + (rem >> 3) * kAttnHalfBytes + r * 128 + ((rem & 7) << 4)) =
+                        make_uint4(0u, 0u, 0u, 0u);
+                }
             }
             fence_proxy_async_smem();
             __syncwarp();
@@ -182,7 +233,32 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
 
         // ---- S = Q K^T: two 8-row column tiles
         float s0[4] = {0.0f, 0.0f, 0.0f, 0.0f}, s1[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        {
+        if constexpr (kFp8) {
+            // rows n = lane / 4 and n + 8 of the tile, this lane's D/4 bytes of each
+            const uint8_t *kt = smem + (sK - smem_base);
+            const uint32_t *r0 = reinterpret_cast<const uint32_t *>(kt + g * kRowBytes8 + (lane & 3) * (kD / 4));
+            const uint32_t *r1 = reinterpret_cast<const uint32_t *>(kt + (g + 8) * kRowBytes8 + (lane & 3) * (kD / 4));
+            uint32_t w0[kD / 16], w1[kD / 16];
+#pragma unroll
+            for (int i = 0; i < kD / 64; ++i) {
+                const uint4 a = reinterpret_cast<const uint4 *>(r0)[i], b = reinterpret_cast<const uint4 *>(r1)[i];
+                w0[4 * i] = a.x; w0[4 * i + 1] = a.y; w0[4 * i + 2] = a.z; w0[4 * i + 3] = a.w;
+                w1[4 * i] = b.x; w1[4 * i + 1] = b.y; w1[4 * i + 2] = b.z; w1[4 * i + 3] = b.w;
+            }
+#pragma unroll
+            for (int ks = 0; ks < kD / 16; ++ks) {
+                uint32_t k0, k1, k2, k3;
+                e4m3x4_to_bf16(w0[ks], k0, k1);
+                e4m3x4_to_bf16(w1[ks], k2, k3);
+                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, k0, k1);
+                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, k2, k3);
+            }
+            // the K rows' scales: this lane holds columns (rows of the tile) qc, qc + 1 of both column tiles
+            s0[0] *= *reinterpret_cast<const float *>(kt + qc * kRowBytes8 + kD);
+            s0[1] *= *reinterpret_cast<const float *>(kt + (qc + 1) * kRowBytes8 + kD);
+            s1[0] *= *reinterpret_cast<const float *>(kt + (8 + qc) * kRowBytes8 + kD);
+            s1[1] *= *reinterpret_cast<const float *>(kt + (9 + qc) * kRowBytes8 + kD);
+        } else {
             const int mi = lane >> 3, r8 = lane & 7;
             const int krow = (mi >> 1) * 8 + r8;
 #pragma unroll
@@ -215,10 +291,50 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         m_run = m_new;
 #pragma unroll
         for (int i = 0; i < kNTiles; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
-        const uint32_t pa0 = pack_bf16x2(p00, p01), pa2 = pack_bf16x2(p10, p11);
+        uint32_t pa0, pa2;
+        if constexpr (kFp8) {
+            const uint8_t *vt = smem + (sV - smem_base);
+            pa0 = pack_bf16x2(p00 * *reinterpret_cast<const float *>(vt + qc * kRowBytes8 + kD),
+                              p01 * *reinterpret_cast<const float *>(vt + (qc + 1) * kRowBytes8 + kD));
+            pa2 = pack_bf16x2(p10 * *reinterpret_cast<const float *>(vt + (8 + qc) * kRowBytes8 + kD),
+                              p11 * *reinterpret_cast<const float *>(vt + (9 + qc) * kRowBytes8 + kD));
+        } else {
+            pa0 = pack_bf16x2(p00, p01);
+            pa2 = pack_bf16x2(p10, p11);
+        }
 
         // ---- O += P V: two 8-column output tiles per ldmatrix
-        {
+        if constexpr (kFp8) {
+            // V rows 2c, 2c+1 (k = 2c, 2c+1) and 2c+8, 2c+9 of the tile, this lane's D/8 bytes of each;
+            // output tile i takes byte i of each row
+            const uint8_t *vt = smem + (sV - smem_base) + g * (kD / 8);
+            uint32_t ra[kD / 32], rb[kD / 32], rc[kD / 32], rd[kD / 32];
+            if constexpr (kD == 128) {
+                const uint4 a = *reinterpret_cast<const uint4 *>(vt + qc * kRowBytes8);
+                const uint4 b = *reinterpret_cast<const uint4 *>(vt + (qc + 1) * kRowBytes8);
+                const uint4 cc = *reinterpret_cast<const uint4 *>(vt + (qc + 8) * kRowBytes8);
+                const uint4 d = *reinterpret_cast<const uint4 *>(vt + (qc + 9) * kRowBytes8);
+                ra[0] = a.x; ra[1] = a.y; ra[2] = a.z; ra[3] = a.w;
+                rb[0] = b.x; rb[1] = b.y; rb[2] = b.z; rb[3] = b.w;
+                rc[0] = cc.x; rc[1] = cc.y; rc[2] = cc.z; rc[3] = cc.w;
+                rd[0] = d.x; rd[1] = d.y; rd[2] = d.z; rd[3] = d.w;
+            } else {
+                const uint2 a = *reinterpret_cast<const uint2 *>(vt + qc * kRowBytes8);
+                const uint2 b = *reinterpret_cast<const uint2 *>(vt + (qc + 1) * kRowBytes8);
+                const uint2 cc = *reinterpret_cast<const uint2 *>(vt + (qc + 8) * kRowBytes8);
+                const uint2 d = *reinterpret_cast<const uint2 *>(vt + (qc + 9) * kRowBytes8);
+                ra[0] = a.x; ra[1] = a.y; rb[0] = b.x; rb[1] = b.y;
+                rc[0] = cc.x; rc[1] = cc.y; rd[0] = d.x; rd[1] = d.y;
+            }
+#pragma unroll
+            for (int i = 0; i < kNTiles; ++i) {
+                const uint32_t sel = (i & 3) | ((4 + (i & 3)) << 4);
+                const uint32_t quad = __byte_perm(__byte_perm(ra[i >> 2], rb[i >> 2], sel), __byte_perm(rc[i >> 2], rd[i >> 2], sel), 0x5410);
+                uint32_t v0, v1;
+                e4m3x4_to_bf16(quad, v0, v1);
+                mma_bf16_16816(o[i], pa0, 0u, pa2, 0u, v0, v1);
+            }
+        } else {
             const int mi = lane >> 3, r8 = lane & 7;
             const int krow = (mi & 1) * 8 + r8;
 #pragma unroll
@@ -257,8 +373,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         if ((lane & 3) == 0) { mine[g] = m_run; mine[8 + g] = l_run; }
 #pragma unroll
         for (int i = 0; i < kNTiles; ++i) {
-            mine[16 + g * kD + i * 8 + qc] = o[i][0];
-            mine[16 + g * kD + i * 8 + qc + 1] = o[i][1];
+            if constexpr (kFp8) {           // output tile i, column j is element j D/8 + i
+                mine[16 + g * kD + qc * (kD / 8) + i] = o[i][0];
+                mine[16 + g * kD + (qc + 1) * (kD / 8) + i] = o[i][1];
+            } else {
+                mine[16 + g * kD + i * 8 + qc] = o[i][0];
+                mine[16 + g * kD + i * 8 + qc + 1] = o[i][1];
+            }
         }
     }
     __syncthreads();

@@ -239,6 +239,24 @@ static kvzap_status make_tmap8(kvzap_ctx *ctx, CUtensorMap *map, const void *bas
     return KVZAP_OK;
 }
 
+// Tensor map over `rows` rows of `row_bytes` bytes each; box = box_rows whole rows, no swizzle (the attention
+// kernel's tiles of 8-bit rows with their trailers).  row_bytes is a multiple of 16, at most 256.
+static kvzap_status make_tmap_rows(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows, uint32_t row_bytes,
+                                   uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {row_bytes, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {row_bytes, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(ctx, KVZAP_ERR_CUDA, "cuTensorMapEncodeTiled (rows) failed with code %d (rows=%llu row_bytes=%u box_rows=%u)",
+                    static_cast<int>(r), static_cast<unsigned long long>(rows), row_bytes, box_rows);
+    return KVZAP_OK;
+}
+
 // Tensor map over the context's copy of the first-layer weights, stored K block by K block:
 // [k_blocks][rows_total][64] bf16, so that the `box_rows` x 64 tile a CTA stages per K step is one
 // contiguous piece of memory (a decode step reads every weight byte from HBM exactly once; contiguous
@@ -2146,10 +2164,10 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
     return KVZAP_OK;
 }
 
-kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
-                                    const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_)
+static kvzap_status attention_impl(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                   const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_, bool fp8)
 {
-    NvtxRange nvtx_range("kvzap_decode_attention");
+    NvtxRange nvtx_range(fp8 ? "kvzap_decode_attention_fp8" : "kvzap_decode_attention");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
     begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -2164,11 +2182,17 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
                     kAttnMaxGroup);
     if (!(scale == scale) || scale < 0.0f) return fail(ctx, KVZAP_ERR_INVALID_ARG, "attention: scale must be >= 0");
     DeviceGuard guard(c.device);
+    // elements per row as the attention sees them: head_dim bf16 values, or head_dim * 2 - 16 E4M3 codes
+    const int d_attn = fp8 ? c.head_dim * 2 - kAttnTrailerBytes : c.head_dim;
+    if (d_attn != 64 && d_attn != 128)
+        return fail(ctx, KVZAP_ERR_UNSUPPORTED,
+                    fp8 ? "8-bit attention needs head_dim 40 or 72 (64 or 128 codes and a 16-byte trailer per row)"
+                        : "attention needs head_dim 64 or 128");
     if (cache->attn_state == 0) {
         // tiles of 16 rows: pages and the window must be whole numbers of them; rows of 64 or 128 elements
         const int64_t pool_rows = v.n_pages_pool * v.page_tokens;
         const int64_t ring_rows = cache->n_lists * (v.window > 0 ? v.window : 1);
-        const bool ok = (c.head_dim == 64 || c.head_dim == 128) && v.page_tokens % kAttnTileRows == 0 &&
+        const bool ok = (d_attn == 64 || d_attn == 128) && v.page_tokens % kAttnTileRows == 0 &&
                         v.window % kAttnTileRows == 0 && pool_rows < (int64_t{1} << 31) && ring_rows < (int64_t{1} << 31) &&
                         pool_rows >= kAttnTileRows;
         cache->attn_state = -1;
@@ -2176,22 +2200,34 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
             const void *kring = v.window > 0 ? static_cast<const void *>(v.k_ring) : static_cast<const void *>(v.k_pool);
             const void *vring = v.window > 0 ? static_cast<const void *>(v.v_ring) : static_cast<const void *>(v.v_pool);
             const uint64_t rr = v.window > 0 ? static_cast<uint64_t>(ring_rows) : static_cast<uint64_t>(pool_rows);
-            if (make_tmap(ctx, &cache->tm_kpool, v.k_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
-                make_tmap(ctx, &cache->tm_vpool, v.v_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
-                make_tmap(ctx, &cache->tm_kring, kring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK &&
-                make_tmap(ctx, &cache->tm_vring, vring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK) {
-                cudaError_t e = c.head_dim == 128
-                    ? cudaFuncSetAttribute(decode_attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(attn_smem_bytes(128)))
-                    : cudaFuncSetAttribute(decode_attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(attn_smem_bytes(64)));
-                if (e == cudaSuccess) cache->attn_state = 1;
+            const uint32_t rb = static_cast<uint32_t>(c.head_dim) * 2;
+            const bool maps_ok = fp8
+                ? make_tmap_rows(ctx, &cache->tm_kpool, v.k_pool, static_cast<uint64_t>(pool_rows), rb, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap_rows(ctx, &cache->tm_vpool, v.v_pool, static_cast<uint64_t>(pool_rows), rb, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap_rows(ctx, &cache->tm_kring, kring, rr, rb, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap_rows(ctx, &cache->tm_vring, vring, rr, rb, kAttnTileRows) == KVZAP_OK
+                : make_tmap(ctx, &cache->tm_kpool, v.k_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap(ctx, &cache->tm_vpool, v.v_pool, static_cast<uint64_t>(pool_rows), c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap(ctx, &cache->tm_kring, kring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK &&
+                  make_tmap(ctx, &cache->tm_vring, vring, rr, c.head_dim, kAttnTileRows) == KVZAP_OK;
+            if (maps_ok) {
+                const int smem = static_cast<int>(attn_smem_bytes(d_attn, fp8));
+                cudaError_t e;
+                if (fp8)
+                    e = d_attn == 128 ? cudaFuncSetAttribute(decode_attn_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                                      : cudaFuncSetAttribute(decode_attn_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                else
+                    e = d_attn == 128 ? cudaFuncSetAttribute(decode_attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                                      : cudaFuncSetAttribute(decode_attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+                if (e == cudaSuccess) cache->attn_state = fp8 ? 2 : 1;
             }
         }
     }
-    if (cache->attn_state != 1)
+    if (cache->attn_state != (fp8 ? 2 : 1))
         return fail(ctx, KVZAP_ERR_UNSUPPORTED,
-                    "attention needs head_dim 64 or 128, page_tokens and window multiples of %d, fewer than 2^31 rows",
+                    fp8 ? "8-bit attention needs head_dim 40 or 72 (64 or 128 codes and a 16-byte trailer per row), page_tokens and "
+                          "window multiples of %d, fewer than 2^31 rows, and a cache not yet used by kvzap_decode_attention"
+                        : "attention needs head_dim 64 or 128, page_tokens and window multiples of %d, fewer than 2^31 rows",
                     kAttnTileRows);
     AttnParams p;
     memset(&p, 0, sizeof p);
@@ -2232,16 +2268,32 @@ kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     const int64_t n_ctas = n_lists_call * p.n_parts;
     {
         ProfScope prof(ctx, KVZAP_KERNEL_ATTENTION, stream);
-        if (c.head_dim == 128)
-            decode_attn_kernel<128><<<static_cast<unsigned>(n_ctas), kAttnThreads, attn_smem_bytes(128), stream>>>(
-                cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+        const unsigned grid = static_cast<unsigned>(n_ctas);
+        const uint32_t smem = attn_smem_bytes(d_attn, fp8);
+        if (fp8 && d_attn == 128)
+            decode_attn_kernel<128, true><<<grid, kAttnThreads, smem, stream>>>(cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+        else if (fp8)
+            decode_attn_kernel<64, true><<<grid, kAttnThreads, smem, stream>>>(cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+        else if (d_attn == 128)
+            decode_attn_kernel<128, false><<<grid, kAttnThreads, smem, stream>>>(cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
         else
-            decode_attn_kernel<64><<<static_cast<unsigned>(n_ctas), kAttnThreads, attn_smem_bytes(64), stream>>>(
-                cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
+            decode_attn_kernel<64, false><<<grid, kAttnThreads, smem, stream>>>(cache->tm_kpool, cache->tm_vpool, cache->tm_kring, cache->tm_vring, p);
         KVZAP_CUDA(ctx, cudaGetLastError());
     }
     ctx->launches += 1;
     return KVZAP_OK;
+}
+
+kvzap_status kvzap_decode_attention(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                    const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_)
+{
+    return attention_impl(ctx, cache, layer_begin, layer_end, Q, n_q_heads, scale, O, stream_, false);
+}
+
+kvzap_status kvzap_decode_attention_fp8(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                        const void *Q, int32_t n_q_heads, float scale, void *O, void *stream_)
+{
+    return attention_impl(ctx, cache, layer_begin, layer_end, Q, n_q_heads, scale, O, stream_, true);
 }
 
 kvzap_status kvzap_cache_release_seq(kvzap_cache *cache, int32_t seq, void *stream_)

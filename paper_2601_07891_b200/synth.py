@@ -139,3 +139,24 @@ def quantize_e4m3(x: torch.Tensor, per_row: bool = True):
     scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax)).to(torch.float32).contiguous()
     q = (xf / scale[:, None]).to(torch.float8_e4m3fn)
     return q.view(torch.uint8).contiguous(), scale
+
+
+E4M3_ROW_TRAILER = 16
+
+
+def pack_rows_e4m3(x: torch.Tensor) -> torch.Tensor:
+    """Input preparation for the 8-bit cache: x [..., D] (any float dtype) -> bf16 tensor [..., (D + 16) / 2] whose
+    bytes are, per row, D E4M3 codes, the row's fp32 scale and 12 zero bytes (the row layout the 8-bit attention
+    call reads; the other calls move such rows as opaque bytes)."""
+    D = x.shape[-1]
+    codes, scale = quantize_e4m3(x.reshape(-1, D))
+    rows = torch.zeros(codes.shape[0], D + E4M3_ROW_TRAILER, dtype=torch.uint8, device=x.device)
+    rows[:, :D] = codes
+    rows[:, D:D + 4] = scale.view(torch.uint8).view(-1, 4)
+    return rows.view(torch.bfloat16).view(*x.shape[:-1], (D + E4M3_ROW_TRAILER) // 2)
+
+
+def unpack_rows_e4m3(bits: np.ndarray, D: int):
+    """Rows as uint16 words [n, (D + 16) / 2] (a cache export, say) -> (codes uint8 [n, D], scale fp32 [n])."""
+    raw = np.ascontiguousarray(bits).view(np.uint8).reshape(-1, D + E4M3_ROW_TRAILER)
+    return np.ascontiguousarray(raw[:, :D]), np.ascontiguousarray(raw[:, D:D + 4]).view(np.float32).reshape(-1)
