@@ -637,6 +637,10 @@ def run_attention(args, wl, env):
     B, H, D, w, P = wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     L = args.layers if args.layers > 0 else 4
     G = 4                                             # 32 query heads over 8 KV heads
+    fp8 = bool(getattr(args, "fp8", False))           # rows of D E4M3 codes + a 16-byte trailer (fp32 scale first)
+    Dq = D                                            # elements per head, as Q and O have them
+    if fp8:
+        D = (Dq + synth.E4M3_ROW_TRAILER) // 2        # row width in bf16 units, as the context moves rows
     ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index, trusted_producers=True)
     for l in range(L):
         ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
@@ -651,14 +655,26 @@ def run_attention(args, wl, env):
     first = np.concatenate([[0], np.cumsum(pages_of)[:-1]]).astype(np.int64)
     n_pool = int(pages_of.sum())
     max_pages = int(pages_of.max())
-    K_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
-    V_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
+    if fp8:
+        # random codes (top exponent bits cleared: magnitudes below 2, no NaN code) and a scale of 1/2 per row
+        def rows8():
+            t = torch.randint(0, 256, (n_pool * P, 2 * D), dtype=torch.uint8, device=dev)
+            t[:, :Dq] &= 0xBF
+            t[:, Dq:] = 0
+            t[:, Dq + 3] = 0x3F                       # little-endian fp32 0.5
+            return t.view(torch.bfloat16).view(n_pool, P, D)
+        K_pool, V_pool = rows8(), rows8()
+    else:
+        K_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
+        V_pool = torch.empty(n_pool, P, D, dtype=torch.bfloat16, device=dev).normal_()
     table = torch.from_numpy((first[:, None] + np.arange(max_pages)[None, :]).astype(np.int32)).to(dev)
     cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
     # imported page tables are private to each list (contiguous runs); growth pages come from each run's tail
     binding.kvzap_cache_import(ctx.handle, cache, torch.from_numpy(prefix).to(dev), table, n_pool)
     Xd = synth.hidden_states(L * B, wl.d_model, 1, dev).view(L, B, wl.d_model)
-    Kn, Vn = synth.keys_values(L * B, H, D, 2, dev)
+    Kn, Vn = synth.keys_values(L * B, H, Dq, 2, dev)
+    if fp8:
+        Kn, Vn = synth.pack_rows_e4m3(Kn), synth.pack_rows_e4m3(Vn)
     for _ in range(w + 3):            # fill every window; tau = +inf keeps the prefixes as imported
         binding.kvzap_decode_step(ctx.handle, cache, 0, L, Xd, Kn.view(L, B, H, D), Vn.view(L, B, H, D), float("inf"), None)
     lengths = torch.zeros(B, L, H, dtype=torch.int32, device=dev)
@@ -667,9 +683,10 @@ def run_attention(args, wl, env):
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set while the cache was filled")
     rows = float(lengths.sum().item())
-    Qs = [synth.hidden_states(L * B * H * G, D, 50 + i, dev).view(L, B, H * G, D) for i in range(3)]
+    Qs = [synth.hidden_states(L * B * H * G, Dq, 50 + i, dev).view(L, B, H * G, Dq) for i in range(3)]
     Os = [torch.empty_like(q) for q in Qs]
-    calls = [binding.prepare_decode_attention(ctx.handle, cache, 0, L, Qs[i], 1.0 / D ** 0.5, Os[i]) for i in range(3)]
+    prepare = binding.prepare_decode_attention_fp8 if fp8 else binding.prepare_decode_attention
+    calls = [prepare(ctx.handle, cache, 0, L, Qs[i], 1.0 / Dq ** 0.5, Os[i]) for i in range(3)]
     n_warm, steps = max(args.warmup, 3), min(args.steps, 30)
     for i in range(n_warm):
         calls[i % 3]()
@@ -689,12 +706,14 @@ def run_attention(args, wl, env):
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during the timed region")
     peaks, peak_src = load_peaks()
-    alg_bytes = rows * 2 * D * 2 + 2 * L * B * H * G * D * 2        # every K and V row once; Q read, O written
+    alg_bytes = rows * 2 * D * 2 + 2 * L * B * H * G * Dq * 2       # every K and V row once; Q read, O written
     achieved = alg_bytes / (ms * 1e-3) / 1e9
     line = {"metric": "decode attention over the pruned cache, sequences/sec per layer", "value": world * B / (ms * 1e-3 / L),
             "unit": "sequences/s/layer", "n_gpus": world, "steps": steps, "warmup": n_warm, "ms_per_step": ms,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name + " / attention", "n_kv_heads": H, "n_q_heads": H * G, "head_dim": D,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "e4m3 rows (fp32 scale per row), bf16 queries, fp32 accumulation" if fp8 else "bf16", "data": "synthetic",
+            "config": {"workload": wl.name + " / attention" + (" / fp8 rows" if fp8 else ""), "n_kv_heads": H, "n_q_heads": H * G,
+                       "head_dim": Dq, "row_bytes": 2 * D,
                        "n_layers": L, "batch": B, "window": w, "page_tokens": P,
                        "sequence_len": [wl.prefix_min, wl.prefix_max], "kept_fraction": [0.15, 0.35],
                        "rows_per_list_mean": rows / n_lists,
@@ -702,7 +721,7 @@ def run_attention(args, wl, env):
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "gpu_launches": int(ctx.launch_count() - launches0),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": alg_bytes * NCU_ATTENTION_TRAFFIC_RATIO,
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None if fp8 else alg_bytes * NCU_ATTENTION_TRAFFIC_RATIO,
                          "kernel": "decode_attn_kernel", "peak_source": peak_src, "kernel_ms": ms,
                          "algorithmic_bytes_per_step": alg_bytes}}
     binding.kvzap_cache_destroy(cache)

@@ -25,14 +25,20 @@
 //
 // 8-bit rows (Related work, "Quantization": pruning and quantisation of the cache compose).  A cache whose
 // rows are D E4M3 codes followed by a 16-byte trailer (the row's fp32 scale, then 12 unused bytes) is walked
-// by the same kernel with kFp8 = true: a tile is 16 whole rows brought in by one unswizzled TMA box per
-// K and V, the codes are widened to bf16 in registers (E4M3 -> f16 -> f32 -> bf16, every step exact) and the
-// row scales are applied outside the MMAs: logit = scale * ks_i * (q . K8_i), P is multiplied by vs_i before it
-// is rounded to bf16 for P V8 (the softmax denominator uses the unscaled P).  The MMA's summation index and the
+// by the same kernel with kFp8 = true: a tile is 16 whole rows, contiguous in memory, brought in by one
+// unswizzled TMA box of full 128-byte lines per K and V, the codes are widened to f16 in registers (one exact conversion per pair) and the MMAs take f16
+// operands.  Everything that is not a code is kept inside f16's range by factors applied around the MMAs: a
+// query row is divided by the power of two of its largest element (exact; bf16's mantissa fits f16's) and the
+// K row scales join that factor on the logits, logit = scale * 2^e * ks_i * (q 2^-e . K8_i); P is multiplied by
+// vs_i / vref, vref the largest V scale met so far (the accumulator is rescaled when it grows, together with the
+// online softmax's own rescaling, and multiplied by vref at the end), so the second operand lies in [0, 1] and
+// is rounded to f16 (11 bits) where the bf16 path rounds P to 8.  The MMA's summation index and the
 // output columns may be numbered freely as long as both operands agree, so each lane reads whole 16- or 32-byte
 // pieces of a row: for Q K^T lane (n, c) owns bytes [c D/4, (c+1) D/4) of K rows n and n + 8, k-step ks taking
-// four of them; for P V lane (n', c) owns bytes [n' D/8, (n'+1) D/8) of V rows 2c, 2c+1, 2c+8, 2c+9, output
-// tile i holding column n' D/8 + i.  With rows 144 (or 80) bytes apart these reads have no bank conflicts.
+// four of them; the second product is computed transposed, O^T += V^T P^T (P, as the softmax leaves it, is the
+// B operand; no accumulator row is wasted on the padding of the query heads to 16), lane (n', c) owning bytes
+// [n' D/8, (n'+1) D/8) of V rows 2c, 2c+1, 2c+8, 2c+9.  With rows 144 (or 80) bytes apart these reads have no
+// bank conflicts.  Four CTAs fit an SM (128 registers, 56 KB of stages).
 #pragma once
 
 #include <cuda_fp16.h>
@@ -69,27 +75,20 @@ __host__ __device__ constexpr uint32_t attn_stage_bytes(int head_dim, bool fp8 =
 }
 __host__ __device__ constexpr uint32_t attn_smem_bytes(int head_dim, bool fp8 = false)
 {
-    return kAttnWarps * kAttnStages * attn_stage_bytes(head_dim, fp8) + 1024u /* alignment */ + 256u /* barriers */;
+    return kAttnWarps * kAttnStages * attn_stage_bytes(head_dim, fp8) + (fp8 ? 128u : 1024u) /* alignment */ + 256u /* barriers */;
 }
 
-// four E4M3 codes (a 32-bit word, lowest byte first) -> two packed bf16 pairs; every step is exact
-__device__ __forceinline__ uint32_t f16x2_to_bf16x2(uint32_t h2)
+// four E4M3 codes (a 32-bit word, lowest byte first) -> two packed f16 pairs (exact: f16 holds every E4M3 value)
+__device__ __forceinline__ void e4m3x4_to_f16(uint32_t w, uint32_t &lo, uint32_t &hi)
 {
-    const __half2 h = *reinterpret_cast<const __half2 *>(&h2);
-    const float2 f = __half22float2(h);
-    return pack_bf16x2(f.x, f.y);
-}
-__device__ __forceinline__ void e4m3x4_to_bf16(uint32_t w, uint32_t &lo, uint32_t &hi)
-{
-    uint32_t h0, h1;
     asm("{\n\t.reg .b16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.rn.f16x2.e4m3x2 %0, a;\n\tcvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
-        : "=r"(h0), "=r"(h1) : "r"(w));
-    lo = f16x2_to_bf16x2(h0);
-    hi = f16x2_to_bf16x2(h1);
+        : "=r"(lo), "=r"(hi) : "r"(w));
 }
+__device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xffff0000u); }
 
 template <int kD, bool kFp8>
-__global__ void __launch_bounds__(kAttnThreads)
+__global__ void __launch_bounds__(kAttnThreads, kFp8 ? 4 : 1)
 decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_constant__ CUtensorMap tmap_vpool,
                    const __grid_constant__ CUtensorMap tmap_kring, const __grid_constant__ CUtensorMap tmap_vring,
                    const AttnParams p)
@@ -98,10 +97,13 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
     constexpr uint32_t kStageBytes = attn_stage_bytes(kD, kFp8);
     constexpr int kRowBytes8 = kD + kAttnTrailerBytes;              // 8-bit rows
     constexpr uint32_t kTileBytes8 = kAttnTileRows * kRowBytes8;
-    constexpr int kNTiles = kD / 8;              // 8-column tiles of the output
+    // accumulator tiles: 16 x 8 pieces of O (rows = query heads, half of them unused) for bf16 rows,
+    // 16 x 8 pieces of O^T (rows = elements, columns = query heads) for 8-bit rows
+    constexpr int kNTiles = kFp8 ? kD / 16 : kD / 8;
+    constexpr uint32_t kAlign = kFp8 ? 128u : 1024u;            // swizzled tiles need 1024-byte alignment
     extern __shared__ uint8_t attn_smem_raw[];
     const uint32_t raw_addr = smem_u32(attn_smem_raw);
-    const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
+    const uint32_t pad = (kAlign - (raw_addr & (kAlign - 1u))) & (kAlign - 1u);
     uint8_t *smem = attn_smem_raw + pad;
     const uint32_t smem_base = raw_addr + pad;
     const uint32_t bars = smem_base + kAttnWarps * kAttnStages * kStageBytes;      // [warp][stage] mbarriers
@@ -160,10 +162,31 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         }
     }
 
+    float logit_scale = p.scale_log2e;     // 8-bit rows: times the power of two taken out of this lane's query row
+    if constexpr (kFp8) {
+        float qmax = 0.0f;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks)
+            qmax = fmaxf(fmaxf(qmax, fmaxf(fabsf(bf16_lo(qa[ks][0])), fabsf(bf16_hi(qa[ks][0])))),
+                         fmaxf(fabsf(bf16_lo(qa[ks][1])), fabsf(bf16_hi(qa[ks][1]))));
+        qmax = fmaxf(qmax, __shfl_xor_sync(0xffffffffu, qmax, 1));
+        qmax = fmaxf(qmax, __shfl_xor_sync(0xffffffffu, qmax, 2));       // the four lanes of a row hold all its elements
+        uint32_t e = __float_as_uint(qmax) >> 23;                        // biased exponent (qmax >= 0)
+        e = e > 253u ? 253u : e;
+        const float down = __uint_as_float((254u - e) << 23);            // 2^-(e - 127)
+        logit_scale *= __uint_as_float(e << 23);                         // 2^(e - 127); zero for a zero row
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+            qa[ks][0] = pack_f16x2(bf16_lo(qa[ks][0]) * down, bf16_hi(qa[ks][0]) * down);
+            qa[ks][1] = pack_f16x2(bf16_lo(qa[ks][1]) * down, bf16_hi(qa[ks][1]) * down);
+        }
+    }
+
     float o[kNTiles][4];
 #pragma unroll
     for (int i = 0; i < kNTiles; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.0f;
     float m_run = -INFINITY, l_run = 0.0f;
+    float vref = 0.0f;                     // 8-bit rows: the largest V scale met so far; o is in units of it
 
     const uint32_t my_stages = smem_base + warp * kAttnStages * kStageBytes;
     const uint32_t my_bars = bars + 8 * warp * kAttnStages;
@@ -183,8 +206,9 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         const bool prefix = t < n_pt;
         mbar_arrive_expect_tx(bar, kStageBytes);
         if constexpr (kFp8) {
-            tma_load_2d(dst, prefix ? &tmap_kpool : &tmap_kring, bar, 0, row, policy);
-            tma_load_2d(dst + kTileBytes8, prefix ? &tmap_vpool : &tmap_vring, bar, 0, row, policy);
+            // a tile of 8-bit rows is one contiguous piece of memory: coordinates (0, 0, tile)
+            tma_load_3d(dst, prefix ? &tmap_kpool : &tmap_kring, bar, 0, 0, row / kAttnTileRows, policy);
+            tma_load_3d(dst + kTileBytes8, prefix ? &tmap_vpool : &tmap_vring, bar, 0, 0, row / kAttnTileRows, policy);
         } else {
 #pragma unroll
             for (int hf = 0; hf < kHalves; ++hf) {
@@ -248,10 +272,10 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
 #pragma unroll
             for (int ks = 0; ks < kD / 16; ++ks) {
                 uint32_t k0, k1, k2, k3;
-                e4m3x4_to_bf16(w0[ks], k0, k1);
-                e4m3x4_to_bf16(w1[ks], k2, k3);
-                mma_bf16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, k0, k1);
-                mma_bf16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, k2, k3);
+                e4m3x4_to_f16(w0[ks], k0, k1);
+                e4m3x4_to_f16(w1[ks], k2, k3);
+                mma_f16_16816(s0, qa[ks][0], 0u, qa[ks][1], 0u, k0, k1);
+                mma_f16_16816(s1, qa[ks][0], 0u, qa[ks][1], 0u, k2, k3);
             }
             // the K rows' scales: this lane holds columns (rows of the tile) qc, qc + 1 of both column tiles
             s0[0] *= *reinterpret_cast<const float *>(kt + qc * kRowBytes8 + kD);
@@ -272,8 +296,8 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
             }
         }
         // ---- online softmax for row g: this lane holds columns qc, qc + 1 of both column tiles
-        float v00 = s0[0] * p.scale_log2e, v01 = s0[1] * p.scale_log2e;
-        float v10 = s1[0] * p.scale_log2e, v11 = s1[1] * p.scale_log2e;
+        float v00 = s0[0] * logit_scale, v01 = s0[1] * logit_scale;
+        float v10 = s1[0] * logit_scale, v11 = s1[1] * logit_scale;
         if (valid < kAttnTileRows) {
             if (qc >= valid) v00 = -INFINITY;
             if (qc + 1 >= valid) v01 = -INFINITY;
@@ -289,24 +313,39 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         const float p10 = fast_ex2(v10 - m_new), p11 = fast_ex2(v11 - m_new);
         l_run = l_run * alpha + ((p00 + p01) + (p10 + p11));
         m_run = m_new;
-#pragma unroll
-        for (int i = 0; i < kNTiles; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
         uint32_t pa0, pa2;
         if constexpr (kFp8) {
+            // the V rows' scales (zero for rows past the end), relative to the largest one so far
             const uint8_t *vt = smem + (sV - smem_base);
-            pa0 = pack_bf16x2(p00 * *reinterpret_cast<const float *>(vt + qc * kRowBytes8 + kD),
-                              p01 * *reinterpret_cast<const float *>(vt + (qc + 1) * kRowBytes8 + kD));
-            pa2 = pack_bf16x2(p10 * *reinterpret_cast<const float *>(vt + (8 + qc) * kRowBytes8 + kD),
-                              p11 * *reinterpret_cast<const float *>(vt + (9 + qc) * kRowBytes8 + kD));
+            const float vs00 = *reinterpret_cast<const float *>(vt + qc * kRowBytes8 + kD);
+            const float vs01 = *reinterpret_cast<const float *>(vt + (qc + 1) * kRowBytes8 + kD);
+            const float vs10 = *reinterpret_cast<const float *>(vt + (8 + qc) * kRowBytes8 + kD);
+            const float vs11 = *reinterpret_cast<const float *>(vt + (9 + qc) * kRowBytes8 + kD);
+            float vmax = fmaxf(fmaxf(fabsf(vs00), fabsf(vs01)), fmaxf(fabsf(vs10), fabsf(vs11)));
+            vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 1));
+            vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, 2));
+            const float vref_new = fmaxf(vref, vmax);
+            const float rinv = vref_new > 0.0f ? 1.0f / vref_new : 0.0f;
+            const float alpha_o = alpha * (vref * rinv);
+            vref = vref_new;
+            // the accumulator tiles hold O^T: this lane's columns are query heads qc and qc + 1
+            const float a_lo = __shfl_sync(0xffffffffu, alpha_o, qc * 4), a_hi = __shfl_sync(0xffffffffu, alpha_o, qc * 4 + 4);
+#pragma unroll
+            for (int i = 0; i < kNTiles; ++i) { o[i][0] *= a_lo; o[i][1] *= a_hi; o[i][2] *= a_lo; o[i][3] *= a_hi; }
+            pa0 = pack_f16x2(p00 * (vs00 * rinv), p01 * (vs01 * rinv));
+            pa2 = pack_f16x2(p10 * (vs10 * rinv), p11 * (vs11 * rinv));
         } else {
+#pragma unroll
+            for (int i = 0; i < kNTiles; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; }
             pa0 = pack_bf16x2(p00, p01);
             pa2 = pack_bf16x2(p10, p11);
         }
 
         // ---- O += P V: two 8-column output tiles per ldmatrix
         if constexpr (kFp8) {
-            // V rows 2c, 2c+1 (k = 2c, 2c+1) and 2c+8, 2c+9 of the tile, this lane's D/8 bytes of each;
-            // output tile i takes byte i of each row
+            // O^T[D x 8] += V^T[D x 16] P^T[16 x 8]: P as it comes out of the softmax is the B operand (k = row of the
+            // tile, n = query head), V^T is the A operand.  V rows 2c, 2c+1 (k = 2c, 2c+1) and 2c+8, 2c+9 of the tile,
+            // this lane's D/8 bytes of each; accumulator tile i takes bytes 2i (MMA rows 0..7) and 2i+1 (rows 8..15)
             const uint8_t *vt = smem + (sV - smem_base) + g * (kD / 8);
             uint32_t ra[kD / 32], rb[kD / 32], rc[kD / 32], rd[kD / 32];
             if constexpr (kD == 128) {
@@ -328,11 +367,11 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
             }
 #pragma unroll
             for (int i = 0; i < kNTiles; ++i) {
-                const uint32_t sel = (i & 3) | ((4 + (i & 3)) << 4);
-                const uint32_t quad = __byte_perm(__byte_perm(ra[i >> 2], rb[i >> 2], sel), __byte_perm(rc[i >> 2], rd[i >> 2], sel), 0x5410);
-                uint32_t v0, v1;
-                e4m3x4_to_bf16(quad, v0, v1);
-                mma_bf16_16816(o[i], pa0, 0u, pa2, 0u, v0, v1);
+                const uint32_t sel = (i & 1) ? 0x7362u : 0x5140u;       // bytes k, k+1 of both rows, interleaved (k = 0 or 2)
+                uint32_t a0, a1, a2, a3;
+                e4m3x4_to_f16(__byte_perm(ra[i >> 1], rb[i >> 1], sel), a0, a1);
+                e4m3x4_to_f16(__byte_perm(rc[i >> 1], rd[i >> 1], sel), a2, a3);
+                mma_f16_16816(o[i], a0, a1, a2, a3, pa0, pa2);
             }
         } else {
             const int mi = lane >> 3, r8 = lane & 7;
@@ -373,9 +412,11 @@ decode_attn_kernel(const __grid_constant__ CUtensorMap tmap_kpool, const __grid_
         if ((lane & 3) == 0) { mine[g] = m_run; mine[8 + g] = l_run; }
 #pragma unroll
         for (int i = 0; i < kNTiles; ++i) {
-            if constexpr (kFp8) {           // output tile i, column j is element j D/8 + i
-                mine[16 + g * kD + qc * (kD / 8) + i] = o[i][0];
-                mine[16 + g * kD + (qc + 1) * (kD / 8) + i] = o[i][1];
+            if constexpr (kFp8) {           // O^T: rows are elements g D/8 + 2i (+1), columns query heads qc, qc+1; back from units of vref
+                mine[16 + qc * kD + g * (kD / 8) + 2 * i] = o[i][0] * vref;
+                mine[16 + (qc + 1) * kD + g * (kD / 8) + 2 * i] = o[i][1] * vref;
+                mine[16 + qc * kD + g * (kD / 8) + 2 * i + 1] = o[i][2] * vref;
+                mine[16 + (qc + 1) * kD + g * (kD / 8) + 2 * i + 1] = o[i][3] * vref;
             } else {
                 mine[16 + g * kD + i * 8 + qc] = o[i][0];
                 mine[16 + g * kD + i * 8 + qc + 1] = o[i][1];

@@ -239,16 +239,18 @@ static kvzap_status make_tmap8(kvzap_ctx *ctx, CUtensorMap *map, const void *bas
     return KVZAP_OK;
 }
 
-// Tensor map over `rows` rows of `row_bytes` bytes each; box = box_rows whole rows, no swizzle (the attention
-// kernel's tiles of 8-bit rows with their trailers).  row_bytes is a multiple of 16, at most 256.
+// Tensor map over `rows` rows of `row_bytes` bytes each, seen as tiles of box_rows whole rows: a tile is one
+// contiguous, 128-byte aligned piece of memory (box_rows * row_bytes is a multiple of 128), fetched as that many
+// full 128-byte lines and laid out in shared memory as it lies in memory (no swizzle).  Coordinates (0, 0, tile).
 static kvzap_status make_tmap_rows(kvzap_ctx *ctx, CUtensorMap *map, const void *base, uint64_t rows, uint32_t row_bytes,
                                    uint32_t box_rows)
 {
-    const cuuint64_t dims[2] = {row_bytes, rows};
-    const cuuint64_t strides[1] = {row_bytes};
-    const cuuint32_t box[2] = {row_bytes, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+    const uint32_t lines = box_rows * row_bytes / 128;
+    const cuuint64_t dims[3] = {128, lines, rows / box_rows};
+    const cuuint64_t strides[2] = {128, static_cast<cuuint64_t>(lines) * 128};
+    const cuuint32_t box[3] = {128, lines, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = ctx->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(base), dims, strides, box, estr,
                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
