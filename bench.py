@@ -35,11 +35,14 @@ HEADLINE = "qwen3_32b_prefill_128k_paged"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, taken from the ncu
 # capture summarised in the named file under profiles/ (bytes per launch; not measured in this run).
 NCU_TRAFFIC = {
-    "qwen3_8b_prefill_32k": (276.8e6, "profiles/score_kernel_mlp_qwen3_8b_prefill_32k.md"),
-    "qwen3_8b_decode_b128": (227.9e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
+    "qwen3_32b_prefill_128k_paged": (2065.3e6, "profiles/score_kernel_mlp_qwen3_32b_prefill_128k_paged.md"),
+    "qwen3_8b_prefill_32k": (277.2e6, "profiles/score_kernel_mlp_qwen3_8b_prefill_32k.md"),
+    "llama31_8b_prefill_4x16k": (540.8e6, "profiles/score_kernel_linear_llama31_8b_prefill_4x16k.md"),
+    "linear_4k": (39.72e6, "profiles/score_linear_split_kernel_linear_4k.md"),
+    "qwen3_8b_decode_b128": (226.3e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
 }
 # attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
-NCU_ATTENTION_TRAFFIC_RATIO = 2.409 / 2.3986
+NCU_ATTENTION_TRAFFIC_RATIO = 2.4093 / 2.3986
 
 
 def load_peaks():
