@@ -41,8 +41,12 @@ NCU_TRAFFIC = {
     "linear_4k": (39.72e6, "profiles/score_linear_split_kernel_linear_4k.md"),
     "qwen3_8b_decode_b128": (226.3e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
 }
+NCU_TRAFFIC_FP8 = {
+    "qwen3_8b_prefill_32k": (140.4e6, "profiles/score_kernel_mlp_fp8_qwen3_8b_prefill_32k.md"),
+}
 # attention over the pruned cache: DRAM bytes per ALGORITHMIC byte, from a one-layer capture (traffic grows with the rows read)
 NCU_ATTENTION_TRAFFIC_RATIO = 2.4093 / 2.3986
+NCU_ATTENTION_FP8_TRAFFIC_RATIO = 1.3609 / 1.3501
 
 
 def load_peaks():
@@ -407,6 +411,8 @@ def run_prefill(args, wl, env, sub=False):
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "alone_achieved": score_bytes / (score_ms * 1e-3) / 1e9}
     traffic = NCU_TRAFFIC.get(wl.name) if args.layers == 0 and not proj else None
+    if fp8:
+        traffic = NCU_TRAFFIC_FP8.get(wl.name) if args.layers == 0 and not proj else None
     roofline.update({"traffic": traffic[0] if traffic else None,
                      "traffic_source": (traffic[1] + " (ncu capture, not measured in this run)") if traffic else None,
                      "kernel": "score_kernel", "peak_source": peak_src,
@@ -724,7 +730,7 @@ def run_attention(args, wl, env):
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "clocks": clocks, "gpu_launches": int(ctx.launch_count() - launches0),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": None if fp8 else alg_bytes * NCU_ATTENTION_TRAFFIC_RATIO,
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": alg_bytes * (NCU_ATTENTION_FP8_TRAFFIC_RATIO if fp8 else NCU_ATTENTION_TRAFFIC_RATIO),
                          "kernel": "decode_attn_kernel", "peak_source": peak_src, "kernel_ms": ms,
                          "algorithmic_bytes_per_step": alg_bytes}}
     binding.kvzap_cache_destroy(cache)
