@@ -472,6 +472,23 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
                                     float tau, float *scores_out, void *stream);
 
 /*
+ * The same for several prompts (or chunks of prompts) at once, one layer: sequence i of the call is tokens
+ * cu_seqlens[i] .. cu_seqlens[i+1] of the packed buffers and goes to the cache's sequence slot seq_ids[i].
+ * One scoring launch over all tokens instead of one small launch per prompt, and three more launches
+ * for the whole batch (window side, page assignment, compaction).  Each sequence ends up exactly as
+ * kvzap_prefill_to_cache would leave it (which pages a list gets depends on the order of allocation and
+ * may differ).
+ *   seq_ids    [n_seqs] int32, HOST: distinct slots in 0..n_seqs_of_the_cache-1 (checked; read before return)
+ *   cu_seqlens [n_seqs+1] int32 (device); empty sequences are allowed and change nothing
+ *   hidden [n_tokens, d_model] bf16, K, V [H, n_tokens, D] bf16 (packed over the sequences),
+ *   scores_out [n_tokens, H] fp32 (device) -- required
+ * n_seqs <= max_seqs and n_tokens <= max_tokens of the context.
+ */
+kvzap_status kvzap_prefill_to_cache_batch(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, const int32_t *seq_ids,
+                                          const int32_t *cu_seqlens, int32_t n_seqs, const void *hidden, const void *K,
+                                          const void *V, int64_t n_tokens, float tau, float *scores_out, void *stream);
+
+/*
  * Installs prefix bookkeeping produced elsewhere (used to set up synthetic
  * cache states): prefix_len [n_seqs*L*H] and page_table
  * [n_seqs*L*H, max_pages_per_list], device int32 in list order (seq, layer,

@@ -78,6 +78,7 @@ SIGNATURES = {
     "kvzap_cache_lengths": (_i32, [_vp, _vp, _vp]),
     "kvzap_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _i64, _vp, _vp]),
     "kvzap_prefill_to_cache": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
+    "kvzap_prefill_to_cache_batch": (_i32, [_vp, _vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp, _i64, _f32, _vp, _vp]),
     "kvzap_cache_import": (_i32, [_vp, _vp, _vp, _i32, _vp]),
     "kvzap_cache_snapshot": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "kvzap_set_wait_limit": (_i32, [_vp, _i64]),
@@ -368,6 +369,15 @@ def kvzap_cache_export(handle, cache, seq, layer, head, K_out, V_out, n_rows, st
 def kvzap_prefill_to_cache(handle, cache, layer, seq, hidden, K, V, tau, scores_out, stream=None):
     _check(handle, load().kvzap_prefill_to_cache(handle, cache, layer, seq, _ptr(hidden), _ptr(K), _ptr(V), K.shape[1],
                                                  tau, _ptr(scores_out), _stream(stream)))
+
+
+def kvzap_prefill_to_cache_batch(handle, cache, layer, seq_ids, cu_seqlens, hidden, K, V, tau, scores_out, stream=None):
+    """seq_ids: a Python sequence of slot numbers (host); cu_seqlens int32 [len(seq_ids) + 1] on the device;
+    hidden [n_tokens, d_model], K, V [H, n_tokens, D] packed over the sequences."""
+    ids = (ctypes.c_int32 * len(seq_ids))(*[int(x) for x in seq_ids])
+    _check(handle, load().kvzap_prefill_to_cache_batch(handle, cache, layer, ctypes.cast(ids, ctypes.c_void_p), _ptr(cu_seqlens),
+                                                       len(seq_ids), _ptr(hidden), _ptr(K), _ptr(V), K.shape[1], tau,
+                                                       _ptr(scores_out), _stream(stream)))
 
 
 def kvzap_cache_import(handle, cache, prefix_len, page_table, next_free_page, stream=None):

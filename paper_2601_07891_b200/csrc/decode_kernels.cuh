@@ -188,16 +188,26 @@ decode_update_kernel(const CacheView c, int layer0, int n_layers_call, const flo
 //      their absolute positions n_old + chunk index;
 //   3. n_tokens advances by m.
 // The chunk's own tokens before its last w are appended to the prefix afterwards by the compaction.
+// A batch of prompts in one launch (grid (H, n_seqs)): sequence b's chunk is tokens cu_seqlens[b] .. cu_seqlens[b+1]
+// of the packed buffers (K, V [H][n_total][D], scores [n_total][H]) and its lists start at list_map[b];
+// list_map == nullptr: one sequence, lists li0 .. li0+H-1, m = n_total tokens.
 __global__ void __launch_bounds__(256)
 chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scores, const uint4 *__restrict__ K,
-                  const uint4 *__restrict__ V, int64_t m, float tau, int32_t *__restrict__ status)
+                  const uint4 *__restrict__ V, int64_t n_total, float tau, int32_t *__restrict__ status,
+                  const int64_t *__restrict__ list_map, const int32_t *__restrict__ cu_seqlens)
 {
     __shared__ int64_t exit_src[128];       // ring row of an exiting token
     __shared__ int64_t exit_dst[128];       // its pool row, -1 = dropped
     __shared__ int64_t len_s;
     __shared__ int ok_s;
     const int h = blockIdx.x;
-    const int64_t li = li0 + h;
+    const int64_t li = (list_map != nullptr ? list_map[blockIdx.y] : li0) + h;
+    const int64_t tok0 = list_map != nullptr ? static_cast<int64_t>(cu_seqlens[blockIdx.y]) : 0;
+    const int64_t m = list_map != nullptr ? static_cast<int64_t>(cu_seqlens[blockIdx.y + 1]) - tok0 : n_total;
+    if (m <= 0) return;                     // an empty chunk leaves its lists as they are
+    K += tok0 * c.row_units;                // row (h, i) of the chunk is row h * n_total + tok0 + i of the buffers
+    V += tok0 * c.row_units;
+    scores += tok0 * c.n_heads;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int64_t n_old = c.n_tokens[li];
     const int64_t in_ring = n_old < c.window ? n_old : c.window;
@@ -294,7 +304,7 @@ chunk_ring_kernel(const CacheView c, int64_t li0, const float *__restrict__ scor
         for (int j = 0; j < 4; ++j) {
             const int64_t i = i0 + 256 * j;
             if (i < n_win * c.row_units) {
-                const int64_t src = (static_cast<int64_t>(h) * m + m - n_win + i / c.row_units) * c.row_units + i % c.row_units;
+                const int64_t src = (static_cast<int64_t>(h) * n_total + m - n_win + i / c.row_units) * c.row_units + i % c.row_units;
                 kr[j] = __ldg(K + src);
                 vr[j] = __ldg(V + src);
             }
@@ -341,8 +351,14 @@ release_seq_kernel(const CacheView c, int32_t seq)
 }
 
 // no window: only the token count advances
-__global__ void tokens_add_kernel(const CacheView c, int64_t li0, int64_t m)
+__global__ void tokens_add_kernel(const CacheView c, int64_t li0, int64_t m, const int64_t *__restrict__ list_map,
+                                  const int32_t *__restrict__ cu_seqlens)
 {
+    if (list_map != nullptr) {              // one block per sequence of a batch
+        li0 = list_map[blockIdx.x];
+        m = cu_seqlens[blockIdx.x + 1] - cu_seqlens[blockIdx.x];
+        if (m <= 0) return;
+    }
     if (threadIdx.x < c.n_heads) c.n_tokens[li0 + threadIdx.x] += static_cast<int32_t>(m);
     if (threadIdx.x == 0) c.active[li0 / (static_cast<int64_t>(c.n_layers) * c.n_heads)] = 1;
 }

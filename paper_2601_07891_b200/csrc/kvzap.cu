@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <algorithm>
 #include <vector>
 
 #include "attn_kernel.cuh"
@@ -81,6 +82,7 @@ struct kvzap_ctx {
     uint32_t *select_hist = nullptr;     // fixed-budget selection: [4 passes][max_seqs][H][256] histograms
     float *select_tau = nullptr;         //                         [max_seqs][H] cut values when the caller wants none
     float *plan_scores = nullptr;        // kvzap_prefill_plan without scores_out: [max_tokens][H] (allocated on first use)
+    int64_t *batch_map = nullptr;        // kvzap_prefill_to_cache_batch: first list of each sequence of the call [max_seqs]
     float *split_part = nullptr;         // few-token kernel: [sm_count tiles][4 slices][128][8] partial scores
     uint32_t *split_arrive = nullptr;    //                   [sm_count] arrival counts per tile
     uint64_t score_turn = 0;
@@ -386,6 +388,7 @@ static void free_all(kvzap_ctx *ctx)
     cudaFree(ctx->tile_counters);
     cudaFree(ctx->split_part);
     cudaFree(ctx->plan_scores);
+    cudaFree(ctx->batch_map);
     cudaFree(ctx->select_hist);
     cudaFree(ctx->select_tau);
     cudaFree(ctx->split_arrive);
@@ -909,7 +912,8 @@ static kvzap_status launch_compaction(kvzap_ctx *ctx, const uint32_t *mask, cons
                                            static_cast<const int32_t *>(nullptr),
                                            tok_major ? int64_t{1} : n_tokens,
                                            tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
-                                           static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr), 0));
+                                           static_cast<const int32_t *>(nullptr), static_cast<const int32_t *>(nullptr), 0,
+                                           static_cast<const int64_t *>(nullptr)));
     }
     ctx->launches += 1;
     return KVZAP_OK;
@@ -1808,7 +1812,8 @@ extern "C" kvzap_status kvzap_prune_prefill_noalloc(const void *K, const void *V
                                                                      tau, w, 1, maskbits, n_words, nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     scan_kernel<<<1, 1024, 0, stream>>>(maskbits, n_words, n_blocks, n_kv_heads, cu_seqlens, n_seqs, n_tokens,
-                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status, 0, nullptr, nullptr, nullptr);
+                                        blockprefix, seqbase, lengths, 0, 0, 0, 0, nullptr, nullptr, nullptr, nullptr, status, 0, nullptr, nullptr, nullptr,
+                                        nullptr);
     KVZAP_CUDA(nullptr, cudaGetLastError());
     const dim3 grid(static_cast<unsigned>(n_blocks), static_cast<unsigned>(n_kv_heads));
     compact_kernel<false><<<grid, kCompactThreads, 0, stream>>>(
@@ -1858,7 +1863,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                             int32_t *n_pages_used, cudaStream_t stream,
                                             int32_t *page_cursor = nullptr, bool tok_major = false, bool append = false,
                                             bool beside_scoring = true, const int32_t *free_stack = nullptr,
-                                            int32_t *free_top = nullptr)
+                                            int32_t *free_top = nullptr, const int64_t *list_map = nullptr)
 {
     const kvzap_config &c = ctx->cfg;
     const int64_t n_blocks = (n_tokens + kBlockTokens - 1) / kBlockTokens;
@@ -1874,7 +1879,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            static_cast<int32_t *>(nullptr),
                                            lengths, static_cast<int>(page_tokens), first_page, n_pages_pool,
                                            static_cast<int>(max_pages), ctx->list_page0, page_table, n_pages_used,
-                                           page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, free_stack, free_top));
+                                           page_cursor, ctx->status_dev, append ? 1 : 0, ctx->list_base, free_stack, free_top, list_map));
     }
     // the same resident-at-once grid as the dense-ragged output (see launch_compaction)
     const int64_t max_ctas = static_cast<int64_t>(ctx->sm_count) * (!beside_scoring ? 8 : (c.hidden > 0 ? 2 : 6));
@@ -1896,7 +1901,7 @@ static kvzap_status launch_compaction_paged(kvzap_ctx *ctx, const uint32_t *mask
                                            tok_major ? int64_t{1} : n_tokens,
                                            tok_major ? static_cast<int64_t>(c.n_kv_heads) : int64_t{1},
                                            static_cast<const int32_t *>(append ? ctx->list_base : nullptr),
-                                           static_cast<const int32_t *>(page_table), static_cast<int>(max_pages)));
+                                           static_cast<const int32_t *>(page_table), static_cast<int>(max_pages), list_map));
     }
     ctx->launches += 2;
     return KVZAP_OK;
@@ -2408,14 +2413,69 @@ kvzap_status kvzap_prefill_to_cache(kvzap_ctx *ctx, kvzap_cache *cache, int32_t 
     if (st != KVZAP_OK) return st;
     if (v.window > 0)
         chunk_ring_kernel<<<static_cast<unsigned>(v.n_heads), 256, 0, stream>>>(
-            v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens, tau, ctx->status_dev);
+            v, li0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens, tau, ctx->status_dev,
+            nullptr, nullptr);
     else
-        tokens_add_kernel<<<1, 32, 0, stream>>>(v, li0, n_tokens);
+        tokens_add_kernel<<<1, 32, 0, stream>>>(v, li0, n_tokens, nullptr, nullptr);
     KVZAP_CUDA(ctx, cudaGetLastError());
     ctx->launches += 1;
     return launch_compaction_paged(ctx, mask, K, V, nullptr, 1, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool, v.page_tokens, 0,
                                    v.page_table + li0 * v.max_pages, v.max_pages, v.prefix_len + li0, nullptr, stream,
                                    v.page_cursor, false, true, true, v.free_stack, v.free_top);
+}
+
+kvzap_status kvzap_prefill_to_cache_batch(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer, const int32_t *seq_ids,
+                                          const int32_t *cu_seqlens, int32_t n_seqs, const void *hidden, const void *K,
+                                          const void *V, int64_t n_tokens, float tau, float *scores_out, void *stream_)
+{
+    NvtxRange nvtx_range("kvzap_prefill_to_cache_batch");
+    if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
+    begin_op(ctx);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const kvzap_config &c = ctx->cfg;
+    const CacheView &v = cache->v;
+    if (layer < 0 || layer >= c.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache_batch: layer %d out of range", layer);
+    if (!seq_ids || !cu_seqlens || n_seqs < 1)
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache_batch: seq_ids (host), cu_seqlens (device), n_seqs >= 1 are required");
+    kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
+    if (st != KVZAP_OK) return st;
+    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    // the lists of head 0 of every sequence; slots must be in range and distinct (two chunks for one list in
+    // one launch would race)
+    std::vector<int64_t> map(static_cast<size_t>(n_seqs));
+    {
+        std::vector<int32_t> sorted(seq_ids, seq_ids + n_seqs);
+        std::sort(sorted.begin(), sorted.end());
+        for (int i = 0; i < n_seqs; ++i) {
+            if (sorted[i] < 0 || sorted[i] >= v.n_seqs)
+                return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache_batch: sequence slot %d out of range", sorted[i]);
+            if (i > 0 && sorted[i] == sorted[i - 1])
+                return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache_batch: sequence slot %d given twice", sorted[i]);
+            map[i] = (static_cast<int64_t>(seq_ids[i]) * v.n_layers + layer) * v.n_heads;
+        }
+    }
+    if (n_tokens == 0) return KVZAP_OK;
+    if (!hidden || !K || !V || !scores_out || !aligned16(hidden) || !aligned16(K) || !aligned16(V))
+        return fail(ctx, KVZAP_ERR_INVALID_ARG, "prefill_to_cache_batch: hidden, K, V, scores_out must be non-NULL, aligned");
+    DeviceGuard guard(c.device);
+    if (!ctx->batch_map) KVZAP_CUDA(ctx, cudaMalloc(&ctx->batch_map, sizeof(int64_t) * static_cast<size_t>(c.max_seqs)));
+    // from pageable host memory: staged by the driver before the call returns; ordered on the stream behind the
+    // kernels of an earlier batch that still read the previous map
+    KVZAP_CUDA(ctx, cudaMemcpyAsync(ctx->batch_map, map.data(), sizeof(int64_t) * map.size(), cudaMemcpyHostToDevice, stream));
+    uint32_t *mask = next_mask_slice(ctx);
+    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, v.window, stream, 0);
+    if (st != KVZAP_OK) return st;
+    if (v.window > 0)
+        chunk_ring_kernel<<<dim3(static_cast<unsigned>(v.n_heads), static_cast<unsigned>(n_seqs)), 256, 0, stream>>>(
+            v, 0, scores_out, static_cast<const uint4 *>(K), static_cast<const uint4 *>(V), n_tokens, tau, ctx->status_dev,
+            ctx->batch_map, cu_seqlens);
+    else
+        tokens_add_kernel<<<static_cast<unsigned>(n_seqs), 32, 0, stream>>>(v, 0, 0, ctx->batch_map, cu_seqlens);
+    KVZAP_CUDA(ctx, cudaGetLastError());
+    ctx->launches += 1;
+    return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, v.k_pool, v.v_pool, v.n_pages_pool,
+                                   v.page_tokens, 0, v.page_table, v.max_pages, v.prefix_len, nullptr, stream, v.page_cursor,
+                                   false, true, true, v.free_stack, v.free_top, ctx->batch_map);
 }
 
 }  // extern "C"

@@ -97,6 +97,14 @@ __device__ __forceinline__ int32_t kept_before(const uint32_t *__restrict__ mask
     return n;
 }
 
+// Where list idx (= b * n_heads + h) of a call lives in the caller's per-list arrays (lengths, page tables): at
+// idx itself, or -- appending a batch of prompts to a cache, whose lists are ordered (sequence slot, layer, head) --
+// at list_map[b] + h, list_map [n_seqs] naming the list of head 0 of each of the call's sequences.
+__device__ __forceinline__ int64_t list_at(const int64_t *__restrict__ list_map, int idx, int n_heads)
+{
+    return list_map != nullptr ? list_map[idx / n_heads] + idx % n_heads : static_cast<int64_t>(idx);
+}
+
 // ---------------------------------------------------------------------------
 // Page assignment of the paged output, by all NT threads of one CTA: list idx (= b * n_heads + h) needs
 // ceil(lengths[idx] / page_tokens) pages (less those it owns already when appending); list_page0 receives the
@@ -110,7 +118,7 @@ assign_pages(int n_heads, int n_seqs, int32_t *__restrict__ lengths, int page_to
              int64_t n_pages_pool, int max_pages, int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table,
              int32_t *__restrict__ n_pages_used, int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
              int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top,
-             int fill_table)
+             int fill_table, const int64_t *__restrict__ list_map = nullptr)
 {
     __shared__ int32_t warp_sums[32];
     __shared__ int32_t carry_s;
@@ -148,7 +156,7 @@ assign_pages(int n_heads, int n_seqs, int32_t *__restrict__ lengths, int page_to
         const int idx = base + tid;
         int32_t need = 0;
         if (idx < n_lists) {
-            need = (lengths[idx] + page_tokens - 1) / page_tokens;
+            need = (lengths[list_at(list_map, idx, n_heads)] + page_tokens - 1) / page_tokens;
             if (need > max_pages) fail_s = 1;
             if (append) need -= (list_base[idx] + page_tokens - 1) / page_tokens;     // pages the list already owns
         }
@@ -171,7 +179,7 @@ assign_pages(int n_heads, int n_seqs, int32_t *__restrict__ lengths, int page_to
     if (fail) {
         for (int idx = tid; idx < n_lists; idx += NT) {
             list_page0[idx] = -1;
-            if (append) lengths[idx] = list_base[idx];
+            if (append) lengths[list_at(list_map, idx, n_heads)] = list_base[idx];
         }
         if (tid == 0) {
             atomicCAS(status, 0, 4 /* KVZAP_ERR_OOM_PAGES */);
@@ -190,10 +198,11 @@ assign_pages(int n_heads, int n_seqs, int32_t *__restrict__ lengths, int page_to
     for (int idx = warp; idx < n_lists; idx += NT / 32) {            // a warp per list
         const int32_t p0 = list_page0[idx];
         const int32_t have = append ? (list_base[idx] + page_tokens - 1) / page_tokens : 0;
-        const int32_t need = (lengths[idx] + page_tokens - 1) / page_tokens - have;
+        const int64_t li = list_at(list_map, idx, n_heads);
+        const int32_t need = (lengths[li] + page_tokens - 1) / page_tokens - have;
         for (int32_t i = lane; i < need; i += 32) {
             const int32_t j = p0 - first_page + i;            // ordinal among the pages assigned by this call
-            page_table[static_cast<int64_t>(idx) * max_pages + have + i] =
+            page_table[li * max_pages + have + i] =
                 j < from_stack ? free_stack[n_free - 1 - j] : first_page + (j - from_stack);
         }
     }
@@ -225,7 +234,8 @@ scan_lists(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blo
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
             int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
-            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top)
+            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top,
+            const int64_t *__restrict__ list_map = nullptr)
 {
     // page_cursor != nullptr: the first page comes from (and the pages used are added to) a device-side
     // allocator cursor instead of the first_page argument
@@ -288,9 +298,10 @@ scan_lists(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blo
             if (lane == 0 && cnt) atomicAdd(&group_sum[grp], cnt);
             __syncthreads();
             if (gt == 0 && idx < n_lists_all) {
-                const int32_t old = append ? lengths[idx] : 0;
+                const int64_t li = list_at(list_map, idx, n_heads);
+                const int32_t old = append ? lengths[li] : 0;
                 if (append) list_base[idx] = old;
-                lengths[idx] = old + group_sum[grp];
+                lengths[li] = old + group_sum[grp];
             }
             __syncthreads();
         }
@@ -325,15 +336,16 @@ scan_lists(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_blo
     __syncthreads();
     for (int idx = tid; idx < n_heads * n_seqs; idx += NT) {
         const int b = idx / n_heads, h = idx % n_heads;
-        const int32_t old = append ? lengths[idx] : 0;
+        const int64_t li = list_at(list_map, idx, n_heads);
+        const int32_t old = append ? lengths[li] : 0;
         if (append) list_base[idx] = old;
-        lengths[idx] = old + seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
+        lengths[li] = old + seqbase[h * (n_seqs + 1) + b + 1] - seqbase[h * (n_seqs + 1) + b];
     }
     }
     if (page_tokens <= 0) return;
     __syncthreads();
     assign_pages<NT>(n_heads, n_seqs, lengths, page_tokens, first_page, n_pages_pool, max_pages, list_page0, page_table,
-                     n_pages_used, page_cursor, status, append, list_base, free_stack, free_top, 1);
+                     n_pages_used, page_cursor, status, append, list_base, free_stack, free_top, 1, list_map);
 }
 
 // The page assignment as a kernel of its own: one CTA of 1024 threads (behind the fused scoring kernels
@@ -345,14 +357,15 @@ scan_kernel(const uint32_t *__restrict__ maskbits, int64_t n_words, int64_t n_bl
             int page_tokens, int32_t first_page, int64_t n_pages_pool, int max_pages,
             int32_t *__restrict__ list_page0, int32_t *__restrict__ page_table, int32_t *__restrict__ n_pages_used,
             int32_t *__restrict__ page_cursor, int32_t *__restrict__ status, int append,
-            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top)
+            int32_t *__restrict__ list_base, const int32_t *__restrict__ free_stack, int32_t *__restrict__ free_top,
+            const int64_t *__restrict__ list_map)
 {
     // may be placed before the kernel that writes the mask has finished; waits for it here
     griddep_launch_dependents();
     griddep_wait();
     scan_lists<1024>(maskbits, n_words, n_blocks, n_heads, cu_seqlens, n_seqs, n_tokens, blockprefix, seqbase, lengths,
                      page_tokens, first_page, n_pages_pool, max_pages, list_page0, page_table, n_pages_used, page_cursor,
-                     status, append, list_base, free_stack, free_top);
+                     status, append, list_base, free_stack, free_top, list_map);
 }
 
 // ---------------------------------------------------------------------------
@@ -475,10 +488,12 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                      int64_t n_blocks, int blocks_per_cta, const int32_t *__restrict__ cu_seqlens, int n_seqs,
                      int64_t n_tokens, int n_heads, int row_units, int32_t *__restrict__ lengths, int page_tokens,
                      const int32_t *__restrict__ list_page0, int64_t in_stride_h, int64_t in_stride_t,
-                     const int32_t *__restrict__ list_base, const int32_t *__restrict__ page_table, int max_pages)
+                     const int32_t *__restrict__ list_base, const int32_t *__restrict__ page_table, int max_pages,
+                     const int64_t *__restrict__ list_map)
 {
     // list_base != nullptr (paged): list (b,h) already holds list_base[] rows; kept rows go behind them,
-    // into the pages that page_table [list][max_pages] names (the scan has entered the new ones).
+    // into the pages that page_table [list][max_pages] names (the scan has entered the new ones); the table
+    // of list (b,h) is row b * H + h of page_table, or row list_map[b] + h (see list_at).
     // Row (h, t) of the inputs starts at row index h * in_stride_h + t * in_stride_t: (n_tokens, 1) for
     // the head-major cache layout [H][T][D], (1, H) for the K/V projection's own output [T][H][D].
     // page_tokens > 0: paged output.  K_out / V_out are the page pools, list (b,h) starts at page
@@ -567,7 +582,8 @@ compact_dense_kernel(const uint4 *__restrict__ K, const uint4 *__restrict__ V, u
                             if (p0 < 0) {
                                 dst_row[r] = -1;
                             } else {
-                                const int64_t page = __ldcg(page_table + static_cast<int64_t>(b * n_heads + h) * max_pages + nn / page_tokens);
+                                const int64_t trow = list_map != nullptr ? list_map[b] + h : static_cast<int64_t>(b * n_heads + h);
+                                const int64_t page = __ldcg(page_table + trow * max_pages + nn / page_tokens);
                                 dst_row[r] = page * page_tokens + nn % page_tokens;
                             }
                         }
