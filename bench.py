@@ -240,8 +240,8 @@ def run_prefill(args, wl, env, sub=False):
     H, D, P = wl.n_kv_heads, wl.head_dim, wl.page_tokens
     proj = args.kv_layout == "proj"
     fp8 = args.fp8 and not sub
-    if fp8 and (wl.page_tokens or proj):
-        raise SystemExit("--fp8 goes with the dense-ragged prefill workloads in the [H,T,D] layout")
+    if fp8 and proj:
+        raise SystemExit("--fp8 goes with the prefill workloads in the [H,T,D] layout")
     ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, n_tokens, max_seqs=B, device=dev.index, trusted_producers=True)
     cu = torch.from_numpy(synth.cu_seqlens([T] * B)).to(dev) if B > 1 else None
 
@@ -304,7 +304,11 @@ def run_prefill(args, wl, env, sub=False):
         for i in (range(n_bufs) if n_bufs > L else [l]):
             prep_paged = binding.prepare_prefill_write_paged if proj else binding.prepare_prefill_fused_paged
             prep_dense = binding.prepare_prefill_write if proj else binding.prepare_prefill_fused
-            if fp8:
+            if fp8 and P:
+                calls[(l, i)] = binding.prepare_prefill_fused_paged_fp8(ctx.handle, l, Xs[i], Xscales[i], Ks[i], Vs[i], cu, B,
+                                                                        wl.tau, wl.window, Kos[i], Vos[i], P, 0, tabs[i],
+                                                                        lens[i], used[i], scs[i])
+            elif fp8:
                 calls[(l, i)] = binding.prepare_prefill_fused_fp8(ctx.handle, l, Xs[i], Xscales[i], Ks[i], Vs[i], cu, B, wl.tau,
                                                                   wl.window, Kos[i], Vos[i], lens[i], scs[i])
             elif P:

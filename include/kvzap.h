@@ -155,6 +155,14 @@ kvzap_status kvzap_prefill_fused_fp8(kvzap_ctx *ctx, int32_t layer, const void *
                                      void *K_out, void *V_out, int32_t *lengths,
                                      float *scores_out, void *stream);
 
+/* The same into pages (arguments as kvzap_prefill_fused_paged, hidden states and x_scale as above). */
+kvzap_status kvzap_prefill_fused_paged_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale,
+                                           const void *K, const void *V, const int32_t *cu_seqlens, int32_t n_seqs,
+                                           int64_t n_tokens, float tau, int32_t w, void *K_pool, void *V_pool,
+                                           int64_t n_pages_pool, int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                           int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                           float *scores_out, void *stream);
+
 /*
  * Threshold + sliding window + per-(sequence, head) ordered compaction
  * (Algorithm 1, the steps after scoring; Method, "KVzap": pairs whose score falls below tau

@@ -65,6 +65,8 @@ SIGNATURES = {
                                          _vp, _i32, _vp, _vp, _vp]),
     "kvzap_prefill_fused_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
                                          _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
+    "kvzap_prefill_fused_paged_fp8": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
+                                             _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "kvzap_prune_prefill_topk": (_i32, [_vp, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_write": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _vp, _vp, _vp]),
     "kvzap_prefill_write_paged": (_i32, [_vp, _i32, _vp, _vp, _vp, _vp, _i32, _i64, _f32, _i32, _vp, _vp, _i64, _i32,
@@ -439,6 +441,30 @@ def prepare_prefill_fused_fp8(handle, layer, hidden_e4m3, x_scale, K, V, cu_seql
             _ptr(K_out), _ptr(V_out), _ptr(lengths), _ptr(scores_out), _stream(stream))
     return PreparedCall("kvzap_prefill_fused_fp8", handle, args,
                         (hidden_e4m3, x_scale, K, V, cu_seqlens, K_out, V_out, lengths, scores_out))
+
+
+def _paged_fp8_args(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                    first_page, page_table, lengths, n_pages_used, scores_out, stream):
+    return (handle, layer, _ptr(hidden_e4m3), _ptr(x_scale), _ptr(K), _ptr(V), _ptr(cu_seqlens), n_seqs, K.shape[1], tau, w,
+            _ptr(K_pool), _ptr(V_pool), K_pool.shape[0], page_tokens, first_page, _ptr(page_table), page_table.shape[1],
+            _ptr(lengths), _ptr(n_pages_used), _ptr(scores_out), _stream(stream))
+
+
+def kvzap_prefill_fused_paged_fp8(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool,
+                                  page_tokens, first_page, page_table, lengths, n_pages_used, scores_out=None, stream=None):
+    """kvzap_prefill_fused_paged with hidden states as E4M3 bytes [n_tokens, d_model] and x_scale fp32 [n_tokens] or None."""
+    _check(handle, load().kvzap_prefill_fused_paged_fp8(*_paged_fp8_args(
+        handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens, first_page,
+        page_table, lengths, n_pages_used, scores_out, stream)))
+
+
+def prepare_prefill_fused_paged_fp8(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool,
+                                    page_tokens, first_page, page_table, lengths, n_pages_used, scores_out=None,
+                                    stream=None) -> PreparedCall:
+    args = _paged_fp8_args(handle, layer, hidden_e4m3, x_scale, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,
+                           first_page, page_table, lengths, n_pages_used, scores_out, stream)
+    return PreparedCall("kvzap_prefill_fused_paged_fp8", handle, args,
+                        (hidden_e4m3, x_scale, K, V, cu_seqlens, K_pool, V_pool, page_table, lengths, n_pages_used, scores_out))
 
 
 def prepare_prefill_fused_paged(handle, layer, hidden, K, V, cu_seqlens, n_seqs, tau, w, K_pool, V_pool, page_tokens,

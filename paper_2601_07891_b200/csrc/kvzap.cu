@@ -1959,7 +1959,8 @@ static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, cons
                                              float tau, int32_t w, void *K_pool, void *V_pool, int64_t n_pages_pool,
                                              int32_t page_tokens, int32_t first_page, int32_t *page_table,
                                              int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
-                                             float *scores_out, void *stream_, bool tok_major)
+                                             float *scores_out, void *stream_, bool tok_major, bool fp8 = false,
+                                             const float *x_scale = nullptr)
 {
     NvtxRange nvtx_range("kvzap_prefill_fused_paged / kvzap_prefill_write_paged");
     if (!ctx) return KVZAP_ERR_INVALID_ARG;
@@ -1968,7 +1969,8 @@ static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, cons
     if (layer < 0 || layer >= ctx->cfg.n_layers) return fail(ctx, KVZAP_ERR_INVALID_ARG, "layer %d out of range", layer);
     kvzap_status st = check_common(ctx, n_tokens, n_seqs, cu_seqlens);
     if (st != KVZAP_OK) return st;
-    if (!ctx->layer_set[layer]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", layer);
+    if (fp8 ? !ctx->layer_fp8[layer] : !ctx->layer_set[layer])
+        return fail(ctx, KVZAP_ERR_STATE, fp8 ? "layer %d has no 8-bit weights (kvzap_set_weights_fp8)" : "layer %d has no weights", layer);
     if (!lengths || !n_pages_used) return fail(ctx, KVZAP_ERR_INVALID_ARG, "lengths / n_pages_used is NULL");
     DeviceGuard guard(ctx->cfg.device);
     if (n_tokens == 0) {
@@ -1981,7 +1983,8 @@ static kvzap_status prefill_fused_paged_impl(kvzap_ctx *ctx, int32_t layer, cons
     if (st != KVZAP_OK) return st;
     if (!hidden || !aligned16(hidden)) return fail(ctx, KVZAP_ERR_INVALID_ARG, "hidden must be non-NULL, 16-byte aligned");
     uint32_t *mask = next_mask_slice(ctx);
-    st = launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
+    st = fp8 ? launch_score_fp8(ctx, layer, hidden, x_scale, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream)
+             : launch_score(ctx, layer, 1, hidden, n_tokens, scores_out, mask, cu_seqlens, n_seqs, tau, w, stream);
     if (st != KVZAP_OK) return st;
     return launch_compaction_paged(ctx, mask, K, V, cu_seqlens, n_seqs, n_tokens, K_pool, V_pool, n_pages_pool, page_tokens,
                                    first_page, page_table, max_pages_per_list, lengths, n_pages_used, stream, nullptr,
@@ -1998,6 +2001,18 @@ kvzap_status kvzap_prefill_fused_paged(kvzap_ctx *ctx, int32_t layer, const void
     return prefill_fused_paged_impl(ctx, layer, hidden, K, V, cu_seqlens, n_seqs, n_tokens, tau, w, K_pool, V_pool,
                                     n_pages_pool, page_tokens, first_page, page_table, max_pages_per_list, lengths,
                                     n_pages_used, scores_out, stream_, false);
+}
+
+kvzap_status kvzap_prefill_fused_paged_fp8(kvzap_ctx *ctx, int32_t layer, const void *hidden_e4m3, const float *x_scale,
+                                           const void *K, const void *V, const int32_t *cu_seqlens, int32_t n_seqs,
+                                           int64_t n_tokens, float tau, int32_t w, void *K_pool, void *V_pool,
+                                           int64_t n_pages_pool, int32_t page_tokens, int32_t first_page, int32_t *page_table,
+                                           int32_t max_pages_per_list, int32_t *lengths, int32_t *n_pages_used,
+                                           float *scores_out, void *stream_)
+{
+    return prefill_fused_paged_impl(ctx, layer, hidden_e4m3, K, V, cu_seqlens, n_seqs, n_tokens, tau, w, K_pool, V_pool,
+                                    n_pages_pool, page_tokens, first_page, page_table, max_pages_per_list, lengths,
+                                    n_pages_used, scores_out, stream_, false, true, x_scale);
 }
 
 kvzap_status kvzap_prefill_write_paged(kvzap_ctx *ctx, int32_t layer, const void *hidden, const void *K_proj,

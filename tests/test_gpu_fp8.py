@@ -91,6 +91,46 @@ def test_fp8_fused_prefill_matches_oracle(binding, oracle, seq_lens, hidden):
     ctx.close()
 
 
+@pytest.mark.parametrize("seq_lens,hidden,P", [([900], 128, 16), ([37, 0, 300, 129], 0, 4), ([20000], 640, 16)])
+def test_fp8_fused_paged_prefill_matches_oracle(binding, oracle, seq_lens, hidden, P):
+    """E4M3 hidden states into a paged output: scores against the 8-bit oracle, pools, page tables and lengths bit for bit
+    against the oracle's paged compaction on the GPU's scores."""
+    d_model, H, D, tau, w = 512, 8, 64, 0.25, 32
+    T, B = int(sum(seq_lens)), len(seq_lens)
+    ctx = binding.Kvzap(d_model, hidden, H, D, 1, T, max_seqs=B)
+    case = _fp8_case(d_model, hidden, H, T, seed=11 + hidden)
+    X8, sx, W18, sw, b1, W2, b2 = case
+    binding.kvzap_set_weights_fp8(ctx.handle, 0, W18.cuda(), sw.cuda(), b1.cuda(), parity.dev(W2), parity.dev(b2))
+    K, V = synth.keys_values(H, T, D, seed=12)
+    cu = synth.cu_seqlens(seq_lens)
+    cu_dev = torch.from_numpy(cu).cuda() if B > 1 else None
+    cu_arg = cu if B > 1 else None
+    n_pool, max_pages, first_page = H * (T // P + B + 1) + 5, max(seq_lens) // P + 2, 2
+    pool = lambda: torch.full((n_pool, P, D), -5.0, dtype=torch.bfloat16, device="cuda")
+    K_pool, V_pool = pool(), pool()
+    table = torch.full((B * H, max_pages), -1, dtype=torch.int32, device="cuda")
+    lengths = torch.zeros(B, H, dtype=torch.int32, device="cuda")
+    used = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scores = torch.empty(T, H, dtype=torch.float32, device="cuda")
+    binding.kvzap_prefill_fused_paged_fp8(ctx.handle, 0, X8.cuda(), sx.cuda(), parity.dev(K), parity.dev(V), cu_dev, B, tau, w,
+                                          K_pool, V_pool, P, first_page, table, lengths, used, scores)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    want = _oracle_scores(oracle, case, hidden)
+    s = scores.cpu().numpy()
+    assert np.abs(s - want).max() <= parity.SCORE_ATOL
+    keep = parity.check_mask_band(oracle, s, want, tau, w, cu_arg)
+    fill = int(synth.bits(torch.tensor([-5.0], dtype=torch.bfloat16))[0])
+    Kp, Vp, tab, ln, n_used = oracle.compact_paged(synth.bits(K), synth.bits(V), keep, P, n_pool, max_pages,
+                                                   cu_seqlens=cu_arg, first_page=first_page, fill=fill)
+    np.testing.assert_array_equal(lengths.cpu().numpy(), ln)
+    assert int(used.item()) == n_used
+    np.testing.assert_array_equal(table.cpu().numpy(), tab)
+    np.testing.assert_array_equal(synth.bits(K_pool), Kp)
+    np.testing.assert_array_equal(synth.bits(V_pool), Vp)
+    ctx.close()
+
+
 def test_fp8_needs_d_model_multiple_of_128_and_its_own_weights(binding):
     ctx = binding.Kvzap(192, 0, 8, 64, 1, max_tokens=64)
     W = torch.zeros(8, 192, dtype=torch.uint8, device="cuda")
