@@ -38,7 +38,10 @@ constexpr int kOpPairs = 8;
 constexpr int kOpRing = 16;            // scratch sets used in rotation by consecutive calls
 constexpr int kOpRows = 4;             // rows of K and of V per register set of a 16-lane group (two sets in rotation)
 // dynamic shared memory: the list of kept rows of kOpPairs (block, head) pairs, rounded up to whole rounds of the move loop
-constexpr uint32_t kOpDynSmem = (kOpPairs * 128 + (kOpThreads / 16) * kOpRows) * 16;
+constexpr int kOpFlight = 8;             // rows in flight per 16-lane group of the row mover (asynchronous copies)
+constexpr uint32_t kOpListBytes = (kOpPairs * 128 + (kOpThreads / 16) * kOpRows) * 16;
+constexpr uint32_t kOpFlightBytes = (kOpThreads / 16) * kOpFlight * 512;   // a slot: 256 bytes of K, 256 of V
+constexpr uint32_t kOpDynSmem = kOpListBytes + kOpFlightBytes;
 
 struct PruneParams {
     const float *scores;       // [n_tokens][n_heads]
@@ -471,8 +474,44 @@ prune_onepass_kernel(const PruneParams p)
             if (last) p.lengths[b * H + h] = n + (keep ? 1 : 0);
         }
         __syncthreads();
-        for (int u0 = gl; u0 < p.row_units && p.slot_out == nullptr; u0 += 16) {
-            // two register sets: the loads of one are in flight while the other is stored
+        if (p.slot_out == nullptr && p.row_units <= 16) {
+            // Rows of up to 256 bytes: every lane copies its 16 bytes of K and of V asynchronously into the group's
+            // ring of kOpFlight slots and stores a row once its copy has landed, so kOpFlight rows per group are on
+            // their way at any time and no register holds a row.  A lane reads back only the bytes it copied itself.
+            // Exactly kOpFlight copy groups are committed ahead of the row being stored (empty ones at the tail), so
+            // the wait is always for all but the newest kOpFlight - 1.
+            const bool act = gl < p.row_units;
+            const int64_t lane_off = static_cast<int64_t>(gl) * 16;
+            char *ring = reinterpret_cast<char *>(ent_s) + kOpListBytes + group * (kOpFlight * 512) + gl * 16;
+            const uint32_t ring_a = smem_u32(ring);
+            const int n_rows = total > group ? (total - group + kGroups - 1) / kGroups : 0;
+            auto issue = [&](int j) {
+                if (j < n_rows && act) {
+                    const int64_t src = ent_s[group + j * kGroups].x;
+                    const uint32_t slot = ring_a + (j % kOpFlight) * 512;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot), "l"(Kb + src + lane_off) : "memory");
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(slot + 256u), "l"(Vb + src + lane_off) : "memory");
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+#pragma unroll
+            for (int j = 0; j < kOpFlight; ++j) issue(j);
+            for (int j = 0; j < n_rows; ++j) {
+                asm volatile("cp.async.wait_group %0;" ::"n"(kOpFlight - 1) : "memory");
+                const int64_t dst = ent_s[group + j * kGroups].y;
+                if (act && dst >= 0) {
+                    const char *slot = ring + (j % kOpFlight) * 512;
+                    const uint4 kk = *reinterpret_cast<const uint4 *>(slot);
+                    const uint4 vv = *reinterpret_cast<const uint4 *>(slot + 256);
+                    *reinterpret_cast<uint4 *>(Ko + dst + lane_off) = kk;
+                    *reinterpret_cast<uint4 *>(Vo + dst + lane_off) = vv;
+                }
+                issue(j + kOpFlight);                          // into the slot just read (the stores above needed its data)
+            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        for (int u0 = gl; u0 < p.row_units && p.slot_out == nullptr && p.row_units > 16; u0 += 16) {
+            // longer rows -- two register sets: the loads of one are in flight while the other is stored
             const int64_t lane_off = static_cast<int64_t>(u0) * 16;
             uint4 ka[kRows], va[kRows], kb[kRows], vb[kRows];
             int64_t da[kRows], db[kRows];
