@@ -413,6 +413,10 @@ def run_prefill(args, wl, env, sub=False):
                     "frac_of_burst": achieved / (peaks["bf16_tflops"] * (2.0 if fp8 else 1.0)),
                     "frac_of_sustained": achieved / (peaks["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)),
                     "alone_achieved": flops / (score_ms * 1e-3) / 1e12}
+        if clocks.get("sm_mhz") and clocks.get("sm_max_mhz"):
+            # time x clock: the burst figure (measured at the maximum clock) scaled to the clock this region ran at
+            at_clock = peaks["bf16_tflops"] * (2.0 if fp8 else 1.0) * clocks["sm_mhz"] / clocks["sm_max_mhz"]
+            roofline["frac_of_burst_scaled_to_run_clock"] = achieved / at_clock
         if not args.skip_live_peak and not sub:
             # the GPUs of the pool settle at different clocks under the power cap: the same loop on this one, now
             live = live_gemm_tflops(dev)
@@ -517,9 +521,15 @@ def run_decode(args, wl, env, sub=False):
     L, B, H, D, w, P = wl.n_layers, wl.batch, wl.n_kv_heads, wl.head_dim, wl.window, wl.page_tokens
     if args.layers > 0:
         L = min(L, args.layers)
+    fp8 = bool(args.fp8) and not sub          # hidden states and first-layer weights as E4M3 bytes with scales
     ctx = binding.Kvzap(wl.d_model, wl.hidden, H, D, L, max_tokens=B, device=dev.index, trusted_producers=True)
     for l in range(L):
-        ctx.set_weights(l, *synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index))
+        wts = synth.surrogate_weights(wl, l, dev, seed_base=7000 + 100 * args.workload_index)
+        if fp8:
+            W18, sw = synth.quantize_e4m3(wts[0])
+            binding.kvzap_set_weights_fp8(ctx.handle, l, W18, sw, wts[1], *(wts[2:] if len(wts) == 4 else (None, None)))
+        else:
+            ctx.set_weights(l, *wts)
     n_lists = B * L * H
     n_steps = max(args.steps, 1000) if sub else args.steps
     total_steps = w + max(args.warmup, 3) + n_steps + 8 + (max(args.e2e_steps, 10) + 3 if not args.skip_e2e and not sub else 0)
@@ -545,8 +555,14 @@ def run_decode(args, wl, env, sub=False):
     scores = [torch.empty(L, B, H, dtype=torch.float32, device=dev) for _ in range(n_sets)]
     it = [0]
 
-    dcalls = [binding.prepare_decode_step(ctx.handle, cache, 0, L, Xs[i], KVs[i][0].view(L, B, H, D),
-                                          KVs[i][1].view(L, B, H, D), wl.tau, scores[i]) for i in range(n_sets)]
+    if fp8:
+        Xq = [synth.quantize_e4m3(x.view(L * B, wl.d_model)) for x in Xs]
+        dcalls = [binding.prepare_decode_step_fp8(ctx.handle, cache, 0, L, Xq[i][0].view(L, B, wl.d_model), Xq[i][1].view(L, B),
+                                                  KVs[i][0].view(L, B, H, D), KVs[i][1].view(L, B, H, D), wl.tau, scores[i])
+                  for i in range(n_sets)]
+    else:
+        dcalls = [binding.prepare_decode_step(ctx.handle, cache, 0, L, Xs[i], KVs[i][0].view(L, B, H, D),
+                                              KVs[i][1].view(L, B, H, D), wl.tau, scores[i]) for i in range(n_sets)]
 
     def step():
         dcalls[it[0] % n_sets]()
@@ -585,17 +601,18 @@ def run_decode(args, wl, env, sub=False):
 
     peaks, peak_src = load_peaks()
     row = 2 * D
-    w_bytes = wl.hidden * wl.d_model * 2 + wl.hidden * H * 4 + wl.hidden * 4 + H * 4
-    bytes_layer = (w_bytes + B * wl.d_model * 2 + B * H * 4          # weights, hidden states, scores
+    xb = 1 if fp8 else 2                                               # bytes per element of hidden states and W1
+    w_bytes = wl.hidden * wl.d_model * xb + wl.hidden * H * 4 + wl.hidden * 4 + H * 4 + (wl.hidden * 4 if fp8 else 0)
+    bytes_layer = (w_bytes + B * wl.d_model * xb + (B * 4 if fp8 else 0) + B * H * 4          # weights, hidden states, scores
                    + 2 * B * H * row * 2                               # new K and V rows read and written to the window
                    + B * H * 4 * 2                                     # buffered score read, new score written
                    + kept_exit * B * H * 2 * row * 2)                  # kept exiting rows: window -> page
     achieved = bytes_layer * L / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"],
-                "traffic": NCU_TRAFFIC[wl.name][0] if wl.name in NCU_TRAFFIC and args.layers == 0 else None,
+                "traffic": NCU_TRAFFIC[wl.name][0] if wl.name in NCU_TRAFFIC and args.layers == 0 and not fp8 else None,
                 "traffic_source": (NCU_TRAFFIC[wl.name][1] + " (ncu capture, not measured in this run)")
-                if wl.name in NCU_TRAFFIC and args.layers == 0 else None,
+                if wl.name in NCU_TRAFFIC and args.layers == 0 and not fp8 else None,
                 "kernel": "score_split_kernel (scoring + cache update in one launch)", "peak_source": peak_src,
                 "kernel_ms": ms_per_step, "algorithmic_bytes_per_step": bytes_layer * L}
     config = {"workload": wl.name, "surrogate": wl.surrogate, "d_model": wl.d_model, "hidden": wl.hidden,
@@ -606,12 +623,12 @@ def run_decode(args, wl, env, sub=False):
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": n_warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config, "clocks": clocks,
-            "gpu_launches": int(gpu_launches), "roofline": roofline,
+            "dtype": "e4m3 x e4m3 -> f32 (first layer), bf16 K/V" if fp8 else "bf16", "data": "synthetic", "config": config,
+            "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline,
             "breakdown": {"layer_us": ms_per_step * 1e3 / L, "layer_roofline_us": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
                           "layer_frac_of_roofline": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e3 / (ms_per_step / L),
                           "kept_fraction_of_exiting_tokens": kept_exit}}
-    if rank == 0 and world == 1 and not args.skip_e2e and not sub:
+    if rank == 0 and world == 1 and not args.skip_e2e and not sub and not fp8:
         # End to end: the step's inputs start in pinned host memory and its scores end there; the copies
         # (torch, on the stream of the call) are inside the timed region.
         hX = [x.cpu().pin_memory() for x in Xs[:2]]
@@ -869,7 +886,8 @@ def main():
     ap.add_argument("--kv-layout", default="heads", choices=["heads", "proj"],
                     help="prefill workloads: K/V as [H,T,D] (default) or as the projection writes them, [T,H,D]")
     ap.add_argument("--fp8", action="store_true",
-                    help="prefill workloads with dense-ragged output: hidden states and first-layer weights as E4M3 bytes with scales")
+                    help="hidden states and first-layer weights as E4M3 bytes with scales (prefill and decode workloads); "
+                         "with --attention: cache rows of E4M3 codes with a per-row scale")
     ap.add_argument("--attention", action="store_true",
                     help="decode workload: time the attention over the pruned cache instead of the pruning step")
     ap.add_argument("--skip-live-peak", action="store_true",

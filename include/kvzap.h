@@ -398,6 +398,18 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
                                float *scores_out, void *stream);
 
 /*
+ * The same step with the new tokens' hidden states as E4M3 bytes (layers set with kvzap_set_weights_fp8):
+ *   hidden_e4m3 [layer_end - layer_begin, n_seqs, d_model] bytes, x_scale [layer_end - layer_begin, n_seqs]
+ *   fp32 or NULL (= 1), both on the device; everything else as kvzap_decode_step.
+ * A decode step is bound by reading the first-layer weights once per step; with 8-bit weights that is half
+ * the bytes.  Scores as kvzap_score_fp8 gives them (the two scales multiply the first layer's sum before
+ * the bias), the cache update is the same.
+ */
+kvzap_status kvzap_decode_step_fp8(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                   const void *hidden_e4m3, const float *x_scale, const void *K_new, const void *V_new,
+                                   float tau, float *scores_out, void *stream);
+
+/*
  * Attention of the newest token over the pruned cache (Introduction, Criterion 3;
  * Discussion, "Implementation Challenges": lists of different lengths per head
  * need an attention kernel that takes variable-length paged lists).  For every

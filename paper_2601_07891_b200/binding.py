@@ -74,6 +74,7 @@ SIGNATURES = {
     "kvzap_cache_create": (_i32, [_vp, ctypes.POINTER(_vp), _i32, _i32, _i32, _vp, _vp, _i64, _i32]),
     "kvzap_cache_destroy": (_i32, [_vp]),
     "kvzap_decode_step": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _f32, _vp, _vp]),
+    "kvzap_decode_step_fp8": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp, _vp, _vp, _f32, _vp, _vp]),
     "kvzap_decode_attention": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
     "kvzap_decode_attention_fp8": (_i32, [_vp, _vp, _i32, _i32, _vp, _i32, _f32, _vp, _vp]),
     "kvzap_cache_release_seq": (_i32, [_vp, _i32, _vp]),
@@ -355,6 +356,13 @@ def kvzap_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_ne
                                             _ptr(V_new), tau, _ptr(scores_out), _stream(stream)))
 
 
+def kvzap_decode_step_fp8(handle, cache, layer_begin, layer_end, hidden_e4m3, x_scale, K_new, V_new, tau, scores_out=None,
+                          stream=None):
+    """hidden_e4m3: uint8 [layers, n_seqs, d_model] of E4M3 bytes; x_scale fp32 [layers, n_seqs] or None."""
+    _check(handle, load().kvzap_decode_step_fp8(handle, cache, layer_begin, layer_end, _ptr(hidden_e4m3), _ptr(x_scale),
+                                                _ptr(K_new), _ptr(V_new), tau, _ptr(scores_out), _stream(stream)))
+
+
 def kvzap_cache_release_seq(handle, cache, seq, stream=None):
     _check(handle, load().kvzap_cache_release_seq(cache, seq, _stream(stream)))
 
@@ -521,6 +529,13 @@ def prepare_decode_step(handle, cache, layer_begin, layer_end, hidden, K_new, V_
     args = (handle, cache, layer_begin, layer_end, _ptr(hidden), _ptr(K_new), _ptr(V_new), tau, _ptr(scores_out),
             _stream(stream))
     return PreparedCall("kvzap_decode_step", handle, args, (hidden, K_new, V_new, scores_out))
+
+
+def prepare_decode_step_fp8(handle, cache, layer_begin, layer_end, hidden_e4m3, x_scale, K_new, V_new, tau, scores_out=None,
+                            stream=None) -> PreparedCall:
+    args = (handle, cache, layer_begin, layer_end, _ptr(hidden_e4m3), _ptr(x_scale), _ptr(K_new), _ptr(V_new), tau,
+            _ptr(scores_out), _stream(stream))
+    return PreparedCall("kvzap_decode_step_fp8", handle, args, (hidden_e4m3, x_scale, K_new, V_new, scores_out))
 
 
 KERNEL_IDS = {"score": 0, "mask": 1, "scan": 2, "compact": 3, "decode_update": 4, "attention": 5}

@@ -55,6 +55,8 @@ struct kvzap_ctx {
     int split_n = 0, split_k = 1, split_stages = 0, split_tmem_cols = 0;   // cluster = split_n * split_k CTAs
     uint32_t split_smem = 0;
     CUtensorMap split_tmap_w;
+    CUtensorMap split_tmap_w8;           // the 8-bit copy of the weights, same slices (set by kvzap_set_weights_fp8)
+    bool split8_ok = false;
     // the same kernel with eight CTAs per tile (4 slices x 2 halves of K) for launches of even fewer tiles
     // (a short prompt or a chunk of one): set when the shape allows it
     int wide_n = 0, wide_k = 1, wide_stages = 0, wide_tmem_cols = 0;
@@ -496,7 +498,8 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
                                  float *scores, uint32_t *maskbits, const int32_t *cu_seqlens, int32_t n_seqs,
                                  float tau, int32_t w, cudaStream_t stream, int32_t window_keep = 1,
                                  const DecodeFuse *fuse = nullptr, bool *fused = nullptr, bool fuse_chain = false,
-                                 const CompactArgs *compact = nullptr, bool *compacted = nullptr)
+                                 const CompactArgs *compact = nullptr, bool *compacted = nullptr,
+                                 bool fp8 = false, const float *x_scale = nullptr)
 {
     if (fused) *fused = false;
     if (compacted) *compacted = false;
@@ -521,18 +524,24 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // ... and with the K split left out (two CTAs per tile, each a slice of the hidden units over the whole K
     // range) the same kernel serves launches of up to half as many tiles as there are SMs, where CTA pairs
     // would leave most SMs idle.
-    const bool slices_only = ctx->split_n == 2 && ctx->split_k == 2 && fuse == nullptr &&
+    const bool slices_only = ctx->split_n == 2 && ctx->split_k == 2 && fuse == nullptr && !fp8 &&
                              blocks_per_layer * n_layers * 4 > ctx->sm_count && blocks_per_layer * n_layers * 2 <= ctx->sm_count;
+    if (fp8 && !(ctx->split8_ok && blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count))
+        return fail(ctx, KVZAP_ERR_UNSUPPORTED, "8-bit few-token scoring: this shape has no four-CTA layout");
     if (ctx->split_n > 0 && (slices_only || blocks_per_layer * n_layers * ctx->split_n * ctx->split_k <= ctx->sm_count)) {
         // eight CTAs per tile when even those fit (not for the fused decode step, which is laid out for four)
-        const bool wide = ctx->wide_n > 0 && fuse == nullptr &&
+        const bool wide = ctx->wide_n > 0 && fuse == nullptr && !fp8 &&
                           blocks_per_layer * n_layers * ctx->wide_n * ctx->wide_k <= ctx->sm_count;
         const int split_n = wide ? ctx->wide_n : ctx->split_n, split_k = wide ? ctx->wide_k : (slices_only ? 1 : ctx->split_k);
         CUtensorMap tmap_x;
-        kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
+        kvzap_status st = fp8 ? make_tmap8(ctx, &tmap_x, hidden, static_cast<uint64_t>(n_tokens), static_cast<uint64_t>(c.d_model),
+                                           kTileM, static_cast<uint64_t>(n_layers), false)
+                              : hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
         if (st != KVZAP_OK) return st;
         ScoreParams p;
         memset(&p, 0, sizeof p);
+        p.x_scale = x_scale;
+        p.w1_scale = ctx->w1_scale_all;
         p.n_tokens = n_tokens;
         p.n_tiles = static_cast<int32_t>(blocks_per_layer * n_layers);
         p.tiles_per_layer = static_cast<int32_t>(blocks_per_layer);
@@ -598,8 +607,11 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
             cudaLaunchAttribute attrs[2];
             make_launch(&cfg, attrs, dim3(static_cast<unsigned>(p.n_tiles * n_ctas)), dim3(kScoreThreads),
                         wide ? ctx->wide_smem : ctx->split_smem, stream, early, split_k);
-            KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel, tmap_x, wide ? ctx->wide_tmap_w : ctx->split_tmap_w, p,
-                                               split_n, split_k, f));
+            if (fp8)
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel<true>, tmap_x, ctx->split_tmap_w8, p, split_n, split_k, f));
+            else
+                KVZAP_CUDA(ctx, cudaLaunchKernelEx(&cfg, score_split_kernel<false>, tmap_x, wide ? ctx->wide_tmap_w : ctx->split_tmap_w, p,
+                                                   split_n, split_k, f));
         }
         ctx->launches += 1;
         return KVZAP_OK;
@@ -1179,7 +1191,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
     CREATE_CUDA(cudaFuncSetAttribute(decode_update_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
                                      static_cast<int>(cudaSharedmemCarveoutMaxShared)));
     if (c.hidden > 0)
-        CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+        CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                          static_cast<int>(cudaSharedmemCarveoutMaxShared)));
     if (c.hidden > 0) {
         CREATE_CUDA(cudaFuncSetAttribute(score_kernel<true, false>, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -1234,7 +1246,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
             ctx->split_stages = stages;
             ctx->split_smem = split_smem_layout(ns, stages, 4).total + 1024;
             ctx->split_tmem_cols = next_pow2(ns);
-            CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(ctx->split_smem)));
             if (make_tmap_w(ctx, &ctx->split_tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
                             static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns)) == KVZAP_OK) {
@@ -1253,7 +1265,7 @@ kvzap_status kvzap_create(kvzap_ctx **out, const kvzap_config *cfg)
                 ctx->wide_smem = split_smem_layout(ns8, st8, 8).total + 1024;
                 ctx->wide_tmem_cols = next_pow2(ns8);
                 if (ctx->wide_smem > ctx->split_smem)
-                    CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                    CREATE_CUDA(cudaFuncSetAttribute(score_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      static_cast<int>(ctx->wide_smem)));
                 if (make_tmap_w(ctx, &ctx->wide_tmap_w, ctx->w1_all, static_cast<uint64_t>(c.n_layers) * ctx->w1_rows,
                                 static_cast<uint64_t>(c.d_model / kBlockK), static_cast<uint32_t>(ns8)) == KVZAP_OK) {
@@ -1398,6 +1410,16 @@ kvzap_status kvzap_set_weights_fp8(kvzap_ctx *ctx, int32_t layer, const void *W1
             kvzap_status st = make_tmap8(ctx, &ctx->tmap_w8[mode], ctx->w1_fp8_all, static_cast<uint64_t>(rows_total),
                                          static_cast<uint64_t>(c.d_model), static_cast<uint32_t>(ctx->sched[mode].chunk_n / (mode + 1)), 0, true);
             if (st != KVZAP_OK) return st;
+        }
+        if (c.hidden > 0 && ctx->split_n > 0 && (c.d_model / 128) % ctx->split_k == 0) {
+            // the few-token layout (a decode step): the same slices of hidden units, K blocks of 128 codes
+            if (make_tmap8(ctx, &ctx->split_tmap_w8, ctx->w1_fp8_all, static_cast<uint64_t>(rows_total), static_cast<uint64_t>(c.d_model),
+                           static_cast<uint32_t>(c.hidden / ctx->split_n), 0, true) == KVZAP_OK &&
+                cudaFuncSetAttribute(score_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(ctx->split_smem)) == cudaSuccess &&
+                cudaFuncSetAttribute(score_split_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                     static_cast<int>(cudaSharedmemCarveoutMaxShared)) == cudaSuccess)
+                ctx->split8_ok = true;
         }
         if (c.hidden > 0) {
             KVZAP_CUDA(ctx, cudaFuncSetAttribute(score_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(ctx->sched[0].smem)));
@@ -2118,11 +2140,11 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache)
     return KVZAP_OK;
 }
 
-kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
-                               const void *hidden, const void *K_new, const void *V_new, float tau,
-                               float *scores_out, void *stream_)
+static kvzap_status decode_step_impl(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                     const void *hidden, const float *x_scale, const void *K_new, const void *V_new, float tau,
+                                     float *scores_out, void *stream_, bool fp8)
 {
-    NvtxRange nvtx_range("kvzap_decode_step");
+    NvtxRange nvtx_range(fp8 ? "kvzap_decode_step_fp8" : "kvzap_decode_step");
     if (!ctx || !cache || cache->ctx != ctx) return KVZAP_ERR_INVALID_ARG;
     begin_op(ctx);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -2130,7 +2152,8 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
     if (layer_begin < 0 || layer_end > c.n_layers || layer_begin >= layer_end)
         return fail(ctx, KVZAP_ERR_INVALID_ARG, "decode: layer range [%d, %d) invalid", layer_begin, layer_end);
     for (int l = layer_begin; l < layer_end; ++l)
-        if (!ctx->layer_set[l]) return fail(ctx, KVZAP_ERR_STATE, "layer %d has no weights", l);
+        if (fp8 ? !ctx->layer_fp8[l] : !ctx->layer_set[l])
+            return fail(ctx, KVZAP_ERR_STATE, fp8 ? "layer %d has no 8-bit weights (kvzap_set_weights_fp8)" : "layer %d has no weights", l);
     if (!hidden || !K_new || !V_new || !aligned16(hidden) || !aligned16(K_new) || !aligned16(V_new))
         return fail(ctx, KVZAP_ERR_INVALID_ARG, "decode: hidden, K_new, V_new must be non-NULL, 16-byte aligned");
     DeviceGuard guard(c.device);
@@ -2160,8 +2183,18 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
     bool fused = false;
     // the call just before this one was a fused step on this cache: the two may overlap
     const bool chain = ctx->fused_cache == cache && ctx->fused_seq + 1 == ctx->op_seq;
-    kvzap_status st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
-                                   0.0f, 0, stream, 1, can_fuse ? &fuse : nullptr, &fused, chain);
+    kvzap_status st = KVZAP_OK;
+    const int64_t step_tiles = (static_cast<int64_t>(cache->v.n_seqs) + kTileM - 1) / kTileM * n_layers;
+    if (fp8 && !(c.hidden > 0 && ctx->split8_ok && step_tiles * ctx->split_n * ctx->split_k <= ctx->sm_count)) {
+        // no few-token layout for this shape: layer after layer through the prefill scoring kernel
+        for (int l = 0; l < n_layers && st == KVZAP_OK; ++l)
+            st = launch_score_fp8(ctx, layer_begin + l, static_cast<const uint8_t *>(hidden) + static_cast<size_t>(l) * cache->v.n_seqs * c.d_model,
+                                  x_scale ? x_scale + static_cast<size_t>(l) * cache->v.n_seqs : nullptr, cache->v.n_seqs,
+                                  scores + static_cast<size_t>(l) * cache->v.n_seqs * c.n_kv_heads, nullptr, nullptr, 1, 0.0f, 0, stream);
+    } else {
+        st = launch_score(ctx, layer_begin, n_layers, hidden, cache->v.n_seqs, scores, nullptr, nullptr, 1,
+                          0.0f, 0, stream, 1, can_fuse ? &fuse : nullptr, &fused, chain, nullptr, nullptr, fp8, x_scale);
+    }
     if (st != KVZAP_OK) return st;
     if (fused) {
         for (int l = layer_begin; l < layer_end; ++l) cache->steps_done[l] += 1;
@@ -2184,6 +2217,20 @@ kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer
     }
     ctx->launches += 1;
     return KVZAP_OK;
+}
+
+kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                               const void *hidden, const void *K_new, const void *V_new, float tau,
+                               float *scores_out, void *stream_)
+{
+    return decode_step_impl(ctx, cache, layer_begin, layer_end, hidden, nullptr, K_new, V_new, tau, scores_out, stream_, false);
+}
+
+kvzap_status kvzap_decode_step_fp8(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
+                                   const void *hidden_e4m3, const float *x_scale, const void *K_new, const void *V_new,
+                                   float tau, float *scores_out, void *stream_)
+{
+    return decode_step_impl(ctx, cache, layer_begin, layer_end, hidden_e4m3, x_scale, K_new, V_new, tau, scores_out, stream_, true);
 }
 
 static kvzap_status attention_impl(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,

@@ -45,7 +45,7 @@ struct DecodeFuse {
 };
 
 struct SplitSmemLayout {
-    uint32_t stage_bytes, stages_end, w2s, b1s, part, xpart, bars, total;
+    uint32_t stage_bytes, stages_end, w2s, b1s, w1s, part, xpart, bars, total;
 };
 __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stages, int n_split)
 {
@@ -54,7 +54,8 @@ __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stage
     L.stages_end = L.stage_bytes * n_stages;
     L.w2s = L.stages_end;
     L.b1s = L.w2s + static_cast<uint32_t>(ns) * kMaxHeads * 4;
-    L.part = L.b1s + static_cast<uint32_t>(ns) * 4;
+    L.w1s = L.b1s + static_cast<uint32_t>(ns) * 4;            // first-layer row scales (8-bit inputs)
+    L.part = L.w1s + static_cast<uint32_t>(ns) * 4;
     L.xpart = L.part + kTileM * kMaxHeads * 4;
     L.bars = L.xpart + static_cast<uint32_t>(n_split) * kTileM * kMaxHeads * 4;
     L.total = L.bars + 256;
@@ -64,10 +65,14 @@ __host__ __device__ inline SplitSmemLayout split_smem_layout(int ns, int n_stage
 // p.group_w = p.chunk_n = Ns (the MMA's N); p.n_chunks = 1; p.acc_bufs = 1; p.n_tiles = 128-token tiles
 // over all layers of the call; cluster dimension k_split, gridDim.x = n_split * k_split * p.n_tiles.
 // A CTA ends up owning Ns / k_split hidden units: xpart and the W2 / b1 slices are sized for those.
+// kFp8: hidden states and W1 are E4M3 bytes (K blocks of 128 codes, tcgen05.mma kind::f8f6f4); the scales
+// x_scale[token] * w1_scale[hidden unit] multiply the summed pre-activation before the bias.
+template <bool kFp8>
 __global__ void __maxnreg__(128)
 score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                    const ScoreParams p, const int n_split, const int k_split, const DecodeFuse f)
 {
+    constexpr int kElems = kFp8 ? 2 * kBlockK : kBlockK;         // elements per 128-byte K block
     __shared__ int64_t fuse_dst[256];       // fused decode step: page row of the evicted token (-1 = dropped)
     __shared__ int64_t fuse_ring[256];      //                     ring row of the list's current slot (-1 = no list)
     extern __shared__ uint8_t smem_raw[];
@@ -82,6 +87,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     ulonglong2 *w2p = reinterpret_cast<ulonglong2 *>(smem + L.w2s);
     float *w2f = reinterpret_cast<float *>(smem + L.w2s);
     float *b1s = reinterpret_cast<float *>(smem + L.b1s);
+    float *w1s = reinterpret_cast<float *>(smem + L.w1s);
     float *part = reinterpret_cast<float *>(smem + L.part);
     float *xpart = reinterpret_cast<float *>(smem + L.xpart);
     const uint32_t bars = smem_base + L.bars;
@@ -125,7 +131,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         prefetch_tensormap(&tmap_x);
         prefetch_tensormap(&tmap_w);
     }
-    const int k_blocks = p.d_model / kBlockK / k_split;  // K blocks of this CTA
+    const int k_blocks = p.d_model / kElems / k_split;   // K blocks of this CTA
     const int kb_first = kh * k_blocks;
     const uint64_t pol_x = l2_policy_evict_last();        // the other CTAs of the cluster read the same X tile
     const uint64_t pol_w = l2_policy_evict_first();       // every W1 byte is read once per step
@@ -141,7 +147,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                 const uint32_t sa = smem_base + kb * L.stage_bytes;
                 mbar_arrive_expect_tx(bar_full + 8 * kb, L.stage_bytes);
                 tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * kb, 0, w_row, kb_first + kb, pol_w);
-                tma_load_3d(sa, &tmap_x, bar_full + 8 * kb, (kb_first + kb) * kBlockK, row0, l_rel, pol_x);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * kb, (kb_first + kb) * kElems, row0, l_rel, pol_x);
             }
         }
         __syncwarp();
@@ -170,7 +176,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             if (elected) {
                 mbar_arrive_expect_tx(bar_full + 8 * st, L.stage_bytes);
                 tma_load_3d(sa + kATileBytes, &tmap_w, bar_full + 8 * st, 0, w_row, kb_first + kb, pol_w);
-                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, (kb_first + kb) * kBlockK, row0, l_rel, pol_x);
+                tma_load_3d(sa, &tmap_x, bar_full + 8 * st, (kb_first + kb) * kElems, row0, l_rel, pol_x);
             }
             __syncwarp();
             sa += L.stage_bytes;
@@ -183,7 +189,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        const uint32_t idesc = umma_idesc_bf16_f32(kTileM, static_cast<uint32_t>(ns));
+        const uint32_t idesc = kFp8 ? umma_idesc_e4m3_f32(kTileM, static_cast<uint32_t>(ns))
+                                    : umma_idesc_bf16_f32(kTileM, static_cast<uint32_t>(ns));
         const uint64_t desc0 = umma_desc_k_major_sw128(smem_base);
         const uint32_t desc_hi = static_cast<uint32_t>(desc0 >> 32);
         const uint32_t desc_lo0 = static_cast<uint32_t>(desc0);
@@ -198,7 +205,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
             tc_fence_after_sync();
             if (elected) {
-                issue_k_block<false, 1>(tmem_base, a_lo, a_lo + (kATileBytes >> 4), desc_hi, 0, 0, idesc, kb == 0);
+                issue_k_block<false, 1, kFp8>(tmem_base, a_lo, a_lo + (kATileBytes >> 4), desc_hi, 0, 0, idesc, kb == 0);
                 umma_commit(bar_empty + 8 * st);
             }
             __syncwarp();
@@ -232,6 +239,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             w2f[(((j >> 1) * kMaxHeads + h) << 1) + (j & 1)] = __ldg(w2g + i);
         }
         for (int i = etid; i < own_n; i += 256) b1s[i] = __ldg(b1g + i);
+        if constexpr (kFp8)
+            for (int i = etid; i < own_n; i += 256) w1s[i] = __ldg(p.w1_scale + static_cast<int64_t>(layer) * p.n_hidden + j_first + i);
         named_barrier_sync(1, 256);
         if (f.enabled) {
             // ---- the cache update of this CTA's lists, under the MMAs
@@ -366,6 +375,13 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         if (ok) {
             // the first warp of a lane quarter takes the 16-column chunks 0, 2, 4, ..., the second the odd ones
             uint32_t ra[16], rb[16];
+            uint64_t sx2 = 0ull;                                   // 8-bit inputs: this row's token scale, twice
+            if constexpr (kFp8) {
+                float sx = 1.0f;
+                if (p.x_scale != nullptr && row0 + row < p.n_tokens)
+                    sx = __ldg(p.x_scale + static_cast<int64_t>(l_rel) * p.n_tokens + row0 + row);
+                sx2 = f2_pack(sx, sx);
+            }
             int c = hsel;
             if (c < n16) tmem_ld_x16(t_row + own_c0 + c * 16, ra);
             while (c < n16) {
@@ -382,7 +398,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         ra[4 * i + 3] = __float_as_uint(__uint_as_float(ra[4 * i + 3]) + o.w);
                     }
                 }
-                mlp_columns<16>(ra, c * 16, b1s, w2p, acc);
+                if constexpr (kFp8) mlp_columns_scaled<16>(ra, c * 16, b1s, w1s, sx2, w2p, acc);
+                else mlp_columns<16>(ra, c * 16, b1s, w2p, acc);
                 c += 2;
                 if (c < n16) {
                     tmem_wait_ld();
@@ -398,7 +415,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                             rb[4 * i + 3] = __float_as_uint(__uint_as_float(rb[4 * i + 3]) + o.w);
                         }
                     }
-                    mlp_columns<16>(rb, c * 16, b1s, w2p, acc);
+                    if constexpr (kFp8) mlp_columns_scaled<16>(rb, c * 16, b1s, w1s, sx2, w2p, acc);
+                    else mlp_columns<16>(rb, c * 16, b1s, w2p, acc);
                     c += 2;
                 }
             }

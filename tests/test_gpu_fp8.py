@@ -131,6 +131,81 @@ def test_fp8_fused_paged_prefill_matches_oracle(binding, oracle, seq_lens, hidde
     ctx.close()
 
 
+def _export(binding, ctx, cache, b, l, h, cap, D):
+    K_out = torch.zeros(cap, D, dtype=torch.bfloat16, device="cuda")
+    V_out = torch.zeros(cap, D, dtype=torch.bfloat16, device="cuda")
+    n = torch.zeros(1, dtype=torch.int32, device="cuda")
+    binding.kvzap_cache_export(ctx.handle, cache, b, l, h, K_out, V_out, n)
+    torch.cuda.synchronize()
+    n = int(n.item())
+    return synth.bits(K_out)[:n], synth.bits(V_out)[:n], n
+
+
+@pytest.mark.parametrize("d_model,hidden,w,P,B,L", [
+    (256, 128, 8, 4, 3, 2),       # the one-launch step (four CTAs per tile, two halves of K)
+    (512, 512, 16, 16, 5, 3),     # the same with 256 hidden units per slice
+    (256, 64, 0, 4, 2, 2),        # no window: scoring launch, then the general update
+    (256, 0, 5, 16, 2, 1),        # KVzap-Linear: layer after layer through the prefill kernel, then the update
+    (256, 128, 8, 4, 130, 1),     # two token tiles per layer
+])
+def test_fp8_decode_steps_match_decode_oracle(binding, oracle, d_model, hidden, w, P, B, L):
+    """kvzap_decode_step_fp8: scores against the 8-bit oracle, eviction decisions and list contents bit for bit
+    against the decode oracle fed the GPU's scores."""
+    H, D, tau, n_steps = 8, 64, 0.1, 30 if B < 100 else 14
+    ctx = binding.Kvzap(d_model, hidden, H, D, L, max_tokens=max(B, 128), max_seqs=1)
+    cases = []
+    for l in range(L):
+        case = _fp8_case(d_model, hidden, H, 1, seed=90 + l)        # weights of layer l (its one-token input is not used)
+        cases.append(case)
+        _, _, W18, sw, b1, W2, b2 = case
+        binding.kvzap_set_weights_fp8(ctx.handle, l, W18.cuda(), sw.cuda(), b1.cuda(),
+                                      parity.dev(W2) if W2 is not None else None, parity.dev(b2) if b2 is not None else None)
+    max_pages = n_steps // P + 2
+    n_pool = B * L * H * max_pages
+    K_pool = torch.zeros(n_pool, P, D, dtype=torch.bfloat16, device="cuda")
+    V_pool = torch.zeros_like(K_pool)
+    cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
+    dec = oracle.DecodeOracle(B, L, H, D, w)
+    worst = 0.0
+    for step in range(n_steps):
+        X = synth.hidden_states(L * B, d_model, seed=1500 + step)
+        X8, sx = synth.quantize_e4m3(X)
+        if step % 3 == 2:
+            sx = None                                          # NULL scales = 1
+        K_new, V_new = synth.keys_values(L * B, H, D, seed=2500 + step)
+        K_new, V_new = K_new.view(L, B, H, D), V_new.view(L, B, H, D)
+        scores = torch.empty(L, B, H, dtype=torch.float32, device="cuda")
+        binding.kvzap_decode_step_fp8(ctx.handle, cache, 0, L, X8.cuda().view(L, B, d_model),
+                                      sx.cuda().view(L, B) if sx is not None else None, parity.dev(K_new), parity.dev(V_new),
+                                      tau, scores)
+        torch.cuda.synchronize()
+        s = scores.cpu().numpy()
+        X8n = X8.numpy().reshape(L, B, d_model)
+        sxn = sx.numpy().reshape(L, B) if sx is not None else np.ones((L, B), dtype=np.float32)
+        for l in range(L):
+            _, _, W18, sw, b1, W2, b2 = cases[l]
+            if hidden:
+                want = oracle.score_mlp_fp8(X8n[l], sxn[l], W18.numpy(), sw.numpy(), b1.numpy(), synth.bits(W2), b2.numpy())
+            else:
+                want = oracle.score_linear_fp8(X8n[l], sxn[l], W18.numpy(), sw.numpy(), b1.numpy())
+            worst = max(worst, float(np.abs(s[l] - want).max()))
+            Kb, Vb = synth.bits(K_new[l]), synth.bits(V_new[l])
+            for b in range(B):
+                dec.append(b, l, s[l, b], Kb[b], Vb[b], tau)
+    assert worst <= parity.SCORE_ATOL, worst
+    assert ctx.poll_status() == 0
+    lists = [(b, l, h) for b in range(B) for l in range(L) for h in range(H)] if B < 100 else \
+            [(0, 0, 0), (127, 0, 3), (129, 0, 7), (64, 0, 5)]
+    for b, l, h in lists:
+        _pos, Kd, Vd = dec.logical(b, l, h)
+        Kg, Vg, n = _export(binding, ctx, cache, b, l, h, n_steps + 1, D)
+        assert n == len(Kd), (b, l, h)
+        np.testing.assert_array_equal(Kg, Kd)
+        np.testing.assert_array_equal(Vg, Vd)
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
+
+
 def test_fp8_needs_d_model_multiple_of_128_and_its_own_weights(binding):
     ctx = binding.Kvzap(192, 0, 8, 64, 1, max_tokens=64)
     W = torch.zeros(8, 192, dtype=torch.uint8, device="cuda")
