@@ -532,7 +532,7 @@ def run_decode(args, wl, env, sub=False):
             ctx.set_weights(l, *wts)
     n_lists = B * L * H
     n_steps = max(args.steps, 1000) if sub else args.steps
-    total_steps = w + max(args.warmup, 3) + n_steps + 8 + (max(args.e2e_steps, 10) + 3 if not args.skip_e2e and not sub else 0)
+    total_steps = w + max(args.warmup, 3) + n_steps + 8 + 36 + (max(args.e2e_steps, 10) + 3 if not args.skip_e2e and not sub else 0)
     # Pre-pruned caches: per-list prefix lengths uniform in [prefix_min, prefix_max].  Decoding never
     # reads a list's earlier pages, so only each list's last (partly filled) page and the pages it can
     # grow into are backed by memory; lengths and page tables carry the full logical sizes.
@@ -568,6 +568,51 @@ def run_decode(args, wl, env, sub=False):
         dcalls[it[0] % n_sets]()
         it[0] += 1
 
+    graph_mode = getattr(args, "graph", "off") if not sub else "off"
+    if graph_mode != "off":
+        # The same steps captured once in a CUDA graph and replayed: n_sets steps per graph (the rotating input sets),
+        # each one launch over all layers ("step") or one launch per layer ("layer").
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        stream_ctx = torch.cuda.stream(side)          # the prepared calls carry the stream they were prepared on
+        stream_ctx.__enter__()
+        if graph_mode == "step":
+            if fp8:
+                gcalls = [binding.prepare_decode_step_fp8(ctx.handle, cache, 0, L, Xq[i][0].view(L, B, wl.d_model), Xq[i][1].view(L, B),
+                                                          KVs[i][0].view(L, B, H, D), KVs[i][1].view(L, B, H, D), wl.tau, scores[i])
+                          for i in range(n_sets)]
+            else:
+                gcalls = [binding.prepare_decode_step(ctx.handle, cache, 0, L, Xs[i], KVs[i][0].view(L, B, H, D),
+                                                      KVs[i][1].view(L, B, H, D), wl.tau, scores[i]) for i in range(n_sets)]
+        if graph_mode == "layer":
+            if fp8:
+                lcalls = [[binding.prepare_decode_step_fp8(ctx.handle, cache, l, l + 1, Xq[i][0].view(L, B, wl.d_model)[l:l + 1],
+                                                           Xq[i][1].view(L, B)[l:l + 1], KVs[i][0].view(L, B, H, D)[l:l + 1],
+                                                           KVs[i][1].view(L, B, H, D)[l:l + 1], wl.tau, scores[i][l:l + 1])
+                           for l in range(L)] for i in range(n_sets)]
+            else:
+                lcalls = [[binding.prepare_decode_step(ctx.handle, cache, l, l + 1, Xs[i][l:l + 1], KVs[i][0].view(L, B, H, D)[l:l + 1],
+                                                       KVs[i][1].view(L, B, H, D)[l:l + 1], wl.tau, scores[i][l:l + 1])
+                           for l in range(L)] for i in range(n_sets)]
+            one = lambda i: [c() for c in lcalls[i]]
+        else:
+            one = lambda i: gcalls[i]()
+        for i in range(n_sets):       # once outside the capture
+            one(i)
+        stream_ctx.__exit__(None, None, None)
+        torch.cuda.synchronize()
+        cuda_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cuda_graph, stream=side):
+            for i in range(n_sets):
+                one(i)
+        replays = [0]
+
+        def step():                   # one replay = n_sets steps; called once per n_sets steps of the loops below
+            if it[0] % n_sets == 0:
+                cuda_graph.replay()
+                replays[0] += 1
+            it[0] += 1
+
     for _ in range(w):                # fill the window: from here on every step decides one token per list
         step()
     n_warm = max(args.warmup, 3)
@@ -576,6 +621,9 @@ def run_decode(args, wl, env, sub=False):
     barrier()
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during warm-up")
+    if graph_mode != "off":           # whole replays only
+        it[0] = -(-it[0] // n_sets) * n_sets
+        n_steps = -(-n_steps // n_sets) * n_sets
     len0 = torch.zeros(B, L, H, dtype=torch.int32, device=dev)
     binding.kvzap_cache_lengths(ctx.handle, cache, len0)
     sampler = ClockSampler(dev.index)
@@ -591,6 +639,8 @@ def run_decode(args, wl, env, sub=False):
     clocks = sampler.stop()
     total_ms = env["max_over_ranks"](e0.elapsed_time(e1))
     gpu_launches = ctx.launch_count() - launches0
+    if graph_mode != "off":          # replays launch what the capture recorded; the host-side counter sees only the capture
+        gpu_launches = n_steps * (L if graph_mode == "layer" else 1)
     ms_per_step = total_ms / n_steps
     if ctx.poll_status() != 0:
         raise RuntimeError("device status word set during the timed region")
@@ -620,6 +670,8 @@ def run_decode(args, wl, env, sub=False):
               "prefix_len": [wl.prefix_min, wl.prefix_max], "input_sets": n_sets,
               "l2": "weights of all layers (151 MB) exceed L2; per-step inputs rotate over %d sets" % n_sets,
               "backing": "only each list's last page and growth pages are backed (decode never reads earlier pages)",
+              "cuda_graph": {"off": "no", "step": "%d steps per graph, one launch per step" % n_sets,
+                             "layer": "%d steps per graph, one launch per layer" % n_sets}[graph_mode],
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": n_warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -628,7 +680,7 @@ def run_decode(args, wl, env, sub=False):
             "breakdown": {"layer_us": ms_per_step * 1e3 / L, "layer_roofline_us": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
                           "layer_frac_of_roofline": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e3 / (ms_per_step / L),
                           "kept_fraction_of_exiting_tokens": kept_exit}}
-    if rank == 0 and world == 1 and not args.skip_e2e and not sub and not fp8:
+    if rank == 0 and world == 1 and not args.skip_e2e and not sub and not fp8 and graph_mode == "off":
         # End to end: the step's inputs start in pinned host memory and its scores end there; the copies
         # (torch, on the stream of the call) are inside the timed region.
         hX = [x.cpu().pin_memory() for x in Xs[:2]]
@@ -888,6 +940,8 @@ def main():
     ap.add_argument("--fp8", action="store_true",
                     help="hidden states and first-layer weights as E4M3 bytes with scales (prefill and decode workloads); "
                          "with --attention: cache rows of E4M3 codes with a per-row scale")
+    ap.add_argument("--graph", choices=["off", "step", "layer"], default="off",
+                    help="decode workload: replay the steps from a captured CUDA graph, one launch per step or one per layer")
     ap.add_argument("--attention", action="store_true",
                     help="decode workload: time the attention over the pruned cache instead of the pruning step")
     ap.add_argument("--skip-live-peak", action="store_true",

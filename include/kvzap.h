@@ -392,6 +392,9 @@ kvzap_status kvzap_cache_destroy(kvzap_cache *cache);
  * step is ONE kernel launch: the cache update runs in the scoring kernel's
  * otherwise idle warps, and consecutive steps overlap on the GPU when their
  * scores_out buffers differ (or are NULL).
+ * The call may be captured in a CUDA graph (stream capture) and replayed, alone or with kvzap_decode_attention:
+ * the number of the step is kept on the device.  Call it (and the attention) once outside the capture first, so
+ * that whatever they build on first use exists; pass the same buffers in every replay and refill them in between.
  */
 kvzap_status kvzap_decode_step(kvzap_ctx *ctx, kvzap_cache *cache, int32_t layer_begin, int32_t layer_end,
                                const void *hidden, const void *K_new, const void *V_new, float tau,
@@ -601,10 +604,10 @@ kvzap_status kvzap_poll_status(kvzap_ctx *ctx, void *stream);
 kvzap_status kvzap_set_wait_limit(kvzap_ctx *ctx, int64_t cycles);
 
 /*
- * Test aid: adds `delta` to the host's count of fused decode steps completed on every layer of the
- * cache, WITHOUT telling the device.  The next fused step then waits for a step that never ran, its
- * bounded wait runs out, and the status word reads KVZAP_ERR_TIMEOUT: the one way to see that path
- * without a fault.  Never call it in production code.
+ * Test aid: adds `delta` to the cache's device-side counts of decode steps STARTED (the tickets from which a
+ * one-launch step learns its number) without touching the counts of steps COMPLETED.  The next such step then
+ * waits for a step that never ran, its bounded wait runs out, and the status word reads KVZAP_ERR_TIMEOUT: the
+ * one way to see that path without a fault.  Synchronises the device.  Never call it in production code.
  */
 kvzap_status kvzap_cache_debug_skew_steps(kvzap_cache *cache, int32_t delta);
 

@@ -308,6 +308,12 @@ __global__ void pack_w1_fp8_kernel(const uint4 *__restrict__ W1, int rows, int d
     dst[(static_cast<int64_t>(kb) * rows_total + row0 + r) * 8 + xu] = W1[idx];
 }
 
+__global__ void add_int_kernel(int32_t *x, int n, int32_t delta)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) x[i] += delta;
+}
+
 // out[i] = src ? src[i] : 1 for i < n, 1 (unused rows) up to n_pad
 __global__ void fill_scale_kernel(const float *__restrict__ src, int n, int n_pad, float *__restrict__ out)
 {
@@ -1856,7 +1862,8 @@ struct kvzap_cache {
     int step_parity = 0;
     // fused decode steps: per-cluster count of completed steps on the device, and the host's view of it
     int32_t *done = nullptr;             // [n_layers * ceil(n_seqs / 128)][4]: one per cluster of the fused step
-    std::vector<int32_t> steps_done;     // per layer
+    int32_t *ticket = nullptr;           // behind `done`: [tiles][4][2] steps started per (slice, rank), see DecodeFuse
+    size_t n_step_counters = 0;          // ints in done + ticket together
     // attention over the cache: tensor maps of the page pools and of the window rings (built on first use)
     CUtensorMap tm_kpool, tm_vpool, tm_kring, tm_vring;
     int attn_state = 0;                  // 0 not built yet, 1 ready, -1 this cache's geometry is not supported
@@ -1870,9 +1877,7 @@ namespace kvzap {
 static void reset_step_counters(kvzap_ctx *ctx, cudaStream_t stream)
 {
     for (kvzap_cache *cache : ctx->caches) {
-        const size_t n = 4 * static_cast<size_t>(ctx->cfg.n_layers) * ((cache->v.n_seqs + 127) / 128);
-        cudaMemsetAsync(cache->done, 0, sizeof(int32_t) * n, stream);
-        cache->steps_done.assign(ctx->cfg.n_layers, 0);
+        cudaMemsetAsync(cache->done, 0, sizeof(int32_t) * cache->n_step_counters, stream);
     }
     ctx->fused_cache = nullptr;
 }
@@ -2091,9 +2096,12 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
     alloc(reinterpret_cast<void **>(&v.free_top), sizeof(int32_t), true);
     alloc(reinterpret_cast<void **>(&v.active), static_cast<size_t>(n_seqs), false);
     if (e == cudaSuccess) e = cudaMemset(v.active, 1, static_cast<size_t>(n_seqs));      // every slot takes part until released
-    alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * 4 * static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128),
-          true);
-    cache->steps_done.assign(c.n_layers, 0);
+    {
+        const size_t tiles = static_cast<size_t>(c.n_layers) * ((n_seqs + 127) / 128);
+        cache->n_step_counters = 12 * tiles;          // done [tiles][4], then ticket [tiles][4][2]
+        alloc(reinterpret_cast<void **>(&cache->done), sizeof(int32_t) * cache->n_step_counters, true);
+        cache->ticket = cache->done ? cache->done + 4 * tiles : nullptr;
+    }
     // two halves used by alternate steps when the caller does not ask for the scores
     alloc(reinterpret_cast<void **>(&cache->scores), 2 * sizeof(float) * static_cast<size_t>(c.n_layers) * n_seqs * c.n_kv_heads,
           false);
@@ -2116,7 +2124,11 @@ kvzap_status kvzap_cache_create(kvzap_ctx *ctx, kvzap_cache **out, int32_t n_seq
 kvzap_status kvzap_cache_debug_skew_steps(kvzap_cache *cache, int32_t delta)
 {
     if (!cache) return KVZAP_ERR_INVALID_ARG;
-    for (auto &n : cache->steps_done) n += delta;
+    DeviceGuard guard(cache->ctx->cfg.device);
+    if (cudaDeviceSynchronize() != cudaSuccess) return KVZAP_ERR_CUDA;
+    const int n = static_cast<int>(cache->n_step_counters / 3 * 2);
+    add_int_kernel<<<(n + 255) / 256, 256>>>(cache->ticket, n, delta);
+    if (cudaDeviceSynchronize() != cudaSuccess) return KVZAP_ERR_CUDA;
     return KVZAP_OK;
 }
 
@@ -2168,11 +2180,9 @@ static kvzap_status decode_step_impl(kvzap_ctx *ctx, kvzap_cache *cache, int32_t
     // at the same step count.
     DecodeFuse fuse;
     memset(&fuse, 0, sizeof fuse);
-    bool can_fuse = cache->v.window > 0 && c.hidden > 0;
-    for (int l = layer_begin; l < layer_end && can_fuse; ++l)
-        can_fuse = cache->steps_done[l] == cache->steps_done[layer_begin];
+    const bool can_fuse = cache->v.window > 0 && c.hidden > 0;
     if (can_fuse) {
-        fuse.expect = cache->steps_done[layer_begin];
+        fuse.ticket = cache->ticket;
         fuse.c = cache->v;
         fuse.K_new = static_cast<const uint4 *>(K_new);
         fuse.V_new = static_cast<const uint4 *>(V_new);
@@ -2197,7 +2207,6 @@ static kvzap_status decode_step_impl(kvzap_ctx *ctx, kvzap_cache *cache, int32_t
     }
     if (st != KVZAP_OK) return st;
     if (fused) {
-        for (int l = layer_begin; l < layer_end; ++l) cache->steps_done[l] += 1;
         ctx->fused_cache = cache;
         ctx->fused_seq = ctx->op_seq;
         return KVZAP_OK;

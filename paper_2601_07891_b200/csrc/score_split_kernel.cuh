@@ -33,10 +33,13 @@ namespace kvzap {
 // the new scores into the score buffer at the very end (the last cluster of the tile to arrive).
 // Consecutive steps may overlap in time (the next launch starts as SMs become free): `done[cluster]`
 // counts the steps a cluster has completed, and a cluster touches the cache only after all clusters of
-// its tile have published `expect` for the step before.
+// its tile have published the number of the step before.  Which step a CTA is working on it learns on the
+// device: it draws a ticket from a counter of its own (tile, slice, rank) before it lets the next launch be
+// placed, so the CTAs that serve the same slice in consecutive launches draw consecutive numbers whatever the
+// host knows -- a captured CUDA graph of steps can be replayed.
 struct DecodeFuse {
     int32_t enabled;
-    int32_t expect;
+    int32_t *ticket;                // [n_layers * tiles_per_layer][4][2]: steps started, per (slice, rank in the cluster)
     CacheView c;
     const uint4 *K_new, *V_new;     // [n_layers_call][B][H][D] bf16
     float tau;
@@ -75,6 +78,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     constexpr int kElems = kFp8 ? 2 * kBlockK : kBlockK;         // elements per 128-byte K block
     __shared__ int64_t fuse_dst[256];       // fused decode step: page row of the evicted token (-1 = dropped)
     __shared__ int64_t fuse_ring[256];      //                     ring row of the list's current slot (-1 = no list)
+    __shared__ int32_t fuse_step;           //                     number of the step this CTA works on (its ticket)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw_addr & 1023u)) & 1023u;
@@ -100,10 +104,6 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 36);
     volatile int *last_flag = reinterpret_cast<volatile int *>(smem + L.bars + 16 * kMaxStages + 40);
 
-    griddep_launch_dependents();
-    // unless the caller vouches for the producers of its inputs, nothing of them is read before the work
-    // ahead in the stream has completed (every thread waits: the loads below are issued by several warps)
-    if (p.wait_before_load) griddep_wait();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();            // 0 .. k_split - 1
@@ -114,6 +114,17 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int l_rel = tile / p.tiles_per_layer;
     const int m_tile = tile - l_rel * p.tiles_per_layer;
     const int layer = p.layer0 + l_rel;
+    if (f.enabled) {
+        // the step number, drawn before any thread of this CTA lets the next launch be placed: a CTA of that launch
+        // starts only after every CTA of this one has passed the instruction below, hence after this draw
+        if (threadIdx.x == 0)
+            fuse_step = atomicAdd(f.ticket + ((layer * p.tiles_per_layer + m_tile) * 4 + nh) * 2 + kh, 1);
+        __syncthreads();
+    }
+    griddep_launch_dependents();
+    // unless the caller vouches for the producers of its inputs, nothing of them is read before the work
+    // ahead in the stream has completed (every thread waits: the loads below are issued by several warps)
+    if (p.wait_before_load) griddep_wait();
     const int own_n = ns / k_split;                      // accumulator columns this CTA finishes
     const int own_c0 = kh * own_n;                       // the first of them
     const int j_first = nh * ns + own_c0;                // = first hidden unit of this CTA
@@ -248,7 +259,8 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const int cid = layer * p.tiles_per_layer + m_tile;
             if (etid < n_split) {
                 const long long t0 = clock64();
-                while (ld_acquire_gpu(f.done + cid * n_split + etid) != f.expect) {
+                const int32_t expect = fuse_step;
+                while (ld_acquire_gpu(f.done + cid * n_split + etid) != expect) {
                     if (clock64() - t0 > f.wait_limit) { *abort_flag = 1; break; }
                 }
             }
@@ -488,7 +500,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             named_barrier_sync(2, 128);
             if (*last_flag == 0) {
                 // not the last: this cluster's part of the cache update is complete, say so and leave
-                if (f.enabled && threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, f.expect + 1);
+                if (f.enabled && threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, fuse_step + 1);
                 return;
             }
 #pragma unroll
@@ -519,7 +531,7 @@ score_split_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             }
             __threadfence();
             named_barrier_sync(2, 128);
-            if (threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, f.expect + 1);
+            if (threadIdx.x == 64 && *abort_flag == 0) st_release_gpu(f.done + done_i, fuse_step + 1);
         }
         if (valid && p.scores != nullptr) {
             float *dst = p.scores + (static_cast<int64_t>(l_rel) * p.n_tokens + t) * p.n_heads;
