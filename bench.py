@@ -39,7 +39,7 @@ NCU_TRAFFIC = {
     "qwen3_8b_prefill_32k": (277.2e6, "profiles/score_kernel_mlp_qwen3_8b_prefill_32k.md"),
     "llama31_8b_prefill_4x16k": (540.8e6, "profiles/score_kernel_linear_llama31_8b_prefill_4x16k.md"),
     "linear_4k": (39.72e6, "profiles/score_linear_split_kernel_linear_4k.md"),
-    "qwen3_8b_decode_b128": (226.3e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
+    "qwen3_8b_decode_b128": (228.0e6, "profiles/score_split_kernel_qwen3_8b_decode_b128.md"),
 }
 NCU_TRAFFIC_FP8 = {
     "qwen3_8b_prefill_32k": (140.4e6, "profiles/score_kernel_mlp_fp8_qwen3_8b_prefill_32k.md"),
