@@ -38,6 +38,9 @@
  *     that does not itself signal early.  (2) Passing the same scores buffer
  *     to two consecutive calls is allowed in either mode; the library then
  *     launches the second call's scoring kernel without overlap of its stores.
+ *   - Stream capture (CUDA graphs): kvzap_decode_step(_fp8) and kvzap_decode_attention(_fp8) may be captured
+ *     and replayed.  The other calls rotate scratch sets and counters on the host from call to call and must
+ *     be enqueued, not captured.
  *   - Errors the host can see (bad argument, unsupported shape) return at once
  *     and launch nothing.  Conditions only the device can see set a status
  *     word that kvzap_poll_status() reads; kernels never trap and every
