@@ -206,6 +206,84 @@ def test_fp8_decode_steps_match_decode_oracle(binding, oracle, d_model, hidden, 
     ctx.close()
 
 
+def test_fp8_decode_steps_captured_in_a_cuda_graph(binding, oracle):
+    """Two 8-bit decode steps captured once and replayed with refilled static buffers: scores against the 8-bit
+    oracle, lists bit for bit against the decode oracle."""
+    d_model, hidden, H, D, w, P, B, L, tau, n_replays = 256, 128, 8, 64, 8, 4, 6, 2, 0.1, 8
+    ctx = binding.Kvzap(d_model, hidden, H, D, L, max_tokens=128, max_seqs=1, trusted_producers=True)
+    cases = []
+    for l in range(L):
+        case = _fp8_case(d_model, hidden, H, 1, seed=190 + l)
+        cases.append(case)
+        _, _, W18, sw, b1, W2, b2 = case
+        binding.kvzap_set_weights_fp8(ctx.handle, l, W18.cuda(), sw.cuda(), b1.cuda(), parity.dev(W2), parity.dev(b2))
+    n_steps = 2 * n_replays + 2
+    max_pages = n_steps // P + 2
+    n_pool = B * L * H * max_pages
+    K_pool = torch.zeros(n_pool, P, D, dtype=torch.bfloat16, device="cuda")
+    V_pool = torch.zeros_like(K_pool)
+    cache = binding.kvzap_cache_create(ctx.handle, B, w, P, K_pool, V_pool, max_pages)
+    dec = oracle.DecodeOracle(B, L, H, D, w)
+    X8 = [torch.zeros(L, B, d_model, dtype=torch.uint8, device="cuda") for _ in range(2)]
+    SX = [torch.zeros(L, B, dtype=torch.float32, device="cuda") for _ in range(2)]
+    Kn = [torch.zeros(L, B, H, D, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    Vn = [torch.zeros(L, B, H, D, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    sc = [torch.zeros(L, B, H, dtype=torch.float32, device="cuda") for _ in range(2)]
+    feed = {}
+
+    def fill(i, step):
+        x8, sx = synth.quantize_e4m3(synth.hidden_states(L * B, d_model, seed=3500 + step))
+        k, v = synth.keys_values(L * B, H, D, seed=4500 + step)
+        X8[i].copy_(x8.view(L, B, d_model)); SX[i].copy_(sx.view(L, B)); Kn[i].copy_(k.view(L, B, H, D)); Vn[i].copy_(v.view(L, B, H, D))
+        feed[i] = (x8.numpy().reshape(L, B, d_model), sx.numpy().reshape(L, B), synth.bits(k.view(L, B, H, D)), synth.bits(v.view(L, B, H, D)))
+
+    def iteration():
+        for i in range(2):
+            binding.kvzap_decode_step_fp8(ctx.handle, cache, 0, L, X8[i], SX[i], Kn[i], Vn[i], tau, sc[i])
+
+    worst = [0.0]
+
+    def account():
+        assert ctx.poll_status() == 0
+        for i in range(2):
+            s = sc[i].cpu().numpy()
+            x8, sx, kb, vb = feed[i]
+            for l in range(L):
+                _, _, W18, sw, b1, W2, b2 = cases[l]
+                want = oracle.score_mlp_fp8(x8[l], sx[l], W18.numpy(), sw.numpy(), b1.numpy(), synth.bits(W2), b2.numpy())
+                worst[0] = max(worst[0], float(np.abs(s[l] - want).max()))
+                for b in range(B):
+                    dec.append(b, l, s[l, b], kb[l, b], vb[l, b], tau)
+
+    fill(0, 0); fill(1, 1)
+    iteration()
+    torch.cuda.synchronize()
+    account()
+    graph = torch.cuda.CUDAGraph()
+    fill(0, 2); fill(1, 3)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=torch.cuda.Stream()):
+        iteration()
+    for r in range(n_replays):
+        if r > 0:
+            fill(0, 2 + 2 * r); fill(1, 3 + 2 * r)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        account()
+    assert worst[0] <= parity.SCORE_ATOL, worst[0]
+    for b in range(B):
+        for l in range(L):
+            for h in range(H):
+                _pos, Kd, Vd = dec.logical(b, l, h)
+                Kg, Vg, n = _export(binding, ctx, cache, b, l, h, n_steps + 1, D)
+                assert n == len(Kd), (b, l, h)
+                np.testing.assert_array_equal(Kg, Kd)
+                np.testing.assert_array_equal(Vg, Vd)
+    binding.kvzap_cache_destroy(cache)
+    ctx.close()
+
+
 def test_fp8_needs_d_model_multiple_of_128_and_its_own_weights(binding):
     ctx = binding.Kvzap(192, 0, 8, 64, 1, max_tokens=64)
     W = torch.zeros(8, 192, dtype=torch.uint8, device="cuda")
