@@ -625,7 +625,12 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
     // KVzap-Linear on few tiles (a short prompt, or a decode step): four CTAs share a tile, each a quarter
     // of the K range.  The kernel writes only after it has waited for the kernel ahead, so it may always
     // be placed early.
-    if (c.hidden == 0 && ctx->lin_split_ok && blocks_per_layer * n_layers * kLinSplit <= ctx->sm_count) {
+    // (with the compaction in the same launch the CTAs are small enough for several per SM: up to kLinMaxTiles tiles)
+    const bool lin_one_launch = compact != nullptr && n_layers == 1 && n_seqs == 1 && maskbits != nullptr && window_keep == 1 &&
+                                blocks_per_layer <= kLinMaxTiles && c.head_dim * 2 <= 2048;
+    if (c.hidden == 0 && ctx->lin_split_ok &&
+        (blocks_per_layer * n_layers * kLinSplit <= ctx->sm_count ||
+         (lin_one_launch && blocks_per_layer * kLinSplit <= 2 * static_cast<int64_t>(ctx->sm_count)))) {
         CUtensorMap tmap_x;
         kvzap_status st = hidden_tmap(ctx, &tmap_x, hidden, n_tokens, n_layers);
         if (st != KVZAP_OK) return st;
@@ -671,8 +676,7 @@ static kvzap_status launch_score(kvzap_ctx *ctx, int32_t layer, int32_t n_layers
         LinCompact fc;
         memset(&fc, 0, sizeof fc);
         uint32_t smem = kLinSmemBytes;
-        if (compact != nullptr && n_layers == 1 && n_seqs == 1 && maskbits != nullptr && window_keep == 1 &&
-            p.n_tiles <= kLinMaxTiles && c.head_dim * 2 <= 2048) {
+        if (lin_one_launch) {
             const size_t kv_bytes = static_cast<size_t>(c.n_kv_heads) * n_tokens * c.head_dim * 2;
             const int set = static_cast<int>(ctx->op_turn % kOpRing);
             ctx->op_turn += 1;

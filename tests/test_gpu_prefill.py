@@ -127,7 +127,10 @@ def _run_fused(binding, oracle, d_model, hidden, H, D, seq_lens, tau, w, seed, t
 
 @pytest.mark.parametrize("T,w,tau", [(1, 128, 0.43), (2, 0, 0.0), (100, 128, 0.43), (128, 128, 0.43), (129, 128, 0.43),
                                      (700, 128, 0.43), (700, 0, 0.43), (700, 512, -0.5), (700, 1000, 0.43),
-                                     (1300, 128, float("inf")), (1300, 128, float("-inf")), (4097, 128, 0.84)])
+                                     (1300, 128, float("inf")), (1300, 128, float("-inf")), (4097, 128, 0.84),
+                                     # 47, 63 and 64 tiles: scoring and compaction in one launch with several CTAs per SM;
+                                     # 65 tiles: the first length that takes two launches again
+                                     (6000, 128, 0.43), (8001, 64, 0.0), (8192, 128, 0.43), (8200, 128, 0.43)])
 def test_fused_linear_single_sequence(binding, oracle, T, w, tau):
     keep, lengths = _run_fused(binding, oracle, 512, 0, 8, 128, [T], tau, w, seed=T + w)
     assert (lengths >= min(T, w)).all()
