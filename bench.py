@@ -430,7 +430,7 @@ def run_prefill(args, wl, env, sub=False):
     if fp8:
         traffic = NCU_TRAFFIC_FP8.get(wl.name) if args.layers == 0 and not proj else None
     roofline.update({"traffic": traffic[0] if traffic else None,
-                     "traffic_source": (traffic[1] + " (ncu capture, not measured in this run)") if traffic else None,
+                     "traffic_source": (traffic[1] + " (ncu capture of 2026-11-28, not measured in this run)") if traffic else None,
                      "kernel": "score_kernel", "peak_source": peak_src,
                      "kernel_ms": layer_ms, "alone_ms": score_ms,
                      "note": "kernel_ms = layer period in the timed region (compaction overlaps the next "
@@ -661,7 +661,7 @@ def run_decode(args, wl, env, sub=False):
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"],
                 "traffic": NCU_TRAFFIC[wl.name][0] if wl.name in NCU_TRAFFIC and args.layers == 0 and not fp8 else None,
-                "traffic_source": (NCU_TRAFFIC[wl.name][1] + " (ncu capture, not measured in this run)")
+                "traffic_source": (NCU_TRAFFIC[wl.name][1] + " (ncu capture of 2026-11-28, not measured in this run)")
                 if wl.name in NCU_TRAFFIC and args.layers == 0 and not fp8 else None,
                 "kernel": "score_split_kernel (scoring + cache update in one launch)", "peak_source": peak_src,
                 "kernel_ms": ms_per_step, "algorithmic_bytes_per_step": bytes_layer * L}
