@@ -214,6 +214,29 @@ def _roofline_times(wl, n_tokens, kept_rows, peaks, tensor_peak):
     return flops, score_bytes, t_tensor, t_hbm_score, t_hbm_layer
 
 
+def _timed_steps(step, n_steps, block, record_first, record_last):
+    """Runs n_steps steps between two given events and marks every `block` steps with an event of its own: the
+    whole-region time stays the measurement, the marks give the spread (median / min / max per step over blocks)."""
+    import torch
+    marks = []
+    record_first.record()
+    for i in range(n_steps):
+        step()
+        if (i + 1) % block == 0 and i + 1 < n_steps:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            marks.append(ev)
+    record_last.record()
+    return marks
+
+
+def _step_stats(first, marks, last, n_steps, block):
+    evs = [first] + marks + [last]
+    sizes = [block] * len(marks) + [n_steps - block * len(marks)]
+    per = sorted(evs[i].elapsed_time(evs[i + 1]) / sizes[i] for i in range(len(sizes)) if sizes[i] > 0)
+    return {"median": statistics.median(per), "min": per[0], "max": per[-1], "steps_per_sample": block, "samples": len(per)}
+
+
 def _timed(fn, n, stream_sync):
     """Average milliseconds of fn() over n calls, CUDA events on the current stream."""
     import torch
@@ -361,13 +384,12 @@ def run_prefill(args, wl, env, sub=False):
     launches0 = ctx.launch_count()
     sampler.start()
     barrier()
-    e0.record()
-    for _ in range(n_steps):
-        step()
-    e1.record()
+    block = 1 if L * n_tokens >= 1000000 else 100        # a mark per step, or per 100 steps where a step is a few microseconds
+    marks = _timed_steps(step, n_steps, block, e0, e1)
     barrier()
     clocks = sampler.stop()
     total_ms = env["max_over_ranks"](e0.elapsed_time(e1))
+    step_stats = _step_stats(e0, marks, e1, n_steps, block)
     gpu_launches = ctx.launch_count() - launches0
     ms_per_step = total_ms / n_steps
     layer_ms = ms_per_step / L
@@ -450,7 +472,7 @@ def run_prefill(args, wl, env, sub=False):
                     "enough sets that 2.5 x L2 lies between two uses of a buffer)",
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps,
-            "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": n_warm, "ms_per_step": ms_per_step, "step_ms": step_stats, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "e4m3 x e4m3 -> f32 (first layer), bf16 K/V" if fp8 else "bf16", "data": "synthetic",
             "config": config, "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline, "breakdown": extra}
 
@@ -631,13 +653,14 @@ def run_decode(args, wl, env, sub=False):
     launches0 = ctx.launch_count()
     sampler.start()
     barrier()
-    e0.record()
-    for _ in range(n_steps):
-        step()
-    e1.record()
+    block = 100 if n_steps >= 200 else max(1, n_steps // 4)
+    if graph_mode != "off":
+        block = -(-block // n_sets) * n_sets
+    marks = _timed_steps(step, n_steps, block, e0, e1)
     barrier()
     clocks = sampler.stop()
     total_ms = env["max_over_ranks"](e0.elapsed_time(e1))
+    step_stats = _step_stats(e0, marks, e1, n_steps, block)
     gpu_launches = ctx.launch_count() - launches0
     if graph_mode != "off":          # replays launch what the capture recorded; the host-side counter sees only the capture
         gpu_launches = n_steps * (L if graph_mode == "layer" else 1)
@@ -674,7 +697,7 @@ def run_decode(args, wl, env, sub=False):
                              "layer": "%d steps per graph, one launch per layer" % n_sets}[graph_mode],
               "parallelism": "replicas only" if world > 1 else "single GPU"}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": n_steps, "warmup": n_warm,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "step_ms": step_stats, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "e4m3 x e4m3 -> f32 (first layer), bf16 K/V" if fp8 else "bf16", "data": "synthetic", "config": config,
             "clocks": clocks, "gpu_launches": int(gpu_launches), "roofline": roofline,
             "breakdown": {"layer_us": ms_per_step * 1e3 / L, "layer_roofline_us": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
@@ -865,7 +888,7 @@ def summarise(line):
     """The short record of one workload for the headline line's `configs` list."""
     bd, rf = line["breakdown"], line["roofline"]
     rec = {"workload": line["config"]["workload"], "value": line["value"], "unit": line["unit"], "steps": line["steps"],
-           "ms_per_step": line["ms_per_step"], "layer_frac_of_roofline": bd.get("layer_frac_of_roofline"),
+           "ms_per_step": line["ms_per_step"], "step_ms": line.get("step_ms"), "layer_frac_of_roofline": bd.get("layer_frac_of_roofline"),
            "roofline_bound": rf["bound"], "roofline_frac": rf["frac"], "clocks": line["clocks"],
            "gpu_launches": line["gpu_launches"]}
     if "layer_ms" in bd:
